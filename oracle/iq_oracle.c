@@ -1,0 +1,373 @@
+/*
+ * IsoQuant oracle: a plain, slow, fp64 CPU statement of what the hot path computes.
+ *
+ * THIS IS TEST INFRASTRUCTURE. Only the test-suite, the smoke check and the benchmark's CPU
+ * baseline may build, load or call it. The product (the CUDA library) shares no code, header,
+ * table or helper with this file and never calls it.
+ *
+ * Everything is written from the paper's definitions, in the paper's order, with dense matrices
+ * and plain loops: no butterfly, no blocking, no fusion.
+ *   - Algorithm 1 (compression): s = ||x||_2, x^ = x/s, x~ = R_SO4(H_d x^), Lloyd-Max code per
+ *     coordinate, bit-pack.
+ *   - Eq. 2: R = R_SO4 o H_d, H_d the normalised Walsh-Hadamard matrix, R_SO4 block-diagonal with
+ *     one 4x4 block per contiguous group of four coordinates.
+ *   - Section 3.3 "SO(4) parameterization" and Appendix B: a block acts as v -> q_L v conj(q_R)
+ *     with unit quaternions q_L, q_R; 8 floats per block.
+ *   - Appendix A: q~ = R q, alpha = softmax(q~ . k~_j / sqrt(d_k)), o~ = sum_j alpha_j v~_j,
+ *     o = R^T o~.
+ *
+ * Readings taken where the paper is silent (each is also listed in the design notes):
+ *   - H_d in natural (Sylvester) order: H[i][j] = (-1)^popcount(i & j) / sqrt(d).
+ *   - blocks b = 0 .. d/4-1 cover coordinates [4b, 4b+4) (Algorithm 1 prints 1-based "4i:4i+4").
+ *   - quaternion = (w, x, y, z), Hamilton product, block coordinates (y0,y1,y2,y3) <-> y0 + y1 i + y2 j + y3 k.
+ *   - quantiser works in unit-variance units u = sqrt(d) * x~; code = #{ j : u > t_j } over the 7
+ *     ascending thresholds (strict ">", an exact tie takes the lower code); codes 0..7 ascend with level.
+ *   - zero row: s = 0, x^ = 0.
+ *   - stored scale = s rounded to fp32; dequantised coordinate = scale * level[code] / sqrt(d).
+ *   - K and V of one KV head share that head's rotation and the codebook; all query heads of a
+ *     group use their KV head's rotation.
+ *   - packed row layout (3 bits x d, 3d/8 bytes, the paper fixes only the size): the row is a
+ *     sequence of little-endian 32-bit words; coordinates are taken in groups of 32, each group
+ *     owning 3 consecutive words. In group-local numbering, coordinate c < 24 puts its 3-bit code in
+ *     bits [4n, 4n+3) of word c/8, n = c mod 8; coordinate c >= 24 (n = c - 24) spreads its code
+ *     over bit 4n+3 of the three words: bit k of the code goes to word k.
+ *
+ * Parity pins: every function here is pinned by tests/test_oracle_*.py (invariants, closed forms,
+ * library routines, brute force). Not pinned (no published artefact exists): equality of the code
+ * values and codebook with the authors' own files -- "parity unpinned" for those two items.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int iqo_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+void iqo_set_num_threads(int n) {
+#ifdef _OPENMP
+  if (n > 0) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
+/* IEEE binary16 -> double, from the format definition. */
+double iqo_half_to_double(uint16_t h) {
+  int sign = (h >> 15) & 1, e = (h >> 10) & 31, m = h & 1023;
+  double v;
+  if (e == 0) v = ldexp((double)m, -24);
+  else if (e == 31) v = m ? NAN : INFINITY;
+  else v = ldexp((double)(m + 1024), e - 25);
+  return sign ? -v : v;
+}
+
+/* Hamilton product of quaternions stored (w, x, y, z). */
+static void quat_mul(const double* a, const double* b, double* o) {
+  o[0] = a[0] * b[0] - a[1] * b[1] - a[2] * b[2] - a[3] * b[3];
+  o[1] = a[0] * b[1] + a[1] * b[0] + a[2] * b[3] - a[3] * b[2];
+  o[2] = a[0] * b[2] - a[1] * b[3] + a[2] * b[0] + a[3] * b[1];
+  o[3] = a[0] * b[3] + a[1] * b[2] - a[2] * b[1] + a[3] * b[0];
+}
+
+/* Section 3.3 / Appendix B: the 4x4 matrix of v -> q_L v conj(q_R), built column by column by
+ * applying the map to the basis quaternions. q8 = (q_L.wxyz, q_R.wxyz) as stored (fp32); both are
+ * renormalised to unit length in fp64 first. M is row-major [4][4]. */
+void iqo_so4_block(const float* q8, double* M) {
+  double qL[4], qR[4], qRc[4], nL = 0, nR = 0;
+  for (int i = 0; i < 4; i++) { qL[i] = q8[i]; qR[i] = q8[4 + i]; nL += qL[i] * qL[i]; nR += qR[i] * qR[i]; }
+  nL = sqrt(nL); nR = sqrt(nR);
+  for (int i = 0; i < 4; i++) { qL[i] /= nL; qR[i] /= nR; }
+  qRc[0] = qR[0]; qRc[1] = -qR[1]; qRc[2] = -qR[2]; qRc[3] = -qR[3];
+  for (int c = 0; c < 4; c++) {
+    double e[4] = {0, 0, 0, 0}, t[4], r[4];
+    e[c] = 1.0;
+    quat_mul(qL, e, t);
+    quat_mul(t, qRc, r);
+    for (int i = 0; i < 4; i++) M[i * 4 + c] = r[i];
+  }
+}
+
+/* Eq. 2: normalised Walsh-Hadamard matrix, natural order. H is row-major [d][d]. */
+void iqo_hadamard(int d, double* H) {
+  double s = 1.0 / sqrt((double)d);
+  for (int i = 0; i < d; i++)
+    for (int j = 0; j < d; j++)
+      H[(size_t)i * d + j] = (__builtin_popcount((unsigned)(i & j)) & 1) ? -s : s;
+}
+
+/* Eq. 2: R = blockdiag(M_0 .. M_{d/4-1}) * H_d as a dense d x d matrix (row-major).
+ * quats = [d/4][8] fp32 for one KV head. */
+void iqo_rotation_matrix(int d, const float* quats, double* R) {
+  double* H = (double*)malloc(sizeof(double) * d * d);
+  iqo_hadamard(d, H);
+  for (int b = 0; b < d / 4; b++) {
+    double M[16];
+    iqo_so4_block(quats + 8 * b, M);
+    for (int r = 0; r < 4; r++)
+      for (int j = 0; j < d; j++) {
+        double acc = 0;
+        for (int c = 0; c < 4; c++) acc += M[r * 4 + c] * H[(size_t)(4 * b + c) * d + j];
+        R[(size_t)(4 * b + r) * d + j] = acc;
+      }
+  }
+  free(H);
+}
+
+/* Algorithm 1, lines 1-4 and Step 3, for one row. x: d binary16 values. codes: one byte per
+ * coordinate (0..7). Returns the fp32 scale; if u_out != NULL also returns u = sqrt(d) * x~. */
+float iqo_quantize_row(int d, const double* R, const float* thresholds7, const uint16_t* x,
+                       uint8_t* codes, double* u_out) {
+  double* xh = (double*)malloc(sizeof(double) * d);
+  double ss = 0;
+  for (int i = 0; i < d; i++) { xh[i] = iqo_half_to_double(x[i]); ss += xh[i] * xh[i]; }
+  double s = sqrt(ss);
+  for (int i = 0; i < d; i++) xh[i] = (s == 0.0) ? 0.0 : xh[i] / s;
+  double rootd = sqrt((double)d);
+  for (int i = 0; i < d; i++) {
+    double acc = 0;
+    for (int j = 0; j < d; j++) acc += R[(size_t)i * d + j] * xh[j];
+    double u = rootd * acc;
+    int code = 0;
+    for (int j = 0; j < 7; j++) if (u > (double)thresholds7[j]) code++;
+    codes[i] = (uint8_t)code;
+    if (u_out) u_out[i] = u;
+  }
+  free(xh);
+  return (float)s;
+}
+
+static int row_bytes(int d) { return 3 * d / 8; }
+
+static void put_word(uint8_t* p, uint32_t w) { p[0] = w & 255; p[1] = (w >> 8) & 255; p[2] = (w >> 16) & 255; p[3] = (w >> 24) & 255; }
+static uint32_t get_word(const uint8_t* p) { return (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24); }
+
+/* Step 4 (bit-pack), layout as described at the top of this file. */
+void iqo_pack_row(int d, const uint8_t* codes, uint8_t* row) {
+  for (int g = 0; g < d / 32; g++) {
+    uint32_t w[3] = {0, 0, 0};
+    for (int c = 0; c < 32; c++) {
+      uint32_t code = codes[32 * g + c] & 7u;
+      if (c < 24) {
+        w[c / 8] |= code << (4 * (c % 8));
+      } else {
+        int n = c - 24;
+        for (int k = 0; k < 3; k++) w[k] |= ((code >> k) & 1u) << (4 * n + 3);
+      }
+    }
+    for (int k = 0; k < 3; k++) put_word(row + 4 * (3 * g + k), w[k]);
+  }
+}
+
+void iqo_unpack_row(int d, const uint8_t* row, uint8_t* codes) {
+  for (int g = 0; g < d / 32; g++) {
+    uint32_t w[3];
+    for (int k = 0; k < 3; k++) w[k] = get_word(row + 4 * (3 * g + k));
+    for (int c = 0; c < 32; c++) {
+      uint32_t code = 0;
+      if (c < 24) {
+        code = (w[c / 8] >> (4 * (c % 8))) & 7u;
+      } else {
+        int n = c - 24;
+        for (int k = 0; k < 3; k++) code |= ((w[k] >> (4 * n + 3)) & 1u) << k;
+      }
+      codes[32 * g + c] = (uint8_t)code;
+    }
+  }
+}
+
+/* Algorithm 1 applied to the new K and V rows of every sequence and KV head, appended to the cache.
+ * k_new, v_new: binary16, element (b, i, h, c) at b*stride_b + i*stride_t + h*stride_h + c (element strides).
+ * Row i < n_new[b] of sequence b goes to cache row append_pos[b] + i (rows >= t_cap are skipped).
+ * quats: [H_kv][d/4][8]. codes: [B][H_kv][t_cap][3d/8], scales: [B][H_kv][t_cap].
+ * Returns the number of rows skipped because they fell outside the cache. */
+int64_t iqo_quantize_append(int B, int H_kv, int d, int t_cap, const float* quats, const float* thresholds7,
+                            const uint16_t* k_new, const uint16_t* v_new,
+                            int64_t stride_b, int64_t stride_t, int64_t stride_h,
+                            const int32_t* append_pos, const int32_t* n_new, int n_new_max,
+                            uint8_t* k_codes, float* k_scales, uint8_t* v_codes, float* v_scales) {
+  int P = row_bytes(d);
+  int64_t skipped = 0;
+  for (int h = 0; h < H_kv; h++) {
+    double* R = (double*)malloc(sizeof(double) * d * d);
+    iqo_rotation_matrix(d, quats + (size_t)h * (d / 4) * 8, R);
+    for (int b = 0; b < B; b++) {
+      int n = n_new ? n_new[b] : n_new_max;
+      if (n > n_new_max) n = n_new_max;
+      int64_t sk = 0;
+#pragma omp parallel for schedule(static) reduction(+ : sk)
+      for (int i = 0; i < n; i++) {
+        int64_t t = (int64_t)append_pos[b] + i;
+        if (t < 0 || t >= t_cap) { sk += 2; continue; }
+        uint8_t codes[512];
+        size_t src = (size_t)(b * stride_b + i * stride_t + h * stride_h);
+        size_t row = ((size_t)b * H_kv + h) * t_cap + t;
+        k_scales[row] = iqo_quantize_row(d, R, thresholds7, k_new + src, codes, NULL);
+        iqo_pack_row(d, codes, k_codes + row * P);
+        v_scales[row] = iqo_quantize_row(d, R, thresholds7, v_new + src, codes, NULL);
+        iqo_pack_row(d, codes, v_codes + row * P);
+      }
+      skipped += sk;
+    }
+    free(R);
+  }
+  return skipped;
+}
+
+/* Dequantised rotated vector of one cached row: x~_i = scale * level[code_i] / sqrt(d). */
+static void dequant_row(int d, const uint8_t* row, float scale, const float* levels8, double* out) {
+  uint8_t codes[512];
+  iqo_unpack_row(d, row, codes);
+  double f = (double)scale / sqrt((double)d);
+  for (int i = 0; i < d; i++) out[i] = f * (double)levels8[codes[i]];
+}
+
+/* Appendix A, one query head against the first len rows of its KV head's packed cache.
+ * z_out (optional, [len]) receives the scaled scores; o_rot (optional, [d]) the rotated-space output. */
+static void decode_one(int d, const double* R, const float* levels8, double sm_scale, const uint16_t* q,
+                       const uint8_t* k_codes, const float* k_scales, const uint8_t* v_codes,
+                       const float* v_scales, int len, double* out, double* lse, int32_t* argmax,
+                       double* z_out, double* o_rot_out) {
+  int P = row_bytes(d);
+  double* qt = (double*)malloc(sizeof(double) * d);
+  double* z = (double*)malloc(sizeof(double) * (len > 0 ? len : 1));
+  double* row = (double*)malloc(sizeof(double) * d);
+  double* orot = (double*)calloc(d, sizeof(double));
+  for (int i = 0; i < d; i++) {           /* q~ = R q */
+    double acc = 0;
+    for (int j = 0; j < d; j++) acc += R[(size_t)i * d + j] * iqo_half_to_double(q[j]);
+    qt[i] = acc;
+  }
+  int best = -1;
+  double zmax = -INFINITY;
+  for (int j = 0; j < len; j++) {         /* z_j = sm_scale * q~ . k~_j */
+    dequant_row(d, k_codes + (size_t)j * P, k_scales[j], levels8, row);
+    double acc = 0;
+    for (int i = 0; i < d; i++) acc += qt[i] * row[i];
+    z[j] = sm_scale * acc;
+    if (z[j] > zmax) { zmax = z[j]; best = j; }
+    if (z_out) z_out[j] = z[j];
+  }
+  double denom = 0;
+  for (int j = 0; j < len; j++) denom += exp(z[j] - zmax);
+  for (int j = 0; j < len; j++) {         /* o~ = sum_j alpha_j v~_j */
+    double a = exp(z[j] - zmax) / denom;
+    dequant_row(d, v_codes + (size_t)j * P, v_scales[j], levels8, row);
+    for (int i = 0; i < d; i++) orot[i] += a * row[i];
+  }
+  for (int j = 0; j < d; j++) {           /* o = R^T o~ */
+    double acc = 0;
+    for (int i = 0; i < d; i++) acc += R[(size_t)i * d + j] * orot[i];
+    out[j] = (len > 0) ? acc : 0.0;
+  }
+  if (o_rot_out) for (int i = 0; i < d; i++) o_rot_out[i] = orot[i];
+  if (lse) *lse = (len > 0) ? zmax + log(denom) : -INFINITY;
+  if (argmax) *argmax = best;
+  free(qt); free(z); free(row); free(orot);
+}
+
+/* One decode step for every sequence and query head. q: [B][H_q][d] binary16. out: [B][H_q][d],
+ * lse: [B][H_q], argmax: [B][H_q] (lowest row index attaining the maximum score; -1 if len = 0).
+ * sm_scale <= 0 selects 1/sqrt(d). o_rot (optional): [B][H_q][d], the output before R^T. */
+void iqo_decode_attention(int B, int H_q, int H_kv, int d, int t_cap, double sm_scale, const float* quats,
+                          const float* levels8, const uint16_t* q, const uint8_t* k_codes,
+                          const float* k_scales, const uint8_t* v_codes, const float* v_scales,
+                          const int32_t* seq_lens, double* out, double* lse, int32_t* argmax, double* o_rot) {
+  int P = row_bytes(d), G = H_q / H_kv;
+  if (sm_scale <= 0) sm_scale = 1.0 / sqrt((double)d);
+  double* Rs = (double*)malloc(sizeof(double) * (size_t)H_kv * d * d);
+  for (int g = 0; g < H_kv; g++) iqo_rotation_matrix(d, quats + (size_t)g * (d / 4) * 8, Rs + (size_t)g * d * d);
+#pragma omp parallel for schedule(dynamic) collapse(2)
+  for (int b = 0; b < B; b++)
+    for (int h = 0; h < H_q; h++) {
+      int g = h / G;
+      int len = seq_lens[b];
+      if (len > t_cap) len = t_cap;
+      if (len < 0) len = 0;
+      size_t base = ((size_t)b * H_kv + g) * t_cap;
+      size_t o = ((size_t)b * H_q + h);
+      decode_one(d, Rs + (size_t)g * d * d, levels8, sm_scale, q + o * d, k_codes + base * P, k_scales + base,
+                 v_codes + base * P, v_scales + base, len, out + o * d, lse ? lse + o : NULL,
+                 argmax ? argmax + o : NULL, NULL, o_rot ? o_rot + o * d : NULL);
+    }
+  free(Rs);
+}
+
+/* Scaled scores z_j of one (sequence b, query head h): z_out [len]. */
+void iqo_scores(int H_q, int H_kv, int d, int t_cap, double sm_scale, const float* quats, const float* levels8,
+                const uint16_t* q_bh, int b, int h, const uint8_t* k_codes, const float* k_scales, int len,
+                double* z_out) {
+  int P = row_bytes(d), G = H_q / H_kv, g = h / G;
+  if (sm_scale <= 0) sm_scale = 1.0 / sqrt((double)d);
+  double* R = (double*)malloc(sizeof(double) * d * d);
+  iqo_rotation_matrix(d, quats + (size_t)g * (d / 4) * 8, R);
+  size_t base = ((size_t)b * H_kv + g) * t_cap;
+  double* qt = (double*)malloc(sizeof(double) * d);
+  double* row = (double*)malloc(sizeof(double) * d);
+  for (int i = 0; i < d; i++) {
+    double acc = 0;
+    for (int j = 0; j < d; j++) acc += R[(size_t)i * d + j] * iqo_half_to_double(q_bh[j]);
+    qt[i] = acc;
+  }
+  for (int j = 0; j < len; j++) {
+    dequant_row(d, k_codes + (base + j) * P, k_scales[base + j], levels8, row);
+    double acc = 0;
+    for (int i = 0; i < d; i++) acc += qt[i] * row[i];
+    z_out[j] = sm_scale * acc;
+  }
+  free(R); free(qt); free(row);
+}
+
+/* Merge of split-softmax partials from the definition of softmax (not in the paper: the paper's
+ * pipeline is unsplit; the split is the flash-decoding decomposition of the same sums).
+ * part_acc [B][H_q][S][d] = sum_{j in split} exp(z_j - m_s) v~_j (rotated space), part_ml [B][H_q][S][2]
+ * = (m_s, l_s) with m_s = max z_j (-inf if empty), l_s = sum exp(z_j - m_s); part_argmax [B][H_q][S]
+ * (row index attaining m_s, -1 if empty) or NULL.
+ * out = R^T ( sum_s acc_s e^{m_s - m} / sum_s l_s e^{m_s - m} ), m = max_s m_s. */
+void iqo_combine_splits(int B, int H_q, int H_kv, int d, int S, const float* quats, const float* part_acc,
+                        const float* part_ml, const int32_t* part_argmax, double* out, double* lse,
+                        int32_t* argmax) {
+  int G = H_q / H_kv;
+  for (int b = 0; b < B; b++)
+    for (int h = 0; h < H_q; h++) {
+      size_t o = (size_t)b * H_q + h;
+      double m = -INFINITY;
+      int best = -1;
+      for (int s = 0; s < S; s++) {
+        double ms = part_ml[(o * S + s) * 2];
+        double ls = part_ml[(o * S + s) * 2 + 1];
+        if (!(ls > 0)) continue;
+        int idx = part_argmax ? part_argmax[o * S + s] : -1;
+        if (ms > m) { m = ms; best = idx; }
+        else if (ms == m && idx >= 0 && (best < 0 || idx < best)) best = idx;
+      }
+      double l = 0;
+      double* orot = (double*)calloc(d, sizeof(double));
+      for (int s = 0; s < S; s++) {
+        double ms = part_ml[(o * S + s) * 2];
+        double ls = part_ml[(o * S + s) * 2 + 1];
+        if (!(ls > 0)) continue;
+        double w = exp(ms - m);
+        l += ls * w;
+        for (int i = 0; i < d; i++) orot[i] += w * (double)part_acc[(o * S + s) * d + i];
+      }
+      double* R = (double*)malloc(sizeof(double) * d * d);
+      iqo_rotation_matrix(d, quats + (size_t)(h / G) * (d / 4) * 8, R);
+      for (int j = 0; j < d; j++) {
+        double acc = 0;
+        if (l > 0) for (int i = 0; i < d; i++) acc += R[(size_t)i * d + j] * orot[i] / l;
+        out[o * d + j] = acc;
+      }
+      if (lse) lse[o] = (l > 0) ? m + log(l) : -INFINITY;
+      if (argmax) argmax[o] = (l > 0) ? best : -1;
+      free(R); free(orot);
+    }
+}

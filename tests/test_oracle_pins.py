@@ -1,0 +1,393 @@
+"""Pins for the fp64 oracle: every check here is against something other than the oracle itself --
+the paper's printed counts, mathematical invariants, library routines, closed forms typed out
+independently, or brute force on tiny inputs. CPU only."""
+import math
+import os
+
+import numpy as np
+import pytest
+import scipy.linalg
+
+import oracle
+import workloads
+from oracle import lloyd_max
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _counts():
+    out = {}
+    for line in open(os.path.join(GOLD, "paper_counts.txt")):
+        line = line.split("#")[0].split()
+        if len(line) == 2:
+            out[line[0]] = float(line[1])
+    return out
+
+
+def _rand_quats(seed, n=1):
+    g = np.random.default_rng(seed)
+    q = g.standard_normal((n, 2, 4))
+    q /= np.linalg.norm(q, axis=-1, keepdims=True)
+    return q.reshape(n, 8).astype(np.float32)
+
+
+# ---------------------------------------------------------------- H_d (Eq. 2)
+@pytest.mark.parametrize("d", [4, 32, 128, 256])
+def test_hadamard_matches_library_and_is_orthogonal(d):
+    H = oracle.hadamard(d)
+    Hint = np.rint(H * math.sqrt(d)).astype(np.int64)
+    assert np.array_equal(Hint @ Hint.T, d * np.eye(d, dtype=np.int64))       # H H^T = d I exactly
+    assert np.array_equal(Hint, scipy.linalg.hadamard(d))                      # Sylvester order
+    assert np.allclose(H, H.T, atol=0) and np.allclose(H @ H, np.eye(d), atol=1e-14)
+    assert np.allclose(H[:, 0], 1 / math.sqrt(d), atol=1e-16)
+
+
+# ---------------------------------------------------------------- SO(4) block (Section 3.3, Appendix B)
+def _closed_form_block(q8):
+    q8 = np.asarray(q8, np.float64)
+    a, b, c, d = q8[:4] / np.linalg.norm(q8[:4])
+    e, f, g, h = q8[4:] / np.linalg.norm(q8[4:])
+    L = np.array([[a, -b, -c, -d], [b, a, -d, c], [c, d, a, -b], [d, -c, b, a]])           # v -> qL v
+    Rm = np.array([[e, f, g, h], [-f, e, -h, g], [-g, h, e, -f], [-h, -g, f, e]])          # v -> v conj(qR)
+    return L @ Rm
+
+
+def test_so4_block_is_a_rotation_and_matches_closed_form():
+    for q8 in _rand_quats(1, 50):
+        M = oracle.so4_block(q8)
+        assert np.allclose(M.T @ M, np.eye(4), atol=1e-14)
+        assert abs(np.linalg.det(M) - 1.0) < 1e-13
+        assert np.allclose(M, _closed_form_block(q8), atol=1e-15)
+        assert np.allclose(oracle.so4_block(-q8), M, atol=1e-15)                # double cover (Appendix B)
+
+
+def test_so4_special_cases():
+    ident = np.array([1, 0, 0, 0, 1, 0, 0, 0], np.float32)
+    assert np.allclose(oracle.so4_block(ident), np.eye(4), atol=0)
+    for q8 in _rand_quats(2, 10):
+        q8[4:] = q8[:4]                                                         # single-quaternion conjugation
+        M = oracle.so4_block(q8)
+        assert np.allclose(M[0], [1, 0, 0, 0], atol=1e-15) and np.allclose(M[:, 0], [1, 0, 0, 0], atol=1e-15)
+        assert abs(np.linalg.det(M[1:, 1:]) - 1) < 1e-13                        # acts as SO(3) on the imaginary part
+    # unnormalised input is renormalised
+    q8 = _rand_quats(3, 1)[0]
+    assert np.allclose(oracle.so4_block(3.0 * q8), oracle.so4_block(q8), atol=1e-7)
+    # a known rotation: qL = qR = (cos t/2, sin t/2, 0, 0) rotates the (j,k) plane by t, fixes (1,i)
+    t = 0.7
+    q = np.array([math.cos(t / 2), math.sin(t / 2), 0, 0] * 2, np.float64)
+    M = _closed_form_block(q)
+    expect = np.eye(4)
+    expect[2:, 2:] = [[math.cos(t), -math.sin(t)], [math.sin(t), math.cos(t)]]
+    assert np.allclose(M, expect, atol=1e-15)
+    assert np.allclose(oracle.so4_block(q.astype(np.float32)), expect, atol=1e-7)
+
+
+# ---------------------------------------------------------------- R = R_SO4 o H_d (Eq. 2, Appendix A)
+@pytest.mark.parametrize("d", [128, 256])
+def test_rotation_is_orthogonal_and_composed_in_the_stated_order(d):
+    quats = workloads.quaternion_pairs(np.random.default_rng(5), 1, d)[0]
+    R = oracle.rotation_matrix(d, quats)
+    assert np.allclose(R.T @ R, np.eye(d), atol=1e-13)
+    g = np.random.default_rng(6)
+    x, y = g.standard_normal(d), g.standard_normal(d)
+    assert abs((R @ x) @ (R @ y) - x @ y) < 1e-12                               # inner products preserved
+    # independent composition: WHT first, then each block on its four contiguous coordinates
+    hx = scipy.linalg.hadamard(d) @ x / math.sqrt(d)
+    ref = np.concatenate([_closed_form_block(quats[b]) @ hx[4 * b:4 * b + 4] for b in range(d // 4)])
+    assert np.allclose(R @ x, ref, atol=1e-13)
+    # identity quaternions leave the WHT alone
+    ident = np.tile(np.array([1, 0, 0, 0, 1, 0, 0, 0], np.float32), (d // 4, 1))
+    assert np.allclose(oracle.rotation_matrix(d, ident), scipy.linalg.hadamard(d) / math.sqrt(d), atol=1e-16)
+
+
+def test_post_wht_coordinate_variance_is_one_over_d():
+    d = 128
+    g = np.random.default_rng(7)
+    x = g.standard_normal((20000, d)) * np.exp(g.standard_normal(d))            # anisotropic rows
+    x /= np.linalg.norm(x, axis=1, keepdims=True)
+    y = x @ oracle.hadamard(d).T
+    assert abs(np.mean(y ** 2) * d - 1) < 1e-12                                  # exact by orthogonality
+    assert np.all(np.abs(np.mean(y ** 2, axis=0) * d - 1) < 0.6)                 # energy spread, no hot channel
+
+
+# ---------------------------------------------------------------- the paper's counts
+def test_paper_counts():
+    c = _counts()
+    d = 128
+    assert oracle.row_bytes(d) == c["packed_row_bytes_d128"] == 3 * d // 8
+    assert 2 * d == c["fp16_row_bytes_d128"]
+    assert round(2 * d / oracle.row_bytes(d), 1) == c["compression_ratio"]
+    quats = workloads.quaternion_pairs(np.random.default_rng(0), 1, d)
+    assert quats.size == c["stored_params_d128"] == c["blocks_d128"] * c["floats_per_block"]
+    assert d * d == c["dense_params_d128"]
+    assert (d // 4) * 6 == c["effective_dof_d128"]
+    assert d * int(math.log2(d)) == c["wht_fmas_d128"]
+    assert (d // 4) * c["so4_fmas_per_block"] == c["so4_fmas_d128"]
+    assert c["wht_fmas_d128"] + c["so4_fmas_d128"] == c["total_fmas_d128"]
+    assert round(c["dense_fmas_d128"] / c["total_fmas_d128"], 1) == c["fma_reduction"]
+    transient_mb = 2 * 28 * 8 * 128 * 2048 * 2 / 1e6                             # Appendix C formula
+    assert abs(transient_mb - c["prefill_transient_mb"]) / c["prefill_transient_mb"] < 0.03
+    assert c["total_fmas_d128"] / (2 * 2048 * 128) < c["inverse_rotation_share_max"]
+
+
+# ---------------------------------------------------------------- Lloyd-Max codebook (Step 3)
+def test_lloyd_max_gaussian_limit_matches_the_textbook_table():
+    rows = [l.split() for l in open(os.path.join(GOLD, "gauss_lloyd_max_8.txt")) if not l.startswith("#")]
+    lv_ref, th_ref, mse_ref = [float(x) for x in rows[0]], [float(x) for x in rows[1]], float(rows[2][0])
+    lv, th, mse = lloyd_max.lloyd_max(0)
+    assert np.allclose(lv[4:], lv_ref, atol=6e-4) and np.allclose(-lv[:4][::-1], lv_ref, atol=6e-4)
+    assert np.allclose(th[4:], th_ref, atol=6e-4) and abs(th[3]) < 1e-9
+    assert abs(mse - mse_ref) < 5e-5
+
+
+@pytest.mark.parametrize("d", [128, 256])
+def test_lloyd_max_is_a_fixed_point_for_the_sphere_marginal(d):
+    from scipy import integrate
+
+    lv, th, mse = lloyd_max.lloyd_max(d)
+    pdf, lim = lloyd_max.sphere_marginal_pdf(d)
+    edges = np.concatenate(([-lim], th, [lim]))
+    for i in range(8):                                                           # centroid condition, independent quadrature
+        xs = np.linspace(edges[i], edges[i + 1], 200001)
+        w = np.array([pdf(x) for x in xs])
+        assert abs(integrate.simpson(xs * w, x=xs) / integrate.simpson(w, x=xs) - lv[i]) < 1e-7
+    assert np.allclose(th, 0.5 * (lv[1:] + lv[:-1]), atol=1e-12)                 # midpoint condition
+    assert np.allclose(lv, -lv[::-1], atol=1e-9)                                 # symmetry
+    g_lv, _, g_mse = lloyd_max.lloyd_max(0)
+    assert np.all(np.abs(lv) < np.abs(g_lv) + 1e-12) and mse < g_mse             # lighter tails than the Gaussian
+    assert np.allclose(lv, g_lv, atol=0.03)
+    # variance of the marginal is 1 in these units (each coordinate of a unit vector has variance 1/d)
+    xs = np.linspace(-lim, lim, 400001)
+    w = np.array([pdf(x) for x in xs])
+    assert abs(integrate.simpson(xs * xs * w, x=xs) / integrate.simpson(w, x=xs) - 1) < 1e-6
+
+
+def test_codebook_as_handed_to_both_sides(codebooks):
+    for d, (lv, th) in codebooks.items():
+        assert lv.dtype == np.float32 and th.dtype == np.float32
+        assert np.array_equal(lv.astype(np.float16).astype(np.float32), lv)      # exactly fp16-representable
+        assert np.all(np.diff(lv) > 0) and np.all(np.diff(th) > 0) and th[3] == 0
+
+
+# ---------------------------------------------------------------- quantise + pack (Algorithm 1)
+@pytest.mark.parametrize("d", [128, 256])
+def test_pack_unpack_roundtrip_and_layout(d):
+    g = np.random.default_rng(11)
+    assert oracle.row_bytes(d) == 3 * d // 8
+    for pattern in [np.zeros(d), np.full(d, 7), np.arange(d) % 8, g.integers(0, 8, d), g.integers(0, 8, d)]:
+        codes = pattern.astype(np.uint8)
+        row = oracle.pack_row(d, codes)
+        assert row.shape == (3 * d // 8,)
+        assert np.array_equal(oracle.unpack_row(d, row), codes)
+    # independent statement of the layout: one coordinate set at a time, every bit accounted for
+    seen = np.zeros(3 * d, dtype=np.int64)
+    for i in range(d):
+        for bit in range(3):
+            codes = np.zeros(d, np.uint8)
+            codes[i] = 1 << bit
+            words = oracle.pack_row(d, codes).view("<u4")
+            grp, c = divmod(i, 32)
+            if c < 24:
+                w, pos = 3 * grp + c // 8, 4 * (c % 8) + bit
+            else:
+                w, pos = 3 * grp + bit, 4 * (c - 24) + 3
+            expect = np.zeros(3 * d // 32, np.uint32)
+            expect[w] = np.uint32(1) << np.uint32(pos)
+            assert np.array_equal(words, expect)
+            seen[32 * w + pos] += 1
+    assert np.all(seen == 1)                                                    # a bijection onto the 3d bits
+
+
+def test_quantize_row_against_an_independent_numpy_statement(codebooks):
+    d = 128
+    lv, th = codebooks[d]
+    w = workloads.config1(T=64)
+    R = oracle.rotation_matrix(d, w.quats[0])
+    for t in range(64):
+        x16 = w.k[0, t, 0]
+        codes, scale, u = oracle.quantize_row(d, R, th, x16)
+        x = x16.astype(np.float64)
+        s = math.sqrt(float(np.sum(x * x)))
+        assert scale == np.float32(s)
+        hx = scipy.linalg.hadamard(d) @ (x / s) / math.sqrt(d)
+        xt = np.concatenate([_closed_form_block(w.quats[0, b]) @ hx[4 * b:4 * b + 4] for b in range(d // 4)])
+        u_ref = math.sqrt(d) * xt
+        assert np.allclose(u, u_ref, atol=1e-12)
+        assert abs(np.sum(u * u) - d) < 1e-9                                     # rotation preserves the unit norm
+        far = np.min(np.abs(u_ref[:, None] - th[None, :].astype(np.float64)), axis=1) > 1e-9
+        nearest = np.argmin(np.abs(u_ref[:, None] - lv[None, :].astype(np.float64)), axis=1)
+        assert np.array_equal(codes[far], nearest[far].astype(np.uint8))        # threshold rule == nearest level
+        assert np.array_equal(codes, np.sum(u_ref[:, None] > th[None, :].astype(np.float64), axis=1))
+
+
+def test_quantizer_ties_and_zero_row(codebooks):
+    d = 128
+    lv, th = codebooks[d]
+    ident = np.tile(np.array([1, 0, 0, 0, 1, 0, 0, 0], np.float32), (d // 4, 1))
+    R = oracle.rotation_matrix(d, ident)
+    codes, scale, u = oracle.quantize_row(d, R, th, np.zeros(d, np.float16))
+    assert scale == 0 and np.all(u == 0) and np.all(codes == 3)                  # 0 > t_3 = 0 is false: lower code
+    # a row whose rotated image sits exactly on thresholds: use R = I-like probe through the definition
+    codes2 = np.sum(np.array([th[5], np.nextafter(th[5], np.float32(9))], np.float64)[:, None] > th[None, :].astype(np.float64), axis=1)
+    assert list(codes2) == [5, 6]
+
+
+@pytest.mark.parametrize("maker,lo,hi", [
+    (lambda: workloads.tiny(1, 1, 1, 1, 128, 512), 0.030, 0.038),               # Gaussian rows: the codebook's own MSE
+    (lambda: workloads.config1(T=512), 0.025, 0.045),                            # x20 outlier channels
+    (lambda: workloads.config3(T=256), 0.02, 0.08),                              # Student-t, d = 256
+])
+def test_roundtrip_reconstruction_error(codebooks, maker, lo, hi):
+    w = maker()
+    lv, th = codebooks[w.d]
+    cache = oracle.new_cache(w.B, w.H_kv, w.d, w.t_cap)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(w.B, np.int32), None, cache)
+    errs = []
+    for g in range(w.H_kv):
+        R = oracle.rotation_matrix(w.d, w.quats[g])
+        for t in range(0, w.k.shape[1], 7):
+            codes = oracle.unpack_row(w.d, cache["k_codes"][0, g, t])
+            xr = R.T @ (float(cache["k_scales"][0, g, t]) * lv[codes].astype(np.float64) / math.sqrt(w.d))
+            x = w.k[0, t, g].astype(np.float64)
+            errs.append(np.sum((x - xr) ** 2) / np.sum(x * x))
+    assert lo < float(np.mean(errs)) < hi
+
+
+# ---------------------------------------------------------------- attention (Appendix A)
+def _reconstruct_then_attend(w, lv, cache, sm_scale=None):
+    """Brute force in numpy: dequantise every row, undo the rotation per row, textbook softmax attention."""
+    d = w.d
+    out = np.zeros((w.B, w.H_q, d))
+    am = np.zeros((w.B, w.H_q), np.int64)
+    for b in range(w.B):
+        n = int(w.seq_lens[b])
+        for h in range(w.H_q):
+            g = h // w.G
+            R = oracle.rotation_matrix(d, w.quats[g])
+            K = np.stack([R.T @ (float(cache["k_scales"][b, g, t]) * lv[oracle.unpack_row(d, cache["k_codes"][b, g, t])].astype(np.float64) / math.sqrt(d)) for t in range(n)]) if n else np.zeros((0, d))
+            V = np.stack([R.T @ (float(cache["v_scales"][b, g, t]) * lv[oracle.unpack_row(d, cache["v_codes"][b, g, t])].astype(np.float64) / math.sqrt(d)) for t in range(n)]) if n else np.zeros((0, d))
+            if n == 0:
+                am[b, h] = -1
+                continue
+            z = (K @ w.q[b, h].astype(np.float64)) * (sm_scale or 1 / math.sqrt(d))
+            p = np.exp(z - z.max())
+            p /= p.sum()
+            out[b, h] = p @ V
+            am[b, h] = int(np.argmax(z))
+    return out, am
+
+
+@pytest.mark.parametrize("d,T,H_q,H_kv,lens", [(128, 64, 4, 1, None), (128, 37, 4, 2, [37, 5]), (256, 16, 2, 2, None),
+                                               (128, 8, 2, 1, [0])])
+def test_compressed_space_attention_equals_reconstruct_then_compute(codebooks, d, T, H_q, H_kv, lens):
+    B = 1 if lens is None else len(lens)
+    w = workloads.tiny(3, B, H_q, H_kv, d, T, lens)
+    lv, th = codebooks[d]
+    cache = oracle.new_cache(B, H_kv, d, T)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), w.seq_lens, cache)
+    r = oracle.decode_attention(w.quats, lv, w.q, cache, w.seq_lens, H_kv, want_rot=True)
+    ref, am = _reconstruct_then_attend(w, lv, cache)
+    assert np.allclose(r["out"], ref, atol=1e-12)
+    assert np.array_equal(r["argmax"], am)
+    # omitting the inverse rotation must NOT reproduce the output (the paper's PPL 7.05 -> 15,369 remark)
+    if w.seq_lens.max() > 0:
+        assert np.max(np.abs(r["o_rot"] - ref)) > 0.05
+
+
+def test_attention_special_cases(codebooks):
+    d = 128
+    lv, th = codebooks[d]
+    w = workloads.tiny(4, 1, 2, 1, d, 16)
+    cache = oracle.new_cache(1, 1, d, 16)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(1, np.int32), None, cache)
+    R = oracle.rotation_matrix(d, w.quats[0])
+    recon = lambda c, s: R.T @ (float(s) * lv[oracle.unpack_row(d, c)].astype(np.float64) / math.sqrt(d))
+    # T = 1: the output is the reconstruction of v_0
+    r = oracle.decode_attention(w.quats, lv, w.q, cache, np.array([1], np.int32), 1)
+    assert np.allclose(r["out"][0, 0], recon(cache["v_codes"][0, 0, 0], cache["v_scales"][0, 0, 0]), atol=1e-13)
+    assert np.all(r["argmax"] == 0)
+    # all keys equal: uniform weights -> mean of reconstructed V, argmax = lowest index
+    cache["k_codes"][0, 0, :] = cache["k_codes"][0, 0, 0]
+    cache["k_scales"][0, 0, :] = cache["k_scales"][0, 0, 0]
+    r = oracle.decode_attention(w.quats, lv, w.q, cache, np.array([16], np.int32), 1)
+    mean_v = np.mean([recon(cache["v_codes"][0, 0, t], cache["v_scales"][0, 0, t]) for t in range(16)], axis=0)
+    assert np.allclose(r["out"][0, 1], mean_v, atol=1e-13) and np.all(r["argmax"] == 0)
+    for h in range(2):
+        assert abs(r["lse"][0, h] - (oracle.scores(w.quats, lv, w.q, cache, 0, h, 16, 1)[0] + math.log(16))) < 1e-12
+    # empty sequence
+    r = oracle.decode_attention(w.quats, lv, w.q, cache, np.array([0], np.int32), 1)
+    assert np.all(r["out"] == 0) and np.all(r["argmax"] == -1) and np.all(np.isneginf(r["lse"]))
+
+
+def test_score_error_statistics_against_the_bound(codebooks):
+    """Eq. 3 / Appendix A: E|q.k - q.k_hat|^2 = sigma_q^2 ||q||^2 (derivation), <= d_k sigma_q^2 ||q||^2 (as printed),
+    with sigma_q^2 the per-coordinate quantisation variance of the de-normalised rotated key."""
+    d = 128
+    lv, th = codebooks[d]
+    w = workloads.tiny(5, 1, 1, 1, d, 4096)
+    cache = oracle.new_cache(1, 1, d, 4096)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(1, np.int32), None, cache)
+    z = oracle.scores(w.quats, lv, w.q, cache, 0, 0, 4096, 1, sm_scale=1.0)
+    q = w.q[0, 0].astype(np.float64)
+    exact = w.k[0, :, 0].astype(np.float64) @ q
+    s2 = np.mean(cache["k_scales"][0, 0].astype(np.float64) ** 2)
+    _, _, mse = lloyd_max.lloyd_max(d)
+    sigma2 = s2 * mse / d
+    measured = float(np.mean((z - exact) ** 2))
+    tight = sigma2 * float(q @ q)
+    assert 0.7 * tight < measured < 1.3 * tight
+    assert measured < d * tight
+
+
+def test_split_merge_equals_unsplit_softmax(codebooks):
+    d = 128
+    lv, th = codebooks[d]
+    w = workloads.tiny(6, 2, 4, 2, d, 100, lens=[100, 63])
+    cache = oracle.new_cache(2, 2, d, 100)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(2, np.int32), w.seq_lens, cache)
+    full = oracle.decode_attention(w.quats, lv, w.q, cache, w.seq_lens, 2, want_rot=True)
+    g = np.random.default_rng(1)
+    for S in (1, 3, 7):
+        pa = np.zeros((2, 4, S, d), np.float32)
+        pm = np.zeros((2, 4, S, 2), np.float32)
+        pg = np.full((2, 4, S), -1, np.int32)
+        for b in range(2):
+            n = int(w.seq_lens[b])
+            cuts = np.sort(np.concatenate(([0, n], g.integers(0, n + 1, S - 1))))     # arbitrary partition, may have empty splits
+            for h in range(4):
+                z = oracle.scores(w.quats, lv, w.q, cache, b, h, n, 2)
+                R = oracle.rotation_matrix(d, w.quats[h // 2])
+                for s in range(S):
+                    lo, hi = cuts[s], cuts[s + 1]
+                    if hi == lo:
+                        pm[b, h, s] = (-np.inf, 0)
+                        continue
+                    m = z[lo:hi].max()
+                    p = np.exp(z[lo:hi] - m)
+                    vt = np.stack([float(cache["v_scales"][b, h // 2, t]) * lv[oracle.unpack_row(d, cache["v_codes"][b, h // 2, t])].astype(np.float64) / math.sqrt(d) for t in range(lo, hi)])
+                    pa[b, h, s] = p @ vt
+                    pm[b, h, s] = (m, p.sum())
+                    pg[b, h, s] = lo + int(np.argmax(z[lo:hi]))
+        r = oracle.combine_splits(w.quats, pa, pm, pg, 2)
+        assert np.allclose(r["out"], full["out"], atol=2e-6)                      # fp32 partials
+        assert np.allclose(r["lse"], full["lse"], atol=1e-5)
+        assert np.array_equal(r["argmax"], full["argmax"])
+
+
+def test_retrieval_margins_config4_shape(codebooks):
+    """Planted key scores ~ 4 ||q||^2 / sqrt(d) ~ 45, far above the Gaussian background: argmax is unambiguous."""
+    d = 128
+    lv, th = codebooks[d]
+    w = workloads.config4(T=2048, H_q=8, H_kv=2)
+    cache = oracle.new_cache(1, 2, d, 2048)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(1, np.int32), None, cache)
+    r = oracle.decode_attention(w.quats, lv, w.q, cache, w.seq_lens, 2)
+    assert np.array_equal(r["argmax"][0], w.extra["needle_pos"])
+    for h in range(8):
+        z = oracle.scores(w.quats, lv, w.q, cache, 0, h, 2048, 2)
+        top2 = np.sort(z)[-2:]
+        assert top2[1] - top2[0] > 15
+        o = r["out"][0, h]
+        assert int(np.argmax(np.abs(o))) == int(w.extra["needle_chan"][h])
+        vn = w.v[0, w.extra["needle_pos"][h], h // 4].astype(np.float64)
+        assert (o @ vn) / (np.linalg.norm(o) * np.linalg.norm(vn)) > 0.9
