@@ -1,0 +1,181 @@
+/*
+ * isoquant.h -- C ABI of the IsoQuant compressed-space decode-attention library (CUDA, sm_100a).
+ *
+ * The library implements the data-parallel hot path of IsoQuant KV-cache compression:
+ *
+ *   quantize-append   Algorithm 1 of the paper: s = ||x||_2, x^ = x/s, x~ = R_SO4(H_d x^) (Eq. 2),
+ *                     3-bit Lloyd-Max code per coordinate (Step 3), bit-pack (Step 4).
+ *   fused decode      Appendix A: q~ = R q once, scores q~ . k~_j / sqrt(d_k) taken directly on the
+ *                     packed codes, softmax, o~ = sum_j alpha_j v~_j accumulated directly on the packed
+ *                     codes, o = R^T o~ once (Table 2, kernels A-D). FP16 K/V are never materialised.
+ *                     The context is split flash-decoding style; the partial results are merged by
+ *                     iq_combine_splits, which also applies the single inverse rotation.
+ *
+ * Conventions
+ *   - Every pointer named *_dev (and every cache / partial / q / out pointer) is DEVICE memory owned by
+ *     the caller. Pointers named *_host and the iq_shape / iq_codebook / iq_cache structs are HOST memory,
+ *     read during the call only. The library allocates nothing and keeps no state between calls.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream). Calls enqueue work on it
+ *     and return without synchronising. They never throw or abort.
+ *   - Every entry point returns IQ_OK (0) or a negative IQ_ERR_* code. Arguments are validated on the host
+ *     before anything is launched; on an error nothing has been enqueued.
+ *   - Device-side conditions that cannot be known on the host are reported through an optional
+ *     `status_dev` array of 4 uint32 (zeroed by the caller): [0] bit mask of IQ_STATUS_* flags,
+ *     [1] rows whose codes were re-decided in fp64 (see iq_quantize_append), [2] rows skipped because
+ *     they fell outside the cache, [3] reserved. Nothing on the device traps or spins without a bound.
+ *
+ * Rotation (Eq. 2, Section 3.3 "SO(4) parameterization", Appendix B)
+ *   R = R_SO4 o H_d. H_d is the normalised Walsh-Hadamard matrix in natural (Sylvester) order,
+ *   H[i][j] = (-1)^popcount(i & j) / sqrt(d). R_SO4 is block diagonal: block b = 0 .. d/4-1 acts on
+ *   coordinates [4b, 4b+4) as v -> q_L v conj(q_R) with unit quaternions stored (w, x, y, z), Hamilton
+ *   product, the four coordinates read as y0 + y1 i + y2 j + y3 k. Storage: [n_kv_heads][d/4][8] fp32 =
+ *   (q_L.wxyz, q_R.wxyz): 8 floats per block, 256 per head at d = 128 (Appendix B). K and V of a KV head
+ *   and all query heads of its group share that head's rotation.
+ *
+ * Codebook (Section 3.2, Step 3)
+ *   8 ascending levels and 7 ascending decision thresholds in unit-variance units u = sqrt(d) * x~.
+ *   code = #{ j : u > t_j } (strict: an exact tie takes the lower code). The 8 levels must be exactly
+ *   representable in IEEE binary16: the decode kernel feeds them to fp16 tensor-core operands and must
+ *   not round them (IQ_ERR_CODEBOOK otherwise). A dequantised coordinate is scale * level[code] / sqrt(d).
+ *
+ * Packed cache (Section 3.2, Step 4 fixes the size only: 3d/8 bytes per row, 48 at d = 128)
+ *   codes  [batch][n_kv_heads][t_cap][3d/8] uint8, scales [batch][n_kv_heads][t_cap] fp32 (= ||x||_2),
+ *   separately for K and V. A row is a sequence of little-endian 32-bit words; coordinates are taken in
+ *   groups of 32, each group owning 3 consecutive words. In group-local numbering, coordinate c < 24
+ *   stores its code in bits [4n, 4n+3) of word c/8, n = c mod 8; coordinate c >= 24 (n = c - 24) stores
+ *   bit k of its code in bit 4n+3 of word k. t_cap must be a multiple of 4 and all four arrays 16-byte
+ *   aligned, so that every tile the decode kernel copies starts on a 16-byte boundary.
+ */
+#ifndef ISOQUANT_H_
+#define ISOQUANT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define IQ_VERSION 100
+
+enum {
+  IQ_OK = 0,
+  IQ_ERR_NULL = -1,     /* a required pointer is NULL */
+  IQ_ERR_SHAPE = -2,    /* unsupported head_dim / bits, n_q_heads % n_kv_heads != 0, bad sizes or strides */
+  IQ_ERR_ALIGN = -3,    /* a pointer or stride breaks the stated alignment */
+  IQ_ERR_CODEBOOK = -4, /* levels / thresholds not ascending, or a level not representable in binary16 */
+  IQ_ERR_CUDA = -5,     /* the CUDA runtime reported an error for the launch */
+  IQ_ERR_LIMIT = -6     /* a size exceeds a documented maximum of the entry point */
+};
+
+enum {
+  IQ_STATUS_ROW_OUT_OF_RANGE = 1u, /* quantize-append: append_pos + i >= t_cap, row skipped */
+  IQ_STATUS_WAIT_TIMEOUT = 2u      /* decode: a bounded wait on an asynchronous copy ran out; results invalid */
+};
+
+typedef struct iq_shape {
+  int32_t batch;
+  int32_t n_q_heads;
+  int32_t n_kv_heads; /* n_q_heads % n_kv_heads == 0 */
+  int32_t head_dim;   /* 128 or 256 */
+  int32_t t_cap;      /* rows allocated per (sequence, KV head); multiple of 4 */
+  int32_t bits;       /* 3 */
+  float sm_scale;     /* softmax scale; <= 0 selects 1/sqrt(head_dim) (Appendix A) */
+} iq_shape;
+
+typedef struct iq_codebook {
+  float levels[8];
+  float thresholds[7];
+} iq_codebook;
+
+typedef struct iq_cache {
+  uint8_t* k_codes;
+  float* k_scales;
+  uint8_t* v_codes;
+  float* v_scales;
+} iq_cache;
+
+int iq_version(void);
+const char* iq_strerror(int code);
+
+/* Bytes of one packed row: 3 * head_dim / 8 (Section 3.2, Step 4). 0 for an unsupported head_dim. */
+size_t iq_row_bytes(int32_t head_dim);
+/* Floats of the rotation parameter buffer: n_kv_heads * (head_dim / 4) * 8 (Appendix B). */
+size_t iq_rotation_floats(int32_t head_dim, int32_t n_kv_heads);
+
+/*
+ * Lloyd-Max codebook for the post-rotation marginal (Section 3.2, Step 3): one coordinate of a uniform
+ * point on S^{d-1} in unit-variance units, density ~ (1 - u^2/d)^((d-3)/2). Levels are rounded to
+ * binary16-representable values, thresholds are the midpoints of the rounded levels. Host only.
+ */
+int iq_default_codebook(int32_t head_dim, iq_codebook* out_host);
+
+/*
+ * Rotation parameters (Appendix B). If quats_host != NULL it holds [n_kv_heads][d/4][8] floats which are
+ * scaled to unit length per quaternion and copied to rot_dev; otherwise the quaternions are drawn on the
+ * device from `seed` (4 iid N(0,1) components per quaternion from a counter-based generator, scaled to
+ * unit length: Haar measure on S^3). rot_dev: device, iq_rotation_floats() floats, 16-byte aligned.
+ */
+int iq_make_rotation(int32_t head_dim, int32_t n_kv_heads, uint64_t seed, const float* quats_host,
+                     float* rot_dev, void* stream);
+
+/*
+ * Algorithm 1 for the new K and V rows of every sequence and KV head; results appended to the cache.
+ *   k_new, v_new   device, binary16; element (b, i, h, c) at b*stride_b + i*stride_t + h*stride_h + c
+ *                  (strides in elements, multiples of 8; base pointers 16-byte aligned).
+ *   append_pos_dev device int32 [batch]: cache row that receives new row 0 of sequence b.
+ *   n_new_dev      device int32 [batch] rows to append per sequence (clamped to n_new_max), or NULL for
+ *                  n_new_max everywhere. n_new_max = 0 is a no-op.
+ *   cache          host struct of device pointers; rows append_pos[b] + i are overwritten. The call does
+ *                  not touch any sequence-length array: the caller advances its lengths.
+ *   status_dev     optional (see top). Rows with append_pos + i outside [0, t_cap) are skipped and flagged.
+ * Arithmetic: fp32 butterfly WHT and 4x4 block products; any row with a coordinate closer than 2^-15 to a
+ * decision threshold is re-decided in fp64 inside the kernel, so the codes equal those of an fp64
+ * evaluation except for ties at the fp64 rounding level. The stored scale is sqrt(sum x^2) accumulated
+ * in fp64 and rounded to fp32. A zero row stores scale 0 and the code of u = 0 everywhere.
+ */
+int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook,
+                       const void* k_new, const void* v_new, int64_t stride_b, int64_t stride_t,
+                       int64_t stride_h, const int32_t* append_pos_dev, const int32_t* n_new_dev,
+                       int32_t n_new_max, const iq_cache* cache, uint32_t* status_dev, void* stream);
+
+/*
+ * Fused decode step on the packed cache (Appendix A; Table 2, kernels A-C), split over the context.
+ *   q              device binary16 [batch][n_q_heads][head_dim], 16-byte aligned; not quantised.
+ *   seq_lens_dev   device int32 [batch]: rows 0 .. len-1 of each sequence are attended to (clamped to
+ *                  [0, t_cap]); the row appended last is attended to like any other.
+ *   num_splits     S >= 1. Sequence b is cut into S consecutive chunks of
+ *                  64 * ceil(ceil(len_b / S) / 64) rows; trailing chunks may be empty.
+ *   part_acc       device fp32 [batch][n_q_heads][S][head_dim]: sum_j exp(z_j - m) v~_j over the chunk,
+ *                  in the rotated space, natural coordinate order. 16-byte aligned.
+ *   part_ml        device fp32 [batch][n_q_heads][S][2] = (m, l): m = max_j z_j, l = sum_j exp(z_j - m),
+ *                  z_j = sm_scale * q~ . k~_j. An empty chunk holds (-inf, 0) and acc = 0.
+ *   part_argmax    device int32 [batch][n_q_heads][S] or NULL: row index attaining m (lowest on ties), -1 if empty.
+ *   status_dev     optional (see top).
+ * Arithmetic: q~ and the probabilities enter fp16 tensor-core operands (q~ as a two-term fp16 sum),
+ * codebook levels are exact fp16 values, every accumulation is fp32.
+ */
+int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook,
+                        const void* q, const iq_cache* cache, const int32_t* seq_lens_dev,
+                        int32_t num_splits, float* part_acc, float* part_ml, int32_t* part_argmax,
+                        uint32_t* status_dev, void* stream);
+
+/*
+ * Merge of the split partials and the single inverse rotation (Table 2, kernel D):
+ *   m = max_s m_s, l = sum_s l_s e^{m_s - m}, o~ = sum_s acc_s e^{m_s - m} / l, o = R^T o~ = H_d blockdiag(M_b^T) o~.
+ *   out            device [batch][n_q_heads][head_dim], fp32 or (out_is_fp16 != 0) binary16; 16-byte aligned.
+ *   lse_out        device fp32 [batch][n_q_heads] or NULL: m + log(l) (-inf for an empty sequence).
+ *   argmax_out     device int32 [batch][n_q_heads] or NULL (needs part_argmax): row with the largest score.
+ * A sequence of length 0 yields out = 0, lse = -inf, argmax = -1.
+ */
+int iq_combine_splits(const iq_shape* shape, const float* rot_dev, int32_t num_splits,
+                      const float* part_acc, const float* part_ml, const int32_t* part_argmax,
+                      void* out, int32_t out_is_fp16, float* lse_out, int32_t* argmax_out, void* stream);
+
+/* A split count that fills the GPU for this shape when the longest sequence has max_seq_len rows. */
+int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ISOQUANT_H_ */

@@ -1,0 +1,27 @@
+"""IsoQuant compressed-space decode attention for B200 (sm_100a).
+
+A thin Python binding over the C-ABI CUDA library `libisoquant.so` (declared in include/isoquant.h). Every
+step of the path runs in the library's kernels; this package only marshals arguments (torch tensors ->
+device pointers, the current torch stream -> cudaStream_t). There is no CPU fallback: if the compiled
+library is missing or fails to load, importing `paper_2608_08081_b200.binding` raises.
+"""
+from .binding import (  # noqa: F401
+    IQError,
+    Cache,
+    Codebook,
+    Shape,
+    iq_combine_splits,
+    iq_decode_attention,
+    iq_default_codebook,
+    iq_make_rotation,
+    iq_quantize_append,
+    iq_rotation_floats,
+    iq_row_bytes,
+    iq_strerror,
+    iq_suggest_splits,
+    iq_version,
+    lib_path,
+    new_cache,
+    DecodeWorkspace,
+    decode_step,
+)

@@ -1,0 +1,216 @@
+"""ctypes binding of libisoquant.so: same names as the C ABI, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+from . import build as _build
+
+_vp = ctypes.c_void_p
+_i32 = ctypes.c_int32
+_i64 = ctypes.c_int64
+
+
+class _IqShape(ctypes.Structure):
+    _fields_ = [("batch", _i32), ("n_q_heads", _i32), ("n_kv_heads", _i32), ("head_dim", _i32),
+                ("t_cap", _i32), ("bits", _i32), ("sm_scale", ctypes.c_float)]
+
+
+class _IqCodebook(ctypes.Structure):
+    _fields_ = [("levels", ctypes.c_float * 8), ("thresholds", ctypes.c_float * 7)]
+
+
+class _IqCache(ctypes.Structure):
+    _fields_ = [("k_codes", _vp), ("k_scales", _vp), ("v_codes", _vp), ("v_scales", _vp)]
+
+
+class IQError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {iq_strerror(code)} ({code})")
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def _load():
+    path = lib_path()
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -m paper_2608_08081_b200.build` (needs nvcc). "
+            "There is no fallback implementation.")
+    lib = ctypes.CDLL(path)
+    lib.iq_version.restype = ctypes.c_int
+    lib.iq_strerror.restype = ctypes.c_char_p
+    lib.iq_strerror.argtypes = [ctypes.c_int]
+    lib.iq_row_bytes.restype = ctypes.c_size_t
+    lib.iq_row_bytes.argtypes = [_i32]
+    lib.iq_rotation_floats.restype = ctypes.c_size_t
+    lib.iq_rotation_floats.argtypes = [_i32, _i32]
+    lib.iq_default_codebook.argtypes = [_i32, ctypes.POINTER(_IqCodebook)]
+    lib.iq_make_rotation.argtypes = [_i32, _i32, ctypes.c_uint64, _vp, _vp, _vp]
+    lib.iq_quantize_append.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp, _vp, _i64, _i64,
+                                       _i64, _vp, _vp, _i32, ctypes.POINTER(_IqCache), _vp, _vp]
+    lib.iq_decode_attention.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp,
+                                        ctypes.POINTER(_IqCache), _vp, _i32, _vp, _vp, _vp, _vp, _vp]
+    lib.iq_combine_splits.argtypes = [ctypes.POINTER(_IqShape), _vp, _i32, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
+    lib.iq_suggest_splits.restype = _i32
+    lib.iq_suggest_splits.argtypes = [ctypes.POINTER(_IqShape), _i32]
+    return lib
+
+
+_lib = _load()
+
+
+@dataclass
+class Shape:
+    batch: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    t_cap: int
+    bits: int = 3
+    sm_scale: float = 0.0
+
+    def c(self) -> _IqShape:
+        return _IqShape(self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.t_cap, self.bits, self.sm_scale)
+
+
+@dataclass
+class Codebook:
+    levels: tuple
+    thresholds: tuple
+
+    def c(self) -> _IqCodebook:
+        cb = _IqCodebook()
+        for i in range(8):
+            cb.levels[i] = float(self.levels[i])
+        for i in range(7):
+            cb.thresholds[i] = float(self.thresholds[i])
+        return cb
+
+
+@dataclass
+class Cache:
+    k_codes: torch.Tensor   # uint8 [B][H_kv][t_cap][3d/8]
+    k_scales: torch.Tensor  # fp32  [B][H_kv][t_cap]
+    v_codes: torch.Tensor
+    v_scales: torch.Tensor
+
+    def c(self) -> _IqCache:
+        return _IqCache(self.k_codes.data_ptr(), self.k_scales.data_ptr(), self.v_codes.data_ptr(), self.v_scales.data_ptr())
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise IQError(rc, where)
+
+
+def iq_version() -> int:
+    return int(_lib.iq_version())
+
+
+def iq_strerror(code: int) -> str:
+    return _lib.iq_strerror(int(code)).decode()
+
+
+def iq_row_bytes(head_dim: int) -> int:
+    return int(_lib.iq_row_bytes(head_dim))
+
+
+def iq_rotation_floats(head_dim: int, n_kv_heads: int) -> int:
+    return int(_lib.iq_rotation_floats(head_dim, n_kv_heads))
+
+
+def iq_default_codebook(head_dim: int) -> Codebook:
+    cb = _IqCodebook()
+    _check(_lib.iq_default_codebook(head_dim, ctypes.byref(cb)), "iq_default_codebook")
+    return Codebook(tuple(cb.levels), tuple(cb.thresholds))
+
+
+def iq_make_rotation(head_dim: int, n_kv_heads: int, seed: int, quats_host, rot_dev: torch.Tensor, stream=None) -> None:
+    """quats_host: None or a contiguous fp32 numpy array [n_kv_heads][head_dim/4][8]."""
+    qp = None
+    if quats_host is not None:
+        assert quats_host.dtype.name == "float32" and quats_host.flags["C_CONTIGUOUS"]
+        assert quats_host.size == iq_rotation_floats(head_dim, n_kv_heads)
+        qp = quats_host.ctypes.data
+    _check(_lib.iq_make_rotation(head_dim, n_kv_heads, ctypes.c_uint64(seed), qp, _ptr(rot_dev), _stream(stream)),
+           "iq_make_rotation")
+
+
+def iq_quantize_append(shape: Shape, rot_dev, codebook: Codebook, k_new, v_new, append_pos_dev, n_new_dev,
+                       n_new_max: int, cache: Cache, status_dev=None, stream=None) -> None:
+    """k_new, v_new: fp16 device tensors [B][n_new_max][H_kv][d] (any strides with a contiguous last dim)."""
+    assert k_new.dtype == torch.float16 and v_new.dtype == torch.float16
+    assert k_new.stride() == v_new.stride() and k_new.stride(3) == 1
+    sb, st, sh = k_new.stride(0), k_new.stride(1), k_new.stride(2)
+    cs, cb, cc = shape.c(), codebook.c(), cache.c()
+    _check(_lib.iq_quantize_append(ctypes.byref(cs), _ptr(rot_dev), ctypes.byref(cb), _ptr(k_new), _ptr(v_new), sb, st, sh,
+                                   _ptr(append_pos_dev), _ptr(n_new_dev), n_new_max, ctypes.byref(cc), _ptr(status_dev),
+                                   _stream(stream)), "iq_quantize_append")
+
+
+def iq_decode_attention(shape: Shape, rot_dev, codebook: Codebook, q, cache: Cache, seq_lens_dev, num_splits: int,
+                        part_acc, part_ml, part_argmax=None, status_dev=None, stream=None) -> None:
+    cs, cb, cc = shape.c(), codebook.c(), cache.c()
+    _check(_lib.iq_decode_attention(ctypes.byref(cs), _ptr(rot_dev), ctypes.byref(cb), _ptr(q), ctypes.byref(cc),
+                                    _ptr(seq_lens_dev), num_splits, _ptr(part_acc), _ptr(part_ml), _ptr(part_argmax),
+                                    _ptr(status_dev), _stream(stream)), "iq_decode_attention")
+
+
+def iq_combine_splits(shape: Shape, rot_dev, num_splits: int, part_acc, part_ml, part_argmax, out, lse_out=None,
+                      argmax_out=None, stream=None) -> None:
+    cs = shape.c()
+    _check(_lib.iq_combine_splits(ctypes.byref(cs), _ptr(rot_dev), num_splits, _ptr(part_acc), _ptr(part_ml),
+                                  _ptr(part_argmax), _ptr(out), 1 if out.dtype == torch.float16 else 0, _ptr(lse_out),
+                                  _ptr(argmax_out), _stream(stream)), "iq_combine_splits")
+
+
+def iq_suggest_splits(shape: Shape, max_seq_len: int) -> int:
+    cs = shape.c()
+    return int(_lib.iq_suggest_splits(ctypes.byref(cs), max_seq_len))
+
+
+# ------------------------------------------------------------------ small conveniences (allocation only)
+def new_cache(shape: Shape, device="cuda") -> Cache:
+    P = iq_row_bytes(shape.head_dim)
+    n = (shape.batch, shape.n_kv_heads, shape.t_cap)
+    return Cache(torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=torch.float32, device=device),
+                 torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=torch.float32, device=device))
+
+
+class DecodeWorkspace:
+    """Caller-owned partial buffers for a fixed shape and split count."""
+
+    def __init__(self, shape: Shape, num_splits: int, want_argmax: bool = False, device="cuda"):
+        B, H, d, S = shape.batch, shape.n_q_heads, shape.head_dim, num_splits
+        self.num_splits = S
+        self.part_acc = torch.empty((B, H, S, d), dtype=torch.float32, device=device)
+        self.part_ml = torch.empty((B, H, S, 2), dtype=torch.float32, device=device)
+        self.part_argmax = torch.empty((B, H, S), dtype=torch.int32, device=device) if want_argmax else None
+        self.out = torch.empty((B, H, d), dtype=torch.float32, device=device)
+        self.lse = torch.empty((B, H), dtype=torch.float32, device=device)
+        self.argmax = torch.empty((B, H), dtype=torch.int32, device=device) if want_argmax else None
+        self.status = torch.zeros(4, dtype=torch.int32, device=device)
+
+
+def decode_step(shape: Shape, rot_dev, codebook: Codebook, q, cache: Cache, seq_lens_dev, ws: DecodeWorkspace, stream=None):
+    """iq_decode_attention followed by iq_combine_splits into the workspace's output buffers."""
+    iq_decode_attention(shape, rot_dev, codebook, q, cache, seq_lens_dev, ws.num_splits, ws.part_acc, ws.part_ml,
+                        ws.part_argmax, ws.status, stream)
+    iq_combine_splits(shape, rot_dev, ws.num_splits, ws.part_acc, ws.part_ml, ws.part_argmax, ws.out, ws.lse, ws.argmax, stream)
+    return ws.out

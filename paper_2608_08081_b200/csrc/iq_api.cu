@@ -1,0 +1,285 @@
+// C ABI of the IsoQuant library: argument validation and kernel launches. See include/isoquant.h for the
+// contract of every entry point. Nothing here allocates device memory or keeps state between calls.
+#include <cmath>
+#include <cstring>
+
+#include "iq_common.cuh"
+#include "iq_kernels.h"
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(const iq_shape* s) {
+  if (!s) return IQ_ERR_NULL;
+  if (s->head_dim != 128 && s->head_dim != 256) return IQ_ERR_SHAPE;
+  if (s->bits != 3) return IQ_ERR_SHAPE;
+  if (s->batch < 0 || s->batch > 65535) return IQ_ERR_SHAPE;
+  if (s->n_kv_heads <= 0 || s->n_q_heads <= 0 || s->n_q_heads % s->n_kv_heads != 0) return IQ_ERR_SHAPE;
+  if (s->t_cap <= 0 || (s->t_cap & 3) != 0) return IQ_ERR_SHAPE;
+  const int hg = (s->n_q_heads / s->n_kv_heads + iq::DEC_HEADS - 1) / iq::DEC_HEADS;
+  if ((long long)s->n_kv_heads * hg > 32767) return IQ_ERR_SHAPE;
+  return IQ_OK;
+}
+
+bool fp16_exact(float x) { return std::isfinite(x) && __half2float(__float2half_rn(x)) == x; }
+
+int check_codebook(const iq_codebook* cb, bool need_fp16_levels) {
+  if (!cb) return IQ_ERR_NULL;
+  for (int i = 0; i < 8; i++) {
+    if (!std::isfinite(cb->levels[i])) return IQ_ERR_CODEBOOK;
+    if (i && !(cb->levels[i] > cb->levels[i - 1])) return IQ_ERR_CODEBOOK;
+    if (need_fp16_levels && !fp16_exact(cb->levels[i])) return IQ_ERR_CODEBOOK;
+  }
+  for (int i = 0; i < 7; i++) {
+    if (!std::isfinite(cb->thresholds[i])) return IQ_ERR_CODEBOOK;
+    if (i && !(cb->thresholds[i] > cb->thresholds[i - 1])) return IQ_ERR_CODEBOOK;
+  }
+  return IQ_OK;
+}
+
+int check_cache(const iq_cache* c) {
+  if (!c || !c->k_codes || !c->k_scales || !c->v_codes || !c->v_scales) return IQ_ERR_NULL;
+  if (!aligned16(c->k_codes) || !aligned16(c->k_scales) || !aligned16(c->v_codes) || !aligned16(c->v_scales)) return IQ_ERR_ALIGN;
+  return IQ_OK;
+}
+
+// Lloyd's iteration for the marginal of one coordinate of a uniform point on S^{d-1}, unit-variance units:
+// density ~ (1 - u^2/d)^((d-3)/2). Cell integrals by composite Simpson on a fixed fine grid.
+struct SphereMarginal {
+  double d;
+  double pdf(double u) const {
+    const double b = 1.0 - u * u / d;
+    return b > 0.0 ? std::exp(0.5 * (d - 3.0) * std::log(b)) : 0.0;
+  }
+  void cell(double a, double b, double& mass, double& mom) const {
+    const int n = 2048;
+    const double hstep = (b - a) / n;
+    double m0 = 0, m1 = 0;
+    for (int i = 0; i <= n; i++) {
+      const double u = a + hstep * i;
+      const double w = (i == 0 || i == n) ? 1.0 : ((i & 1) ? 4.0 : 2.0);
+      const double f = pdf(u);
+      m0 += w * f;
+      m1 += w * f * u;
+    }
+    mass = m0 * hstep / 3.0;
+    mom = m1 * hstep / 3.0;
+  }
+};
+
+void lloyd_max_sphere(int d, double (&lv)[8]) {
+  SphereMarginal f{(double)d};
+  const double lim = std::sqrt((double)d);
+  for (int i = 0; i < 8; i++) lv[i] = -2.1 + 0.6 * i;
+  for (int iter = 0; iter < 5000; iter++) {
+    double edge[9];
+    edge[0] = -lim;
+    edge[8] = lim;
+    for (int i = 1; i < 8; i++) edge[i] = 0.5 * (lv[i - 1] + lv[i]);
+    double delta = 0;
+    for (int i = 0; i < 8; i++) {
+      double mass, mom;
+      f.cell(edge[i], edge[i + 1], mass, mom);
+      const double c = mom / mass;
+      delta = std::fmax(delta, std::fabs(c - lv[i]));
+      lv[i] = c;
+    }
+    if (delta < 1e-13) break;
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+int iq_version(void) { return IQ_VERSION; }
+
+const char* iq_strerror(int code) {
+  switch (code) {
+    case IQ_OK: return "ok";
+    case IQ_ERR_NULL: return "a required pointer is NULL";
+    case IQ_ERR_SHAPE: return "unsupported shape (head_dim 128/256, bits 3, n_q_heads % n_kv_heads == 0, t_cap % 4 == 0, strides % 8 == 0)";
+    case IQ_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
+    case IQ_ERR_CODEBOOK: return "codebook not ascending or a level is not representable in binary16";
+    case IQ_ERR_CUDA: return "CUDA runtime error at launch";
+    case IQ_ERR_LIMIT: return "size exceeds the documented maximum of this entry point";
+    default: return "unknown error code";
+  }
+}
+
+size_t iq_row_bytes(int32_t head_dim) { return (head_dim == 128 || head_dim == 256) ? (size_t)(3 * head_dim / 8) : 0; }
+
+size_t iq_rotation_floats(int32_t head_dim, int32_t n_kv_heads) {
+  if ((head_dim != 128 && head_dim != 256) || n_kv_heads <= 0) return 0;
+  return (size_t)n_kv_heads * (size_t)(head_dim / 4) * 8;
+}
+
+int iq_default_codebook(int32_t head_dim, iq_codebook* out_host) {
+  if (!out_host) return IQ_ERR_NULL;
+  if (head_dim != 128 && head_dim != 256) return IQ_ERR_SHAPE;
+  double lv[8];
+  lloyd_max_sphere(head_dim, lv);
+  for (int i = 0; i < 4; i++) {  // enforce exact symmetry, then round to binary16
+    const double a = 0.5 * (lv[7 - i] - lv[i]);
+    const float r = __half2float(__float2half_rn((float)a));
+    out_host->levels[7 - i] = r;
+    out_host->levels[i] = -r;
+  }
+  for (int i = 0; i < 7; i++)
+    out_host->thresholds[i] = (float)(0.5 * ((double)out_host->levels[i] + (double)out_host->levels[i + 1]));
+  return IQ_OK;
+}
+
+int iq_make_rotation(int32_t head_dim, int32_t n_kv_heads, uint64_t seed, const float* quats_host, float* rot_dev,
+                     void* stream) {
+  const size_t nfl = iq_rotation_floats(head_dim, n_kv_heads);
+  if (nfl == 0) return IQ_ERR_SHAPE;
+  if (!rot_dev) return IQ_ERR_NULL;
+  if (!aligned16(rot_dev)) return IQ_ERR_ALIGN;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int n_quats = (int)(nfl / 4);
+  cudaError_t e;
+  if (quats_host) {
+    e = cudaMemcpyAsync(rot_dev, quats_host, nfl * sizeof(float), cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return IQ_ERR_CUDA;
+    e = iq::launch_normalize_rotation(rot_dev, n_quats, st);
+  } else {
+    e = iq::launch_make_rotation(rot_dev, n_quats, seed, st);
+  }
+  return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
+int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook, const void* k_new,
+                       const void* v_new, int64_t stride_b, int64_t stride_t, int64_t stride_h,
+                       const int32_t* append_pos_dev, const int32_t* n_new_dev, int32_t n_new_max,
+                       const iq_cache* cache, uint32_t* status_dev, void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (!rot_dev || !append_pos_dev) return IQ_ERR_NULL;
+  if ((rc = check_codebook(codebook, false))) return rc;
+  if ((rc = check_cache(cache))) return rc;
+  if (n_new_max < 0) return IQ_ERR_SHAPE;
+  if (n_new_max == 0 || shape->batch == 0) return IQ_OK;
+  if (!k_new || !v_new) return IQ_ERR_NULL;
+  if (!aligned16(k_new) || !aligned16(v_new) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
+  if (stride_b < 0 || stride_t < 0 || stride_h < 0) return IQ_ERR_SHAPE;
+  if ((stride_b & 7) || (stride_t & 7) || (stride_h & 7)) return IQ_ERR_ALIGN;
+
+  iq::QuantizeParams p;
+  p.k_new = static_cast<const __half*>(k_new);
+  p.v_new = static_cast<const __half*>(v_new);
+  p.stride_b = stride_b;
+  p.stride_t = stride_t;
+  p.stride_h = stride_h;
+  p.append_pos = append_pos_dev;
+  p.n_new = n_new_dev;
+  p.n_new_max = n_new_max;
+  p.rot = rot_dev;
+  std::memcpy(p.thresholds, codebook->thresholds, sizeof(p.thresholds));
+  p.k_codes = cache->k_codes;
+  p.k_scales = cache->k_scales;
+  p.v_codes = cache->v_codes;
+  p.v_scales = cache->v_scales;
+  p.status = status_dev;
+  p.n_kv_heads = shape->n_kv_heads;
+  p.t_cap = shape->t_cap;
+  const cudaError_t e = iq::launch_quantize_append(p, shape->head_dim, shape->batch, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
+int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook, const void* q,
+                        const iq_cache* cache, const int32_t* seq_lens_dev, int32_t num_splits, float* part_acc,
+                        float* part_ml, int32_t* part_argmax, uint32_t* status_dev, void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (!rot_dev || !q || !seq_lens_dev || !part_acc || !part_ml) return IQ_ERR_NULL;
+  if ((rc = check_codebook(codebook, true))) return rc;
+  if ((rc = check_cache(cache))) return rc;
+  if (num_splits < 1 || num_splits > 65535) return IQ_ERR_SHAPE;
+  if (!aligned16(q) || !aligned16(part_acc) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
+  if (shape->batch == 0) return IQ_OK;
+
+  iq::DecodeParams p;
+  p.k_codes = cache->k_codes;
+  p.k_scales = cache->k_scales;
+  p.v_codes = cache->v_codes;
+  p.v_scales = cache->v_scales;
+  p.q = static_cast<const __half*>(q);
+  p.rot = rot_dev;
+  p.seq_lens = seq_lens_dev;
+  p.part_acc = part_acc;
+  p.part_ml = part_ml;
+  p.part_argmax = part_argmax;
+  p.status = status_dev;
+  p.batch = shape->batch;
+  p.n_q_heads = shape->n_q_heads;
+  p.n_kv_heads = shape->n_kv_heads;
+  p.group = shape->n_q_heads / shape->n_kv_heads;
+  p.head_groups = (p.group + iq::DEC_HEADS - 1) / iq::DEC_HEADS;
+  p.t_cap = shape->t_cap;
+  p.splits = num_splits;
+  p.sm_scale = shape->sm_scale > 0.f ? shape->sm_scale : 1.0f / std::sqrt((float)shape->head_dim);
+  p.lut_lo[0] = p.lut_lo[1] = p.lut_hi[0] = p.lut_hi[1] = 0u;
+  for (int i = 0; i < 8; i++) {
+    const __half hv = __float2half_rn(codebook->levels[i]);
+    uint16_t bits;
+    std::memcpy(&bits, &hv, 2);
+    p.lut_lo[i >> 2] |= (uint32_t)(bits & 0xFFu) << (8 * (i & 3));
+    p.lut_hi[i >> 2] |= (uint32_t)(bits >> 8) << (8 * (i & 3));
+  }
+  const cudaError_t e = iq::launch_decode_attention(p, shape->head_dim, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
+int iq_combine_splits(const iq_shape* shape, const float* rot_dev, int32_t num_splits, const float* part_acc,
+                      const float* part_ml, const int32_t* part_argmax, void* out, int32_t out_is_fp16, float* lse_out,
+                      int32_t* argmax_out, void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (!rot_dev || !part_acc || !part_ml || !out) return IQ_ERR_NULL;
+  if (argmax_out && !part_argmax) return IQ_ERR_NULL;
+  if (num_splits < 1) return IQ_ERR_SHAPE;
+  if (!aligned16(part_acc) || !aligned16(out) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
+  if (shape->batch == 0) return IQ_OK;
+
+  iq::CombineParams p;
+  p.part_acc = part_acc;
+  p.part_ml = part_ml;
+  p.part_argmax = part_argmax;
+  p.rot = rot_dev;
+  p.out = out;
+  p.lse = lse_out;
+  p.argmax = argmax_out;
+  p.batch = shape->batch;
+  p.n_q_heads = shape->n_q_heads;
+  p.n_kv_heads = shape->n_kv_heads;
+  p.splits = num_splits;
+  p.out_is_fp16 = out_is_fp16;
+  const cudaError_t e = iq::launch_combine_splits(p, shape->head_dim, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
+int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len) {
+  if (check_shape(shape) != IQ_OK || max_seq_len <= 0) return 1;
+  static int n_sm_cached[64] = {};
+  int dev = 0, n_sm = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
+    if (n_sm_cached[dev] == 0) {
+      int v = 0;
+      if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n_sm_cached[dev] = v;
+    }
+    if (n_sm_cached[dev] > 0) n_sm = n_sm_cached[dev];
+  }
+  const int group = shape->n_q_heads / shape->n_kv_heads;
+  const long long items = (long long)(shape->batch > 0 ? shape->batch : 1) * shape->n_kv_heads * ((group + iq::DEC_HEADS - 1) / iq::DEC_HEADS);
+  const long long slots = (long long)n_sm * iq::decode_ctas_per_sm(shape->head_dim);
+  long long s = (3 * slots + items - 1) / items;           // about three CTAs per resident slot
+  const long long cap = (max_seq_len + 511) / 512;         // at least 512 rows (two tiles per warp) per split
+  if (s > cap) s = cap;
+  if (s < 1) s = 1;
+  if (s > 256) s = 256;
+  return (int32_t)s;
+}
+
+}  // extern "C"

@@ -1,0 +1,137 @@
+// Merge of the context-split partials and the single inverse rotation o = R^T o~ (Table 2, kernel D;
+// Appendix A), plus the small kernels that prepare the rotation parameters (Appendix B).
+#include "iq_common.cuh"
+#include "iq_kernels.h"
+
+namespace iq {
+
+constexpr int CMB_WARPS = 4;
+
+// One warp per (sequence, query head). Lane l owns rotated coordinates l*E .. l*E+E-1, i.e. whole SO(4)
+// blocks, so M_b^T is applied in registers and H_d by the warp butterfly.
+template <int D>
+__global__ void __launch_bounds__(CMB_WARPS * 32) combine_kernel(const CombineParams p) {
+  constexpr int E = D / 32;
+  const int lane = threadIdx.x & 31;
+  const int bh = blockIdx.x * CMB_WARPS + (threadIdx.x >> 5);
+  if (bh >= p.batch * p.n_q_heads) return;
+  const int h = bh % p.n_q_heads;
+  const int kvh = h / (p.n_q_heads / p.n_kv_heads);
+  const int S = p.splits;
+  const float* ml = p.part_ml + (size_t)bh * S * 2;
+
+  float m = -INFINITY;
+  int best = -1;
+  for (int s = 0; s < S; s++) {
+    const float ms = ml[2 * s], ls = ml[2 * s + 1];
+    if (!(ls > 0.f)) continue;
+    const int idx = p.part_argmax ? p.part_argmax[(size_t)bh * S + s] : -1;
+    if (ms > m) { m = ms; best = idx; }
+    else if (ms == m && idx >= 0 && (best < 0 || idx < best)) best = idx;
+  }
+  float l = 0.f;
+  float v[E];
+#pragma unroll
+  for (int e = 0; e < E; e++) v[e] = 0.f;
+  for (int s = 0; s < S; s++) {
+    const float ms = ml[2 * s], ls = ml[2 * s + 1];
+    if (!(ls > 0.f)) continue;
+    const float w = __expf(ms - m);
+    l += ls * w;
+    const float* a = p.part_acc + ((size_t)bh * S + s) * D + lane * E;
+#pragma unroll
+    for (int e4 = 0; e4 < E; e4 += 4) {
+      const float4 f = *reinterpret_cast<const float4*>(a + e4);
+      v[e4] += w * f.x; v[e4 + 1] += w * f.y; v[e4 + 2] += w * f.z; v[e4 + 3] += w * f.w;
+    }
+  }
+  const bool empty = !(l > 0.f);
+  const float inv = empty ? 0.f : 1.f / l;
+#pragma unroll
+  for (int e = 0; e < E; e++) v[e] *= inv;
+
+  // o = H_d * blockdiag(M_b^T) * o~   (H_d symmetric, R^T = H_d^T R_SO4^T)
+  float M[E / 4][4][4];
+  const float* qb = p.rot + ((size_t)kvh * (D / 4) + (size_t)lane * (E / 4)) * 8;
+#pragma unroll
+  for (int j = 0; j < E / 4; j++) so4_matrix<float>(qb + 8 * j, M[j]);
+  so4_apply<float, E, true>(M, v);
+  wht_warp<float, E>(v, lane);
+  const float inv_root_d = rsqrtf((float)D);
+#pragma unroll
+  for (int e = 0; e < E; e++) v[e] *= inv_root_d;
+
+  if (p.out_is_fp16) {
+    __half* o = reinterpret_cast<__half*>(p.out) + (size_t)bh * D + lane * E;
+#pragma unroll
+    for (int e = 0; e < E; e += 2) *reinterpret_cast<__half2*>(o + e) = __floats2half2_rn(v[e], v[e + 1]);
+  } else {
+    float* o = reinterpret_cast<float*>(p.out) + (size_t)bh * D + lane * E;
+#pragma unroll
+    for (int e4 = 0; e4 < E; e4 += 4) *reinterpret_cast<float4*>(o + e4) = make_float4(v[e4], v[e4 + 1], v[e4 + 2], v[e4 + 3]);
+  }
+  if (lane == 0) {
+    if (p.lse) p.lse[bh] = empty ? -INFINITY : m + __logf(l);
+    if (p.argmax) p.argmax[bh] = empty ? -1 : best;
+  }
+}
+
+cudaError_t launch_combine_splits(const CombineParams& p, int head_dim, cudaStream_t stream) {
+  const int n = p.batch * p.n_q_heads;
+  if (n <= 0) return cudaSuccess;
+  dim3 grid((n + CMB_WARPS - 1) / CMB_WARPS), block(CMB_WARPS * 32);
+  if (head_dim == 128)
+    combine_kernel<128><<<grid, block, 0, stream>>>(p);
+  else
+    combine_kernel<256><<<grid, block, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Rotation parameters: unit quaternion pairs (Appendix B). Counter-based generator: splitmix64 of
+// (seed, quaternion index, component) -> two uniforms -> Box-Muller normal.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+
+__global__ void make_rotation_kernel(float* rot, int n_quats, uint64_t seed) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_quats) return;
+  float q[4];
+  float nn = 0.f;
+#pragma unroll
+  for (int c = 0; c < 4; c++) {
+    const uint64_t r = splitmix64(splitmix64(seed) ^ ((uint64_t)i * 4 + c));
+    const float u1 = ((float)(uint32_t)(r >> 40) + 0.5f) * (1.0f / 16777216.0f);
+    const float u2 = ((float)(uint32_t)((r >> 8) & 0xFFFFFFu) + 0.5f) * (1.0f / 16777216.0f);
+    q[c] = sqrtf(-2.f * logf(u1)) * cospif(2.f * u2);
+    nn += q[c] * q[c];
+  }
+  const float inv = rsqrtf(nn);
+#pragma unroll
+  for (int c = 0; c < 4; c++) rot[(size_t)i * 4 + c] = q[c] * inv;
+}
+
+__global__ void normalize_rotation_kernel(float* rot, int n_quats) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_quats) return;
+  float4 q = *reinterpret_cast<float4*>(rot + (size_t)i * 4);
+  const float inv = rsqrtf(q.x * q.x + q.y * q.y + q.z * q.z + q.w * q.w);
+  q.x *= inv; q.y *= inv; q.z *= inv; q.w *= inv;
+  *reinterpret_cast<float4*>(rot + (size_t)i * 4) = q;
+}
+
+cudaError_t launch_make_rotation(float* rot, int n_quats, uint64_t seed, cudaStream_t stream) {
+  make_rotation_kernel<<<(n_quats + 127) / 128, 128, 0, stream>>>(rot, n_quats, seed);
+  return cudaGetLastError();
+}
+cudaError_t launch_normalize_rotation(float* rot, int n_quats, cudaStream_t stream) {
+  normalize_rotation_kernel<<<(n_quats + 127) / 128, 128, 0, stream>>>(rot, n_quats);
+  return cudaGetLastError();
+}
+
+}  // namespace iq

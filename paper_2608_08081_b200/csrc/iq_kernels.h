@@ -1,0 +1,71 @@
+// Internal interface between the C ABI (iq_api.cu) and the kernel translation units.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace iq {
+
+// ---- quantize-append
+constexpr int QA_WARPS = 4;
+constexpr int QA_ROWS_PER_WARP = 8;
+
+struct QuantizeParams {
+  const __half* k_new;
+  const __half* v_new;
+  long long stride_b, stride_t, stride_h;
+  const int32_t* append_pos;
+  const int32_t* n_new;
+  int n_new_max;
+  const float* rot;
+  float thresholds[7];
+  uint8_t* k_codes;
+  float* k_scales;
+  uint8_t* v_codes;
+  float* v_scales;
+  uint32_t* status;
+  int n_kv_heads, t_cap;
+};
+cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int batch, cudaStream_t stream);
+
+// ---- fused decode
+constexpr int DEC_BLOCK_TOKENS = 64;  // rows per pipeline stage of one warp
+constexpr int DEC_HEADS = 8;          // query heads per CTA (the N extent of the m16n8k16 tile)
+
+struct DecodeParams {
+  const uint8_t* k_codes;
+  const float* k_scales;
+  const uint8_t* v_codes;
+  const float* v_scales;
+  const __half* q;
+  const float* rot;
+  const int32_t* seq_lens;
+  float* part_acc;
+  float* part_ml;
+  int32_t* part_argmax;
+  uint32_t* status;
+  int batch, n_q_heads, n_kv_heads, group, head_groups, t_cap, splits;
+  float sm_scale;
+  uint32_t lut_lo[2], lut_hi[2];  // low / high bytes of the 8 fp16 levels, 4 per register
+};
+cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream);
+int decode_ctas_per_sm(int head_dim);
+
+// ---- combine + inverse rotation
+struct CombineParams {
+  const float* part_acc;
+  const float* part_ml;
+  const int32_t* part_argmax;
+  const float* rot;
+  void* out;
+  float* lse;
+  int32_t* argmax;
+  int batch, n_q_heads, n_kv_heads, splits, out_is_fp16;
+};
+cudaError_t launch_combine_splits(const CombineParams& p, int head_dim, cudaStream_t stream);
+
+// ---- rotation parameters
+cudaError_t launch_make_rotation(float* rot, int n_quats, uint64_t seed, cudaStream_t stream);
+cudaError_t launch_normalize_rotation(float* rot, int n_quats, cudaStream_t stream);
+
+}  // namespace iq

@@ -1,0 +1,184 @@
+// Quantize-append kernel: Algorithm 1 (normalise, WHT, SO(4) blocks, 3-bit Lloyd-Max, bit-pack) for new
+// K and V rows, one warp per row, appended to the packed cache.
+#include "iq_common.cuh"
+#include "iq_kernels.h"
+
+namespace iq {
+
+// Distance (in unit-variance units) from a decision threshold below which the fp32 decision is not
+// trusted and the row is re-decided in fp64. The fp32 butterfly + block product carry at most a few
+// 1e-6 of absolute error in these units for head_dim <= 256.
+constexpr float GUARD_BAND = 3.0517578125e-05f;  // 2^-15
+
+template <typename T>
+__device__ __forceinline__ int decide_code(T u, const float (&th)[7], bool& near_boundary, T guard) {
+  // Binary search over the 7 ascending thresholds; code = #{ j : u > t_j }. The three pivots visited
+  // include both bounds of the final cell, so checking them covers every decision that could flip.
+  const bool b2 = u > (T)th[3];
+  const T p1 = b2 ? (T)th[5] : (T)th[1];
+  const bool b1 = u > p1;
+  const T p0 = b2 ? (b1 ? (T)th[6] : (T)th[4]) : (b1 ? (T)th[2] : (T)th[0]);
+  const bool b0 = u > p0;
+  T dmin = fabs(u - (T)th[3]);
+  dmin = fmin(dmin, fabs(u - p1));
+  dmin = fmin(dmin, fabs(u - p0));
+  near_boundary = dmin <= guard;
+  return (b2 ? 4 : 0) + (b1 ? 2 : 0) + (b0 ? 1 : 0);
+}
+
+template <int D>
+__global__ void __launch_bounds__(QA_WARPS * 32) quantize_append_kernel(const QuantizeParams p) {
+  constexpr int E = D / 32;        // coordinates per lane
+  constexpr int NB = E / 4;        // SO(4) blocks per lane
+  constexpr int LPU = 32 / E;      // lanes per 32-coordinate packing unit
+  constexpr int WPR = 3 * D / 32;  // 32-bit words per packed row
+
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int b = blockIdx.z;
+  const int h = blockIdx.y >> 1;
+  const int is_v = blockIdx.y & 1;
+
+  int n_new = p.n_new ? p.n_new[b] : p.n_new_max;
+  n_new = min(n_new, p.n_new_max);
+  const int row_begin = (blockIdx.x * QA_WARPS + warp) * QA_ROWS_PER_WARP;
+  if (row_begin >= n_new) return;
+  const int row_end = min(n_new, row_begin + QA_ROWS_PER_WARP);
+  const int pos0 = p.append_pos[b];
+
+  // SO(4) blocks of this lane (fp32), and the raw quaternions for the fp64 re-decision.
+  const float* qbase = p.rot + ((size_t)h * (D / 4) + (size_t)lane * NB) * 8;
+  float q8[NB][8];
+  float M[NB][4][4];
+#pragma unroll
+  for (int j = 0; j < NB; j++) {
+#pragma unroll
+    for (int i = 0; i < 8; i++) q8[j][i] = qbase[j * 8 + i];
+    so4_matrix<float>(q8[j], M[j]);
+  }
+  float th[7];
+#pragma unroll
+  for (int i = 0; i < 7; i++) th[i] = p.thresholds[i];
+
+  const __half* src_base = (is_v ? p.v_new : p.k_new) + (size_t)b * p.stride_b + (size_t)h * p.stride_h + lane * E;
+  uint8_t* codes_out = is_v ? p.v_codes : p.k_codes;
+  float* scales_out = is_v ? p.v_scales : p.k_scales;
+  const size_t slab = ((size_t)b * p.n_kv_heads + h) * (size_t)p.t_cap;
+
+  for (int i = row_begin; i < row_end; i++) {
+    const long long t = (long long)pos0 + i;
+    if (t < 0 || t >= p.t_cap) {
+      if (lane == 0 && p.status) {
+        atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
+        atomicAdd(&p.status[2], 1u);
+      }
+      continue;
+    }
+    // ---- load E contiguous fp16 values (8 or 16 bytes per lane, 256/512 bytes per warp)
+    const __half* src = src_base + (size_t)i * p.stride_t;
+    float x[E];
+    if (E == 4) {
+      const uint2 raw = *reinterpret_cast<const uint2*>(src);
+      const __half2 h0 = *reinterpret_cast<const __half2*>(&raw.x), h1 = *reinterpret_cast<const __half2*>(&raw.y);
+      x[0] = __low2float(h0); x[1] = __high2float(h0); x[2] = __low2float(h1); x[3] = __high2float(h1);
+    } else {
+      const uint4 raw = *reinterpret_cast<const uint4*>(src);
+      const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+      for (int k = 0; k < 4; k++) {
+        const __half2 hh = *reinterpret_cast<const __half2*>(&r[k]);
+        x[2 * k] = __low2float(hh);
+        x[2 * k + 1] = __high2float(hh);
+      }
+    }
+    // ---- Step 1: s = ||x||_2. Squares of fp16 values are exact in fp64; the sum is accumulated in fp64
+    // so that the stored fp32 scale is the correctly rounded norm.
+    double ss = 0.0;
+#pragma unroll
+    for (int e = 0; e < E; e++) ss += (double)x[e] * (double)x[e];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(FULL, ss, o);
+    const double s64 = sqrt(ss);
+    const float s = (float)s64;
+    const float inv_s = (s64 > 0.0) ? (float)(1.0 / s64) : 0.f;
+
+    // ---- Step 2: u = sqrt(d) * R x^ = M_b (H_unnormalised x) / s  (the two sqrt(d) factors cancel)
+    float v[E];
+#pragma unroll
+    for (int e = 0; e < E; e++) v[e] = x[e];
+    wht_warp<float, E>(v, lane);
+    so4_apply<float, E, false>(M, v);
+
+    // ---- Step 3: codes, with a guard band around the thresholds
+    int code[E];
+    bool any_near = false;
+#pragma unroll
+    for (int e = 0; e < E; e++) {
+      bool nb;
+      code[e] = decide_code<float>(v[e] * inv_s, th, nb, GUARD_BAND);
+      any_near |= nb;
+    }
+    if (__any_sync(FULL, any_near)) {
+      // Re-decide the whole row in fp64: the +-1 sums of fp16 values are exact in fp64.
+      double vd[E];
+      double Md[NB][4][4];
+#pragma unroll
+      for (int e = 0; e < E; e++) vd[e] = (double)x[e];
+#pragma unroll
+      for (int j = 0; j < NB; j++) so4_matrix<double>(q8[j], Md[j]);
+      wht_warp<double, E>(vd, lane);
+      so4_apply<double, E, false>(Md, vd);
+#pragma unroll
+      for (int e = 0; e < E; e++) {
+        bool nb;
+        const double u = (s64 > 0.0) ? vd[e] / s64 : 0.0;
+        code[e] = decide_code<double>(u, th, nb, 0.0);
+      }
+      if (lane == 0 && p.status) atomicAdd(&p.status[1], 1u);
+    }
+
+    // ---- Step 4: bit-pack. A packing unit is 32 coordinates = LPU lanes = 3 words.
+    uint32_t w[3] = {0u, 0u, 0u};
+    const int c0 = (lane % LPU) * E;  // unit-local coordinate of this lane's first element
+#pragma unroll
+    for (int e = 0; e < E; e++) {
+      const int c = c0 + e;
+      const uint32_t cd = (uint32_t)code[e];
+      if (c < 24) {
+        const uint32_t val = cd << (4 * (c & 7));
+        if ((c >> 3) == 0) w[0] |= val;
+        else if ((c >> 3) == 1) w[1] |= val;
+        else w[2] |= val;
+      } else {
+        const int sh = 4 * (c - 24) + 3;
+        w[0] |= (cd & 1u) << sh;
+        w[1] |= ((cd >> 1) & 1u) << sh;
+        w[2] |= ((cd >> 2) & 1u) << sh;
+      }
+    }
+#pragma unroll
+    for (int o = 1; o < LPU; o <<= 1) {
+      w[0] |= __shfl_xor_sync(FULL, w[0], o);
+      w[1] |= __shfl_xor_sync(FULL, w[1], o);
+      w[2] |= __shfl_xor_sync(FULL, w[2], o);
+    }
+    const int k = lane % LPU;
+    uint32_t* row_words = reinterpret_cast<uint32_t*>(codes_out + (slab + (size_t)t) * (size_t)(WPR * 4));
+    if (k < 3) row_words[3 * (lane / LPU) + k] = (k == 0) ? w[0] : (k == 1 ? w[1] : w[2]);
+    if (lane == 0) scales_out[slab + (size_t)t] = s;
+  }
+}
+
+cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int batch, cudaStream_t stream) {
+  if (p.n_new_max <= 0 || batch <= 0) return cudaSuccess;
+  const int rows_per_cta = QA_WARPS * QA_ROWS_PER_WARP;
+  dim3 grid((p.n_new_max + rows_per_cta - 1) / rows_per_cta, p.n_kv_heads * 2, batch);
+  dim3 block(QA_WARPS * 32);
+  if (head_dim == 128)
+    quantize_append_kernel<128><<<grid, block, 0, stream>>>(p);
+  else
+    quantize_append_kernel<256><<<grid, block, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace iq

@@ -1,0 +1,134 @@
+"""Shared helpers for the parity tests: run the CUDA path through the C-ABI binding, run the oracle on
+the same seeded inputs, compare."""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+import oracle
+
+OUT_ATOL = 2e-3   # |o - o_ref| <= OUT_ATOL + OUT_RTOL * |o_ref| element-wise
+OUT_RTOL = 1e-3
+TIE_FRACTION_MAX = 1e-5
+
+
+def codebook_for(iq, codebooks, d):
+    lv, th = codebooks[d]
+    return iq.Codebook(tuple(float(x) for x in lv), tuple(float(x) for x in th))
+
+
+def gpu_quantize(iq, torch, w, cb, t_cap=None, append_pos=None, n_new=None, cache=None, status=None):
+    """Quantize-append workload rows on the GPU; returns (shape, rot_dev, cache, status tensor)."""
+    dev = "cuda"
+    t_cap = t_cap or w.t_cap
+    shape = iq.Shape(w.B, w.H_q, w.H_kv, w.d, t_cap)
+    rot = torch.empty(iq.iq_rotation_floats(w.d, w.H_kv), dtype=torch.float32, device=dev)
+    iq.iq_make_rotation(w.d, w.H_kv, 0, np.ascontiguousarray(w.quats), rot)
+    cache = cache or iq.new_cache(shape)
+    status = status if status is not None else torch.zeros(4, dtype=torch.int32, device=dev)
+    k = torch.from_numpy(w.k).to(dev)
+    v = torch.from_numpy(w.v).to(dev)
+    pos = torch.from_numpy(np.asarray(append_pos if append_pos is not None else np.zeros(w.B), np.int32)).to(dev)
+    nn = None if n_new is None else torch.from_numpy(np.asarray(n_new, np.int32)).to(dev)
+    iq.iq_quantize_append(shape, rot, cb, k, v, pos, nn, k.shape[1], cache, status)
+    torch.cuda.synchronize()
+    return shape, rot, cache, status
+
+
+def cache_to_numpy(cache):
+    return dict(k_codes=cache.k_codes.cpu().numpy(), k_scales=cache.k_scales.cpu().numpy(),
+                v_codes=cache.v_codes.cpu().numpy(), v_scales=cache.v_scales.cpu().numpy())
+
+
+def oracle_quantize(w, th, t_cap=None, append_pos=None, n_new=None):
+    cache = oracle.new_cache(w.B, w.H_kv, w.d, t_cap or w.t_cap)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.asarray(append_pos if append_pos is not None else np.zeros(w.B), np.int32),
+                           n_new, cache)
+    return cache
+
+
+def ulp_diff_f32(a, b):
+    ai = a.view(np.int32).astype(np.int64)
+    bi = b.view(np.int32).astype(np.int64)
+    return np.abs(ai - bi)
+
+
+def compare_caches(w, th, gpu, ref, lens):
+    """Codes bit-exact except excused ties; scales equal to within 1 ulp on a vanishing fraction. Returns stats."""
+    d, P = w.d, oracle.row_bytes(w.d)
+    total_codes = 0
+    excused = 0
+    unexcused = 0
+    scale_off = 0
+    rows = 0
+    Rs = {}
+    for which, src in (("k", w.k), ("v", w.v)):
+        gc, rc = gpu[which + "_codes"], ref[which + "_codes"]
+        gs, rs = gpu[which + "_scales"], ref[which + "_scales"]
+        for b in range(w.B):
+            n = int(lens[b])
+            if n == 0:
+                continue
+            total_codes += n * w.H_kv * d
+            rows += n * w.H_kv
+            ud = ulp_diff_f32(np.ascontiguousarray(gs[b, :, :n]), np.ascontiguousarray(rs[b, :, :n]))
+            assert ud.max() <= 1, f"{which} scale differs by {ud.max()} ulp"
+            scale_off += int((ud > 0).sum())
+            neq = np.any(gc[b, :, :n] != rc[b, :, :n], axis=-1)
+            for g, t in zip(*np.nonzero(neq)):
+                cg = oracle.unpack_row(d, gc[b, g, t]).astype(np.int64)
+                cr = oracle.unpack_row(d, rc[b, g, t]).astype(np.int64)
+                if g not in Rs:
+                    Rs[g] = oracle.rotation_matrix(d, w.quats[g])
+                _, _, u = oracle.quantize_row(d, Rs[g], th, src[b, t, g])
+                for i in np.nonzero(cg != cr)[0]:
+                    tj = float(th[min(cg[i], cr[i])])          # threshold separating the two adjacent codes
+                    ok = abs(int(cg[i]) - int(cr[i])) == 1 and abs(u[i] - tj) <= 2.0 ** -23 * max(1.0, abs(tj))
+                    excused += int(ok)
+                    unexcused += int(not ok)
+    assert unexcused == 0, f"{unexcused} code mismatches that are not ties"
+    assert excused <= TIE_FRACTION_MAX * max(total_codes, 1) + 0.999, f"{excused} tie mismatches in {total_codes} codes"
+    assert scale_off <= 1e-5 * rows + 1, f"{scale_off} scales off by 1 ulp in {rows} rows"
+    return dict(total_codes=total_codes, excused=excused, scale_off=scale_off)
+
+
+def gpu_decode(iq, torch, shape, rot, cb, q_np, cache, lens, num_splits, want_argmax=True):
+    dev = "cuda"
+    ws = iq.DecodeWorkspace(shape, num_splits, want_argmax=want_argmax)
+    q = torch.from_numpy(q_np).to(dev)
+    sl = torch.from_numpy(np.asarray(lens, np.int32)).to(dev)
+    iq.decode_step(shape, rot, cb, q, cache, sl, ws)
+    torch.cuda.synchronize()
+    assert int(ws.status[0].item()) == 0, "device status flags set"
+    return dict(out=ws.out.cpu().numpy().astype(np.float64), lse=ws.lse.cpu().numpy().astype(np.float64),
+                argmax=None if ws.argmax is None else ws.argmax.cpu().numpy(), ws=ws)
+
+
+def check_decode(w, lv, q_np, gpu_res, cache_np, lens, sm_scale=0.0, argmax_tol=2e-3):
+    """Outputs within tolerance of the fp64 oracle run on the same packed cache; argmax identical wherever the
+    oracle's maximum is separated from the runner-up by more than argmax_tol, valid (a near-maximal row) otherwise."""
+    ref = oracle.decode_attention(w.quats, lv, q_np, cache_np, lens, w.H_kv, sm_scale)
+    err = np.abs(gpu_res["out"] - ref["out"])
+    bound = OUT_ATOL + OUT_RTOL * np.abs(ref["out"])
+    assert np.all(err <= bound), f"max err {err.max():.3e} (worst excess {np.max(err - bound):.3e})"
+    nz = np.asarray(lens) > 0
+    if nz.any():
+        num = np.linalg.norm((gpu_res["out"] - ref["out"])[nz], axis=-1)
+        den = np.linalg.norm(ref["out"][nz], axis=-1)
+        assert np.all(num <= OUT_RTOL * den + 1e-6), f"relative l2 error {np.max(num / np.maximum(den, 1e-30)):.3e}"
+        assert np.allclose(gpu_res["lse"][nz], ref["lse"][nz], atol=2e-3, rtol=0)
+    assert np.all(np.isneginf(gpu_res["lse"][~nz])) and np.all(gpu_res["out"][~nz] == 0)
+    exact = 0
+    if gpu_res["argmax"] is not None:
+        B, H_q = ref["argmax"].shape
+        for b in range(B):
+            for h in range(H_q):
+                ga, ra = int(gpu_res["argmax"][b, h]), int(ref["argmax"][b, h])
+                if ga == ra:
+                    exact += 1
+                    continue
+                assert lens[b] > 0 and 0 <= ga < lens[b], f"argmax {ga} outside the sequence"
+                z = oracle.scores(w.quats, lv, q_np, cache_np, b, h, int(lens[b]), w.H_kv, sm_scale)
+                assert z[ra] - z[ga] <= argmax_tol, f"argmax differs: gpu row {ga} scores {z[ga]}, oracle row {ra} scores {z[ra]}"
+    return dict(max_err=float(err.max()), argmax_exact=exact, ref=ref)

@@ -1,0 +1,109 @@
+"""C-ABI boundary on the CPU: the library loads, exports every declared symbol, validates arguments
+before any launch, and its host-side codebook matches the oracle-side tool. No kernel is launched."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def iq():
+    import paper_2608_08081_b200 as m
+    return m
+
+
+def test_library_exports_every_declared_symbol(iq):
+    header = open(os.path.join(ROOT, "include", "isoquant.h")).read()
+    names = set(re.findall(r"\b(iq_[a-z_0-9]+)\s*\(", header))
+    assert {"iq_make_rotation", "iq_quantize_append", "iq_decode_attention", "iq_combine_splits"} <= names
+    lib = ctypes.CDLL(iq.lib_path())
+    for n in sorted(names):
+        assert hasattr(lib, n), f"{n} declared in isoquant.h but not exported"
+    assert iq.iq_version() == 100
+    for n in sorted(names):
+        assert hasattr(iq, n) or n in ("iq_shape", "iq_codebook", "iq_cache"), f"binding lacks {n}"
+
+
+def test_sizes(iq):
+    assert iq.iq_row_bytes(128) == 48 and iq.iq_row_bytes(256) == 96 and iq.iq_row_bytes(64) == 0
+    assert iq.iq_rotation_floats(128, 1) == 256 and iq.iq_rotation_floats(256, 8) == 8 * 512
+
+
+def test_default_codebook_matches_oracle_tool(iq, codebooks):
+    for d in (128, 256):
+        cb = iq.iq_default_codebook(d)
+        lv, th = codebooks[d]
+        assert np.array_equal(np.array(cb.levels, np.float32), lv)      # two independent Lloyd-Max implementations
+        assert np.allclose(np.array(cb.thresholds, np.float32), th, atol=0)
+    with pytest.raises(iq.IQError):
+        iq.iq_default_codebook(96)
+
+
+class _P:
+    """Fake tensor: just a device-pointer-like integer (never dereferenced: validation fails first)."""
+    def __init__(self, p): self._p = p
+    def data_ptr(self): return self._p
+
+
+def _call(iq, fn, *a):
+    try:
+        fn(*a)
+    except iq.IQError as e:
+        return e.code
+    return 0
+
+
+def test_argument_validation_happens_before_any_launch(iq, monkeypatch):
+    import paper_2608_08081_b200.binding as B
+    monkeypatch.setattr(B, "_stream", lambda s=None: None)
+    lib = B._lib
+    cb = iq.iq_default_codebook(128).c()
+    good = B._IqShape(1, 4, 1, 128, 1024, 3, 0.0)
+    cache = B._IqCache(0x1000, 0x2000, 0x3000, 0x4000)
+    A = 0x10000  # aligned fake pointer
+    def qa(shape, rot=A, cbk=cb, k=A, v=A, sb=1024 * 128, st=128, sh=128, pos=A, nn=None, n=1, c=cache):
+        return lib.iq_quantize_append(ctypes.byref(shape), rot, ctypes.byref(cbk), k, v, sb, st, sh, pos, nn, n, ctypes.byref(c), None, None)
+    assert qa(B._IqShape(1, 4, 1, 64, 1024, 3, 0.0)) == -2          # head_dim
+    assert qa(B._IqShape(1, 4, 1, 128, 1024, 4, 0.0)) == -2         # bits
+    assert qa(B._IqShape(1, 5, 2, 128, 1024, 3, 0.0)) == -2         # n_q % n_kv
+    assert qa(B._IqShape(1, 4, 1, 128, 1022, 3, 0.0)) == -2         # t_cap % 4
+    assert qa(good, rot=None) == -1
+    assert qa(good, k=None) == -1
+    assert qa(good, k=A + 2) == -3
+    assert qa(good, st=130) == -3
+    assert qa(good, n=-1) == -2
+    assert qa(good, c=B._IqCache(0x1000, 0x2004, 0x3000, 0x4000)) == -3
+    assert qa(good, c=B._IqCache(0x1000, 0, 0x3000, 0x4000)) == -1
+    assert qa(good, n=0) == 0                                        # no-op, nothing launched
+    bad = iq.iq_default_codebook(128).c(); bad.levels[3] = -0.2443    # ascending but not fp16-representable: fine for quantize...
+    assert qa(good, cbk=bad, n=0) == 0
+    bad2 = iq.iq_default_codebook(128).c(); bad2.thresholds[2] = 5.0  # ...but thresholds must ascend
+    assert qa(good, cbk=bad2) == -4
+
+    def da(shape, cbk=cb, q=A, S=2, pa=A, pm=A, lens=A):
+        return lib.iq_decode_attention(ctypes.byref(shape), A, ctypes.byref(cbk), q, ctypes.byref(cache), lens, S, pa, pm, None, None, None)
+    assert da(good, cbk=bad) == -4                                   # decode needs fp16-exact levels
+    assert da(good, S=0) == -2
+    assert da(good, q=None) == -1
+    assert da(good, pa=A + 4) == -3
+    assert da(B._IqShape(0, 4, 1, 128, 1024, 3, 0.0)) == 0           # empty batch: nothing launched
+
+    def cs(shape, S=2, out=A, pg=None, ao=None):
+        return lib.iq_combine_splits(ctypes.byref(shape), A, S, A, A, pg, out, 0, None, ao, None)
+    assert cs(good, S=0) == -2
+    assert cs(good, out=None) == -1
+    assert cs(good, ao=A) == -1                                      # argmax_out without part_argmax
+    assert "binary16" in iq.iq_strerror(-4)
+    assert lib.iq_make_rotation(96, 1, 0, None, A, None) == -2
+    assert lib.iq_make_rotation(128, 1, 0, None, None, None) == -1
+
+
+def test_suggest_splits_is_sane(iq):
+    s = iq.iq_suggest_splits(iq.Shape(1, 32, 8, 128, 32768), 32768)
+    assert 1 <= s <= 64
+    assert iq.iq_suggest_splits(iq.Shape(1, 4, 1, 128, 1024), 100) == 1
+    assert iq.iq_suggest_splits(iq.Shape(32, 64, 8, 128, 32768), 32768) >= 1

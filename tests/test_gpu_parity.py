@@ -1,0 +1,234 @@
+"""GPU-vs-oracle parity through the C ABI: packed codes bit-exact (ties excused and counted), attention
+outputs within 2e-3 + 1e-3 |ref| of the fp64 oracle run on the same packed cache, argmax identical."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+from helpers import (cache_to_numpy, check_decode, codebook_for, compare_caches, gpu_decode, gpu_quantize,
+                     oracle_quantize)
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch as t
+    if not t.cuda.is_available():
+        pytest.skip("no CUDA device")
+    return t
+
+
+@pytest.fixture(scope="module")
+def iq(torch):
+    import paper_2608_08081_b200 as m
+    return m
+
+
+def _roundtrip(iq, torch, codebooks, w, splits_list, n_new=None, t_cap=None):
+    lv, th = codebooks[w.d]
+    cb = codebook_for(iq, codebooks, w.d)
+    lens = w.seq_lens if n_new is None else np.asarray(n_new, np.int32)
+    shape, rot, cache, status = gpu_quantize(iq, torch, w, cb, t_cap=t_cap, n_new=n_new if n_new is not None else w.seq_lens)
+    st = status.cpu().numpy()
+    assert st[0] == 0 and st[2] == 0
+    g = cache_to_numpy(cache)
+    ref = oracle_quantize(w, th, t_cap=t_cap, n_new=lens)
+    stats = compare_caches(w, th, g, ref, lens)
+    stats["rechecked_rows"] = int(st[1])
+    for S in splits_list:
+        res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, lens, S)
+        stats[f"S{S}"] = check_decode(w, lv, w.q, res, g, lens)["max_err"]
+    return stats
+
+
+def test_config1_tiny_decode(iq, torch, codebooks):
+    w = workloads.config1()
+    stats = _roundtrip(iq, torch, codebooks, w, [1, 2, 3, 16])
+    assert stats["total_codes"] == 2 * 1024 * 128
+    print(stats)
+
+
+@pytest.mark.parametrize("d", [128, 256])
+@pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 63, 64, 65, 127, 128, 129, 1000])
+def test_shape_sweep_context_lengths(iq, torch, codebooks, d, T):
+    w = workloads.tiny(100 + T, 1, 8 if d == 128 else 4, 2, d, ((T + 3) // 4) * 4, lens=[T])
+    _roundtrip(iq, torch, codebooks, w, [1, 3], n_new=[T])
+
+
+@pytest.mark.parametrize("G", [1, 2, 4, 8, 16])
+def test_shape_sweep_group_sizes(iq, torch, codebooks, G):
+    w = workloads.tiny(200 + G, 2, 2 * G, 2, 128, 300, lens=[300, 123])
+    _roundtrip(iq, torch, codebooks, w, [1, 4], n_new=[300, 123])
+
+
+def test_ragged_batch_with_empty_and_full_sequences(iq, torch, codebooks):
+    lens = [0, 1, 64, 257, 512, 100, 0, 511]
+    w = workloads.tiny(300, 8, 8, 2, 128, 512, lens=lens)
+    _roundtrip(iq, torch, codebooks, w, [1, 2, 5, 9], n_new=lens)
+
+
+def test_large_scale_rows_and_zero_rows(iq, torch, codebooks):
+    w = workloads.tiny(301, 1, 4, 1, 128, 256, scale=300.0)
+    w.k[0, 5] = 0
+    w.v[0, 7] = 0
+    w.k[0, 9] = np.float16(60000.0)
+    w.v[0, 11, 0, :3] = np.float16(-65504.0)
+    _roundtrip(iq, torch, codebooks, w, [1, 2])
+
+
+def test_append_positions_strides_and_out_of_range_rows(iq, torch, codebooks):
+    """Append in two calls at non-zero positions, from a strided source; rows beyond t_cap are skipped and flagged."""
+    d, T = 128, 96
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    w = workloads.tiny(302, 2, 4, 2, d, T)
+    shape = iq.Shape(2, 4, 2, d, 80)
+    rot = torch.empty(iq.iq_rotation_floats(d, 2), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, 2, 0, np.ascontiguousarray(w.quats), rot)
+    cache = iq.new_cache(shape)
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    big_k = torch.zeros((2, T, 2, 2 * d), dtype=torch.float16, device="cuda")      # strided view: every other 128-slab
+    big_v = torch.zeros_like(big_k)
+    big_k[..., :d] = torch.from_numpy(w.k).cuda()
+    big_v[..., :d] = torch.from_numpy(w.v).cuda()
+    kview, vview = big_k[..., :d], big_v[..., :d]
+    pos0 = torch.zeros(2, dtype=torch.int32, device="cuda")
+    n0 = torch.tensor([40, 17], dtype=torch.int32, device="cuda")
+    iq.iq_quantize_append(shape, rot, cb, kview[:, :40], vview[:, :40], pos0, n0, 40, cache, status)
+    pos1 = n0.clone()
+    n1 = torch.tensor([56, 30], dtype=torch.int32, device="cuda")                  # sequence 0: rows 80..95 fall outside t_cap = 80
+    k2 = torch.stack([kview[0, 40:96], kview[1, 17:73]])
+    v2 = torch.stack([vview[0, 40:96], vview[1, 17:73]])
+    iq.iq_quantize_append(shape, rot, cb, k2, v2, pos1, n1, 56, cache, status)
+    torch.cuda.synchronize()
+    st = status.cpu().numpy()
+    assert st[0] & 1 and st[2] == 16 * 2 * 2                                        # 16 rows x 2 KV heads x (K, V)
+    g = cache_to_numpy(cache)
+    lens = np.array([80, 47], np.int32)
+    ref = oracle.new_cache(2, 2, d, 80)
+    wk = np.zeros((2, 80, 2, d), np.float16); wv = np.zeros_like(wk)
+    wk[0], wv[0] = w.k[0, :80], w.v[0, :80]
+    wk[1, :47], wv[1, :47] = w.k[1, :47], w.v[1, :47]
+    oracle.quantize_append(w.quats, th, wk, wv, np.zeros(2, np.int32), lens, ref)
+    w2 = workloads.Workload("x", 2, 4, 2, d, 80, wk, wv, w.q, w.quats, lens)
+    compare_caches(w2, th, g, ref, lens)
+    res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, lens, 2)
+    check_decode(w2, lv, w.q, res, g, lens)
+
+
+def test_combine_splits_in_isolation(iq, torch, codebooks):
+    d, B, H_q, H_kv, S = 128, 3, 8, 2, 5
+    g = np.random.default_rng(7)
+    pa = g.standard_normal((B, H_q, S, d)).astype(np.float32)
+    pm = np.stack([g.standard_normal((B, H_q, S)) * 3, g.uniform(0.5, 40, (B, H_q, S))], -1).astype(np.float32)
+    pg = g.integers(0, 10000, (B, H_q, S)).astype(np.int32)
+    pm[0, 0, 2] = (-np.inf, 0); pg[0, 0, 2] = -1                                     # an empty split
+    pm[1, 3, :] = (-np.inf, 0); pg[1, 3, :] = -1; pa[1, 3] = 0                        # an empty sequence
+    pm[2, 1, 0, 0] = pm[2, 1, 4, 0] = 50.0; pg[2, 1, 0], pg[2, 1, 4] = 77, 12        # tie on the maximum: lowest row wins
+    quats = workloads.quaternion_pairs(g, H_kv, d)
+    ref = oracle.combine_splits(quats, pa, pm, pg, H_kv)
+    shape = iq.Shape(B, H_q, H_kv, d, 16)
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(quats), rot)
+    out = torch.empty((B, H_q, d), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, H_q), dtype=torch.float32, device="cuda")
+    am = torch.empty((B, H_q), dtype=torch.int32, device="cuda")
+    tt = lambda a: torch.from_numpy(a).cuda()
+    iq.iq_combine_splits(shape, rot, S, tt(pa), tt(pm), tt(pg), out, lse, am)
+    assert np.allclose(out.cpu().numpy(), ref["out"], atol=2e-5, rtol=1e-5)
+    assert np.allclose(lse.cpu().numpy(), ref["lse"], atol=1e-4)
+    assert np.array_equal(am.cpu().numpy(), ref["argmax"]) and am[2, 1].item() == 12 and am[1, 3].item() == -1
+    out16 = torch.empty((B, H_q, d), dtype=torch.float16, device="cuda")
+    iq.iq_combine_splits(shape, rot, S, tt(pa), tt(pm), None, out16)
+    assert np.allclose(out16.float().cpu().numpy(), ref["out"], atol=2e-3, rtol=2e-3)
+
+
+def test_make_rotation_from_seed(iq, torch):
+    d, H = 128, 4
+    a = torch.empty(iq.iq_rotation_floats(d, H), dtype=torch.float32, device="cuda")
+    b = torch.empty_like(a); c = torch.empty_like(a)
+    iq.iq_make_rotation(d, H, 1234, None, a)
+    iq.iq_make_rotation(d, H, 1234, None, b)
+    iq.iq_make_rotation(d, H, 1235, None, c)
+    q = a.cpu().numpy().reshape(-1, 4)
+    assert np.allclose(np.linalg.norm(q, axis=1), 1, atol=1e-6)
+    assert torch.equal(a, b) and not torch.equal(a, c)
+    assert abs(q.mean()) < 0.05 and abs(np.mean(q ** 2) - 0.25) < 0.02                # isotropic on S^3
+
+
+def test_config2_prefill_then_64_decode_steps(iq, torch, codebooks):
+    w = workloads.config2()
+    lv, th = codebooks[w.d]
+    cb = codebook_for(iq, codebooks, w.d)
+    T, steps = 8192, w.extra["steps"]
+    shape, rot, cache, status = gpu_quantize(iq, torch, w, cb, t_cap=w.t_cap)
+    ref = oracle_quantize(w, th, t_cap=w.t_cap)
+    S = iq.iq_suggest_splits(shape, T)
+    ws = iq.DecodeWorkspace(shape, S, want_argmax=True)
+    lens = torch.tensor([T], dtype=torch.int32, device="cuda")
+    worst = 0.0
+    for i in range(steps):
+        k1 = torch.from_numpy(w.extra["step_k"][i]).cuda()
+        v1 = torch.from_numpy(w.extra["step_v"][i]).cuda()
+        q1 = torch.from_numpy(w.extra["step_q"][i]).cuda()
+        iq.iq_quantize_append(shape, rot, cb, k1, v1, lens, None, 1, cache, status)
+        lens += 1
+        iq.decode_step(shape, rot, cb, q1, cache, lens, ws)
+        torch.cuda.synchronize()
+        oracle.quantize_append(w.quats, th, w.extra["step_k"][i], w.extra["step_v"][i], np.array([T + i], np.int32), None, ref)
+        if i % 9 == 0 or i == steps - 1:                                              # every 9th step checked in full
+            g = cache_to_numpy(cache)
+            res = dict(out=ws.out.cpu().numpy().astype(np.float64), lse=ws.lse.cpu().numpy().astype(np.float64),
+                       argmax=ws.argmax.cpu().numpy())
+            worst = max(worst, check_decode(w, lv, w.extra["step_q"][i], res, g, np.array([T + i + 1], np.int32))["max_err"])
+    g = cache_to_numpy(cache)
+    full = workloads.Workload("c2", 1, w.H_q, w.H_kv, w.d, w.t_cap,
+                              np.concatenate([w.k] + [w.extra["step_k"][i] for i in range(steps)], axis=1),
+                              np.concatenate([w.v] + [w.extra["step_v"][i] for i in range(steps)], axis=1), w.q, w.quats,
+                              np.array([T + steps], np.int32))
+    print(compare_caches(full, th, g, ref, full.seq_lens), "worst decode err", worst)
+    assert status.cpu().numpy()[0] == 0
+
+
+def test_config3_wide_heads(iq, torch, codebooks):
+    w = workloads.config3()
+    S = None
+    stats = _roundtrip(iq, torch, codebooks, w, [1, 19])
+    print(stats)
+
+
+def test_config4_long_context_retrieval(iq, torch, codebooks):
+    w = workloads.config4()
+    lv, th = codebooks[w.d]
+    cb = codebook_for(iq, codebooks, w.d)
+    shape, rot, cache, status = gpu_quantize(iq, torch, w, cb)
+    g = cache_to_numpy(cache)
+    ref = oracle_quantize(w, th)
+    print(compare_caches(w, th, g, ref, w.seq_lens))
+    S = iq.iq_suggest_splits(shape, w.t_cap)
+    res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, w.seq_lens, S)
+    chk = check_decode(w, lv, w.q, res, g, w.seq_lens)
+    assert np.array_equal(res["argmax"][0], w.extra["needle_pos"])                    # identical to the planted positions
+    assert np.array_equal(res["argmax"], chk["ref"]["argmax"])                        # and to the oracle's
+    for h in range(w.H_q):
+        o = res["out"][0, h]
+        assert int(np.argmax(np.abs(o))) == int(w.extra["needle_chan"][h])            # dominant V channel = planted channel
+        vn = w.v[0, w.extra["needle_pos"][h], h // w.G].astype(np.float64)
+        assert (o @ vn) / (np.linalg.norm(o) * np.linalg.norm(vn)) > 0.9
+
+
+@pytest.mark.parametrize("B,ctx", [(1, 4096), (8, 4096), (1, 32768)])
+def test_config5_small_points_in_full(iq, torch, codebooks, B, ctx):
+    w = workloads.config5(B, ctx)
+    lv, th = codebooks[w.d]
+    cb = codebook_for(iq, codebooks, w.d)
+    shape, rot, cache, status = gpu_quantize(iq, torch, w, cb, n_new=w.seq_lens)
+    g = cache_to_numpy(cache)
+    ref = oracle_quantize(w, th, n_new=w.seq_lens)
+    print(compare_caches(w, th, g, ref, w.seq_lens))
+    S = iq.iq_suggest_splits(shape, ctx)
+    res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, w.seq_lens, S)
+    print(check_decode(w, lv, w.q, res, g, w.seq_lens)["max_err"])
