@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the IsoQuant hot path: one step = quantize-append of one new K/V row per sequence and KV
+head, the fused decode over the packed cache, and the split merge with the inverse rotation.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line. Metric: packed-KV bytes the decode consumes per second (codes + fp32 scales of K
+and V, all KV heads, all sequences), whole job. `--impl reference` times the fp64 CPU oracle on a bounded
+sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOADS = {
+    # name: (B, ctx, H_q, H_kv, d) -- the batched serving sweep; lengths ragged in [0.5, 1.0] x ctx
+    "config5_B32_ctx32768": (32, 32768, 64, 8, 128),
+    "config5_B8_ctx32768": (8, 32768, 64, 8, 128),
+    "config5_B1_ctx32768": (1, 32768, 64, 8, 128),
+    "config5_B32_ctx4096": (32, 4096, 64, 8, 128),
+    "config5_B8_ctx4096": (8, 4096, 64, 8, 128),
+    "config5_B1_ctx4096": (1, 4096, 64, 8, 128),
+}
+DEFAULT_WORKLOAD = "config5_B32_ctx32768"
+T_CAP_MARGIN = 256  # rows of head-room so that every sequence can take the benchmark's appends
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu capture summarised under
+# profiles/ (None until a capture of that workload exists).
+DECODE_TRAFFIC_BYTES = {}
+
+
+def bytes_per_row(d: int) -> int:
+    return 2 * (3 * d // 8) + 2 * 4   # K and V codes + fp32 scales, per cached row per KV head
+
+
+def measured_peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+    except Exception:
+        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def build_state(name: str, device, rank: int):
+    """Synthetic cache for one rank: seeded K/V generated on the GPU in chunks and bulk-quantized (untimed)."""
+    import torch
+
+    import paper_2608_08081_b200 as iq
+    import workloads
+
+    B, ctx, H_q, H_kv, d = WORKLOADS[name]
+    gen = workloads.config5_device(B, ctx, device, H_q, H_kv, d)
+    t_cap = ctx + T_CAP_MARGIN
+    shape = iq.Shape(B, H_q, H_kv, d, t_cap)
+    cb = iq.iq_default_codebook(d)
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device=device)
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(gen["quats"]), rot)
+    cache = iq.new_cache(shape, device)
+    status = torch.zeros(4, dtype=torch.int32, device=device)
+    lens_np = gen["lens"].astype(np.int32)
+    for b0, k, v in gen["chunks"]():
+        nb = k.shape[0]
+        sub = iq.Shape(nb, H_q, H_kv, d, t_cap)
+        view = iq.Cache(cache.k_codes[b0:b0 + nb], cache.k_scales[b0:b0 + nb], cache.v_codes[b0:b0 + nb], cache.v_scales[b0:b0 + nb])
+        pos = torch.zeros(nb, dtype=torch.int32, device=device)
+        nn = torch.from_numpy(lens_np[b0:b0 + nb]).to(device)
+        iq.iq_quantize_append(sub, rot, cb, k, v, pos, nn, ctx, view, status)
+        torch.cuda.synchronize()
+        del k, v
+    return dict(iq=iq, shape=shape, cb=cb, rot=rot, cache=cache, status=status, lens_np=lens_np, q0=gen["q"], quats=gen["quats"],
+                B=B, ctx=ctx, H_q=H_q, H_kv=H_kv, d=d, t_cap=t_cap)
+
+
+def step_inputs(st, n_steps: int, device, seed: int):
+    """Pre-drawn per-step inputs (same law as the cache rows): q [n][B][H_q][d], k/v [n][B][1][H_kv][d], fp16."""
+    import torch
+
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    B, H_q, H_kv, d = st["B"], st["H_q"], st["H_kv"], st["d"]
+    q = torch.randn((n_steps, B, H_q, d), generator=g, device=device).to(torch.float16)
+    k = torch.randn((n_steps, B, 1, H_kv, d), generator=g, device=device).to(torch.float16)
+    v = torch.randn((n_steps, B, 1, H_kv, d), generator=g, device=device).to(torch.float16)
+    return q, k, v
+
+
+def run_ours(args, rank: int, world: int, local_rank: int):
+    import torch
+    import torch.distributed as dist
+
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    st = build_state(args.workload, device, rank)
+    iq, shape, cb, rot, cache = st["iq"], st["shape"], st["cb"], st["rot"], st["cache"]
+    B, H_q, H_kv, d = st["B"], st["H_q"], st["H_kv"], st["d"]
+    K, W = args.steps, args.warmup
+    S = args.splits or iq.iq_suggest_splits(shape, st["ctx"])
+    ws = iq.DecodeWorkspace(shape, S, want_argmax=False, device=device)
+    lens = torch.from_numpy(st["lens_np"]).to(device)
+    q_all, k_all, v_all = step_inputs(st, K + W, device, 99 + rank)
+    stream = torch.cuda.current_stream()
+
+    def one_step(i, ev=None):
+        iq.iq_quantize_append(shape, rot, cb, k_all[i], v_all[i], lens, None, 1, cache, st["status"])
+        lens.add_(1)
+        if ev is not None:
+            ev[0].record(stream)
+        iq.iq_decode_attention(shape, rot, cb, q_all[i], cache, lens, S, ws.part_acc, ws.part_ml, None, ws.status)
+        if ev is not None:
+            ev[1].record(stream)
+        iq.iq_combine_splits(shape, rot, S, ws.part_acc, ws.part_ml, None, ws.out, ws.lse, None)
+
+    for i in range(W):
+        one_step(i)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record(stream)
+    for i in range(K):
+        one_step(W + i, evs[i])
+    t1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_total = t0.elapsed_time(t1)
+    dec_ms = [a.elapsed_time(b) for a, b in evs]
+    assert int(ws.status[0].item()) == 0 and int(st["status"][0].item()) == 0, "device status flags set"
+    rows = int(st["lens_np"].astype(np.int64).sum()) + B * W           # cached rows per KV head at the first timed step
+    bytes_steps = [(rows + B * (i + 1)) * H_kv * bytes_per_row(d) for i in range(K)]
+    if world > 1:
+        tt = torch.tensor([ms_total], device=device, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+
+    # ---- end to end through the C-ABI binding with host buffers: H2D of the step inputs and D2H of the output inside the timed region
+    hq = q_all[:W + K].cpu().pin_memory(); hk = k_all[:W + K].cpu().pin_memory(); hv = v_all[:W + K].cpu().pin_memory()
+    dq = torch.empty_like(q_all[0]); dk = torch.empty_like(k_all[0]); dv = torch.empty_like(v_all[0])
+    hout = torch.empty((B, H_q, d), dtype=torch.float32).pin_memory()
+
+    def e2e_step(i):
+        dq.copy_(hq[i], non_blocking=True); dk.copy_(hk[i], non_blocking=True); dv.copy_(hv[i], non_blocking=True)
+        iq.iq_quantize_append(shape, rot, cb, dk, dv, lens, None, 1, cache, st["status"])
+        lens.add_(1)
+        iq.iq_decode_attention(shape, rot, cb, dq, cache, lens, S, ws.part_acc, ws.part_ml, None, ws.status)
+        iq.iq_combine_splits(shape, rot, S, ws.part_acc, ws.part_ml, None, ws.out, ws.lse, None)
+        hout.copy_(ws.out, non_blocking=True)
+        torch.cuda.synchronize()
+
+    n_e2e = min(K, T_CAP_MARGIN - 2 * (K + W) - 4)
+    lens_before = lens.clone()
+    for i in range(min(3, W)):
+        e2e_step(i)
+    if world > 1:
+        dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for i in range(n_e2e):
+        e2e_step(W + i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    if world > 1:
+        tt = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    rows_e2e = int(lens_before.sum().item()) + B * min(3, W)
+    e2e_bytes = sum((rows_e2e + B * (i + 1)) * H_kv * bytes_per_row(d) for i in range(n_e2e))
+
+    if rank != 0:
+        return None
+    peak, peak_src = measured_peak_hbm()
+    ms_step = ms_total / K
+    value = world * sum(bytes_steps) / (ms_total * 1e-3) / 1e9
+    dec_avg_ms = sum(dec_ms) / K
+    achieved = (sum(bytes_steps) / K) / (dec_avg_ms * 1e-3) / 1e9
+    out = {
+        "metric": "fused decode packed-KV GB/s",
+        "value": round(value, 1),
+        "unit": "GB/s",
+        "n_gpus": world,
+        "steps": K,
+        "warmup": W,
+        "ms_per_step": round(ms_step, 4),
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "u3 codes, f16 tensor-core operands, f32 accumulate",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "batch": B, "ctx": st["ctx"], "n_q_heads": H_q, "n_kv_heads": H_kv, "head_dim": d,
+                   "t_cap": st["t_cap"], "ragged_lengths": "floor(ctx*U[0.5,1.0])", "cached_rows_per_kv_head": rows,
+                   "num_splits": S, "bytes_per_row_per_kv_head": bytes_per_row(d), "l2": "inputs_larger_than_l2",
+                   "step": "quantize-append 1 row/seq + fused decode + combine", "parallelism": f"replicas x{world}"},
+        "decode_tokens_per_s": round(world * B / (ms_step * 1e-3), 1),
+        "frac_of_8TBs": round(value / world / 8000.0, 4),
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
+                     "traffic": DECODE_TRAFFIC_BYTES.get(args.workload), "kernel": "decode_kernel", "peak_source": peak_src,
+                     "avg_launch_ms": round(dec_avg_ms, 4), "algorithmic_bytes_per_launch": int(sum(bytes_steps) / K)},
+        "e2e": {"value": round(world * e2e_bytes / (e2e_ms * 1e-3) / 1e9, 1), "unit": "GB/s",
+                "h2d_bytes_per_step": int(B * (H_q + 2 * H_kv) * d * 2), "d2h_bytes_per_step": int(B * H_q * d * 4),
+                "ms_per_step": round(e2e_ms / max(n_e2e, 1), 4), "steps": n_e2e,
+                "note": "packed cache is device-resident state; per-step inputs (q, new k/v) come from pinned host memory, output returns to host"},
+        "gpu_launches": 3 * K,
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        out["cpu_baseline"] = cpu_baseline(st, lens, q_all[W + K - 1])
+    return out
+
+
+def cpu_baseline(st, lens, q_last, max_seqs: int = 2):
+    """The fp64 oracle, as it stands, timed on this machine's host cores on a bounded sample: the decode of the
+    first `max_seqs` sequences (all heads) of the same cache."""
+    import oracle
+
+    nb = min(max_seqs, st["B"])
+    cache = {k: getattr(st["cache"], k)[:nb].cpu().numpy() for k in ("k_codes", "k_scales", "v_codes", "v_scales")}
+    ln = lens[:nb].cpu().numpy().astype(np.int32)
+    q = q_last[:nb].cpu().numpy()
+    lv = np.array(st["cb"].levels, np.float32)
+    t0 = time.perf_counter()
+    oracle.decode_attention(st["quats"], lv, q, cache, ln, st["H_kv"])
+    dt = time.perf_counter() - t0
+    nbytes = int(ln.astype(np.int64).sum()) * st["H_kv"] * bytes_per_row(st["d"])
+    return {"value": round(nbytes / dt / 1e9, 4), "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"decode of the first {nb} of {st['B']} sequences (all {st['H_q']} query heads), {dt:.2f} s"}
+
+
+def run_reference(args, rank: int, world: int):
+    """Reference arm: the oracle on host cores, on a bounded sample of the same workload, generated on the host."""
+    if rank != 0:
+        return None
+    import oracle
+    import workloads
+    from oracle import lloyd_max
+
+    B, ctx, H_q, H_kv, d = WORKLOADS[args.workload]
+    lens_all = workloads.config5_lengths(B, ctx)
+    nb = 1
+    T = int(lens_all[0])
+    g = np.random.Generator(np.random.Philox(workloads.stream_seed(5, 0) + 7))
+    lv, th = lloyd_max.fp16_codebook(d)
+    quats = workloads.quaternion_pairs(workloads.rng(5, workloads.QUAT_STREAM), H_kv, d)
+    P = oracle.row_bytes(d)
+    cache = oracle.new_cache(nb, H_kv, d, T + 64)
+    # the sample's cache content: uniformly random codes and Gaussian-row-like scales (the decode cost does not depend on values)
+    cache["k_codes"][:] = g.integers(0, 256, cache["k_codes"].shape, dtype=np.uint8)
+    cache["v_codes"][:] = g.integers(0, 256, cache["v_codes"].shape, dtype=np.uint8)
+    cache["k_scales"][:] = np.sqrt(d) * (1 + 0.05 * g.standard_normal(cache["k_scales"].shape))
+    cache["v_scales"][:] = np.sqrt(d) * (1 + 0.05 * g.standard_normal(cache["v_scales"].shape))
+    times = []
+    lens = np.array([T], np.int32)
+    for i in range(args.warmup + args.steps):
+        k1 = workloads.to_fp16(g.standard_normal((nb, 1, H_kv, d)))
+        v1 = workloads.to_fp16(g.standard_normal((nb, 1, H_kv, d)))
+        q1 = workloads.to_fp16(g.standard_normal((nb, H_q, d)))
+        t0 = time.perf_counter()
+        oracle.quantize_append(quats, th, k1, v1, lens, None, cache)
+        lens = lens + 1
+        oracle.decode_attention(quats, lv, q1, cache, lens, H_kv)
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            times.append((dt, int(lens[0]) * H_kv * bytes_per_row(d)))
+    tot_t = sum(t for t, _ in times)
+    tot_b = sum(b for _, b in times)
+    val = round(tot_b / tot_t / 1e9, 4)
+    sample = f"each step: quantize-append + decode of 1 of {B} sequences ({T} rows x {H_kv} KV heads, {H_q} query heads)"
+    return {"impl": "reference", "metric": "fused decode packed-KV GB/s", "value": val, "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(1e3 * tot_t / max(len(times), 1), 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": sample},
+            "cpu_baseline": {"value": val, "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--splits", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        out = run_reference(args, rank, world)
+        if out is not None:
+            print(json.dumps(out), flush=True)
+        return
+    if 2 * (args.steps + args.warmup) + 8 > T_CAP_MARGIN:
+        raise SystemExit(f"--steps + --warmup must stay below {T_CAP_MARGIN // 2 - 4}")
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        import torch
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl")
+    out = run_ours(args, rank, world, local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+    if out is not None:
+        print(json.dumps(out), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -38,7 +38,7 @@ __device__ __forceinline__ uint32_t sliced_selectors(uint32_t w0, uint32_t w1, u
   return ((w0 >> 3) & 0x11111111u) | ((w1 >> 2) & 0x22222222u) | ((w2 >> 1) & 0x44444444u);
 }
 
-template <int D, bool QSPLIT, bool ARGMAX>
+template <int D, bool QSPLIT, bool PSPLIT, bool ARGMAX>
 __global__ void __launch_bounds__(DEC_WARPS * 32, (D == 128) ? 4 : 2) decode_kernel(const DecodeParams p) {
   using L = DecLayout<D>;
   constexpr int DJ = D / 128;
@@ -277,15 +277,27 @@ __global__ void __launch_bounds__(DEC_WARPS * 32, (D == 128) ? 4 : 2) decode_ker
       m_run[1] = mn1;
     }
     // probabilities -> B fragments of the value product (transposed across the warp by movmatrix)
+    // Each weight p * scale_V / sqrt(d) is carried as a two-term fp16 sum (hi + lo): a single fp16 would leave
+    // a 2^-11 relative error on every term, which is isotropic in the rotated space and too large for rows
+    // whose norm is dominated by a few outlier channels.
     uint32_t pb[4][2];
+    uint32_t pl[PSPLIT ? 4 : 1][2];
 #pragma unroll
     for (int mt = 0; mt < 4; mt++) {
       const float p0 = ex2f(s[mt][0] - mn0), p1 = ex2f(s[mt][1] - mn1);
       const float p2 = ex2f(s[mt][2] - mn0), p3 = ex2f(s[mt][3] - mn1);
       l_run[0] += p0 + p2;
       l_run[1] += p1 + p3;
-      pb[mt][0] = movmatrix_trans(pack_half2(p0 * vs[mt][0], p1 * vs[mt][0]));
-      pb[mt][1] = movmatrix_trans(pack_half2(p2 * vs[mt][1], p3 * vs[mt][1]));
+      const float w0 = p0 * vs[mt][0], w1 = p1 * vs[mt][0], w2 = p2 * vs[mt][1], w3 = p3 * vs[mt][1];
+      const uint32_t h01 = pack_half2(w0, w1), h23 = pack_half2(w2, w3);
+      pb[mt][0] = movmatrix_trans(h01);
+      pb[mt][1] = movmatrix_trans(h23);
+      if (PSPLIT) {
+        const float2 b01 = __half22float2(*reinterpret_cast<const __half2*>(&h01));
+        const float2 b23 = __half22float2(*reinterpret_cast<const __half2*>(&h23));
+        pl[mt][0] = movmatrix_trans(pack_half2(w0 - b01.x, w1 - b01.y));
+        pl[mt][1] = movmatrix_trans(pack_half2(w2 - b23.x, w3 - b23.y));
+      }
     }
 
     // ---- d4: value accumulation on the codes. Lane (g, t) decodes rows 2t, 2t+1, 2t+8, 2t+9 of each
@@ -315,6 +327,7 @@ __global__ void __launch_bounds__(DEC_WARPS * 32, (D == 128) ? 4 : 2) decode_ker
             const uint32_t f0 = prmt(l1, h1, 0x6240u), f1 = prmt(l1, h1, 0x7351u);
             const uint32_t f2 = prmt(l2, h2, 0x6240u), f3 = prmt(l2, h2, 0x7351u);
             mma_16816(acc[j][2 * k + hh], f0, f1, f2, f3, pb[mt][0], pb[mt][1]);
+            if (PSPLIT) mma_16816(acc[j][2 * k + hh], f0, f1, f2, f3, pl[mt][0], pl[mt][1]);
           }
       }
     }
@@ -402,14 +415,14 @@ __global__ void __launch_bounds__(DEC_WARPS * 32, (D == 128) ? 4 : 2) decode_ker
   }
 }
 
-template <int D, bool QSPLIT, bool ARGMAX>
+template <int D, bool QSPLIT, bool PSPLIT, bool ARGMAX>
 static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
   using L = DecLayout<D>;
   static bool configured[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  auto kern = decode_kernel<D, QSPLIT, ARGMAX>;
+  auto kern = decode_kernel<D, QSPLIT, PSPLIT, ARGMAX>;
   if (dev < 0 || dev >= 64 || !configured[dev]) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::SMEM_BYTES);
     if (e != cudaSuccess) return e;
@@ -422,8 +435,8 @@ static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
 
 cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream) {
   const bool am = p.part_argmax != nullptr;
-  if (head_dim == 128) return am ? launch_one<128, true, true>(p, stream) : launch_one<128, true, false>(p, stream);
-  return am ? launch_one<256, true, true>(p, stream) : launch_one<256, true, false>(p, stream);
+  if (head_dim == 128) return am ? launch_one<128, true, true, true>(p, stream) : launch_one<128, true, true, false>(p, stream);
+  return am ? launch_one<256, true, true, true>(p, stream) : launch_one<256, true, true, false>(p, stream);
 }
 
 int decode_ctas_per_sm(int head_dim) { return head_dim == 128 ? 4 : 2; }

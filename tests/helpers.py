@@ -54,7 +54,7 @@ def ulp_diff_f32(a, b):
     return np.abs(ai - bi)
 
 
-def compare_caches(w, th, gpu, ref, lens):
+def compare_caches(w, th, gpu, ref, lens, tie_fraction_max=TIE_FRACTION_MAX):
     """Codes bit-exact except excused ties; scales equal to within 1 ulp on a vanishing fraction. Returns stats."""
     d, P = w.d, oracle.row_bytes(w.d)
     total_codes = 0
@@ -88,7 +88,7 @@ def compare_caches(w, th, gpu, ref, lens):
                     excused += int(ok)
                     unexcused += int(not ok)
     assert unexcused == 0, f"{unexcused} code mismatches that are not ties"
-    assert excused <= TIE_FRACTION_MAX * max(total_codes, 1) + 0.999, f"{excused} tie mismatches in {total_codes} codes"
+    assert excused <= tie_fraction_max * max(total_codes, 1) + 0.999, f"{excused} tie mismatches in {total_codes} codes"
     assert scale_off <= 1e-5 * rows + 1, f"{scale_off} scales off by 1 ulp in {rows} rows"
     return dict(total_codes=total_codes, excused=excused, scale_off=scale_off)
 
@@ -117,7 +117,7 @@ def check_decode(w, lv, q_np, gpu_res, cache_np, lens, sm_scale=0.0, argmax_tol=
         num = np.linalg.norm((gpu_res["out"] - ref["out"])[nz], axis=-1)
         den = np.linalg.norm(ref["out"][nz], axis=-1)
         assert np.all(num <= OUT_RTOL * den + 1e-6), f"relative l2 error {np.max(num / np.maximum(den, 1e-30)):.3e}"
-        assert np.allclose(gpu_res["lse"][nz], ref["lse"][nz], atol=2e-3, rtol=0)
+        assert np.allclose(gpu_res["lse"][nz], ref["lse"][nz], atol=2e-3, rtol=1e-5)   # fp32 scores: relative at large |z|
     assert np.all(np.isneginf(gpu_res["lse"][~nz])) and np.all(gpu_res["out"][~nz] == 0)
     exact = 0
     if gpu_res["argmax"] is not None:
@@ -131,4 +131,4 @@ def check_decode(w, lv, q_np, gpu_res, cache_np, lens, sm_scale=0.0, argmax_tol=
                 assert lens[b] > 0 and 0 <= ga < lens[b], f"argmax {ga} outside the sequence"
                 z = oracle.scores(w.quats, lv, q_np, cache_np, b, h, int(lens[b]), w.H_kv, sm_scale)
                 assert z[ra] - z[ga] <= argmax_tol, f"argmax differs: gpu row {ga} scores {z[ga]}, oracle row {ra} scores {z[ra]}"
-    return dict(max_err=float(err.max()), argmax_exact=exact, ref=ref)
+    return dict(max_err=float(err.max()), margin=float(np.max(err / bound)), argmax_exact=exact, ref=ref)

@@ -27,7 +27,7 @@ def iq(torch):
     return m
 
 
-def _roundtrip(iq, torch, codebooks, w, splits_list, n_new=None, t_cap=None):
+def _roundtrip(iq, torch, codebooks, w, splits_list, n_new=None, t_cap=None, tie_fraction_max=1e-5):
     lv, th = codebooks[w.d]
     cb = codebook_for(iq, codebooks, w.d)
     lens = w.seq_lens if n_new is None else np.asarray(n_new, np.int32)
@@ -36,11 +36,12 @@ def _roundtrip(iq, torch, codebooks, w, splits_list, n_new=None, t_cap=None):
     assert st[0] == 0 and st[2] == 0
     g = cache_to_numpy(cache)
     ref = oracle_quantize(w, th, t_cap=t_cap, n_new=lens)
-    stats = compare_caches(w, th, g, ref, lens)
+    stats = compare_caches(w, th, g, ref, lens, tie_fraction_max)
     stats["rechecked_rows"] = int(st[1])
     for S in splits_list:
         res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, lens, S)
-        stats[f"S{S}"] = check_decode(w, lv, w.q, res, g, lens)["max_err"]
+        c = check_decode(w, lv, w.q, res, g, lens)
+        stats[f"S{S}"] = (c["max_err"], c["margin"])
     return stats
 
 
@@ -55,13 +56,13 @@ def test_config1_tiny_decode(iq, torch, codebooks):
 @pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 63, 64, 65, 127, 128, 129, 1000])
 def test_shape_sweep_context_lengths(iq, torch, codebooks, d, T):
     w = workloads.tiny(100 + T, 1, 8 if d == 128 else 4, 2, d, ((T + 3) // 4) * 4, lens=[T])
-    _roundtrip(iq, torch, codebooks, w, [1, 3], n_new=[T])
+    print(_roundtrip(iq, torch, codebooks, w, [1, 3], n_new=[T]))
 
 
 @pytest.mark.parametrize("G", [1, 2, 4, 8, 16])
 def test_shape_sweep_group_sizes(iq, torch, codebooks, G):
     w = workloads.tiny(200 + G, 2, 2 * G, 2, 128, 300, lens=[300, 123])
-    _roundtrip(iq, torch, codebooks, w, [1, 4], n_new=[300, 123])
+    print(_roundtrip(iq, torch, codebooks, w, [1, 4], n_new=[300, 123]))
 
 
 def test_ragged_batch_with_empty_and_full_sequences(iq, torch, codebooks):
@@ -74,9 +75,9 @@ def test_large_scale_rows_and_zero_rows(iq, torch, codebooks):
     w = workloads.tiny(301, 1, 4, 1, 128, 256, scale=300.0)
     w.k[0, 5] = 0
     w.v[0, 7] = 0
-    w.k[0, 9] = np.float16(60000.0)
-    w.v[0, 11, 0, :3] = np.float16(-65504.0)
-    _roundtrip(iq, torch, codebooks, w, [1, 2])
+    w.k[0, 9] = np.float16(60000.0)   # a constant row rotates onto a multiple of e_0: 127 coordinates sit EXACTLY on the
+    w.v[0, 11, 0, :3] = np.float16(-65504.0)  # threshold 0 -- genuine ties, so only "every mismatch is a tie" is asserted here
+    print(_roundtrip(iq, torch, codebooks, w, [1, 2], tie_fraction_max=1e-2))
 
 
 def test_append_positions_strides_and_out_of_range_rows(iq, torch, codebooks):
@@ -231,4 +232,5 @@ def test_config5_small_points_in_full(iq, torch, codebooks, B, ctx):
     print(compare_caches(w, th, g, ref, w.seq_lens))
     S = iq.iq_suggest_splits(shape, ctx)
     res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, w.seq_lens, S)
-    print(check_decode(w, lv, w.q, res, g, w.seq_lens)["max_err"])
+    c = check_decode(w, lv, w.q, res, g, w.seq_lens)
+    print(c["max_err"], c["margin"])
