@@ -35,7 +35,7 @@ WORKLOADS = {
     "config5_B1_ctx4096": (1, 4096, 64, 8, 128),
 }
 DEFAULT_WORKLOAD = "config5_B32_ctx32768"
-T_CAP_MARGIN = 256  # rows of head-room so that every sequence can take the benchmark's appends
+T_CAP_MARGIN = 2048  # rows of head-room so that every sequence can take the benchmark's appends
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu capture summarised under
 # profiles/ (None until a capture of that workload exists).
@@ -56,50 +56,57 @@ def measured_peak_hbm():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks, power and throttle reasons through NVML (read-only) every few ms while the timed region runs."""
 
-    def __init__(self, gpu_index: int):
-        self.gpu = gpu_index
-        self.proc = None
-        self.lines = []
+    def __init__(self, gpu_index: int, period_s: float = 0.004):
+        self.gpu, self.period = gpu_index, period_s
+        self.samples, self.reasons, self.stop_flag, self.thread, self.err = [], set(), False, None, None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
-            self.thread.start()
-        except Exception:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.gpu
+            if vis:
+                try:
+                    idx = int(vis.split(",")[self.gpu])
+                except ValueError:
+                    idx = self.gpu
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.nv = pynvml
+            self.smax = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:  # noqa: BLE001
+            self.err = repr(e)
+            return
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown, "hw_thermal_slowdown": nv.nvmlClocksEventReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksEventReasonSwThermalSlowdown, "sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap}
+        while not self.stop_flag:
+            try:
+                self.samples.append((nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM), nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0))
+                r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception as e:  # noqa: BLE001
+                self.err = repr(e)
+                break
+            time.sleep(self.period)
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=2)
-        except Exception:
-            self.proc.kill()
-        sm, smax, reasons = [], [], set()
-        for ln in self.lines:
-            f = [x.strip() for x in ln.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1])); smax.append(float(f[2]))
-            except ValueError:
-                continue
-            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        self.stop_flag = True
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "error": self.err}
+        sm = [c for c, _ in self.samples]
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": self.smax, "reasons": sorted(self.reasons), "samples": len(sm),
+                "power_w_max": round(max(p for _, p in self.samples), 1)}
 
 
 def build_state(name: str, device, rank: int):
@@ -212,7 +219,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         hout.copy_(ws.out, non_blocking=True)
         torch.cuda.synchronize()
 
-    n_e2e = min(K, T_CAP_MARGIN - 2 * (K + W) - 4)
+    n_e2e = K
+    lens.copy_(torch.from_numpy(st["lens_np"]).to(device))               # rewind: the e2e leg re-appends over the same rows
     lens_before = lens.clone()
     for i in range(min(3, W)):
         e2e_step(i)
@@ -342,8 +350,8 @@ def run_reference(args, rank: int, world: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--splits", type=int, default=0)
@@ -358,8 +366,8 @@ def main():
         if out is not None:
             print(json.dumps(out), flush=True)
         return
-    if 2 * (args.steps + args.warmup) + 8 > T_CAP_MARGIN:
-        raise SystemExit(f"--steps + --warmup must stay below {T_CAP_MARGIN // 2 - 4}")
+    if args.steps + args.warmup + 8 > T_CAP_MARGIN:
+        raise SystemExit(f"--steps + --warmup must stay below {T_CAP_MARGIN - 8}")
     if world > 1:
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")

@@ -15,10 +15,19 @@
 
 namespace iq {
 
-constexpr int DEC_WARPS = 4;
-constexpr int DEC_STAGES = 2;
+#ifndef IQ_DEC_WARPS
+#define IQ_DEC_WARPS 4
+#endif
+#ifndef IQ_DEC_STAGES
+#define IQ_DEC_STAGES 2
+#endif
+#ifndef IQ_DEC_MINB128
+#define IQ_DEC_MINB128 4
+#endif
+constexpr int DEC_WARPS = IQ_DEC_WARPS;
+constexpr int DEC_STAGES = IQ_DEC_STAGES;
 constexpr uint32_t DEC_WAIT_LIMIT = 1u << 22;
-constexpr int DEC_HDR_BYTES = 1024;  // barriers + cross-warp merge scalars
+constexpr int DEC_HDR_BYTES = 512;  // barriers + cross-warp merge scalars
 
 template <int D>
 struct DecLayout {
@@ -30,7 +39,8 @@ struct DecLayout {
   static constexpr int PIPE_BYTES = DEC_WARPS * DEC_STAGES * STAGE_BYTES;
   static constexpr int Q_BYTES = DEC_HEADS * D * 4;
   static constexpr int MERGE_BYTES = DEC_WARPS * DEC_HEADS * D * 4;
-  static constexpr int SMEM_BYTES = DEC_HDR_BYTES + Q_BYTES + (PIPE_BYTES > MERGE_BYTES ? PIPE_BYTES : MERGE_BYTES);
+  // the rotated-query staging and the cross-warp merge buffer alias the pipeline stages (used before / after them)
+  static constexpr int SMEM_BYTES = DEC_HDR_BYTES + (PIPE_BYTES > MERGE_BYTES ? PIPE_BYTES : MERGE_BYTES);
 };
 
 // Selectors of the 8 coordinates whose code bits sit in bit 3 of the nibbles of the unit's three words.
@@ -38,8 +48,10 @@ __device__ __forceinline__ uint32_t sliced_selectors(uint32_t w0, uint32_t w1, u
   return ((w0 >> 3) & 0x11111111u) | ((w1 >> 2) & 0x22222222u) | ((w2 >> 1) & 0x44444444u);
 }
 
+static_assert(DecLayout<128>::Q_BYTES <= DecLayout<128>::PIPE_BYTES && DecLayout<256>::Q_BYTES <= DecLayout<256>::PIPE_BYTES, "q staging must fit");
+
 template <int D, bool QSPLIT, bool PSPLIT, bool ARGMAX>
-__global__ void __launch_bounds__(DEC_WARPS * 32, (D == 128) ? 4 : 2) decode_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(DEC_WARPS * 32, (D == 128) ? IQ_DEC_MINB128 : 2) decode_kernel(const DecodeParams p) {
   using L = DecLayout<D>;
   constexpr int DJ = D / 128;
   constexpr int E = D / 32;
@@ -52,8 +64,8 @@ __global__ void __launch_bounds__(DEC_WARPS * 32, (D == 128) ? 4 : 2) decode_ker
   float* wm = reinterpret_cast<float*>(smem + 128);           // [warps][8] running max (log2 units)
   float* wl = wm + DEC_WARPS * DEC_HEADS;                     // [warps][8] running sum
   int* wi = reinterpret_cast<int*>(wl + DEC_WARPS * DEC_HEADS);  // [warps][8] argmax row
-  float* qs = reinterpret_cast<float*>(smem + DEC_HDR_BYTES);  // [8][D] rotated queries
-  uint8_t* pipe = smem + DEC_HDR_BYTES + L::Q_BYTES;
+  uint8_t* pipe = smem + DEC_HDR_BYTES;
+  float* qs = reinterpret_cast<float*>(pipe);  // [8][D] rotated queries, consumed before the first tile copy is issued
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int g = lane >> 2, t = lane & 3;
@@ -108,10 +120,6 @@ __global__ void __launch_bounds__(DEC_WARPS * 32, (D == 128) ? 4 : 2) decode_ker
 #pragma unroll
     for (int st = 0; st < DEC_STAGES; st++) mbar_init(&mybar[st], 1);
     fence_mbar_init();
-    fence_proxy_async();
-#pragma unroll
-    for (int st = 0; st < DEC_STAGES; st++)
-      if (warp + st * DEC_WARPS < nblk) issue(warp + st * DEC_WARPS, st);
   }
 
   // ---------------------------------------------------------------- d1: q~ = R q for the CTA's heads
@@ -158,6 +166,14 @@ __global__ void __launch_bounds__(DEC_WARPS * 32, (D == 128) ? 4 : 2) decode_ker
         qlo[j][i][1] = pack_half2(f.z - b23.x, f.w - b23.y);
       }
     }
+
+  __syncthreads();  // every warp has read its q~ fragments: the staging area becomes pipeline memory
+  if (lane == 0) {
+    fence_proxy_async();
+#pragma unroll
+    for (int st = 0; st < DEC_STAGES; st++)
+      if (warp + st * DEC_WARPS < nblk) issue(warp + st * DEC_WARPS, st);
+  }
 
   const uint32_t lut_lo0 = p.lut_lo[0], lut_lo1 = p.lut_lo[1], lut_hi0 = p.lut_hi[0], lut_hi1 = p.lut_hi[1];
   const float kfac = p.sm_scale * LOG2E * rsqrtf((float)D);  // scores in log2 units: z2 = S_raw * scale_K * kfac
@@ -439,6 +455,6 @@ cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStr
   return am ? launch_one<256, true, true, true>(p, stream) : launch_one<256, true, true, false>(p, stream);
 }
 
-int decode_ctas_per_sm(int head_dim) { return head_dim == 128 ? 4 : 2; }
+int decode_ctas_per_sm(int head_dim) { return head_dim == 128 ? IQ_DEC_MINB128 : 2; }
 
 }  // namespace iq
