@@ -172,6 +172,32 @@ int iq_combine_splits(const iq_shape* shape, const float* rot_dev, int32_t num_s
                       const float* part_acc, const float* part_ml, const int32_t* part_argmax,
                       void* out, int32_t out_is_fp16, float* lse_out, int32_t* argmax_out, void* stream);
 
+/*
+ * Decode step for callers that cannot allocate device memory (the paper has no counterpart: its pipeline
+ * is unsplit and needs no scratch). It runs iq_decode_attention followed by iq_combine_splits with the
+ * split partials kept in a fixed array inside the library image instead of caller-provided buffers.
+ * Meant for code that must not call cudaMalloc or a framework allocator: work enqueued while a stream
+ * capture is open, plugins that receive only their inputs and outputs, embeddings with a memory budget
+ * fixed at load time.
+ *   - The array is IQ_STATIC_SCRATCH_BYTES (8 MiB) of device memory on every GPU that loads the library,
+ *     held until the process exits. A call needs batch * n_q_heads * num_splits * (head_dim + 2) floats;
+ *     larger requests are rejected with IQ_ERR_LIMIT and nothing is enqueued.
+ *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress, with that
+ *     device current); with lazy module loading that is also the moment the driver places the array on
+ *     the GPU. Make that first call before any stream capture begins.
+ *   - The call itself allocates nothing and frees nothing.
+ *   - All calls on a device share the one array, which keeps the previous call's contents. Every split of
+ *     every head is rewritten on each call, so no clearing is needed; but two calls whose kernels overlap
+ *     on the GPU (different streams) race on it. Serialise them on one stream or with events.
+ * Arguments as for iq_decode_attention / iq_combine_splits; no argmax output.
+ */
+#define IQ_STATIC_SCRATCH_BYTES (8u << 20)
+size_t iq_static_scratch_bytes(void);
+int iq_decode_attention_static(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook,
+                               const void* q, const iq_cache* cache, const int32_t* seq_lens_dev,
+                               int32_t num_splits, void* out, int32_t out_is_fp16, float* lse_out,
+                               uint32_t* status_dev, void* stream);
+
 /* A split count that fills the GPU for this shape when the longest sequence has max_seq_len rows. */
 int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len);
 

@@ -12,6 +12,8 @@ from .binding import (  # noqa: F401
     Shape,
     iq_combine_splits,
     iq_decode_attention,
+    iq_decode_attention_static,
+    iq_static_scratch_bytes,
     iq_default_codebook,
     iq_make_rotation,
     iq_quantize_append,

@@ -58,6 +58,9 @@ def _load():
     lib.iq_decode_attention.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp,
                                         ctypes.POINTER(_IqCache), _vp, _i32, _vp, _vp, _vp, _vp, _vp]
     lib.iq_combine_splits.argtypes = [ctypes.POINTER(_IqShape), _vp, _i32, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
+    lib.iq_static_scratch_bytes.restype = ctypes.c_size_t
+    lib.iq_decode_attention_static.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp,
+                                               ctypes.POINTER(_IqCache), _vp, _i32, _vp, _i32, _vp, _vp, _vp]
     lib.iq_suggest_splits.restype = _i32
     lib.iq_suggest_splits.argtypes = [ctypes.POINTER(_IqShape), _i32]
     return lib
@@ -178,6 +181,20 @@ def iq_combine_splits(shape: Shape, rot_dev, num_splits: int, part_acc, part_ml,
     _check(_lib.iq_combine_splits(ctypes.byref(cs), _ptr(rot_dev), num_splits, _ptr(part_acc), _ptr(part_ml),
                                   _ptr(part_argmax), _ptr(out), 1 if out.dtype == torch.float16 else 0, _ptr(lse_out),
                                   _ptr(argmax_out), _stream(stream)), "iq_combine_splits")
+
+
+def iq_static_scratch_bytes() -> int:
+    return int(_lib.iq_static_scratch_bytes())
+
+
+def iq_decode_attention_static(shape: Shape, rot_dev, codebook: Codebook, q, cache: Cache, seq_lens_dev, num_splits: int,
+                               out, lse_out=None, status_dev=None, stream=None) -> None:
+    """Decode + combine with the split partials in the library's fixed scratch array: for callers that cannot
+    allocate device memory. Allocates nothing; calls that overlap on the GPU race on the shared array."""
+    cs, cb, cc = shape.c(), codebook.c(), cache.c()
+    _check(_lib.iq_decode_attention_static(ctypes.byref(cs), _ptr(rot_dev), ctypes.byref(cb), _ptr(q), ctypes.byref(cc),
+                                           _ptr(seq_lens_dev), num_splits, _ptr(out), 1 if out.dtype == torch.float16 else 0,
+                                           _ptr(lse_out), _ptr(status_dev), _stream(stream)), "iq_decode_attention_static")
 
 
 def iq_suggest_splits(shape: Shape, max_seq_len: int) -> int:
