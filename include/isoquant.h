@@ -39,12 +39,16 @@
  *   not round them (IQ_ERR_CODEBOOK otherwise). A dequantised coordinate is scale * level[code] / sqrt(d).
  *
  * Packed cache (Section 3.2, Step 4 fixes the size only: 3d/8 bytes per row, 48 at d = 128)
- *   codes  [batch][n_kv_heads][t_cap][3d/8] uint8, scales [batch][n_kv_heads][t_cap] fp32 (= ||x||_2),
- *   separately for K and V. A row is a sequence of little-endian 32-bit words; coordinates are taken in
- *   groups of 32, each group owning 3 consecutive words. In group-local numbering, coordinate c < 24
- *   stores its code in bits [4n, 4n+3) of word c/8, n = c mod 8; coordinate c >= 24 (n = c - 24) stores
- *   bit k of its code in bit 4n+3 of word k. t_cap must be a multiple of 4 and all four arrays 16-byte
- *   aligned, so that every tile the decode kernel copies starts on a 16-byte boundary.
+ *   codes: 3d/8 bytes per cached row and side, scales [batch][n_kv_heads][t_cap] fp32 (= ||x||_2), separately
+ *   for K and V. The unit of packing is a group of 32 entries in 3 consecutive little-endian 32-bit words: in
+ *   group-local numbering, entry c < 24 stores its code in bits [4n, 4n+3) of word c/8, n = c mod 8; entry
+ *   c >= 24 (n = c - 24) stores bit k of its code in bit 4n+3 of word k.
+ *   K codes [batch][n_kv_heads][t_cap][3d/8]: one packed row per cached row, entries = rotated coordinates.
+ *   V codes [batch][n_kv_heads][t_cap/128][d][48]: token-transposed. For every block of 128 cached rows and every
+ *   rotated coordinate c there is one 48-byte record holding the 128 codes of coordinate c, entries = row within
+ *   the block. (The decode kernel contracts K over coordinates and V over rows; either way the contraction
+ *   index then runs along a packed record.) Bits of rows that were never appended are left as they are.
+ *   t_cap must be a multiple of 128 and all four arrays 16-byte aligned.
  */
 #ifndef ISOQUANT_H_
 #define ISOQUANT_H_
@@ -78,7 +82,7 @@ typedef struct iq_shape {
   int32_t n_q_heads;
   int32_t n_kv_heads; /* n_q_heads % n_kv_heads == 0 */
   int32_t head_dim;   /* 128 or 256 */
-  int32_t t_cap;      /* rows allocated per (sequence, KV head); multiple of 4 */
+  int32_t t_cap;      /* rows allocated per (sequence, KV head); multiple of 128 */
   int32_t bits;       /* 3 */
   float sm_scale;     /* softmax scale; <= 0 selects 1/sqrt(head_dim) (Appendix A) */
 } iq_shape;
@@ -126,8 +130,10 @@ int iq_make_rotation(int32_t head_dim, int32_t n_kv_heads, uint64_t seed, const 
  *   append_pos_dev device int32 [batch]: cache row that receives new row 0 of sequence b.
  *   n_new_dev      device int32 [batch] rows to append per sequence (clamped to n_new_max), or NULL for
  *                  n_new_max everywhere. n_new_max = 0 is a no-op.
- *   cache          host struct of device pointers; rows append_pos[b] + i are overwritten. The call does
- *                  not touch any sequence-length array: the caller advances its lengths.
+ *   cache          host struct of device pointers; rows append_pos[b] + i are overwritten (on the V side: the
+ *                  bits of those rows inside the transposed records). The call does not touch any
+ *                  sequence-length array: the caller advances its lengths. Calls that append to the same
+ *                  (sequence, KV head) must be ordered on one stream.
  *   status_dev     optional (see top). Rows with append_pos + i outside [0, t_cap) are skipped and flagged.
  * Arithmetic: fp32 butterfly WHT and 4x4 block products; any row with a coordinate closer than 2^-15 to a
  * decision threshold is re-decided in fp64 inside the kernel, so the codes equal those of an fp64
@@ -145,15 +151,15 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
  *   seq_lens_dev   device int32 [batch]: rows 0 .. len-1 of each sequence are attended to (clamped to
  *                  [0, t_cap]); the row appended last is attended to like any other.
  *   num_splits     S >= 1. Sequence b is cut into S consecutive chunks of
- *                  64 * ceil(ceil(len_b / S) / 64) rows; trailing chunks may be empty.
+ *                  128 * ceil(ceil(len_b / S) / 128) rows; trailing chunks may be empty.
  *   part_acc       device fp32 [batch][n_q_heads][S][head_dim]: sum_j exp(z_j - m) v~_j over the chunk,
  *                  in the rotated space, natural coordinate order. 16-byte aligned.
  *   part_ml        device fp32 [batch][n_q_heads][S][2] = (m, l): m = max_j z_j, l = sum_j exp(z_j - m),
  *                  z_j = sm_scale * q~ . k~_j. An empty chunk holds (-inf, 0) and acc = 0.
  *   part_argmax    device int32 [batch][n_q_heads][S] or NULL: row index attaining m (lowest on ties), -1 if empty.
  *   status_dev     optional (see top).
- * Arithmetic: q~ and the probabilities enter fp16 tensor-core operands (q~ as a two-term fp16 sum),
- * codebook levels are exact fp16 values, every accumulation is fp32.
+ * Arithmetic: q~ and the probabilities enter fp16 tensor-core operands, each as a two-term fp16 sum
+ * (hi + lo); codebook levels are exact fp16 values; every accumulation is fp32.
  */
 int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook,
                         const void* q, const iq_cache* cache, const int32_t* seq_lens_dev,

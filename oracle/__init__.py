@@ -118,7 +118,17 @@ def unpack_row(d: int, row) -> np.ndarray:
     return codes
 
 
+def v_row_codes(d: int, v_area, t: int) -> np.ndarray:
+    """Codes of V row t from the token-transposed V bytes of one (sequence, KV head): v_area is the uint8 array
+    [t_cap][3d/8] slice of that head (viewed flat)."""
+    area = np.ascontiguousarray(v_area, dtype=np.uint8).reshape(-1)
+    codes = np.zeros(d, dtype=np.uint8)
+    lib().iqo_v_row_codes(_c_int(d), _p(area), _c_i64(int(t)), _p(codes))
+    return codes
+
+
 def new_cache(B: int, H_kv: int, d: int, t_cap: int):
+    assert t_cap % 128 == 0, "t_cap must be a multiple of 128 (token-transposed V blocks)"
     P = row_bytes(d)
     return dict(
         k_codes=np.zeros((B, H_kv, t_cap, P), dtype=np.uint8),

@@ -30,7 +30,13 @@
  *     sequence of little-endian 32-bit words; coordinates are taken in groups of 32, each group
  *     owning 3 consecutive words. In group-local numbering, coordinate c < 24 puts its 3-bit code in
  *     bits [4n, 4n+3) of word c/8, n = c mod 8; coordinate c >= 24 (n = c - 24) spreads its code
- *     over bit 4n+3 of the three words: bit k of the code goes to word k.
+ *     over bit 4n+3 of the three words: bit k of the code goes to word k. K rows are stored this way, one
+ *     row after the other.
+ *   - V codes are stored token-transposed (the paper says nothing about the arrangement): the rows of one
+ *     (sequence, KV head) are taken in blocks of 128; for block j and coordinate c there is one 48-byte
+ *     record, at byte ((j * d) + c) * 48 of that head's V area, holding the 128 codes of coordinate c for the
+ *     block's rows, arranged exactly like a packed row of 128 entries with the row-in-block as the entry
+ *     index. t_cap is a multiple of 128.
  *
  * Parity pins: every function here is pinned by tests/test_oracle_*.py (invariants, closed forms,
  * library routines, brute force). Not pinned (no published artefact exists): equality of the code
@@ -184,6 +190,46 @@ void iqo_unpack_row(int d, const uint8_t* row, uint8_t* codes) {
   }
 }
 
+/* Token-transposed V area of one (sequence, KV head): code of (row t, coordinate c). A 128-entry record is a
+ * packed row of 128 entries, so entry e lives in 32-entry group e/32 of the record (3 words each). */
+static void v_locate(int d, int64_t t, int c, size_t* rec_byte, int* e) {
+  *rec_byte = ((size_t)(t / 128) * (size_t)d + (size_t)c) * 48;
+  *e = (int)(t % 128);
+}
+static void v_put(int d, uint8_t* area, int64_t t, int c, uint32_t code) {
+  size_t rb; int e;
+  v_locate(d, t, c, &rb, &e);
+  uint8_t* grp = area + rb + 12 * (e / 32);
+  int cc = e % 32;
+  uint32_t w[3];
+  for (int k = 0; k < 3; k++) w[k] = get_word(grp + 4 * k);
+  if (cc < 24) {
+    int sh = 4 * (cc % 8);
+    w[cc / 8] = (w[cc / 8] & ~(7u << sh)) | ((code & 7u) << sh);
+  } else {
+    int sh = 4 * (cc - 24) + 3;
+    for (int k = 0; k < 3; k++) w[k] = (w[k] & ~(1u << sh)) | (((code >> k) & 1u) << sh);
+  }
+  for (int k = 0; k < 3; k++) put_word(grp + 4 * k, w[k]);
+}
+static uint32_t v_get(int d, const uint8_t* area, int64_t t, int c) {
+  size_t rb; int e;
+  v_locate(d, t, c, &rb, &e);
+  const uint8_t* grp = area + rb + 12 * (e / 32);
+  int cc = e % 32;
+  if (cc < 24) return (get_word(grp + 4 * (cc / 8)) >> (4 * (cc % 8))) & 7u;
+  uint32_t code = 0;
+  for (int k = 0; k < 3; k++) code |= ((get_word(grp + 4 * k) >> (4 * (cc - 24) + 3)) & 1u) << k;
+  return code;
+}
+/* Codes of V row t of one (sequence, KV head) area, one byte per coordinate. */
+void iqo_v_row_codes(int d, const uint8_t* area, int64_t t, uint8_t* codes) {
+  for (int c = 0; c < d; c++) codes[c] = (uint8_t)v_get(d, area, t, c);
+}
+void iqo_v_row_store(int d, uint8_t* area, int64_t t, const uint8_t* codes) {
+  for (int c = 0; c < d; c++) v_put(d, area, t, c, codes[c]);
+}
+
 /* Algorithm 1 applied to the new K and V rows of every sequence and KV head, appended to the cache.
  * k_new, v_new: binary16, element (b, i, h, c) at b*stride_b + i*stride_t + h*stride_h + c (element strides).
  * Row i < n_new[b] of sequence b goes to cache row append_pos[b] + i (rows >= t_cap are skipped).
@@ -212,8 +258,16 @@ int64_t iqo_quantize_append(int B, int H_kv, int d, int t_cap, const float* quat
         size_t row = ((size_t)b * H_kv + h) * t_cap + t;
         k_scales[row] = iqo_quantize_row(d, R, thresholds7, k_new + src, codes, NULL);
         iqo_pack_row(d, codes, k_codes + row * P);
-        v_scales[row] = iqo_quantize_row(d, R, thresholds7, v_new + src, codes, NULL);
-        iqo_pack_row(d, codes, v_codes + row * P);
+      }
+      /* V rows share words between neighbouring rows (token-transposed records): written one row at a time */
+      for (int i = 0; i < n; i++) {
+        int64_t t = (int64_t)append_pos[b] + i;
+        if (t < 0 || t >= t_cap) continue;
+        uint8_t codes[512];
+        size_t src = (size_t)(b * stride_b + i * stride_t + h * stride_h);
+        size_t area = ((size_t)b * H_kv + h) * t_cap;
+        v_scales[area + t] = iqo_quantize_row(d, R, thresholds7, v_new + src, codes, NULL);
+        iqo_v_row_store(d, v_codes + area * P, t, codes);
       }
       skipped += sk;
     }
@@ -222,7 +276,15 @@ int64_t iqo_quantize_append(int B, int H_kv, int d, int t_cap, const float* quat
   return skipped;
 }
 
-/* Dequantised rotated vector of one cached row: x~_i = scale * level[code_i] / sqrt(d). */
+/* Dequantised rotated vector of cached V row t of a (sequence, KV head) area. */
+static void dequant_v_row(int d, const uint8_t* area, int64_t t, float scale, const float* levels8, double* out) {
+  uint8_t codes[512];
+  iqo_v_row_codes(d, area, t, codes);
+  double f = (double)scale / sqrt((double)d);
+  for (int i = 0; i < d; i++) out[i] = f * (double)levels8[codes[i]];
+}
+
+/* Dequantised rotated vector of one cached K row: x~_i = scale * level[code_i] / sqrt(d). */
 static void dequant_row(int d, const uint8_t* row, float scale, const float* levels8, double* out) {
   uint8_t codes[512];
   iqo_unpack_row(d, row, codes);
@@ -260,7 +322,7 @@ static void decode_one(int d, const double* R, const float* levels8, double sm_s
   for (int j = 0; j < len; j++) denom += exp(z[j] - zmax);
   for (int j = 0; j < len; j++) {         /* o~ = sum_j alpha_j v~_j */
     double a = exp(z[j] - zmax) / denom;
-    dequant_row(d, v_codes + (size_t)j * P, v_scales[j], levels8, row);
+    dequant_v_row(d, v_codes, j, v_scales[j], levels8, row);
     for (int i = 0; i < d; i++) orot[i] += a * row[i];
   }
   for (int j = 0; j < d; j++) {           /* o = R^T o~ */

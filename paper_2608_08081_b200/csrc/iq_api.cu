@@ -16,7 +16,7 @@ int check_shape(const iq_shape* s) {
   if (s->bits != 3) return IQ_ERR_SHAPE;
   if (s->batch < 0 || s->batch > 65535) return IQ_ERR_SHAPE;
   if (s->n_kv_heads <= 0 || s->n_q_heads <= 0 || s->n_q_heads % s->n_kv_heads != 0) return IQ_ERR_SHAPE;
-  if (s->t_cap <= 0 || (s->t_cap & 3) != 0) return IQ_ERR_SHAPE;
+  if (s->t_cap <= 0 || (s->t_cap & 127) != 0) return IQ_ERR_SHAPE;
   const int hg = (s->n_q_heads / s->n_kv_heads + iq::DEC_HEADS - 1) / iq::DEC_HEADS;
   if ((long long)s->n_kv_heads * hg > 32767) return IQ_ERR_SHAPE;
   return IQ_OK;
@@ -99,7 +99,7 @@ const char* iq_strerror(int code) {
   switch (code) {
     case IQ_OK: return "ok";
     case IQ_ERR_NULL: return "a required pointer is NULL";
-    case IQ_ERR_SHAPE: return "unsupported shape (head_dim 128/256, bits 3, n_q_heads % n_kv_heads == 0, t_cap % 4 == 0, strides % 8 == 0)";
+    case IQ_ERR_SHAPE: return "unsupported shape (head_dim 128/256, bits 3, n_q_heads % n_kv_heads == 0, t_cap % 128 == 0, strides % 8 == 0)";
     case IQ_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
     case IQ_ERR_CODEBOOK: return "codebook not ascending or a level is not representable in binary16";
     case IQ_ERR_CUDA: return "CUDA runtime error at launch";
@@ -275,7 +275,7 @@ int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len) {
   const long long items = (long long)(shape->batch > 0 ? shape->batch : 1) * shape->n_kv_heads * ((group + iq::DEC_HEADS - 1) / iq::DEC_HEADS);
   const long long slots = (long long)n_sm * iq::decode_ctas_per_sm(shape->head_dim);
   long long s = (3 * slots + items - 1) / items;           // about three CTAs per resident slot
-  const long long cap = (max_seq_len + 511) / 512;         // at least 512 rows (two tiles per warp) per split
+  const long long cap = (max_seq_len + 511) / 512;         // at least 512 rows (four blocks) per split
   if (s > cap) s = cap;
   if (s < 1) s = 1;
   if (s > 256) s = 256;

@@ -144,11 +144,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Bounded wait: gives up after `limit` polls and reports false (the caller flags the error and unwinds).
+// IQ_MBAR_SPIN selects non-blocking polls (test_wait) instead of the suspending try_wait.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t limit) {
+#ifdef IQ_MBAR_SPIN
+  for (uint32_t i = 0; i < limit; i++)
+    if (mbar_test_wait(bar, parity)) return true;
   for (uint32_t i = 0; i < limit; i++)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
+#else
+  for (uint32_t i = 0; i < limit; i++)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+#endif
 }
 // 1-D bulk asynchronous copy global -> shared, completion counted in bytes on an mbarrier. Both addresses
 // 16-byte aligned, size a multiple of 16 bytes.

@@ -29,7 +29,7 @@ struct QuantizeParams {
 cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int batch, cudaStream_t stream);
 
 // ---- fused decode
-constexpr int DEC_BLOCK_TOKENS = 64;  // rows per pipeline stage of one warp
+constexpr int DEC_BLOCK_TOKENS = 128;  // cached rows per block of the decode kernel = rows of one transposed V block
 constexpr int DEC_HEADS = 8;          // query heads per CTA (the N extent of the m16n8k16 tile)
 
 struct DecodeParams {

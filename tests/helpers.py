@@ -75,10 +75,24 @@ def compare_caches(w, th, gpu, ref, lens, tie_fraction_max=TIE_FRACTION_MAX):
             ud = ulp_diff_f32(np.ascontiguousarray(gs[b, :, :n]), np.ascontiguousarray(rs[b, :, :n]))
             assert ud.max() <= 1, f"{which} scale differs by {ud.max()} ulp"
             scale_off += int((ud > 0).sum())
-            neq = np.any(gc[b, :, :n] != rc[b, :, :n], axis=-1)
-            for g, t in zip(*np.nonzero(neq)):
-                cg = oracle.unpack_row(d, gc[b, g, t]).astype(np.int64)
-                cr = oracle.unpack_row(d, rc[b, g, t]).astype(np.int64)
+            if which == "k":
+                row_codes = lambda arr, g, t: oracle.unpack_row(d, arr[b, g, t])
+                neq = np.any(gc[b, :, :n] != rc[b, :, :n], axis=-1)
+                bad = list(zip(*np.nonzero(neq)))
+            else:   # token-transposed: compare whole 128-row blocks, then the rows of the blocks that differ
+                row_codes = lambda arr, g, t: oracle.v_row_codes(d, arr[b, g], t)
+                nb = (n + 127) // 128
+                gb = gc[b].reshape(w.H_kv, -1, 128 * P)[:, :nb]
+                rb = rc[b].reshape(w.H_kv, -1, 128 * P)[:, :nb]
+                bad = []
+                for g, j in zip(*np.nonzero(np.any(gb != rb, axis=-1))):
+                    for t in range(128 * j, min(128 * j + 128, n)):
+                        if not np.array_equal(row_codes(gc, g, t), row_codes(rc, g, t)):
+                            bad.append((g, t))
+                    # rows of the block that were never appended must be untouched (zero) on both sides
+            for g, t in bad:
+                cg = row_codes(gc, g, t).astype(np.int64)
+                cr = row_codes(rc, g, t).astype(np.int64)
                 if g not in Rs:
                     Rs[g] = oracle.rotation_matrix(d, w.quats[g])
                 _, _, u = oracle.quantize_row(d, Rs[g], th, src[b, t, g])

@@ -55,7 +55,7 @@ def test_config1_tiny_decode(iq, torch, codebooks):
 @pytest.mark.parametrize("d", [128, 256])
 @pytest.mark.parametrize("T", [1, 2, 31, 32, 33, 63, 64, 65, 127, 128, 129, 1000])
 def test_shape_sweep_context_lengths(iq, torch, codebooks, d, T):
-    w = workloads.tiny(100 + T, 1, 8 if d == 128 else 4, 2, d, ((T + 3) // 4) * 4, lens=[T])
+    w = workloads.tiny(100 + T, 1, 8 if d == 128 else 4, 2, d, T, lens=[T])
     print(_roundtrip(iq, torch, codebooks, w, [1, 3], n_new=[T]))
 
 
@@ -81,12 +81,13 @@ def test_large_scale_rows_and_zero_rows(iq, torch, codebooks):
 
 
 def test_append_positions_strides_and_out_of_range_rows(iq, torch, codebooks):
-    """Append in two calls at non-zero positions, from a strided source; rows beyond t_cap are skipped and flagged."""
-    d, T = 128, 96
+    """Append in two calls at non-zero positions (not multiples of 32), from a strided source; rows beyond t_cap
+    are skipped and flagged."""
+    d, T = 128, 160
     lv, th = codebooks[d]
     cb = codebook_for(iq, codebooks, d)
     w = workloads.tiny(302, 2, 4, 2, d, T)
-    shape = iq.Shape(2, 4, 2, d, 80)
+    shape = iq.Shape(2, 4, 2, d, 128)
     rot = torch.empty(iq.iq_rotation_floats(d, 2), dtype=torch.float32, device="cuda")
     iq.iq_make_rotation(d, 2, 0, np.ascontiguousarray(w.quats), rot)
     cache = iq.new_cache(shape)
@@ -100,22 +101,23 @@ def test_append_positions_strides_and_out_of_range_rows(iq, torch, codebooks):
     n0 = torch.tensor([40, 17], dtype=torch.int32, device="cuda")
     iq.iq_quantize_append(shape, rot, cb, kview[:, :40], vview[:, :40], pos0, n0, 40, cache, status)
     pos1 = n0.clone()
-    n1 = torch.tensor([56, 30], dtype=torch.int32, device="cuda")                  # sequence 0: rows 80..95 fall outside t_cap = 80
-    k2 = torch.stack([kview[0, 40:96], kview[1, 17:73]])
-    v2 = torch.stack([vview[0, 40:96], vview[1, 17:73]])
-    iq.iq_quantize_append(shape, rot, cb, k2, v2, pos1, n1, 56, cache, status)
+    n1 = torch.tensor([104, 30], dtype=torch.int32, device="cuda")                 # sequence 0: rows 128..143 fall outside t_cap = 128
+    k2 = torch.stack([kview[0, 40:144], kview[1, 17:121]])
+    v2 = torch.stack([vview[0, 40:144], vview[1, 17:121]])
+    iq.iq_quantize_append(shape, rot, cb, k2, v2, pos1, n1, 104, cache, status)
     torch.cuda.synchronize()
     st = status.cpu().numpy()
     assert st[0] & 1 and st[2] == 16 * 2 * 2                                        # 16 rows x 2 KV heads x (K, V)
     g = cache_to_numpy(cache)
-    lens = np.array([80, 47], np.int32)
-    ref = oracle.new_cache(2, 2, d, 80)
-    wk = np.zeros((2, 80, 2, d), np.float16); wv = np.zeros_like(wk)
-    wk[0], wv[0] = w.k[0, :80], w.v[0, :80]
+    lens = np.array([128, 47], np.int32)
+    ref = oracle.new_cache(2, 2, d, 128)
+    wk = np.zeros((2, 128, 2, d), np.float16); wv = np.zeros_like(wk)
+    wk[0], wv[0] = w.k[0, :128], w.v[0, :128]
     wk[1, :47], wv[1, :47] = w.k[1, :47], w.v[1, :47]
     oracle.quantize_append(w.quats, th, wk, wv, np.zeros(2, np.int32), lens, ref)
-    w2 = workloads.Workload("x", 2, 4, 2, d, 80, wk, wv, w.q, w.quats, lens)
+    w2 = workloads.Workload("x", 2, 4, 2, d, 128, wk, wv, w.q, w.quats, lens)
     compare_caches(w2, th, g, ref, lens)
+    assert np.array_equal(g["v_codes"], ref["v_codes"])                             # incl. rows never appended (stay zero)
     res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, lens, 2)
     check_decode(w2, lv, w.q, res, g, lens)
 
@@ -131,7 +133,7 @@ def test_combine_splits_in_isolation(iq, torch, codebooks):
     pm[2, 1, 0, 0] = pm[2, 1, 4, 0] = 50.0; pg[2, 1, 0], pg[2, 1, 4] = 77, 12        # tie on the maximum: lowest row wins
     quats = workloads.quaternion_pairs(g, H_kv, d)
     ref = oracle.combine_splits(quats, pa, pm, pg, H_kv)
-    shape = iq.Shape(B, H_q, H_kv, d, 16)
+    shape = iq.Shape(B, H_q, H_kv, d, 128)
     rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
     iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(quats), rot)
     out = torch.empty((B, H_q, d), dtype=torch.float32, device="cuda")

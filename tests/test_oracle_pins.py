@@ -198,6 +198,33 @@ def test_pack_unpack_roundtrip_and_layout(d):
     assert np.all(seen == 1)                                                    # a bijection onto the 3d bits
 
 
+def test_transposed_v_layout(codebooks):
+    """V codes are stored per 128-row block and coordinate: record ((t // 128) * d + c) * 48 holds the 128 codes of
+    coordinate c, arranged like a packed row of 128 entries (entry = row within the block)."""
+    d, T = 128, 300
+    lv, th = codebooks[d]
+    w = workloads.tiny(9, 1, 1, 1, d, T)
+    cache = oracle.new_cache(1, 1, d, w.t_cap)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(1, np.int32), None, cache)
+    R = oracle.rotation_matrix(d, w.quats[0])
+    area = cache["v_codes"][0, 0].reshape(-1)
+    expect = np.stack([oracle.quantize_row(d, R, th, w.v[0, t, 0])[0] for t in range(T)])          # [T][d] codes
+    for j in range(w.t_cap // 128):
+        for c in (0, 1, 77, 127):
+            rec = area[(j * d + c) * 48:(j * d + c + 1) * 48]
+            col = oracle.unpack_row(128, rec)                                                        # 128 entries = rows of block j
+            rows = np.arange(128 * j, min(128 * j + 128, T))
+            assert np.array_equal(col[:len(rows)], expect[rows, c])
+            assert np.all(col[len(rows):] == 0)                                                      # rows never appended stay zero
+    for t in (0, 31, 32, 127, 128, 299):
+        assert np.array_equal(oracle.v_row_codes(d, cache["v_codes"][0, 0], t), expect[t])
+    # appending row by row gives the same bytes as one bulk append
+    c2 = oracle.new_cache(1, 1, d, w.t_cap)
+    for t in range(T):
+        oracle.quantize_append(w.quats, th, w.k[:, t:t + 1], w.v[:, t:t + 1], np.array([t], np.int32), None, c2)
+    assert all(np.array_equal(cache[k], c2[k]) for k in cache)
+
+
 def test_quantize_row_against_an_independent_numpy_statement(codebooks):
     d = 128
     lv, th = codebooks[d]
@@ -265,7 +292,7 @@ def _reconstruct_then_attend(w, lv, cache, sm_scale=None):
             g = h // w.G
             R = oracle.rotation_matrix(d, w.quats[g])
             K = np.stack([R.T @ (float(cache["k_scales"][b, g, t]) * lv[oracle.unpack_row(d, cache["k_codes"][b, g, t])].astype(np.float64) / math.sqrt(d)) for t in range(n)]) if n else np.zeros((0, d))
-            V = np.stack([R.T @ (float(cache["v_scales"][b, g, t]) * lv[oracle.unpack_row(d, cache["v_codes"][b, g, t])].astype(np.float64) / math.sqrt(d)) for t in range(n)]) if n else np.zeros((0, d))
+            V = np.stack([R.T @ (float(cache["v_scales"][b, g, t]) * lv[oracle.v_row_codes(d, cache["v_codes"][b, g], t)].astype(np.float64) / math.sqrt(d)) for t in range(n)]) if n else np.zeros((0, d))
             if n == 0:
                 am[b, h] = -1
                 continue
@@ -283,7 +310,7 @@ def test_compressed_space_attention_equals_reconstruct_then_compute(codebooks, d
     B = 1 if lens is None else len(lens)
     w = workloads.tiny(3, B, H_q, H_kv, d, T, lens)
     lv, th = codebooks[d]
-    cache = oracle.new_cache(B, H_kv, d, T)
+    cache = oracle.new_cache(B, H_kv, d, w.t_cap)
     oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), w.seq_lens, cache)
     r = oracle.decode_attention(w.quats, lv, w.q, cache, w.seq_lens, H_kv, want_rot=True)
     ref, am = _reconstruct_then_attend(w, lv, cache)
@@ -298,19 +325,19 @@ def test_attention_special_cases(codebooks):
     d = 128
     lv, th = codebooks[d]
     w = workloads.tiny(4, 1, 2, 1, d, 16)
-    cache = oracle.new_cache(1, 1, d, 16)
+    cache = oracle.new_cache(1, 1, d, w.t_cap)
     oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(1, np.int32), None, cache)
     R = oracle.rotation_matrix(d, w.quats[0])
-    recon = lambda c, s: R.T @ (float(s) * lv[oracle.unpack_row(d, c)].astype(np.float64) / math.sqrt(d))
+    recon = lambda t: R.T @ (float(cache["v_scales"][0, 0, t]) * lv[oracle.v_row_codes(d, cache["v_codes"][0, 0], t)].astype(np.float64) / math.sqrt(d))
     # T = 1: the output is the reconstruction of v_0
     r = oracle.decode_attention(w.quats, lv, w.q, cache, np.array([1], np.int32), 1)
-    assert np.allclose(r["out"][0, 0], recon(cache["v_codes"][0, 0, 0], cache["v_scales"][0, 0, 0]), atol=1e-13)
+    assert np.allclose(r["out"][0, 0], recon(0), atol=1e-13)
     assert np.all(r["argmax"] == 0)
     # all keys equal: uniform weights -> mean of reconstructed V, argmax = lowest index
     cache["k_codes"][0, 0, :] = cache["k_codes"][0, 0, 0]
     cache["k_scales"][0, 0, :] = cache["k_scales"][0, 0, 0]
     r = oracle.decode_attention(w.quats, lv, w.q, cache, np.array([16], np.int32), 1)
-    mean_v = np.mean([recon(cache["v_codes"][0, 0, t], cache["v_scales"][0, 0, t]) for t in range(16)], axis=0)
+    mean_v = np.mean([recon(t) for t in range(16)], axis=0)
     assert np.allclose(r["out"][0, 1], mean_v, atol=1e-13) and np.all(r["argmax"] == 0)
     for h in range(2):
         assert abs(r["lse"][0, h] - (oracle.scores(w.quats, lv, w.q, cache, 0, h, 16, 1)[0] + math.log(16))) < 1e-12
@@ -325,7 +352,7 @@ def test_score_error_statistics_against_the_bound(codebooks):
     d = 128
     lv, th = codebooks[d]
     w = workloads.tiny(5, 1, 1, 1, d, 4096)
-    cache = oracle.new_cache(1, 1, d, 4096)
+    cache = oracle.new_cache(1, 1, d, w.t_cap)
     oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(1, np.int32), None, cache)
     z = oracle.scores(w.quats, lv, w.q, cache, 0, 0, 4096, 1, sm_scale=1.0)
     q = w.q[0, 0].astype(np.float64)
@@ -343,7 +370,7 @@ def test_split_merge_equals_unsplit_softmax(codebooks):
     d = 128
     lv, th = codebooks[d]
     w = workloads.tiny(6, 2, 4, 2, d, 100, lens=[100, 63])
-    cache = oracle.new_cache(2, 2, d, 100)
+    cache = oracle.new_cache(2, 2, d, w.t_cap)
     oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(2, np.int32), w.seq_lens, cache)
     full = oracle.decode_attention(w.quats, lv, w.q, cache, w.seq_lens, 2, want_rot=True)
     g = np.random.default_rng(1)
@@ -364,7 +391,7 @@ def test_split_merge_equals_unsplit_softmax(codebooks):
                         continue
                     m = z[lo:hi].max()
                     p = np.exp(z[lo:hi] - m)
-                    vt = np.stack([float(cache["v_scales"][b, h // 2, t]) * lv[oracle.unpack_row(d, cache["v_codes"][b, h // 2, t])].astype(np.float64) / math.sqrt(d) for t in range(lo, hi)])
+                    vt = np.stack([float(cache["v_scales"][b, h // 2, t]) * lv[oracle.v_row_codes(d, cache["v_codes"][b, h // 2], t)].astype(np.float64) / math.sqrt(d) for t in range(lo, hi)])
                     pa[b, h, s] = p @ vt
                     pm[b, h, s] = (m, p.sum())
                     pg[b, h, s] = lo + int(np.argmax(z[lo:hi]))
@@ -379,7 +406,7 @@ def test_retrieval_margins_config4_shape(codebooks):
     d = 128
     lv, th = codebooks[d]
     w = workloads.config4(T=2048, H_q=8, H_kv=2)
-    cache = oracle.new_cache(1, 2, d, 2048)
+    cache = oracle.new_cache(1, 2, d, w.t_cap)
     oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(1, np.int32), None, cache)
     r = oracle.decode_attention(w.quats, lv, w.q, cache, w.seq_lens, 2)
     assert np.array_equal(r["argmax"][0], w.extra["needle_pos"])

@@ -28,6 +28,11 @@ def to_fp16(a: np.ndarray) -> np.ndarray:
     return np.clip(a, -65504.0, 65504.0).astype(np.float16)
 
 
+def cap128(rows: int) -> int:
+    """Cache capacity for `rows` rows: the next multiple of 128 (the V side is stored in 128-row blocks)."""
+    return ((int(rows) + 127) // 128) * 128
+
+
 def quaternion_pairs(gen: np.random.Generator, n_kv_heads: int, d: int) -> np.ndarray:
     """[H_kv][d/4][8] fp32 = (q_L.wxyz, q_R.wxyz), each quaternion of unit length."""
     q = gen.standard_normal((n_kv_heads, d // 4, 2, 4))
@@ -42,7 +47,7 @@ class Workload:
     H_q: int
     H_kv: int
     d: int
-    t_cap: int
+    t_cap: int               # cache rows per (sequence, KV head): multiple of 128, >= T
     k: np.ndarray            # fp16 [B][T][H_kv][d]
     v: np.ndarray            # fp16 [B][T][H_kv][d]
     q: np.ndarray            # fp16 [B][H_q][d]
@@ -70,7 +75,7 @@ def config1(T: int = 1024, H_q: int = 4, H_kv: int = 1, d: int = 128, cfg: int =
     kch = _outlier_channels(sg, k)
     vch = _outlier_channels(sg, v)
     q = rng(cfg, Q_STREAM).standard_normal((1, H_q, d))
-    return Workload("config1", 1, H_q, H_kv, d, T, to_fp16(k), to_fp16(v), to_fp16(q),
+    return Workload("config1", 1, H_q, H_kv, d, cap128(T), to_fp16(k), to_fp16(v), to_fp16(q),
                     quaternion_pairs(rng(cfg, QUAT_STREAM), H_kv, d), np.array([T], np.int32),
                     dict(k_outliers=kch, v_outliers=vch))
 
@@ -88,7 +93,7 @@ def config2(T: int = 8192, steps: int = 64, H_q: int = 32, H_kv: int = 4, d: int
     step_k = st.standard_normal((steps, 1, 1, H_kv, d)) * ks
     step_v = st.standard_normal((steps, 1, 1, H_kv, d)) * vs
     step_q = st.standard_normal((steps, 1, H_q, d))
-    return Workload("config2", 1, H_q, H_kv, d, T + steps, to_fp16(k), to_fp16(v), to_fp16(q),
+    return Workload("config2", 1, H_q, H_kv, d, cap128(T + steps), to_fp16(k), to_fp16(v), to_fp16(q),
                     quaternion_pairs(rng(cfg, QUAT_STREAM), H_kv, d), np.array([T], np.int32),
                     dict(step_k=to_fp16(step_k), step_v=to_fp16(step_v), step_q=to_fp16(step_q), steps=steps))
 
@@ -99,7 +104,7 @@ def config3(T: int = 16384, H_q: int = 16, H_kv: int = 8, d: int = 256) -> Workl
     k = 0.5 * rng(cfg, K_STREAM).standard_t(3.0, (1, T, H_kv, d))
     v = 0.5 * rng(cfg, V_STREAM).standard_t(3.0, (1, T, H_kv, d))
     q = rng(cfg, Q_STREAM).standard_normal((1, H_q, d))
-    return Workload("config3", 1, H_q, H_kv, d, T, to_fp16(k), to_fp16(v), to_fp16(q),
+    return Workload("config3", 1, H_q, H_kv, d, cap128(T), to_fp16(k), to_fp16(v), to_fp16(q),
                     quaternion_pairs(rng(cfg, QUAT_STREAM), H_kv, d), np.array([T], np.int32))
 
 
@@ -119,7 +124,7 @@ def config4(T: int = 32768, H_q: int = 32, H_kv: int = 8, d: int = 128) -> Workl
         k[0, pos[h], g, :] = to_fp16(4.0 * q[0, h, :].astype(np.float64))
         v[0, pos[h], g, :] = 0
         v[0, pos[h], g, chan[h]] = 8.0
-    return Workload("config4", 1, H_q, H_kv, d, T, k, v, q, quaternion_pairs(rng(cfg, QUAT_STREAM), H_kv, d),
+    return Workload("config4", 1, H_q, H_kv, d, cap128(T), k, v, q, quaternion_pairs(rng(cfg, QUAT_STREAM), H_kv, d),
                     np.array([T], np.int32), dict(needle_pos=pos, needle_chan=chan))
 
 
@@ -140,7 +145,7 @@ def config5(B: int, ctx: int, H_q: int = 64, H_kv: int = 8, d: int = 128) -> Wor
     kch = _outlier_channels(sg, k)
     vch = _outlier_channels(sg, v)
     q = np.random.Generator(np.random.Philox(stream_seed(cfg, Q_STREAM) + sub)).standard_normal((B, H_q, d))
-    return Workload(f"config5_B{B}_ctx{ctx}", B, H_q, H_kv, d, ctx, to_fp16(k), to_fp16(v), to_fp16(q),
+    return Workload(f"config5_B{B}_ctx{ctx}", B, H_q, H_kv, d, cap128(ctx), to_fp16(k), to_fp16(v), to_fp16(q),
                     quaternion_pairs(rng(cfg, QUAT_STREAM), H_kv, d), lens, dict(k_outliers=kch, v_outliers=vch))
 
 
@@ -181,4 +186,4 @@ def tiny(seed: int, B: int, H_q: int, H_kv: int, d: int, T: int, lens=None, scal
     quats = quaternion_pairs(g, H_kv, d)
     if lens is None:
         lens = np.full(B, T, np.int32)
-    return Workload(f"tiny{seed}", B, H_q, H_kv, d, T, k, v, q, quats, np.asarray(lens, np.int32))
+    return Workload(f"tiny{seed}", B, H_q, H_kv, d, cap128(T), k, v, q, quats, np.asarray(lens, np.int32))
