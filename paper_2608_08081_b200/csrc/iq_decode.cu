@@ -16,15 +16,15 @@
 //         O[c][n] = sum_row A_V[c][row] * B_P[n][row]
 //   5. thread c folds O (hi + lo columns) into its running accumulator for coordinate c.
 // Packed tiles arrive through a 1-D bulk-copy (TMA) pipeline; every wait is bounded.
-#include <cstdio>
-
 #include "iq_common.cuh"
 #include "iq_kernels.h"
 
 namespace iq {
 
+// Tuning knob: 1 = the K and V operand tiles share TMEM columns at d = 128 (4 CTAs per SM, measured fastest),
+// 0 = separate tiles (3 CTAs per SM, the dequantisation of one tile overlaps the MMAs on the other).
 #ifndef IQ_DEC_SHARED128
-#define IQ_DEC_SHARED128 0
+#define IQ_DEC_SHARED128 1
 #endif
 constexpr int DEC_COMPUTE_THREADS = 128;  // 4 warps: dequantisation, softmax, accumulation (thread = TMEM lane)
 constexpr int DEC_THREADS = 160;          // + 1 control warp: issues the bulk copies and the MMAs
@@ -376,14 +376,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode
       tc_fence_before();
     };
 
-#ifdef IQ_DEC_TIMING
-    long long tph[10] = {0,0,0,0,0,0,0,0,0,0}; long long tc0 = clock64();
-#define TPH(i) { long long tnow = clock64(); tph[i] += tnow - tc0; tc0 = tnow; }
-#else
-#define TPH(i)
-#endif
     k_phase(0);
-    TPH(0)
     bool folded = true;  // is the value product of the previous block already in acc?
     for (int blk = 0; blk < nblk; blk++) {
       const uint8_t* sp = stages + (blk % NST) * L::STAGE_BYTES;
@@ -393,7 +386,6 @@ __global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode
         if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)blk & 1u, DEC_WAIT_LIMIT);
       }
       if (!folded) { fold(blk - 1); folded = true; }  // also: the value MMAs of the previous block have released A_V and B_P
-      TPH(1)
 
       // ---- V coordinate tid (+128) of this block -> TMEM lane tid (A_V), while the score MMAs run
 #pragma unroll
@@ -412,7 +404,6 @@ __global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode
           tc_st16(tmem_a + lane_sel + L::AV_COL + 64 * j + 16 * u, f);
         }
       }
-      TPH(2)
       const float ksc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES)[tid];
       const float vsc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES)[tid];
 
@@ -420,7 +411,6 @@ __global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode
       if (!L::SHARED_A) {
         if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)blk & 1u, DEC_WAIT_LIMIT);
       }
-      TPH(3)
       tc_fence_after();
       float s[8];
       {
@@ -442,7 +432,6 @@ __global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode
       // The running reference m_run is raised only when some score of the block exceeds it by more than
       // DEC_MAX_SLACK (log2 units): exp2(s - m_run) then stays below 2^DEC_MAX_SLACK and nothing has to be
       // exchanged between the warps in the common case (one barrier with an OR reduction).
-      TPH(4)
       bool exceed = false;
 #pragma unroll
       for (int h = 0; h < 8; h++) exceed |= (s[h] - m_run[h] > DEC_MAX_SLACK);
@@ -465,7 +454,6 @@ __global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode
 #pragma unroll
         for (int h = 0; h < 8; h++) alpha[h] = 1.f;
       }
-      TPH(5)
       {
         const float vf = (tid < n) ? vsc * vfac : 0.f;
         float wv[8];
@@ -491,26 +479,18 @@ __global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode
         *reinterpret_cast<uint4*>(bp + (TB / 8) * 128 + off) = lo4;
         fence_proxy_async();
       }
-      TPH(6)
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(p_ready);                 // V tile in TMEM, probabilities in shared memory
       mbar_arrive(&empty_bar[blk % NST]);   // this thread is done with the staged tile
       folded = false;
-      TPH(7)
       // ---- next block's K tile, while the value MMAs run
       if (blk + 1 < nblk) {
         if (L::SHARED_A) { fold(blk); folded = true; }  // the value MMAs read the tile that K is about to overwrite
         k_phase(blk + 1);
       }
-      TPH(0)
     }
     if (!folded) fold(nblk - 1);
-#ifdef IQ_DEC_TIMING
-    TPH(1)
-    if (tid == 0 && blockIdx.x == 1 && blockIdx.y == 3 && blockIdx.z == 2)
-      printf("nblk %d: kphase %lld fold %lld vdequant %lld wait_s %lld ldS+best %lld max-barrier %lld P %lld waitst+arrive %lld (cycles per block)\n", nblk, tph[0]/nblk, tph[1]/nblk, tph[2]/nblk, tph[3]/nblk, tph[4]/nblk, tph[5]/nblk, tph[6]/nblk, tph[7]/nblk);
-#endif
   }
 
   if (__syncthreads_or(failed) && tid == 0 && p.status) atomicOr(&p.status[0], IQ_STATUS_WAIT_TIMEOUT);
