@@ -71,8 +71,18 @@ struct RowQuantizer {
     for (int e = 0; e < E; e++) ss += (double)x[e] * (double)x[e];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(FULL, ss, o);
-    const double s64 = sqrt(ss);
-    const float inv_s = (s64 > 0.0) ? (float)(1.0 / s64) : 0.f;
+    // Stored scale = sqrt(ss) rounded to fp32. An fp32 estimate is corrected with exact fp64 midpoint tests
+    // (x and its neighbours are fp32, so (x +- ulp/2)^2 is exact in fp64 up to one rounding): this avoids the
+    // software double-precision square root on every row.
+    float s = sqrtf((float)ss);
+    {
+      const float up = __uint_as_float(__float_as_uint(s) + 1u);
+      const float dn = (s > 0.f) ? __uint_as_float(__float_as_uint(s) - 1u) : 0.f;
+      const double mu = 0.5 * ((double)s + (double)up), md = 0.5 * ((double)s + (double)dn);
+      if (ss > mu * mu) s = up;
+      else if (s > 0.f && ss < md * md) s = dn;
+    }
+    const float inv_s = (s > 0.f) ? __frcp_rn(s) : 0.f;
 
     // Step 2: u = sqrt(d) * R x^ = M_b (H_unnormalised x) / s  (the two sqrt(d) factors cancel)
     float v[E];
@@ -102,12 +112,12 @@ struct RowQuantizer {
 #pragma unroll
       for (int e = 0; e < E; e++) {
         bool nb;
-        const double u = (s64 > 0.0) ? vd[e] / s64 : 0.0;
+        const double u = (ss > 0.0) ? vd[e] / sqrt(ss) : 0.0;
         code[e] = decide_code<double>(u, th, nb, 0.0);
       }
       if (lane == 0 && status) atomicAdd(&status[1], 1u);
     }
-    return (float)s64;
+    return s;
   }
 };
 

@@ -236,3 +236,55 @@ def test_config5_small_points_in_full(iq, torch, codebooks, B, ctx):
     res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, w.seq_lens, S)
     c = check_decode(w, lv, w.q, res, g, w.seq_lens)
     print(c["max_err"], c["margin"])
+
+
+def test_full_size_bench_configuration_sampled(iq, torch, codebooks):
+    """Config 5 at B = 32, ctx = 32768 (the workload bench.py times), same launch configuration (library codebook,
+    iq_suggest_splits, no argmax). The oracle checks sampled (sequence, KV head) slabs: their packed rows are
+    re-quantised and every query head of the group is decoded from the GPU's own cache."""
+    import bench
+
+    name = bench.DEFAULT_WORKLOAD
+    B, ctx, H_q, H_kv, d = bench.WORKLOADS[name]
+    st = bench.build_state(name, torch.device("cuda", 0), 0)
+    shape, cb, rot, cache = st["shape"], st["cb"], st["rot"], st["cache"]
+    lv = np.array(cb.levels, np.float32)
+    th = np.array(cb.thresholds, np.float32)
+    S = iq.iq_suggest_splits(shape, ctx)
+    ws = iq.DecodeWorkspace(shape, S, want_argmax=False)
+    lens = torch.from_numpy(st["lens_np"]).cuda()
+    q = st["q0"]
+    iq.decode_step(shape, rot, cb, q, cache, lens, ws)
+    torch.cuda.synchronize()
+    assert int(ws.status[0]) == 0 and int(st["status"][0]) == 0
+    out = ws.out.cpu().numpy().astype(np.float64)
+    lse = ws.lse.cpu().numpy().astype(np.float64)
+    G = H_q // H_kv
+    g = np.random.default_rng(3)
+    for b, kvh in [(0, 0), (int(np.argmax(st["lens_np"])), 7), (int(np.argmin(st["lens_np"])), 3), (int(g.integers(B)), int(g.integers(H_kv)))]:
+        n = int(st["lens_np"][b])
+        sub = {k: np.ascontiguousarray(getattr(cache, k)[b:b + 1, kvh:kvh + 1].cpu().numpy()) for k in ("k_codes", "k_scales", "v_codes", "v_scales")}
+        qs = np.ascontiguousarray(q[b:b + 1, kvh * G:(kvh + 1) * G].cpu().numpy())
+        ref = oracle.decode_attention(st["quats"][kvh:kvh + 1], lv, qs, sub, np.array([n], np.int32), 1)
+        o = out[b, kvh * G:(kvh + 1) * G]
+        err = np.abs(o - ref["out"][0])
+        assert np.all(err <= 2e-3 + 1e-3 * np.abs(ref["out"][0])), f"(b={b}, kvh={kvh}) max err {err.max():.3e}"
+        assert np.allclose(lse[b, kvh * G:(kvh + 1) * G], ref["lse"][0], atol=2e-3, rtol=1e-5)
+    # quantize parity on sampled rows of the same cache: the generator is replayed for the first chunk of sequences
+    gen = workloads.config5_device(B, ctx, torch.device("cuda", 0), H_q, H_kv, d)
+    b0, k, v = next(iter(gen["chunks"]()))
+    k, v = k.cpu().numpy(), v.cpu().numpy()
+    kc = cache.k_codes[:k.shape[0]].cpu().numpy()
+    vc = cache.v_codes[:k.shape[0]].cpu().numpy()
+    ks = cache.k_scales[:k.shape[0]].cpu().numpy()
+    Rs = {h: oracle.rotation_matrix(d, st["quats"][h]) for h in range(H_kv)}
+    checked = 0
+    for _ in range(400):
+        b, h = int(g.integers(k.shape[0])), int(g.integers(H_kv))
+        t = int(g.integers(int(st["lens_np"][b])))
+        ck, sk, _ = oracle.quantize_row(d, Rs[h], th, k[b, t, h])
+        cv, _, _ = oracle.quantize_row(d, Rs[h], th, v[b, t, h])
+        assert np.array_equal(oracle.unpack_row(d, kc[b, h, t]), ck) and ks[b, h, t] == sk
+        assert np.array_equal(oracle.v_row_codes(d, vc[b, h], t), cv)
+        checked += 1
+    assert checked == 400
