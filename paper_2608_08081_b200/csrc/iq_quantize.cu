@@ -26,56 +26,122 @@ __device__ __forceinline__ int decide_code(T u, const float (&th)[7], bool& near
   return (b2 ? 4 : 0) + (b1 ? 2 : 0) + (b0 ? 1 : 0);
 }
 
-// Per-warp state that does not change from row to row: the lane's SO(4) blocks and the thresholds.
+// Work mapping of the row kernels: a row is shared by LPR = d/16 lanes, 16 consecutive coordinates (4 whole SO(4)
+// blocks) per lane, so a warp holds 32/LPR rows at a time (4 at d = 128, 2 at d = 256). The Walsh-Hadamard
+// butterfly runs 4 stages inside the lane and log2(LPR) xor-shuffle stages across the row's lanes; a 32-coordinate
+// packing unit is a pair of lanes.
 template <int D>
 struct RowQuantizer {
-  static constexpr int E = D / 32;  // coordinates per lane: lane l owns coordinates l*E .. l*E+E-1
-  static constexpr int NB = E / 4;  // SO(4) blocks per lane
-  float q8[NB][8];
+  static constexpr int E = 16;
+  static constexpr int LPR = D / E;        // lanes per row: 8 or 16
+  static constexpr int RPW = 32 / LPR;     // rows per warp: 4 or 2
+  static constexpr int NB = E / 4;         // SO(4) blocks per lane
+  const float* qbase;      // this lane's NB quaternion pairs
+  const float* th_global;  // the 7 thresholds in memory (for the out-of-line fp64 path)
   float M[NB][4][4];
   float th[7];
 
   __device__ __forceinline__ void init(const float* rot_head, const float* thresholds, int lane) {
-    const float* qbase = rot_head + (size_t)lane * NB * 8;
+    qbase = rot_head + (size_t)(lane % LPR) * NB * 8;
 #pragma unroll
     for (int j = 0; j < NB; j++) {
+      float q8[8];
 #pragma unroll
-      for (int i = 0; i < 8; i++) q8[j][i] = qbase[j * 8 + i];
-      so4_matrix<float>(q8[j], M[j]);
+      for (int i = 0; i < 8; i++) q8[i] = qbase[j * 8 + i];
+      so4_matrix<float>(q8, M[j]);
     }
 #pragma unroll
     for (int i = 0; i < 7; i++) th[i] = thresholds[i];
+    th_global = thresholds;
   }
 
-  // Algorithm 1, steps 1-3 for one row: returns the fp32 scale, fills code[E]. `src` points at this lane's E values.
-  __device__ __forceinline__ float run(const __half* src, int lane, int (&code)[E], uint32_t* status) const {
-    float x[E];
-    if (E == 4) {
-      const uint2 raw = *reinterpret_cast<const uint2*>(src);
-      const __half2 h0 = *reinterpret_cast<const __half2*>(&raw.x), h1 = *reinterpret_cast<const __half2*>(&raw.y);
-      x[0] = __low2float(h0); x[1] = __high2float(h0); x[2] = __low2float(h1); x[3] = __high2float(h1);
-    } else {
-      const uint4 raw = *reinterpret_cast<const uint4*>(src);
-      const uint32_t r[4] = {raw.x, raw.y, raw.z, raw.w};
+  // butterflies across the lanes of one row (strides 16, 32, ...): lane bit b of (lane % LPR) <-> stride 16 << b
+  template <typename T>
+  __device__ __forceinline__ static void wht(T (&v)[E], int lane) {
 #pragma unroll
-      for (int k = 0; k < 4; k++) {
-        const __half2 hh = *reinterpret_cast<const __half2*>(&r[k]);
-        x[2 * k] = __low2float(hh);
-        x[2 * k + 1] = __high2float(hh);
+    for (int s = 1; s < E; s <<= 1)
+#pragma unroll
+      for (int i = 0; i < E; i++)
+        if ((i & s) == 0) {
+          const T a = v[i], c = v[i + s];
+          v[i] = a + c;
+          v[i + s] = a - c;
+        }
+#pragma unroll
+    for (int o = 1; o < LPR; o <<= 1) {
+      const T sgn = (lane & o) ? T(-1) : T(1);  // the upper lane of a pair keeps (other - own)
+#pragma unroll
+      for (int i = 0; i < E; i++) {
+        const T other = shfl_xor_t<T>(v[i], o);
+        v[i] = sgn * v[i] + other;  // one fused multiply-add, exact: sgn is +-1
       }
     }
-    // Step 1: s = ||x||_2. Squares of fp16 values are exact in fp64; the sum is accumulated in fp64 so that
-    // the stored fp32 scale is the correctly rounded norm.
+  }
+
+  __device__ __forceinline__ static void unpack16(const uint4& r0, const uint4& r1, float (&x)[E]) {
+    const uint32_t r[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+    for (int k = 0; k < 8; k++) {
+      const __half2 hh = *reinterpret_cast<const __half2*>(&r[k]);
+      x[2 * k] = __low2float(hh);
+      x[2 * k + 1] = __high2float(hh);
+    }
+  }
+
+  // The rare path: re-decide the warp's rows in fp64, where the +-1 sums of fp16 values are exact. Kept out of line
+  // so that its registers do not count against the common path.
+  __device__ __forceinline__ static uint2 redo_fp64(uint4 r0, uint4 r1, double ss, int lane, const float* qbase,
+                                                 const float* th_global) {
+    float th[7];
+#pragma unroll
+    for (int i = 0; i < 7; i++) th[i] = th_global[i];
+    int code[E];
+    float x[E];
+    unpack16(r0, r1, x);
+    double vd[E];
+#pragma unroll
+    for (int e = 0; e < E; e++) vd[e] = (double)x[e];
+    wht<double>(vd, lane);
+    const double inv_sd = (ss > 0.0) ? 1.0 / sqrt(ss) : 0.0;
+#pragma unroll
+    for (int j = 0; j < NB; j++) {
+      float q8[8];
+#pragma unroll
+      for (int i = 0; i < 8; i++) q8[i] = qbase[j * 8 + i];
+      double Md[1][4][4];
+      so4_matrix<double>(q8, Md[0]);
+      double blk[4] = {vd[4 * j], vd[4 * j + 1], vd[4 * j + 2], vd[4 * j + 3]};
+      so4_apply<double, 4, false>(Md, blk);
+#pragma unroll
+      for (int r = 0; r < 4; r++) {
+        bool nb;
+        code[4 * j + r] = decide_code<double>(blk[r] * inv_sd, th, nb, 0.0);
+      }
+    }
+    uint2 packed = make_uint2(0u, 0u);  // 16 codes as nibbles
+#pragma unroll
+    for (int n = 0; n < 8; n++) {
+      packed.x |= (uint32_t)code[n] << (4 * n);
+      packed.y |= (uint32_t)code[8 + n] << (4 * n);
+    }
+    return packed;
+  }
+
+  // Algorithm 1, steps 1-3 for the row this lane belongs to (r0, r1 = this lane's 16 fp16 values, zeros for the
+  // lanes of a row that is not written; those lanes still take part in the shuffles). Returns the fp32 scale.
+  __device__ __forceinline__ float run(const uint4& r0, const uint4& r1, bool active, int lane, int (&code)[E],
+                                       uint32_t* status) const {
+    float x[E];
+    unpack16(r0, r1, x);
+    // Step 1: s = ||x||_2. Squares of fp16 values are exact in fp32 (22 bits); they are summed in fp64 so that the
+    // stored fp32 scale is the correctly rounded norm.
     double ss = 0.0;
 #pragma unroll
-    for (int e = 0; e < E; e++) ss += (double)x[e] * (double)x[e];
+    for (int e = 0; e < E; e += 2) ss += (double)(x[e] * x[e]) + (double)(x[e + 1] * x[e + 1]);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(FULL, ss, o);
-    // Stored scale = sqrt(ss) rounded to fp32. An fp32 estimate is corrected with exact fp64 midpoint tests
-    // (x and its neighbours are fp32, so (x +- ulp/2)^2 is exact in fp64 up to one rounding): this avoids the
-    // software double-precision square root on every row.
+    for (int o = 1; o < LPR; o <<= 1) ss += __shfl_xor_sync(FULL, ss, o);
     float s = sqrtf((float)ss);
-    {
+    {  // correct the fp32 estimate with exact fp64 midpoint tests instead of a double-precision square root
       const float up = __uint_as_float(__float_as_uint(s) + 1u);
       const float dn = (s > 0.f) ? __uint_as_float(__float_as_uint(s) - 1u) : 0.f;
       const double mu = 0.5 * ((double)s + (double)up), md = 0.5 * ((double)s + (double)dn);
@@ -85,51 +151,61 @@ struct RowQuantizer {
     const float inv_s = (s > 0.f) ? __frcp_rn(s) : 0.f;
 
     // Step 2: u = sqrt(d) * R x^ = M_b (H_unnormalised x) / s  (the two sqrt(d) factors cancel)
-    float v[E];
-#pragma unroll
-    for (int e = 0; e < E; e++) v[e] = x[e];
-    wht_warp<float, E>(v, lane);
-    so4_apply<float, E, false>(M, v);
+    wht<float>(x, lane);
+    so4_apply<float, E, false>(M, x);
 
     // Step 3: codes, with a guard band around the thresholds
     bool any_near = false;
 #pragma unroll
     for (int e = 0; e < E; e++) {
       bool nb;
-      code[e] = decide_code<float>(v[e] * inv_s, th, nb, GUARD_BAND);
+      code[e] = decide_code<float>(x[e] * inv_s, th, nb, GUARD_BAND);
       any_near |= nb;
     }
-    if (__any_sync(FULL, any_near)) {
-      // Re-decide the whole row in fp64: the +-1 sums of fp16 values are exact in fp64.
-      double vd[E];
-      double Md[NB][4][4];
+    const unsigned rows_near = __ballot_sync(FULL, any_near && active);
+    if (rows_near) {
+      const uint2 packed = redo_fp64(r0, r1, ss, lane, qbase, th_global);
 #pragma unroll
-      for (int e = 0; e < E; e++) vd[e] = (double)x[e];
-#pragma unroll
-      for (int j = 0; j < NB; j++) so4_matrix<double>(q8[j], Md[j]);
-      wht_warp<double, E>(vd, lane);
-      so4_apply<double, E, false>(Md, vd);
-#pragma unroll
-      for (int e = 0; e < E; e++) {
-        bool nb;
-        const double u = (ss > 0.0) ? vd[e] / sqrt(ss) : 0.0;
-        code[e] = decide_code<double>(u, th, nb, 0.0);
+      for (int n = 0; n < 8; n++) {
+        code[n] = (packed.x >> (4 * n)) & 7;
+        code[8 + n] = (packed.y >> (4 * n)) & 7;
       }
-      if (lane == 0 && status) atomicAdd(&status[1], 1u);
+      int n_rows = 0;
+#pragma unroll
+      for (int r = 0; r < RPW; r++) n_rows += ((rows_near >> (r * LPR)) & ((1u << (LPR - 1)) * 2u - 1u)) != 0u;
+      if (lane == 0 && status) atomicAdd(&status[1], (unsigned)n_rows);
     }
     return s;
   }
 };
 
+// Packed words of one row from per-lane codes: a packing unit is the lane pair (2p, 2p+1). Returns, for even lanes,
+// words 0 and 1 of the unit in (w0, w1); for odd lanes word 2 in w0.
+__device__ __forceinline__ void pack_pair(const int (&code)[16], int lane, uint32_t& w0, uint32_t& w1) {
+  uint32_t lo = 0, hi = 0;
+#pragma unroll
+  for (int n = 0; n < 8; n++) {
+    lo |= (uint32_t)code[n] << (4 * n);
+    hi |= (uint32_t)code[8 + n] << (4 * n);
+  }
+  // odd lane: lo = entries 16..23 (word 2), hi = entries 24..31 (the bit-sliced ones)
+  const uint32_t xs = __shfl_xor_sync(FULL, hi, 1);  // even lanes receive the odd lane's sliced nibble word
+  if (lane & 1) {
+    w0 = lo | (((hi >> 2) & 0x11111111u) << 3);
+    w1 = 0u;
+  } else {
+    w0 = lo | ((xs & 0x11111111u) << 3);
+    w1 = hi | (((xs >> 1) & 0x11111111u) << 3);
+  }
+}
+
 // ---------------------------------------------------------------------------------------------------------
-// K rows: one warp per row, packed row-major (3d/8 bytes per row).
+// K rows: packed row-major (3d/8 bytes per row).
 // ---------------------------------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(QA_WARPS * 32) quantize_append_k_kernel(const QuantizeParams p) {
-  constexpr int E = D / 32;
-  constexpr int LPU = 32 / E;      // lanes per 32-coordinate packing unit
-  constexpr int WPR = 3 * D / 32;  // 32-bit words per packed row
-
+__global__ void __launch_bounds__(QA_WARPS * 32, 3) quantize_append_k_kernel(const __grid_constant__ QuantizeParams p) {
+  using RQ = RowQuantizer<D>;
+  constexpr int LPR = RQ::LPR, RPW = RQ::RPW;
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int b = blockIdx.z;
@@ -142,67 +218,62 @@ __global__ void __launch_bounds__(QA_WARPS * 32) quantize_append_k_kernel(const 
   const int row_end = min(n_new, row_begin + QA_ROWS_PER_WARP);
   const int pos0 = p.append_pos[b];
 
-  RowQuantizer<D> rq;
+  RQ rq;
   rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane);
-  const __half* src_base = p.k_new + (size_t)b * p.stride_b + (size_t)h * p.stride_h + lane * E;
+  const int li = lane % LPR, sub = lane / LPR;  // lane within the row, row within the warp
+  const __half* src_base = p.k_new + (size_t)b * p.stride_b + (size_t)h * p.stride_h + li * 16;
   const size_t slab = ((size_t)b * p.n_kv_heads + h) * (size_t)p.t_cap;
 
-  for (int i = row_begin; i < row_end; i++) {
+  auto fetch = [&](int i0, uint4& r0, uint4& r1, bool& exists, bool& active) {
+    const int i = i0 + sub;
     const long long t = (long long)pos0 + i;
-    if (t < 0 || t >= p.t_cap) {
-      if (lane == 0 && p.status) {
-        atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
-        atomicAdd(&p.status[2], 1u);
-      }
-      continue;
+    exists = i < row_end;
+    active = exists && t >= 0 && t < p.t_cap;
+    r0 = r1 = make_uint4(0u, 0u, 0u, 0u);
+    if (active) {
+      const uint4* src = reinterpret_cast<const uint4*>(src_base + (size_t)i * p.stride_t);
+      r0 = __ldg(src);
+      r1 = __ldg(src + 1);
     }
-    int code[E];
-    const float s = rq.run(src_base + (size_t)i * p.stride_t, lane, code, p.status);
-
-    // Step 4: bit-pack. A packing unit is 32 coordinates = LPU lanes = 3 words.
-    uint32_t w[3] = {0u, 0u, 0u};
-    const int c0 = (lane % LPU) * E;  // unit-local coordinate of this lane's first element
-#pragma unroll
-    for (int e = 0; e < E; e++) {
-      const int c = c0 + e;
-      const uint32_t cd = (uint32_t)code[e];
-      if (c < 24) {
-        const uint32_t val = cd << (4 * (c & 7));
-        if ((c >> 3) == 0) w[0] |= val;
-        else if ((c >> 3) == 1) w[1] |= val;
-        else w[2] |= val;
-      } else {
-        const int sh = 4 * (c - 24) + 3;
-        w[0] |= (cd & 1u) << sh;
-        w[1] |= ((cd >> 1) & 1u) << sh;
-        w[2] |= ((cd >> 2) & 1u) << sh;
-      }
+  };
+  uint4 n0, n1;
+  bool n_exists, n_active;
+  fetch(row_begin, n0, n1, n_exists, n_active);
+  for (int i0 = row_begin; i0 < row_end; i0 += RPW) {
+    const uint4 r0 = n0, r1 = n1;
+    const bool exists = n_exists, active = n_active;
+    if (i0 + RPW < row_end) fetch(i0 + RPW, n0, n1, n_exists, n_active);  // next rows in flight during this group's math
+    const long long t = (long long)pos0 + i0 + sub;
+    if (exists && !active && li == 0 && p.status) {
+      atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
+      atomicAdd(&p.status[2], 1u);
     }
-#pragma unroll
-    for (int o = 1; o < LPU; o <<= 1) {
-      w[0] |= __shfl_xor_sync(FULL, w[0], o);
-      w[1] |= __shfl_xor_sync(FULL, w[1], o);
-      w[2] |= __shfl_xor_sync(FULL, w[2], o);
+    int code[16];
+    const float s = rq.run(r0, r1, active, lane, code, p.status);
+    uint32_t w0, w1;
+    pack_pair(code, lane, w0, w1);
+    if (active) {
+      uint32_t* unit_words = reinterpret_cast<uint32_t*>(p.k_codes + (slab + (size_t)t) * (size_t)(3 * D / 8)) + 3 * (li >> 1);
+      if (li & 1) unit_words[2] = w0;
+      else { unit_words[0] = w0; unit_words[1] = w1; }
+      if (li == 0) p.k_scales[slab + (size_t)t] = s;
     }
-    const int k = lane % LPU;
-    uint32_t* row_words = reinterpret_cast<uint32_t*>(p.k_codes + (slab + (size_t)t) * (size_t)(WPR * 4));
-    if (k < 3) row_words[3 * (lane / LPU) + k] = (k == 0) ? w[0] : (k == 1 ? w[1] : w[2]);
-    if (lane == 0) p.k_scales[slab + (size_t)t] = s;
   }
 }
 
 // ---------------------------------------------------------------------------------------------------------
 // V rows: stored token-transposed. For every block of 128 cache rows and every coordinate c there is one
-// 48-byte row holding the 128 codes of coordinate c, arranged like a packing unit sequence with the
-// row-in-block in the role of the coordinate. One CTA handles one 32-row unit of one (sequence, KV head):
-// its warps quantise the unit's new rows, the codes go through shared memory, and thread c assembles the
-// three words of (unit, coordinate c). Words that are only partly covered by new rows are read, merged and
-// written back; no other CTA touches them.
+// 48-byte record holding the 128 codes of coordinate c, arranged like a packing unit sequence with the
+// row-in-block in the role of the entry. One CTA handles one 32-row unit of one (sequence, KV head): its warps
+// quantise the unit's new rows, the codes go through shared memory, and thread c assembles the three words of
+// (unit, coordinate c). Words that are only partly covered by new rows are read, merged and written back; no
+// other CTA touches them.
 // ---------------------------------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(128) quantize_append_v_kernel(const QuantizeParams p) {
-  constexpr int E = D / 32;
-  __shared__ uint8_t codes_s[32][D];
+__global__ void __launch_bounds__(128, 3) quantize_append_v_kernel(const __grid_constant__ QuantizeParams p) {
+  using RQ = RowQuantizer<D>;
+  constexpr int LPR = RQ::LPR, RPW = RQ::RPW;
+  __shared__ __align__(16) uint8_t codes_s[32][D + 16];  // +16: the 16-byte stores of different rows hit different banks
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.z;
@@ -217,60 +288,74 @@ __global__ void __launch_bounds__(128) quantize_append_v_kernel(const QuantizePa
   if (t_lo >= t_hi) return;
   const size_t slab = ((size_t)b * p.n_kv_heads + h) * (size_t)p.t_cap;
   const bool in_cache = unit >= 0 && unit * 32 + 32 <= p.t_cap;  // t_cap is a multiple of 128
+  if (!in_cache) {
+    if (tid == 0 && p.status) {
+      atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
+      atomicAdd(&p.status[2], (unsigned)(t_hi - t_lo));
+    }
+    return;
+  }
 
-  RowQuantizer<D> rq;
+  RQ rq;
   rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane);
-  const __half* src_base = p.v_new + (size_t)b * p.stride_b + (size_t)h * p.stride_h + lane * E;
-  for (long long t = t_lo + warp; t < t_hi; t += 4) {
-    if (!in_cache) {
-      if (lane == 0 && p.status) {
-        atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
-        atomicAdd(&p.status[2], 1u);
-      }
-      continue;
-    }
-    int code[E];
-    const float s = rq.run(src_base + (size_t)(t - pos0) * p.stride_t, lane, code, p.status);
-    uint32_t packed = 0;
+  const int li = lane % LPR, sub = lane / LPR;
+  const __half* src_base = p.v_new + (size_t)b * p.stride_b + (size_t)h * p.stride_h + li * 16;
+  uint4 rr[32 / (4 * RPW)][2];  // all of this warp's rows are fetched up front
 #pragma unroll
-    for (int e = 0; e < E; e++) packed |= (uint32_t)code[e] << (8 * (e & 3));
-    if (E == 4) {
-      *reinterpret_cast<uint32_t*>(&codes_s[t & 31][lane * 4]) = packed;
-    } else {
-      uint32_t p0 = 0, p1 = 0;
-#pragma unroll
-      for (int e = 0; e < 4; e++) { p0 |= (uint32_t)code[e] << (8 * e); p1 |= (uint32_t)code[4 + e] << (8 * e); }
-      *reinterpret_cast<uint2*>(&codes_s[t & 31][lane * 8]) = make_uint2(p0, p1);
+  for (int it = 0; it < 32 / (4 * RPW); it++) {
+    const long long t = t_lo + (it * 4 + warp) * RPW + sub;
+    rr[it][0] = rr[it][1] = make_uint4(0u, 0u, 0u, 0u);
+    if (t < t_hi) {
+      const uint4* src = reinterpret_cast<const uint4*>(src_base + (size_t)(t - pos0) * p.stride_t);
+      rr[it][0] = __ldg(src);
+      rr[it][1] = __ldg(src + 1);
     }
-    if (lane == 0) p.v_scales[slab + (size_t)t] = s;
+  }
+#pragma unroll
+  for (int it = 0; it < 32 / (4 * RPW); it++) {
+    const long long t0 = t_lo + (it * 4 + warp) * RPW;
+    if (t0 >= t_hi) break;
+    const long long t = t0 + sub;
+    const bool active = t < t_hi;
+    int code[16];
+    const float s = rq.run(rr[it][0], rr[it][1], active, lane, code, p.status);
+    if (active) {
+      uint32_t pk[4];
+#pragma unroll
+      for (int q = 0; q < 4; q++)
+        pk[q] = (uint32_t)code[4 * q] | ((uint32_t)code[4 * q + 1] << 8) | ((uint32_t)code[4 * q + 2] << 16) | ((uint32_t)code[4 * q + 3] << 24);
+      *reinterpret_cast<uint4*>(&codes_s[t & 31][li * 16]) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      if (li == 0) p.v_scales[slab + (size_t)t] = s;
+    }
   }
   __syncthreads();
-  if (!in_cache) return;
 
   const int c_lo = (int)(t_lo & 31), c_hi = (int)(t_hi - unit * 32);  // rows [c_lo, c_hi) of the unit are new
   const size_t blk = (size_t)(unit * 32) / 128;
   const int u = (int)((unit * 32) % 128) / 32;
+  const bool full = (c_lo == 0 && c_hi == 32);
 #pragma unroll
   for (int j = 0; j < D / 128; j++) {
     const int c = tid + 128 * j;  // coordinate
     uint32_t w[3] = {0u, 0u, 0u}, m[3] = {0u, 0u, 0u};
-    for (int r = c_lo; r < c_hi; r++) {
-      const uint32_t cd = codes_s[r][c];
-      if (r < 24) {
-        const int sh = 4 * (r & 7);
-        w[r >> 3] |= cd << sh;
-        m[r >> 3] |= 7u << sh;
-      } else {
-        const int sh = 4 * (r - 24) + 3;
 #pragma unroll
-        for (int k = 0; k < 3; k++) {
-          w[k] |= ((cd >> k) & 1u) << sh;
-          m[k] |= 1u << sh;
+    for (int r = 0; r < 32; r++) {
+      if (r >= c_lo && r < c_hi) {
+        const uint32_t cd = codes_s[r][c];
+        if (r < 24) {
+          w[r >> 3] |= cd << (4 * (r & 7));
+          m[r >> 3] |= 7u << (4 * (r & 7));
+        } else {
+          const int sh = 4 * (r - 24) + 3;
+#pragma unroll
+          for (int k = 0; k < 3; k++) {
+            w[k] |= ((cd >> k) & 1u) << sh;
+            m[k] |= 1u << sh;
+          }
         }
       }
     }
     uint32_t* dst = reinterpret_cast<uint32_t*>(p.v_codes + ((slab / 128 + blk) * D + c) * 48) + 3 * u;
-    const bool full = (c_lo == 0 && c_hi == 32);
 #pragma unroll
     for (int k = 0; k < 3; k++) {
       if (m[k] == 0u) continue;
