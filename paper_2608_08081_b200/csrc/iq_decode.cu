@@ -188,8 +188,25 @@ __global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode
   const int split = blockIdx.x;
   const int kvh = blockIdx.y / p.head_groups;
   const int hg = blockIdx.y - kvh * p.head_groups;
-  const int b = blockIdx.z;
   const int S = p.splits;
+  // Longest sequences first: CTAs are dispatched in order of blockIdx (z slowest), so slice z of the grid takes the
+  // sequence with the z-th largest length and the short chunks fill the tail of the launch. Every thread ranks one
+  // sequence (ties by index); batches larger than the CTA keep the identity order.
+  int b = blockIdx.z;
+  if (p.batch > 1 && p.batch <= DEC_THREADS) {
+    int* b_slot = reinterpret_cast<int*>(smem + 120);
+    if (tid < p.batch) {
+      const int mine = p.seq_lens[tid];
+      int rank = 0;
+      for (int o = 0; o < p.batch; o++) {
+        const int other = p.seq_lens[o];
+        rank += (other > mine) || (other == mine && o < tid);
+      }
+      if (rank == (int)blockIdx.z) *b_slot = tid;
+    }
+    __syncthreads();
+    b = *b_slot;
+  }
 
   const int len = max(0, min(p.seq_lens[b], p.t_cap));
   const int per = (len + S - 1) / S;
