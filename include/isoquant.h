@@ -150,16 +150,22 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
  *   q              device binary16 [batch][n_q_heads][head_dim], 16-byte aligned; not quantised.
  *   seq_lens_dev   device int32 [batch]: rows 0 .. len-1 of each sequence are attended to (clamped to
  *                  [0, t_cap]); the row appended last is attended to like any other.
- *   num_splits     S >= 1. Sequence b is cut into S consecutive chunks of
- *                  128 * ceil(ceil(len_b / S) / 128) rows; trailing chunks may be empty.
- *   part_acc       device fp32 [batch][n_q_heads][S][head_dim]: sum_j exp(z_j - m) v~_j over the chunk,
+ *   num_splits     S >= 1: partial slots per (sequence, head). The rows of a sequence are covered by at most S
+ *                  consecutive, non-overlapping row ranges (multiples of 128 rows except at the end), one slot per
+ *                  range, in ascending order; which ranges is the library's choice (it balances the launch: every
+ *                  SM takes an equal share of the 128-row blocks of the whole batch).
+ *                  A small S restricts that choice; iq_suggest_splits gives a value that does not.
+ *   part_acc       device fp32 [batch][n_q_heads][S][head_dim]: sum_j exp(z_j - m) v~_j over the slot's rows,
  *                  in the rotated space, natural coordinate order. 16-byte aligned.
  *   part_ml        device fp32 [batch][n_q_heads][S][2] = (m, l): m = max_j z_j, l = sum_j exp(z_j - m),
- *                  z_j = sm_scale * q~ . k~_j. An empty chunk holds (-inf, 0) and acc = 0.
+ *                  z_j = sm_scale * q~ . k~_j. An unused slot holds (-inf, 0) and acc = 0; every slot of every
+ *                  head is written on every call.
  *   part_argmax    device int32 [batch][n_q_heads][S] or NULL: row index attaining m (lowest on ties), -1 if empty.
  *   status_dev     optional (see top).
  * Arithmetic: q~ and the probabilities enter fp16 tensor-core operands, each as a two-term fp16 sum
- * (hi + lo); codebook levels are exact fp16 values; every accumulation is fp32.
+ * (hi + lo); codebook levels are exact fp16 values; every accumulation is fp32. Blocks are handed to the
+ * warps of an SM dynamically, so the order of the fp32 additions -- and with it the last bits of the
+ * result -- can differ between two calls on the same inputs; m and the argmax do not.
  */
 int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook,
                         const void* q, const iq_cache* cache, const int32_t* seq_lens_dev,
@@ -204,7 +210,8 @@ int iq_decode_attention_static(const iq_shape* shape, const float* rot_dev, cons
                                int32_t num_splits, void* out, int32_t out_is_fp16, float* lse_out,
                                uint32_t* status_dev, void* stream);
 
-/* A split count that fills the GPU for this shape when the longest sequence has max_seq_len rows. */
+/* A slot count that leaves the decode kernel free to balance the launch when the longest sequence has
+ * max_seq_len rows (more slots than needed only cost the writing and merging of unused ones). */
 int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len);
 
 #ifdef __cplusplus

@@ -274,10 +274,11 @@ int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len) {
   const int group = shape->n_q_heads / shape->n_kv_heads;
   const long long items = (long long)(shape->batch > 0 ? shape->batch : 1) * shape->n_kv_heads * ((group + iq::DEC_HEADS - 1) / iq::DEC_HEADS);
   const long long slots = (long long)n_sm * iq::decode_ctas_per_sm(shape->head_dim);
-  // About 1.7 CTAs per resident slot: the kernel runs the longest sequences first, so a short second wave is
-  // enough to level the ragged tail, and fewer splits mean fewer per-CTA prologues (measured optimum on B200).
-  long long s = (17 * slots + 10 * items - 1) / (10 * items);
-  const long long cap = (max_seq_len + 511) / 512;         // at least 512 rows (four blocks) per split
+  // The decode kernel gives every SM an equal, contiguous share of the launch's 128-row blocks; an item of nb blocks
+  // then reports to about nb / share + 1 slots. With all sequences at full length share = items * nb / slots; the
+  // factor 1.5 leaves room for batches whose mean length is two thirds of the longest.
+  long long s = (15 * slots + 10 * items - 1) / (10 * items) + 1;
+  const long long cap = (max_seq_len + 255) / 256;         // at least 256 rows (two blocks) per slot
   if (s > cap) s = cap;
   if (s < 1) s = 1;
   if (s > 256) s = 256;

@@ -2,34 +2,37 @@
 // softmax, value accumulation on packed V codes, on the 5th-generation tensor cores (tcgen05) with the
 // dequantised operands resident in tensor memory (TMEM).
 //
-// One CTA of 128 threads per (context split, KV head x head group, sequence); the CTA walks its chunk in
-// blocks of 128 cached rows. Per block:
+// Work decomposition. The 128-row blocks of all (sequence, KV head, head group) items of the launch are laid
+// end to end and every CTA -- one per SM -- takes an equal, contiguous range of that sequence, whatever the length
+// mix of the batch. A range is processed item piece by item piece ("segment"); each segment ends in one partial
+// result (slot) of the item. Inside the CTA, NG groups of 4 compute warps + 1 control warp each run their own
+// tile pipeline and draw the segment's blocks one at a time from a shared-memory counter, so the groups stay
+// busy until the segment is exhausted even though the warp schedulers do not serve them evenly; their partial
+// softmax states are merged in shared memory at the end of the segment.
+//
+// Per block, in group g (thread r of the group = TMEM lane r):
 //   1. thread r dequantises packed K row r (its own 3d/8 bytes from the staged tile) into fp16 and stores it
 //      to TMEM lane r: A_K[128 rows x d].
-//   2. one thread issues tcgen05.mma (M = 128 rows, N = 16, K = 16 per instruction):
+//   2. the control warp issues tcgen05.mma (M = 128 rows, N = 16, K = 16 per instruction):
 //         S[row][n] = sum_i A_K[row][i] * B_Q[n][i],  B_Q = q~ of the <= 8 heads as fp16 hi (n < 8) and lo (n >= 8)
-//   3. every thread reads its row of S back, applies the K scale, joins the block-wide running maximum and
+//   3. every thread reads its row of S back, applies the K scale, joins the group-wide running maximum and
 //      writes its probabilities (times the V scale, again as fp16 hi / lo) into the shared-memory operand
 //      B_P[n][row].
 //   4. thread c dequantises coordinate c of the token-transposed V block (128 codes = one 48-byte row) into
-//      TMEM lane c: A_V[d coords x 128 rows]; one thread issues
-//         O[c][n] = sum_row A_V[c][row] * B_P[n][row]
+//      TMEM lane c: A_V[d coords x 128 rows] (same columns as A_K, once the score MMAs have read them); the
+//      control warp issues   O[c][n] = sum_row A_V[c][row] * B_P[n][row]
 //   5. thread c folds O (hi + lo columns) into its running accumulator for coordinate c.
-// Packed tiles arrive through a 1-D bulk-copy (TMA) pipeline; every wait is bounded.
+// Packed tiles arrive through a 1-D bulk-copy (TMA) pipeline; every mbarrier wait is bounded.
+#include <climits>
+
 #include "iq_common.cuh"
 #include "iq_kernels.h"
 
 namespace iq {
 
-// Tuning knob: 1 = the K and V operand tiles share TMEM columns at d = 128 (4 CTAs per SM, measured fastest),
-// 0 = separate tiles (3 CTAs per SM, the dequantisation of one tile overlaps the MMAs on the other).
-#ifndef IQ_DEC_SHARED128
-#define IQ_DEC_SHARED128 1
-#endif
-constexpr int DEC_COMPUTE_THREADS = 128;  // 4 warps: dequantisation, softmax, accumulation (thread = TMEM lane)
-constexpr int DEC_THREADS = 160;          // + 1 control warp: issues the bulk copies and the MMAs
+constexpr int DEC_GROUP_THREADS = 128;  // 4 warps: dequantisation, softmax, accumulation (thread = TMEM lane)
 constexpr uint32_t DEC_WAIT_LIMIT = 1u << 22;
-constexpr int DEC_HDR_BYTES = 1024;  // barriers, TMEM base, cross-warp scratch
+constexpr int DEC_HDR_BYTES = 4096;    // barriers, TMEM base, work counter, segment and block descriptors, scratch
 constexpr float DEC_MAX_SLACK = 4.0f;  // log2 units a score may exceed the running reference before it is raised
 
 template <int D>
@@ -41,25 +44,31 @@ struct DecLayout {
   static constexpr int VT_BYTES = D * 48;  // token-transposed V block: one 48-byte row (128 codes) per coordinate
   static constexpr int SC_BYTES = DEC_BLOCK_TOKENS * 4;
   static constexpr int STAGE_BYTES = K_BYTES + VT_BYTES + 2 * SC_BYTES;
+  static constexpr int STAGES = 3;
   static constexpr int BQ_BYTES = 16 * D * 2;
   static constexpr int BP_BYTES = 16 * DEC_BLOCK_TOKENS * 2;
-  // TMEM. Separate tiles (d = 128 default): the K tile and the V tile have their own 64 columns each (allocation
-  // 0, 128 columns) and the fp32 results live in a second allocation of 32 columns, so that 3 CTAs fit the SM's
-  // 512 columns and the dequantisation of one tile overlaps the MMAs on the other. Shared tile (d = 256): one
-  // allocation, the K and V tiles share columns (the kernel then waits for the MMAs that read a tile before
-  // overwriting it).
-  static constexpr bool SHARED_A = (D != 128) || (IQ_DEC_SHARED128 != 0);
-  static constexpr int CTAS_PER_SM = (D == 128) ? (SHARED_A ? 4 : 3) : 2;
-  static constexpr int STAGES = (D == 128 && !SHARED_A) ? 4 : 3;
-  static constexpr int SMEM_BYTES = DEC_HDR_BYTES + BQ_BYTES + BP_BYTES + STAGES * STAGE_BYTES;
-  static constexpr int ALLOC0_COLS = SHARED_A ? D : 128;
-  static constexpr int ALLOC1_COLS = SHARED_A ? 0 : 32;
-  static constexpr int AK_COL = 0;
-  static constexpr int AV_COL = SHARED_A ? 0 : 64;
-  static constexpr int S_COL = SHARED_A ? D / 2 : 0;    // in allocation 1 when it exists
-  static constexpr int O_COL = SHARED_A ? D / 2 + 16 : 16;
+  // TMEM columns of one group: the operand tile (K rows, then V coordinates: d fp16 = d/2 columns), 16 columns of
+  // scores, 16 * DJ columns of values. The CTA owns all 512 columns of the SM.
+  static constexpr int GROUP_COLS = D;
+  static constexpr int A_COL = 0;
+  static constexpr int S_COL = D / 2;
+  static constexpr int O_COL = D / 2 + 16;
+  static constexpr int NG = 512 / GROUP_COLS;  // groups per CTA: 4 at d = 128, 2 at d = 256
+  static constexpr int COMPUTE_THREADS = NG * DEC_GROUP_THREADS;
+  static constexpr int THREADS = COMPUTE_THREADS + NG * 32;  // + one control warp per group
+  static constexpr int GROUP_SMEM = BP_BYTES + STAGES * STAGE_BYTES;
+  static constexpr int SMEM_BYTES = DEC_HDR_BYTES + BQ_BYTES + NG * GROUP_SMEM;
+  // header offsets
+  static constexpr int BAR_STRIDE = 96;  // per group: full[3], empty[3], s_bar, o_bar, k_ready, p_ready
+  static constexpr int OFF_TMEM = 384, OFF_NEXT = 388, OFF_SEG = 400, OFF_DESC = 448, OFF_RED = 640, OFF_WALK = 2176;
+  static constexpr int RED_STRIDE = 384;  // per group: 3 x [4 warps][8 heads] words
 };
 static_assert(DEC_BLOCK_TOKENS == 128, "the TMEM operand layout assumes 128-row blocks");
+static_assert(DecLayout<128>::OFF_RED + 4 * DecLayout<128>::RED_STRIDE <= DEC_HDR_BYTES, "header overflow");
+static_assert(DecLayout<128>::O_COL + 16 * DecLayout<128>::DJ <= DecLayout<128>::GROUP_COLS, "TMEM group overflow");
+static_assert(DecLayout<256>::O_COL + 16 * DecLayout<256>::DJ <= DecLayout<256>::GROUP_COLS, "TMEM group overflow");
+static_assert(DecLayout<128>::SMEM_BYTES <= 227 * 1024 && DecLayout<256>::SMEM_BYTES <= 227 * 1024, "shared memory overflow");
+static_assert((DecLayout<128>::THREADS + DecLayout<128>::THREADS / 32) * 4 <= DecLayout<128>::BP_BYTES, "set-up scratch must fit one B_P region");
 
 // ---------------------------------------------------------------------------------------------- tcgen05 wrappers
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -144,14 +153,16 @@ __device__ __forceinline__ bool elect_one() {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Named barrier 1 over the 128 compute threads (the control warp does not take part), with an OR reduction.
-__device__ __forceinline__ bool compute_bar_or(bool pred) {
+// Named barrier `id` over the 128 compute threads of one group, with an OR reduction.
+__device__ __forceinline__ bool group_bar_or(int id, bool pred) {
   uint32_t r;
-  asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbarrier.red.or.pred p, 1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(r) : "r"((uint32_t)pred) : "memory");
+  asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %2, 0;\n\tbarrier.red.or.pred p, %1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(r) : "r"(id), "r"((uint32_t)pred) : "memory");
   return r != 0;
 }
-__device__ __forceinline__ void compute_bar_sync() { asm volatile("barrier.sync 1, 128;" ::: "memory"); }
+// Barrier 0 over the whole CTA, for the places where the control and the compute warps arrive from different code.
+__device__ __forceinline__ void cta_bar_sync() { asm volatile("barrier.sync 0;" ::: "memory"); }
+__device__ __forceinline__ void group_bar_sync(int id) { asm volatile("barrier.sync %0, 128;" ::"r"(id) : "memory"); }
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
@@ -159,121 +170,231 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
+// Segment descriptor in shared memory (written by thread 0 before each segment).
+struct DecSegment {
+  int b, y;          // sequence, item within the sequence (KV head x head group)
+  int blk0, blk1;    // blocks [blk0, blk1) of the item
+  int slot;          // partial slot of the item this segment reports to
+  int len;           // cached rows of the sequence
+  int flags;         // bit 0: blk1 is the end of the item; bit 1: last segment of this CTA
+  int pad;
+};
+
+// Thread 0's position in the CTA's range (kept in shared memory between segments).
+struct DecWalk {
+  int b, y, blk, nb;        // sequence, item within it, block within the item, blocks of sequence b
+  long long left, g, item;  // range mode: blocks to go, launch-wide position; whole-item mode: linear item index
+};
+
 template <int D, bool ARGMAX>
-__global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const DecodeParams p) {
   using L = DecLayout<D>;
   constexpr int DJ = L::DJ;
   constexpr int E = D / 32;
   constexpr int TB = DEC_BLOCK_TOKENS;
   constexpr int NST = L::STAGES;
+  constexpr int NG = L::NG;
   constexpr float LOG2E = 1.4426950408889634f;
   constexpr float LN2 = 0.6931471805599453f;
 
   extern __shared__ __align__(1024) uint8_t smem[];
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem);     // [stages]
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + 64);   // scores ready
-  uint64_t* o_bar = reinterpret_cast<uint64_t*>(smem + 72);   // values ready
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + 80);  // [2] bases of the TMEM allocations
-  uint64_t* k_ready = reinterpret_cast<uint64_t*>(smem + 88);   // K tile in TMEM (128 arrivals)
-  uint64_t* p_ready = reinterpret_cast<uint64_t*>(smem + 96);   // V tile in TMEM + probabilities in smem (128 arrivals)
-  uint64_t* empty_bar = reinterpret_cast<uint64_t*>(smem + 32);  // [stages] staged tile consumed (128 arrivals)
-  float* red = reinterpret_cast<float*>(smem + 128);          // [4 warps][8 heads] cross-warp scratch
-  float* red2 = red + 32;                                     // second scratch (maxima)
-  int* redi = reinterpret_cast<int*>(red2 + 32);              // argmax rows
-  uint8_t* bq = smem + DEC_HDR_BYTES;                         // B_Q: (n, i) MN-major
-  uint8_t* bp = bq + L::BQ_BYTES;                             // B_P: (n, row) MN-major
-  uint8_t* stages = bp + L::BP_BYTES;
-
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int split = blockIdx.x;
-  const int kvh = blockIdx.y / p.head_groups;
-  const int hg = blockIdx.y - kvh * p.head_groups;
+  const bool control = warp >= NG * 4;
+  const int grp = control ? warp - NG * 4 : warp >> 2;  // group of this warp
+  const int gt = tid & (DEC_GROUP_THREADS - 1);         // compute thread within its group = TMEM lane
+  const int bar_id = 1 + grp;                           // named barrier of the group's compute threads
+
+  uint64_t* gbar = reinterpret_cast<uint64_t*>(smem + grp * L::BAR_STRIDE);
+  uint64_t* full_bar = gbar;        // [stages] tile landed (or end marker)
+  uint64_t* empty_bar = gbar + 3;   // [stages] staged tile consumed (128 arrivals)
+  uint64_t* s_bar = gbar + 6;       // scores ready
+  uint64_t* o_bar = gbar + 7;       // values ready
+  uint64_t* k_ready = gbar + 8;     // K tile in TMEM (128 arrivals)
+  uint64_t* p_ready = gbar + 9;     // V tile in TMEM + probabilities in smem (128 arrivals)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_TMEM);
+  int* next_s = reinterpret_cast<int*>(smem + L::OFF_NEXT);            // next block of the open segment
+  DecSegment* seg_s = reinterpret_cast<DecSegment*>(smem + L::OFF_SEG);
+  int2* desc = reinterpret_cast<int2*>(smem + L::OFF_DESC) + grp * NST;  // [stages] (first row, rows | end marker) of the staged block
+  float* red = reinterpret_cast<float*>(smem + L::OFF_RED + grp * L::RED_STRIDE);  // [4 warps][8 heads] cross-warp scratch
+  float* red2 = red + 32;
+  int* redi = reinterpret_cast<int*>(red2 + 32);
+  uint8_t* bq = smem + DEC_HDR_BYTES;                                  // B_Q: (n, i) MN-major, shared by the groups
+  uint8_t* bp = bq + L::BQ_BYTES + grp * L::GROUP_SMEM;                // B_P: (n, row) MN-major
+  uint8_t* stages = bp + L::BP_BYTES;
+  // Set-up scratch in group 0's B_P region: [THREADS] blocks per slice of the batch, then the per-warp maxima. It is
+  // last read before the first segment opens.
+  int* scan_s = reinterpret_cast<int*>(bq + L::BQ_BYTES);
+
   const int S = p.splits;
-  // Longest sequences first: CTAs are dispatched in order of blockIdx (z slowest), so slice z of the grid takes the
-  // sequence with the z-th largest length and the short chunks fill the tail of the launch. Every thread ranks one
-  // sequence (ties by index); batches larger than the CTA keep the identity order.
-  int b = blockIdx.z;
-  if (p.batch > 1 && p.batch <= DEC_THREADS) {
-    int* b_slot = reinterpret_cast<int*>(smem + 120);
-    if (tid < p.batch) {
-      const int mine = p.seq_lens[tid];
-      int rank = 0;
-      for (int o = 0; o < p.batch; o++) {
-        const int other = p.seq_lens[o];
-        rank += (other > mine) || (other == mine && o < tid);
-      }
-      if (rank == (int)blockIdx.z) *b_slot = tid;
+  const int B = p.batch;
+  const int ips = p.n_kv_heads * p.head_groups;  // items per sequence
+  auto len_of = [&](int b) { return max(0, min(p.seq_lens[b], p.t_cap)); };
+  auto nb_of = [&](int b) { return (len_of(b) + TB - 1) / TB; };
+  // Unused partial slots [slot_lo, S) of the heads [h_lo, h_lo + n_h) of sequence b: (m, l) = (-inf, 0), acc = 0.
+  auto fill_slots = [&](int b, int h_lo, int n_h, int slot_lo, int n_threads, int t) {
+    const int n_slots = S - slot_lo;
+    if (n_slots <= 0) return;
+    for (int idx = t; idx < n_h * n_slots * D; idx += n_threads) {
+      const int c = idx % D, sl = (idx / D) % n_slots, h = idx / (D * n_slots);
+      p.part_acc[(((size_t)b * p.n_q_heads + h_lo + h) * S + slot_lo + sl) * D + c] = 0.f;
     }
-    __syncthreads();
-    b = *b_slot;
-  }
-
-  const int len = max(0, min(p.seq_lens[b], p.t_cap));
-  const int per = (len + S - 1) / S;
-  const int chunk = ((per + TB - 1) / TB) * TB;
-  const int start = split * chunk;
-  const int end = min(len, start + chunk);
-  const int h0 = kvh * p.group + hg * DEC_HEADS;
-  const int nh = min(DEC_HEADS, p.group - hg * DEC_HEADS);
-
-  if (start >= end) {  // empty chunk: (m, l) = (-inf, 0), acc = 0
-    for (int idx = tid; idx < nh * D; idx += DEC_THREADS) {
-      const int head = idx / D, c = idx - head * D;
-      p.part_acc[(((size_t)b * p.n_q_heads + h0 + head) * S + split) * D + c] = 0.f;
-    }
-    if (tid < nh) {
-      const size_t o = ((size_t)b * p.n_q_heads + h0 + tid) * S + split;
+    for (int idx = t; idx < n_h * n_slots; idx += n_threads) {
+      const int sl = idx % n_slots, h = idx / n_slots;
+      const size_t o = ((size_t)b * p.n_q_heads + h_lo + h) * S + slot_lo + sl;
       p.part_ml[2 * o] = -INFINITY;
       p.part_ml[2 * o + 1] = 0.f;
       if (ARGMAX) p.part_argmax[o] = -1;
     }
-    return;
-  }
-
-  // ---------------------------------------------------------------- set-up: barriers, TMEM, tile pipeline
-  const size_t slab = ((size_t)b * p.n_kv_heads + kvh) * (size_t)p.t_cap;  // row index of this (sequence, KV head)
-  const int nblk = (end - start + TB - 1) / TB;
-  const bool control = (warp == 4);
-  auto issue = [&](int blk) {  // elected lane of the control warp only
-    const int st = blk % NST;
-    const int r0 = start + blk * TB;
-    const int n = min(TB, end - r0);
-    const int n4 = (n + 3) & ~3;
-    uint8_t* sp = stages + st * L::STAGE_BYTES;
-    mbar_expect_tx(&full_bar[st], (uint32_t)(n * L::ROWB + L::VT_BYTES + 2 * n4 * 4));
-    bulk_g2s(sp, p.k_codes + (slab + r0) * L::ROWB, (uint32_t)(n * L::ROWB), &full_bar[st]);
-    bulk_g2s(sp + L::K_BYTES, p.v_codes + (slab + r0) * L::ROWB, (uint32_t)L::VT_BYTES, &full_bar[st]);  // whole 128-row V block
-    bulk_g2s(sp + L::K_BYTES + L::VT_BYTES, p.k_scales + slab + r0, (uint32_t)(n4 * 4), &full_bar[st]);
-    bulk_g2s(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES, p.v_scales + slab + r0, (uint32_t)(n4 * 4), &full_bar[st]);
   };
-  if (control && elect_one()) {
+
+  // ---------------------------------------------------------------- the block sequence of the launch and this CTA's range
+  const int per_thread = (B + L::THREADS - 1) / L::THREADS;
+  {
+    int sum = 0, mx = 0;
+    for (int b = tid * per_thread; b < min(B, (tid + 1) * per_thread); b++) {
+      const int n = nb_of(b);
+      sum += n;
+      mx = max(mx, n);
+    }
+    scan_s[tid] = sum;
 #pragma unroll
-    for (int st = 0; st < NST; st++) { mbar_init(&full_bar[st], 1); mbar_init(&empty_bar[st], DEC_COMPUTE_THREADS); }
+    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(FULL, mx, o));
+    if (lane == 0) scan_s[L::THREADS + warp] = mx;
+  }
+  // sequences without cached rows belong to no range: CTA c defines the partial slots of sequences c, c + grid, ...
+  for (int b = blockIdx.x; b < B; b += gridDim.x)
+    if (len_of(b) == 0) fill_slots(b, 0, p.n_q_heads, 0, L::THREADS, tid);
+  __syncthreads();
+  long long n_total;
+  int nb_max = 0;
+  {
+    int v = 0;
+    for (int i = lane; i < L::THREADS; i += 32) v += scan_s[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+    n_total = (long long)v * ips;
+    for (int i = 0; i < L::THREADS / 32; i++) nb_max = max(nb_max, scan_s[L::THREADS + i]);
+  }
+  const bool whole_items = (S == 1);  // one slot per head: an item cannot be shared between CTAs
+  long long per = (n_total + gridDim.x - 1) / gridDim.x;
+  if (!whole_items) per = max(per, (long long)((nb_max - 1) / (S - 1) + 1));  // an item then spans at most S ranges
+  per = max(per, 1ll);
+  const long long g0 = (long long)blockIdx.x * per;
+  if (n_total == 0 || (!whole_items && g0 >= n_total) || (whole_items && (long long)blockIdx.x >= (long long)B * ips)) return;
+
+  // Thread 0 walks the range segment by segment; the walk lives in shared memory between segments. Range mode:
+  // position (b, y, blk) and `left` blocks to go; whole-item mode: items blockIdx.x, blockIdx.x + grid, ... with rows.
+  DecWalk* walk_s = reinterpret_cast<DecWalk*>(smem + L::OFF_WALK);
+  auto next_item_with_rows = [&](DecWalk& w) {  // whole-item mode: settle on the next item that has rows, or b = B
+    for (;; w.item += gridDim.x) {
+      if (w.item >= (long long)B * ips) { w.b = B; w.nb = 0; return; }
+      w.b = (int)(w.item / ips);
+      w.y = (int)(w.item % ips);
+      w.nb = nb_of(w.b);
+      w.blk = 0;
+      if (w.nb > 0) return;
+    }
+  };
+  {
+    DecWalk w = {0, 0, 0, 0, 0, g0, (long long)blockIdx.x};
+    if (whole_items) {
+      next_item_with_rows(w);  // every thread: the CTA leaves together when none of its items has rows
+      if (w.b >= B) return;
+    } else if (tid == 0) {
+      long long before = 0;  // blocks (per item column) of the sequences before w.b
+      int t = 0;
+      while (t < L::THREADS - 1 && (before + scan_s[t]) * ips <= g0) { before += scan_s[t]; t++; }
+      w.b = t * per_thread;
+      w.nb = (w.b < B) ? nb_of(w.b) : 0;
+      while (w.b < B - 1 && (before + w.nb) * ips <= g0) { before += w.nb; w.b++; w.nb = nb_of(w.b); }
+      const long long r = g0 - before * ips;  // offset inside sequence b's blocks (nb per item, ips items)
+      w.y = (int)(r / w.nb);
+      w.blk = (int)(r % w.nb);
+      w.left = min(per, n_total - g0);
+    }
+    if (tid == 0) *walk_s = w;
+  }
+  // thread 0: describe the next segment in seg_s, open its block counter, advance the walk
+  auto open_segment = [&]() {
+    DecWalk w = *walk_s;
+    const int take = whole_items ? w.nb : (int)min((long long)(w.nb - w.blk), w.left);
+    DecSegment sg;
+    sg.b = w.b;
+    sg.y = w.y;
+    sg.blk0 = w.blk;
+    sg.blk1 = w.blk + take;
+    sg.slot = whole_items ? 0 : (int)((long long)blockIdx.x - (w.g - w.blk) / per);
+    sg.len = len_of(w.b);
+    const bool item_end = (sg.blk1 == w.nb);
+    w.g += take;
+    w.left -= take;
+    bool cta_end;
+    if (whole_items) {
+      w.item += gridDim.x;
+      next_item_with_rows(w);
+      cta_end = (w.b >= B);
+    } else {
+      if (item_end) {
+        w.blk = 0;
+        if (++w.y == ips) {
+          w.y = 0;
+          do { w.b++; w.nb = (w.b < B) ? nb_of(w.b) : 0; } while (w.b < B && w.nb == 0);
+        }
+      } else {
+        w.blk = sg.blk1;
+      }
+      cta_end = (w.left <= 0) || (w.b >= B);
+    }
+    sg.flags = (item_end ? 1 : 0) | (cta_end ? 2 : 0);
+    sg.pad = 0;
+    *seg_s = sg;
+    *next_s = sg.blk0;
+    *walk_s = w;
+  };
+
+  // ---------------------------------------------------------------- set-up: barriers, TMEM
+  if (control && elect_one()) {  // every control warp initialises the barriers of its group
+#pragma unroll
+    for (int st = 0; st < NST; st++) { mbar_init(&full_bar[st], 1); mbar_init(&empty_bar[st], DEC_GROUP_THREADS); }
     mbar_init(s_bar, 1);
     mbar_init(o_bar, 1);
-    mbar_init(k_ready, DEC_COMPUTE_THREADS);
-    mbar_init(p_ready, DEC_COMPUTE_THREADS);
+    mbar_init(k_ready, DEC_GROUP_THREADS);
+    mbar_init(p_ready, DEC_GROUP_THREADS);
     fence_mbar_init();
     fence_proxy_async();
-    for (int blk = 0; blk < NST && blk < nblk; blk++) issue(blk);
   }
-  if (control) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(L::ALLOC0_COLS));
-    if (L::ALLOC1_COLS > 0)
-      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot + 1)), "r"(L::ALLOC1_COLS));
+  if (warp == NG * 4) {  // the whole tensor memory of the SM: one CTA per SM
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
   }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot[0];
+  const uint32_t tmem_g = tmem_base + (uint32_t)(grp * L::GROUP_COLS);        // this group's columns
+  const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;                // this warp's 32 TMEM lanes
+  bool failed = false;  // a bounded wait gave up; assumed to hit all threads of a group alike (they wait on the same barriers)
+  int it = 0;           // staged slots of this group consumed so far (tile pipeline phases), end markers included
+  int nbk = 0;          // blocks this group has processed (phases of k_ready, s_bar, p_ready, o_bar)
 
-  // ---------------------------------------------------------------- d1: q~ = R q, written as the operand B_Q
-  if (!control) {
-    float M[E / 4][4][4];
-    const float* qb = p.rot + ((size_t)kvh * (D / 4) + (size_t)lane * (E / 4)) * 8;
-#pragma unroll
-    for (int j = 0; j < E / 4; j++) so4_matrix<float>(qb + 8 * j, M[j]);
-    const float inv_root_d = rsqrtf((float)D);
-    for (int hh = warp; hh < DEC_HEADS; hh += 4) {
+  for (;;) {
+    // ================================================================ one segment: blocks [blk0, blk1) of one item
+    if (tid == 0) open_segment();
+    __syncthreads();  // segment published; the previous segment's merge has finished reading the staging buffers
+    if (!control && warp < DEC_HEADS) {
+      // ---- d1: q~ = R q of head `warp`, written as the operand B_Q (shared by the groups)
+      const int b = seg_s->b;
+      const int kvh = seg_s->y / p.head_groups;
+      const int hg = seg_s->y - kvh * p.head_groups;
+      const int h0 = kvh * p.group + hg * DEC_HEADS;
+      const int nh = min(DEC_HEADS, p.group - hg * DEC_HEADS);
+      const int hh = warp;
       float v[E];
       if (hh < nh) {
+        float M[E / 4][4][4];
+        const float* qb = p.rot + ((size_t)kvh * (D / 4) + (size_t)lane * (E / 4)) * 8;
+#pragma unroll
+        for (int j = 0; j < E / 4; j++) so4_matrix<float>(qb + 8 * j, M[j]);
         const __half* src = p.q + ((size_t)b * p.n_q_heads + h0 + hh) * D + lane * E;
 #pragma unroll
         for (int e = 0; e < E; e++) v[e] = __half2float(src[e]);
@@ -283,6 +404,7 @@ __global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode
 #pragma unroll
         for (int e = 0; e < E; e++) v[e] = 0.f;
       }
+      const float inv_root_d = rsqrtf((float)D);
 #pragma unroll
       for (int e = 0; e < E; e++) {
         const float x = v[e] * inv_root_d;
@@ -290,299 +412,361 @@ __global__ void __launch_bounds__(DEC_THREADS, DecLayout<D>::CTAS_PER_SM) decode
         const __half xl = __float2half_rn(x - __half2float(xh));
         const int i = lane * E + e;  // contraction index = rotated coordinate
         const int off = (i & 7) * 16 + (i >> 3) * 128;
-        *reinterpret_cast<__half*>(bq + (hh & 7) * 2 + off) = xh;                  // n = head (hi part)
-        *reinterpret_cast<__half*>(bq + (hh & 7) * 2 + (D / 8) * 128 + off) = xl;  // n = 8 + head (lo part)
+        *reinterpret_cast<__half*>(bq + hh * 2 + off) = xh;                  // n = head (hi part)
+        *reinterpret_cast<__half*>(bq + hh * 2 + (D / 8) * 128 + off) = xl;  // n = 8 + head (lo part)
       }
+      fence_proxy_async();  // B_Q is written through the generic proxy and read by the tensor core through the async proxy
     }
-  }
-  fence_proxy_async();  // B_Q was written through the generic proxy, the tensor core reads it through the async proxy
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_a = tmem_slot[0];
-  const uint32_t tmem_r = (L::ALLOC1_COLS > 0) ? tmem_slot[1] : tmem_slot[0];  // base of the fp32 result columns
-  const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;  // this warp's 32 TMEM lanes
-
-  float acc[DJ][8];  // thread c: coordinates c (+128), 8 heads
-#pragma unroll
-  for (int j = 0; j < DJ; j++)
-#pragma unroll
-    for (int h = 0; h < 8; h++) acc[j][h] = 0.f;
-  float m_run[8], l_run[8], best_v[8], alpha[8];
-  int best_i[8];
-#pragma unroll
-  for (int h = 0; h < 8; h++) { m_run[h] = -INFINITY; l_run[h] = 0.f; best_v[h] = -INFINITY; best_i[h] = -1; alpha[h] = 1.f; }
-  bool failed = false;
-
-  if (control) {
-    // ================================================================ control warp: issues MMAs and tile refills.
-    // All 32 lanes run the loop and the waits; an elected lane issues.
-    const uint32_t bq_addr = smem_u32(bq), bp_addr = smem_u32(bp);
-    for (int blk = 0; blk < nblk; blk++) {
-      // scores of block blk: S = A_K * B_Q^T once all 128 rows are in TMEM
-      if (!failed) failed = !mbar_wait_bounded(k_ready, (uint32_t)blk & 1u, DEC_WAIT_LIMIT);
-      tc_fence_after();
-      if (elect_one()) {
-#pragma unroll
-        for (int kk = 0; kk < D / 16; kk++)
-          tc_mma_f16(tmem_r + L::S_COL, tmem_a + L::AK_COL + 8 * kk, smem_desc_mn(bq_addr + kk * 256, 128, (D / 8) * 128), DEC_IDESC, kk > 0);
-        tc_commit(s_bar);
-      }
-      __syncwarp();
-      // values of block blk: O = A_V * B_P^T once the V tile is in TMEM and the probabilities are in shared memory
-      if (!failed) failed = !mbar_wait_bounded(p_ready, (uint32_t)blk & 1u, DEC_WAIT_LIMIT);
-      tc_fence_after();
-      if (elect_one()) {
-#pragma unroll
-        for (int j = 0; j < DJ; j++)
-#pragma unroll
-          for (int kk = 0; kk < TB / 16; kk++)
-            tc_mma_f16(tmem_r + L::O_COL + 16 * j, tmem_a + L::AV_COL + 64 * j + 8 * kk,
-                       smem_desc_mn(bp_addr + kk * 256, 128, (TB / 8) * 128), DEC_IDESC, kk > 0);
-        tc_commit(o_bar);
-      }
-      __syncwarp();
-      // the compute threads released the stage when they signalled p_ready: refill it
-      if (blk + NST < nblk) {
-        if (!failed) failed = !mbar_wait_bounded(&empty_bar[blk % NST], (uint32_t)(blk / NST) & 1u, DEC_WAIT_LIMIT);
-        if (elect_one()) {
-          fence_proxy_async();
-          issue(blk + NST);
+    // (the control warps stage their first tiles below before they join the barrier that completes B_Q)
+    if (control) {
+      // ================================================================ control warp of group grp: fetches blocks, issues MMAs.
+      // All 32 lanes run the loop and the waits; an elected lane issues.
+      const int blk1 = seg_s->blk1, len = seg_s->len;
+      const size_t slab = ((size_t)seg_s->b * p.n_kv_heads + (seg_s->y / p.head_groups)) * (size_t)p.t_cap;
+      const uint32_t bq_addr = smem_u32(bq), bp_addr = smem_u32(bp);
+      bool ended = false;   // the segment's counter ran out and the end marker has been staged
+      int it_issue = it;    // slots staged so far (the pipeline is empty between segments)
+      auto stage_next = [&]() {  // draw the next block of the segment into slot it_issue, or the end marker
+        const int st = it_issue % NST;
+        if (it_issue >= NST && !failed)  // the slot's previous occupant has been consumed
+          failed = !mbar_wait_bounded(&empty_bar[st], (uint32_t)(it_issue / NST - 1) & 1u, DEC_WAIT_LIMIT);
+        int j = 0;
+        if (lane == 0) j = atomicAdd(next_s, 1);
+        j = __shfl_sync(FULL, j, 0);
+        if (j < blk1) {
+          const int r0 = j * TB;
+          const int n = min(TB, len - r0);
+          if (elect_one()) {
+            desc[st] = make_int2(r0, n);
+            const int n4 = (n + 3) & ~3;
+            uint8_t* sp = stages + st * L::STAGE_BYTES;
+            fence_proxy_async();
+            mbar_expect_tx(&full_bar[st], (uint32_t)(n * L::ROWB + L::VT_BYTES + 2 * n4 * 4));  // also publishes desc[st]
+            bulk_g2s(sp, p.k_codes + (slab + r0) * L::ROWB, (uint32_t)(n * L::ROWB), &full_bar[st]);
+            bulk_g2s(sp + L::K_BYTES, p.v_codes + (slab + r0) * L::ROWB, (uint32_t)L::VT_BYTES, &full_bar[st]);  // whole 128-row V block
+            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES, p.k_scales + slab + r0, (uint32_t)(n4 * 4), &full_bar[st]);
+            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES, p.v_scales + slab + r0, (uint32_t)(n4 * 4), &full_bar[st]);
+          }
+        } else {
+          ended = true;
+          if (elect_one()) {
+            desc[st] = make_int2(0, -1);  // end marker: no tile, the group closes its part of the segment
+            mbar_arrive(&full_bar[st]);
+          }
         }
         __syncwarp();
+        it_issue++;
+      };
+      while (!ended && it_issue - it < NST) stage_next();  // tiles in flight while q~ is being rotated
+      cta_bar_sync();  // B_Q complete
+      for (;;) {
+        if (it == it_issue) stage_next();  // nothing staged ahead (end of a segment): draw now
+        if (ended && it == it_issue - 1) { it++; break; }  // slot `it` holds the end marker
+        // scores of the block in slot `it`: S = A_K * B_Q^T once all 128 rows are in TMEM
+        if (!failed) failed = !mbar_wait_bounded(k_ready, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
+        tc_fence_after();
+        if (elect_one()) {
+#pragma unroll
+          for (int kk = 0; kk < D / 16; kk++)
+            tc_mma_f16(tmem_g + L::S_COL, tmem_g + L::A_COL + 8 * kk, smem_desc_mn(bq_addr + kk * 256, 128, (D / 8) * 128), DEC_IDESC, kk > 0);
+          tc_commit(s_bar);
+        }
+        __syncwarp();
+        // values: O = A_V * B_P^T once the V tile is in TMEM and the probabilities are in shared memory
+        if (!failed) failed = !mbar_wait_bounded(p_ready, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
+        tc_fence_after();
+        if (elect_one()) {
+#pragma unroll
+          for (int j = 0; j < DJ; j++)
+#pragma unroll
+            for (int kk = 0; kk < TB / 16; kk++)
+              tc_mma_f16(tmem_g + L::O_COL + 16 * j, tmem_g + L::A_COL + 64 * j + 8 * kk,
+                         smem_desc_mn(bp_addr + kk * 256, 128, (TB / 8) * 128), DEC_IDESC, kk > 0);
+          tc_commit(o_bar);
+        }
+        __syncwarp();
+        it++;
+        nbk++;
+        // the compute threads released the slot when they signalled p_ready
+        if (!ended) stage_next();
       }
     }
-  } else {
-    // ================================================================ compute warps
-    const uint32_t lut_lo0 = p.lut_lo[0], lut_lo1 = p.lut_lo[1], lut_hi0 = p.lut_hi[0], lut_hi1 = p.lut_hi[1];
-    const float kfac = p.sm_scale * LOG2E * rsqrtf((float)D);  // scores in log2 units: z2 = S_raw * scale_K * kfac
-    const float vfac = rsqrtf((float)D);
+    float* gacc = reinterpret_cast<float*>(stages);                 // group partial for the merge: acc [DJ][8][128]
+    float* gml = gacc + DJ * 8 * DEC_GROUP_THREADS;                 // then per head: reference, l, exact maximum, its row
+    if (!control) {
+      cta_bar_sync();  // B_Q complete
+      // ================================================================ compute warps of group grp
+      const uint32_t lut_lo0 = p.lut_lo[0], lut_lo1 = p.lut_lo[1], lut_hi0 = p.lut_hi[0], lut_hi1 = p.lut_hi[1];
+      const float kfac = p.sm_scale * LOG2E * rsqrtf((float)D);  // scores in log2 units: z2 = S_raw * scale_K * kfac
+      const float vfac = rsqrtf((float)D);
+      float acc[DJ][8];  // thread c: coordinates c (+128), 8 heads
+      float m_run[8], l_run[8], best_v[8];
+      int best_i[8];
+#pragma unroll
+      for (int j = 0; j < DJ; j++)
+#pragma unroll
+        for (int h = 0; h < 8; h++) acc[j][h] = 0.f;
+#pragma unroll
+      for (int h = 0; h < 8; h++) { m_run[h] = -INFINITY; l_run[h] = 0.f; best_v[h] = -INFINITY; best_i[h] = -1; }
 
-    // K row tid of the staged tile -> TMEM lane tid (A_K), then signal the control warp.
-    auto k_phase = [&](int blk) {
-      const uint8_t* sp = stages + (blk % NST) * L::STAGE_BYTES;
-      if (!failed) failed = !mbar_wait_bounded(&full_bar[blk % NST], (uint32_t)(blk / NST) & 1u, DEC_WAIT_LIMIT);
-      uint32_t w[L::WPR];
-      const uint4* krow = reinterpret_cast<const uint4*>(sp + tid * L::ROWB);
-#pragma unroll
-      for (int i = 0; i < L::WPR / 4; i++) {
-        const uint4 t4 = krow[i];
-        w[4 * i] = t4.x; w[4 * i + 1] = t4.y; w[4 * i + 2] = t4.z; w[4 * i + 3] = t4.w;
-      }
-#pragma unroll
-      for (int u = 0; u < 4 * DJ; u++) {
-        uint32_t f[16];
-        dequant_unit(w[3 * u], w[3 * u + 1], w[3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);
-        tc_st16(tmem_a + lane_sel + L::AK_COL + 16 * u, f);
-      }
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(k_ready);
-    };
-    // Fold the value product of block `blk` (ready on o_bar) into the running accumulator.
-    auto fold = [&](int blk) {
-      if (!failed) failed = !mbar_wait_bounded(o_bar, (uint32_t)blk & 1u, DEC_WAIT_LIMIT);
-      tc_fence_after();
-#pragma unroll
-      for (int j = 0; j < DJ; j++) {
-        float o[16];
-        tc_ld16(tmem_r + lane_sel + L::O_COL + 16 * j, o);
-#pragma unroll
-        for (int h = 0; h < 8; h++) acc[j][h] = acc[j][h] * alpha[h] + (o[h] + o[8 + h]);
-      }
-      tc_fence_before();
-    };
+      for (;;) {
+        if (failed) break;
+        const int st = it % NST;
+        const uint8_t* sp = stages + st * L::STAGE_BYTES;
+        failed = !mbar_wait_bounded(&full_bar[st], (uint32_t)(it / NST) & 1u, DEC_WAIT_LIMIT);
+        const int2 dsc = desc[st];
+        if (dsc.y < 0) {  // end marker: the segment has no more blocks for this group
+          mbar_arrive(&empty_bar[st]);
+          it++;
+          break;
+        }
+        const int r0 = dsc.x, n = dsc.y;
 
-    k_phase(0);
-    bool folded = true;  // is the value product of the previous block already in acc?
-    for (int blk = 0; blk < nblk; blk++) {
-      const uint8_t* sp = stages + (blk % NST) * L::STAGE_BYTES;
-      const int r0 = start + blk * TB;
-      const int n = min(TB, end - r0);
-      if (L::SHARED_A) {  // the score MMAs read the tile that the V dequantisation is about to overwrite
-        if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)blk & 1u, DEC_WAIT_LIMIT);
-      }
-      if (!folded) { fold(blk - 1); folded = true; }  // also: the value MMAs of the previous block have released A_V and B_P
+        // ---- K row gt of the staged tile -> TMEM lane gt (A_K), then signal the control warp
+        {
+          uint32_t w[L::WPR];
+          const uint4* krow = reinterpret_cast<const uint4*>(sp + gt * L::ROWB);
+#pragma unroll
+          for (int i = 0; i < L::WPR / 4; i++) {
+            const uint4 t4 = krow[i];
+            w[4 * i] = t4.x; w[4 * i + 1] = t4.y; w[4 * i + 2] = t4.z; w[4 * i + 3] = t4.w;
+          }
+#pragma unroll
+          for (int u = 0; u < 4 * DJ; u++) {
+            uint32_t f[16];
+            dequant_unit(w[3 * u], w[3 * u + 1], w[3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);
+            tc_st16(tmem_g + lane_sel + L::A_COL + 16 * u, f);
+          }
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(k_ready);
+        }
+        // the score MMAs read the tile that the V dequantisation is about to overwrite
+        if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
 
-      // ---- V coordinate tid (+128) of this block -> TMEM lane tid (A_V), while the score MMAs run
+        // ---- V coordinate gt (+128) of this block -> TMEM lane gt (A_V)
 #pragma unroll
-      for (int j = 0; j < DJ; j++) {
-        const uint4* vrow = reinterpret_cast<const uint4*>(sp + L::K_BYTES + (tid + 128 * j) * 48);
-        uint32_t w[12];
+        for (int j = 0; j < DJ; j++) {
+          const uint4* vrow = reinterpret_cast<const uint4*>(sp + L::K_BYTES + (gt + 128 * j) * 48);
+          uint32_t wd[12];
 #pragma unroll
-        for (int i = 0; i < 3; i++) {
-          const uint4 t4 = vrow[i];
-          w[4 * i] = t4.x; w[4 * i + 1] = t4.y; w[4 * i + 2] = t4.z; w[4 * i + 3] = t4.w;
+          for (int i = 0; i < 3; i++) {
+            const uint4 t4 = vrow[i];
+            wd[4 * i] = t4.x; wd[4 * i + 1] = t4.y; wd[4 * i + 2] = t4.z; wd[4 * i + 3] = t4.w;
+          }
+#pragma unroll
+          for (int u = 0; u < 4; u++) {
+            uint32_t f[16];
+            dequant_unit(wd[3 * u], wd[3 * u + 1], wd[3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);
+            tc_st16(tmem_g + lane_sel + L::A_COL + 64 * j + 16 * u, f);
+          }
         }
-#pragma unroll
-        for (int u = 0; u < 4; u++) {
-          uint32_t f[16];
-          dequant_unit(w[3 * u], w[3 * u + 1], w[3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);
-          tc_st16(tmem_a + lane_sel + L::AV_COL + 64 * j + 16 * u, f);
-        }
-      }
-      const float ksc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES)[tid];
-      const float vsc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES)[tid];
+        const float ksc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES)[gt];
+        const float vsc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES)[gt];
 
-      // ---- online softmax (log2 units); thread tid owns row r0 + tid, all 8 heads
-      if (!L::SHARED_A) {
-        if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)blk & 1u, DEC_WAIT_LIMIT);
-      }
-      tc_fence_after();
-      float s[8];
-      {
-        float raw[16];
-        tc_ld16(tmem_r + lane_sel + L::S_COL, raw);
-        const bool valid = tid < n;  // rows >= n of the last block hold stale bytes
-        const float kf = valid ? ksc * kfac : 0.f;
+        // ---- online softmax (log2 units); thread gt owns row r0 + gt, all 8 heads
+        tc_fence_after();
+        float s[8];
+        {
+          float raw[16];
+          tc_ld16(tmem_g + lane_sel + L::S_COL, raw);
+          const bool valid = gt < n;  // rows >= n of the last block hold stale bytes
+          const float kf = valid ? ksc * kfac : 0.f;
 #pragma unroll
-        for (int h = 0; h < 8; h++) s[h] = valid ? (raw[h] + raw[8 + h]) * kf : -INFINITY;
-      }
-#pragma unroll
-      for (int h = 0; h < 8; h++) {  // exact maximum seen by this thread (the partial's m) and, optionally, its row
-        if (ARGMAX) {
-          if (s[h] > best_v[h]) { best_v[h] = s[h]; best_i[h] = r0 + tid; }
-        } else {
-          best_v[h] = fmaxf(best_v[h], s[h]);
+          for (int h = 0; h < 8; h++) s[h] = valid ? (raw[h] + raw[8 + h]) * kf : -INFINITY;
         }
+#pragma unroll
+        for (int h = 0; h < 8; h++) {  // exact maximum seen by this thread (the partial's m) and, optionally, its row
+          if (ARGMAX) {
+            if (s[h] > best_v[h]) { best_v[h] = s[h]; best_i[h] = r0 + gt; }  // a group sees its blocks in ascending order
+          } else {
+            best_v[h] = fmaxf(best_v[h], s[h]);
+          }
+        }
+        // The running reference m_run is raised only when some score of the block exceeds it by more than
+        // DEC_MAX_SLACK (log2 units): exp2(s - m_run) then stays below 2^DEC_MAX_SLACK and nothing has to be
+        // exchanged between the warps in the common case (one barrier with an OR reduction).
+        bool exceed = false;
+#pragma unroll
+        for (int h = 0; h < 8; h++) exceed |= (s[h] - m_run[h] > DEC_MAX_SLACK);
+        if (group_bar_or(bar_id, exceed)) {
+#pragma unroll
+          for (int h = 0; h < 8; h++) {
+            const float wm = warp_max(s[h]);
+            if (lane == h) red[(warp & 3) * 8 + h] = wm;
+          }
+          group_bar_sync(bar_id);
+#pragma unroll
+          for (int h = 0; h < 8; h++) {
+            const float bm = fmaxf(fmaxf(red[h], red[8 + h]), fmaxf(red[16 + h], red[24 + h]));
+            const float mn = fmaxf(m_run[h], bm);
+            const float alpha = ex2f(m_run[h] - mn);  // the accumulator holds the blocks before this one: rescale it now
+            m_run[h] = mn;
+            l_run[h] *= alpha;
+#pragma unroll
+            for (int j = 0; j < DJ; j++) acc[j][h] *= alpha;
+          }
+        }
+        {
+          const float vf = (gt < n) ? vsc * vfac : 0.f;
+          float wv[8];
+#pragma unroll
+          for (int h = 0; h < 8; h++) {
+            const float pr = ex2f(s[h] - m_run[h]);
+            l_run[h] += pr;
+            wv[h] = pr * vf;
+          }
+          // probabilities (times scale_V / sqrt(d)) as fp16 hi + lo: B_P[n][row], n = head (hi) or 8 + head (lo)
+          uint32_t hp[4], lp[4];
+#pragma unroll
+          for (int h2 = 0; h2 < 4; h2++) {
+            const uint32_t hpk = pack_half2(wv[2 * h2], wv[2 * h2 + 1]);
+            const float2 back = __half22float2(*reinterpret_cast<const __half2*>(&hpk));
+            hp[h2] = hpk;
+            lp[h2] = pack_half2(wv[2 * h2] - back.x, wv[2 * h2 + 1] - back.y);
+          }
+          const int off = (gt & 7) * 16 + (gt >> 3) * 128;
+          *reinterpret_cast<uint4*>(bp + off) = make_uint4(hp[0], hp[1], hp[2], hp[3]);
+          *reinterpret_cast<uint4*>(bp + (TB / 8) * 128 + off) = make_uint4(lp[0], lp[1], lp[2], lp[3]);
+          fence_proxy_async();
+        }
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(p_ready);          // V tile in TMEM, probabilities in shared memory
+        mbar_arrive(&empty_bar[st]);   // this thread is done with the staged tile
+
+        // ---- fold the value product into the running accumulator (the value MMAs also release the operand tile)
+        if (!failed) failed = !mbar_wait_bounded(o_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
+        tc_fence_after();
+#pragma unroll
+        for (int j = 0; j < DJ; j++) {
+          float o[16];
+          tc_ld16(tmem_g + lane_sel + L::O_COL + 16 * j, o);
+#pragma unroll
+          for (int h = 0; h < 8; h++) acc[j][h] += o[h] + o[8 + h];
+        }
+        tc_fence_before();
+        it++;
+        nbk++;
       }
-      // The running reference m_run is raised only when some score of the block exceeds it by more than
-      // DEC_MAX_SLACK (log2 units): exp2(s - m_run) then stays below 2^DEC_MAX_SLACK and nothing has to be
-      // exchanged between the warps in the common case (one barrier with an OR reduction).
-      bool exceed = false;
+
+      // ---- close the group's part of the segment: reduce l and the exact maximum (and argmax) over the 128 rows and
+      // leave the group partial in the group's (drained) staging buffer for the merge
 #pragma unroll
-      for (int h = 0; h < 8; h++) exceed |= (s[h] - m_run[h] > DEC_MAX_SLACK);
-      if (compute_bar_or(exceed)) {
+      for (int h = 0; h < 8; h++) {
+        float v = l_run[h];
 #pragma unroll
-        for (int h = 0; h < 8; h++) {
-          const float wm = warp_max(s[h]);
-          if (lane == h) red[warp * 8 + h] = wm;
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+        float bv = best_v[h];
+        int bi = best_i[h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float ov = __shfl_xor_sync(FULL, bv, o);
+          const int oi = ARGMAX ? __shfl_xor_sync(FULL, bi, o) : -1;
+          if (ov > bv || (ARGMAX && ov == bv && oi >= 0 && (bi < 0 || oi < bi))) { bv = ov; bi = oi; }
         }
-        compute_bar_sync();
-#pragma unroll
-        for (int h = 0; h < 8; h++) {
-          const float bm = fmaxf(fmaxf(red[h], red[8 + h]), fmaxf(red[16 + h], red[24 + h]));
-          const float mn = fmaxf(m_run[h], bm);
-          alpha[h] = ex2f(m_run[h] - mn);
-          m_run[h] = mn;
-          l_run[h] *= alpha[h];
-        }
-      } else {
-#pragma unroll
-        for (int h = 0; h < 8; h++) alpha[h] = 1.f;
+        if (lane == h) { red[(warp & 3) * 8 + h] = v; red2[(warp & 3) * 8 + h] = bv; redi[(warp & 3) * 8 + h] = bi; }
       }
-      {
-        const float vf = (tid < n) ? vsc * vfac : 0.f;
-        float wv[8];
 #pragma unroll
-        for (int h = 0; h < 8; h++) {
-          const float pr = ex2f(s[h] - m_run[h]);
-          l_run[h] += pr;
-          wv[h] = pr * vf;
-        }
-        // probabilities (times scale_V / sqrt(d)) as fp16 hi + lo: B_P[n][row], n = head (hi) or 8 + head (lo)
-        uint4 hi4, lo4;
-        uint32_t* hp = reinterpret_cast<uint32_t*>(&hi4);
-        uint32_t* lp = reinterpret_cast<uint32_t*>(&lo4);
+      for (int j = 0; j < DJ; j++)
 #pragma unroll
-        for (int h2 = 0; h2 < 4; h2++) {
-          const uint32_t hpk = pack_half2(wv[2 * h2], wv[2 * h2 + 1]);
-          const float2 back = __half22float2(*reinterpret_cast<const __half2*>(&hpk));
-          hp[h2] = hpk;
-          lp[h2] = pack_half2(wv[2 * h2] - back.x, wv[2 * h2 + 1] - back.y);
+        for (int h = 0; h < 8; h++) gacc[(j * 8 + h) * DEC_GROUP_THREADS + gt] = acc[j][h];
+      group_bar_sync(bar_id);
+      if (gt < 8) {
+        const int h = gt;
+        float mt = -INFINITY;
+        int bi = -1;
+        for (int wq = 0; wq < 4; wq++) {
+          const float ov = red2[wq * 8 + h];
+          const int oi = redi[wq * 8 + h];
+          if (ov > mt || (ov == mt && oi >= 0 && (bi < 0 || oi < bi))) { mt = ov; bi = oi; }
         }
-        const int off = (tid & 7) * 16 + (tid >> 3) * 128;
-        *reinterpret_cast<uint4*>(bp + off) = hi4;
-        *reinterpret_cast<uint4*>(bp + (TB / 8) * 128 + off) = lo4;
-        fence_proxy_async();
-      }
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(p_ready);                 // V tile in TMEM, probabilities in shared memory
-      mbar_arrive(&empty_bar[blk % NST]);   // this thread is done with the staged tile
-      folded = false;
-      // ---- next block's K tile, while the value MMAs run
-      if (blk + 1 < nblk) {
-        if (L::SHARED_A) { fold(blk); folded = true; }  // the value MMAs read the tile that K is about to overwrite
-        k_phase(blk + 1);
+        gml[4 * h] = m_run[h];  // every thread of the group holds the same reference
+        gml[4 * h + 1] = red[h] + red[8 + h] + red[16 + h] + red[24 + h];
+        gml[4 * h + 2] = mt;
+        reinterpret_cast<int*>(gml)[4 * h + 3] = bi;
       }
     }
-    if (!folded) fold(nblk - 1);
+    // ================================================================ merge the groups' partials into the item's partial slot
+    const int seg_b = seg_s->b, seg_y = seg_s->y, seg_slot = seg_s->slot, seg_flags = seg_s->flags;  // before thread 0 reopens seg_s
+    __syncthreads();  // every group has closed its part
+    if (!control) {
+      const int kvh = seg_y / p.head_groups;
+      const int hg = seg_y - kvh * p.head_groups;
+      const int h0 = kvh * p.group + hg * DEC_HEADS;
+      const int nh = min(DEC_HEADS, p.group - hg * DEC_HEADS);
+      const uint8_t* group0 = bq + L::BQ_BYTES + L::BP_BYTES;  // staging buffer of group 0; the others follow at GROUP_SMEM
+      auto gacc_of = [&](int g) { return reinterpret_cast<const float*>(group0 + (size_t)g * L::GROUP_SMEM); };
+      auto gml_of = [&](int g) { return gacc_of(g) + DJ * 8 * DEC_GROUP_THREADS; };
+      // thread (c, hsel): coordinate c (+128), heads hsel, hsel + NG, ...
+      const int c = tid & (DEC_GROUP_THREADS - 1);
+      for (int h = tid >> 7; h < nh; h += NG) {
+        float mt = -INFINITY;  // the exact maximum of the segment: the partial is reported relative to it
+#pragma unroll
+        for (int g = 0; g < NG; g++) mt = fmaxf(mt, gml_of(g)[4 * h + 2]);
+        float sc[NG];
+#pragma unroll
+        for (int g = 0; g < NG; g++) sc[g] = ex2f(gml_of(g)[4 * h] - mt);  // a group without blocks: exp2(-inf) = 0
+#pragma unroll
+        for (int j = 0; j < DJ; j++) {
+          float v = 0.f;
+#pragma unroll
+          for (int g = 0; g < NG; g++) v += gacc_of(g)[(j * 8 + h) * DEC_GROUP_THREADS + c] * sc[g];
+          p.part_acc[(((size_t)seg_b * p.n_q_heads + h0 + h) * S + seg_slot) * D + c + 128 * j] = v;
+        }
+      }
+      if (tid < nh) {
+        const int h = tid;
+        float mt = -INFINITY;
+        int bi = -1;
+#pragma unroll
+        for (int g = 0; g < NG; g++) {
+          const float ov = gml_of(g)[4 * h + 2];
+          const int oi = reinterpret_cast<const int*>(gml_of(g))[4 * h + 3];
+          if (ov > mt || (ov == mt && oi >= 0 && (bi < 0 || oi < bi))) { mt = ov; bi = oi; }
+        }
+        float l = 0.f;
+#pragma unroll
+        for (int g = 0; g < NG; g++) l += gml_of(g)[4 * h + 1] * ex2f(gml_of(g)[4 * h] - mt);
+        const size_t o = ((size_t)seg_b * p.n_q_heads + h0 + h) * S + seg_slot;
+        p.part_ml[2 * o] = mt * LN2;
+        p.part_ml[2 * o + 1] = l;
+        if (ARGMAX) p.part_argmax[o] = bi;
+      }
+      if (seg_flags & 1) fill_slots(seg_b, h0, nh, seg_slot + 1, L::COMPUTE_THREADS, tid);  // end of the item: its unused slots
+    }
+    if (seg_flags & 2) break;  // last segment of this CTA
   }
 
   if (__syncthreads_or(failed) && tid == 0 && p.status) atomicOr(&p.status[0], IQ_STATUS_WAIT_TIMEOUT);
-
-  // ---------------------------------------------------------------- reduce l, the exact maximum (and argmax) over the 128 rows
-  if (!control) {
-#pragma unroll
-  for (int h = 0; h < 8; h++) {
-    float v = l_run[h];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
-    float bv = best_v[h];
-    int bi = best_i[h];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(FULL, bv, o);
-      const int oi = ARGMAX ? __shfl_xor_sync(FULL, bi, o) : -1;
-      if (ov > bv || (ARGMAX && ov == bv && oi >= 0 && (bi < 0 || oi < bi))) { bv = ov; bi = oi; }
-    }
-    if (lane == h) { red[warp * 8 + h] = v; red2[warp * 8 + h] = bv; redi[warp * 8 + h] = bi; }
-  }
-  }
-  __syncthreads();
-  if (!control) {
-  // The partial is reported relative to the exact maximum m = max_j z_j: rescale from the running reference.
-  float fix[8];
-#pragma unroll
-  for (int h = 0; h < 8; h++) {
-    const float mt = fmaxf(fmaxf(red2[h], red2[8 + h]), fmaxf(red2[16 + h], red2[24 + h]));
-    fix[h] = ex2f(m_run[h] - mt);
-    if (h < nh) {
-#pragma unroll
-      for (int j = 0; j < DJ; j++)
-        p.part_acc[(((size_t)b * p.n_q_heads + h0 + h) * S + split) * D + tid + 128 * j] = acc[j][h] * fix[h];
-    }
-  }
-  if (tid < nh) {
-    const int h = tid;
-    float mt = -INFINITY;
-    int bi = -1;
-    for (int w = 0; w < 4; w++) {
-      const float ov = red2[w * 8 + h];
-      const int oi = redi[w * 8 + h];
-      if (ov > mt || (ov == mt && oi >= 0 && (bi < 0 || oi < bi))) { mt = ov; bi = oi; }
-    }
-    const float l = (red[h] + red[8 + h] + red[16 + h] + red[24 + h]) * ex2f(m_run[h] - mt);
-    const size_t o = ((size_t)b * p.n_q_heads + h0 + h) * S + split;
-    p.part_ml[2 * o] = mt * LN2;
-    p.part_ml[2 * o + 1] = l;
-    if (ARGMAX) p.part_argmax[o] = bi;
-  }
-  }
   tc_fence_before();
   __syncthreads();
-  if (control) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_a), "r"(L::ALLOC0_COLS));
-    if (L::ALLOC1_COLS > 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_r), "r"(L::ALLOC1_COLS));
-  }
+  if (warp == NG * 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
 }
 
 template <int D, bool ARGMAX>
 static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
   using L = DecLayout<D>;
   static bool configured[64] = {};
+  static int n_sm[64] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
   auto kern = decode_kernel<D, ARGMAX>;
-  if (dev < 0 || dev >= 64 || !configured[dev]) {
+  if (!configured[dev]) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64) configured[dev] = true;
+    e = cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    configured[dev] = true;
   }
-  dim3 grid(p.splits, p.n_kv_heads * p.head_groups, p.batch);
-  kern<<<grid, DEC_THREADS, L::SMEM_BYTES, stream>>>(p);
+  // One CTA per SM; each takes an equal share of the launch's 128-row blocks. No more CTAs than blocks.
+  const long long max_blocks = (long long)p.batch * p.n_kv_heads * p.head_groups * ((p.t_cap + DEC_BLOCK_TOKENS - 1) / DEC_BLOCK_TOKENS);
+  long long ctas = n_sm[dev];
+  if (ctas > max_blocks) ctas = max_blocks;
+  if (ctas < 1) ctas = 1;
+  kern<<<dim3((unsigned)ctas), L::THREADS, L::SMEM_BYTES, stream>>>(p);
   return cudaGetLastError();
 }
 
@@ -592,6 +776,7 @@ cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStr
   return am ? launch_one<256, true>(p, stream) : launch_one<256, false>(p, stream);
 }
 
-int decode_ctas_per_sm(int head_dim) { return head_dim == 128 ? DecLayout<128>::CTAS_PER_SM : DecLayout<256>::CTAS_PER_SM; }
+// CTAs the decode kernel keeps resident per SM (it sizes its grid as one CTA per SM).
+int decode_ctas_per_sm(int head_dim) { (void)head_dim; return 1; }
 
 }  // namespace iq

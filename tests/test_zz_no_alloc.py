@@ -44,8 +44,10 @@ def test_static_scratch_decode_matches_regular_path_twice(codebooks):
         torch.cuda.synchronize()
         assert torch.cuda.mem_get_info()[0] == free_before            # after set-up, a call takes no device memory
         assert int(status[0]) == 0
-        assert torch.equal(out, ref) and torch.equal(lse, ref_lse)    # same kernels, same partials: bit-identical
-        assert np.allclose(out.cpu().numpy(), ref.cpu().numpy(), atol=2e-3, rtol=1e-3)
+        # same kernels on the same inputs; the decode kernel hands out blocks dynamically, so the fp32 summation order
+        # (and nothing else) may differ between two calls
+        assert np.allclose(out.cpu().numpy(), ref.cpu().numpy(), atol=1e-5, rtol=1e-5)
+        assert np.allclose(lse.cpu().numpy(), ref_lse.cpu().numpy(), atol=1e-5, rtol=1e-6)
         out16 = torch.empty((B, H_q, d), dtype=torch.float16, device="cuda")
         iq.iq_decode_attention_static(shape, rot, cb, q, cache, sl, S, out16)
         torch.cuda.synchronize()
