@@ -572,8 +572,9 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           tc_ld16(tmem_g + lane_sel + L::S_COL, raw);
           const bool valid = gt < n;  // rows >= n of the last block hold stale bytes
           const float kf = valid ? ksc * kfac : 0.f;
+          const float mask = valid ? 0.f : -INFINITY;  // stale rows: 0 * finite - inf = -inf
 #pragma unroll
-          for (int h = 0; h < 8; h++) s[h] = valid ? (raw[h] + raw[8 + h]) * kf : -INFINITY;
+          for (int h = 0; h < 8; h++) s[h] = fmaf(raw[h] + raw[8 + h], kf, mask);
         }
 #pragma unroll
         for (int h = 0; h < 8; h++) {  // exact maximum seen by this thread (the partial's m) and, optionally, its row
