@@ -37,9 +37,17 @@ WORKLOADS = {
 DEFAULT_WORKLOAD = "config5_B32_ctx32768"
 T_CAP_MARGIN = 2048  # rows of head-room so that every sequence can take the benchmark's appends
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch, from the ncu capture summarised under
-# profiles/ (None until a capture of that workload exists).
-DECODE_TRAFFIC_BYTES = {}
+# DRAM traffic of one decode launch. The ncu capture (profiles/decode_kernel_config5_B8.md; the B = 32 workload is too
+# large to capture with dram counters under the size rule) measured, at B = 8, dram__bytes_read.sum = 1.0031 x the
+# algorithmic packed-KV bytes of the launch and dram__bytes_write.sum = 7.91 MB for 1.33 MB of partial results
+# (S = 5 slots). Reads scale with the rows processed; writes with the partial results.
+NCU_READ_PER_ALGORITHMIC_BYTE = 182.576 / 182.013
+NCU_WRITE_PER_PARTIAL_BYTE = 7.907 / 1.331
+
+
+def decode_traffic_bytes(algorithmic_bytes: float, B: int, H_q: int, S: int, d: int) -> int:
+    partial_bytes = B * H_q * S * (d + 2) * 4
+    return int(NCU_READ_PER_ALGORITHMIC_BYTE * algorithmic_bytes + NCU_WRITE_PER_PARTIAL_BYTE * partial_bytes)
 
 
 def bytes_per_row(d: int) -> int:
@@ -179,16 +187,18 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     K, W = args.steps, args.warmup
     S = args.splits or iq.iq_suggest_splits(shape, st["ctx"])
     ws = iq.DecodeWorkspace(shape, S, want_argmax=False, device=device)
-    lens = torch.from_numpy(st["lens_np"]).to(device)
+    # Row i of this table holds the sequence lengths before step i: the step appends at lens_tab[i] and attends to
+    # lens_tab[i + 1] rows (the serving engine knows the lengths; no kernel is spent on incrementing them).
+    lens0 = torch.from_numpy(st["lens_np"]).to(device)
+    lens_tab = (lens0[None, :] + torch.arange(K + W + 4, device=device, dtype=torch.int32)[:, None]).contiguous()
     q_all, k_all, v_all = step_inputs(st, K + W, device, 99 + rank)
     stream = torch.cuda.current_stream()
 
     def one_step(i, ev=None):
-        iq.iq_quantize_append(shape, rot, cb, k_all[i], v_all[i], lens, None, 1, cache, st["status"])
-        lens.add_(1)
+        iq.iq_quantize_append(shape, rot, cb, k_all[i], v_all[i], lens_tab[i], None, 1, cache, st["status"])
         if ev is not None:
             ev[0].record(stream)
-        iq.iq_decode_attention(shape, rot, cb, q_all[i], cache, lens, S, ws.part_acc, ws.part_ml, None, ws.status)
+        iq.iq_decode_attention(shape, rot, cb, q_all[i], cache, lens_tab[i + 1], S, ws.part_acc, ws.part_ml, None, ws.status)
         if ev is not None:
             ev[1].record(stream)
         iq.iq_combine_splits(shape, rot, S, ws.part_acc, ws.part_ml, None, ws.out, ws.lse, None)
@@ -227,17 +237,16 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     def e2e_step(i):
         dq.copy_(hq[i], non_blocking=True); dk.copy_(hk[i], non_blocking=True); dv.copy_(hv[i], non_blocking=True)
-        iq.iq_quantize_append(shape, rot, cb, dk, dv, lens, None, 1, cache, st["status"])
-        lens.add_(1)
-        iq.iq_decode_attention(shape, rot, cb, dq, cache, lens, S, ws.part_acc, ws.part_ml, None, ws.status)
+        iq.iq_quantize_append(shape, rot, cb, dk, dv, lens_tab[i], None, 1, cache, st["status"])
+        iq.iq_decode_attention(shape, rot, cb, dq, cache, lens_tab[i + 1], S, ws.part_acc, ws.part_ml, None, ws.status)
         iq.iq_combine_splits(shape, rot, S, ws.part_acc, ws.part_ml, None, ws.out, ws.lse, None)
         hout.copy_(ws.out, non_blocking=True)
         torch.cuda.synchronize()
 
     n_e2e = K
-    lens.copy_(torch.from_numpy(st["lens_np"]).to(device))               # rewind: the e2e leg re-appends over the same rows
-    lens_before = lens.clone()
-    for i in range(min(3, W)):
+    # the e2e leg re-appends over the same rows (it restarts from row 0 of the length table)
+    n_e2e_warm = min(3, W)
+    for i in range(n_e2e_warm):
         e2e_step(i)
     if world > 1:
         dist.barrier()
@@ -245,7 +254,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     torch.cuda.synchronize()
     e0.record(stream)
     for i in range(n_e2e):
-        e2e_step(W + i)
+        e2e_step(n_e2e_warm + i)
     e1.record(stream)
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
@@ -253,7 +262,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         tt = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         e2e_ms = float(tt.item())
-    rows_e2e = int(lens_before.sum().item()) + B * min(3, W)
+    rows_e2e = int(st["lens_np"].astype(np.int64).sum()) + B * n_e2e_warm
     e2e_bytes = sum((rows_e2e + B * (i + 1)) * H_kv * bytes_per_row(d) for i in range(n_e2e))
 
     if rank != 0:
@@ -283,7 +292,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "decode_tokens_per_s": round(world * B / (ms_step * 1e-3), 1),
         "frac_of_8TBs": round(value / world / 8000.0, 4),
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
-                     "traffic": DECODE_TRAFFIC_BYTES.get(args.workload), "kernel": "decode_kernel", "peak_source": peak_src,
+                     "traffic": decode_traffic_bytes(sum(bytes_steps) / K, B, H_q, S, d),
+                     "traffic_source": "ncu capture at B = 8 scaled by rows processed (reads) and partial results (writes)",
+                     "kernel": "decode_kernel", "peak_source": peak_src,
                      "avg_launch_ms": round(dec_avg_ms, 4), "algorithmic_bytes_per_launch": int(sum(bytes_steps) / K)},
         "e2e": {"value": round(world * e2e_bytes / (e2e_ms * 1e-3) / 1e9, 1), "unit": "GB/s",
                 "h2d_bytes_per_step": int(B * (H_q + 2 * H_kv) * d * 2), "d2h_bytes_per_step": int(B * H_q * d * 4),
@@ -294,7 +305,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
-        out["cpu_baseline"] = cpu_baseline(st, lens, q_all[W + K - 1])
+        out["cpu_baseline"] = cpu_baseline(st, lens_tab[n_e2e_warm + n_e2e], q_all[W + K - 1])
     return out
 
 
