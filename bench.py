@@ -117,6 +117,36 @@ class ClockSampler:
                 "power_w_max": round(max(p for _, p in self.samples), 1)}
 
 
+def init_distributed(world: int, local_rank: int, backend: str = "nccl") -> None:
+    """One process per GPU; rendezvous on 127.0.0.1 unless the launcher says otherwise. The data path has no
+    collective: the group is used for the barrier around the timed region and the max-over-ranks time."""
+    if world <= 1:
+        return
+    import torch.distributed as dist
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29531")
+    if backend == "nccl":
+        import torch
+        torch.cuda.set_device(local_rank)
+    dist.init_process_group(backend)
+
+
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """The slowest rank's time: every multi-GPU number is reported against it."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    tt = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return float(tt.item())
+
+
+def aggregate_gbs(bytes_per_rank: float, ms: float, world: int) -> float:
+    """Whole-job throughput of `world` replicas that each moved bytes_per_rank in ms (weak scaling)."""
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
+
+
 def build_state(name: str, device, rank: int):
     """Synthetic cache for one rank: seeded K/V generated on the GPU in chunks and bulk-quantized (untimed)."""
     import torch
@@ -225,10 +255,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     assert int(ws.status[0].item()) == 0 and int(st["status"][0].item()) == 0, "device status flags set"
     rows = int(st["lens_np"].astype(np.int64).sum()) + B * W           # cached rows per KV head at the first timed step
     bytes_steps = [(rows + B * (i + 1)) * H_kv * bytes_per_row(d) for i in range(K)]
-    if world > 1:
-        tt = torch.tensor([ms_total], device=device, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total, world, device)
 
     # ---- end to end through the C-ABI binding with host buffers: H2D of the step inputs and D2H of the output inside the timed region
     hq = q_all[:W + K].cpu().pin_memory(); hk = k_all[:W + K].cpu().pin_memory(); hv = v_all[:W + K].cpu().pin_memory()
@@ -258,10 +285,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     e1.record(stream)
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        tt = torch.tensor([e2e_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, device)
     rows_e2e = int(st["lens_np"].astype(np.int64).sum()) + B * n_e2e_warm
     e2e_bytes = sum((rows_e2e + B * (i + 1)) * H_kv * bytes_per_row(d) for i in range(n_e2e))
 
@@ -269,7 +293,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         return None
     peak, peak_src = measured_peak_hbm()
     ms_step = ms_total / K
-    value = world * sum(bytes_steps) / (ms_total * 1e-3) / 1e9
+    value = aggregate_gbs(sum(bytes_steps), ms_total, world)
     dec_avg_ms = sum(dec_ms) / K
     achieved = (sum(bytes_steps) / K) / (dec_avg_ms * 1e-3) / 1e9
     out = {
@@ -296,7 +320,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                      "traffic_source": "ncu capture at B = 8 scaled by rows processed (reads) and partial results (writes)",
                      "kernel": "decode_kernel", "peak_source": peak_src,
                      "avg_launch_ms": round(dec_avg_ms, 4), "algorithmic_bytes_per_launch": int(sum(bytes_steps) / K)},
-        "e2e": {"value": round(world * e2e_bytes / (e2e_ms * 1e-3) / 1e9, 1), "unit": "GB/s",
+        "e2e": {"value": round(aggregate_gbs(e2e_bytes, e2e_ms, world), 1), "unit": "GB/s",
                 "h2d_bytes_per_step": int(B * (H_q + 2 * H_kv) * d * 2), "d2h_bytes_per_step": int(B * H_q * d * 4),
                 "ms_per_step": round(e2e_ms / max(n_e2e, 1), 4), "steps": n_e2e,
                 "note": "packed cache is device-resident state; per-step inputs (q, new k/v) come from pinned host memory, output returns to host"},
@@ -343,7 +367,7 @@ def run_reference(args, rank: int, world: int):
     lv, th = lloyd_max.fp16_codebook(d)
     quats = workloads.quaternion_pairs(workloads.rng(5, workloads.QUAT_STREAM), H_kv, d)
     P = oracle.row_bytes(d)
-    cache = oracle.new_cache(nb, H_kv, d, T + 64)
+    cache = oracle.new_cache(nb, H_kv, d, workloads.cap128(T + args.warmup + args.steps + 1))
     # the sample's cache content: uniformly random codes and Gaussian-row-like scales (the decode cost does not depend on values)
     cache["k_codes"][:] = g.integers(0, 256, cache["k_codes"].shape, dtype=np.uint8)
     cache["v_codes"][:] = g.integers(0, 256, cache["v_codes"].shape, dtype=np.uint8)
@@ -395,12 +419,7 @@ def main():
         return
     if args.steps + args.warmup + 8 > T_CAP_MARGIN:
         raise SystemExit(f"--steps + --warmup must stay below {T_CAP_MARGIN - 8}")
-    if world > 1:
-        import torch.distributed as dist
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        import torch
-        torch.cuda.set_device(local_rank)
-        dist.init_process_group("nccl")
+    init_distributed(world, local_rank, "nccl")
     out = run_ours(args, rank, world, local_rank)
     if world > 1:
         import torch.distributed as dist
