@@ -157,9 +157,11 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
  *                  A small S restricts that choice; iq_suggest_splits gives a value that does not.
  *   part_acc       device fp32 [batch][n_q_heads][S][head_dim]: sum_j exp(z_j - m) v~_j over the slot's rows,
  *                  in the rotated space, natural coordinate order. 16-byte aligned.
- *   part_ml        device fp32 [batch][n_q_heads][S][2] = (m, l): m = max_j z_j, l = sum_j exp(z_j - m),
- *                  z_j = sm_scale * q~ . k~_j. An unused slot holds (-inf, 0) and acc = 0; every slot of every
- *                  head is written on every call.
+ *   part_ml        device fp32 [batch][n_q_heads][S][2] = (m, l): the slot's reference m and l = sum_j exp(z_j - m),
+ *                  z_j = sm_scale * q~ . k~_j. With part_argmax, m = max_j z_j exactly; without it m is the kernel's
+ *                  running reference, max_j z_j - 4 ln 2 <= m <= max_j z_j (acc and l are relative to the same m
+ *                  either way). An unused slot holds (-inf, 0) and acc = 0; every slot of every head is written on
+ *                  every call.
  *   part_argmax    device int32 [batch][n_q_heads][S] or NULL: row index attaining m (lowest on ties), -1 if empty.
  *   status_dev     optional (see top).
  * Arithmetic: q~ and the probabilities enter fp16 tensor-core operands, each as a two-term fp16 sum

@@ -164,6 +164,11 @@ __device__ __forceinline__ bool group_bar_or(int id, bool pred) {
 __device__ __forceinline__ void cta_bar_sync() { asm volatile("barrier.sync 0;" ::: "memory"); }
 __device__ __forceinline__ void group_bar_sync(int id) { asm volatile("barrier.sync %0, 128;" ::"r"(id) : "memory"); }
 
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(FULL, v, o));
@@ -509,15 +514,16 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 #pragma unroll
       for (int h = 0; h < 8; h++) { m_run[h] = -INFINITY; l_run[h] = 0.f; best_v[h] = -INFINITY; best_i[h] = -1; }
 
+      int st = it % NST;                      // stage of slot `it` and its phase, kept incrementally
+      uint32_t st_ph = (uint32_t)(it / NST) & 1u;
       for (;;) {
         if (failed) break;
-        const int st = it % NST;
         const uint8_t* sp = stages + st * L::STAGE_BYTES;
-        failed = !mbar_wait_bounded(&full_bar[st], (uint32_t)(it / NST) & 1u, DEC_WAIT_LIMIT);
+        failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
         const int2 dsc = desc[st];
         if (dsc.y < 0) {  // end marker: the segment has no more blocks for this group
           mbar_arrive(&empty_bar[st]);
-          it++;
+          it++;  // (st and st_ph are recomputed from `it` when the next segment starts)
           break;
         }
         const int r0 = dsc.x, n = dsc.y;
@@ -576,20 +582,18 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 #pragma unroll
           for (int h = 0; h < 8; h++) s[h] = fmaf(raw[h] + raw[8 + h], kf, mask);
         }
+        if (ARGMAX) {  // exact maximum seen by this thread and its row (a group sees its blocks in ascending order)
 #pragma unroll
-        for (int h = 0; h < 8; h++) {  // exact maximum seen by this thread (the partial's m) and, optionally, its row
-          if (ARGMAX) {
-            if (s[h] > best_v[h]) { best_v[h] = s[h]; best_i[h] = r0 + gt; }  // a group sees its blocks in ascending order
-          } else {
-            best_v[h] = fmaxf(best_v[h], s[h]);
-          }
+          for (int h = 0; h < 8; h++)
+            if (s[h] > best_v[h]) { best_v[h] = s[h]; best_i[h] = r0 + gt; }
         }
         // The running reference m_run is raised only when some score of the block exceeds it by more than
         // DEC_MAX_SLACK (log2 units): exp2(s - m_run) then stays below 2^DEC_MAX_SLACK and nothing has to be
         // exchanged between the warps in the common case (one barrier with an OR reduction).
-        bool exceed = false;
+        float over[8];
 #pragma unroll
-        for (int h = 0; h < 8; h++) exceed |= (s[h] - m_run[h] > DEC_MAX_SLACK);
+        for (int h = 0; h < 8; h++) over[h] = s[h] - m_run[h];  // NaN (-inf - -inf) for a stale row of an unopened reference: max ignores it
+        const bool exceed = max3f(max3f(over[0], over[1], over[2]), max3f(over[3], over[4], over[5]), fmaxf(over[6], over[7])) > DEC_MAX_SLACK;
         if (group_bar_or(bar_id, exceed)) {
 #pragma unroll
           for (int h = 0; h < 8; h++) {
@@ -649,6 +653,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         tc_fence_before();
         it++;
         nbk++;
+        if (++st == NST) { st = 0; st_ph ^= 1u; }
       }
 
       // ---- close the group's part of the segment: reduce l and the exact maximum (and argmax) over the 128 rows and
@@ -684,7 +689,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         }
         gml[4 * h] = m_run[h];  // every thread of the group holds the same reference
         gml[4 * h + 1] = red[h] + red[8 + h] + red[16 + h] + red[24 + h];
-        gml[4 * h + 2] = mt;
+        gml[4 * h + 2] = ARGMAX ? mt : m_run[h];  // without the argmax output the reference stands in for the maximum
         reinterpret_cast<int*>(gml)[4 * h + 3] = bi;
       }
     }
