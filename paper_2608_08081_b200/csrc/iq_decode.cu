@@ -95,6 +95,15 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&o)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; i++) o[i] = __uint_as_float(r[i]);
 }
+// The same load without the wait: the registers are valid after tc_wait_ld().
+__device__ __forceinline__ void tc_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 // D[tmem] (+)= A[tmem] * B[smem descriptor]; fp16 operands, fp32 accumulate, M = 128, N and majors in idesc.
 __device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -550,37 +559,42 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         // the score MMAs read the tile that the V dequantisation is about to overwrite
         if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
 
-        // ---- V coordinate gt (+128) of this block -> TMEM lane gt (A_V)
+        // ---- V coordinate gt (+128) of this block -> TMEM lane gt (A_V), interleaved with the softmax of the block: the
+        // lookups load the shift/logic pipe, the softmax the FMA and special-function pipes, and the read-back of the
+        // scores and the group barrier have latencies worth covering.
+        uint32_t wd[DJ][12];
 #pragma unroll
         for (int j = 0; j < DJ; j++) {
           const uint4* vrow = reinterpret_cast<const uint4*>(sp + L::K_BYTES + (gt + 128 * j) * 48);
-          uint32_t wd[12];
 #pragma unroll
           for (int i = 0; i < 3; i++) {
             const uint4 t4 = vrow[i];
-            wd[4 * i] = t4.x; wd[4 * i + 1] = t4.y; wd[4 * i + 2] = t4.z; wd[4 * i + 3] = t4.w;
-          }
-#pragma unroll
-          for (int u = 0; u < 4; u++) {
-            uint32_t f[16];
-            dequant_unit(wd[3 * u], wd[3 * u + 1], wd[3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);
-            tc_st16(tmem_g + lane_sel + L::A_COL + 64 * j + 16 * u, f);
+            wd[j][4 * i] = t4.x; wd[j][4 * i + 1] = t4.y; wd[j][4 * i + 2] = t4.z; wd[j][4 * i + 3] = t4.w;
           }
         }
         const float ksc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES)[gt];
         const float vsc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES)[gt];
+        auto v_unit = [&](int q) {  // unit q of the thread's V coordinates: dequantise and store
+          const int j = q >> 2, u = q & 3;
+          uint32_t f[16];
+          dequant_unit(wd[j][3 * u], wd[j][3 * u + 1], wd[j][3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);
+          tc_st16(tmem_g + lane_sel + L::A_COL + 64 * j + 16 * u, f);
+        };
+        tc_fence_after();
+        uint32_t raw_u[16];
+        tc_ld16_issue(tmem_g + lane_sel + L::S_COL, raw_u);  // scores of row gt: in flight during the first units
+#pragma unroll
+        for (int q = 0; q < 2 * DJ; q++) v_unit(q);
 
         // ---- online softmax (log2 units); thread gt owns row r0 + gt, all 8 heads
-        tc_fence_after();
+        tc_wait_ld();
         float s[8];
         {
-          float raw[16];
-          tc_ld16(tmem_g + lane_sel + L::S_COL, raw);
           const bool valid = gt < n;  // rows >= n of the last block hold stale bytes
           const float kf = valid ? ksc * kfac : 0.f;
           const float mask = valid ? 0.f : -INFINITY;  // stale rows: 0 * finite - inf = -inf
 #pragma unroll
-          for (int h = 0; h < 8; h++) s[h] = fmaf(raw[h] + raw[8 + h], kf, mask);
+          for (int h = 0; h < 8; h++) s[h] = fmaf(__uint_as_float(raw_u[h]) + __uint_as_float(raw_u[8 + h]), kf, mask);
         }
         if (ARGMAX) {  // exact maximum seen by this thread and its row (a group sees its blocks in ascending order)
 #pragma unroll
@@ -612,6 +626,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
             for (int j = 0; j < DJ; j++) acc[j][h] *= alpha;
           }
         }
+#pragma unroll
+        for (int q = 2 * DJ; q < 4 * DJ; q++) v_unit(q);  // the other half of the V units, next to the exponentials
         {
           const float vf = (gt < n) ? vsc * vfac : 0.f;
           float wv[8];
