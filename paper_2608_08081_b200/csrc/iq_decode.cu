@@ -53,6 +53,7 @@ struct DecLayout {
   static constexpr int A_COL = 0;
   static constexpr int S_COL = D / 2;
   static constexpr int O_COL = D / 2 + 16;
+  static constexpr int V_COL = O_COL + 16 * (D / 128);  // rows 0..63 of the V tile (32 columns per 128 coordinates)
   static constexpr int NG = 512 / GROUP_COLS;  // groups per CTA: 4 at d = 128, 2 at d = 256
   static constexpr int COMPUTE_THREADS = NG * DEC_GROUP_THREADS;
   static constexpr int THREADS = COMPUTE_THREADS + NG * 32;  // + one control warp per group
@@ -65,8 +66,8 @@ struct DecLayout {
 };
 static_assert(DEC_BLOCK_TOKENS == 128, "the TMEM operand layout assumes 128-row blocks");
 static_assert(DecLayout<128>::OFF_RED + 4 * DecLayout<128>::RED_STRIDE <= DEC_HDR_BYTES, "header overflow");
-static_assert(DecLayout<128>::O_COL + 16 * DecLayout<128>::DJ <= DecLayout<128>::GROUP_COLS, "TMEM group overflow");
-static_assert(DecLayout<256>::O_COL + 16 * DecLayout<256>::DJ <= DecLayout<256>::GROUP_COLS, "TMEM group overflow");
+static_assert(DecLayout<128>::V_COL + 32 * DecLayout<128>::DJ <= DecLayout<128>::GROUP_COLS, "TMEM group overflow");
+static_assert(DecLayout<256>::V_COL + 32 * DecLayout<256>::DJ <= DecLayout<256>::GROUP_COLS, "TMEM group overflow");
 static_assert(DecLayout<128>::SMEM_BYTES <= 227 * 1024 && DecLayout<256>::SMEM_BYTES <= 227 * 1024, "shared memory overflow");
 static_assert((DecLayout<128>::THREADS + DecLayout<128>::THREADS / 32) * 4 <= DecLayout<128>::BP_BYTES, "set-up scratch must fit one B_P region");
 
@@ -494,7 +495,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           for (int j = 0; j < DJ; j++)
 #pragma unroll
             for (int kk = 0; kk < TB / 16; kk++)
-              tc_mma_f16(tmem_g + L::O_COL + 16 * j, tmem_g + L::A_COL + 64 * j + 8 * kk,
+              tc_mma_f16(tmem_g + L::O_COL + 16 * j,  // rows 0..63 of the V tile sit in V_COL, rows 64..127 in the operand columns
+                         tmem_g + (kk < 4 ? L::V_COL + 32 * j + 8 * kk : L::A_COL + 64 * j + 8 * (kk - 4)),
                          smem_desc_mn(bp_addr + kk * 256, 128, (TB / 8) * 128), DEC_IDESC, kk > 0);
           tc_commit(o_bar);
         }
@@ -523,45 +525,53 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 #pragma unroll
       for (int h = 0; h < 8; h++) { m_run[h] = -INFINITY; l_run[h] = 0.f; best_v[h] = -INFINITY; best_i[h] = -1; }
 
+      // The group's 128 TMEM columns: [0, 64 DJ) operand tile, then scores, values, and V_COL.. a second home for the first
+      // half of the V tile. Schedule of one block (K tile complete, k_ready signalled):
+      //   V rows 0..63 -> V_COL columns               while the score MMAs read the K tile
+      //   wait for the scores; V rows 64..127 -> lower half of the operand columns, interleaved with the softmax
+      //   signal p_ready; next block's K coordinates 32..63 (+64..) -> upper half of the operand columns
+      //                                                while the value MMAs read the lower half and V_COL
+      //   wait for the values, fold them; next block's other K coordinates -> lower half; signal k_ready
       int st = it % NST;                      // stage of slot `it` and its phase, kept incrementally
       uint32_t st_ph = (uint32_t)(it / NST) & 1u;
-      for (;;) {
-        if (failed) break;
-        const uint8_t* sp = stages + st * L::STAGE_BYTES;
-        failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
-        const int2 dsc = desc[st];
-        if (dsc.y < 0) {  // end marker: the segment has no more blocks for this group
-          mbar_arrive(&empty_bar[st]);
-          it++;  // (st and st_ph are recomputed from `it` when the next segment starts)
-          break;
+      uint32_t kw[L::WPR];                    // packed K row of the block being staged into TMEM
+      auto k_load = [&](const uint8_t* sp_) {
+        const uint4* krow = reinterpret_cast<const uint4*>(sp_ + gt * L::ROWB);
+#pragma unroll
+        for (int i = 0; i < L::WPR / 4; i++) {
+          const uint4 t4 = krow[i];
+          kw[4 * i] = t4.x; kw[4 * i + 1] = t4.y; kw[4 * i + 2] = t4.z; kw[4 * i + 3] = t4.w;
         }
-        const int r0 = dsc.x, n = dsc.y;
-
-        // ---- K row gt of the staged tile -> TMEM lane gt (A_K), then signal the control warp
-        {
-          uint32_t w[L::WPR];
-          const uint4* krow = reinterpret_cast<const uint4*>(sp + gt * L::ROWB);
+      };
+      auto k_unit = [&](int u) {
+        uint32_t f[16];
+        dequant_unit(kw[3 * u], kw[3 * u + 1], kw[3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);
+        tc_st16(tmem_g + lane_sel + L::A_COL + 16 * u, f);
+      };
+      // first block of the group in this segment: the whole K tile
+      bool have_block = false;
+      int2 dsc = make_int2(0, -1);
+      if (!failed) {
+        failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
+        dsc = desc[st];
+        if (dsc.y < 0) {  // end marker: the segment has no blocks for this group
+          mbar_arrive(&empty_bar[st]);
+          it++;
+        } else {
+          have_block = true;
+          k_load(stages + st * L::STAGE_BYTES);
 #pragma unroll
-          for (int i = 0; i < L::WPR / 4; i++) {
-            const uint4 t4 = krow[i];
-            w[4 * i] = t4.x; w[4 * i + 1] = t4.y; w[4 * i + 2] = t4.z; w[4 * i + 3] = t4.w;
-          }
-#pragma unroll
-          for (int u = 0; u < 4 * DJ; u++) {
-            uint32_t f[16];
-            dequant_unit(w[3 * u], w[3 * u + 1], w[3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);
-            tc_st16(tmem_g + lane_sel + L::A_COL + 16 * u, f);
-          }
+          for (int u = 0; u < 4 * DJ; u++) k_unit(u);
           tc_wait_st();
           tc_fence_before();
           mbar_arrive(k_ready);
         }
-        // the score MMAs read the tile that the V dequantisation is about to overwrite
-        if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
-
-        // ---- V coordinate gt (+128) of this block -> TMEM lane gt (A_V), interleaved with the softmax of the block: the
-        // lookups load the shift/logic pipe, the softmax the FMA and special-function pipes, and the read-back of the
-        // scores and the group barrier have latencies worth covering.
+      }
+      while (have_block) {
+        const uint8_t* sp = stages + st * L::STAGE_BYTES;
+        const int r0 = dsc.x, n = dsc.y;
+        (void)r0;
+        // ---- V coordinate gt (+128): rows 0..63 now, rows 64..127 with the softmax
         uint32_t wd[DJ][12];
 #pragma unroll
         for (int j = 0; j < DJ; j++) {
@@ -574,17 +584,22 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         }
         const float ksc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES)[gt];
         const float vsc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES)[gt];
-        auto v_unit = [&](int q) {  // unit q of the thread's V coordinates: dequantise and store
-          const int j = q >> 2, u = q & 3;
+        auto v_unit = [&](int j, int u) {  // rows 32u .. 32u+31 of coordinate gt + 128 j
           uint32_t f[16];
           dequant_unit(wd[j][3 * u], wd[j][3 * u + 1], wd[j][3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);
-          tc_st16(tmem_g + lane_sel + L::A_COL + 64 * j + 16 * u, f);
+          const uint32_t col = (u < 2) ? (uint32_t)(L::V_COL + 32 * j + 16 * u) : (uint32_t)(L::A_COL + 64 * j + 16 * (u - 2));
+          tc_st16(tmem_g + lane_sel + col, f);
         };
+#pragma unroll
+        for (int j = 0; j < DJ; j++) { v_unit(j, 0); v_unit(j, 1); }
+
+        // the score MMAs read the K tile that the rest of the V tile is about to overwrite
+        if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
         tc_fence_after();
         uint32_t raw_u[16];
-        tc_ld16_issue(tmem_g + lane_sel + L::S_COL, raw_u);  // scores of row gt: in flight during the first units
+        tc_ld16_issue(tmem_g + lane_sel + L::S_COL, raw_u);  // scores of row gt: in flight during the next unit
 #pragma unroll
-        for (int q = 0; q < 2 * DJ; q++) v_unit(q);
+        for (int j = 0; j < DJ; j++) v_unit(j, 2);
 
         // ---- online softmax (log2 units); thread gt owns row r0 + gt, all 8 heads
         tc_wait_ld();
@@ -627,7 +642,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           }
         }
 #pragma unroll
-        for (int q = 2 * DJ; q < 4 * DJ; q++) v_unit(q);  // the other half of the V units, next to the exponentials
+        for (int j = 0; j < DJ; j++) v_unit(j, 3);  // the last V unit, next to the exponentials
         {
           const float vf = (gt < n) ? vsc * vfac : 0.f;
           float wv[8];
@@ -656,7 +671,20 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         mbar_arrive(p_ready);          // V tile in TMEM, probabilities in shared memory
         mbar_arrive(&empty_bar[st]);   // this thread is done with the staged tile
 
-        // ---- fold the value product into the running accumulator (the value MMAs also release the operand tile)
+        // ---- next slot: its K coordinates that live in the upper half of the operand columns, while the value MMAs run
+        it++;
+        if (++st == NST) { st = 0; st_ph ^= 1u; }
+        if (!failed) failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
+        dsc = failed ? make_int2(0, -1) : desc[st];
+        have_block = dsc.y >= 0;
+        if (have_block) {
+          k_load(stages + st * L::STAGE_BYTES);
+#pragma unroll
+          for (int u = 0; u < 4 * DJ; u++)
+            if (u & 2) k_unit(u);
+        }
+
+        // ---- fold the value product into the running accumulator (the value MMAs also release the lower half)
         if (!failed) failed = !mbar_wait_bounded(o_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
         tc_fence_after();
 #pragma unroll
@@ -667,9 +695,18 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           for (int h = 0; h < 8; h++) acc[j][h] += o[h] + o[8 + h];
         }
         tc_fence_before();
-        it++;
         nbk++;
-        if (++st == NST) { st = 0; st_ph ^= 1u; }
+        if (have_block) {
+#pragma unroll
+          for (int u = 0; u < 4 * DJ; u++)
+            if (!(u & 2)) k_unit(u);
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(k_ready);
+        } else if (!failed) {
+          mbar_arrive(&empty_bar[st]);  // the end marker's slot
+          it++;
+        }
       }
 
       // ---- close the group's part of the segment: reduce l and the exact maximum (and argmax) over the 128 rows and
