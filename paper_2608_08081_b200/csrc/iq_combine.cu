@@ -20,6 +20,12 @@ __global__ void __launch_bounds__(CMB_WARPS * 32) combine_kernel(const CombinePa
   const int S = p.splits;
   const float* ml = p.part_ml + (size_t)bh * S * 2;
 
+  // the rotation block of this lane first: its loads do not depend on the partials and overlap with theirs
+  float M[E / 4][4][4];
+  const float* qb = p.rot + ((size_t)kvh * (D / 4) + (size_t)lane * (E / 4)) * 8;
+#pragma unroll
+  for (int j = 0; j < E / 4; j++) so4_matrix<float>(qb + 8 * j, M[j]);
+
   float m = -INFINITY;
   int best = -1;
   for (int s = 0; s < S; s++) {
@@ -51,10 +57,6 @@ __global__ void __launch_bounds__(CMB_WARPS * 32) combine_kernel(const CombinePa
   for (int e = 0; e < E; e++) v[e] *= inv;
 
   // o = H_d * blockdiag(M_b^T) * o~   (H_d symmetric, R^T = H_d^T R_SO4^T)
-  float M[E / 4][4][4];
-  const float* qb = p.rot + ((size_t)kvh * (D / 4) + (size_t)lane * (E / 4)) * 8;
-#pragma unroll
-  for (int j = 0; j < E / 4; j++) so4_matrix<float>(qb + 8 * j, M[j]);
   so4_apply<float, E, true>(M, v);
   wht_warp<float, E>(v, lane);
   const float inv_root_d = rsqrtf((float)D);

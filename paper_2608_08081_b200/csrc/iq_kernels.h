@@ -8,6 +8,7 @@ namespace iq {
 
 // ---- quantize-append
 constexpr int QA_WARPS = 4;
+constexpr int QA_FEW_ROWS = 4;        // calls with at most this many new rows per sequence take the one-warp-per-row latency path
 constexpr int QA_ROWS_PER_WARP = 16;  // K rows per warp and launch (a warp holds 4 rows at a time at head_dim 128)
 
 struct QuantizeParams {
