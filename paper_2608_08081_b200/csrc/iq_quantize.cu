@@ -469,7 +469,7 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
     }
     const long long t = pos0 + i;
     if (t < 0 || t >= p.t_cap) {
-      if (lane == 0 && !is_v && p.status) {  // counted once per row, by the K warp
+      if (lane == 0 && p.status) {  // counted per (row, KV head, tensor), like the bulk kernels
         atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
         atomicAdd(&p.status[2], 1u);
       }

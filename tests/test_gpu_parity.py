@@ -71,6 +71,26 @@ def test_ragged_batch_with_empty_and_full_sequences(iq, torch, codebooks):
     _roundtrip(iq, torch, codebooks, w, [1, 2, 5, 9], n_new=lens)
 
 
+def test_more_sequences_than_sms_and_than_threads(iq, torch, codebooks):
+    # the decode kernel gives every SM a range of the batch's 128-row blocks: here there are more sequences than CTAs
+    # and than threads of a CTA (each thread then sums several sequences for the range boundaries), many of them empty
+    B = 700
+    g = np.random.Generator(np.random.Philox(77))
+    lens = g.integers(0, 300, B).astype(np.int64)
+    lens[g.integers(0, B, 60)] = 0
+    lens[5] = 300
+    w = workloads.tiny(302, B, 4, 2, 128, 300, lens=[int(x) for x in lens])
+    _roundtrip(iq, torch, codebooks, w, [1, 2, 3], n_new=[int(x) for x in lens])
+
+
+def test_few_slots_for_a_long_sequence_next_to_short_ones(iq, torch, codebooks):
+    # with S = 2 an item may span at most two ranges, which forces ranges longer than an equal share of the blocks;
+    # with S = 7 the long sequence is cut into many pieces and the short ones share ranges with it
+    lens = [5000, 17, 0, 129, 2300]
+    w = workloads.tiny(303, 5, 16, 2, 128, 5000, lens=lens)
+    _roundtrip(iq, torch, codebooks, w, [2, 7, 40], n_new=lens)
+
+
 def test_large_scale_rows_and_zero_rows(iq, torch, codebooks):
     w = workloads.tiny(301, 1, 4, 1, 128, 256, scale=300.0)
     w.k[0, 5] = 0
@@ -120,6 +140,45 @@ def test_append_positions_strides_and_out_of_range_rows(iq, torch, codebooks):
     assert np.array_equal(g["v_codes"], ref["v_codes"])                             # incl. rows never appended (stay zero)
     res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, lens, 2)
     check_decode(w2, lv, w.q, res, g, lens)
+
+
+@pytest.mark.parametrize("d", [128, 256])
+def test_small_appends_take_the_same_codes_as_one_bulk_append(iq, torch, codebooks, d):
+    """Calls with a few new rows per sequence (the decode-step path: one warp per row, V written by read-modify-write
+    into the transposed records) must leave exactly the cache a single bulk append leaves, at every row-in-unit
+    position, with ragged per-sequence counts and rows beyond t_cap skipped and flagged."""
+    T, t_cap = 140, 128
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    w = workloads.tiny(310 + d, 3, 4, 2, d, T)
+    shape = iq.Shape(3, 4, 2, d, t_cap)
+    rot = torch.empty(iq.iq_rotation_floats(d, 2), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, 2, 0, np.ascontiguousarray(w.quats), rot)
+    cache = iq.new_cache(shape)
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    k, v = torch.from_numpy(w.k).cuda(), torch.from_numpy(w.v).cuda()
+    pos = np.zeros(3, np.int64)
+    total = np.array([T, 75, 0])                       # sequence 0 runs 12 rows past t_cap, sequence 2 never appends
+    step = 0
+    while (pos < total).any():
+        nmax = 1 + step % 4                            # 1..4 rows per call
+        n = np.minimum(nmax, total - pos).astype(np.int32)
+        idx = (pos[:, None] + np.arange(nmax)[None, :]).clip(max=T - 1)
+        kk = torch.stack([k[b, idx[b]] for b in range(3)])
+        vv = torch.stack([v[b, idx[b]] for b in range(3)])
+        iq.iq_quantize_append(shape, rot, cb, kk, vv, torch.from_numpy(pos.astype(np.int32)).cuda(),
+                              torch.from_numpy(n).cuda(), nmax, cache, status)
+        pos += n
+        step += 1
+    torch.cuda.synchronize()
+    st = status.cpu().numpy()
+    assert st[0] & 1 and st[2] == 12 * 2 * 2           # 12 rows x 2 KV heads x (K, V) beyond t_cap
+    g = cache_to_numpy(cache)
+    lens = np.array([t_cap, 75, 0], np.int32)
+    ref = oracle.new_cache(3, 2, d, t_cap)
+    oracle.quantize_append(w.quats, th, w.k[:, :t_cap], w.v[:, :t_cap], np.zeros(3, np.int32), lens, ref)
+    w2 = workloads.Workload("x", 3, 4, 2, d, t_cap, w.k[:, :t_cap], w.v[:, :t_cap], w.q, w.quats, lens)
+    compare_caches(w2, th, g, ref, lens)
 
 
 def test_combine_splits_in_isolation(iq, torch, codebooks):
