@@ -325,7 +325,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                 "ms_per_step": round(e2e_ms / max(n_e2e, 1), 4), "steps": n_e2e,
                 "note": "packed cache is device-resident state; per-step inputs (q, new k/v) come from pinned host memory, output returns to host"},
         "quantize_append": st["quantize_append"],
-        "gpu_launches": 4 * K,
+        "gpu_launches": 3 * K,   # per step: quantize_append_few_kernel, decode_kernel, combine_kernel
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
