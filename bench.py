@@ -37,8 +37,8 @@ WORKLOADS = {
 DEFAULT_WORKLOAD = "config5_B32_ctx32768"
 T_CAP_MARGIN = 2048  # rows of head-room so that every sequence can take the benchmark's appends
 
-# DRAM traffic of one decode launch. The ncu capture (profiles/decode_kernel_config5_B8.md; the B = 32 workload is too
-# large to capture with dram counters under the size rule) measured, at B = 8, dram__bytes_read.sum = 1.0031 x the
+# DRAM traffic of one decode launch. The ncu capture of the decode kernel (summarised under profiles/; taken at B = 8
+# because a B = 32 launch is too large for a multi-pass capture) measured dram__bytes_read.sum = 1.0031 x the
 # algorithmic packed-KV bytes of the launch and dram__bytes_write.sum = 7.91 MB for 1.33 MB of partial results
 # (S = 5 slots). Reads scale with the rows processed; writes with the partial results.
 NCU_READ_PER_ALGORITHMIC_BYTE = 182.576 / 182.013
