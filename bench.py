@@ -147,6 +147,9 @@ def aggregate_gbs(bytes_per_rank: float, ms: float, world: int) -> float:
     return world * bytes_per_rank / (ms * 1e-3) / 1e9
 
 
+CODEBOOK = "int8"   # "int8": Lloyd-Max levels on an 8-bit grid (integer tensor-core decode path); "fp16": exact fp16 levels
+
+
 def build_state(name: str, device, rank: int):
     """Synthetic cache for one rank: seeded K/V generated on the GPU in chunks and bulk-quantized (untimed)."""
     import torch
@@ -158,7 +161,7 @@ def build_state(name: str, device, rank: int):
     gen = workloads.config5_device(B, ctx, device, H_q, H_kv, d)
     t_cap = ctx + T_CAP_MARGIN
     shape = iq.Shape(B, H_q, H_kv, d, t_cap)
-    cb = iq.iq_default_codebook(d)
+    cb = iq.iq_int8_codebook(d) if CODEBOOK == "int8" else iq.iq_default_codebook(d)
     rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device=device)
     iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(gen["quats"]), rot)
     cache = iq.new_cache(shape, device)
@@ -412,7 +415,10 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--codebook", default="int8", choices=["int8", "fp16"])
     args = ap.parse_args()
+    global CODEBOOK
+    CODEBOOK = args.codebook
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -115,6 +115,15 @@ size_t iq_rotation_floats(int32_t head_dim, int32_t n_kv_heads);
 int iq_default_codebook(int32_t head_dim, iq_codebook* out_host);
 
 /*
+ * The same Lloyd-Max codebook with its levels snapped to an 8-bit grid: level_j = n_j * delta, n_j integer,
+ * |n_j| <= 127, delta = max|level| / 127 (fp32); thresholds = midpoints of the snapped levels. The snapping moves a
+ * level by at most delta / 2 (0.4 % of the largest level). iq_decode_attention runs codebooks of this form on the
+ * integer tensor-core path (int8 operands, int32 accumulation); any other codebook must have levels that are exact
+ * binary16 values and runs on the fp16 path.
+ */
+int iq_int8_codebook(int32_t head_dim, iq_codebook* out_host);
+
+/*
  * Rotation parameters (Appendix B). If quats_host != NULL it holds [n_kv_heads][d/4][8] floats which are
  * scaled to unit length per quaternion and copied to rot_dev; otherwise the quaternions are drawn on the
  * device from `seed` (4 iid N(0,1) components per quaternion from a counter-based generator, scaled to

@@ -15,6 +15,7 @@ from .binding import (  # noqa: F401
     iq_decode_attention_static,
     iq_static_scratch_bytes,
     iq_default_codebook,
+    iq_int8_codebook,
     iq_make_rotation,
     iq_quantize_append,
     iq_rotation_floats,

@@ -52,6 +52,7 @@ def _load():
     lib.iq_rotation_floats.restype = ctypes.c_size_t
     lib.iq_rotation_floats.argtypes = [_i32, _i32]
     lib.iq_default_codebook.argtypes = [_i32, ctypes.POINTER(_IqCodebook)]
+    lib.iq_int8_codebook.argtypes = [_i32, ctypes.POINTER(_IqCodebook)]
     lib.iq_make_rotation.argtypes = [_i32, _i32, ctypes.c_uint64, _vp, _vp, _vp]
     lib.iq_quantize_append.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp, _vp, _i64, _i64,
                                        _i64, _vp, _vp, _i32, ctypes.POINTER(_IqCache), _vp, _vp]
@@ -141,6 +142,12 @@ def iq_rotation_floats(head_dim: int, n_kv_heads: int) -> int:
 def iq_default_codebook(head_dim: int) -> Codebook:
     cb = _IqCodebook()
     _check(_lib.iq_default_codebook(head_dim, ctypes.byref(cb)), "iq_default_codebook")
+    return Codebook(tuple(cb.levels), tuple(cb.thresholds))
+
+
+def iq_int8_codebook(head_dim: int) -> Codebook:
+    cb = _IqCodebook()
+    _check(_lib.iq_int8_codebook(head_dim, ctypes.byref(cb)), "iq_int8_codebook")
     return Codebook(tuple(cb.levels), tuple(cb.thresholds))
 
 

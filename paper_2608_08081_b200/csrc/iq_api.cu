@@ -38,6 +38,22 @@ int check_codebook(const iq_codebook* cb, bool need_fp16_levels) {
   return IQ_OK;
 }
 
+// Levels on an 8-bit grid: level_j = n_j * delta with integer |n_j| <= 127 and delta = max|level| / 127 (to fp32
+// rounding). Fills n[8] and delta.
+bool int8_grid(const iq_codebook* cb, int (&n)[8], float& delta) {
+  float mx = 0.f;
+  for (int i = 0; i < 8; i++) mx = std::fmax(mx, std::fabs(cb->levels[i]));
+  if (!(mx > 0.f)) return false;
+  delta = mx / 127.0f;
+  for (int i = 0; i < 8; i++) {
+    const double r = (double)cb->levels[i] / (double)delta;
+    const double ri = std::nearbyint(r);
+    if (std::fabs(r - ri) > 1e-4 || std::fabs(ri) > 127.0) return false;
+    n[i] = (int)ri;
+  }
+  return true;
+}
+
 int check_cache(const iq_cache* c) {
   if (!c || !c->k_codes || !c->k_scales || !c->v_codes || !c->v_scales) return IQ_ERR_NULL;
   if (!aligned16(c->k_codes) || !aligned16(c->k_scales) || !aligned16(c->v_codes) || !aligned16(c->v_scales)) return IQ_ERR_ALIGN;
@@ -131,6 +147,24 @@ int iq_default_codebook(int32_t head_dim, iq_codebook* out_host) {
   return IQ_OK;
 }
 
+int iq_int8_codebook(int32_t head_dim, iq_codebook* out_host) {
+  if (!out_host) return IQ_ERR_NULL;
+  if (head_dim != 128 && head_dim != 256) return IQ_ERR_SHAPE;
+  double lv[8];
+  lloyd_max_sphere(head_dim, lv);
+  double a[4];
+  for (int i = 0; i < 4; i++) a[i] = 0.5 * (lv[7 - i] - lv[i]);  // exact symmetry; a[0] is the largest magnitude
+  const float delta = (float)(a[0] / 127.0);
+  for (int i = 0; i < 4; i++) {
+    const float r = (float)std::nearbyint(a[i] / (double)delta) * delta;
+    out_host->levels[7 - i] = r;
+    out_host->levels[i] = -r;
+  }
+  for (int i = 0; i < 7; i++)
+    out_host->thresholds[i] = (float)(0.5 * ((double)out_host->levels[i] + (double)out_host->levels[i + 1]));
+  return IQ_OK;
+}
+
 int iq_make_rotation(int32_t head_dim, int32_t n_kv_heads, uint64_t seed, const float* quats_host, float* rot_dev,
                      void* stream) {
   const size_t nfl = iq_rotation_floats(head_dim, n_kv_heads);
@@ -194,7 +228,11 @@ int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_co
   int rc = check_shape(shape);
   if (rc) return rc;
   if (!rot_dev || !q || !seq_lens_dev || !part_acc || !part_ml) return IQ_ERR_NULL;
-  if ((rc = check_codebook(codebook, true))) return rc;
+  if ((rc = check_codebook(codebook, false))) return rc;
+  int n8[8];
+  float delta = 0.f;
+  const bool grid8 = int8_grid(codebook, n8, delta);  // integer tensor-core path; otherwise the levels must be exact fp16 values
+  if (!grid8 && (rc = check_codebook(codebook, true))) return rc;
   if ((rc = check_cache(cache))) return rc;
   if (num_splits < 1 || num_splits > 65535) return IQ_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(part_acc) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
@@ -228,6 +266,11 @@ int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_co
     p.lut_lo[i >> 2] |= (uint32_t)(bits & 0xFFu) << (8 * (i & 3));
     p.lut_hi[i >> 2] |= (uint32_t)(bits >> 8) << (8 * (i & 3));
   }
+  p.use_i8 = grid8 ? 1 : 0;
+  p.delta = delta;
+  p.lut8[0] = p.lut8[1] = 0u;
+  if (grid8)
+    for (int i = 0; i < 8; i++) p.lut8[i >> 2] |= (uint32_t)(uint8_t)(int8_t)n8[i] << (8 * (i & 3));
   const cudaError_t e = iq::launch_decode_attention(p, shape->head_dim, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }

@@ -34,6 +34,7 @@ constexpr int DEC_GROUP_THREADS = 128;  // 4 warps: dequantisation, softmax, acc
 constexpr uint32_t DEC_WAIT_LIMIT = 1u << 22;
 constexpr int DEC_HDR_BYTES = 4096;    // barriers, TMEM base, work counter, segment and block descriptors, scratch
 constexpr float DEC_MAX_SLACK = 4.0f;  // log2 units a score may exceed the running reference before it is raised
+constexpr float DEC_MAX_SLACK_I8 = 1.0f;  // the same on the integer path, where the probabilities are fixed-point numbers
 
 template <int D>
 struct DecLayout {
@@ -54,6 +55,11 @@ struct DecLayout {
   static constexpr int S_COL = D / 2;
   static constexpr int O_COL = D / 2 + 16;
   static constexpr int V_COL = O_COL + 16 * (D / 128);  // rows 0..63 of the V tile (32 columns per 128 coordinates)
+  // Integer path (int8 operands: 4 elements per column, separate K and V tiles, 32 result columns = 8 heads x 4 digits)
+  static constexpr int I8_K_COL = 0;                   // K tile: d/4 columns
+  static constexpr int I8_V_COL = D / 4;               // V tile: 32 columns per 128 coordinates
+  static constexpr int I8_S_COL = D / 4 + 32 * (D / 128);
+  static constexpr int I8_O_COL = I8_S_COL + 32;       // 32 columns per 128 coordinates
   static constexpr int NG = 512 / GROUP_COLS;  // groups per CTA: 4 at d = 128, 2 at d = 256
   static constexpr int COMPUTE_THREADS = NG * DEC_GROUP_THREADS;
   static constexpr int THREADS = COMPUTE_THREADS + NG * 32;  // + one control warp per group
@@ -61,13 +67,15 @@ struct DecLayout {
   static constexpr int SMEM_BYTES = DEC_HDR_BYTES + BQ_BYTES + NG * GROUP_SMEM;
   // header offsets
   static constexpr int BAR_STRIDE = 96;  // per group: full[3], empty[3], s_bar, o_bar, k_ready, p_ready
-  static constexpr int OFF_TMEM = 384, OFF_NEXT = 388, OFF_SEG = 400, OFF_DESC = 448, OFF_RED = 640, OFF_WALK = 2176;
+  static constexpr int OFF_TMEM = 384, OFF_NEXT = 388, OFF_SEG = 400, OFF_DESC = 448, OFF_QFAC = 576, OFF_RED = 640, OFF_WALK = 2176;
   static constexpr int RED_STRIDE = 384;  // per group: 3 x [4 warps][8 heads] words
 };
 static_assert(DEC_BLOCK_TOKENS == 128, "the TMEM operand layout assumes 128-row blocks");
 static_assert(DecLayout<128>::OFF_RED + 4 * DecLayout<128>::RED_STRIDE <= DEC_HDR_BYTES, "header overflow");
 static_assert(DecLayout<128>::V_COL + 32 * DecLayout<128>::DJ <= DecLayout<128>::GROUP_COLS, "TMEM group overflow");
 static_assert(DecLayout<256>::V_COL + 32 * DecLayout<256>::DJ <= DecLayout<256>::GROUP_COLS, "TMEM group overflow");
+static_assert(DecLayout<128>::I8_O_COL + 32 * DecLayout<128>::DJ <= DecLayout<128>::GROUP_COLS, "TMEM group overflow");
+static_assert(DecLayout<256>::I8_O_COL + 32 * DecLayout<256>::DJ <= DecLayout<256>::GROUP_COLS, "TMEM group overflow");
 static_assert(DecLayout<128>::SMEM_BYTES <= 227 * 1024 && DecLayout<256>::SMEM_BYTES <= 227 * 1024, "shared memory overflow");
 static_assert((DecLayout<128>::THREADS + DecLayout<128>::THREADS / 32) * 4 <= DecLayout<128>::BP_BYTES, "set-up scratch must fit one B_P region");
 
@@ -96,6 +104,11 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&o)[16]) {
 #pragma unroll
   for (int i = 0; i < 16; i++) o[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]),
+               "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
 // The same load without the wait: the registers are valid after tc_wait_ld().
 __device__ __forceinline__ void tc_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
@@ -113,6 +126,14 @@ __device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint32_t a_tmem, uin
       "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0)
       : "memory");
 }
+// D[tmem] (+)= A[tmem] * B[smem descriptor]; int8 operands, int32 accumulate, K = 32 per instruction.
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0)
+      : "memory");
+}
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -123,6 +144,9 @@ __device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, uint32_t lbo, ui
 }
 // Instruction descriptor: D = f32, A = B = f16, A K-major (TMEM), B MN-major, N = 16, M = 128.
 constexpr uint32_t DEC_IDESC = (1u << 4) | (1u << 16) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
+// Integer path: D = s32, A = s8 (K-major, TMEM), B MN-major, N = 32, M = 128; B = s8 (query digits) or u8 (probability digits).
+constexpr uint32_t DEC_IDESC_I8_SS = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t DEC_IDESC_I8_SU = (2u << 4) | (1u << 7) | (0u << 10) | (1u << 16) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
 
 // ---------------------------------------------------------------------------------------------- dequantisation
 // x >> s for a compile-time s, computed as the high word of x * 2^(32-s): the multiply issues on the integer
@@ -152,6 +176,18 @@ __device__ __forceinline__ void dequant_unit(uint32_t w0, uint32_t w1, uint32_t 
       out[4 * k + 2 * hh + 1] = prmt(l, h, 0x7362u);
     }
 }
+
+// Integer path: one packing unit -> 8 registers of four int8 levels each, entries in natural order (one prmt per 4 codes).
+__device__ __forceinline__ void dequant_unit8(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t l0, uint32_t l1, uint32_t (&out)[8]) {
+  const uint32_t sel[4] = {w0 & 0x77777777u, w1 & 0x77777777u, w2 & 0x77777777u, sliced_selectors(w0, w1, w2)};
+#pragma unroll
+  for (int k = 0; k < 4; k++) {
+    out[2 * k] = prmt(l0, l1, sel[k]);
+    out[2 * k + 1] = prmt(l0, l1, shr_mul<16>(sel[k]));
+  }
+}
+// int32 -> float for |x| < 2^22, on the integer and FMA pipes (the conversion instruction runs at a quarter of their rate).
+__device__ __forceinline__ float i2f_small(uint32_t x) { return __uint_as_float(x + 0x4B400000u) - 12582912.0f; }
 
 // One lane of a converged warp. Issuing the MMAs / bulk copies from an elected lane of a converged warp keeps
 // their operands in uniform registers; a lone divergent thread issues the same sequence about 3x slower.
@@ -201,7 +237,7 @@ struct DecWalk {
   long long left, g, item;  // range mode: blocks to go, launch-wide position; whole-item mode: linear item index
 };
 
-template <int D, bool ARGMAX>
+template <int D, bool ARGMAX, bool I8>
 __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const DecodeParams p) {
   using L = DecLayout<D>;
   constexpr int DJ = L::DJ;
@@ -420,15 +456,38 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         for (int e = 0; e < E; e++) v[e] = 0.f;
       }
       const float inv_root_d = rsqrtf((float)D);
+      if constexpr (I8) {
+        // q~ of the head as three balanced base-128 digits (int8) of round(q~ * (2^20 - 1) / max|q~|); the head's factor
+        // max|q~| / (2^20 - 1) * delta * (sm_scale log2 e / sqrt d) goes to shared memory for the score read-back
+        float qmax = 0.f;
 #pragma unroll
-      for (int e = 0; e < E; e++) {
-        const float x = v[e] * inv_root_d;
-        const __half xh = __float2half_rn(x);
-        const __half xl = __float2half_rn(x - __half2float(xh));
-        const int i = lane * E + e;  // contraction index = rotated coordinate
-        const int off = (i & 7) * 16 + (i >> 3) * 128;
-        *reinterpret_cast<__half*>(bq + hh * 2 + off) = xh;                  // n = head (hi part)
-        *reinterpret_cast<__half*>(bq + hh * 2 + (D / 8) * 128 + off) = xl;  // n = 8 + head (lo part)
+        for (int e = 0; e < E; e++) qmax = fmaxf(qmax, fabsf(v[e] * inv_root_d));
+        qmax = warp_max(qmax);
+        const float qs = qmax > 0.f ? 1048575.0f / qmax : 0.f;
+#pragma unroll
+        for (int e = 0; e < E; e++) {
+          const int Q = __float2int_rn(v[e] * inv_root_d * qs);
+          const int d2 = (Q + 8192) >> 14;
+          const int r = Q - (d2 << 14);
+          const int d1 = (r + 64) >> 7;
+          const int d0 = r - (d1 << 7);
+          const int i = lane * E + e;  // contraction index = rotated coordinate; column n = 4 * head + digit
+          const uint32_t word = (uint32_t)(d0 & 0xff) | ((uint32_t)(d1 & 0xff) << 8) | ((uint32_t)(d2 & 0xff) << 16);
+          *reinterpret_cast<uint32_t*>(bq + 4 * (hh & 3) + (hh >> 2) * ((D / 8) * 128) + (i & 7) * 16 + (i >> 3) * 128) = word;
+        }
+        if (lane == 0)
+          reinterpret_cast<float*>(smem + L::OFF_QFAC)[hh] = (qmax * (1.0f / 1048575.0f)) * p.delta * (p.sm_scale * LOG2E * inv_root_d);
+      } else {
+#pragma unroll
+        for (int e = 0; e < E; e++) {
+          const float x = v[e] * inv_root_d;
+          const __half xh = __float2half_rn(x);
+          const __half xl = __float2half_rn(x - __half2float(xh));
+          const int i = lane * E + e;  // contraction index = rotated coordinate
+          const int off = (i & 7) * 16 + (i >> 3) * 128;
+          *reinterpret_cast<__half*>(bq + hh * 2 + off) = xh;                  // n = head (hi part)
+          *reinterpret_cast<__half*>(bq + hh * 2 + (D / 8) * 128 + off) = xl;  // n = 8 + head (lo part)
+        }
       }
       fence_proxy_async();  // B_Q is written through the generic proxy and read by the tensor core through the async proxy
     }
@@ -481,9 +540,16 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         if (!failed) failed = !mbar_wait_bounded(k_ready, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
         tc_fence_after();
         if (elect_one()) {
+          if constexpr (I8) {
 #pragma unroll
-          for (int kk = 0; kk < D / 16; kk++)
-            tc_mma_f16(tmem_g + L::S_COL, tmem_g + L::A_COL + 8 * kk, smem_desc_mn(bq_addr + kk * 256, 128, (D / 8) * 128), DEC_IDESC, kk > 0);
+            for (int kk = 0; kk < D / 32; kk++)
+              tc_mma_i8(tmem_g + L::I8_S_COL, tmem_g + L::I8_K_COL + 8 * kk, smem_desc_mn(bq_addr + kk * 512, 128, (D / 8) * 128),
+                        DEC_IDESC_I8_SS, kk > 0);
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < D / 16; kk++)
+              tc_mma_f16(tmem_g + L::S_COL, tmem_g + L::A_COL + 8 * kk, smem_desc_mn(bq_addr + kk * 256, 128, (D / 8) * 128), DEC_IDESC, kk > 0);
+          }
           tc_commit(s_bar);
         }
         __syncwarp();
@@ -491,13 +557,22 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         if (!failed) failed = !mbar_wait_bounded(p_ready, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
         tc_fence_after();
         if (elect_one()) {
+          if constexpr (I8) {
 #pragma unroll
-          for (int j = 0; j < DJ; j++)
+            for (int j = 0; j < DJ; j++)
 #pragma unroll
-            for (int kk = 0; kk < TB / 16; kk++)
-              tc_mma_f16(tmem_g + L::O_COL + 16 * j,  // rows 0..63 of the V tile sit in V_COL, rows 64..127 in the operand columns
-                         tmem_g + (kk < 4 ? L::V_COL + 32 * j + 8 * kk : L::A_COL + 64 * j + 8 * (kk - 4)),
-                         smem_desc_mn(bp_addr + kk * 256, 128, (TB / 8) * 128), DEC_IDESC, kk > 0);
+              for (int kk = 0; kk < TB / 32; kk++)
+                tc_mma_i8(tmem_g + L::I8_O_COL + 32 * j, tmem_g + L::I8_V_COL + 32 * j + 8 * kk,
+                          smem_desc_mn(bp_addr + kk * 512, 128, (TB / 8) * 128), DEC_IDESC_I8_SU, kk > 0);
+          } else {
+#pragma unroll
+            for (int j = 0; j < DJ; j++)
+#pragma unroll
+              for (int kk = 0; kk < TB / 16; kk++)
+                tc_mma_f16(tmem_g + L::O_COL + 16 * j,  // rows 0..63 of the V tile sit in V_COL, rows 64..127 in the operand columns
+                           tmem_g + (kk < 4 ? L::V_COL + 32 * j + 8 * kk : L::A_COL + 64 * j + 8 * (kk - 4)),
+                           smem_desc_mn(bp_addr + kk * 256, 128, (TB / 8) * 128), DEC_IDESC, kk > 0);
+          }
           tc_commit(o_bar);
         }
         __syncwarp();
@@ -525,6 +600,179 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 #pragma unroll
       for (int h = 0; h < 8; h++) { m_run[h] = -INFINITY; l_run[h] = 0.f; best_v[h] = -INFINITY; best_i[h] = -1; }
 
+      if constexpr (I8) {
+      // Integer path. The group's TMEM columns: K tile (d/4), V tile (32 per 128 coordinates), scores (32 = 8 heads x 4
+      // digit columns), values (32 per 128 coordinates). The tiles do not share columns: the V tile of a block is
+      // dequantised while its score MMAs run, the K tile of the next block while its value MMAs run.
+      int st = it % NST;                      // stage of slot `it` and its phase, kept incrementally
+      uint32_t st_ph = (uint32_t)(it / NST) & 1u;
+      const uint32_t l8_0 = p.lut8[0], l8_1 = p.lut8[1];
+      const float* qfac = reinterpret_cast<const float*>(smem + L::OFF_QFAC);  // per head: digits -> log2-domain score per unit K scale
+      float vref = 0.f;    // power of two >= every V scale (x 1/sqrt d) seen by the group in this segment
+      float pscale = 0.f;  // probabilities are written as round(p * vscale * pscale) < 2^23: pscale = 2^21 / vref
+      auto k_tile = [&](const uint8_t* sp_) {  // K row gt of the staged tile -> TMEM lane gt, then signal the control warp
+        uint32_t kw[L::WPR];
+        const uint4* krow = reinterpret_cast<const uint4*>(sp_ + gt * L::ROWB);
+#pragma unroll
+        for (int i = 0; i < L::WPR / 4; i++) {
+          const uint4 t4 = krow[i];
+          kw[4 * i] = t4.x; kw[4 * i + 1] = t4.y; kw[4 * i + 2] = t4.z; kw[4 * i + 3] = t4.w;
+        }
+#pragma unroll
+        for (int u = 0; u < 4 * DJ; u++) {
+          uint32_t f[8];
+          dequant_unit8(kw[3 * u], kw[3 * u + 1], kw[3 * u + 2], l8_0, l8_1, f);
+          tc_st8(tmem_g + lane_sel + L::I8_K_COL + 8 * u, f);
+        }
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(k_ready);
+      };
+      bool have_block = false;
+      int2 dsc = make_int2(0, -1);
+      if (!failed) {
+        failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
+        dsc = desc[st];
+        if (dsc.y < 0) {  // end marker: the segment has no blocks for this group
+          mbar_arrive(&empty_bar[st]);
+          it++;
+        } else {
+          have_block = true;
+          k_tile(stages + st * L::STAGE_BYTES);
+        }
+      }
+      while (have_block) {
+        const uint8_t* sp = stages + st * L::STAGE_BYTES;
+        const int r0 = dsc.x, n = dsc.y;
+        (void)r0;
+        // ---- V coordinate gt (+128) of this block -> TMEM lane gt, while the score MMAs run
+#pragma unroll
+        for (int j = 0; j < DJ; j++) {
+          const uint4* vrow = reinterpret_cast<const uint4*>(sp + L::K_BYTES + (gt + 128 * j) * 48);
+          uint32_t wd[12];
+#pragma unroll
+          for (int i = 0; i < 3; i++) {
+            const uint4 t4 = vrow[i];
+            wd[4 * i] = t4.x; wd[4 * i + 1] = t4.y; wd[4 * i + 2] = t4.z; wd[4 * i + 3] = t4.w;
+          }
+#pragma unroll
+          for (int u = 0; u < 4; u++) {
+            uint32_t f[8];
+            dequant_unit8(wd[3 * u], wd[3 * u + 1], wd[3 * u + 2], l8_0, l8_1, f);
+            tc_st8(tmem_g + lane_sel + L::I8_V_COL + 32 * j + 8 * u, f);
+          }
+        }
+        const float ksc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES)[gt];
+        const float vsc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES)[gt];
+        const bool valid = gt < n;  // rows >= n of the last block hold stale bytes
+        const float kf = valid ? ksc : 0.f;
+        const float mask = valid ? 0.f : -INFINITY;  // stale rows: 0 * finite - inf = -inf
+        const float vf = valid ? vsc * vfac : 0.f;
+
+        // ---- scores: three int32 digit columns per head -> log2-domain score of row gt
+        if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
+        tc_fence_after();
+        float s[8];
+#pragma unroll
+        for (int half = 0; half < 2; half++) {
+          uint32_t raw_u[16];
+          tc_ld16_issue(tmem_g + lane_sel + L::I8_S_COL + 16 * half, raw_u);
+          tc_wait_ld();
+#pragma unroll
+          for (int hq = 0; hq < 4; hq++) {
+            const float sf = fmaf(fmaf(i2f_small(raw_u[4 * hq + 2]), 128.f, i2f_small(raw_u[4 * hq + 1])), 128.f, i2f_small(raw_u[4 * hq]));
+            s[4 * half + hq] = fmaf(sf * qfac[4 * half + hq], kf, mask);
+          }
+        }
+        if (ARGMAX) {  // exact maximum seen by this thread and its row (a group sees its blocks in ascending order)
+#pragma unroll
+          for (int h = 0; h < 8; h++)
+            if (s[h] > best_v[h]) { best_v[h] = s[h]; best_i[h] = r0 + gt; }
+        }
+        // The running reference m_run is raised when a score exceeds it by more than one log2 unit, the V-scale bound vref
+        // when a row exceeds it: both are rare after the first blocks (one barrier with an OR reduction otherwise).
+        float over[8];
+#pragma unroll
+        for (int h = 0; h < 8; h++) over[h] = s[h] - m_run[h];  // NaN (-inf - -inf) for a stale row of an unopened reference: max ignores it
+        const bool exceed = max3f(max3f(over[0], over[1], over[2]), max3f(over[3], over[4], over[5]), fmaxf(over[6], over[7])) > DEC_MAX_SLACK_I8 ||
+                            vf > vref;
+        if (group_bar_or(bar_id, exceed)) {
+#pragma unroll
+          for (int h = 0; h < 8; h++) {
+            const float wm = warp_max(s[h]);
+            if (lane == h) red[(warp & 3) * 8 + h] = wm;
+          }
+          const float wv_max = warp_max(vf);
+          if (lane == 0) red2[warp & 3] = wv_max;
+          group_bar_sync(bar_id);
+#pragma unroll
+          for (int h = 0; h < 8; h++) {
+            const float bm = fmaxf(fmaxf(red[h], red[8 + h]), fmaxf(red[16 + h], red[24 + h]));
+            const float mn = fmaxf(m_run[h], bm);
+            const float alpha = ex2f(m_run[h] - mn);  // the accumulator holds the blocks before this one: rescale it now
+            m_run[h] = mn;
+            l_run[h] *= alpha;
+#pragma unroll
+            for (int j = 0; j < DJ; j++) acc[j][h] *= alpha;
+          }
+          const float bv = fmaxf(fmaxf(red2[0], red2[1]), fmaxf(red2[2], red2[3]));
+          if (bv > vref) vref = __uint_as_float((__float_as_uint(bv) + 0x007FFFFFu) & 0x7F800000u);  // next power of two
+          pscale = vref > 0.f ? 2097152.0f / vref : 0.f;
+        }
+        {
+          // probabilities (times scale_V / sqrt(d)) as 23-bit fixed point: the bytes of the float p * pscale + 2^23 are the base-256
+          // digits of round(p * pscale) (byte 3 is the float's exponent: its result column is ignored). B_P[n][row], n = 4 head + digit.
+          uint32_t pb[8];
+#pragma unroll
+          for (int h = 0; h < 8; h++) {
+            const float pr = ex2f(s[h] - m_run[h]);
+            l_run[h] += pr;
+            pb[h] = __float_as_uint(fmaf(pr * vf, pscale, 8388608.0f));
+          }
+          const int off = (gt & 7) * 16 + (gt >> 3) * 128;
+          *reinterpret_cast<uint4*>(bp + off) = make_uint4(pb[0], pb[1], pb[2], pb[3]);
+          *reinterpret_cast<uint4*>(bp + (TB / 8) * 128 + off) = make_uint4(pb[4], pb[5], pb[6], pb[7]);
+          fence_proxy_async();
+        }
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(p_ready);          // V tile in TMEM, probabilities in shared memory
+        mbar_arrive(&empty_bar[st]);   // this thread is done with the staged tile
+        const float ofac = p.delta * vref * (1.0f / 2097152.0f);  // value digits -> real units: delta / pscale
+
+        // ---- next slot: its K tile, while the value MMAs run
+        it++;
+        if (++st == NST) { st = 0; st_ph ^= 1u; }
+        if (!failed) failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
+        dsc = failed ? make_int2(0, -1) : desc[st];
+        have_block = dsc.y >= 0;
+        if (have_block) k_tile(stages + st * L::STAGE_BYTES);
+
+        // ---- fold the value product into the running accumulator
+        if (!failed) failed = !mbar_wait_bounded(o_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
+        tc_fence_after();
+#pragma unroll
+        for (int j = 0; j < DJ; j++)
+#pragma unroll
+          for (int half = 0; half < 2; half++) {
+            uint32_t o_u[16];
+            tc_ld16_issue(tmem_g + lane_sel + L::I8_O_COL + 32 * j + 16 * half, o_u);
+            tc_wait_ld();
+#pragma unroll
+            for (int hq = 0; hq < 4; hq++) {
+              const float of = fmaf(fmaf(i2f_small(o_u[4 * hq + 2]), 256.f, i2f_small(o_u[4 * hq + 1])), 256.f, i2f_small(o_u[4 * hq]));
+              acc[j][4 * half + hq] = fmaf(of, ofac, acc[j][4 * half + hq]);
+            }
+          }
+        tc_fence_before();
+        nbk++;
+        if (!have_block && !failed) {
+          mbar_arrive(&empty_bar[st]);  // the end marker's slot
+          it++;
+        }
+      }
+
+      } else {
       // The group's 128 TMEM columns: [0, 64 DJ) operand tile, then scores, values, and V_COL.. a second home for the first
       // half of the V tile. Schedule of one block (K tile complete, k_ready signalled):
       //   V rows 0..63 -> V_COL columns               while the score MMAs read the K tile
@@ -709,6 +957,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         }
       }
 
+      }
       // ---- close the group's part of the segment: reduce l and the exact maximum (and argmax) over the 128 rows and
       // leave the group partial in the group's (drained) staging buffer for the merge
 #pragma unroll
@@ -803,7 +1052,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
   if (warp == NG * 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
 }
 
-template <int D, bool ARGMAX>
+template <int D, bool ARGMAX, bool I8>
 static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
   using L = DecLayout<D>;
   static bool configured[64] = {};
@@ -812,7 +1061,7 @@ static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  auto kern = decode_kernel<D, ARGMAX>;
+  auto kern = decode_kernel<D, ARGMAX, I8>;
   if (!configured[dev]) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::SMEM_BYTES);
     if (e != cudaSuccess) return e;
@@ -831,8 +1080,12 @@ static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
 
 cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream) {
   const bool am = p.part_argmax != nullptr;
-  if (head_dim == 128) return am ? launch_one<128, true>(p, stream) : launch_one<128, false>(p, stream);
-  return am ? launch_one<256, true>(p, stream) : launch_one<256, false>(p, stream);
+  if (p.use_i8) {  // levels on an 8-bit grid: int8 operands, int32 accumulation
+    if (head_dim == 128) return am ? launch_one<128, true, true>(p, stream) : launch_one<128, false, true>(p, stream);
+    return am ? launch_one<256, true, true>(p, stream) : launch_one<256, false, true>(p, stream);
+  }
+  if (head_dim == 128) return am ? launch_one<128, true, false>(p, stream) : launch_one<128, false, false>(p, stream);
+  return am ? launch_one<256, true, false>(p, stream) : launch_one<256, false, false>(p, stream);
 }
 
 // CTAs the decode kernel keeps resident per SM (it sizes its grid as one CTA per SM).

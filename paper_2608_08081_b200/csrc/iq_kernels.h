@@ -48,6 +48,10 @@ struct DecodeParams {
   int batch, n_q_heads, n_kv_heads, group, head_groups, t_cap, splits;
   float sm_scale;
   uint32_t lut_lo[2], lut_hi[2];  // low / high bytes of the 8 fp16 levels, 4 per register
+  // integer path (levels on an 8-bit grid): level_j = lut8 byte j (int8) * delta
+  uint32_t lut8[2];
+  float delta;
+  int use_i8;
 };
 cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream);
 int decode_ctas_per_sm(int head_dim);

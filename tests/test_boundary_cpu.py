@@ -35,7 +35,7 @@ def test_sizes(iq):
 
 def test_default_codebook_matches_oracle_tool(iq, codebooks):
     for d in (128, 256):
-        cb = iq.iq_default_codebook(d)
+        cb = iq.iq_default_codebook(d) if codebooks["kind"] == "fp16" else iq.iq_int8_codebook(d)
         lv, th = codebooks[d]
         assert np.array_equal(np.array(cb.levels, np.float32), lv)      # two independent Lloyd-Max implementations
         assert np.allclose(np.array(cb.thresholds, np.float32), th, atol=0)

@@ -163,9 +163,24 @@ def test_lloyd_max_is_a_fixed_point_for_the_sphere_marginal(d):
 
 
 def test_codebook_as_handed_to_both_sides(codebooks):
-    for d, (lv, th) in codebooks.items():
+    from oracle import lloyd_max
+    for d in (128, 256):
+        lv, th = codebooks[d]
         assert lv.dtype == np.float32 and th.dtype == np.float32
-        assert np.array_equal(lv.astype(np.float16).astype(np.float32), lv)      # exactly fp16-representable
+        if codebooks["kind"] == "fp16":
+            assert np.array_equal(lv.astype(np.float16).astype(np.float32), lv)  # exactly fp16-representable
+        else:                                                                    # integer multiples of max / 127
+            delta = np.float32(lv[-1]) / np.float32(127.0)
+            n = lv.astype(np.float64) / np.float64(delta)
+            assert np.allclose(n, np.rint(n), atol=1e-4) and np.abs(np.rint(n)).max() == 127
+            exact, _, mse = lloyd_max.lloyd_max(d)
+            assert np.abs(lv - exact).max() <= 0.5 * delta * 1.0001              # each level moved by at most half a grid step
+            pdf = lambda u: (1 - u * u / d) ** ((d - 3) / 2) if u * u < d else 0.0
+            from scipy import integrate
+            edges = np.concatenate(([-np.sqrt(d)], th.astype(np.float64), [np.sqrt(d)]))
+            tot = integrate.quad(pdf, -np.sqrt(d), np.sqrt(d))[0]
+            mse8 = sum(integrate.quad(lambda u: (u - lv[i]) ** 2 * pdf(u), edges[i], edges[i + 1])[0] for i in range(8)) / tot
+            assert mse8 <= mse * 1.002                                           # the snapping costs < 0.2 % of the distortion
         assert np.all(np.diff(lv) > 0) and np.all(np.diff(th) > 0) and th[3] == 0
 
 
