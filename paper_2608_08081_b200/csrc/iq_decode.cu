@@ -208,6 +208,8 @@ __device__ __forceinline__ bool group_bar_or(int id, bool pred) {
 }
 // Barrier 0 over the whole CTA, for the places where the control and the compute warps arrive from different code.
 __device__ __forceinline__ void cta_bar_sync() { asm volatile("barrier.sync 0;" ::: "memory"); }
+// Named barrier `id` over `count` threads (a multiple of 32).
+__device__ __forceinline__ void cta_bar_sync_n(int id, int count) { asm volatile("barrier.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 __device__ __forceinline__ void group_bar_sync(int id) { asm volatile("barrier.sync %0, 128;" ::"r"(id) : "memory"); }
 
 __device__ __forceinline__ float max3f(float a, float b, float c) {
@@ -254,6 +256,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
   const int grp = control ? warp - NG * 4 : warp >> 2;  // group of this warp
   const int gt = tid & (DEC_GROUP_THREADS - 1);         // compute thread within its group = TMEM lane
   const int bar_id = 1 + grp;                           // named barrier of the group's compute threads
+  constexpr int HEADS_BAR = 8;                          // named barrier of the eight warps that rotate the query heads
 
   uint64_t* gbar = reinterpret_cast<uint64_t*>(smem + grp * L::BAR_STRIDE);
   uint64_t* full_bar = gbar;        // [stages] tile landed (or end marker)
@@ -457,12 +460,18 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
       }
       const float inv_root_d = rsqrtf((float)D);
       if constexpr (I8) {
-        // q~ of the head as three balanced base-128 digits (int8) of round(q~ * (2^20 - 1) / max|q~|); the head's factor
-        // max|q~| / (2^20 - 1) * delta * (sm_scale log2 e / sqrt d) goes to shared memory for the score read-back
+        // q~ as three balanced base-128 digits (int8) of round(q~ * (2^20 - 1) / qmax), qmax = max |q~| over the item's
+        // heads: one scale for all heads, so that the score read-back needs a single factor. (Two base-256 digits would
+        // halve the read-back, but 16 bits are not enough for lse at the logit magnitudes of outlier rows.)
         float qmax = 0.f;
 #pragma unroll
         for (int e = 0; e < E; e++) qmax = fmaxf(qmax, fabsf(v[e] * inv_root_d));
         qmax = warp_max(qmax);
+        float* qtmp = reinterpret_cast<float*>(smem + L::OFF_QFAC);  // [8] per-head maxima, then [8] = the common factor
+        if (lane == 0) qtmp[hh] = qmax;
+        cta_bar_sync_n(HEADS_BAR, DEC_HEADS * 32);
+#pragma unroll
+        for (int h2 = 0; h2 < DEC_HEADS; h2++) qmax = fmaxf(qmax, qtmp[h2]);
         const float qs = qmax > 0.f ? 1048575.0f / qmax : 0.f;
 #pragma unroll
         for (int e = 0; e < E; e++) {
@@ -475,8 +484,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           const uint32_t word = (uint32_t)(d0 & 0xff) | ((uint32_t)(d1 & 0xff) << 8) | ((uint32_t)(d2 & 0xff) << 16);
           *reinterpret_cast<uint32_t*>(bq + 4 * (hh & 3) + (hh >> 2) * ((D / 8) * 128) + (i & 7) * 16 + (i >> 3) * 128) = word;
         }
-        if (lane == 0)
-          reinterpret_cast<float*>(smem + L::OFF_QFAC)[hh] = (qmax * (1.0f / 1048575.0f)) * p.delta * (p.sm_scale * LOG2E * inv_root_d);
+        if (hh == 0 && lane == 0)  // digits -> log2-domain score per unit K scale
+          qtmp[8] = (qmax * (1.0f / 1048575.0f)) * p.delta * (p.sm_scale * LOG2E * inv_root_d);
       } else {
 #pragma unroll
         for (int e = 0; e < E; e++) {
@@ -607,7 +616,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
       int st = it % NST;                      // stage of slot `it` and its phase, kept incrementally
       uint32_t st_ph = (uint32_t)(it / NST) & 1u;
       const uint32_t l8_0 = p.lut8[0], l8_1 = p.lut8[1];
-      const float* qfac = reinterpret_cast<const float*>(smem + L::OFF_QFAC);  // per head: digits -> log2-domain score per unit K scale
+      const float sfac = reinterpret_cast<const float*>(smem + L::OFF_QFAC)[8];  // score digits -> log2-domain score per unit K scale
       float vref = 0.f;    // power of two >= every V scale (x 1/sqrt d) seen by the group in this segment
       float pscale = 0.f;  // probabilities are written as round(p * vscale * pscale) < 2^23: pscale = 2^21 / vref
       auto k_tile = [&](const uint8_t* sp_) {  // K row gt of the staged tile -> TMEM lane gt, then signal the control warp
@@ -665,7 +674,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         const float ksc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES)[gt];
         const float vsc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES)[gt];
         const bool valid = gt < n;  // rows >= n of the last block hold stale bytes
-        const float kf = valid ? ksc : 0.f;
+        const float kfs = valid ? ksc * sfac : 0.f;
         const float mask = valid ? 0.f : -INFINITY;  // stale rows: 0 * finite - inf = -inf
         const float vf = valid ? vsc * vfac : 0.f;
 
@@ -679,9 +688,9 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           tc_ld16_issue(tmem_g + lane_sel + L::I8_S_COL + 16 * half, raw_u);
           tc_wait_ld();
 #pragma unroll
-          for (int hq = 0; hq < 4; hq++) {
-            const float sf = fmaf(fmaf(i2f_small(raw_u[4 * hq + 2]), 128.f, i2f_small(raw_u[4 * hq + 1])), 128.f, i2f_small(raw_u[4 * hq]));
-            s[4 * half + hq] = fmaf(sf * qfac[4 * half + hq], kf, mask);
+          for (int hq = 0; hq < 4; hq++) {  // S = S0 + 128 (S1 + 128 S2): the upper two digits combine in an int32
+            const float hi = __int2float_rn((int)raw_u[4 * hq + 2] * 128 + (int)raw_u[4 * hq + 1]);
+            s[4 * half + hq] = fmaf(fmaf(hi, 128.f, i2f_small(raw_u[4 * hq])), kfs, mask);
           }
         }
         if (ARGMAX) {  // exact maximum seen by this thread and its row (a group sees its blocks in ascending order)
@@ -723,11 +732,12 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           // probabilities (times scale_V / sqrt(d)) as 23-bit fixed point: the bytes of the float p * pscale + 2^23 are the base-256
           // digits of round(p * pscale) (byte 3 is the float's exponent: its result column is ignored). B_P[n][row], n = 4 head + digit.
           uint32_t pb[8];
+          const float vfp = vf * pscale;
 #pragma unroll
           for (int h = 0; h < 8; h++) {
             const float pr = ex2f(s[h] - m_run[h]);
             l_run[h] += pr;
-            pb[h] = __float_as_uint(fmaf(pr * vf, pscale, 8388608.0f));
+            pb[h] = __float_as_uint(fmaf(pr, vfp, 8388608.0f));
           }
           const int off = (gt & 7) * 16 + (gt >> 3) * 128;
           *reinterpret_cast<uint4*>(bp + off) = make_uint4(pb[0], pb[1], pb[2], pb[3]);
@@ -760,7 +770,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
             tc_wait_ld();
 #pragma unroll
             for (int hq = 0; hq < 4; hq++) {
-              const float of = fmaf(fmaf(i2f_small(o_u[4 * hq + 2]), 256.f, i2f_small(o_u[4 * hq + 1])), 256.f, i2f_small(o_u[4 * hq]));
+              const float of = fmaf(i2f_small(o_u[4 * hq + 2]), 65536.f, __int2float_rn((int)o_u[4 * hq + 1] * 256 + (int)o_u[4 * hq]));
               acc[j][4 * half + hq] = fmaf(of, ofac, acc[j][4 * half + hq]);
             }
           }
