@@ -67,7 +67,7 @@ struct DecLayout {
   static constexpr int SMEM_BYTES = DEC_HDR_BYTES + BQ_BYTES + NG * GROUP_SMEM;
   // header offsets
   static constexpr int BAR_STRIDE = 96;  // per group: full[3], empty[3], s_bar, o_bar, k_ready, p_ready
-  static constexpr int OFF_TMEM = 384, OFF_NEXT = 388, OFF_SEG = 400, OFF_DESC = 448, OFF_QFAC = 576, OFF_RED = 640, OFF_WALK = 2176;
+  static constexpr int OFF_TMEM = 384, OFF_NEXT = 388, OFF_SEG = 400, OFF_DESC = 448, OFF_ACCF = 544, OFF_QFAC = 576, OFF_RED = 640, OFF_WALK = 2176;
   static constexpr int RED_STRIDE = 384;  // per group: 3 x [4 warps][8 heads] words
 };
 static_assert(DEC_BLOCK_TOKENS == 128, "the TMEM operand layout assumes 128-row blocks");
@@ -565,14 +565,15 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         // values: O = A_V * B_P^T once the V tile is in TMEM and the probabilities are in shared memory
         if (!failed) failed = !mbar_wait_bounded(p_ready, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
         tc_fence_after();
+        const bool keep_values = I8 && *reinterpret_cast<volatile int*>(smem + L::OFF_ACCF + 4 * grp) != 0;
         if (elect_one()) {
           if constexpr (I8) {
 #pragma unroll
             for (int j = 0; j < DJ; j++)
 #pragma unroll
-              for (int kk = 0; kk < TB / 32; kk++)
+              for (int kk = 0; kk < TB / 32; kk++)  // the values stay in TMEM (int32) over the blocks until the compute threads read them
                 tc_mma_i8(tmem_g + L::I8_O_COL + 32 * j, tmem_g + L::I8_V_COL + 32 * j + 8 * kk,
-                          smem_desc_mn(bp_addr + kk * 512, 128, (TB / 8) * 128), DEC_IDESC_I8_SU, kk > 0);
+                          smem_desc_mn(bp_addr + kk * 512, 128, (TB / 8) * 128), DEC_IDESC_I8_SU, (kk > 0) || keep_values);
           } else {
 #pragma unroll
             for (int j = 0; j < DJ; j++)
@@ -619,6 +620,31 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
       const float sfac = reinterpret_cast<const float*>(smem + L::OFF_QFAC)[8];  // score digits -> log2-domain score per unit K scale
       float vref = 0.f;    // power of two >= every V scale (x 1/sqrt d) seen by the group in this segment
       float pscale = 0.f;  // probabilities are written as round(p * vscale * pscale) < 2^23: pscale = 2^21 / vref
+      // The value products of consecutive blocks accumulate in TMEM as int32 (exact) for as long as the references they are
+      // relative to (m_run, vref) stand; nacc counts the blocks in there. A block adds at most 128 * 127 * 255 < 2^22 per
+      // column, so 384 blocks stay below 2^31. flush() adds the accumulated digits to the float accumulator.
+      int nacc = 0;
+      int* accf = reinterpret_cast<int*>(smem + L::OFF_ACCF + 4 * grp);  // tells the control warp to accumulate onto TMEM
+      auto flush = [&]() {
+        const float ofac = p.delta * vref * (1.0f / 2097152.0f);  // value digits -> real units: delta / pscale
+        tc_fence_after();
+#pragma unroll
+        for (int j = 0; j < DJ; j++)
+#pragma unroll
+          for (int half = 0; half < 2; half++) {
+            uint32_t o_u[16];
+            tc_ld16_issue(tmem_g + lane_sel + L::I8_O_COL + 32 * j + 16 * half, o_u);
+            tc_wait_ld();
+#pragma unroll
+            for (int hq = 0; hq < 4; hq++) {
+              const float of = fmaf(fmaf(__int2float_rn((int)o_u[4 * hq + 2]), 256.f, __int2float_rn((int)o_u[4 * hq + 1])), 256.f,
+                                    __int2float_rn((int)o_u[4 * hq]));
+              acc[j][4 * half + hq] = fmaf(of, ofac, acc[j][4 * half + hq]);
+            }
+          }
+        tc_fence_before();
+        nacc = 0;
+      };
       auto k_tile = [&](const uint8_t* sp_) {  // K row gt of the staged tile -> TMEM lane gt, then signal the control warp
         uint32_t kw[L::WPR];
         const uint4* krow = reinterpret_cast<const uint4*>(sp_ + gt * L::ROWB);
@@ -682,16 +708,21 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
         tc_fence_after();
         float s[8];
+        {
+          auto digits_to_scores = [&](const uint32_t (&raw_u)[16], int half) {
 #pragma unroll
-        for (int half = 0; half < 2; half++) {
-          uint32_t raw_u[16];
-          tc_ld16_issue(tmem_g + lane_sel + L::I8_S_COL + 16 * half, raw_u);
+            for (int hq = 0; hq < 4; hq++) {  // S = S0 + 128 (S1 + 128 S2): the upper two digits combine in an int32
+              const float hi = __int2float_rn((int)raw_u[4 * hq + 2] * 128 + (int)raw_u[4 * hq + 1]);
+              s[4 * half + hq] = fmaf(fmaf(hi, 128.f, i2f_small(raw_u[4 * hq])), kfs, mask);
+            }
+          };
+          uint32_t raw0[16], raw1[16];
+          tc_ld16_issue(tmem_g + lane_sel + L::I8_S_COL, raw0);
           tc_wait_ld();
-#pragma unroll
-          for (int hq = 0; hq < 4; hq++) {  // S = S0 + 128 (S1 + 128 S2): the upper two digits combine in an int32
-            const float hi = __int2float_rn((int)raw_u[4 * hq + 2] * 128 + (int)raw_u[4 * hq + 1]);
-            s[4 * half + hq] = fmaf(fmaf(hi, 128.f, i2f_small(raw_u[4 * hq])), kfs, mask);
-          }
+          tc_ld16_issue(tmem_g + lane_sel + L::I8_S_COL + 16, raw1);  // heads 4..7 in flight while heads 0..3 are converted
+          digits_to_scores(raw0, 0);
+          tc_wait_ld();
+          digits_to_scores(raw1, 1);
         }
         if (ARGMAX) {  // exact maximum seen by this thread and its row (a group sees its blocks in ascending order)
 #pragma unroll
@@ -704,8 +735,9 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 #pragma unroll
         for (int h = 0; h < 8; h++) over[h] = s[h] - m_run[h];  // NaN (-inf - -inf) for a stale row of an unopened reference: max ignores it
         const bool exceed = max3f(max3f(over[0], over[1], over[2]), max3f(over[3], over[4], over[5]), fmaxf(over[6], over[7])) > DEC_MAX_SLACK_I8 ||
-                            vf > vref;
+                            vf > vref || nacc >= 384;
         if (group_bar_or(bar_id, exceed)) {
+          if (nacc > 0) flush();  // what TMEM holds is relative to the old references (the previous value MMAs have completed)
 #pragma unroll
           for (int h = 0; h < 8; h++) {
             const float wm = warp_max(s[h]);
@@ -744,11 +776,12 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           *reinterpret_cast<uint4*>(bp + (TB / 8) * 128 + off) = make_uint4(pb[4], pb[5], pb[6], pb[7]);
           fence_proxy_async();
         }
+        if (gt == 0) *accf = nacc;     // 0: this block's value product starts a new accumulation
+        nacc++;
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(p_ready);          // V tile in TMEM, probabilities in shared memory
         mbar_arrive(&empty_bar[st]);   // this thread is done with the staged tile
-        const float ofac = p.delta * vref * (1.0f / 2097152.0f);  // value digits -> real units: delta / pscale
 
         // ---- next slot: its K tile, while the value MMAs run
         it++;
@@ -758,29 +791,15 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         have_block = dsc.y >= 0;
         if (have_block) k_tile(stages + st * L::STAGE_BYTES);
 
-        // ---- fold the value product into the running accumulator
+        // ---- the value MMAs of this block must have completed before its V tile and B_P are overwritten; their result stays in TMEM
         if (!failed) failed = !mbar_wait_bounded(o_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
-        tc_fence_after();
-#pragma unroll
-        for (int j = 0; j < DJ; j++)
-#pragma unroll
-          for (int half = 0; half < 2; half++) {
-            uint32_t o_u[16];
-            tc_ld16_issue(tmem_g + lane_sel + L::I8_O_COL + 32 * j + 16 * half, o_u);
-            tc_wait_ld();
-#pragma unroll
-            for (int hq = 0; hq < 4; hq++) {
-              const float of = fmaf(i2f_small(o_u[4 * hq + 2]), 65536.f, __int2float_rn((int)o_u[4 * hq + 1] * 256 + (int)o_u[4 * hq]));
-              acc[j][4 * half + hq] = fmaf(of, ofac, acc[j][4 * half + hq]);
-            }
-          }
-        tc_fence_before();
         nbk++;
         if (!have_block && !failed) {
           mbar_arrive(&empty_bar[st]);  // the end marker's slot
           it++;
         }
       }
+      if (nacc > 0) flush();
 
       } else {
       // The group's 128 TMEM columns: [0, 64 DJ) operand tile, then scores, values, and V_COL.. a second home for the first
