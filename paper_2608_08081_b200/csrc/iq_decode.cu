@@ -34,7 +34,10 @@ constexpr int DEC_GROUP_THREADS = 128;  // 4 warps: dequantisation, softmax, acc
 constexpr uint32_t DEC_WAIT_LIMIT = 1u << 22;
 constexpr int DEC_HDR_BYTES = 4096;    // barriers, TMEM base, work counter, segment and block descriptors, scratch
 constexpr float DEC_MAX_SLACK = 4.0f;  // log2 units a score may exceed the running reference before it is raised
-constexpr float DEC_MAX_SLACK_I8 = 1.0f;  // the same on the integer path, where the probabilities are fixed-point numbers
+#ifndef IQ_SLACK_I8
+#define IQ_SLACK_I8 4
+#endif
+constexpr float DEC_MAX_SLACK_I8 = (float)IQ_SLACK_I8;  // the same on the integer path, where the probabilities are fixed-point numbers
 
 template <int D>
 struct DecLayout {
@@ -619,14 +622,14 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
       const uint32_t l8_0 = p.lut8[0], l8_1 = p.lut8[1];
       const float sfac = reinterpret_cast<const float*>(smem + L::OFF_QFAC)[8];  // score digits -> log2-domain score per unit K scale
       float vref = 0.f;    // power of two >= every V scale (x 1/sqrt d) seen by the group in this segment
-      float pscale = 0.f;  // probabilities are written as round(p * vscale * pscale) < 2^23: pscale = 2^21 / vref
+      float pscale = 0.f;  // probabilities are written as round(p * vscale * pscale) <= 2^30: pscale = 2^(30 - slack) / vref
       // The value products of consecutive blocks accumulate in TMEM as int32 (exact) for as long as the references they are
       // relative to (m_run, vref) stand; nacc counts the blocks in there. A block adds at most 128 * 127 * 255 < 2^22 per
       // column, so 384 blocks stay below 2^31. flush() adds the accumulated digits to the float accumulator.
       int nacc = 0;
       int* accf = reinterpret_cast<int*>(smem + L::OFF_ACCF + 4 * grp);  // tells the control warp to accumulate onto TMEM
       auto flush = [&]() {
-        const float ofac = p.delta * vref * (1.0f / 2097152.0f);  // value digits -> real units: delta / pscale
+        const float ofac = p.delta * vref * ((float)(1 << IQ_SLACK_I8) / 1073741824.0f);  // value digits -> real units: delta / pscale
         tc_fence_after();
 #pragma unroll
         for (int j = 0; j < DJ; j++)
@@ -637,8 +640,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
             tc_wait_ld();
 #pragma unroll
             for (int hq = 0; hq < 4; hq++) {
-              const float of = fmaf(fmaf(__int2float_rn((int)o_u[4 * hq + 2]), 256.f, __int2float_rn((int)o_u[4 * hq + 1])), 256.f,
-                                    __int2float_rn((int)o_u[4 * hq]));
+              const float of = fmaf(fmaf(fmaf(__int2float_rn((int)o_u[4 * hq + 3]), 256.f, __int2float_rn((int)o_u[4 * hq + 2])), 256.f,
+                                         __int2float_rn((int)o_u[4 * hq + 1])), 256.f, __int2float_rn((int)o_u[4 * hq]));
               acc[j][4 * half + hq] = fmaf(of, ofac, acc[j][4 * half + hq]);
             }
           }
@@ -758,18 +761,18 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           }
           const float bv = fmaxf(fmaxf(red2[0], red2[1]), fmaxf(red2[2], red2[3]));
           if (bv > vref) vref = __uint_as_float((__float_as_uint(bv) + 0x007FFFFFu) & 0x7F800000u);  // next power of two
-          pscale = vref > 0.f ? 2097152.0f / vref : 0.f;
+          pscale = vref > 0.f ? (1073741824.0f / (float)(1 << IQ_SLACK_I8)) / vref : 0.f;  // p * vscale * pscale <= 2^30
         }
         {
-          // probabilities (times scale_V / sqrt(d)) as 23-bit fixed point: the bytes of the float p * pscale + 2^23 are the base-256
-          // digits of round(p * pscale) (byte 3 is the float's exponent: its result column is ignored). B_P[n][row], n = 4 head + digit.
+          // probabilities (times scale_V / sqrt(d)) as 30-bit fixed point: the bytes of round(p * vscale * pscale) are its four
+          // base-256 digits. B_P[n][row], n = 4 head + digit.
           uint32_t pb[8];
           const float vfp = vf * pscale;
 #pragma unroll
           for (int h = 0; h < 8; h++) {
             const float pr = ex2f(s[h] - m_run[h]);
             l_run[h] += pr;
-            pb[h] = __float_as_uint(fmaf(pr, vfp, 8388608.0f));
+            pb[h] = __float2uint_rn(pr * vfp);
           }
           const int off = (gt & 7) * 16 + (gt >> 3) * 128;
           *reinterpret_cast<uint4*>(bp + off) = make_uint4(pb[0], pb[1], pb[2], pb[3]);
