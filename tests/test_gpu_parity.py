@@ -91,6 +91,23 @@ def test_few_slots_for_a_long_sequence_next_to_short_ones(iq, torch, codebooks):
     _roundtrip(iq, torch, codebooks, w, [2, 7, 40], n_new=lens)
 
 
+def test_dominant_row_over_a_long_tail_of_equal_values(iq, torch, codebooks):
+    """One key far above a long flat tail whose total probability mass still matters, and value rows that all point the
+    same way: every small probability adds with the same sign, so a path that rounds them away (fixed-point or
+    half-precision probabilities) shows a bias here; and the flat tail makes the lazily raised softmax reference and
+    the in-TMEM accumulation run over many blocks without a raise."""
+    T, d = 12000, 128
+    w = workloads.tiny(320, 1, 8, 1, d, T)
+    g = np.random.Generator(np.random.Philox(321))
+    w.k[:] = workloads.to_fp16(0.02 * g.standard_normal(w.k.shape))                 # flat scores near 0
+    base = g.standard_normal(d)
+    w.v[:] = workloads.to_fp16(base[None, None, None, :] * (1 + 0.01 * g.standard_normal((1, T, 1, 1))))
+    for h in range(8):                                                              # the needle of head h: z ~ 11 nats above the tail
+        w.k[0, 1000 + 997 * h, 0] = workloads.to_fp16(11.0 * np.sqrt(d) * w.q[0, h].astype(np.float64) / np.dot(w.q[0, h].astype(np.float64), w.q[0, h].astype(np.float64)))
+    stats = _roundtrip(iq, torch, codebooks, w, [1, 2, 9])
+    print(stats)
+
+
 def test_large_scale_rows_and_zero_rows(iq, torch, codebooks):
     w = workloads.tiny(301, 1, 4, 1, 128, 256, scale=300.0)
     w.k[0, 5] = 0
