@@ -38,11 +38,11 @@ DEFAULT_WORKLOAD = "config5_B32_ctx32768"
 T_CAP_MARGIN = 2048  # rows of head-room so that every sequence can take the benchmark's appends
 
 # DRAM traffic of one decode launch. The ncu capture of the decode kernel (summarised under profiles/; taken at B = 8
-# because a B = 32 launch is too large for a multi-pass capture) measured dram__bytes_read.sum = 1.0031 x the
-# algorithmic packed-KV bytes of the launch and dram__bytes_write.sum = 7.91 MB for 1.33 MB of partial results
+# because a B = 32 launch is too large for a multi-pass capture) measured dram__bytes_read.sum = 1.0032 x the
+# algorithmic packed-KV bytes of the launch and dram__bytes_write.sum = 5.69 MB for 1.33 MB of partial results
 # (S = 5 slots). Reads scale with the rows processed; writes with the partial results.
-NCU_READ_PER_ALGORITHMIC_BYTE = 182.576 / 182.013
-NCU_WRITE_PER_PARTIAL_BYTE = 7.907 / 1.331
+NCU_READ_PER_ALGORITHMIC_BYTE = 182.599 / 182.013
+NCU_WRITE_PER_PARTIAL_BYTE = 5.689 / 1.331
 
 
 def decode_traffic_bytes(algorithmic_bytes: float, B: int, H_q: int, S: int, d: int) -> int:
@@ -310,12 +310,13 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "higher_is_better": True,
         "scaling": "weak",
         "vs_baseline": None,
-        "dtype": "u3 codes, f16 tensor-core operands, f32 accumulate",
+        "dtype": ("u3 codes, int8 tensor-core operands, int32 accumulate" if CODEBOOK == "int8"
+                  else "u3 codes, f16 tensor-core operands, f32 accumulate"),
         "data": "synthetic",
         "config": {"workload": args.workload, "batch": B, "ctx": st["ctx"], "n_q_heads": H_q, "n_kv_heads": H_kv, "head_dim": d,
                    "t_cap": st["t_cap"], "ragged_lengths": "floor(ctx*U[0.5,1.0])", "cached_rows_per_kv_head": rows,
                    "num_splits": S, "bytes_per_row_per_kv_head": bytes_per_row(d), "l2": "inputs_larger_than_l2",
-                   "step": "quantize-append 1 row/seq + fused decode + combine", "parallelism": f"replicas x{world}"},
+                   "step": "quantize-append 1 row/seq + fused decode + combine", "codebook": CODEBOOK, "parallelism": f"replicas x{world}"},
         "decode_tokens_per_s": round(world * B / (ms_step * 1e-3), 1),
         "frac_of_8TBs": round(value / world / 8000.0, 4),
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
@@ -372,7 +373,7 @@ def run_reference(args, rank: int, world: int):
     nb = 1
     T = int(lens_all[0])
     g = np.random.Generator(np.random.Philox(workloads.stream_seed(5, 0) + 7))
-    lv, th = lloyd_max.fp16_codebook(d)
+    lv, th = lloyd_max.int8_codebook(d) if CODEBOOK == "int8" else lloyd_max.fp16_codebook(d)
     quats = workloads.quaternion_pairs(workloads.rng(5, workloads.QUAT_STREAM), H_kv, d)
     P = oracle.row_bytes(d)
     cache = oracle.new_cache(nb, H_kv, d, workloads.cap128(T + args.warmup + args.steps + 1))
