@@ -173,8 +173,11 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
  *                  every call.
  *   part_argmax    device int32 [batch][n_q_heads][S] or NULL: row index attaining m (lowest on ties), -1 if empty.
  *   status_dev     optional (see top).
- * Arithmetic: q~ and the probabilities enter fp16 tensor-core operands, each as a two-term fp16 sum
- * (hi + lo); codebook levels are exact fp16 values; every accumulation is fp32. Blocks are handed to the
+ * Arithmetic, codebook levels on an 8-bit grid (iq_int8_codebook): int8 tensor-core operands and int32
+ * accumulation -- the levels as integers, q~ as three base-128 digits of a 21-bit fixed-point number (one scale per
+ * KV head group), the probabilities times V scale as four base-256 digits of a 30-bit fixed-point number; softmax
+ * statistics and the running output in fp32. Other codebooks: levels must be exact binary16 values; q~ and the
+ * probabilities enter fp16 operands as two-term sums (hi + lo), every accumulation is fp32. Blocks are handed to the
  * warps of an SM dynamically, so the order of the fp32 additions -- and with it the last bits of the
  * result -- can differ between two calls on the same inputs; m and the argmax do not.
  */
