@@ -25,13 +25,12 @@
 // Packed tiles arrive through a 1-D bulk-copy (TMA) pipeline; every mbarrier wait is bounded.
 #include <climits>
 
-#include "iq_common.cuh"
+#include "iq_decode_common.cuh"
 #include "iq_kernels.h"
 
 namespace iq {
 
 constexpr int DEC_GROUP_THREADS = 128;  // 4 warps: dequantisation, softmax, accumulation (thread = TMEM lane)
-constexpr uint32_t DEC_WAIT_LIMIT = 1u << 22;
 constexpr int DEC_HDR_BYTES = 4096;    // barriers, TMEM base, work counter, segment and block descriptors, scratch
 constexpr float DEC_MAX_SLACK = 4.0f;  // log2 units a score may exceed the running reference before it is raised
 #ifndef IQ_SLACK_I8
@@ -81,166 +80,6 @@ static_assert(DecLayout<128>::I8_O_COL + 32 * DecLayout<128>::DJ <= DecLayout<12
 static_assert(DecLayout<256>::I8_O_COL + 32 * DecLayout<256>::DJ <= DecLayout<256>::GROUP_COLS, "TMEM group overflow");
 static_assert(DecLayout<128>::SMEM_BYTES <= 227 * 1024 && DecLayout<256>::SMEM_BYTES <= 227 * 1024, "shared memory overflow");
 static_assert((DecLayout<128>::THREADS + DecLayout<128>::THREADS / 32) * 4 <= DecLayout<128>::BP_BYTES, "set-up scratch must fit one B_P region");
-
-// ---------------------------------------------------------------------------------------------- tcgen05 wrappers
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
-      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float (&o)[16]) {
-  uint32_t r[16];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
-        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-  tc_wait_ld();
-#pragma unroll
-  for (int i = 0; i < 16; i++) o[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&r)[8]) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]),
-               "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
-               : "memory");
-}
-// The same load without the wait: the registers are valid after tc_wait_ld().
-__device__ __forceinline__ void tc_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
-        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem descriptor]; fp16 operands, fp32 accumulate, M = 128, N and majors in idesc.
-__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0)
-      : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem descriptor]; int8 operands, int32 accumulate, K = 32 per instruction.
-__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0), "r"(0), "r"(0), "r"(0)
-      : "memory");
-}
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// Shared-memory operand descriptor, MN-major, no swizzle: element (n, k) of a 16-bit operand sits at
-// (n % 8) * 2 + (n / 8) * sbo + (k % 8) * 16 + (k / 8) * lbo bytes from the start address.
-__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, uint32_t lbo, uint32_t sbo) {
-  return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
-}
-// Instruction descriptor: D = f32, A = B = f16, A K-major (TMEM), B MN-major, N = 16, M = 128.
-constexpr uint32_t DEC_IDESC = (1u << 4) | (1u << 16) | ((16u >> 3) << 17) | ((128u >> 4) << 24);
-// Integer path: D = s32, A = s8 (K-major, TMEM), B MN-major, N = 32, M = 128; B = s8 (query digits) or u8 (probability digits).
-constexpr uint32_t DEC_IDESC_I8_SS = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t DEC_IDESC_I8_SU = (2u << 4) | (1u << 7) | (0u << 10) | (1u << 16) | ((32u >> 3) << 17) | ((128u >> 4) << 24);
-
-// ---------------------------------------------------------------------------------------------- dequantisation
-// x >> s for a compile-time s, computed as the high word of x * 2^(32-s): the multiply issues on the integer
-// multiply-add pipe, which idles here, instead of the shift/logic pipe that carries the byte lookups.
-template <int SH>
-__device__ __forceinline__ uint32_t shr_mul(uint32_t x) {
-  uint32_t hi;
-  asm("{\n\t.reg .b64 t;\n\t.reg .b32 lo;\n\tmul.wide.u32 t, %1, %2;\n\tmov.b64 {lo, %0}, t;\n\t}" : "=r"(hi) : "r"(x), "n"(1u << (32 - SH)));
-  return hi;
-}
-// Selectors of the 8 entries whose code bits sit in bit 3 of the nibbles of the unit's three words.
-__device__ __forceinline__ uint32_t sliced_selectors(uint32_t w0, uint32_t w1, uint32_t w2) {
-  return (shr_mul<3>(w0) & 0x11111111u) | (shr_mul<2>(w1) & 0x22222222u) | (shr_mul<1>(w2) & 0x44444444u);
-}
-// One packing unit (32 codes in 3 words) -> 16 registers of two fp16 levels each, entries in natural order:
-// out[r] = (level[code 2r], level[code 2r+1]). Byte lookups with prmt: 8 levels x (low byte, high byte).
-__device__ __forceinline__ void dequant_unit(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t lo0, uint32_t lo1, uint32_t hi0,
-                                             uint32_t hi1, uint32_t (&out)[16]) {
-  const uint32_t sel[4] = {w0 & 0x77777777u, w1 & 0x77777777u, w2 & 0x77777777u, sliced_selectors(w0, w1, w2)};
-#pragma unroll
-  for (int k = 0; k < 4; k++)
-#pragma unroll
-    for (int hh = 0; hh < 2; hh++) {
-      const uint32_t x = hh ? shr_mul<16>(sel[k]) : sel[k];
-      const uint32_t l = prmt(lo0, lo1, x), h = prmt(hi0, hi1, x);
-      out[4 * k + 2 * hh] = prmt(l, h, 0x5140u);
-      out[4 * k + 2 * hh + 1] = prmt(l, h, 0x7362u);
-    }
-}
-
-// Integer path: one packing unit -> 8 registers of four int8 levels each, entries in natural order (one prmt per 4 codes).
-__device__ __forceinline__ void dequant_unit8(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t l0, uint32_t l1, uint32_t (&out)[8]) {
-  const uint32_t sel[4] = {w0 & 0x77777777u, w1 & 0x77777777u, w2 & 0x77777777u, sliced_selectors(w0, w1, w2)};
-#pragma unroll
-  for (int k = 0; k < 4; k++) {
-    out[2 * k] = prmt(l0, l1, sel[k]);
-    out[2 * k + 1] = prmt(l0, l1, shr_mul<16>(sel[k]));
-  }
-}
-// int32 -> float for |x| < 2^22, on the integer and FMA pipes (the conversion instruction runs at a quarter of their rate).
-__device__ __forceinline__ float i2f_small(uint32_t x) { return __uint_as_float(x + 0x4B400000u) - 12582912.0f; }
-
-// One lane of a converged warp. Issuing the MMAs / bulk copies from an elected lane of a converged warp keeps
-// their operands in uniform registers; a lone divergent thread issues the same sequence about 3x slower.
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
-  return pred != 0;
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// Named barrier `id` over the 128 compute threads of one group, with an OR reduction.
-__device__ __forceinline__ bool group_bar_or(int id, bool pred) {
-  uint32_t r;
-  asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %2, 0;\n\tbarrier.red.or.pred p, %1, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(r) : "r"(id), "r"((uint32_t)pred) : "memory");
-  return r != 0;
-}
-// Barrier 0 over the whole CTA, for the places where the control and the compute warps arrive from different code.
-__device__ __forceinline__ void cta_bar_sync() { asm volatile("barrier.sync 0;" ::: "memory"); }
-// Named barrier `id` over `count` threads (a multiple of 32).
-__device__ __forceinline__ void cta_bar_sync_n(int id, int count) { asm volatile("barrier.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
-__device__ __forceinline__ void group_bar_sync(int id) { asm volatile("barrier.sync %0, 128;" ::"r"(id) : "memory"); }
-
-__device__ __forceinline__ float max3f(float a, float b, float c) {
-  float r;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-  return r;
-}
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(FULL, v, o));
-  return v;
-}
-
-// Segment descriptor in shared memory (written by thread 0 before each segment).
-struct DecSegment {
-  int b, y;          // sequence, item within the sequence (KV head x head group)
-  int blk0, blk1;    // blocks [blk0, blk1) of the item
-  int slot;          // partial slot of the item this segment reports to
-  int len;           // cached rows of the sequence
-  int flags;         // bit 0: blk1 is the end of the item; bit 1: last segment of this CTA
-  int pad;
-};
-
-// Thread 0's position in the CTA's range (kept in shared memory between segments).
-struct DecWalk {
-  int b, y, blk, nb;        // sequence, item within it, block within the item, blocks of sequence b
-  long long left, g, item;  // range mode: blocks to go, launch-wide position; whole-item mode: linear item index
-};
 
 template <int D, bool ARGMAX, bool I8>
 __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const DecodeParams p) {
