@@ -349,6 +349,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
       const int blk1 = seg_s->blk1, len = seg_s->len;
       const size_t slab = ((size_t)seg_s->b * p.n_kv_heads + (seg_s->y / p.head_groups)) * (size_t)p.t_cap;
       const uint32_t bq_addr = smem_u32(bq), bp_addr = smem_u32(bp);
+      // operand descriptors of the first k-step, built before the waits: a k-step further on adds its byte offset / 16
+      const uint64_t bq_desc0 = smem_desc_mn(bq_addr, 128, (D / 8) * 128), bp_desc0 = smem_desc_mn(bp_addr, 128, (TB / 8) * 128);
       bool ended = false;   // the segment's counter ran out and the end marker has been staged
       int it_issue = it;    // slots staged so far (the pipeline is empty between segments)
       auto stage_next = [&]() {  // draw the next block of the segment into slot it_issue, or the end marker
@@ -394,12 +396,11 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           if constexpr (I8) {
 #pragma unroll
             for (int kk = 0; kk < D / 32; kk++)
-              tc_mma_i8(tmem_g + L::I8_S_COL, tmem_g + L::I8_K_COL + 8 * kk, smem_desc_mn(bq_addr + kk * 512, 128, (D / 8) * 128),
-                        DEC_IDESC_I8_SS, kk > 0);
+              tc_mma_i8(tmem_g + L::I8_S_COL, tmem_g + L::I8_K_COL + 8 * kk, bq_desc0 + 32 * kk, DEC_IDESC_I8_SS, kk > 0);
           } else {
 #pragma unroll
             for (int kk = 0; kk < D / 16; kk++)
-              tc_mma_f16(tmem_g + L::S_COL, tmem_g + L::A_COL + 8 * kk, smem_desc_mn(bq_addr + kk * 256, 128, (D / 8) * 128), DEC_IDESC, kk > 0);
+              tc_mma_f16(tmem_g + L::S_COL, tmem_g + L::A_COL + 8 * kk, bq_desc0 + 16 * kk, DEC_IDESC, kk > 0);
           }
           tc_commit(s_bar);
         }
@@ -414,8 +415,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
             for (int j = 0; j < DJ; j++)
 #pragma unroll
               for (int kk = 0; kk < TB / 32; kk++)  // the values stay in TMEM (int32) over the blocks until the compute threads read them
-                tc_mma_i8(tmem_g + L::I8_O_COL + 32 * j, tmem_g + L::I8_V_COL + 32 * j + 8 * kk,
-                          smem_desc_mn(bp_addr + kk * 512, 128, (TB / 8) * 128), DEC_IDESC_I8_SU, (kk > 0) || keep_values);
+                tc_mma_i8(tmem_g + L::I8_O_COL + 32 * j, tmem_g + L::I8_V_COL + 32 * j + 8 * kk, bp_desc0 + 32 * kk, DEC_IDESC_I8_SU,
+                          (kk > 0) || keep_values);
           } else {
 #pragma unroll
             for (int j = 0; j < DJ; j++)
@@ -423,7 +424,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
               for (int kk = 0; kk < TB / 16; kk++)
                 tc_mma_f16(tmem_g + L::O_COL + 16 * j,  // rows 0..63 of the V tile sit in V_COL, rows 64..127 in the operand columns
                            tmem_g + (kk < 4 ? L::V_COL + 32 * j + 8 * kk : L::A_COL + 64 * j + 8 * (kk - 4)),
-                           smem_desc_mn(bp_addr + kk * 256, 128, (TB / 8) * 128), DEC_IDESC, kk > 0);
+                           bp_desc0 + 16 * kk, DEC_IDESC, kk > 0);
           }
           tc_commit(o_bar);
         }
