@@ -261,12 +261,15 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     ms_total = max_over_ranks(ms_total, world, device)
 
     # ---- end to end through the C-ABI binding with host buffers: H2D of the step inputs and D2H of the output inside the timed region
-    hq = q_all[:W + K].cpu().pin_memory(); hk = k_all[:W + K].cpu().pin_memory(); hv = v_all[:W + K].cpu().pin_memory()
-    dq = torch.empty_like(q_all[0]); dk = torch.empty_like(k_all[0]); dv = torch.empty_like(v_all[0])
+    # the step's host inputs (q, new k, new v) sit in one pinned staging buffer per step and travel in one copy
+    nq, nk = B * H_q * d, B * H_kv * d
+    hin = torch.cat([q_all[:W + K].reshape(W + K, nq), k_all[:W + K].reshape(W + K, nk), v_all[:W + K].reshape(W + K, nk)], dim=1).cpu().pin_memory()
+    din = torch.empty(nq + 2 * nk, dtype=torch.float16, device=device)
+    dq = din[:nq].view(B, H_q, d); dk = din[nq:nq + nk].view(B, 1, H_kv, d); dv = din[nq + nk:].view(B, 1, H_kv, d)
     hout = torch.empty((B, H_q, d), dtype=torch.float32).pin_memory()
 
     def e2e_step(i):
-        dq.copy_(hq[i], non_blocking=True); dk.copy_(hk[i], non_blocking=True); dv.copy_(hv[i], non_blocking=True)
+        din.copy_(hin[i], non_blocking=True)
         iq.iq_quantize_append(shape, rot, cb, dk, dv, lens_tab[i], None, 1, cache, st["status"])
         iq.iq_decode_attention(shape, rot, cb, dq, cache, lens_tab[i + 1], S, ws.part_acc, ws.part_ml, None, ws.status)
         iq.iq_combine_splits(shape, rot, S, ws.part_acc, ws.part_ml, None, ws.out, ws.lse, None)
