@@ -70,7 +70,9 @@ def _load():
 _lib = _load()
 
 
-@dataclass
+# Shape and Codebook are immutable, so each builds its C struct once: a decode step of a short batch is bound by the
+# host's time per call, not by the kernels.
+@dataclass(frozen=True)
 class Shape:
     batch: int
     n_q_heads: int
@@ -81,20 +83,27 @@ class Shape:
     sm_scale: float = 0.0
 
     def c(self) -> _IqShape:
-        return _IqShape(self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.t_cap, self.bits, self.sm_scale)
+        cs = self.__dict__.get("_c")
+        if cs is None:
+            cs = _IqShape(self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.t_cap, self.bits, self.sm_scale)
+            object.__setattr__(self, "_c", cs)
+        return cs
 
 
-@dataclass
+@dataclass(frozen=True)
 class Codebook:
     levels: tuple
     thresholds: tuple
 
     def c(self) -> _IqCodebook:
-        cb = _IqCodebook()
-        for i in range(8):
-            cb.levels[i] = float(self.levels[i])
-        for i in range(7):
-            cb.thresholds[i] = float(self.thresholds[i])
+        cb = self.__dict__.get("_c")
+        if cb is None:
+            cb = _IqCodebook()
+            for i in range(8):
+                cb.levels[i] = float(self.levels[i])
+            for i in range(7):
+                cb.thresholds[i] = float(self.thresholds[i])
+            object.__setattr__(self, "_c", cb)
         return cb
 
 

@@ -272,6 +272,68 @@ def test_config2_prefill_then_64_decode_steps(iq, torch, codebooks):
     assert status.cpu().numpy()[0] == 0
 
 
+def test_decode_step_replayed_from_a_cuda_graph(iq, torch, codebooks):
+    """One decode step (append one row per sequence, attend, combine) captured once into a CUDA graph and replayed with
+    new rows, new queries and growing lengths: the grids depend on the shape alone and every length is read on the
+    device, so the replays must match the oracle step by step, across a 128-row block boundary, with one sequence
+    that starts empty."""
+    d, B, H_q, H_kv, T0, steps = 128, 3, 8, 2, 250, 12
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    w = workloads.tiny(77, B, H_q, H_kv, d, T0 + steps)
+    lens0 = np.array([T0, 97, 0], np.int32)
+    t_cap = workloads.cap128(T0 + steps)
+    shape = iq.Shape(B, H_q, H_kv, d, t_cap)
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(w.quats), rot)
+    cache, status = iq.new_cache(shape), torch.zeros(4, dtype=torch.int32, device="cuda")
+    iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(w.k[:, :T0]).cuda(), torch.from_numpy(w.v[:, :T0]).cuda(),
+                          torch.zeros(B, dtype=torch.int32, device="cuda"), torch.from_numpy(lens0).cuda(), T0, cache, status)
+    ref = oracle.new_cache(B, H_kv, d, t_cap)
+    oracle.quantize_append(w.quats, th, w.k[:, :T0], w.v[:, :T0], np.zeros(B, np.int32), lens0, ref)
+    S = iq.iq_suggest_splits(shape, t_cap)
+    ws = iq.DecodeWorkspace(shape, S, want_argmax=True)
+    lens = torch.from_numpy(lens0).cuda()
+    k1 = torch.zeros((B, 1, H_kv, d), dtype=torch.float16, device="cuda")
+    v1, q1 = torch.zeros_like(k1), torch.zeros((B, H_q, d), dtype=torch.float16, device="cuda")
+
+    def step():
+        iq.iq_quantize_append(shape, rot, cb, k1, v1, lens, None, 1, cache, status)
+        lens.add_(1)
+        iq.decode_step(shape, rot, cb, q1, cache, lens, ws)
+
+    g = np.random.default_rng(5)
+    rows = lens0.astype(np.int64).copy()                  # next row of w.k / w.v each sequence appends
+    graph = None
+    for i in range(steps):
+        kn = np.stack([w.k[b, rows[b]] for b in range(B)])[:, None]
+        vn = np.stack([w.v[b, rows[b]] for b in range(B)])[:, None]
+        qn = workloads.to_fp16(g.standard_normal((B, H_q, d)))
+        k1.copy_(torch.from_numpy(kn)); v1.copy_(torch.from_numpy(vn)); q1.copy_(torch.from_numpy(qn))
+        if i == 0:
+            step()                                        # eager once: one-time kernel attributes are set outside a capture
+        elif graph is None:
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            graph.replay()                                # capturing runs nothing
+        else:
+            graph.replay()
+        torch.cuda.synchronize()
+        oracle.quantize_append(w.quats, th, kn, vn, rows.astype(np.int32), None, ref)
+        rows += 1
+        now = rows.astype(np.int32)
+        assert np.array_equal(lens.cpu().numpy(), now)
+        res = dict(out=ws.out.cpu().numpy().astype(np.float64), lse=ws.lse.cpu().numpy().astype(np.float64),
+                   argmax=ws.argmax.cpu().numpy())
+        check_decode(w, lv, qn, res, cache_to_numpy(cache), now)
+    gnp = cache_to_numpy(cache)
+    w2 = workloads.Workload("g", B, H_q, H_kv, d, t_cap, w.k, w.v, w.q, w.quats, rows.astype(np.int32))
+    compare_caches(w2, th, gnp, ref, w2.seq_lens)         # prefill rows and the rows the graph appended
+    assert status.cpu().numpy()[0] == 0
+
+
 def test_config3_wide_heads(iq, torch, codebooks):
     w = workloads.config3()
     S = None
