@@ -33,7 +33,12 @@ WORKLOADS = {
     "config5_B32_ctx4096": (32, 4096, 64, 8, 128),
     "config5_B8_ctx4096": (8, 4096, 64, 8, 128),
     "config5_B1_ctx4096": (1, 4096, 64, 8, 128),
+    # single-sequence shapes (configs 3 and 4) as a stack of 48 per-layer caches of full length, every layer with its own
+    # three launches of batch 1: the caches of the stack exceed L2 together, a step is one pass over the layers
+    "config3_48layers": (48, 16384, 16, 8, 256),
+    "config4_48layers": (48, 32768, 32, 8, 128),
 }
+PER_SEQUENCE_LAUNCHES = {"config3_48layers", "config4_48layers"}
 DEFAULT_WORKLOAD = "config5_B32_ctx32768"
 T_CAP_MARGIN = 2048  # rows of head-room so that every sequence can take the benchmark's appends
 
@@ -161,7 +166,7 @@ def build_state(name: str, device, rank: int):
     import workloads
 
     B, ctx, H_q, H_kv, d = WORKLOADS[name]
-    gen = workloads.config5_device(B, ctx, device, H_q, H_kv, d)
+    gen = workloads.config5_device(B, ctx, device, H_q, H_kv, d, full_lengths=name in PER_SEQUENCE_LAUNCHES)
     t_cap = ctx + T_CAP_MARGIN
     shape = iq.Shape(B, H_q, H_kv, d, t_cap)
     cb = iq.iq_int8_codebook(d) if CODEBOOK == "int8" else iq.iq_default_codebook(d)
@@ -221,7 +226,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     iq, shape, cb, rot, cache = st["iq"], st["shape"], st["cb"], st["rot"], st["cache"]
     B, H_q, H_kv, d = st["B"], st["H_q"], st["H_kv"], st["d"]
     K, W = args.steps, args.warmup
-    S = args.splits or iq.iq_suggest_splits(shape, st["ctx"])
+    # Launch groups: the whole batch in one set of launches, or (stack-of-layers workloads) one set per sequence.
+    per_seq = args.workload in PER_SEQUENCE_LAUNCHES
+    gshape = iq.Shape(1, H_q, H_kv, d, st["t_cap"]) if per_seq else shape
+    S = args.splits or iq.iq_suggest_splits(gshape, st["ctx"])
     ws = iq.DecodeWorkspace(shape, S, want_argmax=False, device=device)
     # Row i of this table holds the sequence lengths before step i: the step appends at lens_tab[i] and attends to
     # lens_tab[i + 1] rows (the serving engine knows the lengths; no kernel is spent on incrementing them).
@@ -229,15 +237,24 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     lens_tab = (lens0[None, :] + torch.arange(K + W + 4, device=device, dtype=torch.int32)[:, None]).contiguous()
     q_all, k_all, v_all = step_inputs(st, K + W, device, 99 + rank)
     stream = torch.cuda.current_stream()
+    groups = [slice(b, b + 1) for b in range(B)] if per_seq else [slice(0, B)]
+    gcache = [iq.Cache(cache.k_codes[g], cache.k_scales[g], cache.v_codes[g], cache.v_scales[g]) for g in groups]
+    n_groups = len(groups)
+
+    def launches(i, q, k, v, ev=None):
+        """The step's launches on device inputs q [B][H_q][d], k, v [B][1][H_kv][d]: append, decode, combine per group;
+        ev = (group, event pair) brackets that group's decode launch."""
+        for j, g in enumerate(groups):
+            iq.iq_quantize_append(gshape, rot, cb, k[g], v[g], lens_tab[i][g], None, 1, gcache[j], st["status"])
+            if ev is not None and ev[0] == j:
+                ev[1][0].record(torch.cuda.current_stream())
+            iq.iq_decode_attention(gshape, rot, cb, q[g], gcache[j], lens_tab[i + 1][g], S, ws.part_acc[g], ws.part_ml[g], None, ws.status)
+            if ev is not None and ev[0] == j:
+                ev[1][1].record(torch.cuda.current_stream())
+            iq.iq_combine_splits(gshape, rot, S, ws.part_acc[g], ws.part_ml[g], None, ws.out[g], ws.lse[g], None)
 
     def one_step(i, ev=None):
-        iq.iq_quantize_append(shape, rot, cb, k_all[i], v_all[i], lens_tab[i], None, 1, cache, st["status"])
-        if ev is not None:
-            ev[0].record(torch.cuda.current_stream())
-        iq.iq_decode_attention(shape, rot, cb, q_all[i], cache, lens_tab[i + 1], S, ws.part_acc, ws.part_ml, None, ws.status)
-        if ev is not None:
-            ev[1].record(torch.cuda.current_stream())
-        iq.iq_combine_splits(shape, rot, S, ws.part_acc, ws.part_ml, None, ws.out, ws.lse, None)
+        launches(i, q_all[i], k_all[i], v_all[i], None if ev is None else (i % n_groups, ev))
 
     def timed(run_k_steps, evs):
         """Times one call of run_k_steps (exactly K steps) between two events on the launching stream; the event pairs
@@ -308,9 +325,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
 
     def e2e_step(i):
         din.copy_(hin[i], non_blocking=True)
-        iq.iq_quantize_append(shape, rot, cb, dk, dv, lens_tab[i], None, 1, cache, st["status"])
-        iq.iq_decode_attention(shape, rot, cb, dq, cache, lens_tab[i + 1], S, ws.part_acc, ws.part_ml, None, ws.status)
-        iq.iq_combine_splits(shape, rot, S, ws.part_acc, ws.part_ml, None, ws.out, ws.lse, None)
+        launches(i, dq, dk, dv)
         hout.copy_(ws.out, non_blocking=True)
         torch.cuda.synchronize()
 
@@ -339,7 +354,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     ms_step = ms_total / K
     value = aggregate_gbs(sum(bytes_steps), ms_total, world)
     dec_avg_ms = sum(dec_ms) / len(dec_ms)
-    timed_launch_bytes = bytes_steps[::GRAPH_EVENT_STRIDE] if graph is not None else bytes_steps   # the bracketed launches
+    # the bracketed launches: one decode launch per bracketed step, over 1 / n_groups of the step's rows
+    timed_launch_bytes = [x / n_groups for x in (bytes_steps[::GRAPH_EVENT_STRIDE] if graph is not None else bytes_steps)]
     assert len(timed_launch_bytes) == len(dec_ms)
     achieved = (sum(timed_launch_bytes) / len(dec_ms)) / (dec_avg_ms * 1e-3) / 1e9
     out = {
@@ -357,7 +373,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                   else "u3 codes, f16 tensor-core operands, f32 accumulate"),
         "data": "synthetic",
         "config": {"workload": args.workload, "batch": B, "ctx": st["ctx"], "n_q_heads": H_q, "n_kv_heads": H_kv, "head_dim": d,
-                   "t_cap": st["t_cap"], "ragged_lengths": "floor(ctx*U[0.5,1.0])", "cached_rows_per_kv_head": rows,
+                   "t_cap": st["t_cap"], "lengths": "ctx" if per_seq else "ragged, floor(ctx*U[0.5,1.0])",
+                   "launch_groups": n_groups, "ms_per_launch_group": round(ms_step / n_groups, 5), "cached_rows_per_kv_head": rows,
                    "num_splits": S, "bytes_per_row_per_kv_head": bytes_per_row(d), "l2": "inputs_larger_than_l2",
                    "step": "quantize-append 1 row/seq + fused decode + combine", "codebook": CODEBOOK, "parallelism": f"replicas x{world}",
                    "timed_region": ("one replay of a CUDA graph holding the K steps" if graph is not None
@@ -365,7 +382,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "decode_tokens_per_s": round(world * B / (ms_step * 1e-3), 1),
         "frac_of_8TBs": round(value / world / 8000.0, 4),
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
-                     "traffic": decode_traffic_bytes(sum(bytes_steps) / K, B, H_q, S, d),
+                     "traffic": decode_traffic_bytes(sum(timed_launch_bytes) / len(dec_ms), B // n_groups, H_q, S, d),
                      "traffic_source": "ncu capture at B = 8 scaled by rows processed (reads) and partial results (writes)",
                      "kernel": "decode_kernel", "peak_source": peak_src,
                      "avg_launch_ms": round(dec_avg_ms, 4), "launches_timed": len(dec_ms),
@@ -378,7 +395,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                           "ms_per_step": round(eager_ms / K, 4), "decode_launch_ms": round(sum(eager_dec_ms) / K, 4),
                           "note": "the same K steps launched call by call from the host (three binding calls per step)"},
         "quantize_append": st["quantize_append"],
-        "gpu_launches": 3 * K,   # per step: quantize_append_few_kernel, decode_kernel, combine_kernel
+        "gpu_launches": 3 * K * n_groups,   # per step and launch group: quantize_append_few_kernel, decode_kernel, combine_kernel
         "clocks": clocks,
     }
     if graph_error:

@@ -12,6 +12,8 @@ constexpr int CMB_WARPS = 4;
 template <int D>
 __global__ void __launch_bounds__(CMB_WARPS * 32) combine_kernel(const CombineParams p) {
   constexpr int E = D / 32;
+  grid_dependency_wait();
+  allow_dependent_launch();
   const int lane = threadIdx.x & 31;
   const int bh = blockIdx.x * CMB_WARPS + (threadIdx.x >> 5);
   if (bh >= p.batch * p.n_q_heads) return;
@@ -82,11 +84,8 @@ cudaError_t launch_combine_splits(const CombineParams& p, int head_dim, cudaStre
   const int n = p.batch * p.n_q_heads;
   if (n <= 0) return cudaSuccess;
   dim3 grid((n + CMB_WARPS - 1) / CMB_WARPS), block(CMB_WARPS * 32);
-  if (head_dim == 128)
-    combine_kernel<128><<<grid, block, 0, stream>>>(p);
-  else
-    combine_kernel<256><<<grid, block, 0, stream>>>(p);
-  return cudaGetLastError();
+  if (head_dim == 128) return launch_after_predecessor(combine_kernel<128>, grid, block, 0, stream, p);
+  return launch_after_predecessor(combine_kernel<256>, grid, block, 0, stream, p);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -143,6 +143,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     }
   };
 
+  grid_dependency_wait();  // nothing written by an earlier kernel (lengths, queries, cache rows) is read above this line
+
   // ---------------------------------------------------------------- the block sequence of the launch and this CTA's range
   const int per_thread = (B + L::THREADS - 1) / L::THREADS;
   {
@@ -918,6 +920,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     if (seg_flags & 2) break;  // last segment of this CTA
   }
 
+  allow_dependent_launch();
   if (__syncthreads_or(failed) && tid == 0 && p.status) atomicOr(&p.status[0], IQ_STATUS_WAIT_TIMEOUT);
   tc_fence_before();
   __syncthreads();
@@ -946,8 +949,7 @@ static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
   long long ctas = n_sm[dev];
   if (ctas > max_blocks) ctas = max_blocks;
   if (ctas < 1) ctas = 1;
-  kern<<<dim3((unsigned)ctas), L::THREADS, L::SMEM_BYTES, stream>>>(p);
-  return cudaGetLastError();
+  return launch_after_predecessor(kern, dim3((unsigned)ctas), dim3(L::THREADS), L::SMEM_BYTES, stream, p);
 }
 
 cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream) {

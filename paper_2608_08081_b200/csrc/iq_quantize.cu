@@ -206,6 +206,8 @@ template <int D>
 __global__ void __launch_bounds__(QA_WARPS * 32, 3) quantize_append_k_kernel(const __grid_constant__ QuantizeParams p) {
   using RQ = RowQuantizer<D>;
   constexpr int LPR = RQ::LPR, RPW = RQ::RPW;
+  grid_dependency_wait();
+  allow_dependent_launch();
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int b = blockIdx.z;
@@ -275,6 +277,8 @@ __global__ void __launch_bounds__(128, 3) quantize_append_v_kernel(const __grid_
   constexpr int LPR = RQ::LPR, RPW = RQ::RPW;
   __shared__ __align__(16) uint8_t codes_s[32][D + 16];  // +16: the 16-byte stores of different rows hit different banks
 
+  grid_dependency_wait();
+  allow_dependent_launch();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.z;
   const int h = blockIdx.y;
@@ -448,6 +452,8 @@ template <int D>
 __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_constant__ QuantizeParams p) {
   constexpr int E = D / 32;
   constexpr int LPU = 32 / E;  // lanes per 32-coordinate packing unit
+  grid_dependency_wait();
+  allow_dependent_launch();
   const int lane = threadIdx.x;
   const bool is_v = blockIdx.x != 0;
   const int h = blockIdx.y, b = blockIdx.z;
@@ -534,16 +540,15 @@ cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int ba
   dim3 vgrid((p.n_new_max + 31) / 32 + 1, p.n_kv_heads, batch);  // +1: the first row may sit in the middle of a unit
   if (p.n_new_max <= QA_FEW_ROWS) {
     dim3 grid(2, p.n_kv_heads, batch);  // x = 0: the K rows, x = 1: the V rows of (sequence, KV head)
-    if (head_dim == 128) quantize_append_few_kernel<128><<<grid, 32, 0, stream>>>(p);
-    else quantize_append_few_kernel<256><<<grid, 32, 0, stream>>>(p);
-  } else if (head_dim == 128) {
-    quantize_append_k_kernel<128><<<kgrid, QA_WARPS * 32, 0, stream>>>(p);
-    quantize_append_v_kernel<128><<<vgrid, 128, 0, stream>>>(p);
-  } else {
-    quantize_append_k_kernel<256><<<kgrid, QA_WARPS * 32, 0, stream>>>(p);
-    quantize_append_v_kernel<256><<<vgrid, 128, 0, stream>>>(p);
+    return head_dim == 128 ? launch_after_predecessor(quantize_append_few_kernel<128>, grid, dim3(32), 0, stream, p)
+                           : launch_after_predecessor(quantize_append_few_kernel<256>, grid, dim3(32), 0, stream, p);
   }
-  return cudaGetLastError();
+  // (the V kernel may start under the K kernel: they write different arrays)
+  cudaError_t e = head_dim == 128 ? launch_after_predecessor(quantize_append_k_kernel<128>, kgrid, dim3(QA_WARPS * 32), 0, stream, p)
+                                  : launch_after_predecessor(quantize_append_k_kernel<256>, kgrid, dim3(QA_WARPS * 32), 0, stream, p);
+  if (e != cudaSuccess) return e;
+  return head_dim == 128 ? launch_after_predecessor(quantize_append_v_kernel<128>, vgrid, dim3(128), 0, stream, p)
+                         : launch_after_predecessor(quantize_append_v_kernel<256>, vgrid, dim3(128), 0, stream, p);
 }
 
 }  // namespace iq

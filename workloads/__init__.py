@@ -149,13 +149,15 @@ def config5(B: int, ctx: int, H_q: int = 64, H_kv: int = 8, d: int = 128) -> Wor
                     quaternion_pairs(rng(cfg, QUAT_STREAM), H_kv, d), lens, dict(k_outliers=kch, v_outliers=vch))
 
 
-def config5_device(B: int, ctx: int, device, H_q: int = 64, H_kv: int = 8, d: int = 128, chunk_seqs: int = 4):
+def config5_device(B: int, ctx: int, device, H_q: int = 64, H_kv: int = 8, d: int = 128, chunk_seqs: int = 4,
+                   full_lengths: bool = False):
     """Generator of the large serving points on the GPU (seeded torch generator): yields, per chunk of
-    sequences, (b0, k, v) fp16 device tensors [nb][ctx][H_kv][d]; also returns q, lengths and quaternions."""
+    sequences, (b0, k, v) fp16 device tensors [nb][ctx][H_kv][d]; also returns q, lengths and quaternions.
+    full_lengths: every sequence holds ctx rows (a stack of per-layer caches instead of a ragged batch)."""
     import torch
 
     cfg = 5
-    lens = config5_lengths(B, ctx)
+    lens = np.full(B, ctx, np.int32) if full_lengths else config5_lengths(B, ctx)
     sub = 100 * B + ctx // 1024
     sg = np.random.Generator(np.random.Philox(stream_seed(cfg, STRUCT_STREAM) + sub))
     kch = sg.choice(d, size=4, replace=False)
