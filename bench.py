@@ -33,6 +33,8 @@ WORKLOADS = {
     "config5_B32_ctx4096": (32, 4096, 64, 8, 128),
     "config5_B8_ctx4096": (8, 4096, 64, 8, 128),
     "config5_B1_ctx4096": (1, 4096, 64, 8, 128),
+    # the wide-head shape of config 3 (d = 256, 16 query / 8 KV heads) as a ragged batch that exceeds L2
+    "d256_B32_ctx16384": (32, 16384, 16, 8, 256),
     # single-sequence shapes (configs 3 and 4) as a stack of 48 per-layer caches of full length, every layer with its own
     # three launches of batch 1: the caches of the stack exceed L2 together, a step is one pass over the layers
     "config3_48layers": (48, 16384, 16, 8, 256),

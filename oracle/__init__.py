@@ -182,6 +182,24 @@ def decode_attention(quats, levels, q, cache, seq_lens, H_kv: int, sm_scale: flo
     return r
 
 
+def reconstruct_rows(quats, levels, cache, seq_lens, H_kv: int):
+    """Figure 1 (top), the reconstruct-then-compute model: every cached row of every (sequence, KV head) dequantised
+    and rotated back, x_hat = R^T (scale * level[code] / sqrt(d)). Returns (K, V), fp64 [B][t_cap][H_kv][d]; rows
+    beyond a sequence's length are zero."""
+    B, _, t_cap = cache["k_scales"].shape
+    d = cache["k_codes"].shape[3] * 8 // 3
+    quats = _f32(quats).reshape(H_kv, d // 4, 8)
+    lv = _f32(levels).reshape(8)
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32).reshape(B)
+    k = np.zeros((B, t_cap, H_kv, d), dtype=np.float64)
+    v = np.zeros((B, t_cap, H_kv, d), dtype=np.float64)
+    for a in cache.values():
+        assert a.flags["C_CONTIGUOUS"]
+    lib().iqo_reconstruct_rows(_c_int(B), _c_int(H_kv), _c_int(d), _c_int(t_cap), _p(quats), _p(lv), _p(cache["k_codes"]),
+                               _p(cache["k_scales"]), _p(cache["v_codes"]), _p(cache["v_scales"]), _p(lens), _p(k), _p(v))
+    return k, v
+
+
 def scores(quats, levels, q, cache, b: int, h: int, length: int, H_kv: int, sm_scale: float = 0.0) -> np.ndarray:
     qq = _u16(q)
     B, H_q, d = qq.shape

@@ -363,6 +363,39 @@ void iqo_decode_attention(int B, int H_q, int H_kv, int d, int t_cap, double sm_
   free(Rs);
 }
 
+/* Reconstruct-then-compute, first half (Figure 1, top; the execution model the fused path replaces): every cached
+ * row back in the original space, x_hat = R^T x~ with x~_i = scale * level[code_i] / sqrt(d) (Algorithm 1 read
+ * backwards; R is orthogonal, so R^-1 = R^T). k_out, v_out: [B][t_cap][H_kv][d] doubles; rows >= seq_lens[b] are
+ * left untouched. */
+void iqo_reconstruct_rows(int B, int H_kv, int d, int t_cap, const float* quats, const float* levels8,
+                          const uint8_t* k_codes, const float* k_scales, const uint8_t* v_codes,
+                          const float* v_scales, const int32_t* seq_lens, double* k_out, double* v_out) {
+  int P = row_bytes(d);
+  double* Rs = (double*)malloc(sizeof(double) * (size_t)H_kv * d * d);
+  for (int g = 0; g < H_kv; g++) iqo_rotation_matrix(d, quats + (size_t)g * (d / 4) * 8, Rs + (size_t)g * d * d);
+#pragma omp parallel for schedule(dynamic) collapse(2)
+  for (int b = 0; b < B; b++)
+    for (int g = 0; g < H_kv; g++) {
+      int len = seq_lens[b];
+      if (len > t_cap) len = t_cap;
+      const double* R = Rs + (size_t)g * d * d;
+      size_t base = ((size_t)b * H_kv + g) * t_cap;
+      double xt[512];
+      for (int t = 0; t < len; t++)
+        for (int which = 0; which < 2; which++) {
+          if (which == 0) dequant_row(d, k_codes + (base + t) * P, k_scales[base + t], levels8, xt);
+          else dequant_v_row(d, v_codes + base * P, t, v_scales[base + t], levels8, xt);
+          double* o = (which == 0 ? k_out : v_out) + (((size_t)b * t_cap + t) * H_kv + g) * d;
+          for (int i = 0; i < d; i++) {  /* (R^T x~)_i = sum_j R[j][i] x~_j */
+            double acc = 0;
+            for (int j = 0; j < d; j++) acc += R[(size_t)j * d + i] * xt[j];
+            o[i] = acc;
+          }
+        }
+    }
+  free(Rs);
+}
+
 /* Scaled scores z_j of one (sequence b, query head h): z_out [len]. */
 void iqo_scores(int H_q, int H_kv, int d, int t_cap, double sm_scale, const float* quats, const float* levels8,
                 const uint16_t* q_bh, int b, int h, const uint8_t* k_codes, const float* k_scales, int len,

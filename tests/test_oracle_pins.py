@@ -336,6 +336,44 @@ def test_compressed_space_attention_equals_reconstruct_then_compute(codebooks, d
         assert np.max(np.abs(r["o_rot"] - ref)) > 0.05
 
 
+@pytest.mark.parametrize("d,T,H_q,H_kv,lens", [(128, 150, 4, 2, [150, 33, 0]), (256, 40, 2, 2, None)])
+def test_reconstructed_rows_give_the_same_attention_and_the_codebook_error(codebooks, d, T, H_q, H_kv, lens):
+    """The reconstruct-then-compute model (Figure 1, top) pinned from three sides: rows are the quantiser's input up to
+    the codebook's distortion, K and V agree with the row-by-row numpy statement, and textbook softmax attention on
+    the reconstructed tensors reproduces the compressed-space result (Appendix A) -- a transposed rotation, a V row
+    read from the wrong record or a missing 1/sqrt(d) fails at least one of them."""
+    B = 1 if lens is None else len(lens)
+    w = workloads.tiny(11, B, H_q, H_kv, d, T, lens)
+    lv, th = codebooks[d]
+    cache = oracle.new_cache(B, H_kv, d, w.t_cap)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), w.seq_lens, cache)
+    K, V = oracle.reconstruct_rows(w.quats, lv, cache, w.seq_lens, H_kv)
+    assert K.shape == (B, w.t_cap, H_kv, d)
+    for b in range(B):
+        n = int(w.seq_lens[b])
+        assert not K[b, n:].any() and not V[b, n:].any()                          # rows beyond the length stay zero
+        if n == 0:
+            continue
+        for x, xr in ((w.k[b, :n].astype(np.float64), K[b, :n]), (w.v[b, :n].astype(np.float64), V[b, :n])):
+            rel = np.sum((x - xr) ** 2, axis=-1) / np.sum(x * x, axis=-1)
+            assert 0.028 < float(rel.mean()) < 0.040                              # 3-bit Lloyd-Max on N(0,1): 0.0345
+        g, t = H_kv - 1, n - 1                                                    # one row, restated with the dense rotation
+        R = oracle.rotation_matrix(d, w.quats[g])
+        xt = float(cache["v_scales"][b, g, t]) * lv[oracle.v_row_codes(d, cache["v_codes"][b, g], t)].astype(np.float64) / math.sqrt(d)
+        assert np.allclose(V[b, t, g], R.T @ xt, atol=1e-13)
+    r = oracle.decode_attention(w.quats, lv, w.q, cache, w.seq_lens, H_kv)
+    for b in range(B):
+        n = int(w.seq_lens[b])
+        for h in range(H_q):
+            if n == 0:
+                assert not r["out"][b, h].any()
+                continue
+            z = K[b, :n, h // w.G] @ w.q[b, h].astype(np.float64) / math.sqrt(d)
+            p = np.exp(z - z.max())
+            assert np.allclose((p / p.sum()) @ V[b, :n, h // w.G], r["out"][b, h], atol=1e-12)
+            assert np.isclose(z.max() + math.log(p.sum()), r["lse"][b, h], atol=1e-12)
+
+
 def test_attention_special_cases(codebooks):
     d = 128
     lv, th = codebooks[d]
