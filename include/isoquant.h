@@ -199,6 +199,22 @@ int iq_combine_splits(const iq_shape* shape, const float* rot_dev, int32_t num_s
                       void* out, int32_t out_is_fp16, float* lse_out, int32_t* argmax_out, void* stream);
 
 /*
+ * Reconstruct-then-compute, first half (Figure 1, top; the execution model that Section 3 argues against and the
+ * fused path replaces): rows [0, seq_lens[b]) of every (sequence, KV head) dequantised and rotated back to the
+ * original space, x_hat = R^T x~ with x~_i = scale * level[code_i] / sqrt(d) (Algorithm 1 read backwards; R is
+ * orthogonal). The fp16 tensors it writes are what a standard attention kernel consumes; the call exists to measure
+ * that model against iq_decode_attention on the same packed cache, and as a way to read the cache back.
+ *   k_out, v_out   device binary16, element (b, t, g, i) at b*stride_b + t*stride_t + g*stride_h + i (strides in
+ *                  elements, multiples of 8; pointers 16-byte aligned), out_rows rows per sequence. Rows
+ *                  t >= min(seq_lens[b], out_rows) are not written.
+ *   codebook       only the levels are used (any fp32 values).
+ * fp32 arithmetic, one rounding to binary16 at the end.
+ */
+int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook,
+                        const iq_cache* cache, const int32_t* seq_lens_dev, void* k_out, void* v_out,
+                        int32_t out_rows, int64_t stride_b, int64_t stride_t, int64_t stride_h, void* stream);
+
+/*
  * Decode step for callers that cannot allocate device memory (the paper has no counterpart: its pipeline
  * is unsplit and needs no scratch). It runs iq_decode_attention followed by iq_combine_splits with the
  * split partials kept in a fixed array inside the library image instead of caller-provided buffers.

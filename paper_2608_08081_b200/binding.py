@@ -62,6 +62,8 @@ def _load():
     lib.iq_static_scratch_bytes.restype = ctypes.c_size_t
     lib.iq_decode_attention_static.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp,
                                                ctypes.POINTER(_IqCache), _vp, _i32, _vp, _i32, _vp, _vp, _vp]
+    lib.iq_reconstruct_rows.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), ctypes.POINTER(_IqCache), _vp,
+                                        _vp, _vp, _i32, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, _vp]
     lib.iq_suggest_splits.restype = _i32
     lib.iq_suggest_splits.argtypes = [ctypes.POINTER(_IqShape), _i32]
     return lib
@@ -211,6 +213,18 @@ def iq_decode_attention_static(shape: Shape, rot_dev, codebook: Codebook, q, cac
     _check(_lib.iq_decode_attention_static(ctypes.byref(cs), _ptr(rot_dev), ctypes.byref(cb), _ptr(q), ctypes.byref(cc),
                                            _ptr(seq_lens_dev), num_splits, _ptr(out), 1 if out.dtype == torch.float16 else 0,
                                            _ptr(lse_out), _ptr(status_dev), _stream(stream)), "iq_decode_attention_static")
+
+
+def iq_reconstruct_rows(shape: Shape, rot_dev, codebook: Codebook, cache: Cache, seq_lens_dev, k_out, v_out, stream=None) -> None:
+    """k_out, v_out: fp16 device tensors [B][T][H_kv][d] (any strides with a contiguous last dim): rows
+    [0, min(seq_lens[b], T)) receive the reconstructed K and V rows, the others are left as they are."""
+    assert k_out.dtype == torch.float16 and v_out.dtype == torch.float16 and k_out.shape == v_out.shape
+    assert k_out.stride() == v_out.stride() and k_out.stride(3) == 1
+    cs, cb, cc = shape.c(), codebook.c(), cache.c()
+    _check(_lib.iq_reconstruct_rows(ctypes.byref(cs), _ptr(rot_dev), ctypes.byref(cb), ctypes.byref(cc), _ptr(seq_lens_dev),
+                                    _ptr(k_out), _ptr(v_out), k_out.shape[1], k_out.stride(0), k_out.stride(1), k_out.stride(2),
+                                    _stream(stream)),
+           "iq_reconstruct_rows")
 
 
 def iq_suggest_splits(shape: Shape, max_seq_len: int) -> int:

@@ -303,6 +303,40 @@ int iq_combine_splits(const iq_shape* shape, const float* rot_dev, int32_t num_s
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }
 
+int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook, const iq_cache* cache,
+                        const int32_t* seq_lens_dev, void* k_out, void* v_out, int32_t out_rows, int64_t stride_b,
+                        int64_t stride_t, int64_t stride_h, void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (!rot_dev || !seq_lens_dev || !k_out || !v_out) return IQ_ERR_NULL;
+  if (out_rows < 0) return IQ_ERR_SHAPE;
+  if ((rc = check_codebook(codebook, false))) return rc;
+  if ((rc = check_cache(cache))) return rc;
+  if (!aligned16(k_out) || !aligned16(v_out) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
+  if (stride_b < 0 || stride_t < 0 || stride_h < 0) return IQ_ERR_SHAPE;
+  if ((stride_b & 7) || (stride_t & 7) || (stride_h & 7)) return IQ_ERR_ALIGN;
+  if (shape->batch == 0 || out_rows == 0) return IQ_OK;
+
+  iq::ReconstructParams p;
+  p.k_codes = cache->k_codes;
+  p.k_scales = cache->k_scales;
+  p.v_codes = cache->v_codes;
+  p.v_scales = cache->v_scales;
+  p.rot = rot_dev;
+  p.seq_lens = seq_lens_dev;
+  p.k_out = static_cast<__half*>(k_out);
+  p.v_out = static_cast<__half*>(v_out);
+  p.stride_b = stride_b;
+  p.stride_t = stride_t;
+  p.stride_h = stride_h;
+  p.n_kv_heads = shape->n_kv_heads;
+  p.t_cap = shape->t_cap;
+  p.out_rows = out_rows;
+  std::memcpy(p.levels, codebook->levels, sizeof(p.levels));
+  const cudaError_t e = iq::launch_reconstruct_rows(p, shape->head_dim, shape->batch, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
 int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len) {
   if (check_shape(shape) != IQ_OK || max_seq_len <= 0) return 1;
   static int n_sm_cached[64] = {};

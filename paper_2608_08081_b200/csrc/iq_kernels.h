@@ -69,6 +69,22 @@ struct CombineParams {
 };
 cudaError_t launch_combine_splits(const CombineParams& p, int head_dim, cudaStream_t stream);
 
+// ---- reconstruction of fp16 K/V rows from the packed cache (the reconstruct-then-compute model)
+struct ReconstructParams {
+  const uint8_t* k_codes;
+  const float* k_scales;
+  const uint8_t* v_codes;
+  const float* v_scales;
+  const float* rot;
+  const int32_t* seq_lens;
+  __half* k_out;
+  __half* v_out;
+  long long stride_b, stride_t, stride_h;  // in elements
+  int n_kv_heads, t_cap, out_rows;
+  float levels[8];
+};
+cudaError_t launch_reconstruct_rows(const ReconstructParams& p, int head_dim, int batch, cudaStream_t stream);
+
 // ---- rotation parameters
 cudaError_t launch_make_rotation(float* rot, int n_quats, uint64_t seed, cudaStream_t stream);
 cudaError_t launch_normalize_rotation(float* rot, int n_quats, cudaStream_t stream);

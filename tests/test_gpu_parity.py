@@ -198,6 +198,37 @@ def test_small_appends_take_the_same_codes_as_one_bulk_append(iq, torch, codeboo
     compare_caches(w2, th, g, ref, lens)
 
 
+@pytest.mark.parametrize("d", [128, 256])
+def test_reconstructed_rows_match_the_oracle(iq, torch, codebooks, d):
+    """iq_reconstruct_rows (the reconstruct-then-compute model's first half) against the oracle's dense R^T per row:
+    fp32 arithmetic and one rounding to binary16. Ragged lengths with an empty sequence, a partial last block, an
+    output shorter than the longest sequence, K and V interleaved in one strided buffer; rows that must not be
+    written keep their sentinel."""
+    B, H_q, H_kv, T, T_out = 3, 4, 2, 300, 256
+    lens = np.array([300, 129, 0], np.int32)
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    w = workloads.tiny(500 + d, B, H_q, H_kv, d, T, lens)
+    shape, rot, cache, status = gpu_quantize(iq, torch, w, cb, n_new=lens)
+    kv = torch.full((B, T_out, H_kv, 2 * d), 7.0, dtype=torch.float16, device="cuda")
+    k_out, v_out = kv[..., :d], kv[..., d:]
+    iq.iq_reconstruct_rows(shape, rot, cb, cache, torch.from_numpy(lens).cuda(), k_out, v_out)
+    torch.cuda.synchronize()
+    K, V = oracle.reconstruct_rows(w.quats, lv, cache_to_numpy(cache), lens, H_kv)
+    for got, ref in ((k_out.cpu().numpy().astype(np.float64), K), (v_out.cpu().numpy().astype(np.float64), V)):
+        for b in range(B):
+            n = min(int(lens[b]), T_out)
+            assert np.all(got[b, n:] == 7.0)
+            if n == 0:
+                continue
+            r = ref[b, :n]
+            bound = 2.0 ** -11 * 1.001 * np.abs(r) + 1e-5 * np.abs(r).max(axis=-1, keepdims=True)   # fp16 rounding + fp32 sums
+            assert np.all(np.abs(got[b, :n] - r) <= bound), float(np.max(np.abs(got[b, :n] - r) / bound))
+            x = (w.k if ref is K else w.v)[b, :n].astype(np.float64)
+            rel = np.sum((x - got[b, :n]) ** 2, axis=-1) / np.sum(x * x, axis=-1)
+            assert 0.025 < float(rel.mean()) < 0.045                                  # the codebook's distortion, end to end
+
+
 def test_combine_splits_in_isolation(iq, torch, codebooks):
     d, B, H_q, H_kv, S = 128, 3, 8, 2, 5
     g = np.random.default_rng(7)
