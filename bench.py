@@ -402,9 +402,65 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     }
     if graph_error:
         out["graph_error"] = graph_error
+    if not args.no_materialised and world == 1 and not per_seq:
+        out["reconstruct_then_compute"] = materialised_baseline(st, lens_tab[W + K], q_all[W + K - 1], ws, S, peak)
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = cpu_baseline(st, lens_tab[n_e2e_warm + n_e2e], q_all[W + K - 1])
     return out
+
+
+def materialised_baseline(st, lens_dev, q, ws, S, peak):
+    """The execution model the fused path replaces, on the same packed cache and the same step: iq_reconstruct_rows
+    writes the whole cache back as fp16 K/V, a library attention kernel (flash_attn) attends to them. Reported beside
+    the fused step, not part of it."""
+    import torch
+
+    iq, shape, cb, rot, cache = st["iq"], st["shape"], st["cb"], st["rot"], st["cache"]
+    B, H_q, H_kv, d, T = st["B"], st["H_q"], st["H_kv"], st["d"], st["t_cap"]
+    lens_dev = lens_dev.contiguous()
+    rows = int(lens_dev.sum().item())
+    res = {"what": "iq_reconstruct_rows (packed cache -> fp16 K/V, every cached row) + flash_attn_with_kvcache on the fp16 tensors; CUDA events",
+           "fp16_kv_bytes": rows * H_kv * d * 2 * 2}
+    try:
+        k = torch.empty((B, T, H_kv, d), dtype=torch.float16, device=lens_dev.device)
+        v = torch.empty_like(k)
+    except torch.OutOfMemoryError as e:
+        res["unavailable"] = f"fp16 K/V do not fit: {e}"[:160]
+        return res
+
+    def timed(f, reps):
+        f()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            f()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    rec_ms = timed(lambda: iq.iq_reconstruct_rows(shape, rot, cb, cache, lens_dev, k, v), 3)
+    rec_bytes = rows * H_kv * (bytes_per_row(d) + 2 * d * 2)           # packed rows in, fp16 K and V rows out
+    res["reconstruct_ms"] = round(rec_ms, 4)
+    res["reconstruct_gb_per_s"] = round(rec_bytes / (rec_ms * 1e-3) / 1e9, 1)
+    res["fp16_attention_ms_at_hbm_peak"] = round(res["fp16_kv_bytes"] / (peak * 1e9) * 1e3, 4)   # a perfect fp16 kernel
+    iq.decode_step(shape, rot, cb, q, cache, lens_dev, ws)             # the fused path on the same query and lengths
+    try:
+        from flash_attn import flash_attn_with_kvcache
+
+        q4 = q.reshape(B, 1, H_q, d)
+        att_ms = timed(lambda: flash_attn_with_kvcache(q4, k, v, cache_seqlens=lens_dev), 10)
+        o = flash_attn_with_kvcache(q4, k, v, cache_seqlens=lens_dev).reshape(B, H_q, d).float()
+        res["fp16_attention_ms"] = round(att_ms, 4)
+        res["fp16_attention_kernel"] = "flash_attn.flash_attn_with_kvcache"
+        res["max_abs_diff_vs_fused"] = float((o - ws.out.float()).abs().max().item())   # fp16 K/V rounding shifts the logits
+        res["max_abs_out"] = float(ws.out.float().abs().max().item())
+        res["ms_per_step"] = round(rec_ms + att_ms, 4)
+    except Exception as e:  # noqa: BLE001 -- the library kernel is optional; the reconstruction time stands on its own
+        res["fp16_attention_ms"] = None
+        res["fp16_attention_error"] = f"{type(e).__name__}: {e}"[:160]
+    del k, v
+    return res
 
 
 def cpu_baseline(st, lens, q_last, target_s: float = 12.0):
@@ -486,6 +542,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-materialised", action="store_true", help="skip the reconstruct-then-compute comparison")
     ap.add_argument("--no-graph", action="store_true", help="time the host-launched loop instead of a CUDA-graph replay of the K steps")
     ap.add_argument("--codebook", default="int8", choices=["int8", "fp16"])
     args = ap.parse_args()
