@@ -44,12 +44,15 @@ PER_SEQUENCE_LAUNCHES = {"config3_48layers", "config4_48layers"}
 DEFAULT_WORKLOAD = "config5_B32_ctx32768"
 T_CAP_MARGIN = 2048  # rows of head-room so that every sequence can take the benchmark's appends
 
-# DRAM traffic of one decode launch. The ncu capture of the decode kernel (summarised under profiles/; taken at B = 8
-# because a B = 32 launch is too large for a multi-pass capture) measured dram__bytes_read.sum = 1.0032 x the
-# algorithmic packed-KV bytes of the launch and dram__bytes_write.sum = 5.69 MB for 1.33 MB of partial results
-# (S = 5 slots). Reads scale with the rows processed; writes with the partial results.
-NCU_READ_PER_ALGORITHMIC_BYTE = 182.599 / 182.013
-NCU_WRITE_PER_PARTIAL_BYTE = 5.689 / 1.331
+# DRAM traffic of one decode launch, from two ncu captures of the decode kernel (summarised under profiles/): a
+# one-pass capture of the two DRAM byte counters on the full B = 32 launch (dram__bytes_read.sum = 614.22 MB for
+# 612.32 MB of algorithmic packed-KV bytes; dram__bytes_write.sum = 7.8 and 11.0 MB for 2.13 MB of partial results,
+# S = 2 slots) and the multi-pass capture at B = 8 (182.60 MB for 182.01 MB; 5.69 MB for 1.33 MB of partials, S = 5).
+# Both give reads = 1.003 x the algorithmic bytes and writes = 4.3 - 4.4 x the partial results (the rest of the
+# writes are dirty lines of the kernels before it leaving L2). Reads scale with the rows processed, writes with the
+# partial results.
+NCU_READ_PER_ALGORITHMIC_BYTE = 614.22 / 612.32
+NCU_WRITE_PER_PARTIAL_BYTE = 0.5 * (7.76 + 11.02) / 2.13
 
 
 GRAPH_EVENT_STRIDE = 4
@@ -385,7 +388,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "frac_of_8TBs": round(value / world / 8000.0, 4),
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
                      "traffic": decode_traffic_bytes(sum(timed_launch_bytes) / len(dec_ms), B // n_groups, H_q, S, d),
-                     "traffic_source": "ncu capture at B = 8 scaled by rows processed (reads) and partial results (writes)",
+                     "traffic_source": "ncu one-pass DRAM byte counters on the full B = 32 launch, scaled by rows processed (reads) and partial results (writes)",
                      "kernel": "decode_kernel", "peak_source": peak_src,
                      "avg_launch_ms": round(dec_avg_ms, 4), "launches_timed": len(dec_ms),
                      "algorithmic_bytes_per_launch": int(sum(timed_launch_bytes) / len(dec_ms))},
