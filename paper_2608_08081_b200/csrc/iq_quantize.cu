@@ -36,20 +36,30 @@ struct RowQuantizer {
   static constexpr int LPR = D / E;        // lanes per row: 8 or 16
   static constexpr int RPW = 32 / LPR;     // rows per warp: 4 or 2
   static constexpr int NB = E / 4;         // SO(4) blocks per lane
+  // The head's d/4 block matrices live in shared memory, 4 blocks (64 floats) + 4 floats of padding per lane-in-row:
+  // with the padding the 8 or 16 different 16-byte rows a warp reads at a time fall into different banks. Keeping
+  // them in registers (64 per thread) halves the number of resident warps.
+  static constexpr int M_STRIDE = NB * 16 + 4;
+  static constexpr int M_FLOATS = LPR * M_STRIDE;
   const float* qbase;      // this lane's NB quaternion pairs
   const float* th_global;  // the 7 thresholds in memory (for the out-of-line fp64 path)
-  float M[NB][4][4];
+  const float4* Ms;        // this lane's NB matrices in shared memory, row-major
   float th[7];
 
-  __device__ __forceinline__ void init(const float* rot_head, const float* thresholds, int lane) {
-    qbase = rot_head + (size_t)(lane % LPR) * NB * 8;
+  // Called by every thread of the CTA (then __syncthreads()): the matrices of the head's blocks into m_smem.
+  __device__ __forceinline__ static void fill_matrices(const float* rot_head, float* m_smem, int tid, int n_threads) {
+    for (int blk = tid; blk < D / 4; blk += n_threads) {
+      float Mt[4][4];
+      so4_matrix<float>(rot_head + (size_t)blk * 8, Mt);
+      float* dst = m_smem + (blk / NB) * M_STRIDE + (blk % NB) * 16;
 #pragma unroll
-    for (int j = 0; j < NB; j++) {
-      float q8[8];
-#pragma unroll
-      for (int i = 0; i < 8; i++) q8[i] = qbase[j * 8 + i];
-      so4_matrix<float>(q8, M[j]);
+      for (int r = 0; r < 4; r++) *reinterpret_cast<float4*>(dst + 4 * r) = make_float4(Mt[r][0], Mt[r][1], Mt[r][2], Mt[r][3]);
     }
+  }
+
+  __device__ __forceinline__ void init(const float* rot_head, const float* thresholds, int lane, const float* m_smem) {
+    qbase = rot_head + (size_t)(lane % LPR) * NB * 8;
+    Ms = reinterpret_cast<const float4*>(m_smem + (lane % LPR) * M_STRIDE);
 #pragma unroll
     for (int i = 0; i < 7; i++) th[i] = thresholds[i];
     th_global = thresholds;
@@ -152,7 +162,15 @@ struct RowQuantizer {
 
     // Step 2: u = sqrt(d) * R x^ = M_b (H_unnormalised x) / s  (the two sqrt(d) factors cancel)
     wht<float>(x, lane);
-    so4_apply<float, E, false>(M, x);
+#pragma unroll
+    for (int j = 0; j < NB; j++) {
+      const float x0 = x[4 * j], x1 = x[4 * j + 1], x2 = x[4 * j + 2], x3 = x[4 * j + 3];
+#pragma unroll
+      for (int r = 0; r < 4; r++) {
+        const float4 m = Ms[4 * j + r];
+        x[4 * j + r] = m.x * x0 + m.y * x1 + m.z * x2 + m.w * x3;
+      }
+    }
 
     // Step 3: codes, with a guard band around the thresholds
     bool any_near = false;
@@ -203,7 +221,7 @@ __device__ __forceinline__ void pack_pair(const int (&code)[16], int lane, uint3
 // K rows: packed row-major (3d/8 bytes per row).
 // ---------------------------------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(QA_WARPS * 32, 3) quantize_append_k_kernel(const __grid_constant__ QuantizeParams p) {
+__global__ void __launch_bounds__(QA_WARPS * 32, 5) quantize_append_k_kernel(const __grid_constant__ QuantizeParams p) {
   using RQ = RowQuantizer<D>;
   constexpr int LPR = RQ::LPR, RPW = RQ::RPW;
   grid_dependency_wait();
@@ -215,13 +233,17 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 3) quantize_append_k_kernel(con
 
   int n_new = p.n_new ? p.n_new[b] : p.n_new_max;
   n_new = min(n_new, p.n_new_max);
+  if (blockIdx.x * QA_WARPS * QA_ROWS_PER_WARP >= n_new) return;  // the whole CTA
+  __shared__ __align__(16) float m_s[RQ::M_FLOATS];
+  RQ::fill_matrices(p.rot + (size_t)h * (D / 4) * 8, m_s, threadIdx.x, QA_WARPS * 32);
+  __syncthreads();
   const int row_begin = (blockIdx.x * QA_WARPS + warp) * QA_ROWS_PER_WARP;
   if (row_begin >= n_new) return;
   const int row_end = min(n_new, row_begin + QA_ROWS_PER_WARP);
   const int pos0 = p.append_pos[b];
 
   RQ rq;
-  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane);
+  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane, m_s);
   const int li = lane % LPR, sub = lane / LPR;  // lane within the row, row within the warp
   const __half* src_base = p.k_new + (size_t)b * p.stride_b + (size_t)h * p.stride_h + li * 16;
   const size_t slab = ((size_t)b * p.n_kv_heads + h) * (size_t)p.t_cap;
@@ -272,7 +294,7 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 3) quantize_append_k_kernel(con
 // other CTA touches them.
 // ---------------------------------------------------------------------------------------------------------
 template <int D>
-__global__ void __launch_bounds__(128, 3) quantize_append_v_kernel(const __grid_constant__ QuantizeParams p) {
+__global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_constant__ QuantizeParams p) {
   using RQ = RowQuantizer<D>;
   constexpr int LPR = RQ::LPR, RPW = RQ::RPW;
   __shared__ __align__(16) uint8_t codes_s[32][D + 16];  // +16: the 16-byte stores of different rows hit different banks
@@ -300,8 +322,11 @@ __global__ void __launch_bounds__(128, 3) quantize_append_v_kernel(const __grid_
     return;
   }
 
+  __shared__ __align__(16) float m_s[RQ::M_FLOATS];
+  RQ::fill_matrices(p.rot + (size_t)h * (D / 4) * 8, m_s, tid, 128);
+  __syncthreads();
   RQ rq;
-  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane);
+  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane, m_s);
   const int li = lane % LPR, sub = lane / LPR;
   const __half* src_base = p.v_new + (size_t)b * p.stride_b + (size_t)h * p.stride_h + li * 16;
   uint4 rr[32 / (4 * RPW)][2];  // all of this warp's rows are fetched up front
