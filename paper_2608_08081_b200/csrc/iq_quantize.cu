@@ -288,16 +288,18 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 5) quantize_append_k_kernel(con
 // ---------------------------------------------------------------------------------------------------------
 // V rows: stored token-transposed. For every block of 128 cache rows and every coordinate c there is one
 // 48-byte record holding the 128 codes of coordinate c, arranged like a packing unit sequence with the
-// row-in-block in the role of the entry. One CTA handles one 32-row unit of one (sequence, KV head): its warps
-// quantise the unit's new rows, the codes go through shared memory, and thread c assembles the three words of
-// (unit, coordinate c). Words that are only partly covered by new rows are read, merged and written back; no
-// other CTA touches them.
+// row-in-block in the role of the entry. One CTA handles one 128-row block of one (sequence, KV head): its warps
+// quantise the block's new rows, the codes go through shared memory, and thread c assembles the record of
+// coordinate c -- written whole (48 contiguous bytes per thread, 1536 per warp) when the block is entirely new,
+// otherwise unit by unit with the words that keep old entries read, merged and written back; no other CTA touches
+// them.
 // ---------------------------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_constant__ QuantizeParams p) {
   using RQ = RowQuantizer<D>;
   constexpr int LPR = RQ::LPR, RPW = RQ::RPW;
-  __shared__ __align__(16) uint8_t codes_s[32][D + 16];  // +16: the 16-byte stores of different rows hit different banks
+  __shared__ __align__(16) uint8_t codes_s[128][D + 16];  // +16: the 16-byte stores of different rows hit different banks
+  __shared__ __align__(16) float m_s[RQ::M_FLOATS];
 
   grid_dependency_wait();
   allow_dependent_launch();
@@ -308,12 +310,12 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
   n_new = min(n_new, p.n_new_max);
   if (n_new <= 0) return;
   const long long pos0 = p.append_pos[b];
-  const long long unit = (pos0 >= 0 ? pos0 / 32 : -((-pos0 + 31) / 32)) + blockIdx.x;  // floor(pos0 / 32) + x
-  const long long t_lo = max(unit * 32, pos0);                 // first cache row of this unit that is appended
-  const long long t_hi = min(unit * 32 + 32, pos0 + n_new);    // one past the last
+  const long long blkg = (pos0 >= 0 ? pos0 / 128 : -((-pos0 + 127) / 128)) + blockIdx.x;  // floor(pos0 / 128) + x
+  const long long t_lo = max(blkg * 128, pos0);                  // first cache row of this block that is appended
+  const long long t_hi = min(blkg * 128 + 128, pos0 + n_new);    // one past the last
   if (t_lo >= t_hi) return;
   const size_t slab = ((size_t)b * p.n_kv_heads + h) * (size_t)p.t_cap;
-  const bool in_cache = unit >= 0 && unit * 32 + 32 <= p.t_cap;  // t_cap is a multiple of 128
+  const bool in_cache = blkg >= 0 && blkg * 128 + 128 <= p.t_cap;  // t_cap is a multiple of 128
   if (!in_cache) {
     if (tid == 0 && p.status) {
       atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
@@ -322,55 +324,83 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
     return;
   }
 
-  __shared__ __align__(16) float m_s[RQ::M_FLOATS];
   RQ::fill_matrices(p.rot + (size_t)h * (D / 4) * 8, m_s, tid, 128);
   __syncthreads();
   RQ rq;
   rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane, m_s);
   const int li = lane % LPR, sub = lane / LPR;
   const __half* src_base = p.v_new + (size_t)b * p.stride_b + (size_t)h * p.stride_h + li * 16;
-  uint4 rr[32 / (4 * RPW)][2];  // all of this warp's rows are fetched up front
-#pragma unroll
-  for (int it = 0; it < 32 / (4 * RPW); it++) {
-    const long long t = t_lo + (it * 4 + warp) * RPW + sub;
-    rr[it][0] = rr[it][1] = make_uint4(0u, 0u, 0u, 0u);
-    if (t < t_hi) {
-      const uint4* src = reinterpret_cast<const uint4*>(src_base + (size_t)(t - pos0) * p.stride_t);
-      rr[it][0] = __ldg(src);
-      rr[it][1] = __ldg(src + 1);
+  const int n_rows = (int)(t_hi - t_lo);
+  // the warps take the block's new rows RPW at a time, interleaved; the next rows are in flight during the math
+  auto fetch = [&](int i0, uint4& r0, uint4& r1, bool& active) {
+    const int i = i0 + sub;
+    active = i < n_rows;
+    r0 = r1 = make_uint4(0u, 0u, 0u, 0u);
+    if (active) {
+      const uint4* src = reinterpret_cast<const uint4*>(src_base + (size_t)(t_lo + i - pos0) * p.stride_t);
+      r0 = __ldg(src);
+      r1 = __ldg(src + 1);
     }
-  }
-#pragma unroll
-  for (int it = 0; it < 32 / (4 * RPW); it++) {
-    const long long t0 = t_lo + (it * 4 + warp) * RPW;
-    if (t0 >= t_hi) break;
-    const long long t = t0 + sub;
-    const bool active = t < t_hi;
+  };
+  uint4 n0, n1;
+  bool n_active;
+  fetch(warp * RPW, n0, n1, n_active);
+  for (int i0 = warp * RPW; i0 < n_rows; i0 += 4 * RPW) {
+    const uint4 r0 = n0, r1 = n1;
+    const bool active = n_active;
+    if (i0 + 4 * RPW < n_rows) fetch(i0 + 4 * RPW, n0, n1, n_active);
+    const long long t = t_lo + i0 + sub;
     int code[16];
-    const float s = rq.run(rr[it][0], rr[it][1], active, lane, code, p.status);
+    const float s = rq.run(r0, r1, active, lane, code, p.status);
     if (active) {
       uint32_t pk[4];
 #pragma unroll
       for (int q = 0; q < 4; q++)
         pk[q] = (uint32_t)code[4 * q] | ((uint32_t)code[4 * q + 1] << 8) | ((uint32_t)code[4 * q + 2] << 16) | ((uint32_t)code[4 * q + 3] << 24);
-      *reinterpret_cast<uint4*>(&codes_s[t & 31][li * 16]) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      *reinterpret_cast<uint4*>(&codes_s[t & 127][li * 16]) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
       if (li == 0) p.v_scales[slab + (size_t)t] = s;
     }
   }
   __syncthreads();
 
-  const int c_lo = (int)(t_lo & 31), c_hi = (int)(t_hi - unit * 32);  // rows [c_lo, c_hi) of the unit are new
-  const size_t blk = (size_t)(unit * 32) / 128;
-  const int u = (int)((unit * 32) % 128) / 32;
-  const bool full = (c_lo == 0 && c_hi == 32);
+  // Thread c assembles the record of coordinate c: four packing units of three words, the row-in-block as the entry.
+  const int c_lo = (int)(t_lo & 127), c_hi = (int)(t_hi - blkg * 128);  // rows [c_lo, c_hi) of the block are new
 #pragma unroll
   for (int j = 0; j < D / 128; j++) {
     const int c = tid + 128 * j;  // coordinate
-    uint32_t w[3] = {0u, 0u, 0u}, m[3] = {0u, 0u, 0u};
+    uint32_t* rec = reinterpret_cast<uint32_t*>(p.v_codes + ((slab / 128 + (size_t)blkg) * D + c) * 48);
+    if (c_lo == 0 && c_hi == 128) {  // the whole block is new: the record is written with three 16-byte stores
+      uint32_t w[12];
 #pragma unroll
-    for (int r = 0; r < 32; r++) {
-      if (r >= c_lo && r < c_hi) {
-        const uint32_t cd = codes_s[r][c];
+      for (int u = 0; u < 4; u++) {
+        uint32_t w0 = 0u, w1 = 0u, w2 = 0u;
+#pragma unroll
+        for (int r = 0; r < 8; r++) {
+          w0 |= (uint32_t)codes_s[32 * u + r][c] << (4 * r);
+          w1 |= (uint32_t)codes_s[32 * u + 8 + r][c] << (4 * r);
+          w2 |= (uint32_t)codes_s[32 * u + 16 + r][c] << (4 * r);
+        }
+#pragma unroll
+        for (int r = 0; r < 8; r++) {  // entries 24..31: bit k of the code into the top bit of nibble r of word k
+          const uint32_t cd = codes_s[32 * u + 24 + r][c];
+          w0 |= (cd & 1u) << (4 * r + 3);
+          w1 |= ((cd >> 1) & 1u) << (4 * r + 3);
+          w2 |= ((cd >> 2) & 1u) << (4 * r + 3);
+        }
+        w[3 * u] = w0; w[3 * u + 1] = w1; w[3 * u + 2] = w2;
+      }
+      uint4* dst = reinterpret_cast<uint4*>(rec);
+      dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+      dst[2] = make_uint4(w[8], w[9], w[10], w[11]);
+      continue;
+    }
+    for (int u = 0; u < 4; u++) {  // partly covered block: unit by unit, words that keep old entries are merged
+      const int lo = max(c_lo, 32 * u) - 32 * u, hi = min(c_hi, 32 * u + 32) - 32 * u;
+      if (lo >= hi) continue;
+      uint32_t w[3] = {0u, 0u, 0u}, m[3] = {0u, 0u, 0u};
+      for (int r = lo; r < hi; r++) {
+        const uint32_t cd = codes_s[32 * u + r][c];
         if (r < 24) {
           w[r >> 3] |= cd << (4 * (r & 7));
           m[r >> 3] |= 7u << (4 * (r & 7));
@@ -383,12 +413,12 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
           }
         }
       }
-    }
-    uint32_t* dst = reinterpret_cast<uint32_t*>(p.v_codes + ((slab / 128 + blk) * D + c) * 48) + 3 * u;
+      uint32_t* dst = rec + 3 * u;
 #pragma unroll
-    for (int k = 0; k < 3; k++) {
-      if (m[k] == 0u) continue;
-      dst[k] = full ? w[k] : ((dst[k] & ~m[k]) | w[k]);
+      for (int k = 0; k < 3; k++) {
+        if (m[k] == 0u) continue;
+        dst[k] = (m[k] == 0xFFFFFFFFu) ? w[k] : ((dst[k] & ~m[k]) | w[k]);
+      }
     }
   }
 }
@@ -562,7 +592,7 @@ cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int ba
   if (p.n_new_max <= 0 || batch <= 0) return cudaSuccess;
   const int rows_per_cta = QA_WARPS * QA_ROWS_PER_WARP;
   dim3 kgrid((p.n_new_max + rows_per_cta - 1) / rows_per_cta, p.n_kv_heads, batch);
-  dim3 vgrid((p.n_new_max + 31) / 32 + 1, p.n_kv_heads, batch);  // +1: the first row may sit in the middle of a unit
+  dim3 vgrid((p.n_new_max + 127) / 128 + 1, p.n_kv_heads, batch);  // +1: the first row may sit in the middle of a block
   if (p.n_new_max <= QA_FEW_ROWS) {
     dim3 grid(2, p.n_kv_heads, batch);  // x = 0: the K rows, x = 1: the V rows of (sequence, KV head)
     return head_dim == 128 ? launch_after_predecessor(quantize_append_few_kernel<128>, grid, dim3(32), 0, stream, p)
