@@ -26,6 +26,19 @@ __device__ __forceinline__ int decide_code(T u, const float (&th)[7], bool& near
   return (b2 ? 4 : 0) + (b1 ? 2 : 0) + (b0 ? 1 : 0);
 }
 
+// The same decision for a codebook that is symmetric about zero (t_3 = 0, t_{6-k} = -t_k; the Lloyd-Max codebooks of a
+// symmetric density are): two compares on |u| and the sign. Exact ties fall inside the guard band and are re-decided.
+// dmin carries the smallest distance to a threshold seen so far, so that one test serves all coordinates of a lane.
+__device__ __forceinline__ int decide_code_sym(float u, float a1, float a2, float a3, float& dmin) {
+  const float a = fabsf(u);
+  const bool b1 = a > a2;
+  const float p0 = b1 ? a3 : a1;
+  const bool b0 = a > p0;
+  dmin = fminf(fminf(dmin, a), fminf(fabsf(a - a2), fabsf(a - p0)));
+  const int mag = (b1 ? 2 : 0) + (b0 ? 1 : 0);
+  return u > 0.f ? 4 + mag : 3 - mag;
+}
+
 // Work mapping of the row kernels: a row is shared by LPR = d/16 lanes, 16 consecutive coordinates (4 whole SO(4)
 // blocks) per lane, so a warp holds 32/LPR rows at a time (4 at d = 128, 2 at d = 256). The Walsh-Hadamard
 // butterfly runs 4 stages inside the lane and log2(LPR) xor-shuffle stages across the row's lanes; a 32-coordinate
@@ -139,6 +152,7 @@ struct RowQuantizer {
 
   // Algorithm 1, steps 1-3 for the row this lane belongs to (r0, r1 = this lane's 16 fp16 values, zeros for the
   // lanes of a row that is not written; those lanes still take part in the shuffles). Returns the fp32 scale.
+  template <bool SYM>
   __device__ __forceinline__ float run(const uint4& r0, const uint4& r1, bool active, int lane, int (&code)[E],
                                        uint32_t* status) const {
     float x[E];
@@ -174,11 +188,18 @@ struct RowQuantizer {
 
     // Step 3: codes, with a guard band around the thresholds
     bool any_near = false;
+    if (SYM) {
+      float dmin = 1.f;
 #pragma unroll
-    for (int e = 0; e < E; e++) {
-      bool nb;
-      code[e] = decide_code<float>(x[e] * inv_s, th, nb, GUARD_BAND);
-      any_near |= nb;
+      for (int e = 0; e < E; e++) code[e] = decide_code_sym(x[e] * inv_s, th[4], th[5], th[6], dmin);
+      any_near = dmin <= GUARD_BAND;
+    } else {
+#pragma unroll
+      for (int e = 0; e < E; e++) {
+        bool nb;
+        code[e] = decide_code<float>(x[e] * inv_s, th, nb, GUARD_BAND);
+        any_near |= nb;
+      }
     }
     const unsigned rows_near = __ballot_sync(FULL, any_near && active);
     if (rows_near) {
@@ -220,7 +241,7 @@ __device__ __forceinline__ void pack_pair(const int (&code)[16], int lane, uint3
 // ---------------------------------------------------------------------------------------------------------
 // K rows: packed row-major (3d/8 bytes per row).
 // ---------------------------------------------------------------------------------------------------------
-template <int D>
+template <int D, bool SYM>
 __global__ void __launch_bounds__(QA_WARPS * 32, 5) quantize_append_k_kernel(const __grid_constant__ QuantizeParams p) {
   using RQ = RowQuantizer<D>;
   constexpr int LPR = RQ::LPR, RPW = RQ::RPW;
@@ -273,7 +294,7 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 5) quantize_append_k_kernel(con
       atomicAdd(&p.status[2], 1u);
     }
     int code[16];
-    const float s = rq.run(r0, r1, active, lane, code, p.status);
+    const float s = rq.template run<SYM>(r0, r1, active, lane, code, p.status);
     uint32_t w0, w1;
     pack_pair(code, lane, w0, w1);
     if (active) {
@@ -294,7 +315,7 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 5) quantize_append_k_kernel(con
 // otherwise unit by unit with the words that keep old entries read, merged and written back; no other CTA touches
 // them.
 // ---------------------------------------------------------------------------------------------------------
-template <int D>
+template <int D, bool SYM>
 __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_constant__ QuantizeParams p) {
   using RQ = RowQuantizer<D>;
   constexpr int LPR = RQ::LPR, RPW = RQ::RPW;
@@ -351,7 +372,7 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
     if (i0 + 4 * RPW < n_rows) fetch(i0 + 4 * RPW, n0, n1, n_active);
     const long long t = t_lo + i0 + sub;
     int code[16];
-    const float s = rq.run(r0, r1, active, lane, code, p.status);
+    const float s = rq.template run<SYM>(r0, r1, active, lane, code, p.status);
     if (active) {
       uint32_t pk[4];
 #pragma unroll
@@ -599,11 +620,22 @@ cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int ba
                            : launch_after_predecessor(quantize_append_few_kernel<256>, grid, dim3(32), 0, stream, p);
   }
   // (the V kernel may start under the K kernel: they write different arrays)
-  cudaError_t e = head_dim == 128 ? launch_after_predecessor(quantize_append_k_kernel<128>, kgrid, dim3(QA_WARPS * 32), 0, stream, p)
-                                  : launch_after_predecessor(quantize_append_k_kernel<256>, kgrid, dim3(QA_WARPS * 32), 0, stream, p);
+  const float* t = p.thresholds;
+  const bool sym = t[3] == 0.f && t[0] == -t[6] && t[1] == -t[5] && t[2] == -t[4];  // two compares per coordinate instead of three
+  const dim3 kblock(QA_WARPS * 32), vblock(128);
+  cudaError_t e;
+  if (head_dim == 128)
+    e = sym ? launch_after_predecessor(quantize_append_k_kernel<128, true>, kgrid, kblock, 0, stream, p)
+            : launch_after_predecessor(quantize_append_k_kernel<128, false>, kgrid, kblock, 0, stream, p);
+  else
+    e = sym ? launch_after_predecessor(quantize_append_k_kernel<256, true>, kgrid, kblock, 0, stream, p)
+            : launch_after_predecessor(quantize_append_k_kernel<256, false>, kgrid, kblock, 0, stream, p);
   if (e != cudaSuccess) return e;
-  return head_dim == 128 ? launch_after_predecessor(quantize_append_v_kernel<128>, vgrid, dim3(128), 0, stream, p)
-                         : launch_after_predecessor(quantize_append_v_kernel<256>, vgrid, dim3(128), 0, stream, p);
+  if (head_dim == 128)
+    return sym ? launch_after_predecessor(quantize_append_v_kernel<128, true>, vgrid, vblock, 0, stream, p)
+               : launch_after_predecessor(quantize_append_v_kernel<128, false>, vgrid, vblock, 0, stream, p);
+  return sym ? launch_after_predecessor(quantize_append_v_kernel<256, true>, vgrid, vblock, 0, stream, p)
+             : launch_after_predecessor(quantize_append_v_kernel<256, false>, vgrid, vblock, 0, stream, p);
 }
 
 }  // namespace iq

@@ -229,6 +229,38 @@ def test_reconstructed_rows_match_the_oracle(iq, torch, codebooks, d):
             assert 0.025 < float(rel.mean()) < 0.045                                  # the codebook's distortion, end to end
 
 
+@pytest.mark.parametrize("d", [128, 256])
+def test_codebook_that_is_not_symmetric_takes_the_same_codes(iq, torch, codebooks, d):
+    """The bulk kernels decide with two compares on |u| when the thresholds are symmetric about zero and with a
+    three-step search otherwise: shifted thresholds must still give the oracle's codes, in the bulk kernels (300
+    rows at once, a partly filled last block) and in the few-rows kernel (3 more rows)."""
+    lv, th = codebooks[d]
+    th2 = (np.asarray(th, np.float64) + np.array([0.013, -0.02, 0.007, 0.011, 0.0, -0.017, 0.02])).astype(np.float32)
+    assert np.all(np.diff(th2) > 0) and th2[3] != 0
+    cb = iq.Codebook(tuple(float(x) for x in lv), tuple(float(x) for x in th2))
+    T = 303
+    w = workloads.tiny(900 + d, 2, 4, 2, d, T)
+    lens = np.array([300, 170], np.int32)
+    shape, rot, cache, status = gpu_quantize(iq, torch, w, cb, n_new=lens)
+    k, v = torch.from_numpy(w.k).cuda(), torch.from_numpy(w.v).cuda()
+    idx = (lens[:, None] + np.arange(3)[None, :]).clip(max=T - 1)
+    kk = torch.stack([k[b, idx[b]] for b in range(2)])
+    vv = torch.stack([v[b, idx[b]] for b in range(2)])
+    iq.iq_quantize_append(shape, rot, cb, kk, vv, torch.from_numpy(lens).cuda(), None, 3, cache, status)
+    torch.cuda.synchronize()
+    lens2 = lens + 3
+    ref = oracle.new_cache(2, 2, d, w.t_cap)
+    oracle.quantize_append(w.quats, th2, w.k, w.v, np.zeros(2, np.int32), lens, ref)
+    oracle.quantize_append(w.quats, th2, kk.cpu().numpy(), vv.cpu().numpy(), lens, None, ref)
+    full_k = np.zeros_like(w.k); full_v = np.zeros_like(w.v)
+    for b in range(2):
+        full_k[b, :lens[b]] = w.k[b, :lens[b]]; full_v[b, :lens[b]] = w.v[b, :lens[b]]
+        full_k[b, lens[b]:lens2[b]] = w.k[b, idx[b]]; full_v[b, lens[b]:lens2[b]] = w.v[b, idx[b]]
+    w2 = workloads.Workload("asym", 2, 4, 2, d, w.t_cap, full_k, full_v, w.q, w.quats, lens2)
+    print(compare_caches(w2, th2, cache_to_numpy(cache), ref, lens2))
+    assert status.cpu().numpy()[0] == 0
+
+
 def test_combine_splits_in_isolation(iq, torch, codebooks):
     d, B, H_q, H_kv, S = 128, 3, 8, 2, 5
     g = np.random.default_rng(7)
