@@ -215,6 +215,25 @@ int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_co
                         int32_t out_rows, int64_t stride_b, int64_t stride_t, int64_t stride_h, void* stream);
 
 /*
+ * One whole decode step from HOST buffers, in one call: the step's inputs go to the device in one copy, one new row
+ * per sequence is appended (Algorithm 1), the fused decode and the merge run (Appendix A), the output comes back and
+ * the call returns when it has arrived. It is iq_quantize_append (n_new_max = 1) + iq_decode_attention +
+ * iq_combine_splits with the two copies and one cudaStreamSynchronize around them; unlike every other call it blocks.
+ *   inputs_host    host (pinned for a truly asynchronous copy) binary16: q [batch][n_q_heads][head_dim], then
+ *                  k_new [batch][n_kv_heads][head_dim], then v_new [batch][n_kv_heads][head_dim], contiguous.
+ *   inputs_dev     device staging buffer of the same size, 16-byte aligned, caller-owned.
+ *   append_pos_dev device int32 [batch]: row that receives the new K/V row (the sequence's length before the step).
+ *   seq_lens_dev   device int32 [batch]: rows attended to (the length after the step).
+ *   out_dev        device [batch][n_q_heads][head_dim], fp32 or binary16 (out_is_fp16); out_host: host, same size.
+ * part_acc / part_ml / num_splits / status_dev as for iq_decode_attention. No lse or argmax output.
+ */
+int iq_decode_step_host(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook,
+                        const void* inputs_host, void* inputs_dev, const int32_t* append_pos_dev,
+                        const int32_t* seq_lens_dev, const iq_cache* cache, int32_t num_splits, float* part_acc,
+                        float* part_ml, void* out_dev, void* out_host, int32_t out_is_fp16, uint32_t* status_dev,
+                        void* stream);
+
+/*
  * Decode step for callers that cannot allocate device memory (the paper has no counterpart: its pipeline
  * is unsplit and needs no scratch). It runs iq_decode_attention followed by iq_combine_splits with the
  * split partials kept in a fixed array inside the library image instead of caller-provided buffers.

@@ -21,6 +21,7 @@ from .binding import (  # noqa: F401
     iq_rotation_floats,
     iq_row_bytes,
     iq_strerror,
+    iq_decode_step_host,
     iq_reconstruct_rows,
     iq_suggest_splits,
     iq_version,

@@ -64,6 +64,8 @@ def _load():
                                                ctypes.POINTER(_IqCache), _vp, _i32, _vp, _i32, _vp, _vp, _vp]
     lib.iq_reconstruct_rows.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), ctypes.POINTER(_IqCache), _vp,
                                         _vp, _vp, _i32, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, _vp]
+    lib.iq_decode_step_host.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp, _vp, _vp, _vp,
+                                        ctypes.POINTER(_IqCache), _i32, _vp, _vp, _vp, _vp, _i32, _vp, _vp]
     lib.iq_suggest_splits.restype = _i32
     lib.iq_suggest_splits.argtypes = [ctypes.POINTER(_IqShape), _i32]
     return lib
@@ -225,6 +227,20 @@ def iq_reconstruct_rows(shape: Shape, rot_dev, codebook: Codebook, cache: Cache,
                                     _ptr(k_out), _ptr(v_out), k_out.shape[1], k_out.stride(0), k_out.stride(1), k_out.stride(2),
                                     _stream(stream)),
            "iq_reconstruct_rows")
+
+
+def iq_decode_step_host(shape: Shape, rot_dev, codebook: Codebook, inputs_host, inputs_dev, append_pos_dev, seq_lens_dev,
+                        cache: Cache, ws: "DecodeWorkspace", out_dev, out_host, stream=None) -> None:
+    """One decode step from host buffers (blocking): inputs_host = fp16 host tensor holding q, k_new, v_new back to
+    back; inputs_dev a device tensor of the same size; out_dev / out_host fp32 or fp16 [B][H_q][d]."""
+    assert inputs_host.dtype == torch.float16 and inputs_dev.dtype == torch.float16 and inputs_host.is_contiguous()
+    n = shape.batch * (shape.n_q_heads + 2 * shape.n_kv_heads) * shape.head_dim
+    assert inputs_host.numel() == n and inputs_dev.numel() == n and out_dev.dtype == out_host.dtype
+    cs, cb, cc = shape.c(), codebook.c(), cache.c()
+    _check(_lib.iq_decode_step_host(ctypes.byref(cs), _ptr(rot_dev), ctypes.byref(cb), _ptr(inputs_host), _ptr(inputs_dev),
+                                    _ptr(append_pos_dev), _ptr(seq_lens_dev), ctypes.byref(cc), ws.num_splits, _ptr(ws.part_acc),
+                                    _ptr(ws.part_ml), _ptr(out_dev), _ptr(out_host), 1 if out_dev.dtype == torch.float16 else 0,
+                                    _ptr(ws.status), _stream(stream)), "iq_decode_step_host")
 
 
 def iq_suggest_splits(shape: Shape, max_seq_len: int) -> int:

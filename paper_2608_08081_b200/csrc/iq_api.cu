@@ -337,6 +337,34 @@ int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_co
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }
 
+int iq_decode_step_host(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook, const void* inputs_host,
+                        void* inputs_dev, const int32_t* append_pos_dev, const int32_t* seq_lens_dev, const iq_cache* cache,
+                        int32_t num_splits, float* part_acc, float* part_ml, void* out_dev, void* out_host,
+                        int32_t out_is_fp16, uint32_t* status_dev, void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (!inputs_host || !inputs_dev || !out_dev || !out_host) return IQ_ERR_NULL;
+  if (!aligned16(inputs_dev)) return IQ_ERR_ALIGN;
+  if (shape->batch == 0) return IQ_OK;
+  const size_t d = (size_t)shape->head_dim, B = (size_t)shape->batch;
+  const size_t nq = B * (size_t)shape->n_q_heads * d, nk = B * (size_t)shape->n_kv_heads * d;  // elements of q, of k_new
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  __half* in = static_cast<__half*>(inputs_dev);
+  if (cudaMemcpyAsync(in, inputs_host, (nq + 2 * nk) * sizeof(__half), cudaMemcpyHostToDevice, st) != cudaSuccess) return IQ_ERR_CUDA;
+  const int64_t sh = (int64_t)d, sb = (int64_t)shape->n_kv_heads * sh;  // k_new, v_new: [B][1][H_kv][d]
+  rc = iq_quantize_append(shape, rot_dev, codebook, in + nq, in + nq + nk, sb, sb, sh, append_pos_dev, nullptr, 1, cache,
+                          status_dev, stream);
+  if (rc) return rc;
+  rc = iq_decode_attention(shape, rot_dev, codebook, in, cache, seq_lens_dev, num_splits, part_acc, part_ml, nullptr,
+                           status_dev, stream);
+  if (rc) return rc;
+  rc = iq_combine_splits(shape, rot_dev, num_splits, part_acc, part_ml, nullptr, out_dev, out_is_fp16, nullptr, nullptr, stream);
+  if (rc) return rc;
+  const size_t out_bytes = B * (size_t)shape->n_q_heads * d * (out_is_fp16 ? 2 : 4);
+  if (cudaMemcpyAsync(out_host, out_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return IQ_ERR_CUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
 int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len) {
   if (check_shape(shape) != IQ_OK || max_seq_len <= 0) return 1;
   static int n_sm_cached[64] = {};

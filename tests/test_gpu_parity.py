@@ -261,6 +261,54 @@ def test_codebook_that_is_not_symmetric_takes_the_same_codes(iq, torch, codebook
     assert status.cpu().numpy()[0] == 0
 
 
+@pytest.mark.parametrize("out_dtype", ["float32", "float16"])
+def test_decode_step_from_host_buffers(iq, torch, codebooks, out_dtype):
+    """iq_decode_step_host (copy in, append one row per sequence, decode, combine, copy out, wait) against the oracle:
+    the appended rows and the attention output, over three steps with ragged lengths and an empty sequence."""
+    d, B, H_q, H_kv, T0, steps = 128, 3, 8, 2, 200, 3
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    w = workloads.tiny(61, B, H_q, H_kv, d, T0 + steps)
+    lens0 = np.array([T0, 127, 0], np.int32)
+    t_cap = workloads.cap128(T0 + steps)
+    shape = iq.Shape(B, H_q, H_kv, d, t_cap)
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(w.quats), rot)
+    cache, status = iq.new_cache(shape), torch.zeros(4, dtype=torch.int32, device="cuda")
+    iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(w.k[:, :T0]).cuda(), torch.from_numpy(w.v[:, :T0]).cuda(),
+                          torch.zeros(B, dtype=torch.int32, device="cuda"), torch.from_numpy(lens0).cuda(), T0, cache, status)
+    ref = oracle.new_cache(B, H_kv, d, t_cap)
+    oracle.quantize_append(w.quats, th, w.k[:, :T0], w.v[:, :T0], np.zeros(B, np.int32), lens0, ref)
+    ws = iq.DecodeWorkspace(shape, iq.iq_suggest_splits(shape, t_cap))
+    dt = getattr(torch, out_dtype)
+    n_in = B * (H_q + 2 * H_kv) * d
+    h_in = torch.empty(n_in, dtype=torch.float16).pin_memory()
+    d_in = torch.empty(n_in, dtype=torch.float16, device="cuda")
+    out_dev = torch.empty((B, H_q, d), dtype=dt, device="cuda")
+    out_host = torch.full((B, H_q, d), 99.0, dtype=dt).pin_memory()
+    g = np.random.default_rng(9)
+    rows = lens0.astype(np.int64).copy()
+    for i in range(steps):
+        kn = np.stack([w.k[b, rows[b]] for b in range(B)])[:, None]
+        vn = np.stack([w.v[b, rows[b]] for b in range(B)])[:, None]
+        qn = workloads.to_fp16(g.standard_normal((B, H_q, d)))
+        h_in.copy_(torch.from_numpy(np.concatenate([qn.reshape(-1), kn.reshape(-1), vn.reshape(-1)])))
+        pos = torch.from_numpy(rows.astype(np.int32)).cuda()
+        after = torch.from_numpy((rows + 1).astype(np.int32)).cuda()
+        iq.iq_decode_step_host(shape, rot, cb, h_in, d_in, pos, after, cache, ws, out_dev, out_host)
+        # the call has waited for the output: no synchronize here
+        got = out_host.numpy().astype(np.float64).copy()
+        oracle.quantize_append(w.quats, th, kn, vn, rows.astype(np.int32), None, ref)
+        rows += 1
+        now = rows.astype(np.int32)
+        r = oracle.decode_attention(w.quats, lv, qn, cache_to_numpy(cache), now, H_kv)
+        tol = 2e-3 + 1e-3 * np.abs(r["out"]) + (2.0 ** -11 * np.abs(r["out"]) if out_dtype == "float16" else 0)
+        assert np.all(np.abs(got - r["out"]) <= tol), float(np.max(np.abs(got - r["out"])))
+    w2 = workloads.Workload("h", B, H_q, H_kv, d, t_cap, w.k, w.v, w.q, w.quats, rows.astype(np.int32))
+    compare_caches(w2, th, cache_to_numpy(cache), ref, w2.seq_lens)
+    assert status.cpu().numpy()[0] == 0 and ws.status.cpu().numpy()[0] == 0
+
+
 def test_combine_splits_in_isolation(iq, torch, codebooks):
     d, B, H_q, H_kv, S = 128, 3, 8, 2, 5
     g = np.random.default_rng(7)
