@@ -374,6 +374,50 @@ def test_reconstructed_rows_give_the_same_attention_and_the_codebook_error(codeb
             assert np.isclose(z.max() + math.log(p.sum()), r["lse"][b, h], atol=1e-12)
 
 
+def test_histogram_fit_reproduces_closed_forms():
+    """Lloyd's iteration on a histogram, pinned by three densities with known optima: uniform on [-1, 1) (the uniform
+    quantiser: levels (2k+1)/8 - 1, mse (1/4)^2 / 12), the Gaussian (the textbook 8-level table) and a shifted Gaussian
+    fitted without the symmetry constraint (the same table, shifted)."""
+    lv, th, mse = lloyd_max.fit_histogram(np.ones(4096), 1.0)
+    assert np.allclose(lv, (2 * np.arange(8) + 1) / 8 - 1, atol=1e-9) and np.allclose(th, np.arange(1, 8) / 4 - 1, atol=1e-9)
+    assert abs(mse - 1 / 192) < 1e-12
+    rows = [l.split() for l in open(os.path.join(GOLD, "gauss_lloyd_max_8.txt")) if not l.startswith("#")]
+    lv_ref, mse_ref = np.array([float(x) for x in rows[0]]), float(rows[2][0])     # the textbook table (4 positive levels)
+    centres = (np.arange(4096) + 0.5) * (16.0 / 4096) - 8.0
+    lv, th, mse = lloyd_max.fit_histogram(np.exp(-0.5 * centres ** 2) * 1e9, 8.0)
+    assert np.allclose(lv[4:], lv_ref, atol=6e-4) and np.allclose(lv[:4], -lv_ref[::-1], atol=6e-4)
+    assert abs(mse - mse_ref) < 5e-5
+    lv2, _, _ = lloyd_max.fit_histogram(np.exp(-0.5 * (centres - 0.3) ** 2) * 1e9, 8.0, symmetric=False)
+    assert np.allclose(lv2 - 0.3, lv, atol=1e-4)
+    assert np.max(np.abs(lv2 + lv2[::-1])) > 0.5                                  # and it is not symmetric about zero
+
+
+def test_rotated_histogram_counts_what_the_quantiser_sees(codebooks):
+    """The calibration histogram bins u = sqrt(d) R x^ -- the quantity Algorithm 1 compares with the thresholds: its
+    counts equal a direct binning of the u values the row quantiser reports, zero rows are left out, and for Gaussian
+    rows its first two moments are those of the post-rotation marginal (mean 0, variance 1)."""
+    d, T, H_kv = 128, 300, 2
+    w = workloads.tiny(21, 1, 2, H_kv, d, T)
+    x = w.k[0].copy()
+    x[7] = 0                                                                      # a zero row (both heads)
+    bins, R = 256, 6.0
+    h = lloyd_max.rotated_histogram(w.quats, x, bins, R)
+    assert h.sum() == (T - 1) * H_kv * d
+    _, th = codebooks[d]
+    direct = np.zeros(bins, np.int64)
+    for g in range(H_kv):
+        Rm = oracle.rotation_matrix(d, w.quats[g])
+        for t in (0, 1, 150, 299):
+            _, _, u = oracle.quantize_row(d, Rm, th, x[t, g])
+            direct += np.bincount(np.clip(np.floor((u + R) * bins / (2 * R)).astype(np.int64), 0, bins - 1), minlength=bins)
+    part = lloyd_max.rotated_histogram(w.quats, x[[0, 1, 150, 299]], bins, R)
+    assert np.array_equal(part, direct)
+    centres = (np.arange(bins) + 0.5) * (2 * R / bins) - R
+    mean = float((h * centres).sum() / h.sum())
+    var = float((h * centres ** 2).sum() / h.sum())
+    assert abs(mean) < 0.02 and abs(var - 1.0) < 0.01                             # sum of u^2 over a row is exactly d
+
+
 def test_attention_special_cases(codebooks):
     d = 128
     lv, th = codebooks[d]
