@@ -215,6 +215,29 @@ int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_co
                         int32_t out_rows, int64_t stride_b, int64_t stride_t, int64_t stride_h, void* stream);
 
 /*
+ * Calibration of the codebook on data (Section 3.2, Step 3: "Lloyd-Max for the post-rotation distribution"; the paper
+ * does not say how that distribution is obtained -- here it is the empirical marginal of a calibration set).
+ *
+ * iq_rotated_histogram adds to hist_dev the histogram of u = sqrt(d) R x^ (Algorithm 1, lines 1-4: the quantity the
+ * thresholds are compared with) over all coordinates of the given rows: `bins` uniform bins on [-range, range), values
+ * outside counted in the end bins, zero rows left out.
+ *   x              device binary16 rows, element (b, t, g, i) at b*stride_b + t*stride_t + g*stride_h + i (strides in
+ *                  elements, multiples of 8), t < n_rows_dev[b] (NULL: n_rows_max for every sequence), capped at n_rows_max.
+ *   hist_dev       device uint32 [bins], 16 <= bins <= 4096; the caller zeroes it once and may accumulate several calls.
+ * iq_fit_codebook (host only, no CUDA) runs Lloyd's iteration on such a histogram read as a piecewise-constant density
+ * (level = centroid of its cell, threshold = midpoint of neighbouring levels) and writes the codebook in the form the
+ * kernels take: grid = 0: levels exactly representable in binary16; grid = 1: levels on an 8-bit grid as from
+ * iq_int8_codebook; thresholds = midpoints of the final levels. symmetric != 0 averages the histogram with its mirror
+ * image first (a codebook symmetric about zero takes the faster decision path of the bulk quantize kernels).
+ * IQ_ERR_CODEBOOK if the data has too few distinct values for eight ascending levels.
+ */
+int iq_rotated_histogram(const iq_shape* shape, const float* rot_dev, const void* x, int64_t stride_b,
+                         int64_t stride_t, int64_t stride_h, const int32_t* n_rows_dev, int32_t n_rows_max,
+                         uint32_t* hist_dev, int32_t bins, float range, void* stream);
+int iq_fit_codebook(const uint32_t* hist_host, int32_t bins, float range, int32_t symmetric, int32_t grid,
+                    iq_codebook* out_host);
+
+/*
  * One whole decode step from HOST buffers, in one call: the step's inputs go to the device in one copy, one new row
  * per sequence is appended (Algorithm 1), the fused decode and the merge run (Appendix A), the output comes back and
  * the call returns when it has arrived. It is iq_quantize_append (n_new_max = 1) + iq_decode_attention +

@@ -22,7 +22,9 @@ from .binding import (  # noqa: F401
     iq_row_bytes,
     iq_strerror,
     iq_decode_step_host,
+    iq_fit_codebook,
     iq_reconstruct_rows,
+    iq_rotated_histogram,
     iq_suggest_splits,
     iq_version,
     lib_path,

@@ -66,6 +66,9 @@ def _load():
                                         _vp, _vp, _i32, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, _vp]
     lib.iq_decode_step_host.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp, _vp, _vp, _vp,
                                         ctypes.POINTER(_IqCache), _i32, _vp, _vp, _vp, _vp, _i32, _vp, _vp]
+    lib.iq_rotated_histogram.argtypes = [ctypes.POINTER(_IqShape), _vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, _vp,
+                                         _i32, _vp, _i32, ctypes.c_float, _vp]
+    lib.iq_fit_codebook.argtypes = [_vp, _i32, ctypes.c_float, _i32, _i32, ctypes.POINTER(_IqCodebook)]
     lib.iq_suggest_splits.restype = _i32
     lib.iq_suggest_splits.argtypes = [ctypes.POINTER(_IqShape), _i32]
     return lib
@@ -241,6 +244,27 @@ def iq_decode_step_host(shape: Shape, rot_dev, codebook: Codebook, inputs_host, 
                                     _ptr(append_pos_dev), _ptr(seq_lens_dev), ctypes.byref(cc), ws.num_splits, _ptr(ws.part_acc),
                                     _ptr(ws.part_ml), _ptr(out_dev), _ptr(out_host), 1 if out_dev.dtype == torch.float16 else 0,
                                     _ptr(ws.status), _stream(stream)), "iq_decode_step_host")
+
+
+def iq_rotated_histogram(shape: Shape, rot_dev, x, n_rows_dev, hist_dev, rng_half: float, stream=None) -> None:
+    """Adds the histogram of the rotated, normalised coordinates of the rows x (fp16 device tensor [B][T][H_kv][d]) to
+    hist_dev (uint32/int32 device tensor [bins]); n_rows_dev: int32 [B] or None (all T rows)."""
+    assert x.dtype == torch.float16 and x.stride(3) == 1 and hist_dev.dtype in (torch.int32, torch.uint32)
+    cs = shape.c()
+    _check(_lib.iq_rotated_histogram(ctypes.byref(cs), _ptr(rot_dev), _ptr(x), x.stride(0), x.stride(1), x.stride(2),
+                                     _ptr(n_rows_dev), x.shape[1], _ptr(hist_dev), hist_dev.numel(), float(rng_half),
+                                     _stream(stream)), "iq_rotated_histogram")
+
+
+def iq_fit_codebook(hist_host, rng_half: float, symmetric: bool = True, grid: str = "int8") -> Codebook:
+    """Lloyd-Max codebook fitted to a histogram from iq_rotated_histogram (a contiguous int32/uint32 numpy array or CPU
+    tensor). grid: "int8" (integer tensor-core decode path) or "fp16" (exact binary16 levels)."""
+    h = hist_host.numpy() if isinstance(hist_host, torch.Tensor) else hist_host
+    assert h.dtype.itemsize == 4 and h.dtype.kind in "iu" and h.flags["C_CONTIGUOUS"]
+    cb = _IqCodebook()
+    _check(_lib.iq_fit_codebook(h.ctypes.data, h.size, float(rng_half), 1 if symmetric else 0, {"fp16": 0, "int8": 1}[grid],
+                                ctypes.byref(cb)), "iq_fit_codebook")
+    return Codebook(tuple(cb.levels), tuple(cb.thresholds))
 
 
 def iq_suggest_splits(shape: Shape, max_seq_len: int) -> int:

@@ -2,6 +2,7 @@
 // contract of every entry point. Nothing here allocates device memory or keeps state between calls.
 #include <cmath>
 #include <cstring>
+#include <vector>
 
 #include "iq_common.cuh"
 #include "iq_kernels.h"
@@ -103,6 +104,75 @@ void lloyd_max_sphere(int d, double (&lv)[8]) {
     }
     if (delta < 1e-13) break;
   }
+}
+
+// Lloyd's iteration on a histogram with uniform bins on [-range, range), read as a piecewise-constant density: a bin
+// cut by a threshold contributes to both cells in proportion. mass0 / mom0: mass and first moment below bin edge i.
+void lloyd_max_histogram(const std::vector<double>& c, double range, bool symmetric, double (&lv)[8]) {
+  const int bins = (int)c.size();
+  const double w = 2.0 * range / bins;
+  std::vector<double> mass0(bins + 1, 0.0), mom0(bins + 1, 0.0);
+  for (int i = 0; i < bins; i++) {
+    const double lo = i * w - range, hi = lo + w;
+    mass0[i + 1] = mass0[i] + c[i];
+    mom0[i + 1] = mom0[i] + c[i] * 0.5 * (lo + hi);
+  }
+  auto below = [&](double t, double& mass, double& mom) {
+    t = std::fmin(std::fmax(t, -range), range);
+    int i = (int)((t + range) / w);
+    if (i > bins - 1) i = bins - 1;
+    const double lo = i * w - range, dens = c[i] / w;
+    mass = mass0[i] + dens * (t - lo);
+    mom = mom0[i] + dens * 0.5 * (t * t - lo * lo);
+  };
+  const double total = mass0[bins];
+  {  // start: the quantiles (k + 1/2) / 8
+    int i = 0;
+    for (int k = 0; k < 8; k++) {
+      const double target = total * (k + 0.5) / 8.0;
+      while (i < bins - 1 && mass0[i + 1] < target) i++;
+      const double frac = c[i] > 0.0 ? (target - mass0[i]) / c[i] : 0.5;
+      lv[k] = (i + frac) * w - range;
+    }
+  }
+  for (int iter = 0; iter < 5000; iter++) {
+    double cut[9], m[9], f[9];
+    cut[0] = -range;
+    cut[8] = range;
+    for (int i = 1; i < 8; i++) cut[i] = 0.5 * (lv[i - 1] + lv[i]);
+    for (int i = 0; i < 9; i++) below(cut[i], m[i], f[i]);
+    double nl[8];
+    for (int i = 0; i < 8; i++) {
+      const double mass = m[i + 1] - m[i];
+      nl[i] = mass > 0.0 ? (f[i + 1] - f[i]) / mass : lv[i];
+    }
+    if (symmetric)
+      for (int i = 0; i < 4; i++) {
+        const double a = 0.5 * (nl[7 - i] - nl[i]);
+        nl[7 - i] = a;
+        nl[i] = -a;
+      }
+    double delta = 0.0;
+    for (int i = 0; i < 8; i++) {
+      delta = std::fmax(delta, std::fabs(nl[i] - lv[i]));
+      lv[i] = nl[i];
+    }
+    if (delta < 1e-13) break;
+  }
+}
+
+// Levels (fp64, ascending) -> the codebook handed to the kernels: levels exactly representable in binary16 (grid = 0)
+// or on an 8-bit grid (grid = 1: level = n * delta, |n| <= 127, delta = max |level| / 127), thresholds = midpoints.
+void finish_codebook(const double (&lv)[8], int grid, iq_codebook* out) {
+  if (grid == 1) {
+    double amax = 0.0;
+    for (int i = 0; i < 8; i++) amax = std::fmax(amax, std::fabs(lv[i]));
+    const float delta = (float)(amax / 127.0);
+    for (int i = 0; i < 8; i++) out->levels[i] = delta > 0.f ? (float)std::nearbyint(lv[i] / (double)delta) * delta : 0.f;
+  } else {
+    for (int i = 0; i < 8; i++) out->levels[i] = __half2float(__float2half_rn((float)lv[i]));
+  }
+  for (int i = 0; i < 7; i++) out->thresholds[i] = (float)(0.5 * ((double)out->levels[i] + (double)out->levels[i + 1]));
 }
 
 }  // namespace
@@ -363,6 +433,51 @@ int iq_decode_step_host(const iq_shape* shape, const float* rot_dev, const iq_co
   const size_t out_bytes = B * (size_t)shape->n_q_heads * d * (out_is_fp16 ? 2 : 4);
   if (cudaMemcpyAsync(out_host, out_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return IQ_ERR_CUDA;
   return cudaStreamSynchronize(st) == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
+int iq_rotated_histogram(const iq_shape* shape, const float* rot_dev, const void* x, int64_t stride_b, int64_t stride_t,
+                         int64_t stride_h, const int32_t* n_rows_dev, int32_t n_rows_max, uint32_t* hist_dev, int32_t bins,
+                         float range, void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (!rot_dev || !hist_dev) return IQ_ERR_NULL;
+  if (bins < 16 || bins > iq::HIST_MAX_BINS || !(range > 0.f) || n_rows_max < 0) return IQ_ERR_SHAPE;
+  if (n_rows_max == 0 || shape->batch == 0) return IQ_OK;
+  if (!x) return IQ_ERR_NULL;
+  if (!aligned16(x) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
+  if (stride_b < 0 || stride_t < 0 || stride_h < 0) return IQ_ERR_SHAPE;
+  if ((stride_b & 7) || (stride_t & 7) || (stride_h & 7)) return IQ_ERR_ALIGN;
+  iq::HistogramParams p = {};
+  p.x = static_cast<const __half*>(x);
+  p.stride_b = stride_b;
+  p.stride_t = stride_t;
+  p.stride_h = stride_h;
+  p.n_rows = n_rows_dev;
+  p.n_rows_max = n_rows_max;
+  p.rot = rot_dev;
+  p.hist = hist_dev;
+  p.bins = bins;
+  p.range = range;
+  p.n_kv_heads = shape->n_kv_heads;
+  const cudaError_t e = iq::launch_rotated_histogram(p, shape->head_dim, shape->batch, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
+int iq_fit_codebook(const uint32_t* hist_host, int32_t bins, float range, int32_t symmetric, int32_t grid,
+                    iq_codebook* out_host) {
+  if (!hist_host || !out_host) return IQ_ERR_NULL;
+  if (bins < 16 || bins > iq::HIST_MAX_BINS || !(range > 0.f) || (grid != 0 && grid != 1)) return IQ_ERR_SHAPE;
+  std::vector<double> c((size_t)bins);
+  double total = 0.0;
+  for (int i = 0; i < bins; i++) total += (double)hist_host[i];
+  if (!(total > 0.0)) return IQ_ERR_SHAPE;
+  for (int i = 0; i < bins; i++) c[i] = symmetric ? 0.5 * ((double)hist_host[i] + (double)hist_host[bins - 1 - i]) : (double)hist_host[i];
+  double lv[8];
+  lloyd_max_histogram(c, (double)range, symmetric != 0, lv);
+  finish_codebook(lv, grid, out_host);
+  for (int i = 0; i < 7; i++)
+    if (!(out_host->levels[i] < out_host->levels[i + 1])) return IQ_ERR_CODEBOOK;  // too few distinct values in the data
+  return IQ_OK;
 }
 
 int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len) {

@@ -29,6 +29,23 @@ struct QuantizeParams {
 };
 cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int batch, cudaStream_t stream);
 
+// ---- calibration: histogram of the rotated, normalised coordinates of a set of rows
+constexpr int HIST_MAX_BINS = 4096;
+constexpr int HIST_ROWS_PER_WARP = 128;
+struct HistogramParams {
+  const __half* x;
+  long long stride_b, stride_t, stride_h;
+  const int32_t* n_rows;
+  int n_rows_max;
+  const float* rot;
+  float thresholds[7];  // unused (zeros): the row quantizer it shares with the append kernels loads them
+  uint32_t* hist;
+  int bins;
+  float range;
+  int n_kv_heads;
+};
+cudaError_t launch_rotated_histogram(const HistogramParams& p, int head_dim, int batch, cudaStream_t stream);
+
 // ---- fused decode
 constexpr int DEC_BLOCK_TOKENS = 128;  // cached rows per block of the decode kernel = rows of one transposed V block
 constexpr int DEC_HEADS = 8;          // query heads per CTA (the N extent of the m16n8k16 tile)

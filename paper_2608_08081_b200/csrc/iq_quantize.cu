@@ -117,12 +117,10 @@ struct RowQuantizer {
     return packed;
   }
 
-  // Algorithm 1, steps 1-3 for the row this lane belongs to (r0, r1 = this lane's 16 fp16 values, zeros for the
-  // lanes of a row that is not written; those lanes still take part in the shuffles). Returns the fp32 scale.
-  template <bool SYM>
-  __device__ __forceinline__ float run(const uint4& r0, const uint4& r1, bool active, int lane, int (&code)[E],
-                                       uint32_t* status) const {
-    float x[E];
+  // Algorithm 1, steps 1-2 for the row this lane belongs to (r0, r1 = this lane's 16 fp16 values, zeros for the lanes
+  // of a row that is not used; those lanes still take part in the shuffles): returns the fp32 scale s (and its fp64
+  // square sum) and leaves M_b (H x) -- u * s, the rotated coordinates before the division by the norm -- in x.
+  __device__ __forceinline__ float rotate(const uint4& r0, const uint4& r1, int lane, float (&x)[E], double& ss_out) const {
     unpack16(r0, r1, x);
     // Step 1: s = ||x||_2. Squares of fp16 values are exact in fp32 (22 bits); they are summed in fp64 so that the
     // stored fp32 scale is the correctly rounded norm.
@@ -139,8 +137,7 @@ struct RowQuantizer {
       if (ss > mu * mu) s = up;
       else if (s > 0.f && ss < md * md) s = dn;
     }
-    const float inv_s = (s > 0.f) ? __frcp_rn(s) : 0.f;
-
+    ss_out = ss;
     // Step 2: u = sqrt(d) * R x^ = M_b (H_unnormalised x) / s  (the two sqrt(d) factors cancel)
     wht<float>(x, lane);
 #pragma unroll
@@ -152,6 +149,18 @@ struct RowQuantizer {
         x[4 * j + r] = m.x * x0 + m.y * x1 + m.z * x2 + m.w * x3;
       }
     }
+
+    return s;
+  }
+
+  // Algorithm 1, steps 1-3: the codes of this lane's 16 coordinates; returns the fp32 scale.
+  template <bool SYM>
+  __device__ __forceinline__ float run(const uint4& r0, const uint4& r1, bool active, int lane, int (&code)[E],
+                                       uint32_t* status) const {
+    float x[E];
+    double ss;
+    const float s = rotate(r0, r1, lane, x, ss);
+    const float inv_s = (s > 0.f) ? __frcp_rn(s) : 0.f;
 
     // Step 3: codes, with a guard band around the thresholds
     bool any_near = false;
@@ -574,6 +583,68 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
       if (lane == 0) p.v_scales[slab + (size_t)t] = s;
     }
   }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Calibration: histogram of the rotated, normalised coordinates u = sqrt(d) R x^ of a set of rows -- the empirical
+// marginal that Step 3's Lloyd-Max codebook is fitted to. Same row mapping as the K kernel; the CTA counts into a
+// histogram in shared memory and adds its non-empty bins to the caller's at the end. Zero rows are left out.
+// ---------------------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(QA_WARPS * 32, 4) rotated_histogram_kernel(const __grid_constant__ HistogramParams p) {
+  using RQ = RowQuantizer<D>;
+  constexpr int LPR = RQ::LPR, RPW = RQ::RPW;
+  __shared__ uint32_t hist_s[HIST_MAX_BINS];
+  __shared__ __align__(16) float m_s[RQ::M_FLOATS];
+  grid_dependency_wait();
+  allow_dependent_launch();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = blockIdx.z, h = blockIdx.y;
+  int n_rows = p.n_rows ? p.n_rows[b] : p.n_rows_max;
+  n_rows = min(n_rows, p.n_rows_max);
+  const int cta_begin = blockIdx.x * QA_WARPS * HIST_ROWS_PER_WARP;
+  if (cta_begin >= n_rows) return;
+  for (int i = tid; i < p.bins; i += QA_WARPS * 32) hist_s[i] = 0u;
+  RQ::fill_matrices(p.rot + (size_t)h * (D / 4) * 8, m_s, tid, QA_WARPS * 32);
+  __syncthreads();
+  RQ rq;
+  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane, m_s);
+  const int li = lane % LPR, sub = lane / LPR;
+  const __half* src_base = p.x + (size_t)b * p.stride_b + (size_t)h * p.stride_h + li * 16;
+  const int row_begin = cta_begin + warp * HIST_ROWS_PER_WARP, row_end = min(n_rows, row_begin + HIST_ROWS_PER_WARP);
+  const float to_bin = (float)p.bins / (2.f * p.range);
+  for (int i0 = row_begin; i0 < row_end; i0 += RPW) {
+    const int i = i0 + sub;
+    const bool active = i < row_end;
+    uint4 r0 = make_uint4(0u, 0u, 0u, 0u), r1 = r0;
+    if (active) {
+      const uint4* src = reinterpret_cast<const uint4*>(src_base + (size_t)i * p.stride_t);
+      r0 = __ldg(src);
+      r1 = __ldg(src + 1);
+    }
+    float x[16];
+    double ss;
+    const float s = rq.rotate(r0, r1, lane, x, ss);
+    if (active && s > 0.f) {
+      const float inv_s = __frcp_rn(s);
+#pragma unroll
+      for (int e = 0; e < 16; e++) {
+        const int bin = (int)floorf((x[e] * inv_s + p.range) * to_bin);
+        atomicAdd(&hist_s[min(max(bin, 0), p.bins - 1)], 1u);
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < p.bins; i += QA_WARPS * 32)
+    if (hist_s[i]) atomicAdd(&p.hist[i], hist_s[i]);
+}
+
+cudaError_t launch_rotated_histogram(const HistogramParams& p, int head_dim, int batch, cudaStream_t stream) {
+  if (p.n_rows_max <= 0 || batch <= 0) return cudaSuccess;
+  const int rows_per_cta = QA_WARPS * HIST_ROWS_PER_WARP;
+  dim3 grid((p.n_rows_max + rows_per_cta - 1) / rows_per_cta, p.n_kv_heads, batch);
+  return head_dim == 128 ? launch_after_predecessor(rotated_histogram_kernel<128>, grid, dim3(QA_WARPS * 32), 0, stream, p)
+                         : launch_after_predecessor(rotated_histogram_kernel<256>, grid, dim3(QA_WARPS * 32), 0, stream, p);
 }
 
 cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int batch, cudaStream_t stream) {

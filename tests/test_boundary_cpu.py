@@ -43,6 +43,31 @@ def test_default_codebook_matches_oracle_tool(iq, codebooks):
         iq.iq_default_codebook(96)
 
 
+def test_codebook_fitted_to_a_histogram_matches_the_oracle(iq):
+    """iq_fit_codebook is host code: Lloyd's iteration on a histogram against the oracle's independent implementation,
+    for a Gaussian, a heavy-tailed and a skewed histogram, with and without the symmetry constraint, on both grids."""
+    from oracle import lloyd_max
+    bins, R = 2048, 8.0
+    c = (np.arange(bins) + 0.5) * (2 * R / bins) - R
+    hists = {"gauss": np.exp(-0.5 * c * c), "student_t3": (1 + c * c / 3) ** -2.0, "skewed": np.exp(-0.5 * (c - 0.4) ** 2) + 0.3 * np.exp(-2 * (c + 1.5) ** 2)}
+    for name, dens in hists.items():
+        h = np.rint(dens * 1e8).astype(np.uint32)
+        for symmetric in (True, False):
+            lv, _, _ = lloyd_max.fit_histogram(h, R, symmetric=symmetric)
+            cb16 = iq.iq_fit_codebook(h, R, symmetric=symmetric, grid="fp16")
+            assert np.array_equal(np.array(cb16.levels, np.float32), lv.astype(np.float16).astype(np.float32)), (name, symmetric)
+            th16 = 0.5 * (np.array(cb16.levels, np.float64)[1:] + np.array(cb16.levels, np.float64)[:-1])
+            assert np.array_equal(np.array(cb16.thresholds, np.float32), th16.astype(np.float32))
+            cb8 = iq.iq_fit_codebook(h, R, symmetric=symmetric, grid="int8")
+            delta = np.float32(np.max(np.abs(lv)) / 127.0)
+            n = np.rint(lv / np.float64(delta))
+            assert np.array_equal(np.array(cb8.levels, np.float32), (n.astype(np.float32) * delta).astype(np.float32)), (name, symmetric)
+            if symmetric:
+                assert np.array_equal(np.array(cb8.levels)[::-1], -np.array(cb8.levels)) and cb8.thresholds[3] == 0.0
+    with pytest.raises(iq.IQError):
+        iq.iq_fit_codebook(np.zeros(bins, np.uint32), R)                 # no data
+
+
 class _P:
     """Fake tensor: just a device-pointer-like integer (never dereferenced: validation fails first)."""
     def __init__(self, p): self._p = p

@@ -309,6 +309,67 @@ def test_decode_step_from_host_buffers(iq, torch, codebooks, out_dtype):
     assert status.cpu().numpy()[0] == 0 and ws.status.cpu().numpy()[0] == 0
 
 
+@pytest.mark.parametrize("d", [128, 256])
+def test_calibration_histogram_and_fitted_codebook(iq, torch, d):
+    """iq_rotated_histogram against the oracle's dense-rotation histogram on heavy-tailed rows (ragged row counts, a
+    zero row, values beyond the range): the counts may differ only where fp32 puts a value on the other side of a bin
+    edge (a vanishing fraction, neighbouring bins), the codebooks fitted to the two histograms agree, and a
+    quantize + decode round trip with the fitted codebook is parity-exact and beats the default codebook's distortion."""
+    from oracle import lloyd_max
+    B, H_q, H_kv, T = 2, 4, 2, 700
+    g = np.random.Generator(np.random.Philox(4100 + d))
+    x = workloads.to_fp16(0.5 * g.standard_t(3.0, (B, T, H_kv, d)))
+    x[0, 5] = 0
+    n_rows = np.array([T, 333], np.int32)
+    quats = workloads.quaternion_pairs(g, H_kv, d)
+    bins, R = 2048, 6.0
+    shape = iq.Shape(B, H_q, H_kv, d, workloads.cap128(T))
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(quats), rot)
+    hist = torch.zeros(bins, dtype=torch.int32, device="cuda")
+    xd = torch.from_numpy(x).cuda()
+    iq.iq_rotated_histogram(shape, rot, xd, torch.from_numpy(n_rows).cuda(), hist, R)
+    torch.cuda.synchronize()
+    got = hist.cpu().numpy().astype(np.int64)
+    ref = lloyd_max.rotated_histogram(quats, x[0], bins, R) + lloyd_max.rotated_histogram(quats, x[1, :333], bins, R)
+    assert got.sum() == ref.sum() == (T - 1 + 333) * H_kv * d
+    moved = np.abs(np.cumsum(got - ref))                     # a value in the neighbouring bin shows as +1 / -1 next to each other
+    assert moved.max() <= 3 and np.abs(got - ref).sum() <= 2e-4 * ref.sum()
+    hist2 = torch.zeros(64, dtype=torch.int32, device="cuda")   # a narrow range: what falls outside is counted in the end bins
+    iq.iq_rotated_histogram(shape, rot, xd, torch.from_numpy(n_rows).cuda(), hist2, 2.0)
+    got2 = hist2.cpu().numpy().astype(np.int64)
+    ref2 = lloyd_max.rotated_histogram(quats, x[0], 64, 2.0) + lloyd_max.rotated_histogram(quats, x[1, :333], 64, 2.0)
+    assert got2.sum() == ref2.sum() and np.abs(np.cumsum(got2 - ref2)).max() <= 3
+    assert got2[0] > 50 * got2[1] / 10 and got2[-1] > 50 * got2[-2] / 10
+    for grid in ("int8", "fp16"):
+        cb_g = iq.iq_fit_codebook(got.astype(np.uint32), R, grid=grid)
+        cb_r = iq.iq_fit_codebook(ref.astype(np.uint32), R, grid=grid)
+        assert np.allclose(cb_g.levels, cb_r.levels, atol=2e-3)
+    # round trip with the fitted codebook (levels on the 8-bit grid): parity against the oracle, and a lower distortion
+    cb = iq.iq_fit_codebook(got.astype(np.uint32), R, grid="int8")
+    lv, th = np.array(cb.levels, np.float32), np.array(cb.thresholds, np.float32)
+    w = workloads.Workload("cal", B, H_q, H_kv, d, shape.t_cap, x, x[:, ::-1].copy(), workloads.to_fp16(g.standard_normal((B, H_q, d))),
+                           quats, n_rows)
+    shape2, rot2, cache, status = gpu_quantize(iq, torch, w, cb, n_new=n_rows)
+    cache_np = cache_to_numpy(cache)
+    refc = oracle.new_cache(B, H_kv, d, shape.t_cap)
+    oracle.quantize_append(quats, th, w.k, w.v, np.zeros(B, np.int32), n_rows, refc)
+    compare_caches(w, th, cache_np, refc, n_rows)
+    S = iq.iq_suggest_splits(shape2, T)
+    res = gpu_decode(iq, torch, shape2, rot2, cb, w.q, cache, n_rows, S)
+    check_decode(w, lv, w.q, res, cache_np, n_rows)
+    dflt = iq.iq_int8_codebook(d)
+
+    def distortion(levels, thresholds):
+        c = oracle.new_cache(B, H_kv, d, shape.t_cap)
+        oracle.quantize_append(quats, np.array(thresholds, np.float32), w.k, w.v, np.zeros(B, np.int32), n_rows, c)
+        K, _ = oracle.reconstruct_rows(quats, np.array(levels, np.float32), c, n_rows, H_kv)
+        xs = x[1, :333].astype(np.float64)
+        return float(np.mean(np.sum((xs - K[1, :333]) ** 2, -1) / np.sum(xs * xs, -1)))
+
+    assert distortion(cb.levels, cb.thresholds) < distortion(dflt.levels, dflt.thresholds)
+
+
 def test_combine_splits_in_isolation(iq, torch, codebooks):
     d, B, H_q, H_kv, S = 128, 3, 8, 2, 5
     g = np.random.default_rng(7)
