@@ -160,6 +160,7 @@ def aggregate_gbs(bytes_per_rank: float, ms: float, world: int) -> float:
     return world * bytes_per_rank / (ms * 1e-3) / 1e9
 
 
+PAGE_ROWS = 0       # > 0: the cache is a pool of pages of this many rows behind a block table in scrambled order
 CODEBOOK = "int8"   # "int8": Lloyd-Max levels on an 8-bit grid (integer tensor-core decode path); "fp16": exact fp16 levels
 
 
@@ -177,14 +178,23 @@ def build_state(name: str, device, rank: int):
     cb = iq.iq_int8_codebook(d) if CODEBOOK == "int8" else iq.iq_default_codebook(d)
     rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device=device)
     iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(gen["quats"]), rot)
-    cache = iq.new_cache(shape, device)
+    if PAGE_ROWS:
+        assert t_cap % PAGE_ROWS == 0, "--page-rows must divide the capacity (ctx + 2048)"
+        n_tab = t_cap // PAGE_ROWS
+        perm = np.random.Generator(np.random.Philox(77 + rank)).permutation(B * n_tab).astype(np.int32)
+        cache = iq.new_paged_cache(shape, B * n_tab, PAGE_ROWS, torch.from_numpy(perm.reshape(B, n_tab)).to(device), device)
+    else:
+        cache = iq.new_cache(shape, device)
     status = torch.zeros(4, dtype=torch.int32, device=device)
     lens_np = gen["lens"].astype(np.int32)
     qa_ms, qa_rows = 0.0, 0
     for b0, k, v in gen["chunks"]():
         nb = k.shape[0]
         sub = iq.Shape(nb, H_q, H_kv, d, t_cap)
-        view = iq.Cache(cache.k_codes[b0:b0 + nb], cache.k_scales[b0:b0 + nb], cache.v_codes[b0:b0 + nb], cache.v_scales[b0:b0 + nb])
+        if PAGE_ROWS:   # the pool is shared; the chunk's sequences are rows b0 .. b0 + nb of the block table
+            view = iq.Cache(cache.k_codes, cache.k_scales, cache.v_codes, cache.v_scales, cache.block_table[b0:b0 + nb], PAGE_ROWS)
+        else:
+            view = iq.Cache(cache.k_codes[b0:b0 + nb], cache.k_scales[b0:b0 + nb], cache.v_codes[b0:b0 + nb], cache.v_scales[b0:b0 + nb])
         pos = torch.zeros(nb, dtype=torch.int32, device=device)
         nn = torch.from_numpy(lens_np[b0:b0 + nb]).to(device)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -243,7 +253,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     q_all, k_all, v_all = step_inputs(st, K + W, device, 99 + rank)
     stream = torch.cuda.current_stream()
     groups = [slice(b, b + 1) for b in range(B)] if per_seq else [slice(0, B)]
-    gcache = [iq.Cache(cache.k_codes[g], cache.k_scales[g], cache.v_codes[g], cache.v_scales[g]) for g in groups]
+    if PAGE_ROWS:
+        gcache = [iq.Cache(cache.k_codes, cache.k_scales, cache.v_codes, cache.v_scales, cache.block_table[g], PAGE_ROWS) for g in groups]
+    else:
+        gcache = [iq.Cache(cache.k_codes[g], cache.k_scales[g], cache.v_codes[g], cache.v_scales[g]) for g in groups]
     n_groups = len(groups)
 
     def launches(i, q, k, v, ev=None, out=None):
@@ -385,7 +398,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                    "t_cap": st["t_cap"], "lengths": "ctx" if per_seq else "ragged, floor(ctx*U[0.5,1.0])",
                    "launch_groups": n_groups, "ms_per_launch_group": round(ms_step / n_groups, 5), "cached_rows_per_kv_head": rows,
                    "num_splits": S, "bytes_per_row_per_kv_head": bytes_per_row(d), "l2": "inputs_larger_than_l2",
-                   "step": "quantize-append 1 row/seq + fused decode + combine", "codebook": CODEBOOK, "parallelism": f"replicas x{world}",
+                   "step": "quantize-append 1 row/seq + fused decode + combine", "codebook": CODEBOOK, "cache": (f"paged, {PAGE_ROWS} rows per page, scrambled" if PAGE_ROWS else "contiguous"), "parallelism": f"replicas x{world}",
                    "timed_region": ("one replay of a CUDA graph holding the K steps" if graph is not None
                                     else "K steps launched from the host")},
         "decode_tokens_per_s": round(world * B / (ms_step * 1e-3), 1),
@@ -550,11 +563,13 @@ def main():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-materialised", action="store_true", help="skip the reconstruct-then-compute comparison")
+    ap.add_argument("--page-rows", type=int, default=0, help="paged cache: rows per page (multiple of 128 dividing ctx + 2048), pages in scrambled order")
     ap.add_argument("--no-graph", action="store_true", help="time the host-launched loop instead of a CUDA-graph replay of the K steps")
     ap.add_argument("--codebook", default="int8", choices=["int8", "fp16"])
     args = ap.parse_args()
-    global CODEBOOK
+    global CODEBOOK, PAGE_ROWS
     CODEBOOK = args.codebook
+    PAGE_ROWS = args.page_rows
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

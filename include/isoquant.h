@@ -74,7 +74,8 @@ enum {
 
 enum {
   IQ_STATUS_ROW_OUT_OF_RANGE = 1u, /* quantize-append: append_pos + i >= t_cap, row skipped */
-  IQ_STATUS_WAIT_TIMEOUT = 2u      /* decode: a bounded wait on an asynchronous copy ran out; results invalid */
+  IQ_STATUS_WAIT_TIMEOUT = 2u,     /* decode: a bounded wait on an asynchronous copy ran out; results invalid */
+  IQ_STATUS_BAD_PAGE = 4u          /* paged cache: a block-table entry outside [0, num_pages) was met and read as page 0 */
 };
 
 typedef struct iq_shape {
@@ -97,6 +98,16 @@ typedef struct iq_cache {
   float* k_scales;
   uint8_t* v_codes;
   float* v_scales;
+  /* Paged cache (optional; the paper's cache is contiguous per sequence). block_table_dev == NULL: the arrays are
+   * [batch][n_kv_heads][t_cap] rows as described above. Otherwise they are a pool of num_pages pages,
+   * [num_pages][n_kv_heads][page_rows] rows (V: page_rows / 128 token-transposed blocks per page and KV head), and
+   * block_table_dev is a device int32 [batch][t_cap / page_rows]: entry (b, j) is the page that holds rows
+   * [j * page_rows, (j + 1) * page_rows) of sequence b. page_rows is a multiple of 128 and divides t_cap, which is
+   * then the logical capacity of a sequence. Entries that a call can reach (rows below the lengths it is given)
+   * must be valid; an entry outside [0, num_pages) sets IQ_STATUS_BAD_PAGE and is read as page 0. */
+  const int32_t* block_table_dev;
+  int32_t page_rows;
+  int32_t num_pages;
 } iq_cache;
 
 int iq_version(void);

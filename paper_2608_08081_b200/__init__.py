@@ -29,6 +29,7 @@ from .binding import (  # noqa: F401
     iq_version,
     lib_path,
     new_cache,
+    new_paged_cache,
     DecodeWorkspace,
     decode_step,
 )

@@ -4,6 +4,7 @@ from __future__ import annotations
 import ctypes
 import os
 from dataclasses import dataclass
+from typing import Optional
 
 import torch
 
@@ -24,7 +25,8 @@ class _IqCodebook(ctypes.Structure):
 
 
 class _IqCache(ctypes.Structure):
-    _fields_ = [("k_codes", _vp), ("k_scales", _vp), ("v_codes", _vp), ("v_scales", _vp)]
+    _fields_ = [("k_codes", _vp), ("k_scales", _vp), ("v_codes", _vp), ("v_scales", _vp),
+                ("block_table_dev", _vp), ("page_rows", _i32), ("num_pages", _i32)]
 
 
 class IQError(RuntimeError):
@@ -116,13 +118,22 @@ class Codebook:
 
 @dataclass
 class Cache:
-    k_codes: torch.Tensor   # uint8 [B][H_kv][t_cap][3d/8]
-    k_scales: torch.Tensor  # fp32  [B][H_kv][t_cap]
+    """Contiguous: k_codes uint8 [B][H_kv][t_cap][3d/8], k_scales fp32 [B][H_kv][t_cap] (V alike). Paged: the same
+    arrays with a pool of pages in place of the batch, [num_pages][H_kv][page_rows]..., and block_table int32
+    [B][t_cap / page_rows] on the device."""
+    k_codes: torch.Tensor
+    k_scales: torch.Tensor
     v_codes: torch.Tensor
     v_scales: torch.Tensor
+    block_table: Optional[torch.Tensor] = None
+    page_rows: int = 0
 
     def c(self) -> _IqCache:
-        return _IqCache(self.k_codes.data_ptr(), self.k_scales.data_ptr(), self.v_codes.data_ptr(), self.v_scales.data_ptr())
+        if self.block_table is None:
+            return _IqCache(self.k_codes.data_ptr(), self.k_scales.data_ptr(), self.v_codes.data_ptr(), self.v_scales.data_ptr(), None, 0, 0)
+        assert self.block_table.dtype == torch.int32 and self.block_table.is_contiguous()
+        return _IqCache(self.k_codes.data_ptr(), self.k_scales.data_ptr(), self.v_codes.data_ptr(), self.v_scales.data_ptr(),
+                        self.block_table.data_ptr(), self.page_rows, self.k_scales.shape[0])
 
 
 def _ptr(t):
@@ -278,6 +289,18 @@ def new_cache(shape: Shape, device="cuda") -> Cache:
     n = (shape.batch, shape.n_kv_heads, shape.t_cap)
     return Cache(torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=torch.float32, device=device),
                  torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=torch.float32, device=device))
+
+
+def new_paged_cache(shape: Shape, num_pages: int, page_rows: int, block_table: torch.Tensor, device="cuda") -> Cache:
+    """A pool of num_pages pages of page_rows rows (a multiple of 128 that divides shape.t_cap) and the block table
+    (int32 device tensor [batch][t_cap / page_rows]) that maps the sequences' rows onto it."""
+    assert page_rows % 128 == 0 and shape.t_cap % page_rows == 0
+    assert tuple(block_table.shape) == (shape.batch, shape.t_cap // page_rows)
+    P = iq_row_bytes(shape.head_dim)
+    n = (num_pages, shape.n_kv_heads, page_rows)
+    return Cache(torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=torch.float32, device=device),
+                 torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=torch.float32, device=device),
+                 block_table, page_rows)
 
 
 class DecodeWorkspace:

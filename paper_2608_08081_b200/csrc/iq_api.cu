@@ -55,10 +55,23 @@ bool int8_grid(const iq_codebook* cb, int (&n)[8], float& delta) {
   return true;
 }
 
-int check_cache(const iq_cache* c) {
+int check_cache(const iq_cache* c, const iq_shape* shape) {
   if (!c || !c->k_codes || !c->k_scales || !c->v_codes || !c->v_scales) return IQ_ERR_NULL;
   if (!aligned16(c->k_codes) || !aligned16(c->k_scales) || !aligned16(c->v_codes) || !aligned16(c->v_scales)) return IQ_ERR_ALIGN;
+  if (c->block_table_dev) {  // paged: whole 128-row blocks per page, whole pages per sequence
+    if (c->page_rows <= 0 || (c->page_rows % 128) != 0 || c->num_pages <= 0 || (shape->t_cap % c->page_rows) != 0) return IQ_ERR_SHAPE;
+  }
   return IQ_OK;
+}
+
+iq::PageMap page_map(const iq_cache* c, const iq_shape* shape) {
+  iq::PageMap m;
+  m.table = c->block_table_dev;
+  m.page_rows = c->block_table_dev ? c->page_rows : 0;
+  m.num_pages = c->block_table_dev ? c->num_pages : 0;
+  m.n_kv_heads = shape->n_kv_heads;
+  m.t_cap = shape->t_cap;
+  return m;
 }
 
 // Lloyd's iteration for the marginal of one coordinate of a uniform point on S^{d-1}, unit-variance units:
@@ -262,7 +275,7 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
   if (rc) return rc;
   if (!rot_dev || !append_pos_dev) return IQ_ERR_NULL;
   if ((rc = check_codebook(codebook, false))) return rc;
-  if ((rc = check_cache(cache))) return rc;
+  if ((rc = check_cache(cache, shape))) return rc;
   if (n_new_max < 0) return IQ_ERR_SHAPE;
   if (n_new_max == 0 || shape->batch == 0) return IQ_OK;
   if (!k_new || !v_new) return IQ_ERR_NULL;
@@ -288,6 +301,7 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
   p.status = status_dev;
   p.n_kv_heads = shape->n_kv_heads;
   p.t_cap = shape->t_cap;
+  p.pm = page_map(cache, shape);
   const cudaError_t e = iq::launch_quantize_append(p, shape->head_dim, shape->batch, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }
@@ -303,7 +317,7 @@ int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_co
   float delta = 0.f;
   const bool grid8 = int8_grid(codebook, n8, delta);  // integer tensor-core path; otherwise the levels must be exact fp16 values
   if (!grid8 && (rc = check_codebook(codebook, true))) return rc;
-  if ((rc = check_cache(cache))) return rc;
+  if ((rc = check_cache(cache, shape))) return rc;
   if (num_splits < 1 || num_splits > 65535) return IQ_ERR_SHAPE;
   if (!aligned16(q) || !aligned16(part_acc) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
   if (shape->batch == 0) return IQ_OK;
@@ -326,6 +340,7 @@ int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_co
   p.group = shape->n_q_heads / shape->n_kv_heads;
   p.head_groups = (p.group + iq::DEC_HEADS - 1) / iq::DEC_HEADS;
   p.t_cap = shape->t_cap;
+  p.pm = page_map(cache, shape);
   p.splits = num_splits;
   p.sm_scale = shape->sm_scale > 0.f ? shape->sm_scale : 1.0f / std::sqrt((float)shape->head_dim);
   p.lut_lo[0] = p.lut_lo[1] = p.lut_hi[0] = p.lut_hi[1] = 0u;
@@ -381,7 +396,7 @@ int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_co
   if (!rot_dev || !seq_lens_dev || !k_out || !v_out) return IQ_ERR_NULL;
   if (out_rows < 0) return IQ_ERR_SHAPE;
   if ((rc = check_codebook(codebook, false))) return rc;
-  if ((rc = check_cache(cache))) return rc;
+  if ((rc = check_cache(cache, shape))) return rc;
   if (!aligned16(k_out) || !aligned16(v_out) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
   if (stride_b < 0 || stride_t < 0 || stride_h < 0) return IQ_ERR_SHAPE;
   if ((stride_b & 7) || (stride_t & 7) || (stride_h & 7)) return IQ_ERR_ALIGN;
@@ -401,6 +416,8 @@ int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_co
   p.stride_h = stride_h;
   p.n_kv_heads = shape->n_kv_heads;
   p.t_cap = shape->t_cap;
+  p.pm = page_map(cache, shape);
+  p.status = nullptr;
   p.out_rows = out_rows;
   std::memcpy(p.levels, codebook->levels, sizeof(p.levels));
   const cudaError_t e = iq::launch_reconstruct_rows(p, shape->head_dim, shape->batch, static_cast<cudaStream_t>(stream));

@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include "../../include/isoquant.h"
+#include "iq_kernels.h"
 
 namespace iq {
 
@@ -147,6 +148,21 @@ inline cudaError_t launch_after_predecessor(void (*kernel)(Params), dim3 grid, d
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
+// Where cache row t of (sequence b, KV head g) sits in the cache arrays, in rows. Contiguous cache: the arrays are
+// [batch][n_kv_heads][t_cap]. Paged cache: a pool [num_pages][n_kv_heads][page_rows] and a table [batch][t_cap /
+// page_rows] of page numbers; page_rows is a multiple of 128, so a 128-row block never straddles two pages and the
+// row index of a block's first row, times the row size, is also where its token-transposed V records start.
+__device__ __forceinline__ size_t cache_row(const PageMap& m, int b, int g, long long t, uint32_t* status) {
+  if (m.table == nullptr) return ((size_t)b * m.n_kv_heads + g) * (size_t)m.t_cap + (size_t)t;
+  const int j = (int)(t / m.page_rows);
+  int page = m.table[(size_t)b * (m.t_cap / m.page_rows) + j];
+  if ((unsigned)page >= (unsigned)m.num_pages) {  // never turned into an address: flagged and read as page 0
+    if (status) atomicOr(&status[0], IQ_STATUS_BAD_PAGE);
+    page = 0;
+  }
+  return ((size_t)page * m.n_kv_heads + g) * (size_t)m.page_rows + (size_t)(t - (long long)j * m.page_rows);
 }
 
 #ifndef IQ_MBAR_SUSPEND_NS

@@ -349,19 +349,30 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
       // ================================================================ control warp of group grp: fetches blocks, issues MMAs.
       // All 32 lanes run the loop and the waits; an elected lane issues.
       const int blk1 = seg_s->blk1, len = seg_s->len;
-      const size_t slab = ((size_t)seg_s->b * p.n_kv_heads + (seg_s->y / p.head_groups)) * (size_t)p.t_cap;
+      const int seg_b = seg_s->b, seg_kvh = seg_s->y / p.head_groups;
       const uint32_t bq_addr = smem_u32(bq), bp_addr = smem_u32(bp);
       // operand descriptors of the first k-step, built before the waits: a k-step further on adds its byte offset / 16
       const uint64_t bq_desc0 = smem_desc_mn(bq_addr, 128, (D / 8) * 128), bp_desc0 = smem_desc_mn(bp_addr, 128, (TB / 8) * 128);
       bool ended = false;   // the segment's counter ran out and the end marker has been staged
       int it_issue = it;    // slots staged so far (the pipeline is empty between segments)
-      auto stage_next = [&]() {  // draw the next block of the segment into slot it_issue, or the end marker
+      // The next block is drawn (shared counter; with a paged cache also its block-table entry, a load from global
+      // memory) while the compute warps are busy with the softmax of the current one, and staged after the value MMAs.
+      int drawn_j = -1;        // block drawn ahead of its staging, -1: none
+      size_t drawn_row0 = 0;   // its first row in the cache arrays
+      auto draw = [&]() {
+        int j = 0;
+        if (lane == 0) j = atomicAdd(next_s, 1);
+        drawn_j = __shfl_sync(FULL, j, 0);
+        if (drawn_j < blk1) drawn_row0 = cache_row(p.pm, seg_b, seg_kvh, drawn_j * TB, p.status);
+      };
+      auto stage_next = [&]() {  // the next block of the segment into slot it_issue, or the end marker
         const int st = it_issue % NST;
         if (it_issue >= NST && !failed)  // the slot's previous occupant has been consumed
           failed = !mbar_wait_bounded(&empty_bar[st], (uint32_t)(it_issue / NST - 1) & 1u, DEC_WAIT_LIMIT);
-        int j = 0;
-        if (lane == 0) j = atomicAdd(next_s, 1);
-        j = __shfl_sync(FULL, j, 0);
+        if (drawn_j < 0) draw();
+        const int j = drawn_j;
+        const size_t row0 = drawn_row0;
+        drawn_j = -1;
         if (j < blk1) {
           const int r0 = j * TB;
           const int n = min(TB, len - r0);
@@ -371,10 +382,10 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
             uint8_t* sp = stages + st * L::STAGE_BYTES;
             fence_proxy_async();
             mbar_expect_tx(&full_bar[st], (uint32_t)(n * L::ROWB + L::VT_BYTES + 2 * n4 * 4));  // also publishes desc[st]
-            bulk_g2s(sp, p.k_codes + (slab + r0) * L::ROWB, (uint32_t)(n * L::ROWB), &full_bar[st]);
-            bulk_g2s(sp + L::K_BYTES, p.v_codes + (slab + r0) * L::ROWB, (uint32_t)L::VT_BYTES, &full_bar[st]);  // whole 128-row V block
-            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES, p.k_scales + slab + r0, (uint32_t)(n4 * 4), &full_bar[st]);
-            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES, p.v_scales + slab + r0, (uint32_t)(n4 * 4), &full_bar[st]);
+            bulk_g2s(sp, p.k_codes + row0 * L::ROWB, (uint32_t)(n * L::ROWB), &full_bar[st]);
+            bulk_g2s(sp + L::K_BYTES, p.v_codes + row0 * L::ROWB, (uint32_t)L::VT_BYTES, &full_bar[st]);  // whole 128-row V block
+            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES, p.k_scales + row0, (uint32_t)(n4 * 4), &full_bar[st]);
+            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES, p.v_scales + row0, (uint32_t)(n4 * 4), &full_bar[st]);
           }
         } else {
           ended = true;
@@ -407,6 +418,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           tc_commit(s_bar);
         }
         __syncwarp();
+        if (!ended) draw();
         // values: O = A_V * B_P^T once the V tile is in TMEM and the probabilities are in shared memory
         if (!failed) failed = !mbar_wait_bounded(p_ready, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
         tc_fence_after();

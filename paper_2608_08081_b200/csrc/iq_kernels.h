@@ -6,6 +6,13 @@
 
 namespace iq {
 
+// Addressing of the cache arrays: contiguous per sequence (table == nullptr) or a pool of pages with a block table
+// (see cache_row in iq_common.cuh).
+struct PageMap {
+  const int32_t* table;
+  int page_rows, num_pages, n_kv_heads, t_cap;
+};
+
 // ---- quantize-append
 constexpr int QA_WARPS = 4;
 constexpr int QA_FEW_ROWS = 4;        // calls with at most this many new rows per sequence take the one-warp-per-row latency path
@@ -26,6 +33,7 @@ struct QuantizeParams {
   float* v_scales;
   uint32_t* status;
   int n_kv_heads, t_cap;
+  PageMap pm;
 };
 cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int batch, cudaStream_t stream);
 
@@ -63,6 +71,7 @@ struct DecodeParams {
   int32_t* part_argmax;
   uint32_t* status;
   int batch, n_q_heads, n_kv_heads, group, head_groups, t_cap, splits;
+  PageMap pm;
   float sm_scale;
   uint32_t lut_lo[2], lut_hi[2];  // low / high bytes of the 8 fp16 levels, 4 per register
   // integer path (levels on an 8-bit grid): level_j = lut8 byte j (int8) * delta
@@ -98,6 +107,8 @@ struct ReconstructParams {
   __half* v_out;
   long long stride_b, stride_t, stride_h;  // in elements
   int n_kv_heads, t_cap, out_rows;
+  PageMap pm;
+  uint32_t* status;
   float levels[8];
 };
 cudaError_t launch_reconstruct_rows(const ReconstructParams& p, int head_dim, int batch, cudaStream_t stream);

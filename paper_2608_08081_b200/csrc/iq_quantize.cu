@@ -243,7 +243,6 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 5) quantize_append_k_kernel(con
   rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane, m_s);
   const int li = lane % LPR, sub = lane / LPR;  // lane within the row, row within the warp
   const __half* src_base = p.k_new + (size_t)b * p.stride_b + (size_t)h * p.stride_h + li * 16;
-  const size_t slab = ((size_t)b * p.n_kv_heads + h) * (size_t)p.t_cap;
 
   auto fetch = [&](int i0, uint4& r0, uint4& r1, bool& exists, bool& active) {
     const int i = i0 + sub;
@@ -274,10 +273,11 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 5) quantize_append_k_kernel(con
     uint32_t w0, w1;
     pack_pair(code, lane, w0, w1);
     if (active) {
-      uint32_t* unit_words = reinterpret_cast<uint32_t*>(p.k_codes + (slab + (size_t)t) * (size_t)(3 * D / 8)) + 3 * (li >> 1);
+      const size_t row = cache_row(p.pm, b, h, t, p.status);
+      uint32_t* unit_words = reinterpret_cast<uint32_t*>(p.k_codes + row * (size_t)(3 * D / 8)) + 3 * (li >> 1);
       if (li & 1) unit_words[2] = w0;
       else { unit_words[0] = w0; unit_words[1] = w1; }
-      if (li == 0) p.k_scales[slab + (size_t)t] = s;
+      if (li == 0) p.k_scales[row] = s;
     }
   }
 }
@@ -311,7 +311,6 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
   const long long t_lo = max(blkg * 128, pos0);                  // first cache row of this block that is appended
   const long long t_hi = min(blkg * 128 + 128, pos0 + n_new);    // one past the last
   if (t_lo >= t_hi) return;
-  const size_t slab = ((size_t)b * p.n_kv_heads + h) * (size_t)p.t_cap;
   const bool in_cache = blkg >= 0 && blkg * 128 + 128 <= p.t_cap;  // t_cap is a multiple of 128
   if (!in_cache) {
     if (tid == 0 && p.status) {
@@ -320,6 +319,7 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
     }
     return;
   }
+  const size_t block_row0 = cache_row(p.pm, b, h, blkg * 128, p.status);  // the block's first row in the cache arrays
 
   RQ::fill_matrices(p.rot + (size_t)h * (D / 4) * 8, m_s, tid, 128);
   __syncthreads();
@@ -355,7 +355,7 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
       for (int q = 0; q < 4; q++)
         pk[q] = (uint32_t)code[4 * q] | ((uint32_t)code[4 * q + 1] << 8) | ((uint32_t)code[4 * q + 2] << 16) | ((uint32_t)code[4 * q + 3] << 24);
       *reinterpret_cast<uint4*>(&codes_s[t & 127][li * 16]) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-      if (li == 0) p.v_scales[slab + (size_t)t] = s;
+      if (li == 0) p.v_scales[block_row0 + (size_t)(t & 127)] = s;
     }
   }
   __syncthreads();
@@ -365,7 +365,7 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
 #pragma unroll
   for (int j = 0; j < D / 128; j++) {
     const int c = tid + 128 * j;  // coordinate
-    uint32_t* rec = reinterpret_cast<uint32_t*>(p.v_codes + ((slab / 128 + (size_t)blkg) * D + c) * 48);
+    uint32_t* rec = reinterpret_cast<uint32_t*>(p.v_codes + ((block_row0 / 128) * D + c) * 48);
     if (c_lo == 0 && c_hi == 128) {  // the whole block is new: the record is written with three 16-byte stores
       uint32_t w[12];
 #pragma unroll
@@ -519,7 +519,6 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
   for (int k = 0; k < E / 2; k++) raw[k] = reinterpret_cast<const __half2*>(src_base)[k];
   WarpRowQuantizer<D> rq;
   rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane);
-  const size_t slab = ((size_t)b * p.n_kv_heads + h) * (size_t)p.t_cap;
   for (int i = 0; i < n_new; i++) {
     if (i > 0) {
 #pragma unroll
@@ -533,6 +532,7 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
       }
       continue;
     }
+    const size_t row = cache_row(p.pm, b, h, t, p.status);  // the row's place in the cache arrays
     int code[E];
     const float s = rq.run(raw, lane, code, p.status);
     if (!is_v) {
@@ -559,18 +559,18 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
         w[2] |= __shfl_xor_sync(FULL, w[2], o);
       }
       const int k = lane % LPU;
-      uint32_t* row_words = reinterpret_cast<uint32_t*>(p.k_codes + (slab + (size_t)t) * (size_t)(3 * D / 8));
+      uint32_t* row_words = reinterpret_cast<uint32_t*>(p.k_codes + row * (size_t)(3 * D / 8));
       if (k < 3) row_words[3 * (lane / LPU) + k] = (k == 0) ? w[0] : (k == 1 ? w[1] : w[2]);
-      if (lane == 0) p.k_scales[slab + (size_t)t] = s;
+      if (lane == 0) p.k_scales[row] = s;
     } else {
       // transposed records: row t is entry r = t % 32 of unit u = (t % 128) / 32 of block t / 128, for every coordinate
-      const size_t blk = (size_t)t / 128;
+      const size_t blk = row / 128;  // (a page holds whole 128-row blocks: row / 128 is the block's index in the V array)
       const int u = (int)(t % 128) / 32, r = (int)(t % 32);
 #pragma unroll
       for (int e = 0; e < E; e++) {
         const int c = lane * E + e;
         const uint32_t cd = (uint32_t)code[e];
-        uint32_t* dst = reinterpret_cast<uint32_t*>(p.v_codes + ((slab / 128 + blk) * D + c) * 48) + 3 * u;
+        uint32_t* dst = reinterpret_cast<uint32_t*>(p.v_codes + (blk * D + c) * 48) + 3 * u;
         if (r < 24) {
           const int sh = 4 * (r & 7);
           dst[r >> 3] = (dst[r >> 3] & ~(7u << sh)) | (cd << sh);
@@ -580,7 +580,7 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
           for (int k = 0; k < 3; k++) dst[k] = (dst[k] & ~(1u << sh)) | (((cd >> k) & 1u) << sh);
         }
       }
-      if (lane == 0) p.v_scales[slab + (size_t)t] = s;
+      if (lane == 0) p.v_scales[row] = s;
     }
   }
 }

@@ -36,16 +36,16 @@ __global__ void __launch_bounds__(RC_WARPS * 32) reconstruct_kernel(const Recons
   const int r_begin = blockIdx.x * TB;
   if (r_begin >= len) return;
   const int n = min(TB, len - r_begin);
-  const size_t slab = ((size_t)b * p.n_kv_heads + g) * (size_t)p.t_cap;
+  const size_t row0 = cache_row(p.pm, b, g, r_begin, p.status);  // the block's first row in the cache arrays
 
   {  // stage the block: n packed K rows, the whole V record set of the block (128 * ROWB = D * 48 bytes), the scales
-    const uint4* ksrc = reinterpret_cast<const uint4*>(p.k_codes + (slab + r_begin) * ROWB);
-    const uint4* vsrc = reinterpret_cast<const uint4*>(p.v_codes + (slab + r_begin) * ROWB);
+    const uint4* ksrc = reinterpret_cast<const uint4*>(p.k_codes + row0 * ROWB);
+    const uint4* vsrc = reinterpret_cast<const uint4*>(p.v_codes + row0 * ROWB);
     for (int i = tid; i < n * ROWB / 16; i += RC_WARPS * 32) reinterpret_cast<uint4*>(k_s)[i] = ksrc[i];
     for (int i = tid; i < D * 48 / 16; i += RC_WARPS * 32) reinterpret_cast<uint4*>(v_s)[i] = vsrc[i];
     if (tid < n) {
-      ks_s[tid] = p.k_scales[slab + r_begin + tid];
-      vs_s[tid] = p.v_scales[slab + r_begin + tid];
+      ks_s[tid] = p.k_scales[row0 + tid];
+      vs_s[tid] = p.v_scales[row0 + tid];
     }
     if (tid < 8) lv_s[tid] = p.levels[tid];
   }

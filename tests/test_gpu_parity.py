@@ -370,6 +370,73 @@ def test_calibration_histogram_and_fitted_codebook(iq, torch, d):
     assert distortion(cb.levels, cb.thresholds) < distortion(dflt.levels, dflt.thresholds)
 
 
+def _gather_pages(cache, table, page_rows):
+    """The paged pool read back as the contiguous cache [B][H_kv][t_cap] the oracle works on."""
+    tb = np.asarray(table)
+    out = {}
+    for name in ("k_codes", "k_scales", "v_codes", "v_scales"):
+        pool = getattr(cache, name).cpu().numpy()                                     # [pages][H_kv][page_rows](...)
+        out[name] = np.ascontiguousarray(np.concatenate([pool[tb[:, j]] for j in range(tb.shape[1])], axis=2))
+    return out
+
+
+@pytest.mark.parametrize("d,page_rows", [(128, 128), (128, 256), (256, 128)])
+def test_paged_cache_gives_the_contiguous_results(iq, torch, codebooks, d, page_rows):
+    """A pool of pages in scrambled order behind a block table: bulk append with ragged lengths, two single-row steps
+    (one of them lands on the first row of a fresh page), decode, and reconstruction must give exactly what the
+    contiguous cache gives -- the gathered pool is compared with the oracle's cache and the oracle's decode."""
+    B, H_q, H_kv, T = 3, 8, 2, 768
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    lens = np.array([700, 255, 0], np.int32)
+    w = workloads.tiny(1200 + d + page_rows, B, H_q, H_kv, d, T, lens)
+    n_tab = T // page_rows
+    num_pages = B * n_tab + 3
+    g = np.random.default_rng(page_rows + d)
+    table = g.permutation(num_pages)[:B * n_tab].reshape(B, n_tab).astype(np.int32)   # every (sequence, slot) its own page
+    shape = iq.Shape(B, H_q, H_kv, d, T)
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(w.quats), rot)
+    cache = iq.new_paged_cache(shape, num_pages, page_rows, torch.from_numpy(table).cuda())
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    k, v = torch.from_numpy(w.k).cuda(), torch.from_numpy(w.v).cuda()
+    iq.iq_quantize_append(shape, rot, cb, k, v, torch.zeros(B, dtype=torch.int32, device="cuda"), torch.from_numpy(lens).cuda(), T, cache, status)
+    ref = oracle.new_cache(B, H_kv, d, T)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), lens, ref)
+    now = lens.copy()
+    for step in range(2):                                                            # sequence 1: rows 255 and 256
+        kn = np.stack([w.k[b, now[b]] for b in range(B)])[:, None]
+        vn = np.stack([w.v[b, now[b]] for b in range(B)])[:, None]
+        iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(),
+                              torch.from_numpy(now).cuda(), None, 1, cache, status)
+        oracle.quantize_append(w.quats, th, kn, vn, now, None, ref)
+        now = now + 1
+    torch.cuda.synchronize()
+    assert status.cpu().numpy()[0] == 0
+    gathered = _gather_pages(cache, table, page_rows)
+    w2 = workloads.Workload("paged", B, H_q, H_kv, d, T, w.k, w.v, w.q, w.quats, now)
+    compare_caches(w2, th, gathered, ref, now)
+    used = np.zeros(num_pages, bool); used[table.ravel()] = True                     # pages outside the table stay untouched
+    assert not cache.k_codes.cpu().numpy()[~used].any() and not cache.v_codes.cpu().numpy()[~used].any()
+    S = iq.iq_suggest_splits(shape, T)
+    res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, now, S)
+    check_decode(w2, lv, w.q, res, gathered, now)
+    k_out = torch.zeros((B, T, H_kv, d), dtype=torch.float16, device="cuda")
+    v_out = torch.zeros_like(k_out)
+    iq.iq_reconstruct_rows(shape, rot, cb, cache, torch.from_numpy(now).cuda(), k_out, v_out)
+    K, V = oracle.reconstruct_rows(w.quats, lv, gathered, now, H_kv)
+    for got, r in ((k_out.cpu().numpy().astype(np.float64), K), (v_out.cpu().numpy().astype(np.float64), V)):
+        bound = 2.0 ** -11 * 1.001 * np.abs(r) + 1e-5 * np.abs(r).max(axis=-1, keepdims=True) + 1e-30
+        assert np.all(np.abs(got - r) <= bound)
+    # a block-table entry outside the pool is never turned into an address: flagged, read as page 0
+    bad = table.copy(); bad[0, 1] = num_pages + 5
+    cache_bad = iq.Cache(cache.k_codes, cache.k_scales, cache.v_codes, cache.v_scales, torch.from_numpy(bad).cuda(), page_rows)
+    ws = iq.DecodeWorkspace(shape, S)
+    iq.decode_step(shape, rot, cb, torch.from_numpy(w.q).cuda(), cache_bad, torch.from_numpy(now).cuda(), ws)
+    torch.cuda.synchronize()
+    assert int(ws.status[0].item()) & 4
+
+
 def test_combine_splits_in_isolation(iq, torch, codebooks):
     d, B, H_q, H_kv, S = 128, 3, 8, 2, 5
     g = np.random.default_rng(7)
