@@ -437,6 +437,58 @@ def test_paged_cache_gives_the_contiguous_results(iq, torch, codebooks, d, page_
     assert int(ws.status[0].item()) & 4
 
 
+def test_context_sharded_decode_on_one_gpu(iq, torch, codebooks):
+    """The context-sharded path with the two ranks' work done one after the other on one GPU: rows [0, 256) and
+    [256, T) of every sequence in two caches, the fused decode over each, the partials laid out as the all-gather
+    lays them out (rank-major along the split axis, argmax rows made global), one merge: the unsharded result. Then
+    sharded_decode_step itself under a one-rank process group: the same as the plain step."""
+    import torch.distributed as dist
+    from paper_2608_08081_b200 import sharded
+    d, B, H_q, H_kv, T, cut = 128, 2, 8, 2, 700, 256
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    lens = np.array([700, 130], np.int32)                                           # the second sequence ends inside the first slice
+    w = workloads.tiny(77, B, H_q, H_kv, d, T, lens)
+    t_cap = workloads.cap128(T)
+    shape = iq.Shape(B, H_q, H_kv, d, t_cap)
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(w.quats), rot)
+    q = torch.from_numpy(w.q).cuda()
+    S = 3
+    parts = []
+    for lo, hi in ((0, cut), (cut, T)):
+        my = np.clip(lens - lo, 0, hi - lo).astype(np.int32)
+        cache, status = iq.new_cache(shape), torch.zeros(4, dtype=torch.int32, device="cuda")
+        iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(w.k[:, lo:hi].copy()).cuda(), torch.from_numpy(w.v[:, lo:hi].copy()).cuda(),
+                              torch.zeros(B, dtype=torch.int32, device="cuda"), torch.from_numpy(my).cuda(), hi - lo, cache, status)
+        ws = iq.DecodeWorkspace(shape, S, want_argmax=True)
+        iq.iq_decode_attention(shape, rot, cb, q, cache, torch.from_numpy(my).cuda(), S, ws.part_acc, ws.part_ml, ws.part_argmax, ws.status)
+        am = torch.where(ws.part_argmax >= 0, ws.part_argmax + lo, ws.part_argmax)
+        parts.append((ws.part_acc.clone(), ws.part_ml.clone(), am, cache, my, ws))
+    acc = torch.cat([p[0] for p in parts], dim=2)
+    ml = torch.cat([p[1] for p in parts], dim=2)
+    am = torch.cat([p[2] for p in parts], dim=2)
+    out = torch.empty((B, H_q, d), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, H_q), dtype=torch.float32, device="cuda")
+    amx = torch.empty((B, H_q), dtype=torch.int32, device="cuda")
+    iq.iq_combine_splits(shape, rot, 2 * S, acc, ml, am, out, lse, amx)
+    torch.cuda.synchronize()
+    full = oracle.new_cache(B, H_kv, d, t_cap)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), lens, full)
+    res = dict(out=out.cpu().numpy().astype(np.float64), lse=lse.cpu().numpy().astype(np.float64), argmax=amx.cpu().numpy())
+    check_decode(w, lv, w.q, res, full, lens)
+    # the library's function under a process group of one rank
+    if not dist.is_initialized():
+        dist.init_process_group("gloo", init_method="tcp://127.0.0.1:29557", rank=0, world_size=1)
+    _, _, _, cache0, my0, ws0 = parts[0]
+    o1, l1, a1 = sharded.sharded_decode_step(iq, shape, rot, cb, q, cache0, torch.from_numpy(my0).cuda(), ws0,
+                                             row_offset=torch.zeros(B, dtype=torch.int32, device="cuda"))
+    iq.decode_step(shape, rot, cb, q, cache0, torch.from_numpy(my0).cuda(), ws0)
+    torch.cuda.synchronize()
+    assert torch.allclose(o1, ws0.out, atol=1e-5) and torch.equal(a1, ws0.argmax)
+    dist.destroy_process_group()
+
+
 def test_combine_splits_in_isolation(iq, torch, codebooks):
     d, B, H_q, H_kv, S = 128, 3, 8, 2, 5
     g = np.random.default_rng(7)

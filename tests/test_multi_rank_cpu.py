@@ -1,6 +1,7 @@
-"""The N > 1 path of bench.py on CPU: two gloo ranks rendezvous on 127.0.0.1, agree on the slowest rank's time,
-and only rank 0 reports. (The data path shards by sequence with no collective, so this is all the distributed
-logic there is; the kernels themselves are covered by the single-GPU parity tests.)"""
+"""The N > 1 paths on CPU, two gloo ranks on 127.0.0.1: bench.py's replicas (the data path shards by sequence with no
+collective: the ranks agree on the slowest rank's time and only rank 0 reports) and the one exchange step the method
+has when the context itself is sharded (an all-gather of the split partials, merged on every rank). The kernels
+themselves are covered by the single-GPU parity tests."""
 import json
 import os
 import subprocess
@@ -56,3 +57,60 @@ def test_reference_arm_under_two_ranks_reports_once():
     line = json.loads(outs[0].strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+SHARD_SCRIPT = r"""
+import json, os, sys
+import numpy as np, torch
+sys.path.insert(0, os.environ["IQ_REPO"]); sys.path.insert(0, os.path.join(os.environ["IQ_REPO"], "tests"))
+import torch.distributed as dist
+import importlib.util
+spec = importlib.util.spec_from_file_location("sharded", os.path.join(os.environ["IQ_REPO"], "paper_2608_08081_b200", "sharded.py"))
+sharded = importlib.util.module_from_spec(spec); spec.loader.exec_module(sharded)      # (the package itself needs the CUDA library)
+import oracle, workloads
+from oracle import lloyd_max
+rank = int(os.environ["RANK"]); world = int(os.environ["WORLD_SIZE"])
+dist.init_process_group("gloo", rank=rank, world_size=world)
+d, B, H_q, H_kv, T = 128, 2, 4, 2, 300
+lens = np.array([300, 41], np.int32)                       # the second sequence lives on rank 0 alone
+w = workloads.tiny(33, B, H_q, H_kv, d, T, lens)
+lv, th = lloyd_max.fp16_codebook(d)
+cut = 128                                                  # rank 0: rows [0, 128), rank 1: rows [128, T)
+lo = 0 if rank == 0 else cut
+my_lens = np.clip(lens - lo, 0, cut if rank == 0 else T - cut).astype(np.int32)
+cache = oracle.new_cache(B, H_kv, d, workloads.cap128(T))
+oracle.quantize_append(w.quats, th, w.k[:, lo:], w.v[:, lo:], np.zeros(B, np.int32), my_lens, cache)
+r = oracle.decode_attention(w.quats, lv, w.q, cache, my_lens, H_kv, want_rot=True)
+# this rank's slice as one split partial per head: m = max score, l = sum exp(z - m), acc = l * (normalised rotated
+# output); an empty slice: (-inf, 0, 0)
+S = 1
+m = np.full((B, H_q), -np.inf); l = np.zeros((B, H_q))
+for b in range(B):
+    for h in range(H_q):
+        if my_lens[b] > 0:
+            z = oracle.scores(w.quats, lv, w.q, cache, b, h, int(my_lens[b]), H_kv)
+            m[b, h] = z.max(); l[b, h] = np.exp(z - z.max()).sum()
+acc = torch.from_numpy((r["o_rot"] * l[:, :, None]).astype(np.float32)).reshape(B, H_q, S, d)
+ml = torch.from_numpy(np.stack([m, l], -1).astype(np.float32)).reshape(B, H_q, S, 2)
+am = torch.from_numpy(r["argmax"].astype(np.int32)).reshape(B, H_q, S)
+off = torch.full((B,), lo, dtype=torch.int32)
+g_acc, g_ml, g_am = sharded.gather_partials(acc, ml, am, off)
+dist.barrier(); dist.destroy_process_group()
+merged = oracle.combine_splits(w.quats, g_acc.numpy(), g_ml.numpy(), g_am.numpy(), H_kv)
+full = oracle.new_cache(B, H_kv, d, workloads.cap128(T))
+oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), lens, full)
+ref = oracle.decode_attention(w.quats, lv, w.q, full, lens, H_kv)
+print(json.dumps({"rank": rank, "splits": int(g_acc.shape[2]), "err": float(np.abs(merged["out"] - ref["out"]).max()),
+                  "lse_err": float(np.abs(merged["lse"] - ref["lse"]).max()), "argmax_equal": bool(np.array_equal(merged["argmax"], ref["argmax"]))}), flush=True)
+"""
+
+
+def test_context_sharded_partials_merge_to_the_unsharded_result():
+    """Two ranks hold rows [0, 128) and [128, 300) of every sequence (one sequence ends inside the first slice, so the
+    second rank contributes an empty partial for it): the gathered partials, merged, must be the unsharded attention
+    output -- on both ranks, with global argmax rows."""
+    outs = _spawn(2, ["-c", SHARD_SCRIPT], extra_env={"MASTER_PORT": "29551"})
+    res = [json.loads(o.strip().splitlines()[-1]) for o in outs]
+    assert {r["rank"] for r in res} == {0, 1}
+    for r in res:
+        assert r["splits"] == 2 and r["err"] < 2e-6 and r["lse_err"] < 2e-6 and r["argmax_equal"]   # partials travel as fp32
