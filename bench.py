@@ -407,7 +407,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                      "traffic": decode_traffic_bytes(sum(timed_launch_bytes) / len(dec_ms), B // n_groups, H_q, S, d),
                      "traffic_source": "ncu one-pass DRAM byte counters on the full B = 32 launch, scaled by rows processed (reads) and partial results (writes)",
                      "kernel": "decode_kernel", "peak_source": peak_src,
-                     "avg_launch_ms": round(dec_avg_ms, 4), "launches_timed": len(dec_ms),
+                     "avg_launch_ms": round(dec_avg_ms, 4), "median_launch_ms": round(float(np.median(dec_ms)), 4),
+                     "launch_ms_cv": round(float(np.std(dec_ms) / np.mean(dec_ms)), 4), "launches_timed": len(dec_ms),
                      "algorithmic_bytes_per_launch": int(sum(timed_launch_bytes) / len(dec_ms))},
         "e2e": {"value": round(aggregate_gbs(e2e_bytes, e2e_ms, world), 1), "unit": "GB/s",
                 "h2d_bytes_per_step": int(B * (H_q + 2 * H_kv) * d * 2), "d2h_bytes_per_step": int(B * H_q * d * 2),
@@ -424,7 +425,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         out["graph_error"] = graph_error
     if not args.no_materialised and world == 1 and not per_seq:
         out["reconstruct_then_compute"] = materialised_baseline(st, lens_tab[W + K], q_all[W + K - 1], ws, S, peak)
-    if not args.no_cpu_baseline and world == 1:
+    if not args.no_cpu_baseline and world == 1 and not PAGE_ROWS:
         out["cpu_baseline"] = cpu_baseline(st, lens_tab[n_e2e_warm + n_e2e], q_all[W + K - 1])
     return out
 
@@ -501,9 +502,21 @@ def cpu_baseline(st, lens, q_last, target_s: float = 12.0):
         oracle.decode_attention(st["quats"], lv, q, cache, ln, st["H_kv"])
         total += time.perf_counter() - t0
         reps += 1
-    return {"value": round(reps * nbytes / total / 1e9, 4), "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{reps} x decode of all {nb} sequences (all {st['H_q']} query heads, {nbytes / 1e6:.0f} MB of packed cache), "
-                      f"{total:.1f} s"}
+    res = {"value": round(reps * nbytes / total / 1e9, 4), "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": f"{reps} x decode of all {nb} sequences (all {st['H_q']} query heads, {nbytes / 1e6:.0f} MB of packed cache), "
+                     f"{total:.1f} s"}
+    # the same oracle on one thread, on the first sequence alone
+    threads = oracle.num_threads()
+    oracle.set_num_threads(1)
+    try:
+        one = {k: v[:1] for k, v in cache.items()}
+        t0 = time.perf_counter()
+        oracle.decode_attention(st["quats"], lv, q[:1], one, ln[:1], st["H_kv"])
+        t1 = time.perf_counter() - t0
+        res["value_1_thread"] = round(int(ln[0]) * st["H_kv"] * bytes_per_row(st["d"]) / t1 / 1e9, 4)
+    finally:
+        oracle.set_num_threads(threads)
+    return res
 
 
 def run_reference(args, rank: int, world: int):
