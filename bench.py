@@ -33,6 +33,8 @@ WORKLOADS = {
     "config5_B32_ctx4096": (32, 4096, 64, 8, 128),
     "config5_B8_ctx4096": (8, 4096, 64, 8, 128),
     "config5_B1_ctx4096": (1, 4096, 64, 8, 128),
+    # one sequence of a million rows: the same shape far beyond the paper's 32 K (0.8 GB of packed cache, 4 GB as fp16)
+    "config5_B1_ctx1048576": (1, 1048576, 64, 8, 128),
     # the wide-head shape of config 3 (d = 256, 16 query / 8 KV heads) as a ragged batch that exceeds L2
     "d256_B32_ctx16384": (32, 16384, 16, 8, 256),
     # single-sequence shapes (configs 3 and 4) as a stack of 48 per-layer caches of full length, every layer with its own
