@@ -717,3 +717,28 @@ def test_full_size_bench_configuration_sampled(iq, torch, codebooks):
         assert np.array_equal(oracle.v_row_codes(d, vc[b, h], t), cv)
         checked += 1
     assert checked == 400
+
+
+def test_bench_line_keeps_its_contract():
+    """bench.py on the smallest serving point: one JSON line with the keys the measurement contract names, a roofline
+    object whose fraction is achieved / peak, an end-to-end leg that moved bytes both ways, and launches counted."""
+    import json
+    import os
+    import subprocess
+    import sys
+    repo = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "bench.py", "--workload", "config5_B1_ctx4096", "--steps", "4", "--warmup", "3", "--no-cpu-baseline",
+                        "--no-materialised"], cwd=repo, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling", "vs_baseline", "dtype",
+                "data", "config", "roofline", "e2e", "gpu_launches", "clocks"):
+        assert key in d, key
+    assert d["steps"] == 4 and d["warmup"] == 3 and d["n_gpus"] == 1 and d["vs_baseline"] is None and d["data"] == "synthetic"
+    assert d["config"]["workload"] == "config5_B1_ctx4096" and d["gpu_launches"] == 3 * 4
+    rf = d["roofline"]
+    assert rf["bound"] == "hbm" and rf["unit"] == "GB/s" and abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-3 and rf["traffic"] > 0
+    assert d["e2e"]["h2d_bytes_per_step"] > 0 and d["e2e"]["d2h_bytes_per_step"] > 0 and d["e2e"]["value"] > 0
+    assert d["value"] > 0 and d["ms_per_step"] > 0
