@@ -56,7 +56,7 @@ cudaError_t launch_rotated_histogram(const HistogramParams& p, int head_dim, int
 
 // ---- fused decode
 constexpr int DEC_BLOCK_TOKENS = 128;  // cached rows per block of the decode kernel = rows of one transposed V block
-constexpr int DEC_HEADS = 8;          // query heads per CTA (the N extent of the m16n8k16 tile)
+constexpr int DEC_HEADS = 8;          // query heads of one KV head that a work item covers (they share the N columns of one MMA)
 
 struct DecodeParams {
   const uint8_t* k_codes;
