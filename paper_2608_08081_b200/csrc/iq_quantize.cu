@@ -1,5 +1,6 @@
 // Quantize-append kernels: Algorithm 1 (normalise, WHT, SO(4) blocks, 3-bit Lloyd-Max, bit-pack) for new
-// K and V rows, one warp per row. K rows are packed row-major, V rows token-transposed.
+// K and V rows: bulk kernels (a row shared by d/16 lanes), the few-rows kernel of the decode step (a warp per row) and the
+// calibration histogram. K rows are packed row-major, V rows token-transposed.
 #include "iq_common.cuh"
 #include "iq_kernels.h"
 #include "iq_quantize_common.cuh"
