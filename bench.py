@@ -66,7 +66,7 @@ def decode_traffic_bytes(algorithmic_bytes: float, B: int, H_q: int, S: int, d: 
 
 
 def bytes_per_row(d: int) -> int:
-    return 2 * (3 * d // 8) + 2 * 4   # K and V codes + fp32 scales, per cached row per KV head
+    return 2 * (3 * d // 8) + 2 * (2 if SCALES_F16 else 4)   # K and V codes + scales, per cached row per KV head
 
 
 def measured_peak_hbm():
@@ -162,6 +162,7 @@ def aggregate_gbs(bytes_per_rank: float, ms: float, world: int) -> float:
     return world * bytes_per_rank / (ms * 1e-3) / 1e9
 
 
+SCALES_F16 = False  # binary16 scale arrays: 100 instead of 104 bytes per cached row and KV head
 PAGE_ROWS = 0       # > 0: the cache is a pool of pages of this many rows behind a block table in scrambled order
 CODEBOOK = "int8"   # "int8": Lloyd-Max levels on an 8-bit grid (integer tensor-core decode path); "fp16": exact fp16 levels
 
@@ -184,9 +185,10 @@ def build_state(name: str, device, rank: int):
         assert t_cap % PAGE_ROWS == 0, "--page-rows must divide the capacity (ctx + 2048)"
         n_tab = t_cap // PAGE_ROWS
         perm = np.random.Generator(np.random.Philox(77 + rank)).permutation(B * n_tab).astype(np.int32)
-        cache = iq.new_paged_cache(shape, B * n_tab, PAGE_ROWS, torch.from_numpy(perm.reshape(B, n_tab)).to(device), device)
+        cache = iq.new_paged_cache(shape, B * n_tab, PAGE_ROWS, torch.from_numpy(perm.reshape(B, n_tab)).to(device), device,
+                                   scales_dtype=torch.float16 if SCALES_F16 else torch.float32)
     else:
-        cache = iq.new_cache(shape, device)
+        cache = iq.new_cache(shape, device, scales_dtype=torch.float16 if SCALES_F16 else torch.float32)
     status = torch.zeros(4, dtype=torch.int32, device=device)
     lens_np = gen["lens"].astype(np.int32)
     qa_ms, qa_rows = 0.0, 0
@@ -400,7 +402,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                    "t_cap": st["t_cap"], "lengths": "ctx" if per_seq else "ragged, floor(ctx*U[0.5,1.0])",
                    "launch_groups": n_groups, "ms_per_launch_group": round(ms_step / n_groups, 5), "cached_rows_per_kv_head": rows,
                    "num_splits": S, "bytes_per_row_per_kv_head": bytes_per_row(d), "l2": "inputs_larger_than_l2",
-                   "step": "quantize-append 1 row/seq + fused decode + combine", "codebook": CODEBOOK, "cache": (f"paged, {PAGE_ROWS} rows per page, scrambled" if PAGE_ROWS else "contiguous"), "parallelism": f"replicas x{world}",
+                   "step": "quantize-append 1 row/seq + fused decode + combine", "codebook": CODEBOOK, "scales": "fp16" if SCALES_F16 else "fp32", "cache": (f"paged, {PAGE_ROWS} rows per page, scrambled" if PAGE_ROWS else "contiguous"), "parallelism": f"replicas x{world}",
                    "timed_region": ("one replay of a CUDA graph holding the K steps" if graph is not None
                                     else "K steps launched from the host")},
         "decode_tokens_per_s": round(world * B / (ms_step * 1e-3), 1),
@@ -427,7 +429,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         out["graph_error"] = graph_error
     if not args.no_materialised and world == 1 and not per_seq:
         out["reconstruct_then_compute"] = materialised_baseline(st, lens_tab[W + K], q_all[W + K - 1], ws, S, peak)
-    if not args.no_cpu_baseline and world == 1 and not PAGE_ROWS:
+    if not args.no_cpu_baseline and world == 1 and not PAGE_ROWS and not SCALES_F16:
         out["cpu_baseline"] = cpu_baseline(st, lens_tab[n_e2e_warm + n_e2e], q_all[W + K - 1])
     return out
 
@@ -578,11 +580,13 @@ def main():
     ap.add_argument("--splits", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-materialised", action="store_true", help="skip the reconstruct-then-compute comparison")
+    ap.add_argument("--scales", default="fp32", choices=["fp32", "fp16"], help="precision of the stored row norms")
     ap.add_argument("--page-rows", type=int, default=0, help="paged cache: rows per page (multiple of 128 dividing ctx + 2048), pages in scrambled order")
     ap.add_argument("--no-graph", action="store_true", help="time the host-launched loop instead of a CUDA-graph replay of the K steps")
     ap.add_argument("--codebook", default="int8", choices=["int8", "fp16"])
     args = ap.parse_args()
-    global CODEBOOK, PAGE_ROWS
+    global CODEBOOK, PAGE_ROWS, SCALES_F16
+    SCALES_F16 = args.scales == "fp16"
     CODEBOOK = args.codebook
     PAGE_ROWS = args.page_rows
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -75,6 +75,7 @@ enum {
 enum {
   IQ_STATUS_ROW_OUT_OF_RANGE = 1u, /* quantize-append: append_pos + i >= t_cap, row skipped */
   IQ_STATUS_WAIT_TIMEOUT = 2u,     /* decode: a bounded wait on an asynchronous copy ran out; results invalid */
+  IQ_STATUS_SCALE_OVERFLOW = 8u,   /* binary16 scales: a row norm above 65504 was stored as 65504 */
   IQ_STATUS_BAD_PAGE = 4u          /* paged cache: a block-table entry outside [0, num_pages) was met and read as page 0 */
 };
 
@@ -108,6 +109,11 @@ typedef struct iq_cache {
   const int32_t* block_table_dev;
   int32_t page_rows;
   int32_t num_pages;
+  /* 0: k_scales / v_scales are fp32 arrays (52 bytes per row and side at head_dim 128). 1: they are binary16 arrays of
+   * the same shape (the pointers are then really uint16_t*; 50 bytes per row): the norm is rounded to binary16 when a
+   * row is appended -- the row is still normalised by its exact norm -- and a norm beyond the binary16 range is
+   * stored as 65504 and flagged with IQ_STATUS_SCALE_OVERFLOW. */
+  int32_t scales_fp16;
 } iq_cache;
 
 int iq_version(void);

@@ -138,6 +138,15 @@ def new_cache(B: int, H_kv: int, d: int, t_cap: int):
     )
 
 
+def round_scales_fp16(cache) -> None:
+    """The binary16-scales variant of the cache (50 instead of 52 bytes per row and side): every stored norm rounded to
+    the nearest binary16 value (saturating at 65504), kept in the fp32 arrays. Rows are normalised by their exact norm
+    either way; only the stored scale, which decode multiplies back, is rounded. Idempotent."""
+    for name in ("k_scales", "v_scales"):
+        a = cache[name]
+        a[...] = np.minimum(a, np.float32(65504.0)).astype(np.float16).astype(np.float32)
+
+
 def quantize_append(quats, thresholds, k_new, v_new, append_pos, n_new, cache) -> int:
     """k_new, v_new: fp16 [B][n_new_max][H_kv][d] (any strides, last dim contiguous). Appends in place."""
     k = k_new.view(np.uint16) if k_new.dtype == np.float16 else k_new

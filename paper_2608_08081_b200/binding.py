@@ -26,7 +26,7 @@ class _IqCodebook(ctypes.Structure):
 
 class _IqCache(ctypes.Structure):
     _fields_ = [("k_codes", _vp), ("k_scales", _vp), ("v_codes", _vp), ("v_scales", _vp),
-                ("block_table_dev", _vp), ("page_rows", _i32), ("num_pages", _i32)]
+                ("block_table_dev", _vp), ("page_rows", _i32), ("num_pages", _i32), ("scales_fp16", _i32)]
 
 
 class IQError(RuntimeError):
@@ -129,11 +129,13 @@ class Cache:
     page_rows: int = 0
 
     def c(self) -> _IqCache:
+        assert self.k_scales.dtype == self.v_scales.dtype and self.k_scales.dtype in (torch.float32, torch.float16)
+        f16 = 1 if self.k_scales.dtype == torch.float16 else 0   # binary16 scale arrays: 50 instead of 52 bytes per row
         if self.block_table is None:
-            return _IqCache(self.k_codes.data_ptr(), self.k_scales.data_ptr(), self.v_codes.data_ptr(), self.v_scales.data_ptr(), None, 0, 0)
+            return _IqCache(self.k_codes.data_ptr(), self.k_scales.data_ptr(), self.v_codes.data_ptr(), self.v_scales.data_ptr(), None, 0, 0, f16)
         assert self.block_table.dtype == torch.int32 and self.block_table.is_contiguous()
         return _IqCache(self.k_codes.data_ptr(), self.k_scales.data_ptr(), self.v_codes.data_ptr(), self.v_scales.data_ptr(),
-                        self.block_table.data_ptr(), self.page_rows, self.k_scales.shape[0])
+                        self.block_table.data_ptr(), self.page_rows, self.k_scales.shape[0], f16)
 
 
 def _ptr(t):
@@ -284,22 +286,24 @@ def iq_suggest_splits(shape: Shape, max_seq_len: int) -> int:
 
 
 # ------------------------------------------------------------------ small conveniences (allocation only)
-def new_cache(shape: Shape, device="cuda") -> Cache:
+def new_cache(shape: Shape, device="cuda", scales_dtype=torch.float32) -> Cache:
+    """scales_dtype: torch.float32, or torch.float16 for binary16 scale arrays."""
     P = iq_row_bytes(shape.head_dim)
     n = (shape.batch, shape.n_kv_heads, shape.t_cap)
-    return Cache(torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=torch.float32, device=device),
-                 torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=torch.float32, device=device))
+    return Cache(torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=scales_dtype, device=device),
+                 torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=scales_dtype, device=device))
 
 
-def new_paged_cache(shape: Shape, num_pages: int, page_rows: int, block_table: torch.Tensor, device="cuda") -> Cache:
+def new_paged_cache(shape: Shape, num_pages: int, page_rows: int, block_table: torch.Tensor, device="cuda",
+                    scales_dtype=torch.float32) -> Cache:
     """A pool of num_pages pages of page_rows rows (a multiple of 128 that divides shape.t_cap) and the block table
     (int32 device tensor [batch][t_cap / page_rows]) that maps the sequences' rows onto it."""
     assert page_rows % 128 == 0 and shape.t_cap % page_rows == 0
     assert tuple(block_table.shape) == (shape.batch, shape.t_cap // page_rows)
     P = iq_row_bytes(shape.head_dim)
     n = (num_pages, shape.n_kv_heads, page_rows)
-    return Cache(torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=torch.float32, device=device),
-                 torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=torch.float32, device=device),
+    return Cache(torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=scales_dtype, device=device),
+                 torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=scales_dtype, device=device),
                  block_table, page_rows)
 
 

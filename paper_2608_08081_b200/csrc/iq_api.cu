@@ -302,6 +302,7 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
   p.n_kv_heads = shape->n_kv_heads;
   p.t_cap = shape->t_cap;
   p.pm = page_map(cache, shape);
+  p.scale_f16 = cache->scales_fp16 ? 1 : 0;
   const cudaError_t e = iq::launch_quantize_append(p, shape->head_dim, shape->batch, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }
@@ -341,6 +342,7 @@ int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_co
   p.head_groups = (p.group + iq::DEC_HEADS - 1) / iq::DEC_HEADS;
   p.t_cap = shape->t_cap;
   p.pm = page_map(cache, shape);
+  p.scale_f16 = cache->scales_fp16 ? 1 : 0;
   p.splits = num_splits;
   p.sm_scale = shape->sm_scale > 0.f ? shape->sm_scale : 1.0f / std::sqrt((float)shape->head_dim);
   p.lut_lo[0] = p.lut_lo[1] = p.lut_hi[0] = p.lut_hi[1] = 0u;
@@ -417,6 +419,7 @@ int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_co
   p.n_kv_heads = shape->n_kv_heads;
   p.t_cap = shape->t_cap;
   p.pm = page_map(cache, shape);
+  p.scale_f16 = cache->scales_fp16 ? 1 : 0;
   p.status = nullptr;
   p.out_rows = out_rows;
   std::memcpy(p.levels, codebook->levels, sizeof(p.levels));

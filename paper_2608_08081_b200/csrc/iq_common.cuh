@@ -165,6 +165,22 @@ __device__ __forceinline__ size_t cache_row(const PageMap& m, int b, int g, long
   return ((size_t)page * m.n_kv_heads + g) * (size_t)m.page_rows + (size_t)(t - (long long)j * m.page_rows);
 }
 
+// The scale arrays hold fp32 values or (f16 != 0) binary16 values of the same shape.
+__device__ __forceinline__ void store_scale(float* arr, size_t row, float s, int f16, uint32_t* status) {
+  if (!f16) {
+    arr[row] = s;
+  } else {
+    if (s > 65504.f) {
+      if (status) atomicOr(&status[0], IQ_STATUS_SCALE_OVERFLOW);
+      s = 65504.f;
+    }
+    reinterpret_cast<__half*>(arr)[row] = __float2half_rn(s);
+  }
+}
+__device__ __forceinline__ float load_scale(const void* arr, size_t row, int f16) {
+  return f16 ? __half2float(reinterpret_cast<const __half*>(arr)[row]) : reinterpret_cast<const float*>(arr)[row];
+}
+
 #ifndef IQ_MBAR_SUSPEND_NS
 #define IQ_MBAR_SUSPEND_NS 20000
 #endif

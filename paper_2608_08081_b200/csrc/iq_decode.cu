@@ -378,14 +378,14 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           const int n = min(TB, len - r0);
           if (elect_one()) {
             desc[st] = make_int2(r0, n);
-            const int n4 = (n + 3) & ~3;
+            const uint32_t sc_bytes = p.scale_f16 ? (uint32_t)(((n + 7) & ~7) * 2) : (uint32_t)(((n + 3) & ~3) * 4);  // whole 16-byte pieces
             uint8_t* sp = stages + st * L::STAGE_BYTES;
             fence_proxy_async();
-            mbar_expect_tx(&full_bar[st], (uint32_t)(n * L::ROWB + L::VT_BYTES + 2 * n4 * 4));  // also publishes desc[st]
+            mbar_expect_tx(&full_bar[st], (uint32_t)(n * L::ROWB + L::VT_BYTES) + 2 * sc_bytes);  // also publishes desc[st]
             bulk_g2s(sp, p.k_codes + row0 * L::ROWB, (uint32_t)(n * L::ROWB), &full_bar[st]);
             bulk_g2s(sp + L::K_BYTES, p.v_codes + row0 * L::ROWB, (uint32_t)L::VT_BYTES, &full_bar[st]);  // whole 128-row V block
-            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES, p.k_scales + row0, (uint32_t)(n4 * 4), &full_bar[st]);
-            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES, p.v_scales + row0, (uint32_t)(n4 * 4), &full_bar[st]);
+            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES, reinterpret_cast<const uint8_t*>(p.k_scales) + row0 * (p.scale_f16 ? 2 : 4), sc_bytes, &full_bar[st]);
+            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES, reinterpret_cast<const uint8_t*>(p.v_scales) + row0 * (p.scale_f16 ? 2 : 4), sc_bytes, &full_bar[st]);
           }
         } else {
           ended = true;
@@ -554,8 +554,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
             tc_st8(tmem_g + lane_sel + L::I8_V_COL + 32 * j + 8 * u, f);
           }
         }
-        const float ksc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES)[gt];
-        const float vsc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES)[gt];
+        const float ksc = load_scale(sp + L::K_BYTES + L::VT_BYTES, gt, p.scale_f16);
+        const float vsc = load_scale(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES, gt, p.scale_f16);
         const bool valid = gt < n;  // rows >= n of the last block hold stale bytes
         const float kfs = valid ? ksc * sfac : 0.f;
         const float mask = valid ? 0.f : -INFINITY;  // stale rows: 0 * finite - inf = -inf
@@ -716,8 +716,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
             wd[j][4 * i] = t4.x; wd[j][4 * i + 1] = t4.y; wd[j][4 * i + 2] = t4.z; wd[j][4 * i + 3] = t4.w;
           }
         }
-        const float ksc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES)[gt];
-        const float vsc = reinterpret_cast<const float*>(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES)[gt];
+        const float ksc = load_scale(sp + L::K_BYTES + L::VT_BYTES, gt, p.scale_f16);
+        const float vsc = load_scale(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES, gt, p.scale_f16);
         auto v_unit = [&](int j, int u) {  // rows 32u .. 32u+31 of coordinate gt + 128 j
           uint32_t f[16];
           dequant_unit(wd[j][3 * u], wd[j][3 * u + 1], wd[j][3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);

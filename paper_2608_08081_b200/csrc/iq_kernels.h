@@ -34,6 +34,7 @@ struct QuantizeParams {
   uint32_t* status;
   int n_kv_heads, t_cap;
   PageMap pm;
+  int scale_f16;
 };
 cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int batch, cudaStream_t stream);
 
@@ -72,6 +73,7 @@ struct DecodeParams {
   uint32_t* status;
   int batch, n_q_heads, n_kv_heads, group, head_groups, t_cap, splits;
   PageMap pm;
+  int scale_f16;
   float sm_scale;
   uint32_t lut_lo[2], lut_hi[2];  // low / high bytes of the 8 fp16 levels, 4 per register
   // integer path (levels on an 8-bit grid): level_j = lut8 byte j (int8) * delta
@@ -108,6 +110,7 @@ struct ReconstructParams {
   long long stride_b, stride_t, stride_h;  // in elements
   int n_kv_heads, t_cap, out_rows;
   PageMap pm;
+  int scale_f16;
   uint32_t* status;
   float levels[8];
 };

@@ -278,7 +278,7 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 5) quantize_append_k_kernel(con
       uint32_t* unit_words = reinterpret_cast<uint32_t*>(p.k_codes + row * (size_t)(3 * D / 8)) + 3 * (li >> 1);
       if (li & 1) unit_words[2] = w0;
       else { unit_words[0] = w0; unit_words[1] = w1; }
-      if (li == 0) p.k_scales[row] = s;
+      if (li == 0) store_scale(p.k_scales, row, s, p.scale_f16, p.status);
     }
   }
 }
@@ -356,7 +356,7 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
       for (int q = 0; q < 4; q++)
         pk[q] = (uint32_t)code[4 * q] | ((uint32_t)code[4 * q + 1] << 8) | ((uint32_t)code[4 * q + 2] << 16) | ((uint32_t)code[4 * q + 3] << 24);
       *reinterpret_cast<uint4*>(&codes_s[t & 127][li * 16]) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-      if (li == 0) p.v_scales[block_row0 + (size_t)(t & 127)] = s;
+      if (li == 0) store_scale(p.v_scales, block_row0 + (size_t)(t & 127), s, p.scale_f16, p.status);
     }
   }
   __syncthreads();
@@ -562,7 +562,7 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
       const int k = lane % LPU;
       uint32_t* row_words = reinterpret_cast<uint32_t*>(p.k_codes + row * (size_t)(3 * D / 8));
       if (k < 3) row_words[3 * (lane / LPU) + k] = (k == 0) ? w[0] : (k == 1 ? w[1] : w[2]);
-      if (lane == 0) p.k_scales[row] = s;
+      if (lane == 0) store_scale(p.k_scales, row, s, p.scale_f16, p.status);
     } else {
       // transposed records: row t is entry r = t % 32 of unit u = (t % 128) / 32 of block t / 128, for every coordinate
       const size_t blk = row / 128;  // (a page holds whole 128-row blocks: row / 128 is the block's index in the V array)
@@ -581,7 +581,7 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
           for (int k = 0; k < 3; k++) dst[k] = (dst[k] & ~(1u << sh)) | (((cd >> k) & 1u) << sh);
         }
       }
-      if (lane == 0) p.v_scales[row] = s;
+      if (lane == 0) store_scale(p.v_scales, row, s, p.scale_f16, p.status);
     }
   }
 }

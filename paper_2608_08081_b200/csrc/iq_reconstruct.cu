@@ -44,8 +44,8 @@ __global__ void __launch_bounds__(RC_WARPS * 32) reconstruct_kernel(const Recons
     for (int i = tid; i < n * ROWB / 16; i += RC_WARPS * 32) reinterpret_cast<uint4*>(k_s)[i] = ksrc[i];
     for (int i = tid; i < D * 48 / 16; i += RC_WARPS * 32) reinterpret_cast<uint4*>(v_s)[i] = vsrc[i];
     if (tid < n) {
-      ks_s[tid] = p.k_scales[row0 + tid];
-      vs_s[tid] = p.v_scales[row0 + tid];
+      ks_s[tid] = load_scale(p.k_scales, row0 + tid, p.scale_f16);
+      vs_s[tid] = load_scale(p.v_scales, row0 + tid, p.scale_f16);
     }
     if (tid < 8) lv_s[tid] = p.levels[tid];
   }

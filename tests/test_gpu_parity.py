@@ -489,6 +489,60 @@ def test_context_sharded_decode_on_one_gpu(iq, torch, codebooks):
     dist.destroy_process_group()
 
 
+@pytest.mark.parametrize("d", [128, 256])
+def test_binary16_scales(iq, torch, codebooks, d):
+    """The 50-bytes-per-row variant: scale arrays in binary16. Appends (bulk with ragged lengths and a partly filled
+    block, then a single-row step), decode and reconstruction against the oracle with its stored norms rounded the same
+    way; a row whose norm exceeds the binary16 range is stored as 65504 and flagged."""
+    B, H_q, H_kv, T = 2, 8, 2, 300
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    lens = np.array([297, 130], np.int32)
+    w = workloads.tiny(1500 + d, B, H_q, H_kv, d, T, lens)
+    w.k[0, 11] = (w.k[0, 11].astype(np.float32) * 6000).astype(np.float16)             # norm ~ 6000 * sqrt(d) > 65504
+    shape = iq.Shape(B, H_q, H_kv, d, w.t_cap)
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(w.quats), rot)
+    cache = iq.new_cache(shape, scales_dtype=torch.float16)
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(w.k).cuda(), torch.from_numpy(w.v).cuda(),
+                          torch.zeros(B, dtype=torch.int32, device="cuda"), torch.from_numpy(lens).cuda(), T, cache, status)
+    ref = oracle.new_cache(B, H_kv, d, w.t_cap)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), lens, ref)
+    kn = np.stack([w.k[b, lens[b]] for b in range(B)])[:, None]
+    vn = np.stack([w.v[b, lens[b]] for b in range(B)])[:, None]
+    iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), torch.from_numpy(lens).cuda(), None, 1, cache, status)
+    oracle.quantize_append(w.quats, th, kn, vn, lens, None, ref)
+    oracle.round_scales_fp16(ref)
+    now = lens + 1
+    torch.cuda.synchronize()
+    assert status.cpu().numpy()[0] == 8                                               # IQ_STATUS_SCALE_OVERFLOW, nothing else
+    g = dict(k_codes=cache.k_codes.cpu().numpy(), v_codes=cache.v_codes.cpu().numpy(),
+             k_scales=cache.k_scales.float().cpu().numpy(), v_scales=cache.v_scales.float().cpu().numpy())
+    assert g["k_scales"][0, :, 11].max() == 65504.0
+    for name in ("k_scales", "v_scales"):                                             # equal but for norms that sit on a rounding boundary
+        for b in range(B):
+            a, r = g[name][b, :, :now[b]], ref[name][b, :, :now[b]]
+            off = a != r
+            assert off.mean() <= 2e-3 and np.all(np.abs(a - r)[off] <= 2.0 ** -10 * r[off])
+    assert np.array_equal(g["k_codes"][0, :, :now[0]], ref["k_codes"][0, :, :now[0]])
+    w2 = workloads.Workload("h16", B, H_q, H_kv, d, w.t_cap, w.k, w.v, w.q, w.quats, now)
+    S = iq.iq_suggest_splits(shape, T)
+    ws = iq.DecodeWorkspace(shape, S, want_argmax=True)
+    iq.decode_step(shape, rot, cb, torch.from_numpy(w.q).cuda(), cache, torch.from_numpy(now).cuda(), ws)
+    torch.cuda.synchronize()
+    res = dict(out=ws.out.cpu().numpy().astype(np.float64), lse=ws.lse.cpu().numpy().astype(np.float64), argmax=ws.argmax.cpu().numpy())
+    check_decode(w2, lv, w.q, res, g, now)                                            # the oracle on the GPU's own (rounded) cache
+    k_out = torch.zeros((B, w.t_cap, H_kv, d), dtype=torch.float16, device="cuda")
+    v_out = torch.zeros_like(k_out)
+    iq.iq_reconstruct_rows(shape, rot, cb, cache, torch.from_numpy(now).cuda(), k_out, v_out)
+    K, V = oracle.reconstruct_rows(w.quats, lv, g, now, H_kv)
+    for got, r in ((k_out.cpu().numpy().astype(np.float64), K), (v_out.cpu().numpy().astype(np.float64), V)):
+        fin = np.abs(r) < 6e4                                                         # (the blown-up row overflows binary16 outputs)
+        bound = 2.0 ** -11 * 1.001 * np.abs(r) + 1e-5 * np.abs(r).max(axis=-1, keepdims=True) + 1e-30
+        assert np.all((np.abs(got - r) <= bound)[fin])
+
+
 def test_combine_splits_in_isolation(iq, torch, codebooks):
     d, B, H_q, H_kv, S = 128, 3, 8, 2, 5
     g = np.random.default_rng(7)

@@ -418,6 +418,35 @@ def test_rotated_histogram_counts_what_the_quantiser_sees(codebooks):
     assert abs(mean) < 0.02 and abs(var - 1.0) < 0.01                             # sum of u^2 over a row is exactly d
 
 
+def test_binary16_scales_variant(codebooks):
+    """round_scales_fp16: the stored norms become binary16 values within 2^-11 of the exact ones (saturating at 65504),
+    codes are untouched, the rounding is idempotent, and the attention output moves by no more than the scales did."""
+    d = 128
+    lv, th = codebooks[d]
+    w = workloads.tiny(5, 1, 4, 2, d, 200)
+    w.k[0, 3] = np.clip(w.k[0, 3].astype(np.float32) * 9000, -65504, 65504).astype(np.float16)
+    cache = oracle.new_cache(1, 2, d, w.t_cap)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(1, np.int32), None, cache)
+    exact = {k: v.copy() for k, v in cache.items()}
+    oracle.round_scales_fp16(cache)
+    for name in ("k_scales", "v_scales"):
+        a, e = cache[name], exact[name]
+        assert np.array_equal(a.astype(np.float16).astype(np.float32), a)
+        ok = e <= 65504
+        assert np.all(np.abs(a - e)[ok] <= 2.0 ** -11 * e[ok]) and np.all(a[~ok] == 65504.0) and (~ok).sum() == (2 if name == "k_scales" else 0)
+    assert np.array_equal(cache["k_codes"], exact["k_codes"]) and np.array_equal(cache["v_codes"], exact["v_codes"])
+    again = {k: v.copy() for k, v in cache.items()}
+    oracle.round_scales_fp16(again)
+    assert all(np.array_equal(again[k], cache[k]) for k in cache)
+    lens = np.array([200], np.int32)
+    keep = np.ones(200, bool); keep[3] = False                       # (leave the saturated row out of the comparison)
+    for c in (cache, exact):
+        c["k_scales"][0, :, 3] = 0
+    r16 = oracle.decode_attention(w.quats, lv, w.q, cache, lens, 2)["out"]
+    r32 = oracle.decode_attention(w.quats, lv, w.q, exact, lens, 2)["out"]
+    assert np.max(np.abs(r16 - r32)) <= 4e-3 * np.max(np.abs(r32)) and np.max(np.abs(r16 - r32)) > 0
+
+
 def test_attention_special_cases(codebooks):
     d = 128
     lv, th = codebooks[d]
