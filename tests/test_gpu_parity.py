@@ -543,6 +543,78 @@ def test_binary16_scales(iq, torch, codebooks, d):
         assert np.all((np.abs(got - r) <= bound)[fin])
 
 
+@pytest.mark.parametrize("case", range(16))
+def test_random_configurations(iq, torch, codebooks, case):
+    """Seeded random shapes through the whole path: head counts and group sizes, head_dim, ragged lengths with empty
+    sequences, split counts from 1 upwards, contiguous or paged cache, fp32 or binary16 scales, bulk append followed by
+    single-row steps -- cache and decode output against the oracle every time."""
+    g = np.random.Generator(np.random.Philox(9000 + case))
+    d = int(g.choice([128, 128, 256]))
+    H_kv = int(g.choice([1, 2, 3]))
+    G = int(g.choice([1, 2, 4, 8, 12]))
+    H_q = H_kv * G
+    B = int(g.integers(1, 6))
+    T = int(g.choice([128, 384, 640]))
+    lens = g.integers(0, T - 3, size=B).astype(np.int32)
+    if case % 4 == 0:
+        lens[0] = T - 3
+    paged = bool(case % 2)
+    page_rows = int(g.choice([128, 128 * (T // 128)])) if paged else 0
+    f16 = bool((case // 2) % 2)
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    w = workloads.tiny(9100 + case, B, H_q, H_kv, d, T, lens)
+    shape = iq.Shape(B, H_q, H_kv, d, T)
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(w.quats), rot)
+    sdt = torch.float16 if f16 else torch.float32
+    if paged:
+        n_tab = T // page_rows
+        table = g.permutation(B * n_tab + 2)[:B * n_tab].reshape(B, n_tab).astype(np.int32)
+        cache = iq.new_paged_cache(shape, B * n_tab + 2, page_rows, torch.from_numpy(table).cuda(), scales_dtype=sdt)
+    else:
+        cache = iq.new_cache(shape, scales_dtype=sdt)
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(w.k).cuda(), torch.from_numpy(w.v).cuda(),
+                          torch.zeros(B, dtype=torch.int32, device="cuda"), torch.from_numpy(lens).cuda(), T, cache, status)
+    ref = oracle.new_cache(B, H_kv, d, T)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), lens, ref)
+    now = lens.copy()
+    for step in range(int(g.integers(0, 3))):
+        kn = np.stack([w.k[b, now[b]] for b in range(B)])[:, None]
+        vn = np.stack([w.v[b, now[b]] for b in range(B)])[:, None]
+        iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), torch.from_numpy(now).cuda(), None, 1, cache, status)
+        oracle.quantize_append(w.quats, th, kn, vn, now, None, ref)
+        now = now + 1
+    if f16:
+        oracle.round_scales_fp16(ref)
+    torch.cuda.synchronize()
+    assert status.cpu().numpy()[0] == 0
+    if paged:
+        got = _gather_pages(cache, table, page_rows)
+    else:
+        got = cache_to_numpy(cache)
+    got["k_scales"] = got["k_scales"].astype(np.float32)
+    got["v_scales"] = got["v_scales"].astype(np.float32)
+    # the appended rows, wherever they came from: prefill rows 0 .. lens-1, then the step rows
+    full_k, full_v = w.k.copy(), w.v.copy()
+    w2 = workloads.Workload("rnd", B, H_q, H_kv, d, T, full_k, full_v, w.q, w.quats, now)
+    if not f16:
+        compare_caches(w2, th, got, ref, now)
+    else:
+        for b in range(B):
+            assert np.array_equal(got["k_codes"][b, :, :now[b]], ref["k_codes"][b, :, :now[b]])   # codes do not depend on how the norm is stored
+            nb = (int(now[b]) + 127) // 128
+            vg = got["v_codes"][b].reshape(H_kv, -1)[:, :nb * 128 * oracle.row_bytes(d)]
+            vr = ref["v_codes"][b].reshape(H_kv, -1)[:, :nb * 128 * oracle.row_bytes(d)]
+            assert np.array_equal(vg, vr)
+            a, r = got["k_scales"][b, :, :now[b]], ref["k_scales"][b, :, :now[b]]
+            assert np.all(np.abs(a - r) <= 2.0 ** -10 * r)
+    S = int(g.choice([1, 2, 3, iq.iq_suggest_splits(shape, T)]))
+    res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, now, S)
+    check_decode(w2, lv, w.q, res, got, now)
+
+
 def test_combine_splits_in_isolation(iq, torch, codebooks):
     d, B, H_q, H_kv, S = 128, 3, 8, 2, 5
     g = np.random.default_rng(7)
