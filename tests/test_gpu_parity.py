@@ -1,6 +1,7 @@
 """GPU-vs-oracle parity through the C ABI: packed codes bit-exact (ties excused and counted), attention
 outputs within 2e-3 + 1e-3 |ref| of the fp64 oracle run on the same packed cache, argmax identical."""
 import math
+import os
 
 import numpy as np
 import pytest
@@ -543,7 +544,7 @@ def test_binary16_scales(iq, torch, codebooks, d):
         assert np.all((np.abs(got - r) <= bound)[fin])
 
 
-@pytest.mark.parametrize("case", range(16))
+@pytest.mark.parametrize("case", range(int(os.environ.get("IQ_RANDOM_CASES", "16"))))
 def test_random_configurations(iq, torch, codebooks, case):
     """Seeded random shapes through the whole path: head counts and group sizes, head_dim, ragged lengths with empty
     sequences, split counts from 1 upwards, contiguous or paged cache, fp32 or binary16 scales, bulk append followed by
