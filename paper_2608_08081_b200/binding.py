@@ -43,7 +43,7 @@ def _load():
     path = lib_path()
     if not os.path.exists(path):
         raise ImportError(
-            f"{path} is missing: build it with `python -m paper_2608_08081_b200.build` (needs nvcc). "
+            f"{path} is missing: build it with `python paper_2608_08081_b200/build.py` (needs nvcc). "
             "There is no fallback implementation.")
     lib = ctypes.CDLL(path)
     lib.iq_version.restype = ctypes.c_int
