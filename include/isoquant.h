@@ -176,11 +176,14 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
  *   q              device binary16 [batch][n_q_heads][head_dim], 16-byte aligned; not quantised.
  *   seq_lens_dev   device int32 [batch]: rows 0 .. len-1 of each sequence are attended to (clamped to
  *                  [0, t_cap]); the row appended last is attended to like any other.
- *   num_splits     S >= 1: partial slots per (sequence, head). The rows of a sequence are covered by at most S
- *                  consecutive, non-overlapping row ranges (multiples of 128 rows except at the end), one slot per
- *                  range, in ascending order; which ranges is the library's choice (it balances the launch: every
- *                  SM takes an equal share of the 128-row blocks of the whole batch).
- *                  A small S restricts that choice; iq_suggest_splits gives a value that does not.
+ *   num_splits     S >= 1: partial slots per (sequence, head). Every cached row of a sequence is covered by exactly one
+ *                  slot of each head; which rows a slot covers is the library's choice, and a slot's rows need not be
+ *                  consecutive. With S >= 2 G (G = 4 workers per SM at head_dim 128, 2 at 256) the launch is balanced
+ *                  over the whole batch: every SM takes an equal, contiguous share of all 128-row blocks, and the part of
+ *                  a (sequence, KV head) inside a share reports to G slots, one per worker of that SM. With fewer slots
+ *                  every (sequence, KV head) is cut into S runs of consecutive blocks, one slot each, dealt out to the
+ *                  workers in turn (S = 1: one worker per (sequence, KV head), no merge needed afterwards).
+ *                  iq_suggest_splits gives a value for the balanced mode.
  *   part_acc       device fp32 [batch][n_q_heads][S][head_dim]: sum_j exp(z_j - m) v~_j over the slot's rows,
  *                  in the rotated space, natural coordinate order. 16-byte aligned.
  *   part_ml        device fp32 [batch][n_q_heads][S][2] = (m, l): the slot's reference m and l = sum_j exp(z_j - m),

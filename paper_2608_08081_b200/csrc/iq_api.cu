@@ -513,15 +513,19 @@ int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len) {
   }
   const int group = shape->n_q_heads / shape->n_kv_heads;
   const long long items = (long long)(shape->batch > 0 ? shape->batch : 1) * shape->n_kv_heads * ((group + iq::DEC_HEADS - 1) / iq::DEC_HEADS);
-  const long long slots = (long long)n_sm * iq::decode_ctas_per_sm(shape->head_dim);
-  // The decode kernel gives every SM an equal, contiguous share of the launch's 128-row blocks; an item of nb blocks
-  // then reports to about nb / share + 1 slots. With all sequences at full length share = items * nb / slots; the
-  // factor 1.5 leaves room for batches whose mean length is two thirds of the longest.
-  long long s = (15 * slots + 10 * items - 1) / (10 * items) + 1;
-  const long long cap = (max_seq_len + 255) / 256;         // at least 256 rows (two blocks) per slot
-  if (s > cap) s = cap;
-  if (s < 1) s = 1;
-  if (s > 256) s = 256;
+  const long long ctas = (long long)n_sm * iq::decode_ctas_per_sm(shape->head_dim);
+  const int ng = iq::decode_groups_per_cta(shape->head_dim);
+  // The decode kernel gives every CTA an equal, contiguous share of the launch's 128-row blocks; an item of nb blocks
+  // then has about nb / share + 1 pieces, and every piece reports to one slot per group of its CTA. With all sequences
+  // at full length share = items * nb / ctas; the factor 1.5 leaves room for batches whose mean length is two thirds
+  // of the longest. A piece is not worth less than one block per group.
+  const long long nb = (max_seq_len + iq::DEC_BLOCK_TOKENS - 1) / iq::DEC_BLOCK_TOKENS;
+  long long pieces = (15 * ctas + 10 * items - 1) / (10 * items) + 1;
+  const long long cap = (nb + ng - 1) / ng;
+  if (pieces > cap) pieces = cap;
+  if (pieces < 2) pieces = 2;
+  long long s = pieces * ng;
+  if (s > 1024) s = 1024;
   return (int32_t)s;
 }
 

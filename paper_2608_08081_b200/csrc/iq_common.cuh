@@ -195,7 +195,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after `limit` polls and reports false (the caller flags the error and unwinds).
+// Bounded wait: gives up after `limit` polls and reports false (the caller flags the error and unwinds). A poll that
+// does not find the phase complete suspends the thread for at most IQ_MBAR_SUSPEND_NS, so `limit` polls last at most
+// limit * IQ_MBAR_SUSPEND_NS (plus the polls' own latency) and at least limit times the latency of a poll (tens of
+// nanoseconds). The loop is kept this plain on purpose: a timer read or an out-of-line call in it measurably slows
+// the kernels that wait, whose waits all succeed.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t limit) {
   for (uint32_t i = 0; i < limit; i++)
     if (mbar_try_wait(bar, parity)) return true;

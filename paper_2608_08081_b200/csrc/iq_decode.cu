@@ -2,27 +2,31 @@
 // softmax, value accumulation on packed V codes, on the 5th-generation tensor cores (tcgen05) with the
 // dequantised operands resident in tensor memory (TMEM).
 //
-// Work decomposition. The 128-row blocks of all (sequence, KV head, head group) items of the launch are laid
-// end to end and every CTA -- one per SM -- takes an equal, contiguous range of that sequence, whatever the length
-// mix of the batch. A range is processed item piece by item piece ("segment"); each segment ends in one partial
-// result (slot) of the item. Inside the CTA, NG groups of 4 compute warps + 1 control warp each run their own
-// tile pipeline and draw the segment's blocks one at a time from a shared-memory counter, so the groups stay
-// busy until the segment is exhausted even though the warp schedulers do not serve them evenly; their partial
-// softmax states are merged in shared memory at the end of the segment.
+// Work decomposition. A CTA -- one per SM -- holds NG independent workers ("groups": 4 compute warps + 1 control
+// warp, their own TMEM columns, tile pipeline, query operand and softmax state). After the set-up there is no
+// CTA-wide synchronisation: a group never waits for another group.
+//   Range mode (num_splits >= 2 NG). The 128-row blocks of all (sequence, KV head, head group) items of the launch
+//   are laid end to end and every CTA takes an equal, contiguous range of that sequence, whatever the length mix of
+//   the batch. The groups of the CTA draw the blocks of the range one at a time from a shared-memory counter, so they
+//   stay busy although the warp schedulers do not serve them evenly. The part of one item inside a range is a
+//   "segment"; piece k of an item (its k-th CTA) reports to partial slots k NG .. k NG + NG - 1, one per group. A
+//   group that crosses into another segment writes its partial of the old one straight to its slot, rotates the
+//   queries of the new item into its own operand buffer and goes on, while its tiles keep streaming in.
+//   Unit mode (fewer slots). Every item is cut into num_splits consecutive runs of blocks, run k reports to slot
+//   k, and the runs are dealt out to the groups of all CTAs in turn.
+// Every partial slot of every head is written on every launch: by the group that worked on it, else by the
+// control warp that is responsible for it (unused slots hold m = -inf, l = 0, acc = 0).
 //
 // Per block, in group g (thread r of the group = TMEM lane r):
-//   1. thread r dequantises packed K row r (its own 3d/8 bytes from the staged tile) into fp16 and stores it
-//      to TMEM lane r: A_K[128 rows x d].
-//   2. the control warp issues tcgen05.mma (M = 128 rows, N = 16, K = 16 per instruction):
-//         S[row][n] = sum_i A_K[row][i] * B_Q[n][i],  B_Q = q~ of the <= 8 heads as fp16 hi (n < 8) and lo (n >= 8)
-//   3. every thread reads its row of S back, applies the K scale, joins the group-wide running maximum and
-//      writes its probabilities (times the V scale, again as fp16 hi / lo) into the shared-memory operand
-//      B_P[n][row].
+//   1. thread r dequantises packed K row r (its own 3d/8 bytes from the staged tile) and stores it to TMEM lane r.
+//   2. the control warp issues tcgen05.mma (M = 128 rows): S[row][n] = sum_i A_K[row][i] * B_Q[n][i], the columns n
+//      holding q~ of the <= 8 heads (fp16 hi | lo, or three int8 digits per head).
+//   3. every thread reads its row of S back, applies the K scale, joins the group-wide running reference and
+//      writes its probabilities (times the V scale) into the shared-memory operand B_P[n][row].
 //   4. thread c dequantises coordinate c of the token-transposed V block (128 codes = one 48-byte row) into
-//      TMEM lane c: A_V[d coords x 128 rows] (same columns as A_K, once the score MMAs have read them); the
-//      control warp issues   O[c][n] = sum_row A_V[c][row] * B_P[n][row]
-//   5. thread c folds O (hi + lo columns) into its running accumulator for coordinate c.
-// Packed tiles arrive through a 1-D bulk-copy (TMA) pipeline; every mbarrier wait is bounded.
+//      TMEM lane c; the control warp issues O[c][n] = sum_row A_V[c][row] * B_P[n][row].
+//   5. thread c folds O into its running accumulator for coordinate c.
+// Packed tiles arrive through a 1-D bulk-copy (TMA) pipeline; every mbarrier wait is bounded in time.
 #include <climits>
 
 #include "iq_decode_common.cuh"
@@ -31,12 +35,26 @@
 namespace iq {
 
 constexpr int DEC_GROUP_THREADS = 128;  // 4 warps: dequantisation, softmax, accumulation (thread = TMEM lane)
-constexpr int DEC_HDR_BYTES = 4096;    // barriers, TMEM base, work counter, segment and block descriptors, scratch
+constexpr int DEC_HDR_BYTES = 4096;    // barriers, TMEM base, work counter, block descriptors, scratch
+constexpr int DEC_NPRE = 4;             // query operands prepared at the start of a CTA: those of its range's first segments
+constexpr int DEC_PRE_BAR = 9;          // named barrier of all compute threads (used while those operands are built)
 constexpr float DEC_MAX_SLACK = 4.0f;  // log2 units a score may exceed the running reference before it is raised
 #ifndef IQ_SLACK_I8
 #define IQ_SLACK_I8 4
 #endif
 constexpr float DEC_MAX_SLACK_I8 = (float)IQ_SLACK_I8;  // the same on the integer path, where the probabilities are fixed-point numbers
+
+// What the control warp tells the compute warps about a staged tile.
+struct DecDesc {
+  int n;        // valid rows of the block; n < 0: end marker, the group is done
+  int flags;    // bit 0: first block this group gets of a segment: close the open one, open (b, y, slot)
+  int r0;       // first row of the block in its sequence
+  int slot;     // partial slot of the item this group reports the segment to
+  int b, y;     // sequence, item within it (KV head x head group)
+  int len;      // cached rows of the sequence (unused by the compute warps; kept for diagnosis)
+  int bqbuf;    // which prepared query operand the segment uses, -1: the group builds its own
+};
+static_assert(sizeof(DecDesc) == 32, "descriptor layout");
 
 template <int D>
 struct DecLayout {
@@ -48,10 +66,10 @@ struct DecLayout {
   static constexpr int SC_BYTES = DEC_BLOCK_TOKENS * 4;
   static constexpr int STAGE_BYTES = K_BYTES + VT_BYTES + 2 * SC_BYTES;
   static constexpr int STAGES = 3;
-  static constexpr int BQ_BYTES = 16 * D * 2;
+  static constexpr int BQ_BYTES = 16 * D * 2;  // per group: 16 fp16 columns or 32 int8 columns over d contraction steps
   static constexpr int BP_BYTES = 16 * DEC_BLOCK_TOKENS * 2;
-  // TMEM columns of one group: the operand tile (K rows, then V coordinates: d fp16 = d/2 columns), 16 columns of
-  // scores, 16 * DJ columns of values. The CTA owns all 512 columns of the SM.
+  // TMEM columns of one group, fp16 path: the operand tile (K rows, then V coordinates: d fp16 = d/2 columns), 16
+  // columns of scores, 16 * DJ columns of values. The CTA owns all 512 columns of the SM.
   static constexpr int GROUP_COLS = D;
   static constexpr int A_COL = 0;
   static constexpr int S_COL = D / 2;
@@ -65,15 +83,20 @@ struct DecLayout {
   static constexpr int NG = 512 / GROUP_COLS;  // groups per CTA: 4 at d = 128, 2 at d = 256
   static constexpr int COMPUTE_THREADS = NG * DEC_GROUP_THREADS;
   static constexpr int THREADS = COMPUTE_THREADS + NG * 32;  // + one control warp per group
-  static constexpr int GROUP_SMEM = BP_BYTES + STAGES * STAGE_BYTES;
-  static constexpr int SMEM_BYTES = DEC_HDR_BYTES + BQ_BYTES + NG * GROUP_SMEM;
+  static constexpr int GROUP_SMEM = BQ_BYTES + BP_BYTES + STAGES * STAGE_BYTES;
+  static constexpr int PRE_BYTES = DEC_NPRE * BQ_BYTES;  // the prepared query operands, shared by the groups
+  static constexpr int SMEM_BYTES = DEC_HDR_BYTES + PRE_BYTES + NG * GROUP_SMEM;
   // header offsets
   static constexpr int BAR_STRIDE = 96;  // per group: full[3], empty[3], s_bar, o_bar, k_ready, p_ready
-  static constexpr int OFF_TMEM = 384, OFF_NEXT = 388, OFF_SEG = 400, OFF_DESC = 448, OFF_ACCF = 544, OFF_QFAC = 576, OFF_RED = 640, OFF_WALK = 2176;
-  static constexpr int RED_STRIDE = 384;  // per group: 3 x [4 warps][8 heads] words
+  static constexpr int OFF_TMEM = 384, OFF_NEXT = 388, OFF_ACCF = 400, OFF_START = 448, OFF_DESC = 512, OFF_QFAC = 896, OFF_SEGID = 960, OFF_RED = 1024, OFF_PRE = 2560;
+  // OFF_PRE: count, [DEC_NPRE] (sequence, item), [DEC_NPRE] score factors, [DEC_NPRE][8] per-head maxima
+  static constexpr int DESC_STRIDE = STAGES * 32;  // per group
+  static constexpr int RED_STRIDE = 384;            // per group: 3 x [4 warps][8 heads] words
 };
 static_assert(DEC_BLOCK_TOKENS == 128, "the TMEM operand layout assumes 128-row blocks");
-static_assert(DecLayout<128>::OFF_RED + 4 * DecLayout<128>::RED_STRIDE <= DEC_HDR_BYTES, "header overflow");
+static_assert(DecLayout<128>::OFF_DESC + 4 * DecLayout<128>::DESC_STRIDE <= DecLayout<128>::OFF_QFAC, "header overflow");
+static_assert(DecLayout<128>::OFF_RED + 4 * DecLayout<128>::RED_STRIDE <= DecLayout<128>::OFF_PRE, "header overflow");
+static_assert(DecLayout<128>::OFF_PRE + 8 + 8 * DEC_NPRE + 4 * DEC_NPRE + 32 * DEC_NPRE <= DEC_HDR_BYTES, "header overflow");
 static_assert(DecLayout<128>::V_COL + 32 * DecLayout<128>::DJ <= DecLayout<128>::GROUP_COLS, "TMEM group overflow");
 static_assert(DecLayout<256>::V_COL + 32 * DecLayout<256>::DJ <= DecLayout<256>::GROUP_COLS, "TMEM group overflow");
 static_assert(DecLayout<128>::I8_O_COL + 32 * DecLayout<128>::DJ <= DecLayout<128>::GROUP_COLS, "TMEM group overflow");
@@ -81,8 +104,119 @@ static_assert(DecLayout<256>::I8_O_COL + 32 * DecLayout<256>::DJ <= DecLayout<25
 static_assert(DecLayout<128>::SMEM_BYTES <= 227 * 1024 && DecLayout<256>::SMEM_BYTES <= 227 * 1024, "shared memory overflow");
 static_assert((DecLayout<128>::THREADS + DecLayout<128>::THREADS / 32) * 4 <= DecLayout<128>::BP_BYTES, "set-up scratch must fit one B_P region");
 
+// Marks one partial slot of nh consecutive heads unused: (m, l) = (-inf, 0), acc = 0, argmax = -1. acc / ml / argmax
+// point at the slot of the first head; consecutive heads are S slots apart. Called by n_threads threads, this one t.
+// Kept out of line: it is rare, and the decode kernel's loops should stay small.
+static __device__ __noinline__ void dec_fill_slot(float* acc, float* ml, int32_t* argmax, int nh, int S, int D, int n_threads, int t) {
+  const int q = D / 4;
+  for (int idx = t; idx < nh * q; idx += n_threads) {
+    const int c4 = idx % q, h = idx / q;
+    *reinterpret_cast<float4*>(acc + (size_t)h * S * D + 4 * c4) = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  if (t < nh) {
+    ml[2 * (size_t)t * S] = -INFINITY;
+    ml[2 * (size_t)t * S + 1] = 0.f;
+    if (argmax) argmax[(size_t)t * S] = -1;
+  }
+}
+
+// The control warp's position in its work, and the block it has drawn. All lanes hold the same values.
+struct DecWalk {
+  int range_mode, grp, ng, ips, count;
+  // range mode: item (b, y) of the CTA's range the walk is in, blocks of its sequence, which piece of the item lies in
+  // this range, whether this group has staged a block of the segment
+  int b, y, nb, len, piece, touched;  // (len: cached rows of sequence b)
+  int sidx, n_pre;                    // ordinal of the segment in the range; segments below n_pre have a prepared query operand
+  long long item_g, g0, g_end;  // launch-wide index of block 0 of the item; the range [g0, g_end)
+  // unit mode: run k of item i is unit i * S + k; the walk is in run uk of item (ub, uy), at block ublk of [.., uhi)
+  long long n_units, unit_step, unit;
+  int ub, uy, uk, ublk, uhi, unew, ulen;
+};
+struct DecDrawn {
+  int kind;  // -1: nothing drawn, 0: a block, 1: the work has run out
+  int b, y, blk, slot, len, is_new, bqbuf;
+  size_t row0;  // first row of the block in the cache arrays
+};
+
+// Draws the group's next block. Range mode: the next block of the CTA's range from the shared counter; on the way the
+// walk passes over the segments of the range, and the partial slots this group owes -- its slot of a segment it got
+// no block of, the slots of an item beyond its last piece (those with index = grp mod ng) -- are marked unused. Unit
+// mode: the next block of the worker's current run, else of its next run with blocks (runs without blocks are marked
+// unused). Nothing is loaded from global memory unless the walk moves to another sequence (or the cache is paged).
+__device__ __forceinline__ void dec_draw(const DecodeParams& p, DecWalk& w, DecDrawn& d, int* next_s, int lane, int D, int with_argmax) {
+  constexpr int TB = DEC_BLOCK_TOKENS;
+  const int S = p.splits, B = p.batch;
+  auto len_of = [&](int b) { return max(0, min(p.seq_lens[b], p.t_cap)); };
+  auto warp_fill = [&](int b, int y, int slot) {
+    const int kvh = y / p.head_groups, hg = y - kvh * p.head_groups;
+    const int h0 = kvh * p.group + hg * DEC_HEADS, nh = min(DEC_HEADS, p.group - hg * DEC_HEADS);
+    const size_t o = ((size_t)b * p.n_q_heads + h0) * S + slot;
+    dec_fill_slot(p.part_acc + o * D, p.part_ml + 2 * o, with_argmax ? p.part_argmax + o : nullptr, nh, S, D, 32, lane);
+  };
+  if (w.range_mode) {
+    auto leave_segment = [&](bool item_ends) {
+      if (!w.touched) warp_fill(w.b, w.y, w.piece * w.ng + w.grp);
+      if (item_ends)
+        for (int sl = (w.piece + 1) * w.ng + w.grp; sl < S; sl += w.ng) warp_fill(w.b, w.y, sl);
+    };
+    auto next_item = [&]() {
+      w.item_g += w.nb;
+      w.touched = 0;
+      w.piece = 0;  // the next item starts inside this range
+      w.sidx++;
+      if (++w.y == w.ips) {
+        w.y = 0;
+        do { w.b++; w.len = (w.b < B) ? len_of(w.b) : 0; w.nb = (w.len + TB - 1) / TB; } while (w.b < B && w.nb == 0);
+      }
+    };
+    int n = 0;
+    if (lane == 0) n = atomicAdd(next_s, 1);
+    n = __shfl_sync(FULL, n, 0);
+    if (n >= w.count) {  // walk to the end of the range: the slots this group still owes
+      while (w.b < B && w.item_g + w.nb <= w.g_end) { leave_segment(true); next_item(); }
+      if (w.b < B && max(w.item_g, w.g0) < w.g_end) leave_segment(false);
+      w.b = B;
+      d.kind = 1;
+      return;
+    }
+    const long long g = w.g0 + n;
+    while (g >= w.item_g + w.nb) { leave_segment(true); next_item(); }
+    d.is_new = w.touched ? 0 : 1;
+    w.touched = 1;
+    d.b = w.b;
+    d.y = w.y;
+    d.blk = (int)(g - w.item_g);
+    d.slot = w.piece * w.ng + w.grp;
+    d.len = w.len;
+    d.bqbuf = w.sidx < w.n_pre ? w.sidx : -1;
+  } else {
+    while (w.ublk >= w.uhi) {  // the next run with blocks
+      if (w.unit >= w.n_units) { d.kind = 1; return; }
+      const long long item = w.unit / S;
+      const int k = (int)(w.unit - item * S);
+      w.unit += w.unit_step;
+      const int b = (int)(item / w.ips), y = (int)(item - (long long)b * w.ips);
+      const int len = len_of(b), nb = (len + TB - 1) / TB;
+      if (nb == 0) continue;  // an empty sequence: its slots were written during the set-up
+      const int cb = (nb + S - 1) / S, lo = k * cb, hi = min(nb, lo + cb);
+      if (lo >= hi) { warp_fill(b, y, k); continue; }
+      w.ub = b; w.uy = y; w.uk = k; w.ublk = lo; w.uhi = hi; w.unew = 1; w.ulen = len;
+    }
+    d.b = w.ub; d.y = w.uy; d.blk = w.ublk++; d.slot = w.uk; d.is_new = w.unew; d.len = w.ulen; d.bqbuf = -1;
+    w.unew = 0;
+  }
+  d.row0 = cache_row(p.pm, d.b, d.y / p.head_groups, (long long)d.blk * TB, p.status);
+  d.kind = 0;
+}
+
+// Where the CTA's range starts (thread 0, set-up).
+struct DecStart {
+  int b, y, len, piece;  // sequence, item within it, rows of the sequence, which piece of the item the range starts in
+  long long item_g;     // launch-wide index of block 0 of that item (<= the range's first block)
+};
+
 template <int D, bool ARGMAX, bool I8>
-__global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const __grid_constant__ DecodeParams p) {
   using L = DecLayout<D>;
   constexpr int DJ = L::DJ;
   constexpr int E = D / 32;
@@ -98,7 +232,6 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
   const int grp = control ? warp - NG * 4 : warp >> 2;  // group of this warp
   const int gt = tid & (DEC_GROUP_THREADS - 1);         // compute thread within its group = TMEM lane
   const int bar_id = 1 + grp;                           // named barrier of the group's compute threads
-  constexpr int HEADS_BAR = 8;                          // named barrier of the eight warps that rotate the query heads
 
   uint64_t* gbar = reinterpret_cast<uint64_t*>(smem + grp * L::BAR_STRIDE);
   uint64_t* full_bar = gbar;        // [stages] tile landed (or end marker)
@@ -108,147 +241,122 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
   uint64_t* k_ready = gbar + 8;     // K tile in TMEM (128 arrivals)
   uint64_t* p_ready = gbar + 9;     // V tile in TMEM + probabilities in smem (128 arrivals)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_TMEM);
-  int* next_s = reinterpret_cast<int*>(smem + L::OFF_NEXT);            // next block of the open segment
-  DecSegment* seg_s = reinterpret_cast<DecSegment*>(smem + L::OFF_SEG);
-  int2* desc = reinterpret_cast<int2*>(smem + L::OFF_DESC) + grp * NST;  // [stages] (first row, rows | end marker) of the staged block
+  int* next_s = reinterpret_cast<int*>(smem + L::OFF_NEXT);            // next block of the CTA's range
+  DecStart* start_s = reinterpret_cast<DecStart*>(smem + L::OFF_START);
+  DecDesc* desc = reinterpret_cast<DecDesc*>(smem + L::OFF_DESC + grp * L::DESC_STRIDE);  // [stages]
+  float* qtmp = reinterpret_cast<float*>(smem + L::OFF_QFAC + grp * 16);  // [4] per-warp maxima of |q~|
   float* red = reinterpret_cast<float*>(smem + L::OFF_RED + grp * L::RED_STRIDE);  // [4 warps][8 heads] cross-warp scratch
   float* red2 = red + 32;
   int* redi = reinterpret_cast<int*>(red2 + 32);
-  uint8_t* bq = smem + DEC_HDR_BYTES;                                  // B_Q: (n, i) MN-major, shared by the groups
-  uint8_t* bp = bq + L::BQ_BYTES + grp * L::GROUP_SMEM;                // B_P: (n, row) MN-major
+  int* n_pre_s = reinterpret_cast<int*>(smem + L::OFF_PRE);
+  int2* pre_tab = reinterpret_cast<int2*>(smem + L::OFF_PRE + 8);
+  float* pre_sfac = reinterpret_cast<float*>(smem + L::OFF_PRE + 8 + 8 * DEC_NPRE);
+  float* pre_hmax = pre_sfac + DEC_NPRE;
+  uint8_t* bq_pre = smem + DEC_HDR_BYTES;                                    // B_Q of the range's first segments
+  uint8_t* bq = bq_pre + L::PRE_BYTES + grp * L::GROUP_SMEM;                 // B_Q: (n, i) MN-major, this group's own
+  uint8_t* bp = bq + L::BQ_BYTES;                            // B_P: (n, row) MN-major
   uint8_t* stages = bp + L::BP_BYTES;
-  // Set-up scratch in group 0's B_P region: [THREADS] blocks per slice of the batch, then the per-warp maxima. It is
-  // last read before the first segment opens.
-  int* scan_s = reinterpret_cast<int*>(bq + L::BQ_BYTES);
+  // Set-up scratch in group 0's staging area: [THREADS] blocks per slice of the batch, then the per-warp maxima.
+  // It is last read before the barrier that ends the set-up.
+  int* scan_s = reinterpret_cast<int*>(smem + DEC_HDR_BYTES + L::PRE_BYTES + L::BQ_BYTES);
 
   const int S = p.splits;
   const int B = p.batch;
   const int ips = p.n_kv_heads * p.head_groups;  // items per sequence
+  const bool range_mode = S >= 2 * NG;
   auto len_of = [&](int b) { return max(0, min(p.seq_lens[b], p.t_cap)); };
   auto nb_of = [&](int b) { return (len_of(b) + TB - 1) / TB; };
-  // Unused partial slots [slot_lo, S) of the heads [h_lo, h_lo + n_h) of sequence b: (m, l) = (-inf, 0), acc = 0.
-  auto fill_slots = [&](int b, int h_lo, int n_h, int slot_lo, int n_threads, int t) {
-    const int n_slots = S - slot_lo;
-    if (n_slots <= 0) return;
-    for (int idx = t; idx < n_h * n_slots * D; idx += n_threads) {
-      const int c = idx % D, sl = (idx / D) % n_slots, h = idx / (D * n_slots);
-      p.part_acc[(((size_t)b * p.n_q_heads + h_lo + h) * S + slot_lo + sl) * D + c] = 0.f;
-    }
-    for (int idx = t; idx < n_h * n_slots; idx += n_threads) {
-      const int sl = idx % n_slots, h = idx / n_slots;
-      const size_t o = ((size_t)b * p.n_q_heads + h_lo + h) * S + slot_lo + sl;
-      p.part_ml[2 * o] = -INFINITY;
-      p.part_ml[2 * o + 1] = 0.f;
-      if (ARGMAX) p.part_argmax[o] = -1;
-    }
+  auto item_heads = [&](int y, int& kvh, int& h0, int& nh) {
+    kvh = y / p.head_groups;
+    const int hg = y - kvh * p.head_groups;
+    h0 = kvh * p.group + hg * DEC_HEADS;
+    nh = min(DEC_HEADS, p.group - hg * DEC_HEADS);
+  };
+  // Partial slot `slot` of the heads of item (b, y) marked unused: (m, l) = (-inf, 0), acc = 0. n_threads threads, this one t.
+  auto fill_slot = [&](int b, int y, int slot, int n_threads, int t) {
+    int kvh, h0, nh;
+    item_heads(y, kvh, h0, nh);
+    const size_t o = ((size_t)b * p.n_q_heads + h0) * S + slot;
+    dec_fill_slot(p.part_acc + o * D, p.part_ml + 2 * o, ARGMAX ? p.part_argmax + o : nullptr, nh, S, D, n_threads, t);
   };
 
   grid_dependency_wait();  // nothing written by an earlier kernel (lengths, queries, cache rows) is read above this line
 
-  // ---------------------------------------------------------------- the block sequence of the launch and this CTA's range
-  const int per_thread = (B + L::THREADS - 1) / L::THREADS;
-  {
-    int sum = 0, mx = 0;
-    for (int b = tid * per_thread; b < min(B, (tid + 1) * per_thread); b++) {
-      const int n = nb_of(b);
-      sum += n;
-      mx = max(mx, n);
-    }
-    scan_s[tid] = sum;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(FULL, mx, o));
-    if (lane == 0) scan_s[L::THREADS + warp] = mx;
-  }
-  // sequences without cached rows belong to no range: CTA c defines the partial slots of sequences c, c + grid, ...
+  // sequences without cached rows belong to no range and no unit: CTA c defines their partial slots for sequences c, c + grid, ...
   for (int b = blockIdx.x; b < B; b += gridDim.x)
-    if (len_of(b) == 0) fill_slots(b, 0, p.n_q_heads, 0, L::THREADS, tid);
-  __syncthreads();
-  long long n_total;
-  int nb_max = 0;
-  {
-    int v = 0;
-    for (int i = lane; i < L::THREADS; i += 32) v += scan_s[i];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
-    n_total = (long long)v * ips;
-    for (int i = 0; i < L::THREADS / 32; i++) nb_max = max(nb_max, scan_s[L::THREADS + i]);
-  }
-  const bool whole_items = (S == 1);  // one slot per head: an item cannot be shared between CTAs
-  long long per = (n_total + gridDim.x - 1) / gridDim.x;
-  if (!whole_items) per = max(per, (long long)((nb_max - 1) / (S - 1) + 1));  // an item then spans at most S ranges
-  per = max(per, 1ll);
-  const long long g0 = (long long)blockIdx.x * per;
-  if (n_total == 0 || (!whole_items && g0 >= n_total) || (whole_items && (long long)blockIdx.x >= (long long)B * ips)) return;
+    if (len_of(b) == 0)
+      for (int y = 0; y < ips; y++)
+        for (int sl = 0; sl < S; sl++) fill_slot(b, y, sl, L::THREADS, tid);
 
-  // Thread 0 walks the range segment by segment; the walk lives in shared memory between segments. Range mode:
-  // position (b, y, blk) and `left` blocks to go; whole-item mode: items blockIdx.x, blockIdx.x + grid, ... with rows.
-  DecWalk* walk_s = reinterpret_cast<DecWalk*>(smem + L::OFF_WALK);
-  auto next_item_with_rows = [&](DecWalk& w) {  // whole-item mode: settle on the next item that has rows, or b = B
-    for (;; w.item += gridDim.x) {
-      if (w.item >= (long long)B * ips) { w.b = B; w.nb = 0; return; }
-      w.b = (int)(w.item / ips);
-      w.y = (int)(w.item % ips);
-      w.nb = nb_of(w.b);
-      w.blk = 0;
-      if (w.nb > 0) return;
+  // ---------------------------------------------------------------- range mode: the block sequence of the launch and this CTA's range
+  long long per = 1, g0 = 0;
+  int count = 0;  // blocks of this CTA's range
+  if (range_mode) {
+    const int per_thread = (B + L::THREADS - 1) / L::THREADS;
+    {
+      int sum = 0, mx = 0;
+      for (int b = tid * per_thread; b < min(B, (tid + 1) * per_thread); b++) {
+        const int n = nb_of(b);
+        sum += n;
+        mx = max(mx, n);
+      }
+      scan_s[tid] = sum;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(FULL, mx, o));
+      if (lane == 0) scan_s[L::THREADS + warp] = mx;
     }
-  };
-  {
-    DecWalk w = {0, 0, 0, 0, 0, g0, (long long)blockIdx.x};
-    if (whole_items) {
-      next_item_with_rows(w);  // every thread: the CTA leaves together when none of its items has rows
-      if (w.b >= B) return;
-    } else if (tid == 0) {
-      long long before = 0;  // blocks (per item column) of the sequences before w.b
+    __syncthreads();
+    long long n_total;
+    int nb_max = 0;
+    {
+      int v = 0;
+      for (int i = lane; i < L::THREADS; i += 32) v += scan_s[i];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+      n_total = (long long)v * ips;
+      for (int i = 0; i < L::THREADS / 32; i++) nb_max = max(nb_max, scan_s[L::THREADS + i]);
+    }
+    per = (n_total + gridDim.x - 1) / gridDim.x;
+    per = max(per, (long long)((nb_max - 1) / (S / NG - 1) + 1));  // an item then spans at most S / NG ranges
+    per = max(per, 1ll);
+    g0 = (long long)blockIdx.x * per;
+    if (g0 >= n_total) return;
+    count = (int)min(per, n_total - g0);
+    if (tid == 0) {  // the item that holds block g0
+      long long before = 0;  // blocks (per item column) of the sequences before b
       int t = 0;
       while (t < L::THREADS - 1 && (before + scan_s[t]) * ips <= g0) { before += scan_s[t]; t++; }
-      w.b = t * per_thread;
-      w.nb = (w.b < B) ? nb_of(w.b) : 0;
-      while (w.b < B - 1 && (before + w.nb) * ips <= g0) { before += w.nb; w.b++; w.nb = nb_of(w.b); }
+      int b = t * per_thread;
+      int nb = (b < B) ? nb_of(b) : 0;
+      while (b < B - 1 && (before + nb) * ips <= g0) { before += nb; b++; nb = nb_of(b); }
       const long long r = g0 - before * ips;  // offset inside sequence b's blocks (nb per item, ips items)
-      w.y = (int)(r / w.nb);
-      w.blk = (int)(r % w.nb);
-      w.left = min(per, n_total - g0);
-    }
-    if (tid == 0) *walk_s = w;
-  }
-  // thread 0: describe the next segment in seg_s, open its block counter, advance the walk
-  auto open_segment = [&]() {
-    DecWalk w = *walk_s;
-    const int take = whole_items ? w.nb : (int)min((long long)(w.nb - w.blk), w.left);
-    DecSegment sg;
-    sg.b = w.b;
-    sg.y = w.y;
-    sg.blk0 = w.blk;
-    sg.blk1 = w.blk + take;
-    sg.slot = whole_items ? 0 : (int)((long long)blockIdx.x - (w.g - w.blk) / per);
-    sg.len = len_of(w.b);
-    const bool item_end = (sg.blk1 == w.nb);
-    w.g += take;
-    w.left -= take;
-    bool cta_end;
-    if (whole_items) {
-      w.item += gridDim.x;
-      next_item_with_rows(w);
-      cta_end = (w.b >= B);
-    } else {
-      if (item_end) {
-        w.blk = 0;
-        if (++w.y == ips) {
-          w.y = 0;
-          do { w.b++; w.nb = (w.b < B) ? nb_of(w.b) : 0; } while (w.b < B && w.nb == 0);
+      DecStart s0;
+      s0.b = b;
+      s0.len = (b < B) ? len_of(b) : 0;
+      s0.y = (int)(r / nb);
+      s0.item_g = before * ips + (long long)s0.y * nb;
+      s0.piece = (int)((long long)blockIdx.x - s0.item_g / per);  // CTAs between the item's first block and this range
+      *start_s = s0;
+      *next_s = 0;
+      // the range's first segments: their query operands are prepared once for all groups
+      int np = 0;
+      long long item_g = s0.item_g;
+      int y = s0.y;
+      while (np < DEC_NPRE && b < B && max(item_g, g0) < g0 + count) {
+        pre_tab[np++] = make_int2(b, y);
+        item_g += nb;
+        if (++y == ips) {
+          y = 0;
+          do { b++; nb = (b < B) ? nb_of(b) : 0; } while (b < B && nb == 0);
         }
-      } else {
-        w.blk = sg.blk1;
       }
-      cta_end = (w.left <= 0) || (w.b >= B);
+      *n_pre_s = np;
     }
-    sg.flags = (item_end ? 1 : 0) | (cta_end ? 2 : 0);
-    sg.pad = 0;
-    *seg_s = sg;
-    *next_s = sg.blk0;
-    *walk_s = w;
-  };
+  } else {
+    // unit mode: worker w = grp * grid + CTA takes units w, w + NG * grid, ...; a CTA none of whose groups has a unit leaves
+    if ((long long)blockIdx.x >= (long long)B * ips * S) return;
+    if (tid == 0) *n_pre_s = 0;
+  }
 
   // ---------------------------------------------------------------- set-up: barriers, TMEM
   if (control && elect_one()) {  // every control warp initialises the barriers of its group
@@ -266,215 +374,361 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
   }
   tc_fence_before();
-  __syncthreads();
+  __syncthreads();  // the last CTA-wide barrier before the end of the kernel
   tc_fence_after();
   const uint32_t tmem_base = tmem_slot[0];
   const uint32_t tmem_g = tmem_base + (uint32_t)(grp * L::GROUP_COLS);        // this group's columns
   const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;                // this warp's 32 TMEM lanes
-  bool failed = false;  // a bounded wait gave up; assumed to hit all threads of a group alike (they wait on the same barriers)
-  int it = 0;           // staged slots of this group consumed so far (tile pipeline phases), end markers included
-  int nbk = 0;          // blocks this group has processed (phases of k_ready, s_bar, p_ready, o_bar)
+  bool failed = false;  // a bounded wait gave up; every later wait of this thread is skipped
 
-  for (;;) {
-    // ================================================================ one segment: blocks [blk0, blk1) of one item
-    if (tid == 0) open_segment();
-    __syncthreads();  // segment published; the previous segment's merge has finished reading the staging buffers
-    if (!control && warp < DEC_HEADS) {
-      // ---- d1: q~ = R q of head `warp`, written as the operand B_Q (shared by the groups)
-      const int b = seg_s->b;
-      const int kvh = seg_s->y / p.head_groups;
-      const int hg = seg_s->y - kvh * p.head_groups;
-      const int h0 = kvh * p.group + hg * DEC_HEADS;
-      const int nh = min(DEC_HEADS, p.group - hg * DEC_HEADS);
-      const int hh = warp;
-      float v[E];
-      if (hh < nh) {
+  if (control) {
+    // ================================================================ control warp of group grp: walks the work, fetches blocks, issues MMAs.
+    // All 32 lanes run the loop and the waits (the walk is uniform over the warp); an elected lane issues.
+    const uint32_t bq_addr = smem_u32(bq), bp_addr = smem_u32(bp);
+    // operand descriptors of the first k-step, built before the waits: a k-step further on adds its byte offset / 16
+    const uint64_t bq_desc_own = smem_desc_mn(bq_addr, 128, (D / 8) * 128), bp_desc0 = smem_desc_mn(bp_addr, 128, (TB / 8) * 128);
+    const uint64_t bq_desc_pre = smem_desc_mn(smem_u32(bq_pre), 128, (D / 8) * 128);
+    int it = 0;         // staged slots consumed so far (tile pipeline phases), the end marker included
+    int it_issue = 0;   // slots staged so far
+    int nbk = 0;        // blocks processed (phases of k_ready, s_bar, p_ready, o_bar)
+    bool ended = false; // the work ran out and the end marker has been staged
+    // The walk over the CTA's work lives in a struct and advances in an out-of-line function (dec_draw).
+    DecWalk wk;
+    wk.range_mode = range_mode ? 1 : 0;
+    wk.grp = grp;
+    wk.ng = NG;
+    wk.ips = ips;
+    wk.count = count;
+    wk.g0 = g0;
+    wk.g_end = g0 + count;
+    wk.touched = 0;
+    wk.sidx = 0;
+    wk.n_pre = *n_pre_s;
+    if (range_mode) { wk.b = start_s->b; wk.y = start_s->y; wk.len = start_s->len; wk.nb = (wk.len + TB - 1) / TB; wk.piece = start_s->piece; wk.item_g = start_s->item_g; }
+    else { wk.b = wk.y = wk.nb = wk.len = wk.piece = 0; wk.item_g = 0; }
+    wk.n_units = (long long)B * ips * S;
+    wk.unit_step = (long long)NG * gridDim.x;
+    wk.unit = (long long)grp * gridDim.x + blockIdx.x;
+    wk.ub = wk.uy = wk.uk = wk.ublk = wk.uhi = wk.unew = wk.ulen = 0;
+    // The next block is drawn (shared counter; with a paged cache also its block-table entry, a load from global
+    // memory) while the compute warps are busy with the softmax of the current one, and staged after the value MMAs.
+    DecDrawn dr;
+    dr.kind = -1;
+    auto draw = [&]() { dec_draw(p, wk, dr, next_s, lane, D, ARGMAX ? 1 : 0); };
+    auto stage_next = [&]() {  // the drawn (or next) block into slot it_issue, or the end marker
+      const int st = it_issue % NST;
+      if (it_issue >= NST && !failed)  // the slot's previous occupant has been consumed
+        failed = !mbar_wait_bounded(&empty_bar[st], (uint32_t)(it_issue / NST - 1) & 1u, DEC_WAIT_LIMIT);
+      if (dr.kind < 0 && !failed) draw();
+      if (dr.kind == 0 && !failed) {
+        const int r0 = dr.blk * TB;
+        const int n = min(TB, dr.len - r0);
+        if (elect_one()) {
+          DecDesc dd;
+          dd.n = n; dd.flags = dr.is_new; dd.r0 = r0; dd.slot = dr.slot; dd.b = dr.b; dd.y = dr.y; dd.len = dr.len; dd.bqbuf = dr.bqbuf;
+          desc[st] = dd;
+          const uint32_t sc_bytes = p.scale_f16 ? (uint32_t)(((n + 7) & ~7) * 2) : (uint32_t)(((n + 3) & ~3) * 4);  // whole 16-byte pieces
+          uint8_t* sp = stages + st * L::STAGE_BYTES;
+          const size_t row0 = dr.row0;
+          fence_proxy_async();
+          mbar_expect_tx(&full_bar[st], (uint32_t)(n * L::ROWB + L::VT_BYTES) + 2 * sc_bytes);  // also publishes desc[st]
+          bulk_g2s(sp, p.k_codes + row0 * L::ROWB, (uint32_t)(n * L::ROWB), &full_bar[st]);
+          bulk_g2s(sp + L::K_BYTES, p.v_codes + row0 * L::ROWB, (uint32_t)L::VT_BYTES, &full_bar[st]);  // whole 128-row V block
+          bulk_g2s(sp + L::K_BYTES + L::VT_BYTES, reinterpret_cast<const uint8_t*>(p.k_scales) + row0 * (p.scale_f16 ? 2 : 4), sc_bytes, &full_bar[st]);
+          bulk_g2s(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES, reinterpret_cast<const uint8_t*>(p.v_scales) + row0 * (p.scale_f16 ? 2 : 4), sc_bytes, &full_bar[st]);
+        }
+        dr.kind = -1;
+      } else {
+        ended = true;
+        if (elect_one()) {
+          desc[st].n = -1;  // end marker: no tile, the group closes what it has open and leaves
+          mbar_arrive(&full_bar[st]);
+        }
+      }
+      __syncwarp();
+      it_issue++;
+    };
+    for (;;) {
+#pragma unroll 1
+      while (!ended && it_issue - it < NST) stage_next();  // keep the pipeline full (at the start: tiles in flight while the compute warps open their first segment)
+      if (ended && it == it_issue - 1) { it++; break; }  // slot `it` holds the end marker
+      // scores of the block in slot `it`: S = A_K * B_Q^T once all 128 rows are in TMEM (and B_Q of its segment is complete)
+      if (!failed) failed = !mbar_wait_bounded(k_ready, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
+      if (failed) break;
+      tc_fence_after();
+      const int bqbuf = desc[it % NST].bqbuf;  // the query operand of the block's segment (the start address field counts 16-byte units)
+      const uint64_t bq_desc0 = bqbuf < 0 ? bq_desc_own : bq_desc_pre + (uint64_t)(bqbuf * (L::BQ_BYTES / 16));
+      if (elect_one()) {
+        if constexpr (I8) {
+#pragma unroll
+          for (int kk = 0; kk < D / 32; kk++)
+            tc_mma_i8(tmem_g + L::I8_S_COL, tmem_g + L::I8_K_COL + 8 * kk, bq_desc0 + 32 * kk, DEC_IDESC_I8_SS, kk > 0);
+        } else {
+#pragma unroll
+          for (int kk = 0; kk < D / 16; kk++)
+            tc_mma_f16(tmem_g + L::S_COL, tmem_g + L::A_COL + 8 * kk, bq_desc0 + 16 * kk, DEC_IDESC, kk > 0);
+        }
+        tc_commit(s_bar);
+      }
+      __syncwarp();
+      if (!ended && dr.kind < 0) draw();
+      // values: O = A_V * B_P^T once the V tile is in TMEM and the probabilities are in shared memory
+      failed = !mbar_wait_bounded(p_ready, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
+      if (failed) break;
+      tc_fence_after();
+      const bool keep_values = I8 && *reinterpret_cast<volatile int*>(smem + L::OFF_ACCF + 4 * grp) != 0;
+      if (elect_one()) {
+        if constexpr (I8) {
+#pragma unroll
+          for (int j = 0; j < DJ; j++)
+#pragma unroll
+            for (int kk = 0; kk < TB / 32; kk++)  // the values stay in TMEM (int32) over the blocks until the compute threads read them
+              tc_mma_i8(tmem_g + L::I8_O_COL + 32 * j, tmem_g + L::I8_V_COL + 32 * j + 8 * kk, bp_desc0 + 32 * kk, DEC_IDESC_I8_SU,
+                        (kk > 0) || keep_values);
+        } else {
+#pragma unroll
+          for (int j = 0; j < DJ; j++)
+#pragma unroll
+            for (int kk = 0; kk < TB / 16; kk++)
+              tc_mma_f16(tmem_g + L::O_COL + 16 * j,  // rows 0..63 of the V tile sit in V_COL, rows 64..127 in the operand columns
+                         tmem_g + (kk < 4 ? L::V_COL + 32 * j + 8 * kk : L::A_COL + 64 * j + 8 * (kk - 4)),
+                         bp_desc0 + 16 * kk, DEC_IDESC, kk > 0);
+        }
+        tc_commit(o_bar);
+      }
+      __syncwarp();
+      it++;
+      nbk++;  // the compute threads released the slot when they signalled p_ready: the loop stages the next block into it
+    }
+    if (failed) {
+      // Give-up path. Tiles staged and not consumed may still be landing: wait (bounded) for each of them, so that no
+      // bulk copy targets this CTA's shared memory after it has left. Tensor-core work in flight is covered by the
+      // fence before the TMEM release at the end of the kernel.
+      for (int s = it; s < it_issue; s++) mbar_wait_bounded(&full_bar[s % NST], (uint32_t)(s / NST) & 1u, DEC_WAIT_LIMIT);
+    }
+  }
+  if (!control) {
+    // ================================================================ compute warps of group grp
+    const uint32_t lut_lo0 = p.lut_lo[0], lut_lo1 = p.lut_lo[1], lut_hi0 = p.lut_hi[0], lut_hi1 = p.lut_hi[1];
+    const float inv_root_d = rsqrtf((float)D);
+    const float kfac = p.sm_scale * LOG2E * inv_root_d;  // scores in log2 units: z2 = S_raw * scale_K * kfac
+    const float vfac = inv_root_d;
+    float acc[DJ][8];  // thread c: coordinates c (+128), 8 heads
+    float m_run[8], l_run[8], best_v[8];
+    int best_i[8];
+    float sfac = 0.f;  // integer path: score digits -> log2-domain score per unit K scale (set when a segment is opened)
+    int it = 0;        // staged slots of this group consumed so far (tile pipeline phases), the end marker included
+    int nbk = 0;       // blocks this group has processed (phases of k_ready, s_bar, p_ready, o_bar)
+    int* seg_id = reinterpret_cast<int*>(smem + L::OFF_SEGID + 16 * grp);  // the open segment: (sequence, item, slot); kept in shared memory between open and close
+
+    // ---- d1 (App. A): q~ = R q of one head, as the lane's E coordinates (lane l holds l E .. l E + E - 1), times 1/sqrt(d)
+    auto rotate_head = [&](int b, int kvh, int h_abs, bool present, float (&v)[E]) {
+      if (present) {
         float M[E / 4][4][4];
         const float* qb = p.rot + ((size_t)kvh * (D / 4) + (size_t)lane * (E / 4)) * 8;
 #pragma unroll
         for (int j = 0; j < E / 4; j++) so4_matrix<float>(qb + 8 * j, M[j]);
-        const __half* src = p.q + ((size_t)b * p.n_q_heads + h0 + hh) * D + lane * E;
+        const __half* src = p.q + ((size_t)b * p.n_q_heads + h_abs) * D + lane * E;
 #pragma unroll
         for (int e = 0; e < E; e++) v[e] = __half2float(src[e]);
         wht_warp<float, E>(v, lane);
         so4_apply<float, E, false>(M, v);
+#pragma unroll
+        for (int e = 0; e < E; e++) v[e] *= inv_root_d;
       } else {
 #pragma unroll
         for (int e = 0; e < E; e++) v[e] = 0.f;
       }
-      const float inv_root_d = rsqrtf((float)D);
+    };
+    auto abs_max = [&](const float (&v)[E]) {
+      float m = 0.f;
+#pragma unroll
+      for (int e = 0; e < E; e++) m = fmaxf(m, fabsf(v[e]));
+      return warp_max(m);
+    };
+    // Column block hh (one head) of the operand B_Q in buffer `dst`. Integer path: q~ as three balanced base-128 digits
+    // (int8) of round(q~ * (2^20 - 1) / qmax), qmax = max |q~| over the item's heads: one scale for all heads, so that
+    // the score read-back needs a single factor. (Two base-256 digits would halve the read-back, but 16 bits are not
+    // enough for lse at the logit magnitudes of outlier rows.) fp16 path: q~ as hi + lo.
+    auto write_operand = [&](uint8_t* dst, int hh, const float (&v)[E], float qmax) {
       if constexpr (I8) {
-        // q~ as three balanced base-128 digits (int8) of round(q~ * (2^20 - 1) / qmax), qmax = max |q~| over the item's
-        // heads: one scale for all heads, so that the score read-back needs a single factor. (Two base-256 digits would
-        // halve the read-back, but 16 bits are not enough for lse at the logit magnitudes of outlier rows.)
-        float qmax = 0.f;
-#pragma unroll
-        for (int e = 0; e < E; e++) qmax = fmaxf(qmax, fabsf(v[e] * inv_root_d));
-        qmax = warp_max(qmax);
-        float* qtmp = reinterpret_cast<float*>(smem + L::OFF_QFAC);  // [8] per-head maxima, then [8] = the common factor
-        if (lane == 0) qtmp[hh] = qmax;
-        cta_bar_sync_n(HEADS_BAR, DEC_HEADS * 32);
-#pragma unroll
-        for (int h2 = 0; h2 < DEC_HEADS; h2++) qmax = fmaxf(qmax, qtmp[h2]);
         const float qs = qmax > 0.f ? 1048575.0f / qmax : 0.f;
 #pragma unroll
         for (int e = 0; e < E; e++) {
-          const int Q = __float2int_rn(v[e] * inv_root_d * qs);
+          const int Q = __float2int_rn(v[e] * qs);
           const int d2 = (Q + 8192) >> 14;
           const int r = Q - (d2 << 14);
           const int d1 = (r + 64) >> 7;
           const int d0 = r - (d1 << 7);
           const int i = lane * E + e;  // contraction index = rotated coordinate; column n = 4 * head + digit
           const uint32_t word = (uint32_t)(d0 & 0xff) | ((uint32_t)(d1 & 0xff) << 8) | ((uint32_t)(d2 & 0xff) << 16);
-          *reinterpret_cast<uint32_t*>(bq + 4 * (hh & 3) + (hh >> 2) * ((D / 8) * 128) + (i & 7) * 16 + (i >> 3) * 128) = word;
+          *reinterpret_cast<uint32_t*>(dst + 4 * (hh & 3) + (hh >> 2) * ((D / 8) * 128) + (i & 7) * 16 + (i >> 3) * 128) = word;
         }
-        if (hh == 0 && lane == 0)  // digits -> log2-domain score per unit K scale
-          qtmp[8] = (qmax * (1.0f / 1048575.0f)) * p.delta * (p.sm_scale * LOG2E * inv_root_d);
       } else {
 #pragma unroll
         for (int e = 0; e < E; e++) {
-          const float x = v[e] * inv_root_d;
+          const float x = v[e];
           const __half xh = __float2half_rn(x);
           const __half xl = __float2half_rn(x - __half2float(xh));
           const int i = lane * E + e;  // contraction index = rotated coordinate
           const int off = (i & 7) * 16 + (i >> 3) * 128;
-          *reinterpret_cast<__half*>(bq + hh * 2 + off) = xh;                  // n = head (hi part)
-          *reinterpret_cast<__half*>(bq + hh * 2 + (D / 8) * 128 + off) = xl;  // n = 8 + head (lo part)
+          *reinterpret_cast<__half*>(dst + hh * 2 + off) = xh;                  // n = head (hi part)
+          *reinterpret_cast<__half*>(dst + hh * 2 + (D / 8) * 128 + off) = xl;  // n = 8 + head (lo part)
         }
       }
-      fence_proxy_async();  // B_Q is written through the generic proxy and read by the tensor core through the async proxy
-    }
-    // (the control warps stage their first tiles below before they join the barrier that completes B_Q)
-    if (control) {
-      // ================================================================ control warp of group grp: fetches blocks, issues MMAs.
-      // All 32 lanes run the loop and the waits; an elected lane issues.
-      const int blk1 = seg_s->blk1, len = seg_s->len;
-      const int seg_b = seg_s->b, seg_kvh = seg_s->y / p.head_groups;
-      const uint32_t bq_addr = smem_u32(bq), bp_addr = smem_u32(bp);
-      // operand descriptors of the first k-step, built before the waits: a k-step further on adds its byte offset / 16
-      const uint64_t bq_desc0 = smem_desc_mn(bq_addr, 128, (D / 8) * 128), bp_desc0 = smem_desc_mn(bp_addr, 128, (TB / 8) * 128);
-      bool ended = false;   // the segment's counter ran out and the end marker has been staged
-      int it_issue = it;    // slots staged so far (the pipeline is empty between segments)
-      // The next block is drawn (shared counter; with a paged cache also its block-table entry, a load from global
-      // memory) while the compute warps are busy with the softmax of the current one, and staged after the value MMAs.
-      int drawn_j = -1;        // block drawn ahead of its staging, -1: none
-      size_t drawn_row0 = 0;   // its first row in the cache arrays
-      auto draw = [&]() {
-        int j = 0;
-        if (lane == 0) j = atomicAdd(next_s, 1);
-        drawn_j = __shfl_sync(FULL, j, 0);
-        if (drawn_j < blk1) drawn_row0 = cache_row(p.pm, seg_b, seg_kvh, drawn_j * TB, p.status);
-      };
-      auto stage_next = [&]() {  // the next block of the segment into slot it_issue, or the end marker
-        const int st = it_issue % NST;
-        if (it_issue >= NST && !failed)  // the slot's previous occupant has been consumed
-          failed = !mbar_wait_bounded(&empty_bar[st], (uint32_t)(it_issue / NST - 1) & 1u, DEC_WAIT_LIMIT);
-        if (drawn_j < 0) draw();
-        const int j = drawn_j;
-        const size_t row0 = drawn_row0;
-        drawn_j = -1;
-        if (j < blk1) {
-          const int r0 = j * TB;
-          const int n = min(TB, len - r0);
-          if (elect_one()) {
-            desc[st] = make_int2(r0, n);
-            const uint32_t sc_bytes = p.scale_f16 ? (uint32_t)(((n + 7) & ~7) * 2) : (uint32_t)(((n + 3) & ~3) * 4);  // whole 16-byte pieces
-            uint8_t* sp = stages + st * L::STAGE_BYTES;
-            fence_proxy_async();
-            mbar_expect_tx(&full_bar[st], (uint32_t)(n * L::ROWB + L::VT_BYTES) + 2 * sc_bytes);  // also publishes desc[st]
-            bulk_g2s(sp, p.k_codes + row0 * L::ROWB, (uint32_t)(n * L::ROWB), &full_bar[st]);
-            bulk_g2s(sp + L::K_BYTES, p.v_codes + row0 * L::ROWB, (uint32_t)L::VT_BYTES, &full_bar[st]);  // whole 128-row V block
-            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES, reinterpret_cast<const uint8_t*>(p.k_scales) + row0 * (p.scale_f16 ? 2 : 4), sc_bytes, &full_bar[st]);
-            bulk_g2s(sp + L::K_BYTES + L::VT_BYTES + L::SC_BYTES, reinterpret_cast<const uint8_t*>(p.v_scales) + row0 * (p.scale_f16 ? 2 : 4), sc_bytes, &full_bar[st]);
-          }
-        } else {
-          ended = true;
-          if (elect_one()) {
-            desc[st] = make_int2(0, -1);  // end marker: no tile, the group closes its part of the segment
-            mbar_arrive(&full_bar[st]);
+    };
+    auto score_factor = [&](float qmax) { return (qmax * (1.0f / 1048575.0f)) * p.delta * kfac; };  // digits -> log2-domain score per unit K scale
+
+    // ---- the operands of the range's first segments, built once for all groups of the CTA by all compute warps
+    // (a group that meets a later segment, or works in unit mode, builds the operand itself in open_segment)
+    {
+      const int n_pre = *n_pre_s;
+      if (n_pre > 0) {
+        constexpr int NCW = NG * 4, JOBS = (8 * DEC_NPRE + NCW - 1) / NCW;
+        float v[JOBS][E];
+#pragma unroll
+        for (int t = 0; t < JOBS; t++) {
+          const int job = warp + t * NCW, sg = job >> 3, hh = job & 7;
+          int kvh = 0, h0 = 0, nh = 0, b = 0;
+          if (sg < n_pre) { b = pre_tab[sg].x; item_heads(pre_tab[sg].y, kvh, h0, nh); }
+          rotate_head(b, kvh, h0 + hh, sg < n_pre && hh < nh, v[t]);
+          if (I8 && sg < DEC_NPRE) {
+            const float m = abs_max(v[t]);
+            if (lane == 0) pre_hmax[sg * 8 + hh] = m;
           }
         }
-        __syncwarp();
-        it_issue++;
-      };
-      while (!ended && it_issue - it < NST) stage_next();  // tiles in flight while q~ is being rotated
-      cta_bar_sync();  // B_Q complete
-      for (;;) {
-        if (it == it_issue) stage_next();  // nothing staged ahead (end of a segment): draw now
-        if (ended && it == it_issue - 1) { it++; break; }  // slot `it` holds the end marker
-        // scores of the block in slot `it`: S = A_K * B_Q^T once all 128 rows are in TMEM
-        if (!failed) failed = !mbar_wait_bounded(k_ready, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
-        tc_fence_after();
-        if (elect_one()) {
-          if constexpr (I8) {
+        if (I8) cta_bar_sync_n(DEC_PRE_BAR, L::COMPUTE_THREADS);
 #pragma unroll
-            for (int kk = 0; kk < D / 32; kk++)
-              tc_mma_i8(tmem_g + L::I8_S_COL, tmem_g + L::I8_K_COL + 8 * kk, bq_desc0 + 32 * kk, DEC_IDESC_I8_SS, kk > 0);
-          } else {
+        for (int t = 0; t < JOBS; t++) {
+          const int job = warp + t * NCW, sg = job >> 3, hh = job & 7;
+          if (sg < n_pre) {
+            float qmax = 0.f;
+            if (I8) {
 #pragma unroll
-            for (int kk = 0; kk < D / 16; kk++)
-              tc_mma_f16(tmem_g + L::S_COL, tmem_g + L::A_COL + 8 * kk, bq_desc0 + 16 * kk, DEC_IDESC, kk > 0);
+              for (int h2 = 0; h2 < 8; h2++) qmax = fmaxf(qmax, pre_hmax[sg * 8 + h2]);
+              if (hh == 0 && lane == 0) pre_sfac[sg] = score_factor(qmax);
+            }
+            write_operand(bq_pre + sg * L::BQ_BYTES, hh, v[t], qmax);
           }
-          tc_commit(s_bar);
         }
-        __syncwarp();
-        if (!ended) draw();
-        // values: O = A_V * B_P^T once the V tile is in TMEM and the probabilities are in shared memory
-        if (!failed) failed = !mbar_wait_bounded(p_ready, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
-        tc_fence_after();
-        const bool keep_values = I8 && *reinterpret_cast<volatile int*>(smem + L::OFF_ACCF + 4 * grp) != 0;
-        if (elect_one()) {
-          if constexpr (I8) {
-#pragma unroll
-            for (int j = 0; j < DJ; j++)
-#pragma unroll
-              for (int kk = 0; kk < TB / 32; kk++)  // the values stay in TMEM (int32) over the blocks until the compute threads read them
-                tc_mma_i8(tmem_g + L::I8_O_COL + 32 * j, tmem_g + L::I8_V_COL + 32 * j + 8 * kk, bp_desc0 + 32 * kk, DEC_IDESC_I8_SU,
-                          (kk > 0) || keep_values);
-          } else {
-#pragma unroll
-            for (int j = 0; j < DJ; j++)
-#pragma unroll
-              for (int kk = 0; kk < TB / 16; kk++)
-                tc_mma_f16(tmem_g + L::O_COL + 16 * j,  // rows 0..63 of the V tile sit in V_COL, rows 64..127 in the operand columns
-                           tmem_g + (kk < 4 ? L::V_COL + 32 * j + 8 * kk : L::A_COL + 64 * j + 8 * (kk - 4)),
-                           bp_desc0 + 16 * kk, DEC_IDESC, kk > 0);
-          }
-          tc_commit(o_bar);
-        }
-        __syncwarp();
-        it++;
-        nbk++;
-        // the compute threads released the slot when they signalled p_ready
-        if (!ended) stage_next();
+        fence_proxy_async();  // the operands are written through the generic proxy and read by the tensor core through the async proxy
+        cta_bar_sync_n(DEC_PRE_BAR, L::COMPUTE_THREADS);
       }
     }
-    float* gacc = reinterpret_cast<float*>(stages);                 // group partial for the merge: acc [DJ][8][128]
-    float* gml = gacc + DJ * 8 * DEC_GROUP_THREADS;                 // then per head: reference, l, exact maximum, its row
-    if (!control) {
-      cta_bar_sync();  // B_Q complete
-      // ================================================================ compute warps of group grp
-      const uint32_t lut_lo0 = p.lut_lo[0], lut_lo1 = p.lut_lo[1], lut_hi0 = p.lut_hi[0], lut_hi1 = p.lut_hi[1];
-      const float kfac = p.sm_scale * LOG2E * rsqrtf((float)D);  // scores in log2 units: z2 = S_raw * scale_K * kfac
-      const float vfac = rsqrtf((float)D);
-      float acc[DJ][8];  // thread c: coordinates c (+128), 8 heads
-      float m_run[8], l_run[8], best_v[8];
-      int best_i[8];
+
+    // ---- open a segment: reset the softmax state; the operand B_Q is either one of the prepared ones (dd.bqbuf >= 0)
+    // or written here into the group's own buffer, warp w of the group rotating heads w and w + 4. The operand is read
+    // by the score MMAs of the segment's blocks, which the control warp issues after every thread of the group has
+    // signalled k_ready, i.e. after this function.
+    auto open_segment = [&](const DecDesc& dd) {
+      const int seg_b = dd.b, seg_y = dd.y, bqbuf = dd.bqbuf;
+      if (gt == 0) { seg_id[0] = seg_b; seg_id[1] = seg_y; seg_id[2] = dd.slot; }  // read back in close_segment, barriers in between
 #pragma unroll
       for (int j = 0; j < DJ; j++)
 #pragma unroll
         for (int h = 0; h < 8; h++) acc[j][h] = 0.f;
 #pragma unroll
       for (int h = 0; h < 8; h++) { m_run[h] = -INFINITY; l_run[h] = 0.f; best_v[h] = -INFINITY; best_i[h] = -1; }
-
+      if (bqbuf >= 0) {
+        if (I8) sfac = pre_sfac[bqbuf];
+        return;
+      }
+      int kvh, h0, nh;
+      item_heads(seg_y, kvh, h0, nh);
+      const int wq = warp & 3;
+      float v[2][E];
+#pragma unroll
+      for (int t = 0; t < 2; t++) rotate_head(seg_b, kvh, h0 + wq + 4 * t, wq + 4 * t < nh, v[t]);
+      float qmax = 0.f;
       if constexpr (I8) {
+        qmax = fmaxf(abs_max(v[0]), abs_max(v[1]));
+        if (lane == 0) qtmp[wq] = qmax;
+        group_bar_sync(bar_id);
+        qmax = fmaxf(fmaxf(qtmp[0], qtmp[1]), fmaxf(qtmp[2], qtmp[3]));
+        sfac = score_factor(qmax);
+      }
+#pragma unroll
+      for (int t = 0; t < 2; t++) write_operand(bq, wq + 4 * t, v[t], qmax);
+      fence_proxy_async();  // B_Q is written through the generic proxy and read by the tensor core through the async proxy
+    };
+
+    // ---- close the open segment: reduce l and the exact maximum (and argmax) over the group's 128 rows and write the
+    // group's partial to its slot of the item (d5 merges the slots). Called with the group's value MMAs complete and
+    // acc up to date.
+    auto close_segment = [&]() {
+      const int seg_b = seg_id[0], seg_y = seg_id[1], seg_slot = seg_id[2];
+      int kvh, h0, nh;
+      item_heads(seg_y, kvh, h0, nh);
+#pragma unroll
+      for (int h = 0; h < 8; h++) {
+        float v = l_run[h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+        if (lane == h) red[(warp & 3) * 8 + h] = v;
+        if (ARGMAX) {
+          float bv = best_v[h];
+          int bi = best_i[h];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(FULL, bv, o);
+            const int oi = __shfl_xor_sync(FULL, bi, o);
+            if (ov > bv || (ov == bv && oi >= 0 && (bi < 0 || oi < bi))) { bv = ov; bi = oi; }
+          }
+          if (lane == h) { red2[(warp & 3) * 8 + h] = bv; redi[(warp & 3) * 8 + h] = bi; }
+        }
+      }
+      group_bar_sync(bar_id);
+      float scale[8];  // the partial is reported relative to the exact maximum where that is tracked
+#pragma unroll
+      for (int h = 0; h < 8; h++) {
+        float mt = m_run[h];  // every thread of the group holds the same reference
+        int bi = -1;
+        if (ARGMAX) {
+          mt = -INFINITY;
+#pragma unroll
+          for (int wq = 0; wq < 4; wq++) {
+            const float ov = red2[wq * 8 + h];
+            const int oi = redi[wq * 8 + h];
+            if (ov > mt || (ov == mt && oi >= 0 && (bi < 0 || oi < bi))) { mt = ov; bi = oi; }
+          }
+        }
+        scale[h] = ARGMAX ? ex2f(m_run[h] - mt) : 1.f;
+        if (gt == h && h < nh) {
+          const size_t o = ((size_t)seg_b * p.n_q_heads + h0 + h) * S + seg_slot;
+          p.part_ml[2 * o] = mt * LN2;
+          p.part_ml[2 * o + 1] = (red[h] + red[8 + h] + red[16 + h] + red[24 + h]) * scale[h];
+          if (ARGMAX) p.part_argmax[o] = bi;
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < 8; h++)
+        if (h < nh) {
+#pragma unroll
+          for (int j = 0; j < DJ; j++)
+            p.part_acc[(((size_t)seg_b * p.n_q_heads + h0 + h) * S + seg_slot) * D + gt + 128 * j] = acc[j][h] * scale[h];
+        }
+      group_bar_sync(bar_id);  // the scratch is free again
+    };
+
+    int st = 0;          // stage of slot `it` and its phase, kept incrementally
+    uint32_t st_ph = 0;
+    int2 dsc = make_int2(-1, 0);  // (valid rows | end marker, flags) of slot `it`; the rest of its descriptor is read where it is needed
+    auto next_slot = [&]() {      // wait for slot `it` and read its descriptor
+      if (!failed) failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
+      if (failed) { dsc.x = -1; return; }
+      dsc = *reinterpret_cast<const int2*>(&desc[st]);
+    };
+    auto advance_slot = [&]() {
+      it++;
+      if (++st == NST) { st = 0; st_ph ^= 1u; }
+    };
+    next_slot();
+
+    if constexpr (I8) {
       // Integer path. The group's TMEM columns: K tile (d/4), V tile (32 per 128 coordinates), scores (32 = 8 heads x 4
       // digit columns), values (32 per 128 coordinates). The tiles do not share columns: the V tile of a block is
       // dequantised while its score MMAs run, the K tile of the next block while its value MMAs run.
-      int st = it % NST;                      // stage of slot `it` and its phase, kept incrementally
-      uint32_t st_ph = (uint32_t)(it / NST) & 1u;
       const uint32_t l8_0 = p.lut8[0], l8_1 = p.lut8[1];
-      const float sfac = reinterpret_cast<const float*>(smem + L::OFF_QFAC)[8];  // score digits -> log2-domain score per unit K scale
       float vref = 0.f;    // power of two >= every V scale (x 1/sqrt d) seen by the group in this segment
       float pscale = 0.f;  // probabilities are written as round(p * vscale * pscale) <= 2^30: pscale = 2^(30 - slack) / vref
       // The value products of consecutive blocks accumulate in TMEM as int32 (exact) for as long as the references they are
@@ -520,22 +774,19 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         tc_fence_before();
         mbar_arrive(k_ready);
       };
-      bool have_block = false;
-      int2 dsc = make_int2(0, -1);
-      if (!failed) {
-        failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
-        dsc = desc[st];
-        if (dsc.y < 0) {  // end marker: the segment has no blocks for this group
-          mbar_arrive(&empty_bar[st]);
-          it++;
-        } else {
-          have_block = true;
-          k_tile(stages + st * L::STAGE_BYTES);
-        }
-      }
-      while (have_block) {
+#pragma unroll 1
+      while (dsc.x >= 0) {  // one segment per pass: slot `it` holds the first block this group gets of it
+        open_segment(desc[st]);
+        vref = 0.f;
+        pscale = 0.f;
+        nacc = 0;
+        k_tile(stages + st * L::STAGE_BYTES);
+        bool more = true;
+#pragma unroll 1
+      while (more) {  // the blocks of the segment
         const uint8_t* sp = stages + st * L::STAGE_BYTES;
-        const int r0 = dsc.x, n = dsc.y;
+        const int n = dsc.x;
+        const int r0 = ARGMAX ? desc[st].r0 : 0;
         (void)r0;
         // ---- V coordinate gt (+128) of this block -> TMEM lane gt, while the score MMAs run
 #pragma unroll
@@ -563,6 +814,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 
         // ---- scores: three int32 digit columns per head -> log2-domain score of row gt
         if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
+        if (failed) break;
         tc_fence_after();
         float s[8];
         {
@@ -581,13 +833,14 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           tc_wait_ld();
           digits_to_scores(raw1, 1);
         }
-        if (ARGMAX) {  // exact maximum seen by this thread and its row (a group sees its blocks in ascending order)
+        if (ARGMAX) {  // exact maximum seen by this thread and its row (a group sees the blocks of a segment in ascending order)
 #pragma unroll
           for (int h = 0; h < 8; h++)
             if (s[h] > best_v[h]) { best_v[h] = s[h]; best_i[h] = r0 + gt; }
         }
-        // The running reference m_run is raised when a score exceeds it by more than one log2 unit, the V-scale bound vref
-        // when a row exceeds it: both are rare after the first blocks (one barrier with an OR reduction otherwise).
+        // The running reference m_run is raised when a score exceeds it by more than DEC_MAX_SLACK_I8 log2 units, the
+        // V-scale bound vref when a row exceeds it: both are rare after the first blocks (one barrier with an OR reduction
+        // otherwise).
         float over[8];
 #pragma unroll
         for (int h = 0; h < 8; h++) over[h] = s[h] - m_run[h];  // NaN (-inf - -inf) for a stale row of an unopened reference: max ignores it
@@ -612,6 +865,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
             l_run[h] *= alpha;
 #pragma unroll
             for (int j = 0; j < DJ; j++) acc[j][h] *= alpha;
+            over[h] = s[h] - mn;
           }
           const float bv = fmaxf(fmaxf(red2[0], red2[1]), fmaxf(red2[2], red2[3]));
           if (bv > vref) vref = __uint_as_float((__float_as_uint(bv) + 0x007FFFFFu) & 0x7F800000u);  // next power of two
@@ -624,7 +878,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           const float vfp = vf * pscale;
 #pragma unroll
           for (int h = 0; h < 8; h++) {
-            const float pr = ex2f(s[h] - m_run[h]);
+            const float pr = ex2f(over[h]);
             l_run[h] += pr;
             pb[h] = __float2uint_rn(pr * vfp);
           }
@@ -640,34 +894,28 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         mbar_arrive(p_ready);          // V tile in TMEM, probabilities in shared memory
         mbar_arrive(&empty_bar[st]);   // this thread is done with the staged tile
 
-        // ---- next slot: its K tile, while the value MMAs run
-        it++;
-        if (++st == NST) { st = 0; st_ph ^= 1u; }
-        if (!failed) failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
-        dsc = failed ? make_int2(0, -1) : desc[st];
-        have_block = dsc.y >= 0;
-        if (have_block) k_tile(stages + st * L::STAGE_BYTES);
+        // ---- next slot: if it continues the segment, its K tile now, while the value MMAs run
+        advance_slot();
+        next_slot();
+        more = dsc.x >= 0 && !(dsc.y & 1);
+        if (more) k_tile(stages + st * L::STAGE_BYTES);
 
         // ---- the value MMAs of this block must have completed before its V tile and B_P are overwritten; their result stays in TMEM
         if (!failed) failed = !mbar_wait_bounded(o_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
         nbk++;
-        if (!have_block && !failed) {
-          mbar_arrive(&empty_bar[st]);  // the end marker's slot
-          it++;
-        }
       }
-      if (nacc > 0) flush();
-
-      } else {
-      // The group's 128 TMEM columns: [0, 64 DJ) operand tile, then scores, values, and V_COL.. a second home for the first
-      // half of the V tile. Schedule of one block (K tile complete, k_ready signalled):
+        if (failed) break;
+        if (nacc > 0) flush();
+        close_segment();
+      }
+    } else {
+      // fp16 path. The group's 128 TMEM columns: [0, 64 DJ) operand tile, then scores, values, and V_COL.. a second home for
+      // the first half of the V tile. Schedule of one block (K tile complete, k_ready signalled):
       //   V rows 0..63 -> V_COL columns               while the score MMAs read the K tile
       //   wait for the scores; V rows 64..127 -> lower half of the operand columns, interleaved with the softmax
       //   signal p_ready; next block's K coordinates 32..63 (+64..) -> upper half of the operand columns
       //                                                while the value MMAs read the lower half and V_COL
       //   wait for the values, fold them; next block's other K coordinates -> lower half; signal k_ready
-      int st = it % NST;                      // stage of slot `it` and its phase, kept incrementally
-      uint32_t st_ph = (uint32_t)(it / NST) & 1u;
       uint32_t kw[L::WPR];                    // packed K row of the block being staged into TMEM
       auto k_load = [&](const uint8_t* sp_) {
         const uint4* krow = reinterpret_cast<const uint4*>(sp_ + gt * L::ROWB);
@@ -682,28 +930,21 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         dequant_unit(kw[3 * u], kw[3 * u + 1], kw[3 * u + 2], lut_lo0, lut_lo1, lut_hi0, lut_hi1, f);
         tc_st16(tmem_g + lane_sel + L::A_COL + 16 * u, f);
       };
-      // first block of the group in this segment: the whole K tile
-      bool have_block = false;
-      int2 dsc = make_int2(0, -1);
-      if (!failed) {
-        failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
-        dsc = desc[st];
-        if (dsc.y < 0) {  // end marker: the segment has no blocks for this group
-          mbar_arrive(&empty_bar[st]);
-          it++;
-        } else {
-          have_block = true;
-          k_load(stages + st * L::STAGE_BYTES);
+#pragma unroll 1
+      while (dsc.x >= 0) {  // one segment per pass: slot `it` holds the first block this group gets of it
+        open_segment(desc[st]);
+        k_load(stages + st * L::STAGE_BYTES);  // the whole K tile
 #pragma unroll
-          for (int u = 0; u < 4 * DJ; u++) k_unit(u);
-          tc_wait_st();
-          tc_fence_before();
-          mbar_arrive(k_ready);
-        }
-      }
-      while (have_block) {
+        for (int u = 0; u < 4 * DJ; u++) k_unit(u);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(k_ready);
+        bool more = true;
+#pragma unroll 1
+      while (more) {  // the blocks of the segment
         const uint8_t* sp = stages + st * L::STAGE_BYTES;
-        const int r0 = dsc.x, n = dsc.y;
+        const int n = dsc.x;
+        const int r0 = ARGMAX ? desc[st].r0 : 0;
         (void)r0;
         // ---- V coordinate gt (+128): rows 0..63 now, rows 64..127 with the softmax
         uint32_t wd[DJ][12];
@@ -729,6 +970,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 
         // the score MMAs read the K tile that the rest of the V tile is about to overwrite
         if (!failed) failed = !mbar_wait_bounded(s_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
+        if (failed) break;
         tc_fence_after();
         uint32_t raw_u[16];
         tc_ld16_issue(tmem_g + lane_sel + L::S_COL, raw_u);  // scores of row gt: in flight during the next unit
@@ -745,7 +987,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 #pragma unroll
           for (int h = 0; h < 8; h++) s[h] = fmaf(__uint_as_float(raw_u[h]) + __uint_as_float(raw_u[8 + h]), kf, mask);
         }
-        if (ARGMAX) {  // exact maximum seen by this thread and its row (a group sees its blocks in ascending order)
+        if (ARGMAX) {  // exact maximum seen by this thread and its row (a group sees the blocks of a segment in ascending order)
 #pragma unroll
           for (int h = 0; h < 8; h++)
             if (s[h] > best_v[h]) { best_v[h] = s[h]; best_i[h] = r0 + gt; }
@@ -773,6 +1015,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
             l_run[h] *= alpha;
 #pragma unroll
             for (int j = 0; j < DJ; j++) acc[j][h] *= alpha;
+            over[h] = s[h] - mn;
           }
         }
 #pragma unroll
@@ -782,7 +1025,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           float wv[8];
 #pragma unroll
           for (int h = 0; h < 8; h++) {
-            const float pr = ex2f(s[h] - m_run[h]);
+            const float pr = ex2f(over[h]);
             l_run[h] += pr;
             wv[h] = pr * vf;
           }
@@ -805,13 +1048,12 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         mbar_arrive(p_ready);          // V tile in TMEM, probabilities in shared memory
         mbar_arrive(&empty_bar[st]);   // this thread is done with the staged tile
 
-        // ---- next slot: its K coordinates that live in the upper half of the operand columns, while the value MMAs run
-        it++;
-        if (++st == NST) { st = 0; st_ph ^= 1u; }
-        if (!failed) failed = !mbar_wait_bounded(&full_bar[st], st_ph, DEC_WAIT_LIMIT);
-        dsc = failed ? make_int2(0, -1) : desc[st];
-        have_block = dsc.y >= 0;
-        if (have_block) {
+        // ---- next slot: if it continues the segment, its K coordinates that live in the upper half of the operand
+        // columns, while the value MMAs run
+        advance_slot();
+        next_slot();
+        more = dsc.x >= 0 && !(dsc.y & 1);
+        if (more) {
           k_load(stages + st * L::STAGE_BYTES);
 #pragma unroll
           for (int u = 0; u < 4 * DJ; u++)
@@ -820,6 +1062,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 
         // ---- fold the value product into the running accumulator (the value MMAs also release the lower half)
         if (!failed) failed = !mbar_wait_bounded(o_bar, (uint32_t)nbk & 1u, DEC_WAIT_LIMIT);
+        if (failed) break;
         tc_fence_after();
 #pragma unroll
         for (int j = 0; j < DJ; j++) {
@@ -830,106 +1073,20 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         }
         tc_fence_before();
         nbk++;
-        if (have_block) {
+        if (more) {
 #pragma unroll
           for (int u = 0; u < 4 * DJ; u++)
             if (!(u & 2)) k_unit(u);
           tc_wait_st();
           tc_fence_before();
           mbar_arrive(k_ready);
-        } else if (!failed) {
-          mbar_arrive(&empty_bar[st]);  // the end marker's slot
-          it++;
         }
       }
-
-      }
-      // ---- close the group's part of the segment: reduce l and the exact maximum (and argmax) over the 128 rows and
-      // leave the group partial in the group's (drained) staging buffer for the merge
-#pragma unroll
-      for (int h = 0; h < 8; h++) {
-        float v = l_run[h];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
-        float bv = best_v[h];
-        int bi = best_i[h];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          const float ov = __shfl_xor_sync(FULL, bv, o);
-          const int oi = ARGMAX ? __shfl_xor_sync(FULL, bi, o) : -1;
-          if (ov > bv || (ARGMAX && ov == bv && oi >= 0 && (bi < 0 || oi < bi))) { bv = ov; bi = oi; }
-        }
-        if (lane == h) { red[(warp & 3) * 8 + h] = v; red2[(warp & 3) * 8 + h] = bv; redi[(warp & 3) * 8 + h] = bi; }
-      }
-#pragma unroll
-      for (int j = 0; j < DJ; j++)
-#pragma unroll
-        for (int h = 0; h < 8; h++) gacc[(j * 8 + h) * DEC_GROUP_THREADS + gt] = acc[j][h];
-      group_bar_sync(bar_id);
-      if (gt < 8) {
-        const int h = gt;
-        float mt = -INFINITY;
-        int bi = -1;
-        for (int wq = 0; wq < 4; wq++) {
-          const float ov = red2[wq * 8 + h];
-          const int oi = redi[wq * 8 + h];
-          if (ov > mt || (ov == mt && oi >= 0 && (bi < 0 || oi < bi))) { mt = ov; bi = oi; }
-        }
-        gml[4 * h] = m_run[h];  // every thread of the group holds the same reference
-        gml[4 * h + 1] = red[h] + red[8 + h] + red[16 + h] + red[24 + h];
-        gml[4 * h + 2] = ARGMAX ? mt : m_run[h];  // without the argmax output the reference stands in for the maximum
-        reinterpret_cast<int*>(gml)[4 * h + 3] = bi;
+        if (failed) break;
+        close_segment();
       }
     }
-    // ================================================================ merge the groups' partials into the item's partial slot
-    const int seg_b = seg_s->b, seg_y = seg_s->y, seg_slot = seg_s->slot, seg_flags = seg_s->flags;  // before thread 0 reopens seg_s
-    __syncthreads();  // every group has closed its part
-    if (!control) {
-      const int kvh = seg_y / p.head_groups;
-      const int hg = seg_y - kvh * p.head_groups;
-      const int h0 = kvh * p.group + hg * DEC_HEADS;
-      const int nh = min(DEC_HEADS, p.group - hg * DEC_HEADS);
-      const uint8_t* group0 = bq + L::BQ_BYTES + L::BP_BYTES;  // staging buffer of group 0; the others follow at GROUP_SMEM
-      auto gacc_of = [&](int g) { return reinterpret_cast<const float*>(group0 + (size_t)g * L::GROUP_SMEM); };
-      auto gml_of = [&](int g) { return gacc_of(g) + DJ * 8 * DEC_GROUP_THREADS; };
-      // thread (c, hsel): coordinate c (+128), heads hsel, hsel + NG, ...
-      const int c = tid & (DEC_GROUP_THREADS - 1);
-      for (int h = tid >> 7; h < nh; h += NG) {
-        float mt = -INFINITY;  // the exact maximum of the segment: the partial is reported relative to it
-#pragma unroll
-        for (int g = 0; g < NG; g++) mt = fmaxf(mt, gml_of(g)[4 * h + 2]);
-        float sc[NG];
-#pragma unroll
-        for (int g = 0; g < NG; g++) sc[g] = ex2f(gml_of(g)[4 * h] - mt);  // a group without blocks: exp2(-inf) = 0
-#pragma unroll
-        for (int j = 0; j < DJ; j++) {
-          float v = 0.f;
-#pragma unroll
-          for (int g = 0; g < NG; g++) v += gacc_of(g)[(j * 8 + h) * DEC_GROUP_THREADS + c] * sc[g];
-          p.part_acc[(((size_t)seg_b * p.n_q_heads + h0 + h) * S + seg_slot) * D + c + 128 * j] = v;
-        }
-      }
-      if (tid < nh) {
-        const int h = tid;
-        float mt = -INFINITY;
-        int bi = -1;
-#pragma unroll
-        for (int g = 0; g < NG; g++) {
-          const float ov = gml_of(g)[4 * h + 2];
-          const int oi = reinterpret_cast<const int*>(gml_of(g))[4 * h + 3];
-          if (ov > mt || (ov == mt && oi >= 0 && (bi < 0 || oi < bi))) { mt = ov; bi = oi; }
-        }
-        float l = 0.f;
-#pragma unroll
-        for (int g = 0; g < NG; g++) l += gml_of(g)[4 * h + 1] * ex2f(gml_of(g)[4 * h] - mt);
-        const size_t o = ((size_t)seg_b * p.n_q_heads + h0 + h) * S + seg_slot;
-        p.part_ml[2 * o] = mt * LN2;
-        p.part_ml[2 * o + 1] = l;
-        if (ARGMAX) p.part_argmax[o] = bi;
-      }
-      if (seg_flags & 1) fill_slots(seg_b, h0, nh, seg_slot + 1, L::COMPUTE_THREADS, tid);  // end of the item: its unused slots
-    }
-    if (seg_flags & 2) break;  // last segment of this CTA
+    if (!failed && dsc.x < 0) mbar_arrive(&empty_bar[st]);  // the end marker's slot
   }
 
   allow_dependent_launch();
@@ -974,6 +1131,8 @@ cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStr
   return am ? launch_one<256, true, false>(p, stream) : launch_one<256, false, false>(p, stream);
 }
 
+// Groups (independent workers, one partial slot each per piece of an item) the decode kernel runs per CTA.
+int decode_groups_per_cta(int head_dim) { return head_dim == 128 ? DecLayout<128>::NG : DecLayout<256>::NG; }
 // CTAs the decode kernel keeps resident per SM (it sizes its grid as one CTA per SM).
 int decode_ctas_per_sm(int head_dim) { (void)head_dim; return 1; }
 

@@ -1,11 +1,15 @@
 // Device helpers shared by the decode kernels: tcgen05 / tensor-memory wrappers, the byte-lookup dequantisation of
-// a packing unit, named barriers, and the descriptors of a CTA's position in the launch-wide block sequence.
+// a packing unit, named barriers.
 #pragma once
 #include "iq_common.cuh"
 
 namespace iq {
 
-constexpr uint32_t DEC_WAIT_LIMIT = 1u << 22;
+// Polls one mbarrier wait of the decode kernel may take before the kernel gives up (IQ_STATUS_WAIT_TIMEOUT): with the
+// 20 us suspend hint of a poll that is at most 65536 * 20 us = 1.3 s (and a few milliseconds at least). Waits that
+// work last microseconds. A thread that has given up skips every later wait, so a CTA returns within about that time
+// after its first failed wait.
+constexpr uint32_t DEC_WAIT_LIMIT = 1u << 16;
 
 // ---------------------------------------------------------------------------------------------- tcgen05 wrappers
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -150,22 +154,5 @@ __device__ __forceinline__ float warp_max(float v) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(FULL, v, o));
   return v;
 }
-
-// Segment descriptor in shared memory (written by thread 0 before each segment).
-struct DecSegment {
-  int b, y;          // sequence, item within the sequence (KV head x head group)
-  int blk0, blk1;    // blocks [blk0, blk1) of the item
-  int slot;          // partial slot of the item this segment reports to
-  int len;           // cached rows of the sequence
-  int flags;         // bit 0: blk1 is the end of the item; bit 1: last segment of this CTA
-  int pad;
-};
-
-// Thread 0's position in the CTA's range (kept in shared memory between segments).
-struct DecWalk {
-  int b, y, blk, nb;        // sequence, item within it, block within the item, blocks of sequence b
-  long long left, g, item;  // range mode: blocks to go, launch-wide position; whole-item mode: linear item index
-};
-
 
 }  // namespace iq

@@ -83,6 +83,7 @@ struct DecodeParams {
 };
 cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream);
 int decode_ctas_per_sm(int head_dim);
+int decode_groups_per_cta(int head_dim);
 
 // ---- combine + inverse rotation
 struct CombineParams {

@@ -128,7 +128,10 @@ def test_argument_validation_happens_before_any_launch(iq, monkeypatch):
 
 
 def test_suggest_splits_is_sane(iq):
+    # one slot per piece of an item and group of the CTA that holds it (4 groups at head_dim 128, 2 at 256): a multiple
+    # of the group count, at least two pieces, no more pieces than groups' worth of 128-row blocks
     s = iq.iq_suggest_splits(iq.Shape(1, 32, 8, 128, 32768), 32768)
-    assert 1 <= s <= 64
-    assert iq.iq_suggest_splits(iq.Shape(1, 4, 1, 128, 1024), 100) == 1
-    assert iq.iq_suggest_splits(iq.Shape(32, 64, 8, 128, 32768), 32768) >= 1
+    assert s % 4 == 0 and 8 <= s <= 4 * 64
+    assert iq.iq_suggest_splits(iq.Shape(1, 4, 1, 128, 1024), 100) == 8
+    assert iq.iq_suggest_splits(iq.Shape(32, 64, 8, 128, 32768), 32768) == 8
+    assert iq.iq_suggest_splits(iq.Shape(1, 16, 8, 256, 16384), 16384) % 2 == 0
