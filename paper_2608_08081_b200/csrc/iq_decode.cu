@@ -38,6 +38,7 @@ constexpr int DEC_GROUP_THREADS = 128;  // 4 warps: dequantisation, softmax, acc
 constexpr int DEC_HDR_BYTES = 4096;    // barriers, TMEM base, work counter, block descriptors, scratch
 constexpr int DEC_NPRE = 4;             // query operands prepared at the start of a CTA: those of its range's first segments
 constexpr int DEC_PRE_BAR = 9;          // named barrier of all compute threads (used while those operands are built)
+constexpr float DEC_RAISE_MARGIN = 3.0f;  // log2 units a raised reference is put above the block's maximum
 constexpr float DEC_MAX_SLACK = 4.0f;  // log2 units a score may exceed the running reference before it is raised
 #ifndef IQ_SLACK_I8
 #define IQ_SLACK_I8 4
@@ -659,22 +660,15 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
       const int seg_b = seg_id[0], seg_y = seg_id[1], seg_slot = seg_id[2];
       int kvh, h0, nh;
       item_heads(seg_y, kvh, h0, nh);
-#pragma unroll
-      for (int h = 0; h < 8; h++) {
-        float v = l_run[h];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
-        if (lane == h) red[(warp & 3) * 8 + h] = v;
+      {
+        const int hr = warp_reduce8_head(lane);  // the head whose sums this lane ends up with
+        const float lsum = warp_reduce8(l_run, lane, [](float x, float y) { return x + y; });
+        if ((lane & 3) == 0) red[(warp & 3) * 8 + hr] = lsum;
         if (ARGMAX) {
-          float bv = best_v[h];
-          int bi = best_i[h];
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(FULL, bv, o);
-            const int oi = __shfl_xor_sync(FULL, bi, o);
-            if (ov > bv || (ov == bv && oi >= 0 && (bi < 0 || oi < bi))) { bv = ov; bi = oi; }
-          }
-          if (lane == h) { red2[(warp & 3) * 8 + h] = bv; redi[(warp & 3) * 8 + h] = bi; }
+          float bv;
+          int bi;
+          warp_argmax8(best_v, best_i, lane, bv, bi);
+          if ((lane & 3) == 0) { red2[(warp & 3) * 8 + hr] = bv; redi[(warp & 3) * 8 + hr] = bi; }
         }
       }
       group_bar_sync(bar_id);
@@ -687,9 +681,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           mt = -INFINITY;
 #pragma unroll
           for (int wq = 0; wq < 4; wq++) {
-            const float ov = red2[wq * 8 + h];
-            const int oi = redi[wq * 8 + h];
-            if (ov > mt || (ov == mt && oi >= 0 && (bi < 0 || oi < bi))) { mt = ov; bi = oi; }
+            argmax_merge(mt, bi, red2[wq * 8 + h], redi[wq * 8 + h]);
           }
         }
         scale[h] = ARGMAX ? ex2f(m_run[h] - mt) : 1.f;
@@ -707,7 +699,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           for (int j = 0; j < DJ; j++)
             p.part_acc[(((size_t)seg_b * p.n_q_heads + h0 + h) * S + seg_slot) * D + gt + 128 * j] = acc[j][h] * scale[h];
         }
-      group_bar_sync(bar_id);  // the scratch is free again
+      // (the scratch is written next after the group barrier of the next block's vote)
     };
 
     int st = 0;          // stage of slot `it` and its phase, kept incrementally
@@ -848,10 +840,9 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
                             vf > vref || nacc >= 384;
         if (group_bar_or(bar_id, exceed)) {
           if (nacc > 0) flush();  // what TMEM holds is relative to the old references (the previous value MMAs have completed)
-#pragma unroll
-          for (int h = 0; h < 8; h++) {
-            const float wm = warp_max(s[h]);
-            if (lane == h) red[(warp & 3) * 8 + h] = wm;
+          {
+            const float wm = warp_reduce8(s, lane, [](float x, float y) { return fmaxf(x, y); });
+            if ((lane & 3) == 0) red[(warp & 3) * 8 + warp_reduce8_head(lane)] = wm;
           }
           const float wv_max = warp_max(vf);
           if (lane == 0) red2[warp & 3] = wv_max;
@@ -859,7 +850,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 #pragma unroll
           for (int h = 0; h < 8; h++) {
             const float bm = fmaxf(fmaxf(red[h], red[8 + h]), fmaxf(red[16 + h], red[24 + h]));
-            const float mn = fmaxf(m_run[h], bm);
+            const float mn = (bm > m_run[h] + DEC_MAX_SLACK_I8) ? bm + DEC_RAISE_MARGIN : m_run[h];  // raised beyond the maximum: fewer raises later
             const float alpha = ex2f(m_run[h] - mn);  // the accumulator holds the blocks before this one: rescale it now
             m_run[h] = mn;
             l_run[h] *= alpha;
@@ -1000,16 +991,15 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         for (int h = 0; h < 8; h++) over[h] = s[h] - m_run[h];  // NaN (-inf - -inf) for a stale row of an unopened reference: max ignores it
         const bool exceed = max3f(max3f(over[0], over[1], over[2]), max3f(over[3], over[4], over[5]), fmaxf(over[6], over[7])) > DEC_MAX_SLACK;
         if (group_bar_or(bar_id, exceed)) {
-#pragma unroll
-          for (int h = 0; h < 8; h++) {
-            const float wm = warp_max(s[h]);
-            if (lane == h) red[(warp & 3) * 8 + h] = wm;
+          {
+            const float wm = warp_reduce8(s, lane, [](float x, float y) { return fmaxf(x, y); });
+            if ((lane & 3) == 0) red[(warp & 3) * 8 + warp_reduce8_head(lane)] = wm;
           }
           group_bar_sync(bar_id);
 #pragma unroll
           for (int h = 0; h < 8; h++) {
             const float bm = fmaxf(fmaxf(red[h], red[8 + h]), fmaxf(red[16 + h], red[24 + h]));
-            const float mn = fmaxf(m_run[h], bm);
+            const float mn = (bm > m_run[h] + DEC_MAX_SLACK) ? bm + DEC_RAISE_MARGIN : m_run[h];  // raised beyond the maximum: fewer raises later
             const float alpha = ex2f(m_run[h] - mn);  // the accumulator holds the blocks before this one: rescale it now
             m_run[h] = mn;
             l_run[h] *= alpha;

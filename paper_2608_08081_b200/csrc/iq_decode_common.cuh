@@ -149,6 +149,48 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
+// Reduction of 8 values per lane over the 32 lanes of a warp with 9 shuffles instead of 40: the lanes first trade
+// halves of their value sets (xor 16: four values each way, xor 8: two, xor 4: one), so that lane l ends up with one
+// value of head warp_reduce8_head(l), which two more butterfly steps complete. Every lane gets the result of its head.
+__device__ __forceinline__ int warp_reduce8_head(int lane) { return ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1); }
+template <typename OP>
+__device__ __forceinline__ float warp_reduce8(const float (&v)[8], int lane, OP op) {
+  const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4;
+  float a[4], c[2];
+#pragma unroll
+  for (int i = 0; i < 4; i++) a[i] = op(b4 ? v[i + 4] : v[i], __shfl_xor_sync(FULL, b4 ? v[i] : v[i + 4], 16));
+#pragma unroll
+  for (int i = 0; i < 2; i++) c[i] = op(b3 ? a[i + 2] : a[i], __shfl_xor_sync(FULL, b3 ? a[i] : a[i + 2], 8));
+  float r = op(b2 ? c[1] : c[0], __shfl_xor_sync(FULL, b2 ? c[0] : c[1], 4));
+  r = op(r, __shfl_xor_sync(FULL, r, 2));
+  return op(r, __shfl_xor_sync(FULL, r, 1));
+}
+// The same for (value, row) pairs: the larger value wins, the lower row among equal values (rows < 0 mean "none").
+__device__ __forceinline__ void argmax_merge(float& bv, int& bi, float ov, int oi) {
+  if (ov > bv || (ov == bv && oi >= 0 && (bi < 0 || oi < bi))) { bv = ov; bi = oi; }
+}
+__device__ __forceinline__ void warp_argmax8(const float (&v)[8], const int (&ix)[8], int lane, float& rv, int& ri) {
+  const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4;
+  float a[4], c[2];
+  int ai[4], ci[2];
+#pragma unroll
+  for (int i = 0; i < 4; i++) {
+    a[i] = b4 ? v[i + 4] : v[i];
+    ai[i] = b4 ? ix[i + 4] : ix[i];
+    argmax_merge(a[i], ai[i], __shfl_xor_sync(FULL, b4 ? v[i] : v[i + 4], 16), __shfl_xor_sync(FULL, b4 ? ix[i] : ix[i + 4], 16));
+  }
+#pragma unroll
+  for (int i = 0; i < 2; i++) {
+    c[i] = b3 ? a[i + 2] : a[i];
+    ci[i] = b3 ? ai[i + 2] : ai[i];
+    argmax_merge(c[i], ci[i], __shfl_xor_sync(FULL, b3 ? a[i] : a[i + 2], 8), __shfl_xor_sync(FULL, b3 ? ai[i] : ai[i + 2], 8));
+  }
+  rv = b2 ? c[1] : c[0];
+  ri = b2 ? ci[1] : ci[0];
+  argmax_merge(rv, ri, __shfl_xor_sync(FULL, b2 ? c[0] : c[1], 4), __shfl_xor_sync(FULL, b2 ? ci[0] : ci[1], 4));
+  argmax_merge(rv, ri, __shfl_xor_sync(FULL, rv, 2), __shfl_xor_sync(FULL, ri, 2));
+  argmax_merge(rv, ri, __shfl_xor_sync(FULL, rv, 1), __shfl_xor_sync(FULL, ri, 1));
+}
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(FULL, v, o));
