@@ -660,6 +660,33 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
       const int seg_b = seg_id[0], seg_y = seg_id[1], seg_slot = seg_id[2];
       int kvh, h0, nh;
       item_heads(seg_y, kvh, h0, nh);
+      if constexpr (!ARGMAX) {
+        // without the argmax output the partial is reported relative to the running reference as it stands
+        float* dst = p.part_acc + (((size_t)seg_b * p.n_q_heads + h0) * S + seg_slot) * D + gt;
+        const size_t hstride = (size_t)S * D;
+#pragma unroll
+        for (int h = 0; h < 8; h++)
+          if (h < nh) {
+#pragma unroll
+            for (int j = 0; j < DJ; j++) dst[h * hstride + 128 * j] = acc[j][h];
+          }
+        const int hr = warp_reduce8_head(lane);  // the head whose sum this lane ends up with
+        const float lsum = warp_reduce8(l_run, lane, [](float x, float y) { return x + y; });
+        float msel = m_run[0];  // m_run[hr] (every thread of the group holds the same references)
+#pragma unroll
+        for (int h = 1; h < 8; h++) msel = (hr == h) ? m_run[h] : msel;
+        if ((lane & 3) == 0) {
+          red[(warp & 3) * 8 + hr] = lsum;
+          if ((warp & 3) == 0) red2[hr] = msel;
+        }
+        group_bar_sync(bar_id);
+        if (gt < nh) {
+          const size_t o = ((size_t)seg_b * p.n_q_heads + h0 + gt) * S + seg_slot;
+          p.part_ml[2 * o] = red2[gt] * LN2;
+          p.part_ml[2 * o + 1] = red[gt] + red[8 + gt] + red[16 + gt] + red[24 + gt];
+        }
+        return;  // (the scratch is written next after the group barrier of the next block's vote)
+      }
       {
         const int hr = warp_reduce8_head(lane);  // the head whose sums this lane ends up with
         const float lsum = warp_reduce8(l_run, lane, [](float x, float y) { return x + y; });
@@ -757,10 +784,11 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
           kw[4 * i] = t4.x; kw[4 * i + 1] = t4.y; kw[4 * i + 2] = t4.z; kw[4 * i + 3] = t4.w;
         }
 #pragma unroll
-        for (int u = 0; u < 4 * DJ; u++) {
-          uint32_t f[8];
+        for (int u = 0; u < 4 * DJ; u += 2) {  // two packing units (64 coordinates) per TMEM store
+          uint32_t f[16];
           dequant_unit8(kw[3 * u], kw[3 * u + 1], kw[3 * u + 2], l8_0, l8_1, f);
-          tc_st8(tmem_g + lane_sel + L::I8_K_COL + 8 * u, f);
+          dequant_unit8(kw[3 * u + 3], kw[3 * u + 4], kw[3 * u + 5], l8_0, l8_1, f + 8);
+          tc_st16(tmem_g + lane_sel + L::I8_K_COL + 8 * u, f);
         }
         tc_wait_st();
         tc_fence_before();
@@ -791,10 +819,11 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
             wd[4 * i] = t4.x; wd[4 * i + 1] = t4.y; wd[4 * i + 2] = t4.z; wd[4 * i + 3] = t4.w;
           }
 #pragma unroll
-          for (int u = 0; u < 4; u++) {
-            uint32_t f[8];
+          for (int u = 0; u < 4; u += 2) {  // two packing units (64 rows) per TMEM store
+            uint32_t f[16];
             dequant_unit8(wd[3 * u], wd[3 * u + 1], wd[3 * u + 2], l8_0, l8_1, f);
-            tc_st8(tmem_g + lane_sel + L::I8_V_COL + 32 * j + 8 * u, f);
+            dequant_unit8(wd[3 * u + 3], wd[3 * u + 4], wd[3 * u + 5], l8_0, l8_1, f + 8);
+            tc_st16(tmem_g + lane_sel + L::I8_V_COL + 32 * j + 8 * u, f);
           }
         }
         const float ksc = load_scale(sp + L::K_BYTES + L::VT_BYTES, gt, p.scale_f16);
@@ -812,9 +841,9 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         {
           auto digits_to_scores = [&](const uint32_t (&raw_u)[16], int half) {
 #pragma unroll
-            for (int hq = 0; hq < 4; hq++) {  // S = S0 + 128 (S1 + 128 S2): the upper two digits combine in an int32
-              const float hi = __int2float_rn((int)raw_u[4 * hq + 2] * 128 + (int)raw_u[4 * hq + 1]);
-              s[4 * half + hq] = fmaf(fmaf(hi, 128.f, i2f_small(raw_u[4 * hq])), kfs, mask);
+            for (int hq = 0; hq < 4; hq++) {  // S = (S0 + 128 S1) + 16384 S2: the lower two digits combine in an int32 (< 2^28)
+              const float lo = __int2float_rn((int)raw_u[4 * hq + 1] * 128 + (int)raw_u[4 * hq]);
+              s[4 * half + hq] = fmaf(fmaf(__int2float_rn((int)raw_u[4 * hq + 2]), 16384.f, lo), kfs, mask);
             }
           };
           uint32_t raw0[16], raw1[16];
@@ -838,6 +867,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         for (int h = 0; h < 8; h++) over[h] = s[h] - m_run[h];  // NaN (-inf - -inf) for a stale row of an unopened reference: max ignores it
         const bool exceed = max3f(max3f(over[0], over[1], over[2]), max3f(over[3], over[4], over[5]), fmaxf(over[6], over[7])) > DEC_MAX_SLACK_I8 ||
                             vf > vref || nacc >= 384;
+        
         if (group_bar_or(bar_id, exceed)) {
           if (nacc > 0) flush();  // what TMEM holds is relative to the old references (the previous value MMAs have completed)
           {
@@ -850,7 +880,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 #pragma unroll
           for (int h = 0; h < 8; h++) {
             const float bm = fmaxf(fmaxf(red[h], red[8 + h]), fmaxf(red[16 + h], red[24 + h]));
-            const float mn = (bm > m_run[h] + DEC_MAX_SLACK_I8) ? bm + DEC_RAISE_MARGIN : m_run[h];  // raised beyond the maximum: fewer raises later
+            const float mn = fmaxf(m_run[h], bm + DEC_RAISE_MARGIN);  // every head goes above its block maximum whichever head asked: fewer raises later
             const float alpha = ex2f(m_run[h] - mn);  // the accumulator holds the blocks before this one: rescale it now
             m_run[h] = mn;
             l_run[h] *= alpha;
@@ -999,7 +1029,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
 #pragma unroll
           for (int h = 0; h < 8; h++) {
             const float bm = fmaxf(fmaxf(red[h], red[8 + h]), fmaxf(red[16 + h], red[24 + h]));
-            const float mn = (bm > m_run[h] + DEC_MAX_SLACK) ? bm + DEC_RAISE_MARGIN : m_run[h];  // raised beyond the maximum: fewer raises later
+            const float mn = fmaxf(m_run[h], bm + DEC_RAISE_MARGIN);  // every head goes above its block maximum whichever head asked: fewer raises later
             const float alpha = ex2f(m_run[h] - mn);  // the accumulator holds the blocks before this one: rescale it now
             m_run[h] = mn;
             l_run[h] *= alpha;

@@ -110,7 +110,7 @@ __device__ __forceinline__ void dequant_unit(uint32_t w0, uint32_t w1, uint32_t 
 }
 
 // Integer path: one packing unit -> 8 registers of four int8 levels each, entries in natural order (one prmt per 4 codes).
-__device__ __forceinline__ void dequant_unit8(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t l0, uint32_t l1, uint32_t (&out)[8]) {
+__device__ __forceinline__ void dequant_unit8(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t l0, uint32_t l1, uint32_t* out) {
   const uint32_t sel[4] = {w0 & 0x77777777u, w1 & 0x77777777u, w2 & 0x77777777u, sliced_selectors(w0, w1, w2)};
 #pragma unroll
   for (int k = 0; k < 4; k++) {
