@@ -22,7 +22,10 @@
  *   - Device-side conditions that cannot be known on the host are reported through an optional
  *     `status_dev` array of 4 uint32 (zeroed by the caller): [0] bit mask of IQ_STATUS_* flags,
  *     [1] rows whose codes were re-decided in fp64 (see iq_quantize_append), [2] rows skipped because
- *     they fell outside the cache, [3] reserved. Nothing on the device traps or spins without a bound.
+ *     they fell outside the cache, [3] reserved. Nothing on the device traps or spins without a bound: the
+ *     decode kernel's waits on its asynchronous copies and tensor-core results give up after 65536 polls of at most
+ *     20 us each (about a second at worst; a wait that works lasts microseconds), flag IQ_STATUS_WAIT_TIMEOUT and
+ *     the kernel returns with invalid results.
  *
  * Rotation (Eq. 2, Section 3.3 "SO(4) parameterization", Appendix B)
  *   R = R_SO4 o H_d. H_d is the normalised Walsh-Hadamard matrix in natural (Sylvester) order,
@@ -34,9 +37,12 @@
  *
  * Codebook (Section 3.2, Step 3)
  *   8 ascending levels and 7 ascending decision thresholds in unit-variance units u = sqrt(d) * x~.
- *   code = #{ j : u > t_j } (strict: an exact tie takes the lower code). The 8 levels must be exactly
- *   representable in IEEE binary16: the decode kernel feeds them to fp16 tensor-core operands and must
- *   not round them (IQ_ERR_CODEBOOK otherwise). A dequantised coordinate is scale * level[code] / sqrt(d).
+ *   code = #{ j : u > t_j } (strict: an exact tie takes the lower code). A dequantised coordinate is
+ *   scale * level[code] / sqrt(d). iq_quantize_append uses the thresholds only and takes any ascending set.
+ *   iq_decode_attention feeds the levels to tensor-core operands without rounding them, so it takes two forms:
+ *   levels on an 8-bit grid, level_j = n_j * delta with integers |n_j| <= 127 (iq_int8_codebook, or iq_fit_codebook
+ *   with grid = 1): int8 operands, the faster path; or levels that are all exact IEEE binary16 values
+ *   (iq_default_codebook, iq_fit_codebook with grid = 0): fp16 operands. Anything else is IQ_ERR_CODEBOOK.
  *
  * Packed cache (Section 3.2, Step 4 fixes the size only: 3d/8 bytes per row, 48 at d = 128)
  *   codes: 3d/8 bytes per cached row and side, scales [batch][n_kv_heads][t_cap] fp32 (= ||x||_2), separately
@@ -60,14 +66,18 @@
 extern "C" {
 #endif
 
-#define IQ_VERSION 100
+#define IQ_VERSION 200
+/* Version of the packed-cache byte layout described above and in docs/FORMAT.md (bit order of a packing unit,
+ * token-transposed V records, scale arrays, rotation parameters, partial slots). A cache written under one format
+ * version is read correctly only by a library of the same format version; iq_format_version() reports the library's. */
+#define IQ_FORMAT_VERSION 2
 
 enum {
   IQ_OK = 0,
   IQ_ERR_NULL = -1,     /* a required pointer is NULL */
   IQ_ERR_SHAPE = -2,    /* unsupported head_dim / bits, n_q_heads % n_kv_heads != 0, bad sizes or strides */
   IQ_ERR_ALIGN = -3,    /* a pointer or stride breaks the stated alignment */
-  IQ_ERR_CODEBOOK = -4, /* levels / thresholds not ascending, or a level not representable in binary16 */
+  IQ_ERR_CODEBOOK = -4, /* levels / thresholds not ascending; decode: levels neither on an 8-bit grid nor exact binary16 */
   IQ_ERR_CUDA = -5,     /* the CUDA runtime reported an error for the launch */
   IQ_ERR_LIMIT = -6     /* a size exceeds a documented maximum of the entry point */
 };
@@ -76,7 +86,8 @@ enum {
   IQ_STATUS_ROW_OUT_OF_RANGE = 1u, /* quantize-append: append_pos + i >= t_cap, row skipped */
   IQ_STATUS_WAIT_TIMEOUT = 2u,     /* decode: a bounded wait on an asynchronous copy ran out; results invalid */
   IQ_STATUS_SCALE_OVERFLOW = 8u,   /* binary16 scales: a row norm above 65504 was stored as 65504 */
-  IQ_STATUS_BAD_PAGE = 4u          /* paged cache: a block-table entry outside [0, num_pages) was met and read as page 0 */
+  IQ_STATUS_BAD_PAGE = 4u          /* paged cache: a block-table entry outside [0, num_pages) was met: read as page 0 by
+                                      decode / reconstruct, the rows skipped (and counted in [2]) by quantize-append */
 };
 
 typedef struct iq_shape {
@@ -105,7 +116,8 @@ typedef struct iq_cache {
    * block_table_dev is a device int32 [batch][t_cap / page_rows]: entry (b, j) is the page that holds rows
    * [j * page_rows, (j + 1) * page_rows) of sequence b. page_rows is a multiple of 128 and divides t_cap, which is
    * then the logical capacity of a sequence. Entries that a call can reach (rows below the lengths it is given)
-   * must be valid; an entry outside [0, num_pages) sets IQ_STATUS_BAD_PAGE and is read as page 0. */
+   * must be valid; an entry outside [0, num_pages) sets IQ_STATUS_BAD_PAGE: a reading kernel takes page 0 in its place,
+   * iq_quantize_append skips the rows that would go there and counts them in status[2]. */
   const int32_t* block_table_dev;
   int32_t page_rows;
   int32_t num_pages;
@@ -117,6 +129,7 @@ typedef struct iq_cache {
 } iq_cache;
 
 int iq_version(void);
+int iq_format_version(void);
 const char* iq_strerror(int code);
 
 /* Bytes of one packed row: 3 * head_dim / 8 (Section 3.2, Step 4). 0 for an unsupported head_dim. */
@@ -289,7 +302,8 @@ int iq_decode_step_host(const iq_shape* shape, const float* rot_dev, const iq_co
  *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress, with that
  *     device current); with lazy module loading that is also the moment the driver places the array on
  *     the GPU. Make that first call before any stream capture begins.
- *   - The call itself allocates nothing and frees nothing.
+ *   - The call itself allocates nothing and frees nothing. The address found by the first call is kept until the
+ *     process ends; after a cudaDeviceReset of the device it is stale and the entry point must not be called again.
  *   - All calls on a device share the one array, which keeps the previous call's contents. Every split of
  *     every head is rewritten on each call, so no clearing is needed; but two calls whose kernels overlap
  *     on the GPU (different streams) race on it. Serialise them on one stream or with events.
@@ -301,6 +315,16 @@ int iq_decode_attention_static(const iq_shape* shape, const float* rot_dev, cons
                                const void* q, const iq_cache* cache, const int32_t* seq_lens_dev,
                                int32_t num_splits, void* out, int32_t out_is_fp16, float* lse_out,
                                uint32_t* status_dev, void* stream);
+
+/*
+ * Diagnostic (the paper has no counterpart): exercises the give-up path of the decode kernel's bounded waits without
+ * the decode kernel. A one-warp kernel waits on a barrier that nothing completes -- no copy and no tensor-core work
+ * is in flight -- with `polls` (1 .. 65536) as its poll limit, sets IQ_STATUS_WAIT_TIMEOUT in status_dev[0] when the
+ * wait gives up and writes the polls it took to status_dev[1]. polls == 0 completes the barrier first: the wait
+ * succeeds and status_dev[0] stays as it is. A poll suspends the thread for at most 20 us, so the call lasts at
+ * most polls * 20 us.
+ */
+int iq_selftest_bounded_wait(uint32_t* status_dev, uint32_t polls, void* stream);
 
 /* A slot count that leaves the decode kernel free to balance the launch when the longest sequence has
  * max_seq_len rows (more slots than needed only cost the writing and merging of unused ones). */

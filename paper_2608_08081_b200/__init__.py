@@ -26,6 +26,8 @@ from .binding import (  # noqa: F401
     iq_reconstruct_rows,
     iq_rotated_histogram,
     iq_suggest_splits,
+    iq_format_version,
+    iq_selftest_bounded_wait,
     iq_version,
     lib_path,
     new_cache,

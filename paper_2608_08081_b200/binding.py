@@ -47,6 +47,7 @@ def _load():
             "There is no fallback implementation.")
     lib = ctypes.CDLL(path)
     lib.iq_version.restype = ctypes.c_int
+    lib.iq_format_version.restype = ctypes.c_int
     lib.iq_strerror.restype = ctypes.c_char_p
     lib.iq_strerror.argtypes = [ctypes.c_int]
     lib.iq_row_bytes.restype = ctypes.c_size_t
@@ -73,6 +74,7 @@ def _load():
     lib.iq_fit_codebook.argtypes = [_vp, _i32, ctypes.c_float, _i32, _i32, ctypes.POINTER(_IqCodebook)]
     lib.iq_suggest_splits.restype = _i32
     lib.iq_suggest_splits.argtypes = [ctypes.POINTER(_IqShape), _i32]
+    lib.iq_selftest_bounded_wait.argtypes = [_vp, ctypes.c_uint32, _vp]
     return lib
 
 
@@ -154,6 +156,10 @@ def _check(rc: int, where: str):
 
 def iq_version() -> int:
     return int(_lib.iq_version())
+
+
+def iq_format_version() -> int:
+    return int(_lib.iq_format_version())
 
 
 def iq_strerror(code: int) -> str:
@@ -283,6 +289,10 @@ def iq_fit_codebook(hist_host, rng_half: float, symmetric: bool = True, grid: st
 def iq_suggest_splits(shape: Shape, max_seq_len: int) -> int:
     cs = shape.c()
     return int(_lib.iq_suggest_splits(ctypes.byref(cs), max_seq_len))
+
+
+def iq_selftest_bounded_wait(status, polls: int, stream=None) -> None:
+    _check(_lib.iq_selftest_bounded_wait(_ptr(status), int(polls), _stream(stream)), "iq_selftest_bounded_wait")
 
 
 # ------------------------------------------------------------------ small conveniences (allocation only)

@@ -193,6 +193,7 @@ void finish_codebook(const double (&lv)[8], int grid, iq_codebook* out) {
 extern "C" {
 
 int iq_version(void) { return IQ_VERSION; }
+int iq_format_version(void) { return IQ_FORMAT_VERSION; }
 
 const char* iq_strerror(int code) {
   switch (code) {
@@ -200,7 +201,7 @@ const char* iq_strerror(int code) {
     case IQ_ERR_NULL: return "a required pointer is NULL";
     case IQ_ERR_SHAPE: return "unsupported shape (head_dim 128/256, bits 3, n_q_heads % n_kv_heads == 0, t_cap % 128 == 0, strides % 8 == 0)";
     case IQ_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
-    case IQ_ERR_CODEBOOK: return "codebook not ascending or a level is not representable in binary16";
+    case IQ_ERR_CODEBOOK: return "codebook not ascending, or (decode) its levels are neither on an 8-bit grid nor all exact binary16 values";
     case IQ_ERR_CUDA: return "CUDA runtime error at launch";
     case IQ_ERR_LIMIT: return "size exceeds the documented maximum of this entry point";
     default: return "unknown error code";
@@ -435,6 +436,17 @@ int iq_decode_step_host(const iq_shape* shape, const float* rot_dev, const iq_co
   if (rc) return rc;
   if (!inputs_host || !inputs_dev || !out_dev || !out_host) return IQ_ERR_NULL;
   if (!aligned16(inputs_dev)) return IQ_ERR_ALIGN;
+  // everything the three calls below would refuse is refused here, before the copy and the append are enqueued
+  if (!rot_dev || !append_pos_dev || !seq_lens_dev || !part_acc || !part_ml) return IQ_ERR_NULL;
+  if ((rc = check_codebook(codebook, false))) return rc;
+  {
+    int n8[8];
+    float delta = 0.f;
+    if (!int8_grid(codebook, n8, delta) && (rc = check_codebook(codebook, true))) return rc;
+  }
+  if ((rc = check_cache(cache, shape))) return rc;
+  if (num_splits < 1 || num_splits > 65535) return IQ_ERR_SHAPE;
+  if (!aligned16(part_acc) || !aligned16(rot_dev) || !aligned16(out_dev)) return IQ_ERR_ALIGN;
   if (shape->batch == 0) return IQ_OK;
   const size_t d = (size_t)shape->head_dim, B = (size_t)shape->batch;
   const size_t nq = B * (size_t)shape->n_q_heads * d, nk = B * (size_t)shape->n_kv_heads * d;  // elements of q, of k_new
@@ -498,6 +510,12 @@ int iq_fit_codebook(const uint32_t* hist_host, int32_t bins, float range, int32_
   for (int i = 0; i < 7; i++)
     if (!(out_host->levels[i] < out_host->levels[i + 1])) return IQ_ERR_CODEBOOK;  // too few distinct values in the data
   return IQ_OK;
+}
+
+int iq_selftest_bounded_wait(uint32_t* status_dev, uint32_t polls, void* stream) {
+  if (!status_dev) return IQ_ERR_NULL;
+  if (polls > 65536u) return IQ_ERR_LIMIT;
+  return iq::launch_bounded_wait_selftest(status_dev, polls, static_cast<cudaStream_t>(stream)) == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }
 
 int32_t iq_suggest_splits(const iq_shape* shape, int32_t max_seq_len) {

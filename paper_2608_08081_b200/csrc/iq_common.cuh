@@ -165,6 +165,21 @@ __device__ __forceinline__ size_t cache_row(const PageMap& m, int b, int g, long
   return ((size_t)page * m.n_kv_heads + g) * (size_t)m.page_rows + (size_t)(t - (long long)j * m.page_rows);
 }
 
+// The same for a kernel that WRITES the row. A block-table entry outside the pool must not redirect the write to
+// another page (page 0 may belong to another sequence): the function then returns false and sets IQ_STATUS_BAD_PAGE;
+// the caller skips the row and counts it.
+__device__ __forceinline__ bool cache_row_for_write(const PageMap& m, int b, int g, long long t, uint32_t* status, size_t& row) {
+  if (m.table != nullptr) {
+    const int page = m.table[(size_t)b * (m.t_cap / m.page_rows) + (int)(t / m.page_rows)];
+    if ((unsigned)page >= (unsigned)m.num_pages) {
+      if (status) atomicOr(&status[0], IQ_STATUS_BAD_PAGE);
+      return false;
+    }
+  }
+  row = cache_row(m, b, g, t, status);
+  return true;
+}
+
 // The scale arrays hold fp32 values or (f16 != 0) binary16 values of the same shape.
 __device__ __forceinline__ void store_scale(float* arr, size_t row, float s, int f16, uint32_t* status) {
   if (!f16) {

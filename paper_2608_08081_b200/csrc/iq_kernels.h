@@ -47,7 +47,6 @@ struct HistogramParams {
   const int32_t* n_rows;
   int n_rows_max;
   const float* rot;
-  float thresholds[7];  // unused (zeros): the row quantizer it shares with the append kernels loads them
   uint32_t* hist;
   int bins;
   float range;
@@ -84,6 +83,7 @@ struct DecodeParams {
 cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream);
 int decode_ctas_per_sm(int head_dim);
 int decode_groups_per_cta(int head_dim);
+cudaError_t launch_bounded_wait_selftest(uint32_t* status, uint32_t polls, cudaStream_t stream);
 
 // ---- combine + inverse rotation
 struct CombineParams {

@@ -274,11 +274,15 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 5) quantize_append_k_kernel(con
     uint32_t w0, w1;
     pack_pair(code, lane, w0, w1);
     if (active) {
-      const size_t row = cache_row(p.pm, b, h, t, p.status);
-      uint32_t* unit_words = reinterpret_cast<uint32_t*>(p.k_codes + row * (size_t)(3 * D / 8)) + 3 * (li >> 1);
-      if (li & 1) unit_words[2] = w0;
-      else { unit_words[0] = w0; unit_words[1] = w1; }
-      if (li == 0) store_scale(p.k_scales, row, s, p.scale_f16, p.status);
+      size_t row;
+      if (cache_row_for_write(p.pm, b, h, t, p.status, row)) {
+        uint32_t* unit_words = reinterpret_cast<uint32_t*>(p.k_codes + row * (size_t)(3 * D / 8)) + 3 * (li >> 1);
+        if (li & 1) unit_words[2] = w0;
+        else { unit_words[0] = w0; unit_words[1] = w1; }
+        if (li == 0) store_scale(p.k_scales, row, s, p.scale_f16, p.status);
+      } else if (li == 0 && p.status) {
+        atomicAdd(&p.status[2], 1u);  // a row whose page does not exist is skipped and counted
+      }
     }
   }
 }
@@ -320,7 +324,11 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
     }
     return;
   }
-  const size_t block_row0 = cache_row(p.pm, b, h, blkg * 128, p.status);  // the block's first row in the cache arrays
+  size_t block_row0;  // the block's first row in the cache arrays
+  if (!cache_row_for_write(p.pm, b, h, blkg * 128, p.status, block_row0)) {  // no such page: the block's rows are skipped and counted
+    if (tid == 0 && p.status) atomicAdd(&p.status[2], (unsigned)(t_hi - t_lo));
+    return;
+  }
 
   RQ::fill_matrices(p.rot + (size_t)h * (D / 4) * 8, m_s, tid, 128);
   __syncthreads();
@@ -533,7 +541,11 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
       }
       continue;
     }
-    const size_t row = cache_row(p.pm, b, h, t, p.status);  // the row's place in the cache arrays
+    size_t row;  // the row's place in the cache arrays
+    if (!cache_row_for_write(p.pm, b, h, t, p.status, row)) {  // no such page: skipped and counted
+      if (lane == 0 && p.status) atomicAdd(&p.status[2], 1u);
+      continue;
+    }
     int code[E];
     const float s = rq.run(raw, lane, code, p.status);
     if (!is_v) {
@@ -591,6 +603,9 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
 // marginal that Step 3's Lloyd-Max codebook is fitted to. Same row mapping as the K kernel; the CTA counts into a
 // histogram in shared memory and adds its non-empty bins to the caller's at the end. Zero rows are left out.
 // ---------------------------------------------------------------------------------------------------------
+// The row quantiser the histogram shares with the append kernels loads seven thresholds; the histogram has none.
+__device__ const float g_no_thresholds[7] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+
 template <int D>
 __global__ void __launch_bounds__(QA_WARPS * 32, 4) rotated_histogram_kernel(const __grid_constant__ HistogramParams p) {
   using RQ = RowQuantizer<D>;
@@ -609,7 +624,7 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 4) rotated_histogram_kernel(con
   RQ::fill_matrices(p.rot + (size_t)h * (D / 4) * 8, m_s, tid, QA_WARPS * 32);
   __syncthreads();
   RQ rq;
-  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane, m_s);
+  rq.init(p.rot + (size_t)h * (D / 4) * 8, g_no_thresholds, lane, m_s);  // (the histogram takes u itself, no codes)
   const int li = lane % LPR, sub = lane / LPR;
   const __half* src_base = p.x + (size_t)b * p.stride_b + (size_t)h * p.stride_h + li * 16;
   const int row_begin = cta_begin + warp * HIST_ROWS_PER_WARP, row_end = min(n_rows, row_begin + HIST_ROWS_PER_WARP);

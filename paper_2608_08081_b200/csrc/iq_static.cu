@@ -9,7 +9,8 @@
 //
 // In host code the name of a __device__ array is only a host-side stand-in, not a device address, so the
 // address is looked up once per device with cudaGetSymbolAddress (with that device current) and the
-// pointer is what the kernels receive.
+// pointer is what the kernels receive. The looked-up address is kept for the life of the process: it does
+// not survive a cudaDeviceReset of that device, after which this entry point must not be used again.
 #include <mutex>
 
 #include "iq_common.cuh"
@@ -48,6 +49,9 @@ int iq_decode_attention_static(const iq_shape* shape, const float* rot_dev, cons
                                const iq_cache* cache, const int32_t* seq_lens_dev, int32_t num_splits, void* out,
                                int32_t out_is_fp16, float* lse_out, uint32_t* status_dev, void* stream) {
   if (!shape) return IQ_ERR_NULL;
+  // what the merge would refuse after the decode kernel has been enqueued is refused here instead
+  if (!out) return IQ_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(out) & 15u) != 0) return IQ_ERR_ALIGN;
   if (num_splits < 1) return IQ_ERR_SHAPE;
   if (shape->batch < 0 || shape->n_q_heads <= 0 || (shape->head_dim != 128 && shape->head_dim != 256)) return IQ_ERR_SHAPE;
   // partials: acc [B][H_q][S][d] followed by (m, l) [B][H_q][S][2]

@@ -86,10 +86,13 @@ def compare_caches(w, th, gpu, ref, lens, tie_fraction_max=TIE_FRACTION_MAX):
                 rb = rc[b].reshape(w.H_kv, -1, 128 * P)[:, :nb]
                 bad = []
                 for g, j in zip(*np.nonzero(np.any(gb != rb, axis=-1))):
+                    differing = 0
                     for t in range(128 * j, min(128 * j + 128, n)):
                         if not np.array_equal(row_codes(gc, g, t), row_codes(rc, g, t)):
                             bad.append((g, t))
-                    # rows of the block that were never appended must be untouched (zero) on both sides
+                            differing += 1
+                    # the bits of the block's rows that were never appended must be untouched (as allocated) on both sides
+                    assert differing > 0, f"V block {j} of (sequence {b}, head {g}) differs only in rows that were never appended"
             for g, t in bad:
                 cg = row_codes(gc, g, t).astype(np.int64)
                 cr = row_codes(rc, g, t).astype(np.int64)
@@ -119,9 +122,14 @@ def gpu_decode(iq, torch, shape, rot, cb, q_np, cache, lens, num_splits, want_ar
                 argmax=None if ws.argmax is None else ws.argmax.cpu().numpy(), ws=ws)
 
 
-def check_decode(w, lv, q_np, gpu_res, cache_np, lens, sm_scale=0.0, argmax_tol=2e-3):
-    """Outputs within tolerance of the fp64 oracle run on the same packed cache; argmax identical wherever the
-    oracle's maximum is separated from the runner-up by more than argmax_tol, valid (a near-maximal row) otherwise."""
+ARGMAX_TIE_RTOL = 4e-6   # a different argmax row is a tie iff its fp64 score is within this (relative) of the maximum
+ARGMAX_TIE_ATOL = 2e-6   # ... plus this: the kernel's scores are fp32 values of 21-bit (integer path) or 22-bit (fp16 path) queries
+
+
+def check_decode(w, lv, q_np, gpu_res, cache_np, lens, sm_scale=0.0, argmax_tol=None):
+    """Outputs within tolerance of the fp64 oracle run on the same packed cache; argmax identical, except that a row
+    whose fp64 score ties with the maximum within the rounding of the kernel's fp32 scores is accepted (counted, and
+    at most 2 % of the heads + 1)."""
     ref = oracle.decode_attention(w.quats, lv, q_np, cache_np, lens, w.H_kv, sm_scale)
     err = np.abs(gpu_res["out"] - ref["out"])
     bound = OUT_ATOL + OUT_RTOL * np.abs(ref["out"])
@@ -133,7 +141,7 @@ def check_decode(w, lv, q_np, gpu_res, cache_np, lens, sm_scale=0.0, argmax_tol=
         assert np.all(num <= OUT_RTOL * den + 1e-6), f"relative l2 error {np.max(num / np.maximum(den, 1e-30)):.3e}"
         assert np.allclose(gpu_res["lse"][nz], ref["lse"][nz], atol=2e-3, rtol=1e-5)   # fp32 scores: relative at large |z|
     assert np.all(np.isneginf(gpu_res["lse"][~nz])) and np.all(gpu_res["out"][~nz] == 0)
-    exact = 0
+    exact = ties = 0
     if gpu_res["argmax"] is not None:
         B, H_q = ref["argmax"].shape
         for b in range(B):
@@ -144,5 +152,8 @@ def check_decode(w, lv, q_np, gpu_res, cache_np, lens, sm_scale=0.0, argmax_tol=
                     continue
                 assert lens[b] > 0 and 0 <= ga < lens[b], f"argmax {ga} outside the sequence"
                 z = oracle.scores(w.quats, lv, q_np, cache_np, b, h, int(lens[b]), w.H_kv, sm_scale)
-                assert z[ra] - z[ga] <= argmax_tol, f"argmax differs: gpu row {ga} scores {z[ga]}, oracle row {ra} scores {z[ra]}"
-    return dict(max_err=float(err.max()), margin=float(np.max(err / bound)), argmax_exact=exact, ref=ref)
+                tol = argmax_tol if argmax_tol is not None else ARGMAX_TIE_ATOL + ARGMAX_TIE_RTOL * abs(z[ra])
+                assert z[ra] - z[ga] <= tol, f"argmax differs: gpu row {ga} scores {z[ga]}, oracle row {ra} scores {z[ra]}"
+                ties += 1
+        assert ties <= 0.02 * B * H_q + 1, f"{ties} argmax ties in {B * H_q} heads"
+    return dict(max_err=float(err.max()), margin=float(np.max(err / bound)), argmax_exact=exact, argmax_ties=ties, ref=ref)

@@ -23,7 +23,7 @@ def test_library_exports_every_declared_symbol(iq):
     lib = ctypes.CDLL(iq.lib_path())
     for n in sorted(names):
         assert hasattr(lib, n), f"{n} declared in isoquant.h but not exported"
-    assert iq.iq_version() == 100
+    assert iq.iq_version() == 200 and iq.iq_format_version() == 2
     for n in sorted(names):
         assert hasattr(iq, n) or n in ("iq_shape", "iq_codebook", "iq_cache"), f"binding lacks {n}"
 
@@ -122,7 +122,25 @@ def test_argument_validation_happens_before_any_launch(iq, monkeypatch):
     assert cs(good, S=0) == -2
     assert cs(good, out=None) == -1
     assert cs(good, ao=A) == -1                                      # argmax_out without part_argmax
-    assert "binary16" in iq.iq_strerror(-4)
+    assert "binary16" in iq.iq_strerror(-4) and "8-bit grid" in iq.iq_strerror(-4)
+
+    # the no-allocation entry point: its size limit and its output pointer are checked before any CUDA call
+    def ds(shape, S=2, out=A):
+        return lib.iq_decode_attention_static(ctypes.byref(shape), A, ctypes.byref(cb), A, ctypes.byref(cache), A, S, out, 0, None, None, None)
+    assert ds(B._IqShape(64, 64, 8, 128, 1024, 3, 0.0), S=64) == -6   # 64 * 64 * 64 * 130 floats > the fixed array
+    assert ds(good, out=None) == -1
+    assert ds(good, out=A + 4) == -3
+    assert ds(good, S=0) == -2
+    assert ds(B._IqShape(1, 4, 1, 64, 1024, 3, 0.0)) == -2
+    assert lib.iq_decode_attention_static(None, A, ctypes.byref(cb), A, ctypes.byref(cache), A, 2, A, 0, None, None, None) == -1
+
+    # the host-buffer step refuses what its three parts would refuse before it enqueues the copy and the append
+    def hs(shape, cbk=cb, S=2, pa=A, out=A):
+        return lib.iq_decode_step_host(ctypes.byref(shape), A, ctypes.byref(cbk), A, A, A, A, ctypes.byref(cache), S, pa, A, out, A, 0, None, None)
+    assert hs(good, cbk=bad) == -4
+    assert hs(good, S=0) == -2
+    assert hs(good, pa=None) == -1
+    assert hs(good, out=A + 8) == -3
     assert lib.iq_make_rotation(96, 1, 0, None, A, None) == -2
     assert lib.iq_make_rotation(128, 1, 0, None, None, None) == -1
 

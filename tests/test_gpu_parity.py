@@ -436,6 +436,40 @@ def test_paged_cache_gives_the_contiguous_results(iq, torch, codebooks, d, page_
     iq.decode_step(shape, rot, cb, torch.from_numpy(w.q).cuda(), cache_bad, torch.from_numpy(now).cuda(), ws)
     torch.cuda.synchronize()
     assert int(ws.status[0].item()) & 4
+    # quantize-append through such an entry (also a negative one) writes nothing anywhere: the rows are skipped and counted
+    before = [t.clone() for t in (cache.k_codes, cache.k_scales, cache.v_codes, cache.v_scales)]
+    for entry, n_new in ((num_pages + 5, 1), (-1, 1), (-1, 200)):
+        bad = table.copy(); bad[0, 0] = entry
+        cache_bad = iq.Cache(cache.k_codes, cache.k_scales, cache.v_codes, cache.v_scales, torch.from_numpy(bad).cuda(), page_rows)
+        st2 = torch.zeros(4, dtype=torch.int32, device="cuda")
+        nn = torch.tensor([n_new, 0, 0], dtype=torch.int32, device="cuda")
+        iq.iq_quantize_append(shape, rot, cb, k, v, torch.zeros(B, dtype=torch.int32, device="cuda"), nn, n_new, cache_bad, st2)
+        torch.cuda.synchronize()
+        assert int(st2[0]) & 4 and int(st2[2]) == 2 * H_kv * min(n_new, page_rows)   # K and V rows of every KV head
+        keep = torch.ones(num_pages, dtype=torch.bool, device="cuda")
+        if n_new > page_rows:
+            keep[int(table[0, 1])] = False                                  # rows beyond the missing page have a page and are written
+        for a, bfr in zip((cache.k_codes, cache.k_scales, cache.v_codes, cache.v_scales), before):
+            assert torch.equal(a[keep], bfr[keep])
+
+
+def test_a_wait_that_nothing_completes_gives_up_and_reports(iq, torch):
+    """The decode kernel's mbarrier waits are bounded: a one-warp kernel waits on a barrier that nothing arrives at
+    (no copy, no tensor-core work in flight), gives up after its poll limit and reports IQ_STATUS_WAIT_TIMEOUT; the
+    context stays usable."""
+    import time
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    t0 = time.perf_counter()
+    iq.iq_selftest_bounded_wait(status, 256)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert int(status[0]) == 2 and int(status[1]) == 256                    # the flag, and the polls it took
+    assert dt < 1.0                                                         # 256 polls of at most 20 us each
+    status.zero_()
+    iq.iq_selftest_bounded_wait(status, 0)                                  # limit 0: the barrier is completed first
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    assert float(torch.ones(8, device="cuda").sum()) == 8.0
 
 
 def test_context_sharded_decode_on_one_gpu(iq, torch, codebooks):
@@ -779,7 +813,7 @@ def test_config4_long_context_retrieval(iq, torch, codebooks):
         assert (o @ vn) / (np.linalg.norm(o) * np.linalg.norm(vn)) > 0.9
 
 
-@pytest.mark.parametrize("B,ctx", [(1, 4096), (8, 4096), (1, 32768)])
+@pytest.mark.parametrize("B,ctx", [(1, 4096), (8, 4096), (32, 4096), (1, 32768)])
 def test_config5_small_points_in_full(iq, torch, codebooks, B, ctx):
     w = workloads.config5(B, ctx)
     lv, th = codebooks[w.d]
@@ -794,13 +828,14 @@ def test_config5_small_points_in_full(iq, torch, codebooks, B, ctx):
     print(c["max_err"], c["margin"])
 
 
-def test_full_size_bench_configuration_sampled(iq, torch, codebooks):
-    """Config 5 at B = 32, ctx = 32768 (the workload bench.py times), same launch configuration (library codebook,
-    iq_suggest_splits, no argmax). The oracle checks sampled (sequence, KV head) slabs: their packed rows are
+@pytest.mark.parametrize("name", ["config5_B32_ctx32768", "config5_B8_ctx32768"])
+def test_full_size_bench_configuration_sampled(iq, torch, codebooks, name):
+    """Config 5 at ctx = 32768, B = 32 (the workload bench.py times) and B = 8, same launch configuration (library
+    codebook, iq_suggest_splits, no argmax). The oracle checks sampled (sequence, KV head) slabs: their packed rows are
     re-quantised and every query head of the group is decoded from the GPU's own cache."""
     import bench
 
-    name = bench.DEFAULT_WORKLOAD
+    assert bench.DEFAULT_WORKLOAD == "config5_B32_ctx32768"
     B, ctx, H_q, H_kv, d = bench.WORKLOADS[name]
     st = bench.build_state(name, torch.device("cuda", 0), 0)
     shape, cb, rot, cache = st["shape"], st["cb"], st["rot"], st["cache"]

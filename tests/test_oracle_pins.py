@@ -31,6 +31,19 @@ def _rand_quats(seed, n=1):
     return q.reshape(n, 8).astype(np.float32)
 
 
+# ---------------------------------------------------------------- binary16 inputs
+def test_half_to_double_on_every_bit_pattern():
+    """Every input of both sides passes through the oracle's binary16 reader: all 65536 patterns (subnormals,
+    infinities, NaNs included) against numpy's float16 -> float64 conversion."""
+    L = oracle.lib()
+    bits = np.arange(65536, dtype=np.uint16)
+    want = bits.view(np.float16).astype(np.float64)
+    got = np.array([L.iqo_half_to_double(int(b)) for b in bits])
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan], want[~nan]) and np.array_equal(np.signbit(got[~nan]), np.signbit(want[~nan]))
+
+
 # ---------------------------------------------------------------- H_d (Eq. 2)
 @pytest.mark.parametrize("d", [4, 32, 128, 256])
 def test_hadamard_matches_library_and_is_orthogonal(d):

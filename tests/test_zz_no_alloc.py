@@ -16,7 +16,7 @@ def test_static_scratch_decode_matches_regular_path_twice(codebooks):
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     import paper_2608_08081_b200 as iq
-    from helpers import codebook_for, gpu_quantize
+    from helpers import cache_to_numpy, check_decode, codebook_for, gpu_quantize
 
     outs = []
     # two different problems back to back: the second one (fewer heads, other lengths, other split count)
@@ -48,6 +48,10 @@ def test_static_scratch_decode_matches_regular_path_twice(codebooks):
         # (and nothing else) may differ between two calls
         assert np.allclose(out.cpu().numpy(), ref.cpu().numpy(), atol=1e-5, rtol=1e-5)
         assert np.allclose(lse.cpu().numpy(), ref_lse.cpu().numpy(), atol=1e-5, rtol=1e-6)
+        # and against the fp64 oracle on the same packed cache, at the tolerance of the parity tests
+        lv, _ = codebooks[d]
+        check_decode(w, lv, w.q, dict(out=out.cpu().numpy().astype(np.float64), lse=lse.cpu().numpy().astype(np.float64), argmax=None),
+                     cache_to_numpy(cache), np.asarray(lens, np.int32))
         out16 = torch.empty((B, H_q, d), dtype=torch.float16, device="cuda")
         iq.iq_decode_attention_static(shape, rot, cb, q, cache, sl, S, out16)
         torch.cuda.synchronize()
