@@ -899,7 +899,8 @@ def test_bench_line_keeps_its_contract():
                 "data", "config", "roofline", "e2e", "gpu_launches", "clocks"):
         assert key in d, key
     assert d["steps"] == 4 and d["warmup"] == 3 and d["n_gpus"] == 1 and d["vs_baseline"] is None and d["data"] == "synthetic"
-    assert d["config"]["workload"] == "config5_B1_ctx4096" and d["gpu_launches"] == 3 * 4
+    assert d["config"]["workload"] == "config5_B1_ctx4096" and d["replays"] >= 1 and d["gpu_launches"] == 3 * 4 * d["replays"]
+    assert d["roofline"]["launches_timed"] >= 50 and d["clocks"]["samples"] >= 50
     rf = d["roofline"]
     assert rf["bound"] == "hbm" and rf["unit"] == "GB/s" and abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-3 and rf["traffic"] > 0
     assert d["e2e"]["h2d_bytes_per_step"] > 0 and d["e2e"]["d2h_bytes_per_step"] > 0 and d["e2e"]["value"] > 0
