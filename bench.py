@@ -322,7 +322,7 @@ class StepRunner:
         torch.cuda.synchronize()
         return t0.elapsed_time(t1), [a.elapsed_time(b) for a, b in evs]
 
-    def timed_region(self, min_region_s: float, max_replays: int = 400, barrier=None):
+    def timed_region(self, min_region_s: float, max_replays: int = 100000, barrier=None):
         """The timed region: the K-step graph replayed R times, each replay timed on its own (events and a synchronize
         on both sides), until the replays add up to min_region_s. With no graph: the host-launched K steps, R times.
         Returns (per-replay ms, decode-launch ms of every bracketed launch)."""
@@ -367,7 +367,7 @@ def point_summary(name: str, device, rank: int, K: int = 20, W: int = 3, min_reg
     r = StepRunner(name, device, rank, K, W)
     r.warm_up()
     r.capture()
-    per_replay, dec = r.timed_region(min_region_s, max_replays=100)
+    per_replay, dec = r.timed_region(min_region_s, max_replays=2000)
     assert int(r.ws.status[0].item()) == 0 and int(r.st["status"][0].item()) == 0, "device status flags set"
     ms_step = float(np.mean(per_replay)) / K
     step_bytes = float(np.mean(r.bytes_of_steps()))

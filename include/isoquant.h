@@ -202,8 +202,8 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
  *   part_ml        device fp32 [batch][n_q_heads][S][2] = (m, l): the slot's reference m and l = sum_j exp(z_j - m),
  *                  z_j = sm_scale * q~ . k~_j. With part_argmax, m = max_j z_j exactly; without it m is the kernel's
  *                  running reference, max_j z_j - 4 ln 2 <= m <= max_j z_j (acc and l are relative to the same m
- *                  either way). An unused slot holds (-inf, 0) and acc = 0; every slot of every head is written on
- *                  every call.
+ *                  either way). An unused slot holds (-inf, 0), and its acc is not written (the merge skips a slot
+ *                  with l = 0 without reading acc); (m, l) of every slot of every head is written on every call.
  *   part_argmax    device int32 [batch][n_q_heads][S] or NULL: row index attaining m (lowest on ties), -1 if empty.
  *   status_dev     optional (see top).
  * Arithmetic, codebook levels on an 8-bit grid (iq_int8_codebook): int8 tensor-core operands and int32

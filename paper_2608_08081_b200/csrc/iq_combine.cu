@@ -7,30 +7,34 @@ namespace iq {
 
 constexpr int CMB_WARPS = 4;
 
-// One warp per (sequence, query head). Lane l owns rotated coordinates l*E .. l*E+E-1, i.e. whole SO(4)
-// blocks, so M_b^T is applied in registers and H_d by the warp butterfly.
-template <int D>
-__global__ void __launch_bounds__(CMB_WARPS * 32) combine_kernel(const CombineParams p) {
+// WPH = 1: one warp per (sequence, query head), CMB_WARPS heads per CTA. WPH > 1 (many slots): one CTA of WPH warps
+// per head; warp w merges slots w, w + WPH, ... and warp 0 merges the warps' results. Lane l owns rotated
+// coordinates l*E .. l*E+E-1, i.e. whole SO(4) blocks, so M_b^T is applied in registers and H_d by the warp butterfly.
+template <int D, int WPH>
+__global__ void __launch_bounds__(WPH == 1 ? CMB_WARPS * 32 : WPH * 32) combine_kernel(const CombineParams p) {
   constexpr int E = D / 32;
   grid_dependency_wait();
   allow_dependent_launch();
-  const int lane = threadIdx.x & 31;
-  const int bh = blockIdx.x * CMB_WARPS + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int bh = WPH == 1 ? blockIdx.x * CMB_WARPS + warp : blockIdx.x;
   if (bh >= p.batch * p.n_q_heads) return;
   const int h = bh % p.n_q_heads;
   const int kvh = h / (p.n_q_heads / p.n_kv_heads);
   const int S = p.splits;
   const float* ml = p.part_ml + (size_t)bh * S * 2;
+  const int s0 = WPH == 1 ? 0 : warp;
 
   // the rotation block of this lane first: its loads do not depend on the partials and overlap with theirs
   float M[E / 4][4][4];
-  const float* qb = p.rot + ((size_t)kvh * (D / 4) + (size_t)lane * (E / 4)) * 8;
+  if (WPH == 1 || warp == 0) {
+    const float* qb = p.rot + ((size_t)kvh * (D / 4) + (size_t)lane * (E / 4)) * 8;
 #pragma unroll
-  for (int j = 0; j < E / 4; j++) so4_matrix<float>(qb + 8 * j, M[j]);
+    for (int j = 0; j < E / 4; j++) so4_matrix<float>(qb + 8 * j, M[j]);
+  }
 
   float m = -INFINITY;
   int best = -1;
-  for (int s = 0; s < S; s++) {
+  for (int s = s0; s < S; s += WPH) {
     const float ms = ml[2 * s], ls = ml[2 * s + 1];
     if (!(ls > 0.f)) continue;
     const int idx = p.part_argmax ? p.part_argmax[(size_t)bh * S + s] : -1;
@@ -41,7 +45,7 @@ __global__ void __launch_bounds__(CMB_WARPS * 32) combine_kernel(const CombinePa
   float v[E];
 #pragma unroll
   for (int e = 0; e < E; e++) v[e] = 0.f;
-  for (int s = 0; s < S; s++) {
+  for (int s = s0; s < S; s += WPH) {
     const float ms = ml[2 * s], ls = ml[2 * s + 1];
     if (!(ls > 0.f)) continue;
     const float w = __expf(ms - m);
@@ -51,6 +55,33 @@ __global__ void __launch_bounds__(CMB_WARPS * 32) combine_kernel(const CombinePa
     for (int e4 = 0; e4 < E; e4 += 4) {
       const float4 f = *reinterpret_cast<const float4*>(a + e4);
       v[e4] += w * f.x; v[e4 + 1] += w * f.y; v[e4 + 2] += w * f.z; v[e4 + 3] += w * f.w;
+    }
+  }
+  if constexpr (WPH > 1) {  // the warps' results (relative to their own maxima) merged by warp 0
+    __shared__ float sv[WPH][D];
+    __shared__ float sm[WPH], sl[WPH];
+    __shared__ int sb[WPH];
+#pragma unroll
+    for (int e = 0; e < E; e++) sv[warp][lane * E + e] = v[e];
+    if (lane == 0) { sm[warp] = m; sl[warp] = l; sb[warp] = best; }
+    __syncthreads();
+    if (warp != 0) return;
+    m = -INFINITY;
+    best = -1;
+    for (int w2 = 0; w2 < WPH; w2++) {
+      if (!(sl[w2] > 0.f)) continue;
+      if (sm[w2] > m) { m = sm[w2]; best = sb[w2]; }
+      else if (sm[w2] == m && sb[w2] >= 0 && (best < 0 || sb[w2] < best)) best = sb[w2];
+    }
+    l = 0.f;
+#pragma unroll
+    for (int e = 0; e < E; e++) v[e] = 0.f;
+    for (int w2 = 0; w2 < WPH; w2++) {
+      if (!(sl[w2] > 0.f)) continue;
+      const float w = __expf(sm[w2] - m);
+      l += sl[w2] * w;
+#pragma unroll
+      for (int e = 0; e < E; e++) v[e] += w * sv[w2][lane * E + e];
     }
   }
   const bool empty = !(l > 0.f);
@@ -80,12 +111,19 @@ __global__ void __launch_bounds__(CMB_WARPS * 32) combine_kernel(const CombinePa
   }
 }
 
+constexpr int CMB_WIDE = 8;  // warps per head when there are many slots
+
 cudaError_t launch_combine_splits(const CombineParams& p, int head_dim, cudaStream_t stream) {
   const int n = p.batch * p.n_q_heads;
   if (n <= 0) return cudaSuccess;
+  if (p.splits > 16) {  // many slots per head (small batches cut into many pieces): the slots of a head spread over a CTA
+    dim3 grid(n), block(CMB_WIDE * 32);
+    if (head_dim == 128) return launch_after_predecessor(combine_kernel<128, CMB_WIDE>, grid, block, 0, stream, p);
+    return launch_after_predecessor(combine_kernel<256, CMB_WIDE>, grid, block, 0, stream, p);
+  }
   dim3 grid((n + CMB_WARPS - 1) / CMB_WARPS), block(CMB_WARPS * 32);
-  if (head_dim == 128) return launch_after_predecessor(combine_kernel<128>, grid, block, 0, stream, p);
-  return launch_after_predecessor(combine_kernel<256>, grid, block, 0, stream, p);
+  if (head_dim == 128) return launch_after_predecessor(combine_kernel<128, 1>, grid, block, 0, stream, p);
+  return launch_after_predecessor(combine_kernel<256, 1>, grid, block, 0, stream, p);
 }
 
 // ------------------------------------------------------------------------------------------------

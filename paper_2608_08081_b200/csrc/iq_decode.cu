@@ -15,7 +15,7 @@
 //   Unit mode (fewer slots). Every item is cut into num_splits consecutive runs of blocks, run k reports to slot
 //   k, and the runs are dealt out to the groups of all CTAs in turn.
 // Every partial slot of every head is written on every launch: by the group that worked on it, else by the
-// control warp that is responsible for it (unused slots hold m = -inf, l = 0, acc = 0).
+// control warp that is responsible for it (unused slots hold m = -inf, l = 0; their acc is not written).
 //
 // Per block, in group g (thread r of the group = TMEM lane r):
 //   1. thread r dequantises packed K row r (its own 3d/8 bytes from the staged tile) and stores it to TMEM lane r.
@@ -105,15 +105,10 @@ static_assert(DecLayout<256>::I8_O_COL + 32 * DecLayout<256>::DJ <= DecLayout<25
 static_assert(DecLayout<128>::SMEM_BYTES <= 227 * 1024 && DecLayout<256>::SMEM_BYTES <= 227 * 1024, "shared memory overflow");
 static_assert((DecLayout<128>::THREADS + DecLayout<128>::THREADS / 32) * 4 <= DecLayout<128>::BP_BYTES, "set-up scratch must fit one B_P region");
 
-// Marks one partial slot of nh consecutive heads unused: (m, l) = (-inf, 0), acc = 0, argmax = -1. acc / ml / argmax
-// point at the slot of the first head; consecutive heads are S slots apart. Called by n_threads threads, this one t.
-// Kept out of line: it is rare, and the decode kernel's loops should stay small.
-static __device__ __noinline__ void dec_fill_slot(float* acc, float* ml, int32_t* argmax, int nh, int S, int D, int n_threads, int t) {
-  const int q = D / 4;
-  for (int idx = t; idx < nh * q; idx += n_threads) {
-    const int c4 = idx % q, h = idx / q;
-    *reinterpret_cast<float4*>(acc + (size_t)h * S * D + 4 * c4) = make_float4(0.f, 0.f, 0.f, 0.f);
-  }
+// Marks one partial slot of nh consecutive heads unused: (m, l) = (-inf, 0), argmax = -1 (the merge skips a slot with
+// l = 0 without reading its acc, which is left as it is). ml / argmax point at the slot of the first head; consecutive
+// heads are S slots apart. Thread t of the caller writes head t.
+__device__ __forceinline__ void dec_fill_slot(float* ml, int32_t* argmax, int nh, int S, int t) {
   if (t < nh) {
     ml[2 * (size_t)t * S] = -INFINITY;
     ml[2 * (size_t)t * S + 1] = 0.f;
@@ -152,7 +147,7 @@ __device__ __forceinline__ void dec_draw(const DecodeParams& p, DecWalk& w, DecD
     const int kvh = y / p.head_groups, hg = y - kvh * p.head_groups;
     const int h0 = kvh * p.group + hg * DEC_HEADS, nh = min(DEC_HEADS, p.group - hg * DEC_HEADS);
     const size_t o = ((size_t)b * p.n_q_heads + h0) * S + slot;
-    dec_fill_slot(p.part_acc + o * D, p.part_ml + 2 * o, with_argmax ? p.part_argmax + o : nullptr, nh, S, D, 32, lane);
+    dec_fill_slot(p.part_ml + 2 * o, with_argmax ? p.part_argmax + o : nullptr, nh, S, lane);
   };
   if (w.range_mode) {
     auto leave_segment = [&](bool item_ends) {
@@ -273,12 +268,12 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     h0 = kvh * p.group + hg * DEC_HEADS;
     nh = min(DEC_HEADS, p.group - hg * DEC_HEADS);
   };
-  // Partial slot `slot` of the heads of item (b, y) marked unused: (m, l) = (-inf, 0), acc = 0. n_threads threads, this one t.
-  auto fill_slot = [&](int b, int y, int slot, int n_threads, int t) {
+  // Partial slot `slot` of the heads of item (b, y) marked unused: (m, l) = (-inf, 0). Thread t writes head t.
+  auto fill_slot = [&](int b, int y, int slot, int t) {
     int kvh, h0, nh;
     item_heads(y, kvh, h0, nh);
     const size_t o = ((size_t)b * p.n_q_heads + h0) * S + slot;
-    dec_fill_slot(p.part_acc + o * D, p.part_ml + 2 * o, ARGMAX ? p.part_argmax + o : nullptr, nh, S, D, n_threads, t);
+    dec_fill_slot(p.part_ml + 2 * o, ARGMAX ? p.part_argmax + o : nullptr, nh, S, t);
   };
 
   grid_dependency_wait();  // nothing written by an earlier kernel (lengths, queries, cache rows) is read above this line
@@ -286,8 +281,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
   // sequences without cached rows belong to no range and no unit: CTA c defines their partial slots for sequences c, c + grid, ...
   for (int b = blockIdx.x; b < B; b += gridDim.x)
     if (len_of(b) == 0)
-      for (int y = 0; y < ips; y++)
-        for (int sl = 0; sl < S; sl++) fill_slot(b, y, sl, L::THREADS, tid);
+      for (int i = tid / DEC_HEADS; i < ips * S; i += L::THREADS / DEC_HEADS) fill_slot(b, i / S, i % S, tid % DEC_HEADS);
 
   // ---------------------------------------------------------------- range mode: the block sequence of the launch and this CTA's range
   long long per = 1, g0 = 0;
