@@ -232,6 +232,21 @@ int iq_combine_splits(const iq_shape* shape, const float* rot_dev, int32_t num_s
                       void* out, int32_t out_is_fp16, float* lse_out, int32_t* argmax_out, void* stream);
 
 /*
+ * The same merge over the partials of several ranks that each decoded a slice of every sequence's rows (context
+ * sharding; the paper's system is a single device, the merge is the one exchange step the method has when the context
+ * itself is spread over GPUs). The arrays hold the ranks' partials one after the other, as an all-gather into one
+ * buffer leaves them: part_acc [n_shards][batch][n_q_heads][S][head_dim], part_ml [n_shards][batch][n_q_heads][S][2],
+ * part_argmax [n_shards][batch][n_q_heads][S] or NULL; a head is merged over its n_shards * S slots in place, nothing
+ * is copied or allocated. row_offsets_dev: device int32 [n_shards][batch], the first row of rank r's slice of
+ * sequence b, added to that rank's argmax rows (NULL: the rows are taken as they are). n_shards = 1 is
+ * iq_combine_splits.
+ */
+int iq_combine_splits_sharded(const iq_shape* shape, const float* rot_dev, int32_t num_splits, int32_t n_shards,
+                              const float* part_acc, const float* part_ml, const int32_t* part_argmax,
+                              const int32_t* row_offsets_dev, void* out, int32_t out_is_fp16, float* lse_out,
+                              int32_t* argmax_out, void* stream);
+
+/*
  * Reconstruct-then-compute, first half (Figure 1, top; the execution model that Section 3 argues against and the
  * fused path replaces): rows [0, seq_lens[b]) of every (sequence, KV head) dequantised and rotated back to the
  * original space, x_hat = R^T x~ with x~_i = scale * level[code_i] / sqrt(d) (Algorithm 1 read backwards; R is

@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     Codebook,
     Shape,
     iq_combine_splits,
+    iq_combine_splits_sharded,
     iq_decode_attention,
     iq_decode_attention_static,
     iq_static_scratch_bytes,

@@ -62,6 +62,7 @@ def _load():
     lib.iq_decode_attention.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp,
                                         ctypes.POINTER(_IqCache), _vp, _i32, _vp, _vp, _vp, _vp, _vp]
     lib.iq_combine_splits.argtypes = [ctypes.POINTER(_IqShape), _vp, _i32, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
+    lib.iq_combine_splits_sharded.argtypes = [ctypes.POINTER(_IqShape), _vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _i32, _vp, _vp, _vp]
     lib.iq_static_scratch_bytes.restype = ctypes.c_size_t
     lib.iq_decode_attention_static.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp,
                                                ctypes.POINTER(_IqCache), _vp, _i32, _vp, _i32, _vp, _vp, _vp]
@@ -223,6 +224,15 @@ def iq_combine_splits(shape: Shape, rot_dev, num_splits: int, part_acc, part_ml,
     _check(_lib.iq_combine_splits(ctypes.byref(cs), _ptr(rot_dev), num_splits, _ptr(part_acc), _ptr(part_ml),
                                   _ptr(part_argmax), _ptr(out), 1 if out.dtype == torch.float16 else 0, _ptr(lse_out),
                                   _ptr(argmax_out), _stream(stream)), "iq_combine_splits")
+
+
+def iq_combine_splits_sharded(shape: Shape, rot_dev, num_splits: int, n_shards: int, part_acc, part_ml, part_argmax, row_offsets,
+                              out, lse_out=None, argmax_out=None, stream=None) -> None:
+    """Merge over the partials of n_shards ranks laid out rank after rank ([n_shards][B][H][S][..]), in place."""
+    cs = shape.c()
+    _check(_lib.iq_combine_splits_sharded(ctypes.byref(cs), _ptr(rot_dev), num_splits, n_shards, _ptr(part_acc), _ptr(part_ml),
+                                          _ptr(part_argmax), _ptr(row_offsets), _ptr(out), 1 if out.dtype == torch.float16 else 0,
+                                          _ptr(lse_out), _ptr(argmax_out), _stream(stream)), "iq_combine_splits_sharded")
 
 
 def iq_static_scratch_bytes() -> int:

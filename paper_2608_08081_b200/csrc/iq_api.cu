@@ -363,14 +363,15 @@ int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_co
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }
 
-int iq_combine_splits(const iq_shape* shape, const float* rot_dev, int32_t num_splits, const float* part_acc,
-                      const float* part_ml, const int32_t* part_argmax, void* out, int32_t out_is_fp16, float* lse_out,
-                      int32_t* argmax_out, void* stream) {
+int iq_combine_splits_sharded(const iq_shape* shape, const float* rot_dev, int32_t num_splits, int32_t n_shards,
+                              const float* part_acc, const float* part_ml, const int32_t* part_argmax,
+                              const int32_t* row_offsets_dev, void* out, int32_t out_is_fp16, float* lse_out,
+                              int32_t* argmax_out, void* stream) {
   int rc = check_shape(shape);
   if (rc) return rc;
   if (!rot_dev || !part_acc || !part_ml || !out) return IQ_ERR_NULL;
   if (argmax_out && !part_argmax) return IQ_ERR_NULL;
-  if (num_splits < 1) return IQ_ERR_SHAPE;
+  if (num_splits < 1 || n_shards < 1) return IQ_ERR_SHAPE;
   if (!aligned16(part_acc) || !aligned16(out) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
   if (shape->batch == 0) return IQ_OK;
 
@@ -386,9 +387,18 @@ int iq_combine_splits(const iq_shape* shape, const float* rot_dev, int32_t num_s
   p.n_q_heads = shape->n_q_heads;
   p.n_kv_heads = shape->n_kv_heads;
   p.splits = num_splits;
+  p.shards = n_shards;
+  p.row_offsets = row_offsets_dev;
   p.out_is_fp16 = out_is_fp16;
   const cudaError_t e = iq::launch_combine_splits(p, shape->head_dim, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
+int iq_combine_splits(const iq_shape* shape, const float* rot_dev, int32_t num_splits, const float* part_acc,
+                      const float* part_ml, const int32_t* part_argmax, void* out, int32_t out_is_fp16, float* lse_out,
+                      int32_t* argmax_out, void* stream) {
+  return iq_combine_splits_sharded(shape, rot_dev, num_splits, 1, part_acc, part_ml, part_argmax, nullptr, out, out_is_fp16,
+                                   lse_out, argmax_out, stream);
 }
 
 int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook, const iq_cache* cache,

@@ -20,8 +20,15 @@ __global__ void __launch_bounds__(WPH == 1 ? CMB_WARPS * 32 : WPH * 32) combine_
   if (bh >= p.batch * p.n_q_heads) return;
   const int h = bh % p.n_q_heads;
   const int kvh = h / (p.n_q_heads / p.n_kv_heads);
-  const int S = p.splits;
-  const float* ml = p.part_ml + (size_t)bh * S * 2;
+  const int S1 = p.splits, S = p.splits * p.shards;  // slots of one shard, of all shards
+  const size_t shard_heads = (size_t)p.batch * p.n_q_heads;
+  // slot s of this head: shard s / S1, its slot s % S1 (one shard: s itself)
+  auto slot_index = [&](int s) { return p.shards == 1 ? (size_t)bh * S1 + s : ((size_t)(s / S1) * shard_heads + bh) * S1 + (s % S1); };
+  auto slot_argmax = [&](int s, size_t o) {
+    int idx = p.part_argmax ? p.part_argmax[o] : -1;
+    if (idx >= 0 && p.row_offsets) idx += p.row_offsets[(size_t)(s / S1) * p.batch + bh / p.n_q_heads];
+    return idx;
+  };
   const int s0 = WPH == 1 ? 0 : warp;
 
   // the rotation block of this lane first: its loads do not depend on the partials and overlap with theirs
@@ -35,9 +42,10 @@ __global__ void __launch_bounds__(WPH == 1 ? CMB_WARPS * 32 : WPH * 32) combine_
   float m = -INFINITY;
   int best = -1;
   for (int s = s0; s < S; s += WPH) {
-    const float ms = ml[2 * s], ls = ml[2 * s + 1];
+    const size_t o = slot_index(s);
+    const float ms = p.part_ml[2 * o], ls = p.part_ml[2 * o + 1];
     if (!(ls > 0.f)) continue;
-    const int idx = p.part_argmax ? p.part_argmax[(size_t)bh * S + s] : -1;
+    const int idx = slot_argmax(s, o);
     if (ms > m) { m = ms; best = idx; }
     else if (ms == m && idx >= 0 && (best < 0 || idx < best)) best = idx;
   }
@@ -46,11 +54,12 @@ __global__ void __launch_bounds__(WPH == 1 ? CMB_WARPS * 32 : WPH * 32) combine_
 #pragma unroll
   for (int e = 0; e < E; e++) v[e] = 0.f;
   for (int s = s0; s < S; s += WPH) {
-    const float ms = ml[2 * s], ls = ml[2 * s + 1];
+    const size_t o = slot_index(s);
+    const float ms = p.part_ml[2 * o], ls = p.part_ml[2 * o + 1];
     if (!(ls > 0.f)) continue;
     const float w = __expf(ms - m);
     l += ls * w;
-    const float* a = p.part_acc + ((size_t)bh * S + s) * D + lane * E;
+    const float* a = p.part_acc + o * D + lane * E;
 #pragma unroll
     for (int e4 = 0; e4 < E; e4 += 4) {
       const float4 f = *reinterpret_cast<const float4*>(a + e4);
@@ -116,7 +125,7 @@ constexpr int CMB_WIDE = 8;  // warps per head when there are many slots
 cudaError_t launch_combine_splits(const CombineParams& p, int head_dim, cudaStream_t stream) {
   const int n = p.batch * p.n_q_heads;
   if (n <= 0) return cudaSuccess;
-  if (p.splits > 16) {  // many slots per head (small batches cut into many pieces): the slots of a head spread over a CTA
+  if (p.splits * p.shards > 16) {  // many slots per head (small batches cut into many pieces): the slots of a head spread over a CTA
     dim3 grid(n), block(CMB_WIDE * 32);
     if (head_dim == 128) return launch_after_predecessor(combine_kernel<128, CMB_WIDE>, grid, block, 0, stream, p);
     return launch_after_predecessor(combine_kernel<256, CMB_WIDE>, grid, block, 0, stream, p);

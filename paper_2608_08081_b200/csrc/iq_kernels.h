@@ -95,6 +95,11 @@ struct CombineParams {
   float* lse;
   int32_t* argmax;
   int batch, n_q_heads, n_kv_heads, splits, out_is_fp16;
+  // Context sharding: the partials of `shards` ranks laid out rank after rank (each [batch][n_q_heads][splits][..]);
+  // a head then has shards * splits slots. row_offsets [shards][batch] (or nullptr) turns a shard's argmax rows into
+  // rows of the whole sequence. shards = 1 is the plain layout.
+  int shards;
+  const int32_t* row_offsets;
 };
 cudaError_t launch_combine_splits(const CombineParams& p, int head_dim, cudaStream_t stream);
 

@@ -475,7 +475,8 @@ def test_a_wait_that_nothing_completes_gives_up_and_reports(iq, torch):
 def test_context_sharded_decode_on_one_gpu(iq, torch, codebooks):
     """The context-sharded path with the two ranks' work done one after the other on one GPU: rows [0, 256) and
     [256, T) of every sequence in two caches, the fused decode over each, the partials laid out as the all-gather
-    lays them out (rank-major along the split axis, argmax rows made global), one merge: the unsharded result. Then
+    lays them out (rank after rank, argmax rows local to the slices, the slices' first rows beside them), one merge
+    in place: the unsharded result. Then
     sharded_decode_step itself under a one-rank process group: the same as the plain step."""
     import torch.distributed as dist
     from paper_2608_08081_b200 import sharded
@@ -498,15 +499,16 @@ def test_context_sharded_decode_on_one_gpu(iq, torch, codebooks):
                               torch.zeros(B, dtype=torch.int32, device="cuda"), torch.from_numpy(my).cuda(), hi - lo, cache, status)
         ws = iq.DecodeWorkspace(shape, S, want_argmax=True)
         iq.iq_decode_attention(shape, rot, cb, q, cache, torch.from_numpy(my).cuda(), S, ws.part_acc, ws.part_ml, ws.part_argmax, ws.status)
-        am = torch.where(ws.part_argmax >= 0, ws.part_argmax + lo, ws.part_argmax)
-        parts.append((ws.part_acc.clone(), ws.part_ml.clone(), am, cache, my, ws))
-    acc = torch.cat([p[0] for p in parts], dim=2)
-    ml = torch.cat([p[1] for p in parts], dim=2)
-    am = torch.cat([p[2] for p in parts], dim=2)
+        parts.append((ws.part_acc.clone(), ws.part_ml.clone(), ws.part_argmax.clone(), cache, my, ws, lo))
+    # the buffers as an all-gather into one tensor leaves them: rank after rank, argmax rows local to each slice
+    acc = torch.stack([p[0] for p in parts])
+    ml = torch.stack([p[1] for p in parts])
+    am = torch.stack([p[2] for p in parts])
+    offs = torch.tensor([[p[6]] * B for p in parts], dtype=torch.int32, device="cuda")
     out = torch.empty((B, H_q, d), dtype=torch.float32, device="cuda")
     lse = torch.empty((B, H_q), dtype=torch.float32, device="cuda")
     amx = torch.empty((B, H_q), dtype=torch.int32, device="cuda")
-    iq.iq_combine_splits(shape, rot, 2 * S, acc, ml, am, out, lse, amx)
+    iq.iq_combine_splits_sharded(shape, rot, S, 2, acc, ml, am, offs, out, lse, amx)
     torch.cuda.synchronize()
     full = oracle.new_cache(B, H_kv, d, t_cap)
     oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), lens, full)
@@ -515,9 +517,13 @@ def test_context_sharded_decode_on_one_gpu(iq, torch, codebooks):
     # the library's function under a process group of one rank
     if not dist.is_initialized():
         dist.init_process_group("gloo", init_method="tcp://127.0.0.1:29557", rank=0, world_size=1)
-    _, _, _, cache0, my0, ws0 = parts[0]
-    o1, l1, a1 = sharded.sharded_decode_step(iq, shape, rot, cb, q, cache0, torch.from_numpy(my0).cuda(), ws0,
-                                             row_offset=torch.zeros(B, dtype=torch.int32, device="cuda"))
+    _, _, _, cache0, my0, ws0, _ = parts[0]
+    bufs = sharded.ShardedBuffers(B, H_q, S, d, 1, True, "cuda")
+    bufs.set_row_offsets(torch.zeros(B, dtype=torch.int32, device="cuda"))
+    free_before = torch.cuda.mem_get_info()[0]
+    o1, l1, a1 = sharded.sharded_decode_step(iq, shape, rot, cb, q, cache0, torch.from_numpy(my0).cuda(), ws0, bufs)
+    o1, a1 = o1.clone(), a1.clone()
+    assert torch.cuda.mem_get_info()[0] >= free_before - (4 << 20)                   # (the clones; the step itself takes nothing)
     iq.decode_step(shape, rot, cb, q, cache0, torch.from_numpy(my0).cuda(), ws0)
     torch.cuda.synchronize()
     assert torch.allclose(o1, ws0.out, atol=1e-5) and torch.equal(a1, ws0.argmax)

@@ -93,8 +93,10 @@ for b in range(B):
 acc = torch.from_numpy((r["o_rot"] * l[:, :, None]).astype(np.float32)).reshape(B, H_q, S, d)
 ml = torch.from_numpy(np.stack([m, l], -1).astype(np.float32)).reshape(B, H_q, S, 2)
 am = torch.from_numpy(r["argmax"].astype(np.int32)).reshape(B, H_q, S)
-off = torch.full((B,), lo, dtype=torch.int32)
-g_acc, g_ml, g_am = sharded.gather_partials(acc, ml, am, off)
+bufs = sharded.ShardedBuffers(B, H_q, S, d, world, True, "cpu")             # allocated once; the step below allocates nothing
+bufs.set_row_offsets(torch.full((B,), lo, dtype=torch.int32))
+bufs.gather(acc, ml, am)
+g_acc, g_ml, g_am = bufs.slot_major()
 dist.barrier(); dist.destroy_process_group()
 merged = oracle.combine_splits(w.quats, g_acc.numpy(), g_ml.numpy(), g_am.numpy(), H_kv)
 full = oracle.new_cache(B, H_kv, d, workloads.cap128(T))
