@@ -188,7 +188,10 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
  * Fused decode step on the packed cache (Appendix A; Table 2, kernels A-C), split over the context.
  *   q              device binary16 [batch][n_q_heads][head_dim], 16-byte aligned; not quantised.
  *   seq_lens_dev   device int32 [batch]: rows 0 .. len-1 of each sequence are attended to (clamped to
- *                  [0, t_cap]); the row appended last is attended to like any other.
+ *                  [0, t_cap]); the row appended last is attended to like any other. The lengths are read while the
+ *                  kernel that precedes the call on the stream may still be finishing (the launch overlaps it): they
+ *                  must have been written before that kernel started (by the host, a copy, or earlier work). No kernel
+ *                  of this library writes them. Everything else is read after that kernel has completed.
  *   num_splits     S >= 1: partial slots per (sequence, head). Every cached row of a sequence is covered by exactly one
  *                  slot of each head; which rows a slot covers is the library's choice, and a slot's rows need not be
  *                  consecutive. With S >= 2 G (G = 4 workers per SM at head_dim 128, 2 at 256) the launch is balanced

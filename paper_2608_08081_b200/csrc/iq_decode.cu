@@ -38,6 +38,7 @@ constexpr int DEC_GROUP_THREADS = 128;  // 4 warps: dequantisation, softmax, acc
 constexpr int DEC_HDR_BYTES = 4096;    // barriers, TMEM base, work counter, block descriptors, scratch
 constexpr int DEC_NPRE = 4;             // query operands prepared at the start of a CTA: those of its range's first segments
 constexpr int DEC_PRE_BAR = 9;          // named barrier of all compute threads (used while those operands are built)
+constexpr int DEC_SEG_COST = 8;          // what an item entering a CTA's range costs the CTA, in blocks (range partition)
 constexpr float DEC_RAISE_MARGIN = 3.0f;  // log2 units a raised reference is put above the block's maximum
 constexpr float DEC_MAX_SLACK = 4.0f;  // log2 units a score may exceed the running reference before it is raised
 #ifndef IQ_SLACK_I8
@@ -103,7 +104,7 @@ static_assert(DecLayout<256>::V_COL + 32 * DecLayout<256>::DJ <= DecLayout<256>:
 static_assert(DecLayout<128>::I8_O_COL + 32 * DecLayout<128>::DJ <= DecLayout<128>::GROUP_COLS, "TMEM group overflow");
 static_assert(DecLayout<256>::I8_O_COL + 32 * DecLayout<256>::DJ <= DecLayout<256>::GROUP_COLS, "TMEM group overflow");
 static_assert(DecLayout<128>::SMEM_BYTES <= 227 * 1024 && DecLayout<256>::SMEM_BYTES <= 227 * 1024, "shared memory overflow");
-static_assert((DecLayout<128>::THREADS + DecLayout<128>::THREADS / 32) * 4 <= DecLayout<128>::BP_BYTES, "set-up scratch must fit one B_P region");
+static_assert((2 * DecLayout<128>::THREADS + DecLayout<128>::THREADS / 32) * 4 <= DecLayout<128>::BP_BYTES + DecLayout<128>::STAGE_BYTES, "set-up scratch must fit group 0's B_P region and first stage");
 
 // Marks one partial slot of nh consecutive heads unused: (m, l) = (-inf, 0), argmax = -1 (the merge skips a slot with
 // l = 0 without reading its acc, which is left as it is). ml / argmax point at the slot of the first head; consecutive
@@ -209,6 +210,8 @@ __device__ __forceinline__ void dec_draw(const DecodeParams& p, DecWalk& w, DecD
 struct DecStart {
   int b, y, len, piece;  // sequence, item within it, rows of the sequence, which piece of the item the range starts in
   long long item_g;     // launch-wide index of block 0 of that item (<= the range's first block)
+  long long g0;         // launch-wide index of the range's first block
+  int count, pad;       // blocks of the range
 };
 
 template <int D, bool ARGMAX, bool I8>
@@ -252,8 +255,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
   uint8_t* bq = bq_pre + L::PRE_BYTES + grp * L::GROUP_SMEM;                 // B_Q: (n, i) MN-major, this group's own
   uint8_t* bp = bq + L::BQ_BYTES;                            // B_P: (n, row) MN-major
   uint8_t* stages = bp + L::BP_BYTES;
-  // Set-up scratch in group 0's staging area: [THREADS] blocks per slice of the batch, then the per-warp maxima.
-  // It is last read before the barrier that ends the set-up.
+  // Set-up scratch in group 0's B_P region and first stage: [THREADS] blocks per slice of the batch, the per-warp maxima,
+  // [THREADS] non-empty sequences per slice. It is last read before the barrier that ends the set-up.
   int* scan_s = reinterpret_cast<int*>(smem + DEC_HDR_BYTES + L::PRE_BYTES + L::BQ_BYTES);
 
   const int S = p.splits;
@@ -276,68 +279,95 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     dec_fill_slot(p.part_ml + 2 * o, ARGMAX ? p.part_argmax + o : nullptr, nh, S, t);
   };
 
-  grid_dependency_wait();  // nothing written by an earlier kernel (lengths, queries, cache rows) is read above this line
-
-  // sequences without cached rows belong to no range and no unit: CTA c defines their partial slots for sequences c, c + grid, ...
-  for (int b = blockIdx.x; b < B; b += gridDim.x)
-    if (len_of(b) == 0)
-      for (int i = tid / DEC_HEADS; i < ips * S; i += L::THREADS / DEC_HEADS) fill_slot(b, i / S, i % S, tid % DEC_HEADS);
+  // Everything up to grid_dependency_wait() below runs while the kernel before this one on the stream may still be
+  // running (programmatic dependent launch): it reads seq_lens only -- which no kernel of this library writes and the
+  // caller must have written before that kernel started -- and writes nothing outside shared and tensor memory.
 
   // ---------------------------------------------------------------- range mode: the block sequence of the launch and this CTA's range
-  long long per = 1, g0 = 0;
-  int count = 0;  // blocks of this CTA's range
+  // The ranges are cut at equal COST, not at equal block counts: a block costs 1 and every item a range enters costs
+  // DEC_SEG_COST more (its groups close one partial and open another: measured at 8 - 10 block times per segment and
+  // CTA). Block blk of item y of sequence b (nb blocks per item, ips items) sits at cost position
+  //   C = C_b + y (nb + W) + W + blk,   C_b = sum over the non-empty sequences before b of ips (nb + W),
+  // strictly increasing along the block sequence; CTA c owns the blocks with c * cper <= C < (c + 1) * cper.
+  long long g0 = 0;
+  int count = 0;  // blocks of this CTA's range (read from shared memory after the set-up barrier)
   if (range_mode) {
+    constexpr long long W = DEC_SEG_COST;
+    int* cnt_s = scan_s + L::THREADS + L::THREADS / 32;  // [THREADS] non-empty sequences per slice of the batch
     const int per_thread = (B + L::THREADS - 1) / L::THREADS;
     {
-      int sum = 0, mx = 0;
+      int sum = 0, mx = 0, cnt = 0;
       for (int b = tid * per_thread; b < min(B, (tid + 1) * per_thread); b++) {
         const int n = nb_of(b);
         sum += n;
+        cnt += n > 0;
         mx = max(mx, n);
       }
       scan_s[tid] = sum;
+      cnt_s[tid] = cnt;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(FULL, mx, o));
       if (lane == 0) scan_s[L::THREADS + warp] = mx;
     }
     __syncthreads();
-    long long n_total;
+    long long c_total, n_cols;  // cost of the whole launch; blocks per item column (all sequences)
     int nb_max = 0;
     {
-      int v = 0;
-      for (int i = lane; i < L::THREADS; i += 32) v += scan_s[i];
+      int v = 0, c = 0;
+      for (int i = lane; i < L::THREADS; i += 32) { v += scan_s[i]; c += cnt_s[i]; }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
-      n_total = (long long)v * ips;
+      for (int o = 16; o > 0; o >>= 1) { v += __shfl_xor_sync(FULL, v, o); c += __shfl_xor_sync(FULL, c, o); }
+      c_total = ((long long)v + W * c) * ips;
+      n_cols = v;
       for (int i = 0; i < L::THREADS / 32; i++) nb_max = max(nb_max, scan_s[L::THREADS + i]);
     }
-    per = (n_total + gridDim.x - 1) / gridDim.x;
-    per = max(per, (long long)((nb_max - 1) / (S / NG - 1) + 1));  // an item then spans at most S / NG ranges
-    per = max(per, 1ll);
-    g0 = (long long)blockIdx.x * per;
-    if (g0 >= n_total) return;
-    count = (int)min(per, n_total - g0);
-    if (tid == 0) {  // the item that holds block g0
-      long long before = 0;  // blocks (per item column) of the sequences before b
-      int t = 0;
-      while (t < L::THREADS - 1 && (before + scan_s[t]) * ips <= g0) { before += scan_s[t]; t++; }
-      int b = t * per_thread;
-      int nb = (b < B) ? nb_of(b) : 0;
-      while (b < B - 1 && (before + nb) * ips <= g0) { before += nb; b++; nb = nb_of(b); }
-      const long long r = g0 - before * ips;  // offset inside sequence b's blocks (nb per item, ips items)
+    long long cper = (c_total + gridDim.x - 1) / gridDim.x;
+    cper = max(cper, (long long)((nb_max + W - 1) / (S / NG - 1) + 1));  // an item then spans at most S / NG ranges
+    cper = max(cper, W + 1);                                              // and no range between two ranges of blocks is empty
+    const long long t_lo = (long long)blockIdx.x * cper;
+    if (t_lo >= c_total) return;
+    if (tid == 0) {
+      // the first block at or after cost position t: its sequence, item, block, and launch-wide block index
+      auto locate = [&](long long t, int& b, int& nb, int& y, int& blk, long long& before_nb, long long& c_b) {
+        before_nb = 0;  // blocks (per item column) of the sequences before b
+        long long before_cnt = 0;
+        int i = 0;
+        if (t >= c_total) { b = B; nb = 0; y = 0; blk = 0; before_nb = n_cols; c_b = c_total; return; }  // past the last block
+        while (i < L::THREADS - 1 && ((before_nb + scan_s[i]) + W * (before_cnt + cnt_s[i])) * ips <= t) { before_nb += scan_s[i]; before_cnt += cnt_s[i]; i++; }
+        b = i * per_thread;
+        c_b = (before_nb + W * before_cnt) * ips;
+        for (;; b++) {
+          nb = (b < B) ? nb_of(b) : 0;
+          if (b >= B) break;
+          if (nb == 0) continue;
+          if (c_b + (long long)ips * (nb + W) > t) break;
+          c_b += (long long)ips * (nb + W);
+          before_nb += nb;
+        }
+        if (b >= B) { y = 0; blk = 0; return; }  // past the last block
+        const long long rel = t - c_b;
+        y = (int)(rel / (nb + W));
+        const long long r = rel - (long long)y * (nb + W);
+        blk = (int)max(0ll, r - W);
+      };
+      int b, nb, y, blk, b1, nb1, y1, blk1;
+      long long before, c_b, before1, c_b1;
+      locate(t_lo, b, nb, y, blk, before, c_b);
+      locate(t_lo + cper, b1, nb1, y1, blk1, before1, c_b1);
       DecStart s0;
       s0.b = b;
-      s0.len = (b < B) ? len_of(b) : 0;
-      s0.y = (int)(r / nb);
-      s0.item_g = before * ips + (long long)s0.y * nb;
-      s0.piece = (int)((long long)blockIdx.x - s0.item_g / per);  // CTAs between the item's first block and this range
+      s0.len = len_of(b);
+      s0.y = y;
+      s0.item_g = before * ips + (long long)y * nb;
+      s0.g0 = s0.item_g + blk;
+      s0.count = (int)((b1 < B ? before1 * ips + (long long)y1 * nb1 + blk1 : before1 * ips) - s0.g0);
+      s0.piece = (int)((long long)blockIdx.x - (c_b + (long long)y * (nb + W) + W) / cper);  // CTAs since the one that holds the item's first block
       *start_s = s0;
       *next_s = 0;
       // the range's first segments: their query operands are prepared once for all groups
       int np = 0;
       long long item_g = s0.item_g;
-      int y = s0.y;
-      while (np < DEC_NPRE && b < B && max(item_g, g0) < g0 + count) {
+      while (np < DEC_NPRE && b < B && max(item_g, s0.g0) < s0.g0 + s0.count) {
         pre_tab[np++] = make_int2(b, y);
         item_g += nb;
         if (++y == ips) {
@@ -368,9 +398,17 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::);
   }
+  grid_dependency_wait();  // queries, cache rows and the partial buffers are not touched above this line
+
+  // sequences without cached rows belong to no range and no unit: CTA c defines their partial slots for sequences c, c + grid, ...
+  for (int b = blockIdx.x; b < B; b += gridDim.x)
+    if (len_of(b) == 0)
+      for (int i = tid / DEC_HEADS; i < ips * S; i += L::THREADS / DEC_HEADS) fill_slot(b, i / S, i % S, tid % DEC_HEADS);
+
   tc_fence_before();
   __syncthreads();  // the last CTA-wide barrier before the end of the kernel
   tc_fence_after();
+  if (range_mode) { g0 = start_s->g0; count = start_s->count; }
   const uint32_t tmem_base = tmem_slot[0];
   const uint32_t tmem_g = tmem_base + (uint32_t)(grp * L::GROUP_COLS);        // this group's columns
   const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;                // this warp's 32 TMEM lanes
