@@ -321,6 +321,10 @@ int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_co
   if (!grid8 && (rc = check_codebook(codebook, true))) return rc;
   if ((rc = check_cache(cache, shape))) return rc;
   if (num_splits < 1 || num_splits > 65535) return IQ_ERR_SHAPE;
+  {  // the kernel counts (sequence, KV head group, slot) units and 128-row blocks in 31 bits
+    const long long items = (long long)shape->batch * shape->n_kv_heads * ((shape->n_q_heads / shape->n_kv_heads + iq::DEC_HEADS - 1) / iq::DEC_HEADS);
+    if (items * num_splits >= (1ll << 31) || items * (shape->t_cap / iq::DEC_BLOCK_TOKENS) >= (1ll << 31)) return IQ_ERR_LIMIT;
+  }
   if (!aligned16(q) || !aligned16(part_acc) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
   if (shape->batch == 0) return IQ_OK;
 

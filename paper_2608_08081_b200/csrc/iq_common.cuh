@@ -156,7 +156,7 @@ inline cudaError_t launch_after_predecessor(void (*kernel)(Params), dim3 grid, d
 // row index of a block's first row, times the row size, is also where its token-transposed V records start.
 __device__ __forceinline__ size_t cache_row(const PageMap& m, int b, int g, long long t, uint32_t* status) {
   if (m.table == nullptr) return ((size_t)b * m.n_kv_heads + g) * (size_t)m.t_cap + (size_t)t;
-  const int j = (int)(t / m.page_rows);
+  const int j = (int)t / m.page_rows;  // (t < t_cap: 32-bit arithmetic)
   int page = m.table[(size_t)b * (m.t_cap / m.page_rows) + j];
   if ((unsigned)page >= (unsigned)m.num_pages) {  // never turned into an address: flagged and read as page 0
     if (status) atomicOr(&status[0], IQ_STATUS_BAD_PAGE);
@@ -170,7 +170,7 @@ __device__ __forceinline__ size_t cache_row(const PageMap& m, int b, int g, long
 // the caller skips the row and counts it.
 __device__ __forceinline__ bool cache_row_for_write(const PageMap& m, int b, int g, long long t, uint32_t* status, size_t& row) {
   if (m.table != nullptr) {
-    const int page = m.table[(size_t)b * (m.t_cap / m.page_rows) + (int)(t / m.page_rows)];
+    const int page = m.table[(size_t)b * (m.t_cap / m.page_rows) + (int)t / m.page_rows];
     if ((unsigned)page >= (unsigned)m.num_pages) {
       if (status) atomicOr(&status[0], IQ_STATUS_BAD_PAGE);
       return false;

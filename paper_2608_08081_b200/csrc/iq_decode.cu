@@ -126,7 +126,7 @@ struct DecWalk {
   int sidx, n_pre;                    // ordinal of the segment in the range; segments below n_pre have a prepared query operand
   long long item_g, g0, g_end;  // launch-wide index of block 0 of the item; the range [g0, g_end)
   // unit mode: run k of item i is unit i * S + k; the walk is in run uk of item (ub, uy), at block ublk of [.., uhi)
-  long long n_units, unit_step, unit;
+  int n_units, unit_step, unit;  // (the host refuses launches whose unit count does not fit 31 bits)
   int ub, uy, uk, ublk, uhi, unew, ulen;
 };
 struct DecDrawn {
@@ -189,10 +189,10 @@ __device__ __forceinline__ void dec_draw(const DecodeParams& p, DecWalk& w, DecD
   } else {
     while (w.ublk >= w.uhi) {  // the next run with blocks
       if (w.unit >= w.n_units) { d.kind = 1; return; }
-      const long long item = w.unit / S;
-      const int k = (int)(w.unit - item * S);
-      w.unit += w.unit_step;
-      const int b = (int)(item / w.ips), y = (int)(item - (long long)b * w.ips);
+      const int item = w.unit / S;
+      const int k = w.unit - item * S;
+      w.unit = (w.unit_step > w.n_units - w.unit) ? w.n_units : w.unit + w.unit_step;  // (no overflow)
+      const int b = item / w.ips, y = item - b * w.ips;
       const int len = len_of(b), nb = (len + TB - 1) / TB;
       if (nb == 0) continue;  // an empty sequence: its slots were written during the set-up
       const int cb = (nb + S - 1) / S, lo = k * cb, hi = min(nb, lo + cb);
@@ -204,6 +204,68 @@ __device__ __forceinline__ void dec_draw(const DecodeParams& p, DecWalk& w, DecD
   }
   d.row0 = cache_row(p.pm, d.b, d.y / p.head_groups, (long long)d.blk * TB, p.status);
   d.kind = 0;
+}
+
+// d1 (App. A): q~ = R q of one head times 1/sqrt(d), as the lane's E = D / 32 coordinates (lane l holds l E .. l E + E - 1).
+// Out of line, like dec_write_operand: both run once per segment at most, and the kernel's code should stay small
+// (a launch over a short context spends a good part of its time fetching instructions it executes once).
+template <int D>
+struct DecHeadCoords { float v[D / 32]; };
+template <int D>
+static __device__ __noinline__ DecHeadCoords<D> dec_rotate_head(const __half* q_head, const float* rot_head, int lane) {
+  constexpr int E = D / 32;
+  DecHeadCoords<D> r;
+  if (q_head == nullptr) {
+#pragma unroll
+    for (int e = 0; e < E; e++) r.v[e] = 0.f;
+    return r;
+  }
+  float M[E / 4][4][4];
+  const float* qb = rot_head + (size_t)lane * (E / 4) * 8;
+#pragma unroll
+  for (int j = 0; j < E / 4; j++) so4_matrix<float>(qb + 8 * j, M[j]);
+  const __half* src = q_head + lane * E;
+#pragma unroll
+  for (int e = 0; e < E; e++) r.v[e] = __half2float(src[e]);
+  wht_warp<float, E>(r.v, lane);
+  so4_apply<float, E, false>(M, r.v);
+  const float inv_root_d = rsqrtf((float)D);
+#pragma unroll
+  for (int e = 0; e < E; e++) r.v[e] *= inv_root_d;
+  return r;
+}
+// Column block hh (one head) of the operand B_Q in buffer `dst`. Integer path: q~ as three balanced base-128 digits
+// (int8) of round(q~ * (2^20 - 1) / qmax), qmax = max |q~| over the item's heads: one scale for all heads, so that
+// the score read-back needs a single factor. (Two base-256 digits would halve the read-back, but 16 bits are not
+// enough for lse at the logit magnitudes of outlier rows.) fp16 path: q~ as hi + lo.
+template <int D, bool I8>
+static __device__ __noinline__ void dec_write_operand(uint8_t* dst, int hh, DecHeadCoords<D> c, float qmax, int lane) {
+  constexpr int E = D / 32;
+  if constexpr (I8) {
+    const float qs = qmax > 0.f ? 1048575.0f / qmax : 0.f;
+#pragma unroll
+    for (int e = 0; e < E; e++) {
+      const int Q = __float2int_rn(c.v[e] * qs);
+      const int d2 = (Q + 8192) >> 14;
+      const int r = Q - (d2 << 14);
+      const int d1 = (r + 64) >> 7;
+      const int d0 = r - (d1 << 7);
+      const int i = lane * E + e;  // contraction index = rotated coordinate; column n = 4 * head + digit
+      const uint32_t word = (uint32_t)(d0 & 0xff) | ((uint32_t)(d1 & 0xff) << 8) | ((uint32_t)(d2 & 0xff) << 16);
+      *reinterpret_cast<uint32_t*>(dst + 4 * (hh & 3) + (hh >> 2) * ((D / 8) * 128) + (i & 7) * 16 + (i >> 3) * 128) = word;
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < E; e++) {
+      const float x = c.v[e];
+      const __half xh = __float2half_rn(x);
+      const __half xl = __float2half_rn(x - __half2float(xh));
+      const int i = lane * E + e;  // contraction index = rotated coordinate
+      const int off = (i & 7) * 16 + (i >> 3) * 128;
+      *reinterpret_cast<__half*>(dst + hh * 2 + off) = xh;                  // n = head (hi part)
+      *reinterpret_cast<__half*>(dst + hh * 2 + (D / 8) * 128 + off) = xl;  // n = 8 + head (lo part)
+    }
+  }
 }
 
 // Where the CTA's range starts (thread 0, set-up).
@@ -350,10 +412,18 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
         const long long r = rel - (long long)y * (nb + W);
         blk = (int)max(0ll, r - W);
       };
-      int b, nb, y, blk, b1, nb1, y1, blk1;
-      long long before, c_b, before1, c_b1;
-      locate(t_lo, b, nb, y, blk, before, c_b);
-      locate(t_lo + cper, b1, nb1, y1, blk1, before1, c_b1);
+      int b = 0, nb = 0, y = 0, blk = 0, b1 = 0, nb1 = 0, y1 = 0, blk1 = 0;
+      long long before = 0, c_b = 0, before1 = 0, c_b1 = 0;
+#pragma unroll 1
+      for (int k = 0; k < 2; k++) {  // (a loop so that the search exists once in the code)
+        b = b1; nb = nb1; y = y1; blk = blk1; before = before1; c_b = c_b1;
+        locate(k == 0 ? t_lo + cper : t_lo, b1, nb1, y1, blk1, before1, c_b1);
+      }
+      {  // the first pass found the end of the range, the second its start: swap them into place
+        int ti; long long tl;
+        ti = b; b = b1; b1 = ti; ti = nb; nb = nb1; nb1 = ti; ti = y; y = y1; y1 = ti; ti = blk; blk = blk1; blk1 = ti;
+        tl = before; before = before1; before1 = tl; tl = c_b; c_b = c_b1; c_b1 = tl;
+      }
       DecStart s0;
       s0.b = b;
       s0.len = len_of(b);
@@ -439,9 +509,9 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     wk.n_pre = *n_pre_s;
     if (range_mode) { wk.b = start_s->b; wk.y = start_s->y; wk.len = start_s->len; wk.nb = (wk.len + TB - 1) / TB; wk.piece = start_s->piece; wk.item_g = start_s->item_g; }
     else { wk.b = wk.y = wk.nb = wk.len = wk.piece = 0; wk.item_g = 0; }
-    wk.n_units = (long long)B * ips * S;
-    wk.unit_step = (long long)NG * gridDim.x;
-    wk.unit = (long long)grp * gridDim.x + blockIdx.x;
+    wk.n_units = B * ips * S;
+    wk.unit_step = NG * (int)gridDim.x;
+    wk.unit = min(wk.n_units, grp * (int)gridDim.x + (int)blockIdx.x);
     wk.ub = wk.uy = wk.uk = wk.ublk = wk.uhi = wk.unew = wk.ulen = 0;
     // The next block is drawn (shared counter; with a paged cache also its block-table entry, a load from global
     // memory) while the compute warps are busy with the softmax of the current one, and staged after the value MMAs.
@@ -554,24 +624,11 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     int nbk = 0;       // blocks this group has processed (phases of k_ready, s_bar, p_ready, o_bar)
     int* seg_id = reinterpret_cast<int*>(smem + L::OFF_SEGID + 16 * grp);  // the open segment: (sequence, item, slot); kept in shared memory between open and close
 
-    // ---- d1 (App. A): q~ = R q of one head, as the lane's E coordinates (lane l holds l E .. l E + E - 1), times 1/sqrt(d)
     auto rotate_head = [&](int b, int kvh, int h_abs, bool present, float (&v)[E]) {
-      if (present) {
-        float M[E / 4][4][4];
-        const float* qb = p.rot + ((size_t)kvh * (D / 4) + (size_t)lane * (E / 4)) * 8;
+      const DecHeadCoords<D> c = dec_rotate_head<D>(present ? p.q + ((size_t)b * p.n_q_heads + h_abs) * D : nullptr,
+                                                    p.rot + (size_t)kvh * (D / 4) * 8, lane);
 #pragma unroll
-        for (int j = 0; j < E / 4; j++) so4_matrix<float>(qb + 8 * j, M[j]);
-        const __half* src = p.q + ((size_t)b * p.n_q_heads + h_abs) * D + lane * E;
-#pragma unroll
-        for (int e = 0; e < E; e++) v[e] = __half2float(src[e]);
-        wht_warp<float, E>(v, lane);
-        so4_apply<float, E, false>(M, v);
-#pragma unroll
-        for (int e = 0; e < E; e++) v[e] *= inv_root_d;
-      } else {
-#pragma unroll
-        for (int e = 0; e < E; e++) v[e] = 0.f;
-      }
+      for (int e = 0; e < E; e++) v[e] = c.v[e];
     };
     auto abs_max = [&](const float (&v)[E]) {
       float m = 0.f;
@@ -579,36 +636,11 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
       for (int e = 0; e < E; e++) m = fmaxf(m, fabsf(v[e]));
       return warp_max(m);
     };
-    // Column block hh (one head) of the operand B_Q in buffer `dst`. Integer path: q~ as three balanced base-128 digits
-    // (int8) of round(q~ * (2^20 - 1) / qmax), qmax = max |q~| over the item's heads: one scale for all heads, so that
-    // the score read-back needs a single factor. (Two base-256 digits would halve the read-back, but 16 bits are not
-    // enough for lse at the logit magnitudes of outlier rows.) fp16 path: q~ as hi + lo.
     auto write_operand = [&](uint8_t* dst, int hh, const float (&v)[E], float qmax) {
-      if constexpr (I8) {
-        const float qs = qmax > 0.f ? 1048575.0f / qmax : 0.f;
+      DecHeadCoords<D> c;
 #pragma unroll
-        for (int e = 0; e < E; e++) {
-          const int Q = __float2int_rn(v[e] * qs);
-          const int d2 = (Q + 8192) >> 14;
-          const int r = Q - (d2 << 14);
-          const int d1 = (r + 64) >> 7;
-          const int d0 = r - (d1 << 7);
-          const int i = lane * E + e;  // contraction index = rotated coordinate; column n = 4 * head + digit
-          const uint32_t word = (uint32_t)(d0 & 0xff) | ((uint32_t)(d1 & 0xff) << 8) | ((uint32_t)(d2 & 0xff) << 16);
-          *reinterpret_cast<uint32_t*>(dst + 4 * (hh & 3) + (hh >> 2) * ((D / 8) * 128) + (i & 7) * 16 + (i >> 3) * 128) = word;
-        }
-      } else {
-#pragma unroll
-        for (int e = 0; e < E; e++) {
-          const float x = v[e];
-          const __half xh = __float2half_rn(x);
-          const __half xl = __float2half_rn(x - __half2float(xh));
-          const int i = lane * E + e;  // contraction index = rotated coordinate
-          const int off = (i & 7) * 16 + (i >> 3) * 128;
-          *reinterpret_cast<__half*>(dst + hh * 2 + off) = xh;                  // n = head (hi part)
-          *reinterpret_cast<__half*>(dst + hh * 2 + (D / 8) * 128 + off) = xl;  // n = 8 + head (lo part)
-        }
-      }
+      for (int e = 0; e < E; e++) c.v[e] = v[e];
+      dec_write_operand<D, I8>(dst, hh, c, qmax, lane);
     };
     auto score_factor = [&](float qmax) { return (qmax * (1.0f / 1048575.0f)) * p.delta * kfac; };  // digits -> log2-domain score per unit K scale
 
