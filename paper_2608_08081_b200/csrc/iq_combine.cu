@@ -41,6 +41,56 @@ __global__ void __launch_bounds__(WPH == 1 ? CMB_WARPS * 32 : WPH * 32) combine_
 
   float m = -INFINITY;
   int best = -1;
+  float l = 0.f;
+  float v[E];
+#pragma unroll
+  for (int e = 0; e < E; e++) v[e] = 0.f;
+  if (WPH == 1 && S <= 32) {
+    // few slots: lane s takes (m, l, argmax) of slot s, the reference and the weights come from warp reductions, and the
+    // acc rows are then loaded four at a time (their addresses do not depend on one another)
+    float ms = -INFINITY, ls = 0.f;
+    int idx = -1;
+    size_t o = 0;
+    if (lane < S) {
+      o = slot_index(lane);
+      ms = p.part_ml[2 * o];
+      ls = p.part_ml[2 * o + 1];
+      if (ls > 0.f) idx = slot_argmax(lane, o);
+      else ms = -INFINITY;
+    }
+    m = ms;
+    best = idx;
+#pragma unroll
+    for (int d2 = 16; d2 > 0; d2 >>= 1) {
+      const float om = __shfl_xor_sync(FULL, m, d2);
+      const int ob = __shfl_xor_sync(FULL, best, d2);
+      if (om > m) { m = om; best = ob; }
+      else if (om == m && ob >= 0 && (best < 0 || ob < best)) best = ob;
+    }
+    const float w = (ls > 0.f) ? __expf(ms - m) : 0.f;
+    l = ls * w;
+#pragma unroll
+    for (int d2 = 16; d2 > 0; d2 >>= 1) l += __shfl_xor_sync(FULL, l, d2);
+    for (int sb = 0; sb < S; sb += 4) {
+      float4 f[4][E / 4];
+      float ws[4];
+#pragma unroll
+      for (int k = 0; k < 4; k++) {
+        ws[k] = __shfl_sync(FULL, w, (sb + k) & 31);
+        const size_t ok = __shfl_sync(FULL, o, (sb + k) & 31);
+        if (sb + k >= S) ws[k] = 0.f;
+#pragma unroll
+        for (int e4 = 0; e4 < E / 4; e4++)
+          f[k][e4] = ws[k] != 0.f ? *reinterpret_cast<const float4*>(p.part_acc + ok * D + lane * E + 4 * e4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int k = 0; k < 4; k++)
+#pragma unroll
+        for (int e4 = 0; e4 < E / 4; e4++) {
+          v[4 * e4] += ws[k] * f[k][e4].x; v[4 * e4 + 1] += ws[k] * f[k][e4].y; v[4 * e4 + 2] += ws[k] * f[k][e4].z; v[4 * e4 + 3] += ws[k] * f[k][e4].w;
+        }
+    }
+  } else {
   for (int s = s0; s < S; s += WPH) {
     const size_t o = slot_index(s);
     const float ms = p.part_ml[2 * o], ls = p.part_ml[2 * o + 1];
@@ -49,10 +99,6 @@ __global__ void __launch_bounds__(WPH == 1 ? CMB_WARPS * 32 : WPH * 32) combine_
     if (ms > m) { m = ms; best = idx; }
     else if (ms == m && idx >= 0 && (best < 0 || idx < best)) best = idx;
   }
-  float l = 0.f;
-  float v[E];
-#pragma unroll
-  for (int e = 0; e < E; e++) v[e] = 0.f;
   for (int s = s0; s < S; s += WPH) {
     const size_t o = slot_index(s);
     const float ms = p.part_ml[2 * o], ls = p.part_ml[2 * o + 1];
@@ -65,6 +111,7 @@ __global__ void __launch_bounds__(WPH == 1 ? CMB_WARPS * 32 : WPH * 32) combine_
       const float4 f = *reinterpret_cast<const float4*>(a + e4);
       v[e4] += w * f.x; v[e4 + 1] += w * f.y; v[e4 + 2] += w * f.z; v[e4 + 3] += w * f.w;
     }
+  }
   }
   if constexpr (WPH > 1) {  // the warps' results (relative to their own maxima) merged by warp 0
     __shared__ float sv[WPH][D];
