@@ -557,3 +557,60 @@ def test_retrieval_margins_config4_shape(codebooks):
         assert int(np.argmax(np.abs(o))) == int(w.extra["needle_chan"][h])
         vn = w.v[0, w.extra["needle_pos"][h], h // 4].astype(np.float64)
         assert (o @ vn) / (np.linalg.norm(o) * np.linalg.norm(vn)) > 0.9
+
+
+# ---------------------------------------------------------------- fitting the SO(4) blocks (Section 3.2: 192 learnable parameters)
+def test_quaternion_pair_decomposition_inverts_the_block_matrix():
+    from oracle import so4_fit
+    q = _rand_quats(6, 64)
+    for q8 in q:
+        M = oracle.so4_block(q8)
+        back = so4_fit.matrix_to_quaternion_pair(M)
+        assert abs(np.linalg.norm(back[:4]) - 1) < 1e-12 and abs(np.linalg.norm(back[4:]) - 1) < 1e-12
+        assert np.allclose(oracle.so4_block(back.astype(np.float32)), M, atol=5e-7)      # (the block is built from fp32 parameters)
+        # the pair is determined up to a common sign (double cover)
+        s = np.sign(back[:4] @ q8[:4].astype(np.float64))
+        assert np.allclose(s * back, q8.astype(np.float64), atol=1e-6)
+    assert np.allclose(so4_fit.matrix_to_quaternion_pair(np.eye(4)) ** 2, [1, 0, 0, 0, 1, 0, 0, 0], atol=1e-12)
+
+
+def test_block_distortion_of_isotropic_data_does_not_depend_on_the_rotation():
+    from oracle import so4_fit
+    lv, th, mse = lloyd_max.lloyd_max(0)                       # the Gaussian-limit codebook and its distortion
+    z = np.random.Generator(np.random.Philox(5)).standard_normal((200000, 4))
+    q = _rand_quats(7, 3)
+    ds = [so4_fit.block_distortion(z, oracle.so4_block(q8), lv, th) for q8 in q] + [so4_fit.block_distortion(z, np.eye(4), lv, th)]
+    for dist in ds:
+        assert abs(dist - 4 * mse) < 0.02 * 4 * mse            # four coordinates, each at the codebook's distortion
+    assert max(ds) - min(ds) < 0.01 * 4 * mse
+
+
+def test_rotation_fit_finds_a_planted_rotation_and_never_ends_above_its_start(codebooks):
+    from oracle import so4_fit
+    lv, th = codebooks[128]
+    lv64 = np.asarray(lv, np.float64)
+    g = np.random.Generator(np.random.Philox(11))
+    Mstar = oracle.so4_block(_rand_quats(12, 1)[0])
+    c = lv64[g.integers(0, 8, size=(4000, 4))]                 # points that sit exactly on levels after the planted rotation
+    z = c @ Mstar                                              # u = M* z = c: zero distortion at M*
+    assert so4_fit.block_distortion(z, Mstar, lv, th) < 1e-24
+    start = so4_fit.givens(0, 2, 0.17) @ so4_fit.givens(1, 3, -0.11) @ Mstar
+    M, before, after = so4_fit.fit_block(z, start, lv, th)
+    assert before > 1e-2 and after < 1e-3 * before
+    assert np.allclose(M @ M.T, np.eye(4), atol=1e-12) and abs(np.linalg.det(M) - 1) < 1e-12
+    # structured (non-isotropic) data: the search improves on its start and beats most random rotations
+    zz = g.standard_normal((3000, 4)) * np.array([2.0, 0.3, 1.0, 0.2])
+    zz *= 2.0 / np.sqrt(np.mean(np.sum(zz * zz, axis=1)))      # mean squared norm 4, as for sqrt(d) H x^
+    M2, b2, a2 = so4_fit.fit_block(zz, np.eye(4), lv, th)
+    rand = sorted(so4_fit.block_distortion(zz, oracle.so4_block(q8), lv, th) for q8 in _rand_quats(13, 200))
+    assert a2 <= b2 and a2 <= rand[len(rand) // 10]             # at least as good as the best tenth of 200 random rotations
+
+
+def test_wht_coordinates_have_unit_variance_units():
+    from oracle import so4_fit
+    x = workloads.to_fp16(np.random.Generator(np.random.Philox(3)).standard_normal((64, 128)))
+    z = so4_fit.wht_coordinates(x)
+    assert np.allclose(np.sum(z * z, axis=1), 128.0, rtol=1e-12)          # sqrt(d) times a unit vector
+    R = oracle.rotation_matrix(128, np.tile(np.array([1, 0, 0, 0, 1, 0, 0, 0], np.float32), (32, 1)))   # identity blocks: R = H
+    xs = x.astype(np.float64)
+    assert np.allclose(z, math.sqrt(128) * (xs / np.linalg.norm(xs, axis=1, keepdims=True)) @ R.T, atol=1e-12)
