@@ -289,6 +289,31 @@ int iq_fit_codebook(const uint32_t* hist_host, int32_t bins, float range, int32_
                     iq_codebook* out_host);
 
 /*
+ * Calibration of the rotation (Section 3.2 counts 192 learnable parameters at d = 128: the 6 rotational degrees of
+ * freedom of each of the 32 SO(4) blocks; Appendix B stores them as 8 floats per block. The paper does not say how they
+ * are learned -- here each block's rotation is chosen to minimise the mean squared quantisation error of the block's
+ * four rotated coordinates, under the codebook in use, over a calibration set of rows).
+ *
+ * iq_wht_coordinates writes z = sqrt(d) H_d x^ (Algorithm 1, lines 1-2, in the unit-variance units of the codebook) of
+ * the given rows as fp32: the quantity the blocks rotate.
+ *   x              device binary16 rows, element (b, t, g, i) at b*stride_b + t*stride_t + g*stride_h + i (strides in
+ *                  elements, multiples of 8), t < n_rows_dev[b] (NULL: n_rows_max for every sequence), capped at n_rows_max.
+ *   z_dev          device fp32 [batch][n_rows_max][n_kv_heads][head_dim], 16-byte aligned; rows beyond a sequence's
+ *                  count are not written, zero rows give zeros.
+ * iq_fit_rotation (host only, no CUDA) fits the d/4 blocks of ONE KV head: z_host holds n_rows rows of that head's z,
+ * row r at z_host + r * row_stride (floats); quats_host [d/4][8] holds the starting rotation (q_L.wxyz, q_R.wxyz per
+ * block) and receives the fitted one, as unit quaternion pairs ready for iq_make_rotation. Per block a pattern search
+ * over the six coordinate planes: rotate by +-delta, keep the move if the distortion
+ *     1/N sum_rows sum_{i<4} (u_i - level[code(u_i)])^2,  u = M z,
+ * decreases, halve delta (pi/8 down to 1e-3 rad) when a sweep over the planes improves nothing. The result is never
+ * worse than the start. distortion_host (optional, 2 doubles): mean distortion per coordinate before and after.
+ */
+int iq_wht_coordinates(const iq_shape* shape, const void* x, int64_t stride_b, int64_t stride_t, int64_t stride_h,
+                       const int32_t* n_rows_dev, int32_t n_rows_max, float* z_dev, void* stream);
+int iq_fit_rotation(const float* z_host, int32_t n_rows, int64_t row_stride, int32_t head_dim, const iq_codebook* codebook,
+                    float* quats_host, double* distortion_host);
+
+/*
  * One whole decode step from HOST buffers, in one call: the step's inputs go to the device in one copy, one new row
  * per sequence is appended (Algorithm 1), the fused decode and the merge run (Appendix A), the output comes back and
  * the call returns when it has arrived. It is iq_quantize_append (n_new_max = 1) + iq_decode_attention +

@@ -27,9 +27,11 @@ from .binding import (  # noqa: F401
     iq_reconstruct_rows,
     iq_rotated_histogram,
     iq_suggest_splits,
+    iq_fit_rotation,
     iq_format_version,
     iq_selftest_bounded_wait,
     iq_version,
+    iq_wht_coordinates,
     lib_path,
     new_cache,
     new_paged_cache,

@@ -75,6 +75,8 @@ def _load():
     lib.iq_fit_codebook.argtypes = [_vp, _i32, ctypes.c_float, _i32, _i32, ctypes.POINTER(_IqCodebook)]
     lib.iq_suggest_splits.restype = _i32
     lib.iq_suggest_splits.argtypes = [ctypes.POINTER(_IqShape), _i32]
+    lib.iq_wht_coordinates.argtypes = [ctypes.POINTER(_IqShape), _vp, _i64, _i64, _i64, _vp, _i32, _vp, _vp]
+    lib.iq_fit_rotation.argtypes = [_vp, _i32, _i64, _i32, ctypes.POINTER(_IqCodebook), _vp, _vp]
     lib.iq_selftest_bounded_wait.argtypes = [_vp, ctypes.c_uint32, _vp]
     return lib
 
@@ -299,6 +301,27 @@ def iq_fit_codebook(hist_host, rng_half: float, symmetric: bool = True, grid: st
 def iq_suggest_splits(shape: Shape, max_seq_len: int) -> int:
     cs = shape.c()
     return int(_lib.iq_suggest_splits(ctypes.byref(cs), max_seq_len))
+
+
+def iq_wht_coordinates(shape: Shape, x, n_rows_dev, n_rows_max: int, z_out, stream=None) -> None:
+    """z = sqrt(d) H x^ of the rows x [B][T][H_kv][d] (fp16) into z_out [B][n_rows_max][H_kv][d] (fp32)."""
+    cs = shape.c()
+    _check(_lib.iq_wht_coordinates(ctypes.byref(cs), _ptr(x), x.stride(0), x.stride(1), x.stride(2), _ptr(n_rows_dev), n_rows_max,
+                                   _ptr(z_out), _stream(stream)), "iq_wht_coordinates")
+
+
+def iq_fit_rotation(z_rows, head_dim: int, codebook: Codebook, quats):
+    """Host fit of one KV head's SO(4) blocks: z_rows numpy fp32 [n][d] (that head's rows of iq_wht_coordinates), quats
+    numpy fp32 [d/4][8] the starting rotation. Returns (fitted quats fp32 [d/4][8], distortion before, after)."""
+    import numpy as np
+
+    z = np.ascontiguousarray(z_rows, dtype=np.float32)
+    q = np.ascontiguousarray(quats, dtype=np.float32).copy()
+    dist = (ctypes.c_double * 2)()
+    cb = codebook.c()
+    _check(_lib.iq_fit_rotation(z.ctypes.data, z.shape[0], z.shape[1], head_dim, ctypes.byref(cb), q.ctypes.data,
+                                ctypes.cast(dist, ctypes.c_void_p)), "iq_fit_rotation")
+    return q, float(dist[0]), float(dist[1])
 
 
 def iq_selftest_bounded_wait(status, polls: int, stream=None) -> None:

@@ -188,6 +188,99 @@ void finish_codebook(const double (&lv)[8], int grid, iq_codebook* out) {
   for (int i = 0; i < 7; i++) out->thresholds[i] = (float)(0.5 * ((double)out->levels[i] + (double)out->levels[i + 1]));
 }
 
+// ---- fitting the SO(4) blocks (host, fp64) ---------------------------------------------------------------------
+// A block matrix from its quaternion pair, M = L(q_L) R(conj q_R) (Section 3.3), both quaternions rescaled to unit length.
+void so4_from_pair(const double* q8, double (&M)[4][4]) {
+  double a = q8[0], b = q8[1], c = q8[2], d = q8[3], e = q8[4], f = q8[5], g = q8[6], h = q8[7];
+  const double nl = 1.0 / std::sqrt(a * a + b * b + c * c + d * d), nr = 1.0 / std::sqrt(e * e + f * f + g * g + h * h);
+  a *= nl; b *= nl; c *= nl; d *= nl; e *= nr; f *= nr; g *= nr; h *= nr;
+  const double L[4][4] = {{a, -b, -c, -d}, {b, a, -d, c}, {c, d, a, -b}, {d, -c, b, a}};
+  const double R[4][4] = {{e, f, g, h}, {-f, e, -h, g}, {-g, h, e, -f}, {-h, -g, f, e}};
+  for (int i = 0; i < 4; i++)
+    for (int j = 0; j < 4; j++) {
+      double s = 0;
+      for (int k = 0; k < 4; k++) s += L[i][k] * R[k][j];
+      M[i][j] = s;
+    }
+}
+// The pair back from a rotation matrix: M is bilinear in (q_L, q_R) over the 16 matrices T_ab = L(e_a) R(conj e_b), which
+// are orthogonal under the Frobenius product with squared norm 4, so <M, T_ab> / 4 = l_a r_b.
+void pair_from_so4(const double (&M)[4][4], double* q8) {
+  double P[4][4];
+  for (int a = 0; a < 4; a++)
+    for (int b = 0; b < 4; b++) {
+      double e8[8] = {0, 0, 0, 0, 0, 0, 0, 0}, T[4][4];
+      e8[a] = 1.0;
+      e8[4 + b] = 1.0;
+      so4_from_pair(e8, T);
+      double s = 0;
+      for (int i = 0; i < 4; i++)
+        for (int j = 0; j < 4; j++) s += T[i][j] * M[i][j];
+      P[a][b] = 0.25 * s;
+    }
+  int best = 0;
+  double bn = -1.0;
+  for (int a = 0; a < 4; a++) {
+    const double n = P[a][0] * P[a][0] + P[a][1] * P[a][1] + P[a][2] * P[a][2] + P[a][3] * P[a][3];
+    if (n > bn) { bn = n; best = a; }
+  }
+  double r[4], l[4], rn = std::sqrt(bn), ln = 0;
+  for (int b = 0; b < 4; b++) r[b] = P[best][b] / rn;
+  for (int a = 0; a < 4; a++) {
+    l[a] = P[a][0] * r[0] + P[a][1] * r[1] + P[a][2] * r[2] + P[a][3] * r[3];
+    ln += l[a] * l[a];
+  }
+  ln = std::sqrt(ln);
+  for (int a = 0; a < 4; a++) { q8[a] = l[a] / ln; q8[4 + a] = r[a]; }
+}
+// Mean over the rows of the squared quantisation error of u = M z (four coordinates), z = z4[n * stride .. + 4).
+double block_distortion(const float* z4, size_t stride, int n, const double (&M)[4][4], const iq_codebook& cb) {
+  double total = 0.0;
+  for (int i = 0; i < n; i++) {
+    const float* z = z4 + (size_t)i * stride;
+    for (int r = 0; r < 4; r++) {
+      const double u = M[r][0] * z[0] + M[r][1] * z[1] + M[r][2] * z[2] + M[r][3] * z[3];
+      int code = 0;
+      for (int j = 0; j < 7; j++) code += u > (double)cb.thresholds[j];
+      const double e = u - (double)cb.levels[code];
+      total += e * e;
+    }
+  }
+  return total / n;
+}
+// Pattern search over the six coordinate planes: rotate by +-delta, keep what lowers the distortion, halve delta when a
+// sweep improves nothing (pi/8 down to 1e-3 rad). Returns the distortion reached; M is updated in place.
+double fit_block(const float* z4, size_t stride, int n, double (&M)[4][4], const iq_codebook& cb, double& start) {
+  static const int planes[6][2] = {{0, 1}, {0, 2}, {0, 3}, {1, 2}, {1, 3}, {2, 3}};
+  double best = start = block_distortion(z4, stride, n, M, cb);
+  for (double delta = 3.14159265358979323846 / 8; delta >= 1e-3;) {
+    bool improved = false;
+    for (int pl = 0; pl < 6; pl++) {
+      const int i = planes[pl][0], j = planes[pl][1];
+      for (int sg = 0; sg < 2; sg++) {
+        const double c = std::cos(delta), sn = (sg == 0 ? 1.0 : -1.0) * std::sin(delta);
+        double C[4][4];
+        for (int r = 0; r < 4; r++)
+          for (int k = 0; k < 4; k++) C[r][k] = M[r][k];
+        for (int k = 0; k < 4; k++) {  // G(i, j, angle) M: rows i and j mix
+          C[i][k] = c * M[i][k] - sn * M[j][k];
+          C[j][k] = sn * M[i][k] + c * M[j][k];
+        }
+        const double dist = block_distortion(z4, stride, n, C, cb);
+        if (dist < best) {
+          for (int r = 0; r < 4; r++)
+            for (int k = 0; k < 4; k++) M[r][k] = C[r][k];
+          best = dist;
+          improved = true;
+          break;
+        }
+      }
+    }
+    if (!improved) delta *= 0.5;
+  }
+  return best;
+}
+
 }  // namespace
 
 extern "C" {
@@ -523,6 +616,52 @@ int iq_fit_codebook(const uint32_t* hist_host, int32_t bins, float range, int32_
   finish_codebook(lv, grid, out_host);
   for (int i = 0; i < 7; i++)
     if (!(out_host->levels[i] < out_host->levels[i + 1])) return IQ_ERR_CODEBOOK;  // too few distinct values in the data
+  return IQ_OK;
+}
+
+int iq_wht_coordinates(const iq_shape* shape, const void* x, int64_t stride_b, int64_t stride_t, int64_t stride_h,
+                       const int32_t* n_rows_dev, int32_t n_rows_max, float* z_dev, void* stream) {
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (n_rows_max < 0) return IQ_ERR_SHAPE;
+  if (n_rows_max == 0 || shape->batch == 0) return IQ_OK;
+  if (!x || !z_dev) return IQ_ERR_NULL;
+  if (!aligned16(x) || !aligned16(z_dev)) return IQ_ERR_ALIGN;
+  if (stride_b < 0 || stride_t < 0 || stride_h < 0) return IQ_ERR_SHAPE;
+  if ((stride_b & 7) || (stride_t & 7) || (stride_h & 7)) return IQ_ERR_ALIGN;
+  iq::WhtParams p = {};
+  p.x = static_cast<const __half*>(x);
+  p.stride_b = stride_b;
+  p.stride_t = stride_t;
+  p.stride_h = stride_h;
+  p.n_rows = n_rows_dev;
+  p.n_rows_max = n_rows_max;
+  p.z = z_dev;
+  p.n_kv_heads = shape->n_kv_heads;
+  const cudaError_t e = iq::launch_wht_coordinates(p, shape->head_dim, shape->batch, static_cast<cudaStream_t>(stream));
+  return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
+int iq_fit_rotation(const float* z_host, int32_t n_rows, int64_t row_stride, int32_t head_dim, const iq_codebook* codebook,
+                    float* quats_host, double* distortion_host) {
+  if (!z_host || !codebook || !quats_host) return IQ_ERR_NULL;
+  if ((head_dim != 128 && head_dim != 256) || n_rows < 1 || row_stride < head_dim) return IQ_ERR_SHAPE;
+  const int rc = check_codebook(codebook, false);
+  if (rc) return rc;
+  double before = 0.0, after = 0.0;
+  for (int b = 0; b < head_dim / 4; b++) {
+    double q8[8], M[4][4], start;
+    for (int i = 0; i < 8; i++) q8[i] = (double)quats_host[8 * b + i];
+    so4_from_pair(q8, M);
+    after += fit_block(z_host + 4 * b, (size_t)row_stride, n_rows, M, *codebook, start);
+    before += start;
+    pair_from_so4(M, q8);
+    for (int i = 0; i < 8; i++) quats_host[8 * b + i] = (float)q8[i];
+  }
+  if (distortion_host) {
+    distortion_host[0] = before / head_dim;
+    distortion_host[1] = after / head_dim;
+  }
   return IQ_OK;
 }
 

@@ -54,6 +54,17 @@ struct HistogramParams {
 };
 cudaError_t launch_rotated_histogram(const HistogramParams& p, int head_dim, int batch, cudaStream_t stream);
 
+// ---- calibration of the rotation: z = sqrt(d) H x^ of a set of rows
+struct WhtParams {
+  const __half* x;
+  long long stride_b, stride_t, stride_h;
+  const int32_t* n_rows;
+  int n_rows_max;
+  float* z;  // [batch][n_rows_max][n_kv_heads][head_dim]
+  int n_kv_heads;
+};
+cudaError_t launch_wht_coordinates(const WhtParams& p, int head_dim, int batch, cudaStream_t stream);
+
 // ---- fused decode
 constexpr int DEC_BLOCK_TOKENS = 128;  // cached rows per block of the decode kernel = rows of one transposed V block
 constexpr int DEC_HEADS = 8;          // query heads of one KV head that a work item covers (they share the N columns of one MMA)

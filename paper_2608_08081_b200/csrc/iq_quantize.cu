@@ -663,6 +663,43 @@ cudaError_t launch_rotated_histogram(const HistogramParams& p, int head_dim, int
                          : launch_after_predecessor(rotated_histogram_kernel<256>, grid, dim3(QA_WARPS * 32), 0, stream, p);
 }
 
+// Calibration of the rotation: z = sqrt(d) H_d x^ (Algorithm 1, lines 1-2, in the unit-variance units of the codebook) of
+// a set of rows, written out as fp32. One warp per row, lane l holds coordinates l E .. l E + E - 1.
+template <int D>
+__global__ void __launch_bounds__(QA_WARPS * 32) wht_coordinates_kernel(const __grid_constant__ WhtParams p) {
+  constexpr int E = D / 32;
+  grid_dependency_wait();
+  allow_dependent_launch();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int b = blockIdx.z, h = blockIdx.y;
+  const int t = blockIdx.x * QA_WARPS + warp;
+  int n_rows = p.n_rows ? p.n_rows[b] : p.n_rows_max;
+  n_rows = min(n_rows, p.n_rows_max);
+  if (t >= n_rows) return;
+  const __half* src = p.x + (size_t)b * p.stride_b + (size_t)t * p.stride_t + (size_t)h * p.stride_h + lane * E;
+  float v[E];
+  double ss = 0.0;  // squares of fp16 values are exact in fp32
+#pragma unroll
+  for (int e = 0; e < E; e++) {
+    v[e] = __half2float(src[e]);
+    ss += (double)(v[e] * v[e]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(FULL, ss, o);
+  wht_warp<float, E>(v, lane);  // unnormalised: the 1/sqrt(d) of H_d and the sqrt(d) of the units cancel
+  const float inv_s = ss > 0.0 ? (float)(1.0 / sqrt(ss)) : 0.f;
+  float* dst = p.z + (((size_t)b * p.n_rows_max + t) * p.n_kv_heads + h) * D + lane * E;
+#pragma unroll
+  for (int e = 0; e < E; e++) dst[e] = v[e] * inv_s;
+}
+
+cudaError_t launch_wht_coordinates(const WhtParams& p, int head_dim, int batch, cudaStream_t stream) {
+  if (p.n_rows_max <= 0 || batch <= 0) return cudaSuccess;
+  dim3 grid((p.n_rows_max + QA_WARPS - 1) / QA_WARPS, p.n_kv_heads, batch);
+  return head_dim == 128 ? launch_after_predecessor(wht_coordinates_kernel<128>, grid, dim3(QA_WARPS * 32), 0, stream, p)
+                         : launch_after_predecessor(wht_coordinates_kernel<256>, grid, dim3(QA_WARPS * 32), 0, stream, p);
+}
+
 cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int batch, cudaStream_t stream) {
   if (p.n_new_max <= 0 || batch <= 0) return cudaSuccess;
   const int rows_per_cta = QA_WARPS * QA_ROWS_PER_WARP;

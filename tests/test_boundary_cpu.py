@@ -153,3 +153,36 @@ def test_suggest_splits_is_sane(iq):
     assert iq.iq_suggest_splits(iq.Shape(1, 4, 1, 128, 1024), 100) == 8
     assert iq.iq_suggest_splits(iq.Shape(32, 64, 8, 128, 32768), 32768) == 8
     assert iq.iq_suggest_splits(iq.Shape(1, 16, 8, 256, 16384), 16384) % 2 == 0
+
+
+def test_rotation_fit_on_the_host_matches_the_oracle(iq, codebooks):
+    """iq_fit_rotation is host code: the same pattern search as the oracle's, written independently in C++. On structured
+    calibration rows both must end at the same distortion (the two evaluate the same fp64 sums in a different order, so a
+    comparison at a near-tie may go the other way: distortions are compared, not paths), the product's quaternion pairs
+    must give, under the oracle's distortion, what the product reports, and no block may end above its start."""
+    import oracle
+    import workloads
+    from oracle import so4_fit
+    d = 128
+    lv, th = codebooks[d]
+    cb = iq.Codebook(tuple(float(x) for x in lv), tuple(float(x) for x in th))
+    g = np.random.Generator(np.random.Philox(21))
+    scales = np.where(np.arange(d) % 2 == 1, 4.0, 1.0) * np.exp(0.5 * g.standard_normal(d))   # channel scales that correlate the block's coordinates
+    x = workloads.to_fp16(g.standard_normal((768, d)) * scales)
+    z = so4_fit.wht_coordinates(x).astype(np.float32)
+    q0 = workloads.quaternion_pairs(g, 1, d)[0]
+    q_ref, b_ref, a_ref = so4_fit.fit_rotation(z.astype(np.float64), q0, lv, th)
+    q_lib, b_lib, a_lib = iq.iq_fit_rotation(z, d, cb, q0)
+    assert abs(b_lib - b_ref) < 1e-12 * b_ref
+    assert a_lib <= b_lib and a_ref <= b_ref and a_ref < 0.97 * b_ref          # the fit pays on such data
+    assert abs(a_lib - a_ref) < 2e-3 * a_ref
+    again = sum(so4_fit.block_distortion(z[:, 4 * b:4 * b + 4].astype(np.float64), oracle.so4_block(q_lib[b]), lv, th) for b in range(d // 4)) / d
+    assert abs(again - a_lib) < 1e-5 * a_lib                                   # the pairs it returns are the rotation it found
+    assert np.allclose(np.linalg.norm(q_lib.reshape(-1, 2, 4), axis=-1), 1.0, atol=1e-6)
+    # argument checks, no CUDA involved
+    import ctypes
+    import paper_2608_08081_b200.binding as B
+    c = cb.c()
+    assert B._lib.iq_fit_rotation(None, 4, 128, 128, ctypes.byref(c), q_lib.ctypes.data, None) == -1
+    assert B._lib.iq_fit_rotation(z.ctypes.data, 0, 128, 128, ctypes.byref(c), q_lib.ctypes.data, None) == -2
+    assert B._lib.iq_fit_rotation(z.ctypes.data, 4, 64, 128, ctypes.byref(c), q_lib.ctypes.data, None) == -2

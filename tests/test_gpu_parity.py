@@ -381,6 +381,56 @@ def _gather_pages(cache, table, page_rows):
     return out
 
 
+@pytest.mark.parametrize("d", [128, 256])
+def test_rotation_calibration(iq, torch, codebooks, d):
+    """The 'learnable' SO(4) parameters: iq_wht_coordinates (GPU) against the oracle's sqrt(d) H x^, the host fit on the
+    GPU's coordinates against the oracle's fit, and the effect: rows quantised under the fitted rotation reconstruct
+    with a lower error than under the rotation the fit started from, and decode stays parity-exact with it."""
+    from oracle import so4_fit
+    B, H_q, H_kv, T = 2, 4, 2, 640
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    lens = np.array([640, 500], np.int32)
+    w = workloads.tiny(3100 + d, B, H_q, H_kv, d, T, lens)
+    g = np.random.Generator(np.random.Philox(7 + d))
+    scales = np.where(np.arange(d) % 2 == 1, 4.0, 1.0) * np.exp(0.5 * g.standard_normal(d))     # correlates neighbouring coordinates after H
+    k = workloads.to_fp16(w.k.astype(np.float64) * scales)
+    v = workloads.to_fp16(w.v.astype(np.float64) * scales)
+    shape = iq.Shape(B, H_q, H_kv, d, workloads.cap128(T))
+    kd = torch.from_numpy(k).cuda()
+    z = torch.full((B, T, H_kv, d), float("nan"), dtype=torch.float32, device="cuda")
+    iq.iq_wht_coordinates(shape, kd, torch.from_numpy(lens).cuda(), T, z)
+    torch.cuda.synchronize()
+    zc = z.cpu().numpy()
+    assert np.isnan(zc[1, 500:]).all()                                                          # rows beyond a sequence's count are not written
+    fitted = np.zeros_like(w.quats)
+    for h in range(H_kv):
+        rows = np.concatenate([zc[b, :lens[b], h] for b in range(B)])
+        ref = np.concatenate([so4_fit.wht_coordinates(k[b, :lens[b], h]) for b in range(B)])
+        assert np.all(np.abs(rows - ref) <= 1e-5 + 2e-6 * np.abs(ref))                          # fp32 butterfly against fp64
+        q_lib, before, after = iq.iq_fit_rotation(rows, d, cb, w.quats[h])
+        q_ref, b_ref, a_ref = so4_fit.fit_rotation(rows.astype(np.float64), w.quats[h], lv, th)
+        assert abs(before - b_ref) < 1e-9 * b_ref and abs(after - a_ref) < 5e-3 * a_ref and after < 0.97 * before
+        fitted[h] = q_lib
+    # the same rows through Algorithm 1 under both rotations: reconstruction error of the K rows, and decode parity
+    errs = []
+    for quats in (w.quats, fitted):
+        w2 = workloads.Workload("calib", B, H_q, H_kv, d, T, k, v, w.q, quats, lens)
+        shape2, rot, cache, status = gpu_quantize(iq, torch, w2, cb, n_new=lens)
+        gq = cache_to_numpy(cache)
+        compare_caches(w2, th, gq, oracle_quantize(w2, th, n_new=lens), lens)
+        K, _ = oracle.reconstruct_rows(quats, lv, gq, lens, H_kv)
+        num = den = 0.0
+        for b in range(B):
+            xk = k[b, :lens[b]].astype(np.float64)
+            num += np.sum((K[b, :lens[b]] - xk) ** 2)
+            den += np.sum(xk ** 2)
+        errs.append(num / den)
+        res = gpu_decode(iq, torch, shape2, rot, cb, w.q, cache, lens, iq.iq_suggest_splits(shape2, T))
+        check_decode(w2, lv, w.q, res, gq, lens)
+    assert errs[1] < 0.98 * errs[0], errs
+
+
 @pytest.mark.parametrize("d,page_rows", [(128, 128), (128, 256), (256, 128)])
 def test_paged_cache_gives_the_contiguous_results(iq, torch, codebooks, d, page_rows):
     """A pool of pages in scrambled order behind a block table: bulk append with ragged lengths, two single-row steps
