@@ -20,21 +20,24 @@
  *   - H_d in natural (Sylvester) order: H[i][j] = (-1)^popcount(i & j) / sqrt(d).
  *   - blocks b = 0 .. d/4-1 cover coordinates [4b, 4b+4) (Algorithm 1 prints 1-based "4i:4i+4").
  *   - quaternion = (w, x, y, z), Hamilton product, block coordinates (y0,y1,y2,y3) <-> y0 + y1 i + y2 j + y3 k.
- *   - quantiser works in unit-variance units u = sqrt(d) * x~; code = #{ j : u > t_j } over the 7
- *     ascending thresholds (strict ">", an exact tie takes the lower code); codes 0..7 ascend with level.
+ *   - quantiser works in unit-variance units u = sqrt(d) * x~; code = #{ j : u > t_j } over the 2^b - 1
+ *     ascending thresholds (strict ">", an exact tie takes the lower code); codes 0 .. 2^b - 1 ascend with level.
+ *     b = 3 is the paper's setting; Algorithm 1 is written for a general b, and b = 2 and b = 4 are carried too.
  *   - zero row: s = 0, x^ = 0.
  *   - stored scale = s rounded to fp32; dequantised coordinate = scale * level[code] / sqrt(d).
- *   - K and V of one KV head share that head's rotation and the codebook; all query heads of a
- *     group use their KV head's rotation.
+ *   - K and V of one KV head share that head's rotation; each side has its codebook (the same one unless the caller
+ *     gives two); all query heads of a group use their KV head's rotation.
  *   - packed row layout (3 bits x d, 3d/8 bytes, the paper fixes only the size): the row is a
  *     sequence of little-endian 32-bit words; coordinates are taken in groups of 32, each group
  *     owning 3 consecutive words. In group-local numbering, coordinate c < 24 puts its 3-bit code in
  *     bits [4n, 4n+3) of word c/8, n = c mod 8; coordinate c >= 24 (n = c - 24) spreads its code
  *     over bit 4n+3 of the three words: bit k of the code goes to word k. K rows are stored this way, one
- *     row after the other.
+ *     row after the other. b = 4: entry c puts its code in bits [4n, 4n+4) of word c/8, n = c mod 8 (b d / 8 = d/2
+ *     bytes per row). b = 2: entries are taken in groups of 16, one word each; in group-local numbering entry c < 8
+ *     puts its code in bits [4c, 4c+2), entry c >= 8 in bits [4(c-8)+2, 4(c-8)+4) (d/4 bytes per row).
  *   - V codes are stored token-transposed (the paper says nothing about the arrangement): the rows of one
- *     (sequence, KV head) are taken in blocks of 128; for block j and coordinate c there is one 48-byte
- *     record, at byte ((j * d) + c) * 48 of that head's V area, holding the 128 codes of coordinate c for the
+ *     (sequence, KV head) are taken in blocks of 128; for block j and coordinate c there is one record of 16 b
+ *     bytes (48 at b = 3), at byte ((j * d) + c) * 16 b of that head's V area, holding the 128 codes of coordinate c for the
  *     block's rows, arranged exactly like a packed row of 128 entries with the row-in-block as the entry
  *     index. t_cap is a multiple of 128.
  *
@@ -129,9 +132,10 @@ void iqo_rotation_matrix(int d, const float* quats, double* R) {
 }
 
 /* Algorithm 1, lines 1-4 and Step 3, for one row. x: d binary16 values. codes: one byte per
- * coordinate (0..7). Returns the fp32 scale; if u_out != NULL also returns u = sqrt(d) * x~. */
-float iqo_quantize_row(int d, const double* R, const float* thresholds7, const uint16_t* x,
+ * coordinate (0 .. 2^bits - 1; thresholds: 2^bits - 1 of them). Returns the fp32 scale; if u_out != NULL also returns u = sqrt(d) * x~. */
+float iqo_quantize_row(int d, int bits, const double* R, const float* thresholds, const uint16_t* x,
                        uint8_t* codes, double* u_out) {
+  const int n_th = (1 << bits) - 1;
   double* xh = (double*)malloc(sizeof(double) * d);
   double ss = 0;
   for (int i = 0; i < d; i++) { xh[i] = iqo_half_to_double(x[i]); ss += xh[i] * xh[i]; }
@@ -143,7 +147,7 @@ float iqo_quantize_row(int d, const double* R, const float* thresholds7, const u
     for (int j = 0; j < d; j++) acc += R[(size_t)i * d + j] * xh[j];
     double u = rootd * acc;
     int code = 0;
-    for (int j = 0; j < 7; j++) if (u > (double)thresholds7[j]) code++;
+    for (int j = 0; j < n_th; j++) if (u > (double)thresholds[j]) code++;
     codes[i] = (uint8_t)code;
     if (u_out) u_out[i] = u;
   }
@@ -151,96 +155,89 @@ float iqo_quantize_row(int d, const double* R, const float* thresholds7, const u
   return (float)s;
 }
 
-static int row_bytes(int d) { return 3 * d / 8; }
+static int row_bytes(int d, int bits) { return bits * d / 8; }
 
 static void put_word(uint8_t* p, uint32_t w) { p[0] = w & 255; p[1] = (w >> 8) & 255; p[2] = (w >> 16) & 255; p[3] = (w >> 24) & 255; }
 static uint32_t get_word(const uint8_t* p) { return (uint32_t)p[0] | ((uint32_t)p[1] << 8) | ((uint32_t)p[2] << 16) | ((uint32_t)p[3] << 24); }
 
-/* Step 4 (bit-pack), layout as described at the top of this file. */
-void iqo_pack_row(int d, const uint8_t* codes, uint8_t* row) {
-  for (int g = 0; g < d / 32; g++) {
-    uint32_t w[3] = {0, 0, 0};
-    for (int c = 0; c < 32; c++) {
-      uint32_t code = codes[32 * g + c] & 7u;
-      if (c < 24) {
-        w[c / 8] |= code << (4 * (c % 8));
-      } else {
-        int n = c - 24;
-        for (int k = 0; k < 3; k++) w[k] |= ((code >> k) & 1u) << (4 * n + 3);
-      }
-    }
-    for (int k = 0; k < 3; k++) put_word(row + 4 * (3 * g + k), w[k]);
+/* Entry e of a packed record (a K row: e = coordinate; a V record: e = row within the block), layouts as described at
+ * the top of this file. rec points at the record's first byte. */
+static uint32_t record_get(int bits, const uint8_t* rec, int e) {
+  if (bits == 4) return (get_word(rec + 4 * (e / 8)) >> (4 * (e % 8))) & 15u;
+  if (bits == 2) {
+    int c = e % 16;
+    int sh = (c < 8) ? 4 * c : 4 * (c - 8) + 2;
+    return (get_word(rec + 4 * (e / 16)) >> sh) & 3u;
   }
-}
-
-void iqo_unpack_row(int d, const uint8_t* row, uint8_t* codes) {
-  for (int g = 0; g < d / 32; g++) {
-    uint32_t w[3];
-    for (int k = 0; k < 3; k++) w[k] = get_word(row + 4 * (3 * g + k));
-    for (int c = 0; c < 32; c++) {
-      uint32_t code = 0;
-      if (c < 24) {
-        code = (w[c / 8] >> (4 * (c % 8))) & 7u;
-      } else {
-        int n = c - 24;
-        for (int k = 0; k < 3; k++) code |= ((w[k] >> (4 * n + 3)) & 1u) << k;
-      }
-      codes[32 * g + c] = (uint8_t)code;
-    }
-  }
-}
-
-/* Token-transposed V area of one (sequence, KV head): code of (row t, coordinate c). A 128-entry record is a
- * packed row of 128 entries, so entry e lives in 32-entry group e/32 of the record (3 words each). */
-static void v_locate(int d, int64_t t, int c, size_t* rec_byte, int* e) {
-  *rec_byte = ((size_t)(t / 128) * (size_t)d + (size_t)c) * 48;
-  *e = (int)(t % 128);
-}
-static void v_put(int d, uint8_t* area, int64_t t, int c, uint32_t code) {
-  size_t rb; int e;
-  v_locate(d, t, c, &rb, &e);
-  uint8_t* grp = area + rb + 12 * (e / 32);
-  int cc = e % 32;
-  uint32_t w[3];
-  for (int k = 0; k < 3; k++) w[k] = get_word(grp + 4 * k);
-  if (cc < 24) {
-    int sh = 4 * (cc % 8);
-    w[cc / 8] = (w[cc / 8] & ~(7u << sh)) | ((code & 7u) << sh);
-  } else {
-    int sh = 4 * (cc - 24) + 3;
-    for (int k = 0; k < 3; k++) w[k] = (w[k] & ~(1u << sh)) | (((code >> k) & 1u) << sh);
-  }
-  for (int k = 0; k < 3; k++) put_word(grp + 4 * k, w[k]);
-}
-static uint32_t v_get(int d, const uint8_t* area, int64_t t, int c) {
-  size_t rb; int e;
-  v_locate(d, t, c, &rb, &e);
-  const uint8_t* grp = area + rb + 12 * (e / 32);
+  const uint8_t* grp = rec + 12 * (e / 32);  /* bits == 3: groups of 32 entries in 3 words */
   int cc = e % 32;
   if (cc < 24) return (get_word(grp + 4 * (cc / 8)) >> (4 * (cc % 8))) & 7u;
   uint32_t code = 0;
   for (int k = 0; k < 3; k++) code |= ((get_word(grp + 4 * k) >> (4 * (cc - 24) + 3)) & 1u) << k;
   return code;
 }
-/* Codes of V row t of one (sequence, KV head) area, one byte per coordinate. */
-void iqo_v_row_codes(int d, const uint8_t* area, int64_t t, uint8_t* codes) {
-  for (int c = 0; c < d; c++) codes[c] = (uint8_t)v_get(d, area, t, c);
+static void record_put(int bits, uint8_t* rec, int e, uint32_t code) {
+  if (bits == 4) {
+    uint8_t* wp = rec + 4 * (e / 8);
+    int sh = 4 * (e % 8);
+    put_word(wp, (get_word(wp) & ~(15u << sh)) | ((code & 15u) << sh));
+    return;
+  }
+  if (bits == 2) {
+    uint8_t* wp = rec + 4 * (e / 16);
+    int c = e % 16;
+    int sh = (c < 8) ? 4 * c : 4 * (c - 8) + 2;
+    put_word(wp, (get_word(wp) & ~(3u << sh)) | ((code & 3u) << sh));
+    return;
+  }
+  uint8_t* grp = rec + 12 * (e / 32);
+  int cc = e % 32;
+  if (cc < 24) {
+    uint8_t* wp = grp + 4 * (cc / 8);
+    int sh = 4 * (cc % 8);
+    put_word(wp, (get_word(wp) & ~(7u << sh)) | ((code & 7u) << sh));
+  } else {
+    int sh = 4 * (cc - 24) + 3;
+    for (int k = 0; k < 3; k++) {
+      uint8_t* wp = grp + 4 * k;
+      put_word(wp, (get_word(wp) & ~(1u << sh)) | (((code >> k) & 1u) << sh));
+    }
+  }
 }
-void iqo_v_row_store(int d, uint8_t* area, int64_t t, const uint8_t* codes) {
-  for (int c = 0; c < d; c++) v_put(d, area, t, c, codes[c]);
+
+/* Step 4 (bit-pack) of one K row, and its inverse. */
+void iqo_pack_row(int d, int bits, const uint8_t* codes, uint8_t* row) {
+  memset(row, 0, (size_t)row_bytes(d, bits));
+  for (int c = 0; c < d; c++) record_put(bits, row, c, codes[c]);
+}
+
+void iqo_unpack_row(int d, int bits, const uint8_t* row, uint8_t* codes) {
+  for (int c = 0; c < d; c++) codes[c] = (uint8_t)record_get(bits, row, c);
+}
+
+/* Token-transposed V area of one (sequence, KV head): the record of (block t / 128, coordinate c) holds 128 entries,
+ * the row within the block as the entry. */
+static size_t v_record(int d, int bits, int64_t t, int c) { return ((size_t)(t / 128) * (size_t)d + (size_t)c) * (size_t)(16 * bits); }
+/* Codes of V row t of one (sequence, KV head) area, one byte per coordinate. */
+void iqo_v_row_codes(int d, int bits, const uint8_t* area, int64_t t, uint8_t* codes) {
+  for (int c = 0; c < d; c++) codes[c] = (uint8_t)record_get(bits, area + v_record(d, bits, t, c), (int)(t % 128));
+}
+void iqo_v_row_store(int d, int bits, uint8_t* area, int64_t t, const uint8_t* codes) {
+  for (int c = 0; c < d; c++) record_put(bits, area + v_record(d, bits, t, c), (int)(t % 128), codes[c]);
 }
 
 /* Algorithm 1 applied to the new K and V rows of every sequence and KV head, appended to the cache.
  * k_new, v_new: binary16, element (b, i, h, c) at b*stride_b + i*stride_t + h*stride_h + c (element strides).
  * Row i < n_new[b] of sequence b goes to cache row append_pos[b] + i (rows >= t_cap are skipped).
- * quats: [H_kv][d/4][8]. codes: [B][H_kv][t_cap][3d/8], scales: [B][H_kv][t_cap].
+ * quats: [H_kv][d/4][8]. codes: [B][H_kv][t_cap][bits d/8], scales: [B][H_kv][t_cap]. thresholds_k / thresholds_v: the
+ * 2^bits - 1 thresholds of the K side and of the V side.
  * Returns the number of rows skipped because they fell outside the cache. */
-int64_t iqo_quantize_append(int B, int H_kv, int d, int t_cap, const float* quats, const float* thresholds7,
-                            const uint16_t* k_new, const uint16_t* v_new,
+int64_t iqo_quantize_append(int B, int H_kv, int d, int bits, int t_cap, const float* quats, const float* thresholds_k,
+                            const float* thresholds_v, const uint16_t* k_new, const uint16_t* v_new,
                             int64_t stride_b, int64_t stride_t, int64_t stride_h,
                             const int32_t* append_pos, const int32_t* n_new, int n_new_max,
                             uint8_t* k_codes, float* k_scales, uint8_t* v_codes, float* v_scales) {
-  int P = row_bytes(d);
+  int P = row_bytes(d, bits);
   int64_t skipped = 0;
   for (int h = 0; h < H_kv; h++) {
     double* R = (double*)malloc(sizeof(double) * d * d);
@@ -256,8 +253,8 @@ int64_t iqo_quantize_append(int B, int H_kv, int d, int t_cap, const float* quat
         uint8_t codes[512];
         size_t src = (size_t)(b * stride_b + i * stride_t + h * stride_h);
         size_t row = ((size_t)b * H_kv + h) * t_cap + t;
-        k_scales[row] = iqo_quantize_row(d, R, thresholds7, k_new + src, codes, NULL);
-        iqo_pack_row(d, codes, k_codes + row * P);
+        k_scales[row] = iqo_quantize_row(d, bits, R, thresholds_k, k_new + src, codes, NULL);
+        iqo_pack_row(d, bits, codes, k_codes + row * P);
       }
       /* V rows share words between neighbouring rows (token-transposed records): written one row at a time */
       for (int i = 0; i < n; i++) {
@@ -266,8 +263,8 @@ int64_t iqo_quantize_append(int B, int H_kv, int d, int t_cap, const float* quat
         uint8_t codes[512];
         size_t src = (size_t)(b * stride_b + i * stride_t + h * stride_h);
         size_t area = ((size_t)b * H_kv + h) * t_cap;
-        v_scales[area + t] = iqo_quantize_row(d, R, thresholds7, v_new + src, codes, NULL);
-        iqo_v_row_store(d, v_codes + area * P, t, codes);
+        v_scales[area + t] = iqo_quantize_row(d, bits, R, thresholds_v, v_new + src, codes, NULL);
+        iqo_v_row_store(d, bits, v_codes + area * P, t, codes);
       }
       skipped += sk;
     }
@@ -277,28 +274,28 @@ int64_t iqo_quantize_append(int B, int H_kv, int d, int t_cap, const float* quat
 }
 
 /* Dequantised rotated vector of cached V row t of a (sequence, KV head) area. */
-static void dequant_v_row(int d, const uint8_t* area, int64_t t, float scale, const float* levels8, double* out) {
+static void dequant_v_row(int d, int bits, const uint8_t* area, int64_t t, float scale, const float* levels, double* out) {
   uint8_t codes[512];
-  iqo_v_row_codes(d, area, t, codes);
+  iqo_v_row_codes(d, bits, area, t, codes);
   double f = (double)scale / sqrt((double)d);
-  for (int i = 0; i < d; i++) out[i] = f * (double)levels8[codes[i]];
+  for (int i = 0; i < d; i++) out[i] = f * (double)levels[codes[i]];
 }
 
 /* Dequantised rotated vector of one cached K row: x~_i = scale * level[code_i] / sqrt(d). */
-static void dequant_row(int d, const uint8_t* row, float scale, const float* levels8, double* out) {
+static void dequant_row(int d, int bits, const uint8_t* row, float scale, const float* levels, double* out) {
   uint8_t codes[512];
-  iqo_unpack_row(d, row, codes);
+  iqo_unpack_row(d, bits, row, codes);
   double f = (double)scale / sqrt((double)d);
-  for (int i = 0; i < d; i++) out[i] = f * (double)levels8[codes[i]];
+  for (int i = 0; i < d; i++) out[i] = f * (double)levels[codes[i]];
 }
 
 /* Appendix A, one query head against the first len rows of its KV head's packed cache.
  * z_out (optional, [len]) receives the scaled scores; o_rot (optional, [d]) the rotated-space output. */
-static void decode_one(int d, const double* R, const float* levels8, double sm_scale, const uint16_t* q,
+static void decode_one(int d, int bits, const double* R, const float* levels_k, const float* levels_v, double sm_scale, const uint16_t* q,
                        const uint8_t* k_codes, const float* k_scales, const uint8_t* v_codes,
                        const float* v_scales, int len, double* out, double* lse, int32_t* argmax,
                        double* z_out, double* o_rot_out) {
-  int P = row_bytes(d);
+  int P = row_bytes(d, bits);
   double* qt = (double*)malloc(sizeof(double) * d);
   double* z = (double*)malloc(sizeof(double) * (len > 0 ? len : 1));
   double* row = (double*)malloc(sizeof(double) * d);
@@ -311,7 +308,7 @@ static void decode_one(int d, const double* R, const float* levels8, double sm_s
   int best = -1;
   double zmax = -INFINITY;
   for (int j = 0; j < len; j++) {         /* z_j = sm_scale * q~ . k~_j */
-    dequant_row(d, k_codes + (size_t)j * P, k_scales[j], levels8, row);
+    dequant_row(d, bits, k_codes + (size_t)j * P, k_scales[j], levels_k, row);
     double acc = 0;
     for (int i = 0; i < d; i++) acc += qt[i] * row[i];
     z[j] = sm_scale * acc;
@@ -322,7 +319,7 @@ static void decode_one(int d, const double* R, const float* levels8, double sm_s
   for (int j = 0; j < len; j++) denom += exp(z[j] - zmax);
   for (int j = 0; j < len; j++) {         /* o~ = sum_j alpha_j v~_j */
     double a = exp(z[j] - zmax) / denom;
-    dequant_v_row(d, v_codes, j, v_scales[j], levels8, row);
+    dequant_v_row(d, bits, v_codes, j, v_scales[j], levels_v, row);
     for (int i = 0; i < d; i++) orot[i] += a * row[i];
   }
   for (int j = 0; j < d; j++) {           /* o = R^T o~ */
@@ -339,11 +336,11 @@ static void decode_one(int d, const double* R, const float* levels8, double sm_s
 /* One decode step for every sequence and query head. q: [B][H_q][d] binary16. out: [B][H_q][d],
  * lse: [B][H_q], argmax: [B][H_q] (lowest row index attaining the maximum score; -1 if len = 0).
  * sm_scale <= 0 selects 1/sqrt(d). o_rot (optional): [B][H_q][d], the output before R^T. */
-void iqo_decode_attention(int B, int H_q, int H_kv, int d, int t_cap, double sm_scale, const float* quats,
-                          const float* levels8, const uint16_t* q, const uint8_t* k_codes,
+void iqo_decode_attention(int B, int H_q, int H_kv, int d, int bits, int t_cap, double sm_scale, const float* quats,
+                          const float* levels_k, const float* levels_v, const uint16_t* q, const uint8_t* k_codes,
                           const float* k_scales, const uint8_t* v_codes, const float* v_scales,
                           const int32_t* seq_lens, double* out, double* lse, int32_t* argmax, double* o_rot) {
-  int P = row_bytes(d), G = H_q / H_kv;
+  int P = row_bytes(d, bits), G = H_q / H_kv;
   if (sm_scale <= 0) sm_scale = 1.0 / sqrt((double)d);
   double* Rs = (double*)malloc(sizeof(double) * (size_t)H_kv * d * d);
   for (int g = 0; g < H_kv; g++) iqo_rotation_matrix(d, quats + (size_t)g * (d / 4) * 8, Rs + (size_t)g * d * d);
@@ -356,7 +353,7 @@ void iqo_decode_attention(int B, int H_q, int H_kv, int d, int t_cap, double sm_
       if (len < 0) len = 0;
       size_t base = ((size_t)b * H_kv + g) * t_cap;
       size_t o = ((size_t)b * H_q + h);
-      decode_one(d, Rs + (size_t)g * d * d, levels8, sm_scale, q + o * d, k_codes + base * P, k_scales + base,
+      decode_one(d, bits, Rs + (size_t)g * d * d, levels_k, levels_v, sm_scale, q + o * d, k_codes + base * P, k_scales + base,
                  v_codes + base * P, v_scales + base, len, out + o * d, lse ? lse + o : NULL,
                  argmax ? argmax + o : NULL, NULL, o_rot ? o_rot + o * d : NULL);
     }
@@ -367,10 +364,10 @@ void iqo_decode_attention(int B, int H_q, int H_kv, int d, int t_cap, double sm_
  * row back in the original space, x_hat = R^T x~ with x~_i = scale * level[code_i] / sqrt(d) (Algorithm 1 read
  * backwards; R is orthogonal, so R^-1 = R^T). k_out, v_out: [B][t_cap][H_kv][d] doubles; rows >= seq_lens[b] are
  * left untouched. */
-void iqo_reconstruct_rows(int B, int H_kv, int d, int t_cap, const float* quats, const float* levels8,
+void iqo_reconstruct_rows(int B, int H_kv, int d, int bits, int t_cap, const float* quats, const float* levels_k, const float* levels_v,
                           const uint8_t* k_codes, const float* k_scales, const uint8_t* v_codes,
                           const float* v_scales, const int32_t* seq_lens, double* k_out, double* v_out) {
-  int P = row_bytes(d);
+  int P = row_bytes(d, bits);
   double* Rs = (double*)malloc(sizeof(double) * (size_t)H_kv * d * d);
   for (int g = 0; g < H_kv; g++) iqo_rotation_matrix(d, quats + (size_t)g * (d / 4) * 8, Rs + (size_t)g * d * d);
 #pragma omp parallel for schedule(dynamic) collapse(2)
@@ -383,8 +380,8 @@ void iqo_reconstruct_rows(int B, int H_kv, int d, int t_cap, const float* quats,
       double xt[512];
       for (int t = 0; t < len; t++)
         for (int which = 0; which < 2; which++) {
-          if (which == 0) dequant_row(d, k_codes + (base + t) * P, k_scales[base + t], levels8, xt);
-          else dequant_v_row(d, v_codes + base * P, t, v_scales[base + t], levels8, xt);
+          if (which == 0) dequant_row(d, bits, k_codes + (base + t) * P, k_scales[base + t], levels_k, xt);
+          else dequant_v_row(d, bits, v_codes + base * P, t, v_scales[base + t], levels_v, xt);
           double* o = (which == 0 ? k_out : v_out) + (((size_t)b * t_cap + t) * H_kv + g) * d;
           for (int i = 0; i < d; i++) {  /* (R^T x~)_i = sum_j R[j][i] x~_j */
             double acc = 0;
@@ -397,10 +394,10 @@ void iqo_reconstruct_rows(int B, int H_kv, int d, int t_cap, const float* quats,
 }
 
 /* Scaled scores z_j of one (sequence b, query head h): z_out [len]. */
-void iqo_scores(int H_q, int H_kv, int d, int t_cap, double sm_scale, const float* quats, const float* levels8,
+void iqo_scores(int H_q, int H_kv, int d, int bits, int t_cap, double sm_scale, const float* quats, const float* levels_k,
                 const uint16_t* q_bh, int b, int h, const uint8_t* k_codes, const float* k_scales, int len,
                 double* z_out) {
-  int P = row_bytes(d), G = H_q / H_kv, g = h / G;
+  int P = row_bytes(d, bits), G = H_q / H_kv, g = h / G;
   if (sm_scale <= 0) sm_scale = 1.0 / sqrt((double)d);
   double* R = (double*)malloc(sizeof(double) * d * d);
   iqo_rotation_matrix(d, quats + (size_t)g * (d / 4) * 8, R);
@@ -413,7 +410,7 @@ void iqo_scores(int H_q, int H_kv, int d, int t_cap, double sm_scale, const floa
     qt[i] = acc;
   }
   for (int j = 0; j < len; j++) {
-    dequant_row(d, k_codes + (base + j) * P, k_scales[base + j], levels8, row);
+    dequant_row(d, bits, k_codes + (base + j) * P, k_scales[base + j], levels_k, row);
     double acc = 0;
     for (int i = 0; i < d; i++) acc += qt[i] * row[i];
     z_out[j] = sm_scale * acc;

@@ -55,21 +55,21 @@ def lloyd_max(d: int, n_levels: int = 8, iters: int = 2000, tol: float = 1e-13):
     return levels, th, err / total
 
 
-def fp16_codebook(d: int):
+def fp16_codebook(d: int, n_levels: int = 8):
     """Codebook in the form handed to both the oracle and the CUDA library: levels rounded to values
     exactly representable in binary16 (stored as fp32), thresholds = midpoints of those levels (fp32)."""
-    lv, _, _ = lloyd_max(d)
+    lv, _, _ = lloyd_max(d, n_levels)
     lv16 = lv.astype(np.float16).astype(np.float32)
     th = (0.5 * (lv16[1:].astype(np.float64) + lv16[:-1].astype(np.float64))).astype(np.float32)
     return lv16, th
 
 
-def int8_codebook(d: int):
+def int8_codebook(d: int, n_levels: int = 8):
     """The same codebook with its levels snapped to an 8-bit grid: level_j = n_j * delta with integer |n_j| <= 127 and
     delta = max|level| / 127 (all in fp32, as handed to the oracle and the CUDA library); thresholds = midpoints of the
     snapped levels. The decode kernel's integer tensor-core path needs levels of this form."""
-    lv, _, _ = lloyd_max(d)
-    a = 0.5 * (lv - lv[::-1])                      # exact symmetry first (ascending, a[7] = -a[0] > 0)
+    lv, _, _ = lloyd_max(d, n_levels)
+    a = 0.5 * (lv - lv[::-1])                      # exact symmetry first (ascending, a[-1] = -a[0] > 0)
     delta = np.float32(a[-1] / 127.0)
     n = np.rint(a / np.float64(delta)).astype(np.int32)
     lv8 = (n.astype(np.float32) * delta).astype(np.float32)

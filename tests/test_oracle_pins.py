@@ -614,3 +614,100 @@ def test_wht_coordinates_have_unit_variance_units():
     R = oracle.rotation_matrix(128, np.tile(np.array([1, 0, 0, 0, 1, 0, 0, 0], np.float32), (32, 1)))   # identity blocks: R = H
     xs = x.astype(np.float64)
     assert np.allclose(z, math.sqrt(128) * (xs / np.linalg.norm(xs, axis=1, keepdims=True)) @ R.T, atol=1e-12)
+
+
+# ---------------------------------------------------------------- other bit widths (Algorithm 1 is written for a general b)
+def _gauss_table(n):
+    out = {}
+    for line in open(os.path.join(GOLD, "gauss_lloyd_max_4_16.txt")):
+        f = line.split("#")[0].split()
+        if len(f) >= 3 and f[0] == str(n):
+            out[f[1]] = np.array([float(x) for x in f[2:]])
+    return out
+
+
+@pytest.mark.parametrize("n", [4, 16])
+def test_lloyd_max_gaussian_limit_matches_the_textbook_tables_for_2_and_4_bits(n):
+    lv, th, mse = lloyd_max.lloyd_max(0, n_levels=n)
+    t = _gauss_table(n)
+    assert np.allclose(lv[n // 2:], t["levels"], atol=6e-4) and np.allclose(lv[:n // 2], -t["levels"][::-1], atol=6e-4)
+    assert abs(th[n // 2 - 1]) < 1e-9 and np.allclose(th[n // 2:], t["thresholds"], atol=6e-4)
+    assert abs(mse - t["mse"][0]) < 6e-5
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+@pytest.mark.parametrize("d", [128, 256])
+def test_pack_unpack_roundtrip_and_layout_other_bit_widths(d, bits):
+    g = np.random.default_rng(bits * 100 + d)
+    codes = g.integers(0, 1 << bits, size=d, dtype=np.uint8)
+    row = oracle.pack_row(d, codes, bits)
+    assert row.size == bits * d // 8 and np.array_equal(oracle.unpack_row(d, row, bits), codes)
+    words = row.view("<u4")
+    # the layout, stated bit by bit
+    for c in range(d):
+        if bits == 4:      # entry c: bits [4n, 4n+4) of word c / 8, n = c mod 8
+            got = (int(words[c // 8]) >> (4 * (c % 8))) & 15
+        else:              # groups of 16 entries, one word each: entry e < 8 at bits [4e, 4e+2), entry e >= 8 at bits [4(e-8)+2, 4(e-8)+4)
+            e = c % 16
+            got = (int(words[c // 16]) >> (4 * e if e < 8 else 4 * (e - 8) + 2)) & 3
+        assert got == codes[c]
+    # every bit of the row belongs to exactly one entry: flipping one code changes only that entry's bits
+    for c in (0, 7, 8, 15, 16, d - 1):
+        c2 = codes.copy()
+        c2[c] ^= (1 << bits) - 1
+        diff = np.unpackbits(oracle.pack_row(d, c2, bits) ^ row).sum()
+        assert diff == bits
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_quantize_roundtrip_and_attention_identity_other_bit_widths(bits):
+    """Round-trip error = the codebook's distortion, threshold rule = nearest level, the token-transposed V records, and
+    compressed-space attention = reconstruct-then-compute, at 2 and 4 bits, with separate K and V codebooks."""
+    d, T, H_kv, H_q = 128, 300, 2, 4
+    n = 1 << bits
+    lv_k, th_k = lloyd_max.int8_codebook(d, n)
+    lv_f, _, mse = lloyd_max.lloyd_max(d, n)
+    lv_v = (lv_k.astype(np.float64) * 1.07).astype(np.float32)                     # a different codebook for the V side
+    th_v = (0.5 * (lv_v[1:].astype(np.float64) + lv_v[:-1].astype(np.float64))).astype(np.float32)
+    w = workloads.tiny(500 + bits, 1, H_q, H_kv, d, T)
+    cache = oracle.new_cache(1, H_kv, d, workloads.cap128(T), bits)
+    assert cache["k_codes"].shape[-1] == bits * d // 8
+    oracle.quantize_append(w.quats, th_k, w.k, w.v, np.zeros(1, np.int32), None, cache, thresholds_v=th_v)
+    R = [oracle.rotation_matrix(d, w.quats[g]) for g in range(H_kv)]
+    err = 0.0
+    for t in (0, 1, 127, 128, 129, 299):
+        for g in range(H_kv):
+            ck, s, u = oracle.quantize_row(d, R[g], th_k, w.k[0, t, g])
+            assert np.array_equal(oracle.unpack_row(d, cache["k_codes"][0, g, t], bits), ck)
+            assert np.array_equal(ck, np.argmin(np.abs(u[:, None] - lv_k[None, :].astype(np.float64)), axis=1))   # nearest level
+            cv, sv, uv = oracle.quantize_row(d, R[g], th_v, w.v[0, t, g])
+            assert np.array_equal(oracle.v_row_codes(d, cache["v_codes"][0, g], t, bits), cv)
+            # the V record of (block, coordinate), stated independently: 16 * bits bytes, entry = row in the block
+            for c in (0, 5, d - 1):
+                rec = cache["v_codes"][0, g].reshape(-1)[((t // 128) * d + c) * 16 * bits:][:16 * bits].view("<u4")
+                e = t % 128
+                if bits == 4:
+                    got = (int(rec[e // 8]) >> (4 * (e % 8))) & 15
+                else:
+                    ee = e % 16
+                    got = (int(rec[e // 16]) >> (4 * ee if ee < 8 else 4 * (ee - 8) + 2)) & 3
+                assert got == cv[c]
+            err += np.mean((u - lv_k.astype(np.float64)[ck]) ** 2)
+    err /= 12
+    assert abs(err - mse) < 0.12 * mse                                             # distortion of Gaussian rows = the codebook's
+    # attention identity against a dense numpy restatement with the two codebooks
+    lens = np.array([T], np.int32)
+    res = oracle.decode_attention(w.quats, lv_k, w.q, cache, lens, H_kv, levels_v=lv_v)
+    K, V = oracle.reconstruct_rows(w.quats, lv_k, cache, lens, H_kv, levels_v=lv_v, d=d)
+    for h in range(H_q):
+        g = h // (H_q // H_kv)
+        q = w.q[0, h].astype(np.float64)
+        z = (K[0, :T, g] @ q) / math.sqrt(d)
+        a = np.exp(z - z.max()); a /= a.sum()
+        assert np.allclose(res["out"][0, h], a @ V[0, :T, g], atol=1e-11)
+        # and the reconstruction itself: x_hat = R^T (s * level[code] / sqrt(d))
+        t = 17
+        ck = oracle.unpack_row(d, cache["k_codes"][0, g, t], bits)
+        assert np.allclose(K[0, t, g], R[g].T @ (cache["k_scales"][0, g, t].astype(np.float64) * lv_k.astype(np.float64)[ck] / math.sqrt(d)), atol=1e-12)
+        cv = oracle.v_row_codes(d, cache["v_codes"][0, g], t, bits)
+        assert np.allclose(V[0, t, g], R[g].T @ (cache["v_scales"][0, g, t].astype(np.float64) * lv_v.astype(np.float64)[cv] / math.sqrt(d)), atol=1e-12)
