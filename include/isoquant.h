@@ -333,6 +333,34 @@ int iq_decode_step_host(const iq_shape* shape, const float* rot_dev, const iq_co
                         void* stream);
 
 /*
+ * The decode step with the append folded into the decode launch (Algorithm 1 for the step's new rows; Appendix A): what
+ * iq_quantize_append (one row per sequence) + iq_decode_attention + iq_combine_splits compute, in two launches instead
+ * of three -- at batch 1 the launch boundaries cost as much as the decode itself. One warp per (sequence, KV head) of
+ * the decode kernel quantises the new K and V rows and writes them to the cache while the other warps read the cache
+ * WITHOUT those rows; the new row's contribution is a partial of its own, computed from its codes and stored scale like
+ * a cached row's, which the merge takes as one more slot.
+ *   k_new, v_new   device binary16 [batch][n_kv_heads][head_dim], contiguous, 16-byte aligned: the step's new rows,
+ *                  appended at row seq_lens[b] of every sequence and attended to.
+ *   seq_lens_dev   device int32 [batch]: the lengths BEFORE the step (as for iq_decode_attention they are read early).
+ *                  The caller advances them afterwards. A sequence with seq_lens[b] outside [0, t_cap) gets no new row
+ *                  (IQ_STATUS_ROW_OUT_OF_RANGE, 2 rows per KV head counted in status_dev[2]) and attends to its cached
+ *                  rows only.
+ *   workspace_dev  device, iq_decode_step_workspace_bytes(shape, num_splits) bytes, 16-byte aligned: the partial slots
+ *                  and the new rows' partials; needs no initialisation. Calls that share a workspace must be ordered on
+ *                  one stream.
+ *   out, lse_out, argmax_out   as for iq_combine_splits (argmax_out != NULL also selects exact slot maxima).
+ *   num_splits     as for iq_decode_attention.
+ * With a paged cache the page that receives the new row must be in the block table before the call.
+ * (Merging inside the decode kernel as well -- arrival counters, the last writer merges -- was built and measured
+ * slower than the separate merge launch at every batch size, and is not part of the library.)
+ */
+size_t iq_decode_step_workspace_bytes(const iq_shape* shape, int32_t num_splits);
+int iq_decode_step_fused(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook, const void* q,
+                         const void* k_new, const void* v_new, const iq_cache* cache, const int32_t* seq_lens_dev,
+                         int32_t num_splits, void* workspace_dev, void* out, int32_t out_is_fp16, float* lse_out,
+                         int32_t* argmax_out, uint32_t* status_dev, void* stream);
+
+/*
  * Decode step for callers that cannot allocate device memory (the paper has no counterpart: its pipeline
  * is unsplit and needs no scratch). It runs iq_decode_attention followed by iq_combine_splits with the
  * split partials kept in a fixed array inside the library image instead of caller-provided buffers.

@@ -23,6 +23,8 @@ from .binding import (  # noqa: F401
     iq_row_bytes,
     iq_strerror,
     iq_decode_step_host,
+    iq_decode_step_fused,
+    iq_decode_step_workspace_bytes,
     iq_fit_codebook,
     iq_reconstruct_rows,
     iq_rotated_histogram,

@@ -78,6 +78,10 @@ def _load():
     lib.iq_wht_coordinates.argtypes = [ctypes.POINTER(_IqShape), _vp, _i64, _i64, _i64, _vp, _i32, _vp, _vp]
     lib.iq_fit_rotation.argtypes = [_vp, _i32, _i64, _i32, ctypes.POINTER(_IqCodebook), _vp, _vp]
     lib.iq_selftest_bounded_wait.argtypes = [_vp, ctypes.c_uint32, _vp]
+    lib.iq_decode_step_workspace_bytes.argtypes = [ctypes.POINTER(_IqShape), _i32]
+    lib.iq_decode_step_workspace_bytes.restype = ctypes.c_size_t
+    lib.iq_decode_step_fused.argtypes = [ctypes.POINTER(_IqShape), _vp, ctypes.POINTER(_IqCodebook), _vp, _vp, _vp,
+                                         ctypes.POINTER(_IqCache), _vp, _i32, _vp, _vp, _i32, _vp, _vp, _vp, _vp]
     return lib
 
 
@@ -235,6 +239,23 @@ def iq_combine_splits_sharded(shape: Shape, rot_dev, num_splits: int, n_shards: 
     _check(_lib.iq_combine_splits_sharded(ctypes.byref(cs), _ptr(rot_dev), num_splits, n_shards, _ptr(part_acc), _ptr(part_ml),
                                           _ptr(part_argmax), _ptr(row_offsets), _ptr(out), 1 if out.dtype == torch.float16 else 0,
                                           _ptr(lse_out), _ptr(argmax_out), _stream(stream)), "iq_combine_splits_sharded")
+
+
+def iq_decode_step_workspace_bytes(shape: Shape, num_splits: int) -> int:
+    cs = shape.c()
+    return int(_lib.iq_decode_step_workspace_bytes(ctypes.byref(cs), num_splits))
+
+
+def iq_decode_step_fused(shape: Shape, rot_dev, codebook: Codebook, q, k_new, v_new, cache: Cache, seq_lens_dev, num_splits: int,
+                         workspace, out, lse_out=None, argmax_out=None, status_dev=None, stream=None) -> None:
+    """The decode step in two launches: the decode kernel also appends k_new / v_new [B][H_kv][d] at row seq_lens[b]
+    (the lengths before the step), the merge takes the new row's partial as one more slot and rotates back into `out`.
+    `workspace`: a device uint8 tensor of iq_decode_step_workspace_bytes(shape, num_splits) bytes."""
+    cs, cb, cc = shape.c(), codebook.c(), cache.c()
+    _check(_lib.iq_decode_step_fused(ctypes.byref(cs), _ptr(rot_dev), ctypes.byref(cb), _ptr(q), _ptr(k_new), _ptr(v_new),
+                                     ctypes.byref(cc), _ptr(seq_lens_dev), num_splits, _ptr(workspace), _ptr(out),
+                                     1 if out.dtype == torch.float16 else 0, _ptr(lse_out), _ptr(argmax_out), _ptr(status_dev),
+                                     _stream(stream)), "iq_decode_step_fused")
 
 
 def iq_static_scratch_bytes() -> int:

@@ -401,9 +401,10 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }
 
-int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook, const void* q,
-                        const iq_cache* cache, const int32_t* seq_lens_dev, int32_t num_splits, float* part_acc,
-                        float* part_ml, int32_t* part_argmax, uint32_t* status_dev, void* stream) {
+// Validation and kernel parameters shared by the decode entry points.
+static int decode_params(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook, const void* q,
+                         const iq_cache* cache, const int32_t* seq_lens_dev, int32_t num_splits, float* part_acc,
+                         float* part_ml, int32_t* part_argmax, uint32_t* status_dev, iq::DecodeParams& p) {
   int rc = check_shape(shape);
   if (rc) return rc;
   if (!rot_dev || !q || !seq_lens_dev || !part_acc || !part_ml) return IQ_ERR_NULL;
@@ -419,9 +420,7 @@ int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_co
     if (items * num_splits >= (1ll << 31) || items * (shape->t_cap / iq::DEC_BLOCK_TOKENS) >= (1ll << 31)) return IQ_ERR_LIMIT;
   }
   if (!aligned16(q) || !aligned16(part_acc) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
-  if (shape->batch == 0) return IQ_OK;
 
-  iq::DecodeParams p;
   p.k_codes = cache->k_codes;
   p.k_scales = cache->k_scales;
   p.v_codes = cache->v_codes;
@@ -456,14 +455,86 @@ int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_co
   p.lut8[0] = p.lut8[1] = 0u;
   if (grid8)
     for (int i = 0; i < 8; i++) p.lut8[i >> 2] |= (uint32_t)(uint8_t)(int8_t)n8[i] << (8 * (i & 3));
+  p.k_new = p.v_new = nullptr;
+  p.new_acc = p.new_ml = nullptr;
+  std::memcpy(p.thresholds, codebook->thresholds, sizeof(p.thresholds));
+  std::memcpy(p.levels, codebook->levels, sizeof(p.levels));
+  return IQ_OK;
+}
+
+int iq_decode_attention(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook, const void* q,
+                        const iq_cache* cache, const int32_t* seq_lens_dev, int32_t num_splits, float* part_acc,
+                        float* part_ml, int32_t* part_argmax, uint32_t* status_dev, void* stream) {
+  iq::DecodeParams p;
+  const int rc = decode_params(shape, rot_dev, codebook, q, cache, seq_lens_dev, num_splits, part_acc, part_ml, part_argmax, status_dev, p);
+  if (rc) return rc;
+  if (shape->batch == 0) return IQ_OK;
   const cudaError_t e = iq::launch_decode_attention(p, shape->head_dim, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }
 
-int iq_combine_splits_sharded(const iq_shape* shape, const float* rot_dev, int32_t num_splits, int32_t n_shards,
-                              const float* part_acc, const float* part_ml, const int32_t* part_argmax,
-                              const int32_t* row_offsets_dev, void* out, int32_t out_is_fp16, float* lse_out,
-                              int32_t* argmax_out, void* stream) {
+// Sections of the decode step's workspace, in bytes from its start (each a multiple of 16).
+namespace {
+struct StepWorkspace {
+  size_t part_acc, part_ml, new_acc, new_ml, part_argmax, total;
+};
+StepWorkspace step_workspace(const iq_shape* s, int32_t num_splits) {
+  auto up = [](size_t x) { return (x + 15) & ~(size_t)15; };
+  const size_t bh = (size_t)s->batch * s->n_q_heads, S = (size_t)num_splits, D = (size_t)s->head_dim;
+  StepWorkspace w;
+  size_t o = 0;
+  w.part_acc = o; o += up(bh * S * D * 4);
+  w.part_ml = o; o += up(bh * S * 8);
+  w.new_acc = o; o += up(bh * D * 4);
+  w.new_ml = o; o += up(bh * 8);
+  w.part_argmax = o; o += up(bh * S * 4);
+  w.total = o;
+  return w;
+}
+}  // namespace
+
+size_t iq_decode_step_workspace_bytes(const iq_shape* shape, int32_t num_splits) {
+  if (check_shape(shape) || num_splits < 1 || num_splits > 65535) return 0;
+  return step_workspace(shape, num_splits).total;
+}
+
+static int combine_with_new_row(const iq_shape* shape, const float* rot_dev, int32_t num_splits, int32_t n_shards, const float* part_acc,
+                                const float* part_ml, const int32_t* part_argmax, const int32_t* row_offsets_dev, const float* new_acc,
+                                const float* new_ml, const int32_t* new_rows, void* out, int32_t out_is_fp16, float* lse_out,
+                                int32_t* argmax_out, void* stream);
+
+int iq_decode_step_fused(const iq_shape* shape, const float* rot_dev, const iq_codebook* codebook, const void* q,
+                         const void* k_new, const void* v_new, const iq_cache* cache, const int32_t* seq_lens_dev,
+                         int32_t num_splits, void* workspace_dev, void* out, int32_t out_is_fp16, float* lse_out,
+                         int32_t* argmax_out, uint32_t* status_dev, void* stream) {
+  if (!workspace_dev || !out || !k_new || !v_new) return IQ_ERR_NULL;
+  if (!aligned16(workspace_dev) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new)) return IQ_ERR_ALIGN;
+  int rc = check_shape(shape);
+  if (rc) return rc;
+  if (num_splits < 1 || num_splits > 65535) return IQ_ERR_SHAPE;
+  const StepWorkspace w = step_workspace(shape, num_splits);
+  uint8_t* ws = static_cast<uint8_t*>(workspace_dev);
+  float* part_acc = reinterpret_cast<float*>(ws + w.part_acc);
+  float* part_ml = reinterpret_cast<float*>(ws + w.part_ml);
+  int32_t* part_argmax = argmax_out ? reinterpret_cast<int32_t*>(ws + w.part_argmax) : nullptr;
+  iq::DecodeParams p;
+  rc = decode_params(shape, rot_dev, codebook, q, cache, seq_lens_dev, num_splits, part_acc, part_ml, part_argmax, status_dev, p);
+  if (rc) return rc;
+  if (shape->batch == 0) return IQ_OK;
+  p.k_new = static_cast<const __half*>(k_new);
+  p.v_new = static_cast<const __half*>(v_new);
+  p.new_acc = reinterpret_cast<float*>(ws + w.new_acc);
+  p.new_ml = reinterpret_cast<float*>(ws + w.new_ml);
+  const cudaError_t e = iq::launch_decode_attention(p, shape->head_dim, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return IQ_ERR_CUDA;
+  return combine_with_new_row(shape, rot_dev, num_splits, 1, part_acc, part_ml, part_argmax, nullptr, p.new_acc, p.new_ml, seq_lens_dev,
+                              out, out_is_fp16, lse_out, argmax_out, stream);
+}
+
+static int combine_with_new_row(const iq_shape* shape, const float* rot_dev, int32_t num_splits, int32_t n_shards, const float* part_acc,
+                                const float* part_ml, const int32_t* part_argmax, const int32_t* row_offsets_dev, const float* new_acc,
+                                const float* new_ml, const int32_t* new_rows, void* out, int32_t out_is_fp16, float* lse_out,
+                                int32_t* argmax_out, void* stream) {
   int rc = check_shape(shape);
   if (rc) return rc;
   if (!rot_dev || !part_acc || !part_ml || !out) return IQ_ERR_NULL;
@@ -487,8 +558,19 @@ int iq_combine_splits_sharded(const iq_shape* shape, const float* rot_dev, int32
   p.shards = n_shards;
   p.row_offsets = row_offsets_dev;
   p.out_is_fp16 = out_is_fp16;
+  p.new_acc = new_acc;
+  p.new_ml = new_ml;
+  p.new_rows = new_rows;
   const cudaError_t e = iq::launch_combine_splits(p, shape->head_dim, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
+}
+
+int iq_combine_splits_sharded(const iq_shape* shape, const float* rot_dev, int32_t num_splits, int32_t n_shards,
+                              const float* part_acc, const float* part_ml, const int32_t* part_argmax,
+                              const int32_t* row_offsets_dev, void* out, int32_t out_is_fp16, float* lse_out,
+                              int32_t* argmax_out, void* stream) {
+  return combine_with_new_row(shape, rot_dev, num_splits, n_shards, part_acc, part_ml, part_argmax, row_offsets_dev, nullptr, nullptr,
+                              nullptr, out, out_is_fp16, lse_out, argmax_out, stream);
 }
 
 int iq_combine_splits(const iq_shape* shape, const float* rot_dev, int32_t num_splits, const float* part_acc,

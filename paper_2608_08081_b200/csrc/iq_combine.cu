@@ -45,17 +45,21 @@ __global__ void __launch_bounds__(WPH == 1 ? CMB_WARPS * 32 : WPH * 32) combine_
   float v[E];
 #pragma unroll
   for (int e = 0; e < E; e++) v[e] = 0.f;
-  if (WPH == 1 && S <= 32) {
-    // few slots: lane s takes (m, l, argmax) of slot s, the reference and the weights come from warp reductions, and the
-    // acc rows are then loaded four at a time (their addresses do not depend on one another)
+  // The warp's run of slots: all of them (WPH = 1), else an equal share of consecutive slots.
+  const int chunk = WPH == 1 ? S : (S + WPH - 1) / WPH;
+  const int c0 = WPH == 1 ? 0 : warp * chunk;
+  const int cn = max(0, min(chunk, S - c0));
+  if (chunk <= 32) {
+    // at most 32 slots per warp: lane j takes (m, l, argmax) of slot c0 + j, the reference and the weights come from warp
+    // reductions, and the acc rows are then loaded eight at a time (their addresses do not depend on one another)
     float ms = -INFINITY, ls = 0.f;
     int idx = -1;
     size_t o = 0;
-    if (lane < S) {
-      o = slot_index(lane);
+    if (lane < cn) {
+      o = slot_index(c0 + lane);
       ms = p.part_ml[2 * o];
       ls = p.part_ml[2 * o + 1];
-      if (ls > 0.f) idx = slot_argmax(lane, o);
+      if (ls > 0.f) idx = slot_argmax(c0 + lane, o);
       else ms = -INFINITY;
     }
     m = ms;
@@ -71,20 +75,21 @@ __global__ void __launch_bounds__(WPH == 1 ? CMB_WARPS * 32 : WPH * 32) combine_
     l = ls * w;
 #pragma unroll
     for (int d2 = 16; d2 > 0; d2 >>= 1) l += __shfl_xor_sync(FULL, l, d2);
-    for (int sb = 0; sb < S; sb += 4) {
-      float4 f[4][E / 4];
-      float ws[4];
+    constexpr int NF = 8;  // rows in flight
+    for (int sb = 0; sb < cn; sb += NF) {
+      float4 f[NF][E / 4];
+      float ws[NF];
 #pragma unroll
-      for (int k = 0; k < 4; k++) {
+      for (int k = 0; k < NF; k++) {
         ws[k] = __shfl_sync(FULL, w, (sb + k) & 31);
         const size_t ok = __shfl_sync(FULL, o, (sb + k) & 31);
-        if (sb + k >= S) ws[k] = 0.f;
+        if (sb + k >= cn) ws[k] = 0.f;
 #pragma unroll
         for (int e4 = 0; e4 < E / 4; e4++)
           f[k][e4] = ws[k] != 0.f ? *reinterpret_cast<const float4*>(p.part_acc + ok * D + lane * E + 4 * e4) : make_float4(0.f, 0.f, 0.f, 0.f);
       }
 #pragma unroll
-      for (int k = 0; k < 4; k++)
+      for (int k = 0; k < NF; k++)
 #pragma unroll
         for (int e4 = 0; e4 < E / 4; e4++) {
           v[4 * e4] += ws[k] * f[k][e4].x; v[4 * e4 + 1] += ws[k] * f[k][e4].y; v[4 * e4 + 2] += ws[k] * f[k][e4].z; v[4 * e4 + 3] += ws[k] * f[k][e4].w;
@@ -138,6 +143,26 @@ __global__ void __launch_bounds__(WPH == 1 ? CMB_WARPS * 32 : WPH * 32) combine_
       l += sl[w2] * w;
 #pragma unroll
       for (int e = 0; e < E; e++) v[e] += w * sv[w2][lane * E + e];
+    }
+  }
+  if (p.new_ml) {  // the step's new row: one more slot (its row index is the highest of the sequence: it wins no tie)
+    const float mn = p.new_ml[2 * (size_t)bh], ln = p.new_ml[2 * (size_t)bh + 1];
+    if (ln > 0.f) {
+      const bool had = l > 0.f;
+      const float m2 = had ? fmaxf(m, mn) : mn;
+      const float wa = had ? __expf(m - m2) : 0.f, wn = __expf(mn - m2);
+      const float4* a = reinterpret_cast<const float4*>(p.new_acc + (size_t)bh * D + lane * E);
+#pragma unroll
+      for (int e4 = 0; e4 < E / 4; e4++) {
+        const float4 f = a[e4];
+        v[4 * e4] = fmaf(wn, f.x, wa * v[4 * e4]);
+        v[4 * e4 + 1] = fmaf(wn, f.y, wa * v[4 * e4 + 1]);
+        v[4 * e4 + 2] = fmaf(wn, f.z, wa * v[4 * e4 + 2]);
+        v[4 * e4 + 3] = fmaf(wn, f.w, wa * v[4 * e4 + 3]);
+      }
+      l = fmaf(ln, wn, wa * l);
+      if (!had || mn > m) best = p.new_rows[bh / p.n_q_heads];
+      m = m2;
     }
   }
   const bool empty = !(l > 0.f);

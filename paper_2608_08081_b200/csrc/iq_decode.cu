@@ -29,6 +29,7 @@
 // Packed tiles arrive through a 1-D bulk-copy (TMA) pipeline; every mbarrier wait is bounded in time.
 #include <climits>
 
+#include "iq_append_row.cuh"
 #include "iq_decode_common.cuh"
 #include "iq_kernels.h"
 
@@ -140,7 +141,8 @@ struct DecDrawn {
 // no block of, the slots of an item beyond its last piece (those with index = grp mod ng) -- are marked unused. Unit
 // mode: the next block of the worker's current run, else of its next run with blocks (runs without blocks are marked
 // unused). Nothing is loaded from global memory unless the walk moves to another sequence (or the cache is paged).
-__device__ __forceinline__ void dec_draw(const DecodeParams& p, DecWalk& w, DecDrawn& d, int* next_s, int lane, int D, int with_argmax) {
+template <int D>
+__device__ __forceinline__ void dec_draw(const DecodeParams& p, DecWalk& w, DecDrawn& d, int* next_s, int lane, int with_argmax) {
   constexpr int TB = DEC_BLOCK_TOKENS;
   const int S = p.splits, B = p.batch;
   auto len_of = [&](int b) { return max(0, min(p.seq_lens[b], p.t_cap)); };
@@ -268,6 +270,89 @@ static __device__ __noinline__ void dec_write_operand(uint8_t* dst, int hh, DecH
   }
 }
 
+// Decode with append: the step's new K and V rows are quantised and appended (Algorithm 1) by the launch that attends
+// to them. CTA c takes (sequence, KV head) units c, c + grid, ...; one warp quantises the two rows, writes them to the
+// cache and writes the new row's own partial (m, l) = (z, 1), acc = v~ -- computed from the row's codes and stored
+// scale, like a cached row's -- which the merge reads as one more slot. The blocks of the cache are read WITHOUT that
+// row (rows below seq_lens[b]), so nothing the other warps load depends on these writes.
+template <int D>
+static __device__ __noinline__ void dec_aux_work(const DecodeParams& p, int lane) {
+  constexpr int E = D / 32;
+  const int n_units = p.batch * p.n_kv_heads;
+  for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const int b = u / p.n_kv_heads, kvh = u - b * p.n_kv_heads;
+    const int raw_len = p.seq_lens[b];
+    {
+      bool have_new = false;
+      size_t row = 0;
+      if (raw_len < 0 || raw_len >= p.t_cap) {
+        if (lane == 0 && p.status) {  // counted per (row, KV head, tensor)
+          atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
+          atomicAdd(&p.status[2], 2u);
+        }
+      } else if (!cache_row_for_write(p.pm, b, kvh, raw_len, p.status, row)) {  // no such page: skipped and counted
+        if (lane == 0 && p.status) atomicAdd(&p.status[2], 2u);
+      } else {
+        have_new = true;
+      }
+      if (have_new) {
+        const RowSink sink{const_cast<uint8_t*>(p.k_codes), const_cast<float*>(p.k_scales), const_cast<uint8_t*>(p.v_codes),
+                           const_cast<float*>(p.v_scales), p.status, p.scale_f16};
+        const size_t src = ((size_t)b * p.n_kv_heads + kvh) * D + lane * E;
+        __half2 raw_k[E / 2], raw_v[E / 2];
+#pragma unroll
+        for (int k = 0; k < E / 2; k++) {
+          raw_k[k] = reinterpret_cast<const __half2*>(p.k_new + src)[k];
+          raw_v[k] = reinterpret_cast<const __half2*>(p.v_new + src)[k];
+        }
+        WarpRowQuantizer<D> rq;
+        rq.init(p.rot + (size_t)kvh * (D / 4) * 8, p.thresholds, lane);
+        int code[E];
+        float lk[E], lv[E];
+        float sk = rq.run(raw_k, lane, code, p.status);
+        warp_store_k_row<D>(sink, row, code, sk, lane);
+#pragma unroll
+        for (int e = 0; e < E; e++) lk[e] = p.levels[code[e]];
+        float sv = rq.run(raw_v, lane, code, p.status);
+        warp_store_v_row<D>(sink, row, raw_len, code, sv, lane);
+#pragma unroll
+        for (int e = 0; e < E; e++) lv[e] = p.levels[code[e]];
+        if (p.scale_f16) {  // the scales as the cache holds them
+          sk = __half2float(__float2half_rn(fminf(sk, 65504.f)));
+          sv = __half2float(__float2half_rn(fminf(sv, 65504.f)));
+        }
+        const float vf = sv * rsqrtf((float)D);
+        for (int j = 0; j < p.group; j++) {  // z = sm_scale q~ . k~ of the new row, head by head; (m, l) = (z, 1), acc = v~
+          const size_t bh = (size_t)b * p.n_q_heads + kvh * p.group + j;
+          const DecHeadCoords<D> c = dec_rotate_head<D>(p.q + bh * D, p.rot + (size_t)kvh * (D / 4) * 8, lane);
+          float dot = 0.f;
+#pragma unroll
+          for (int e = 0; e < E; e++) dot = fmaf(c.v[e], lk[e], dot);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(FULL, dot, o);
+          float4* a = reinterpret_cast<float4*>(p.new_acc + bh * D + lane * E);
+#pragma unroll
+          for (int e4 = 0; e4 < E / 4; e4++) a[e4] = make_float4(lv[4 * e4] * vf, lv[4 * e4 + 1] * vf, lv[4 * e4 + 2] * vf, lv[4 * e4 + 3] * vf);
+          if (lane == 0) {
+            p.new_ml[2 * bh] = dot * sk * p.sm_scale * rsqrtf((float)D);  // z = sm_scale q~ . (s level / sqrt d)
+            p.new_ml[2 * bh + 1] = 1.f;
+          }
+        }
+      } else if (lane < p.group) {
+        const size_t bh = (size_t)b * p.n_q_heads + kvh * p.group + lane;
+        p.new_ml[2 * bh] = -INFINITY;
+        p.new_ml[2 * bh + 1] = 0.f;
+      }
+      if (!have_new)
+        for (int j = 32 + lane; j < p.group; j += 32) {  // (more than 32 heads per KV head)
+          const size_t bh = (size_t)b * p.n_q_heads + kvh * p.group + j;
+          p.new_ml[2 * bh] = -INFINITY;
+          p.new_ml[2 * bh + 1] = 0.f;
+        }
+    }
+  }
+}
+
 // Where the CTA's range starts (thread 0, set-up).
 struct DecStart {
   int b, y, len, piece;  // sequence, item within it, rows of the sequence, which piece of the item the range starts in
@@ -276,7 +361,7 @@ struct DecStart {
   int count, pad;       // blocks of the range
 };
 
-template <int D, bool ARGMAX, bool I8>
+template <int D, bool ARGMAX, bool I8, bool APPEND>
 __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const __grid_constant__ DecodeParams p) {
   using L = DecLayout<D>;
   constexpr int DJ = L::DJ;
@@ -291,6 +376,9 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const bool control = warp >= NG * 4;
   const int grp = control ? warp - NG * 4 : warp >> 2;  // group of this warp
+  // decode with append: the last control warp first does the CTA's share of the appends; its group starts that much
+  // later, and the other groups draw the blocks meanwhile
+  const bool aux = APPEND && warp == NG * 5 - 1;
   const int gt = tid & (DEC_GROUP_THREADS - 1);         // compute thread within its group = TMEM lane
   const int bar_id = 1 + grp;                           // named barrier of the group's compute threads
 
@@ -353,6 +441,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
   // strictly increasing along the block sequence; CTA c owns the blocks with c * cper <= C < (c + 1) * cper.
   long long g0 = 0;
   int count = 0;  // blocks of this CTA's range (read from shared memory after the set-up barrier)
+  bool no_work = false;
   if (range_mode) {
     constexpr long long W = DEC_SEG_COST;
     int* cnt_s = scan_s + L::THREADS + L::THREADS / 32;  // [THREADS] non-empty sequences per slice of the batch
@@ -387,8 +476,8 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     cper = max(cper, (long long)((nb_max + W - 1) / (S / NG - 1) + 1));  // an item then spans at most S / NG ranges
     cper = max(cper, W + 1);                                              // and no range between two ranges of blocks is empty
     const long long t_lo = (long long)blockIdx.x * cper;
-    if (t_lo >= c_total) return;
-    if (tid == 0) {
+    if (t_lo >= c_total) no_work = true;
+    if (tid == 0 && !no_work) {
       // the first block at or after cost position t: its sequence, item, block, and launch-wide block index
       auto locate = [&](long long t, int& b, int& nb, int& y, int& blk, long long& before_nb, long long& c_b) {
         before_nb = 0;  // blocks (per item column) of the sequences before b
@@ -449,8 +538,15 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     }
   } else {
     // unit mode: worker w = grp * grid + CTA takes units w, w + NG * grid, ...; a CTA none of whose groups has a unit leaves
-    if ((long long)blockIdx.x >= (long long)B * ips * S) return;
+    if ((long long)blockIdx.x >= (long long)B * ips * S) no_work = true;
     if (tid == 0) *n_pre_s = 0;
+  }
+  if (no_work) {  // a CTA without blocks still has its share of the appends
+    if (aux) {
+      grid_dependency_wait();
+      dec_aux_work<D>(p, lane);
+    }
+    return;
   }
 
   // ---------------------------------------------------------------- set-up: barriers, TMEM
@@ -484,6 +580,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
   const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;                // this warp's 32 TMEM lanes
   bool failed = false;  // a bounded wait gave up; every later wait of this thread is skipped
 
+  if (aux) dec_aux_work<D>(p, lane);
   if (control) {
     // ================================================================ control warp of group grp: walks the work, fetches blocks, issues MMAs.
     // All 32 lanes run the loop and the waits (the walk is uniform over the warp); an elected lane issues.
@@ -517,7 +614,9 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
     // memory) while the compute warps are busy with the softmax of the current one, and staged after the value MMAs.
     DecDrawn dr;
     dr.kind = -1;
-    auto draw = [&]() { dec_draw(p, wk, dr, next_s, lane, D, ARGMAX ? 1 : 0); };
+    auto draw = [&]() {
+      dec_draw<D>(p, wk, dr, next_s, lane, ARGMAX ? 1 : 0);
+    };
     auto stage_next = [&]() {  // the drawn (or next) block into slot it_issue, or the end marker
       const int st = it_issue % NST;
       if (it_issue >= NST && !failed)  // the slot's previous occupant has been consumed
@@ -1180,7 +1279,7 @@ __global__ void __launch_bounds__(DecLayout<D>::THREADS, 1) decode_kernel(const 
   if (warp == NG * 4) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512));
 }
 
-template <int D, bool ARGMAX, bool I8>
+template <int D, bool ARGMAX, bool I8, bool APPEND>
 static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
   using L = DecLayout<D>;
   static bool configured[64] = {};
@@ -1189,7 +1288,7 @@ static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-  auto kern = decode_kernel<D, ARGMAX, I8>;
+  auto kern = decode_kernel<D, ARGMAX, I8, APPEND>;
   if (!configured[dev]) {
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::SMEM_BYTES);
     if (e != cudaSuccess) return e;
@@ -1202,17 +1301,25 @@ static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
   long long ctas = n_sm[dev];
   if (ctas > max_blocks) ctas = max_blocks;
   if (ctas < 1) ctas = 1;
+  if (APPEND) {  // the appends are spread over the CTAs whatever the number of blocks
+    const long long units = (long long)p.batch * p.n_kv_heads;
+    if (ctas < units) ctas = units < n_sm[dev] ? units : n_sm[dev];
+  }
   return launch_after_predecessor(kern, dim3((unsigned)ctas), dim3(L::THREADS), L::SMEM_BYTES, stream, p);
 }
 
-cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream) {
+template <bool APPEND>
+static cudaError_t launch_decode_variant(const DecodeParams& p, int head_dim, cudaStream_t stream) {
   const bool am = p.part_argmax != nullptr;
   if (p.use_i8) {  // levels on an 8-bit grid: int8 operands, int32 accumulation
-    if (head_dim == 128) return am ? launch_one<128, true, true>(p, stream) : launch_one<128, false, true>(p, stream);
-    return am ? launch_one<256, true, true>(p, stream) : launch_one<256, false, true>(p, stream);
+    if (head_dim == 128) return am ? launch_one<128, true, true, APPEND>(p, stream) : launch_one<128, false, true, APPEND>(p, stream);
+    return am ? launch_one<256, true, true, APPEND>(p, stream) : launch_one<256, false, true, APPEND>(p, stream);
   }
-  if (head_dim == 128) return am ? launch_one<128, true, false>(p, stream) : launch_one<128, false, false>(p, stream);
-  return am ? launch_one<256, true, false>(p, stream) : launch_one<256, false, false>(p, stream);
+  if (head_dim == 128) return am ? launch_one<128, true, false, APPEND>(p, stream) : launch_one<128, false, false, APPEND>(p, stream);
+  return am ? launch_one<256, true, false, APPEND>(p, stream) : launch_one<256, false, false, APPEND>(p, stream);
+}
+cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream) {
+  return p.k_new ? launch_decode_variant<true>(p, head_dim, stream) : launch_decode_variant<false>(p, head_dim, stream);
 }
 
 // Self-test of the bounded wait: one warp waits, with `polls` as its limit, on a barrier that nothing completes (no
@@ -1243,3 +1350,4 @@ int decode_groups_per_cta(int head_dim) { return head_dim == 128 ? DecLayout<128
 int decode_ctas_per_sm(int head_dim) { (void)head_dim; return 1; }
 
 }  // namespace iq
+

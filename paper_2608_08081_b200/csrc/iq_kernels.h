@@ -90,6 +90,16 @@ struct DecodeParams {
   uint32_t lut8[2];
   float delta;
   int use_i8;
+  // Decode with append (k_new != nullptr; otherwise none of the following is read): the step's new K and V rows
+  // [batch][n_kv_heads][head_dim] are quantised and appended at row seq_lens[b] by one warp per (sequence, KV head),
+  // which also writes the new row's own partial (new_acc [batch][n_q_heads][head_dim], new_ml [batch][n_q_heads][2]);
+  // the blocks of the cache are read up to row seq_lens[b] - 1.
+  const __half* k_new;
+  const __half* v_new;
+  float* new_acc;
+  float* new_ml;
+  float thresholds[7];
+  float levels[8];
 };
 cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream);
 int decode_ctas_per_sm(int head_dim);
@@ -111,6 +121,10 @@ struct CombineParams {
   // rows of the whole sequence. shards = 1 is the plain layout.
   int shards;
   const int32_t* row_offsets;
+  // Decode with append: the partial of the step's new row, one more slot per head (nullptr: none); its row is new_rows[b].
+  const float* new_acc;
+  const float* new_ml;
+  const int32_t* new_rows;
 };
 cudaError_t launch_combine_splits(const CombineParams& p, int head_dim, cudaStream_t stream);
 
