@@ -66,7 +66,7 @@ def decode_traffic_bytes(algorithmic_bytes: float, B: int, H_q: int, S: int, d: 
 
 
 def bytes_per_row(d: int) -> int:
-    return 2 * (3 * d // 8) + 2 * (2 if SCALES_F16 else 4)   # K and V codes + scales, per cached row per KV head
+    return 2 * (BITS * d // 8) + 2 * (2 if SCALES_F16 else 4)   # K and V codes + scales, per cached row per KV head
 
 
 def measured_peak_hbm():
@@ -164,6 +164,7 @@ def aggregate_gbs(bytes_per_rank: float, ms: float, world: int) -> float:
 
 SCALES_F16 = False  # binary16 scale arrays: 100 instead of 104 bytes per cached row and KV head
 PAGE_ROWS = 0       # > 0: the cache is a pool of pages of this many rows behind a block table in scrambled order
+BITS = 3            # bits per code (Algorithm 1's b); the paper's and the benchmark's configurations are 3-bit
 CODEBOOK = "int8"   # "int8": Lloyd-Max levels on an 8-bit grid (integer tensor-core decode path); "fp16": exact fp16 levels
 
 
@@ -177,8 +178,8 @@ def build_state(name: str, device, rank: int):
     B, ctx, H_q, H_kv, d = WORKLOADS[name]
     gen = workloads.config5_device(B, ctx, device, H_q, H_kv, d, full_lengths=name in PER_SEQUENCE_LAUNCHES)
     t_cap = ctx + T_CAP_MARGIN
-    shape = iq.Shape(B, H_q, H_kv, d, t_cap)
-    cb = iq.iq_int8_codebook(d) if CODEBOOK == "int8" else iq.iq_default_codebook(d)
+    shape = iq.Shape(B, H_q, H_kv, d, t_cap, bits=BITS)
+    cb = iq.iq_lloyd_max_codebook(d, BITS, CODEBOOK)
     rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device=device)
     iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(gen["quats"]), rot)
     if PAGE_ROWS:
@@ -194,7 +195,7 @@ def build_state(name: str, device, rank: int):
     qa_ms, qa_rows = 0.0, 0
     for b0, k, v in gen["chunks"]():
         nb = k.shape[0]
-        sub = iq.Shape(nb, H_q, H_kv, d, t_cap)
+        sub = iq.Shape(nb, H_q, H_kv, d, t_cap, bits=BITS)
         if PAGE_ROWS:   # the pool is shared; the chunk's sequences are rows b0 .. b0 + nb of the block table
             view = iq.Cache(cache.k_codes, cache.k_scales, cache.v_codes, cache.v_scales, cache.block_table[b0:b0 + nb], PAGE_ROWS)
         else:
@@ -213,7 +214,7 @@ def build_state(name: str, device, rank: int):
         del k, v
     qa = None
     if qa_rows:
-        bytes_per_row = 2 * d + 3 * d // 8 + 4   # fp16 in + packed codes + fp32 scale out
+        bytes_per_row = 2 * d + BITS * d // 8 + 4   # fp16 in + packed codes + fp32 scale out
         peak, _ = measured_peak_hbm()
         gbs = qa_rows * bytes_per_row / (qa_ms * 1e-3) / 1e9
         qa = {"rows_per_s": round(qa_rows / (qa_ms * 1e-3), 1), "gb_per_s": round(gbs, 1), "frac_of_hbm_peak": round(gbs / peak, 4),
@@ -249,7 +250,7 @@ class StepRunner:
         self.B, self.H_q, self.H_kv, self.d = st["B"], st["H_q"], st["H_kv"], st["d"]
         # Launch groups: the whole batch in one set of launches, or (stack-of-layers workloads) one set per sequence.
         self.per_seq = name in PER_SEQUENCE_LAUNCHES
-        self.gshape = iq.Shape(1, self.H_q, self.H_kv, self.d, st["t_cap"]) if self.per_seq else st["shape"]
+        self.gshape = iq.Shape(1, self.H_q, self.H_kv, self.d, st["t_cap"], bits=BITS) if self.per_seq else st["shape"]
         self.S = splits or iq.iq_suggest_splits(self.gshape, st["ctx"])
         self.ws = iq.DecodeWorkspace(st["shape"], self.S, want_argmax=False, device=device)
         # Row i of this table holds the sequence lengths before step i: the step appends at lens_tab[i] and attends to
@@ -411,7 +412,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     import torch
     import torch.distributed as dist
 
-    global CODEBOOK
+    global CODEBOOK, BITS
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
     K, W = args.steps, args.warmup
@@ -510,7 +511,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         "higher_is_better": True,
         "scaling": "weak",
         "vs_baseline": None,
-        "dtype": ("u3 codes, int8 tensor-core operands, int32 accumulate" if CODEBOOK == "int8"
+        "dtype": (f"u{BITS} codes, int8 tensor-core operands, int32 accumulate" if CODEBOOK == "int8"
                   else "u3 codes, f16 tensor-core operands, f32 accumulate"),
         "data": "synthetic",
         "config": {"workload": args.workload, "batch": B, "ctx": st["ctx"], "n_q_heads": H_q, "n_kv_heads": H_kv, "head_dim": d,
@@ -569,6 +570,17 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             out["decode_fp16_codebook" if CODEBOOK == "fp16" else "decode_int8_codebook"] = o
         finally:
             CODEBOOK = main_cb
+        # the other bit widths of Algorithm 1 on the same workload (cache rebuilt at that width; the paper's setting is 3 bits)
+        out["other_bit_widths"] = {}
+        for b in (2, 4):
+            BITS = b
+            try:
+                o = point_summary(args.workload, device, rank)
+                o["bits"] = b
+                o["bytes_per_row_per_kv_head"] = bytes_per_row(d)
+                out["other_bit_widths"][str(b)] = o
+            finally:
+                BITS = 3
     return out
 
 
@@ -674,10 +686,10 @@ def run_reference(args, rank: int, world: int):
     nb = 1
     T = int(lens_all[0])
     g = np.random.Generator(np.random.Philox(workloads.stream_seed(5, 0) + 7))
-    lv, th = lloyd_max.int8_codebook(d) if CODEBOOK == "int8" else lloyd_max.fp16_codebook(d)
+    lv, th = lloyd_max.int8_codebook(d, 1 << BITS) if CODEBOOK == "int8" else lloyd_max.fp16_codebook(d, 1 << BITS)
     quats = workloads.quaternion_pairs(workloads.rng(5, workloads.QUAT_STREAM), H_kv, d)
-    P = oracle.row_bytes(d)
-    cache = oracle.new_cache(nb, H_kv, d, workloads.cap128(T + args.warmup + args.steps + 1))
+    P = oracle.row_bytes(d, BITS)
+    cache = oracle.new_cache(nb, H_kv, d, workloads.cap128(T + args.warmup + args.steps + 1), BITS)
     # the sample's cache content: uniformly random codes and Gaussian-row-like scales (the decode cost does not depend on values)
     cache["k_codes"][:] = g.integers(0, 256, cache["k_codes"].shape, dtype=np.uint8)
     cache["v_codes"][:] = g.integers(0, 256, cache["v_codes"].shape, dtype=np.uint8)
@@ -724,8 +736,10 @@ def main():
     ap.add_argument("--min-region", type=float, default=0.5, help="seconds the timed region must last: the K steps are repeated until it does")
     ap.add_argument("--no-sweep", action="store_true", help="skip the other config-5 points and the other codebook's decode path")
     ap.add_argument("--codebook", default="int8", choices=["int8", "fp16"])
+    ap.add_argument("--bits", type=int, default=3, choices=[2, 3, 4], help="bits per code (the headline configuration is 3)")
     args = ap.parse_args()
-    global CODEBOOK, PAGE_ROWS, SCALES_F16
+    global CODEBOOK, PAGE_ROWS, SCALES_F16, BITS
+    BITS = args.bits
     SCALES_F16 = args.scales == "fp16"
     CODEBOOK = args.codebook
     PAGE_ROWS = args.page_rows

@@ -35,24 +35,32 @@
  *   (q_L.wxyz, q_R.wxyz): 8 floats per block, 256 per head at d = 128 (Appendix B). K and V of a KV head
  *   and all query heads of its group share that head's rotation.
  *
- * Codebook (Section 3.2, Step 3)
- *   8 ascending levels and 7 ascending decision thresholds in unit-variance units u = sqrt(d) * x~.
- *   code = #{ j : u > t_j } (strict: an exact tie takes the lower code). A dequantised coordinate is
- *   scale * level[code] / sqrt(d). iq_quantize_append uses the thresholds only and takes any ascending set.
+ * Codebook (Section 3.2, Step 3; Algorithm 1 is written for a general bit width b and codebook C_b)
+ *   2^b ascending levels and 2^b - 1 ascending decision thresholds in unit-variance units u = sqrt(d) * x~, b = bits
+ *   in {2, 3, 4}. code = #{ j : u > t_j } (strict: an exact tie takes the lower code). A dequantised coordinate is
+ *   scale * level[code] / sqrt(d). The K rows and the V rows may have codebooks of their own (separate_v): keys and
+ *   values need not have the same post-rotation marginal. iq_quantize_append uses the thresholds only and takes any
+ *   ascending set.
  *   iq_decode_attention feeds the levels to tensor-core operands without rounding them, so it takes two forms:
  *   levels on an 8-bit grid, level_j = n_j * delta with integers |n_j| <= 127 (iq_int8_codebook, or iq_fit_codebook
- *   with grid = 1): int8 operands, the faster path; or levels that are all exact IEEE binary16 values
- *   (iq_default_codebook, iq_fit_codebook with grid = 0): fp16 operands. Anything else is IQ_ERR_CODEBOOK.
+ *   with grid = 1; with separate_v each side on a grid of its own): int8 operands, the faster path; or levels that
+ *   are all exact IEEE binary16 values (iq_default_codebook, iq_fit_codebook with grid = 0): fp16 operands. Anything
+ *   else is IQ_ERR_CODEBOOK.
  *
- * Packed cache (Section 3.2, Step 4 fixes the size only: 3d/8 bytes per row, 48 at d = 128)
- *   codes: 3d/8 bytes per cached row and side, scales [batch][n_kv_heads][t_cap] fp32 (= ||x||_2), separately
- *   for K and V. The unit of packing is a group of 32 entries in 3 consecutive little-endian 32-bit words: in
- *   group-local numbering, entry c < 24 stores its code in bits [4n, 4n+3) of word c/8, n = c mod 8; entry
- *   c >= 24 (n = c - 24) stores bit k of its code in bit 4n+3 of word k.
- *   K codes [batch][n_kv_heads][t_cap][3d/8]: one packed row per cached row, entries = rotated coordinates.
- *   V codes [batch][n_kv_heads][t_cap/128][d][48]: token-transposed. For every block of 128 cached rows and every
- *   rotated coordinate c there is one 48-byte record holding the 128 codes of coordinate c, entries = row within
- *   the block. (The decode kernel contracts K over coordinates and V over rows; either way the contraction
+ * Packed cache (Section 3.2, Step 4 fixes the size only: b d / 8 bytes per row, 48 at b = 3, d = 128)
+ *   codes: b d / 8 bytes per cached row and side, scales [batch][n_kv_heads][t_cap] fp32 (= ||x||_2), separately
+ *   for K and V. A run of packed entries (a K row, or a V record) is a sequence of little-endian 32-bit words:
+ *     b = 3: groups of 32 entries in 3 consecutive words: in group-local numbering, entry c < 24 stores its code in
+ *            bits [4n, 4n+3) of word c/8, n = c mod 8; entry c >= 24 (n = c - 24) stores bit k of its code in bit 4n+3
+ *            of word k.
+ *     b = 4: entry c stores its code in bits [4n, 4n+4) of word c/8, n = c mod 8.
+ *     b = 2: groups of 16 entries in one word: entry e < 8 of the group in bits [4e, 4e+2), entry e >= 8 in bits
+ *            [4(e-8)+2, 4(e-8)+4).
+ *   (Every layout keeps the codes nibble-aligned, which is what the decode kernel's byte-permute lookups index by.)
+ *   K codes [batch][n_kv_heads][t_cap][b d / 8]: one packed row per cached row, entries = rotated coordinates.
+ *   V codes [batch][n_kv_heads][t_cap/128][d][16 b]: token-transposed. For every block of 128 cached rows and every
+ *   rotated coordinate c there is one record of 16 b bytes (48 at b = 3) holding the 128 codes of coordinate c,
+ *   entries = row within the block. (The decode kernel contracts K over coordinates and V over rows; either way the contraction
  *   index then runs along a packed record.) Bits of rows that were never appended are left as they are.
  *   t_cap must be a multiple of 128 and all four arrays 16-byte aligned.
  */
@@ -66,18 +74,18 @@
 extern "C" {
 #endif
 
-#define IQ_VERSION 200
+#define IQ_VERSION 300
 /* Version of the packed-cache byte layout described above and in docs/FORMAT.md (bit order of a packing unit,
  * token-transposed V records, scale arrays, rotation parameters, partial slots). A cache written under one format
  * version is read correctly only by a library of the same format version; iq_format_version() reports the library's. */
-#define IQ_FORMAT_VERSION 2
+#define IQ_FORMAT_VERSION 3
 
 enum {
   IQ_OK = 0,
   IQ_ERR_NULL = -1,     /* a required pointer is NULL */
   IQ_ERR_SHAPE = -2,    /* unsupported head_dim / bits, n_q_heads % n_kv_heads != 0, bad sizes or strides */
   IQ_ERR_ALIGN = -3,    /* a pointer or stride breaks the stated alignment */
-  IQ_ERR_CODEBOOK = -4, /* levels / thresholds not ascending; decode: levels neither on an 8-bit grid nor exact binary16 */
+  IQ_ERR_CODEBOOK = -4, /* bits differ from the shape's; levels / thresholds not ascending; decode: levels neither on an 8-bit grid nor exact binary16 */
   IQ_ERR_CUDA = -5,     /* the CUDA runtime reported an error for the launch */
   IQ_ERR_LIMIT = -6     /* a size exceeds a documented maximum of the entry point */
 };
@@ -96,13 +104,18 @@ typedef struct iq_shape {
   int32_t n_kv_heads; /* n_q_heads % n_kv_heads == 0 */
   int32_t head_dim;   /* 128 or 256 */
   int32_t t_cap;      /* rows allocated per (sequence, KV head); multiple of 128 */
-  int32_t bits;       /* 3 */
+  int32_t bits;       /* 2, 3 or 4 */
   float sm_scale;     /* softmax scale; <= 0 selects 1/sqrt(head_dim) (Appendix A) */
 } iq_shape;
 
+#define IQ_MAX_LEVELS 16
 typedef struct iq_codebook {
-  float levels[8];
-  float thresholds[7];
+  int32_t bits;                          /* 2, 3 or 4: 2^bits levels, 2^bits - 1 thresholds are read; must equal iq_shape.bits */
+  int32_t separate_v;                    /* 0: the V rows use levels / thresholds too; else v_levels / v_thresholds */
+  float levels[IQ_MAX_LEVELS];           /* K rows (and V rows unless separate_v) */
+  float thresholds[IQ_MAX_LEVELS - 1];
+  float v_levels[IQ_MAX_LEVELS];
+  float v_thresholds[IQ_MAX_LEVELS - 1];
 } iq_codebook;
 
 typedef struct iq_cache {
@@ -132,8 +145,10 @@ int iq_version(void);
 int iq_format_version(void);
 const char* iq_strerror(int code);
 
-/* Bytes of one packed row: 3 * head_dim / 8 (Section 3.2, Step 4). 0 for an unsupported head_dim. */
+/* Bytes of one packed row: bits * head_dim / 8 (Section 3.2, Step 4); iq_row_bytes is the 3-bit case. 0 for an
+ * unsupported head_dim or bit width. The V array of a (sequence, KV head) has the same number of bytes as the K array. */
 size_t iq_row_bytes(int32_t head_dim);
+size_t iq_row_bytes_bits(int32_t head_dim, int32_t bits);
 /* Floats of the rotation parameter buffer: n_kv_heads * (head_dim / 4) * 8 (Appendix B). */
 size_t iq_rotation_floats(int32_t head_dim, int32_t n_kv_heads);
 
@@ -152,6 +167,11 @@ int iq_default_codebook(int32_t head_dim, iq_codebook* out_host);
  * binary16 values and runs on the fp16 path.
  */
 int iq_int8_codebook(int32_t head_dim, iq_codebook* out_host);
+/* The same two codebooks for any bit width (iq_default_codebook / iq_int8_codebook are bits = 3): 2^bits Lloyd-Max
+ * levels for the post-rotation marginal, grid = 0: rounded to binary16, grid = 1: snapped to the 8-bit grid. */
+int iq_lloyd_max_codebook(int32_t head_dim, int32_t bits, int32_t grid, iq_codebook* out_host);
+/* Makes `cb` a two-sided codebook: its V side becomes the K side of `v_side` (same bits). Host only. */
+int iq_codebook_set_v(iq_codebook* cb, const iq_codebook* v_side);
 
 /*
  * Rotation parameters (Appendix B). If quats_host != NULL it holds [n_kv_heads][d/4][8] floats which are
@@ -280,12 +300,13 @@ int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_co
  * kernels take: grid = 0: levels exactly representable in binary16; grid = 1: levels on an 8-bit grid as from
  * iq_int8_codebook; thresholds = midpoints of the final levels. symmetric != 0 averages the histogram with its mirror
  * image first (a codebook symmetric about zero takes the faster decision path of the bulk quantize kernels).
- * IQ_ERR_CODEBOOK if the data has too few distinct values for eight ascending levels.
+ * IQ_ERR_CODEBOOK if the data has too few distinct values for 2^bits ascending levels. Calibrating K and V separately is
+ * two histograms and two fits, joined with iq_codebook_set_v.
  */
 int iq_rotated_histogram(const iq_shape* shape, const float* rot_dev, const void* x, int64_t stride_b,
                          int64_t stride_t, int64_t stride_h, const int32_t* n_rows_dev, int32_t n_rows_max,
                          uint32_t* hist_dev, int32_t bins, float range, void* stream);
-int iq_fit_codebook(const uint32_t* hist_host, int32_t bins, float range, int32_t symmetric, int32_t grid,
+int iq_fit_codebook(const uint32_t* hist_host, int32_t bins, float range, int32_t bits, int32_t symmetric, int32_t grid,
                     iq_codebook* out_host);
 
 /*

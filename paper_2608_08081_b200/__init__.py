@@ -17,6 +17,9 @@ from .binding import (  # noqa: F401
     iq_static_scratch_bytes,
     iq_default_codebook,
     iq_int8_codebook,
+    iq_lloyd_max_codebook,
+    iq_codebook_set_v,
+    iq_row_bytes_bits,
     iq_make_rotation,
     iq_quantize_append,
     iq_rotation_floats,

@@ -21,7 +21,8 @@ class _IqShape(ctypes.Structure):
 
 
 class _IqCodebook(ctypes.Structure):
-    _fields_ = [("levels", ctypes.c_float * 8), ("thresholds", ctypes.c_float * 7)]
+    _fields_ = [("bits", _i32), ("separate_v", _i32), ("levels", ctypes.c_float * 16), ("thresholds", ctypes.c_float * 15),
+                ("v_levels", ctypes.c_float * 16), ("v_thresholds", ctypes.c_float * 15)]
 
 
 class _IqCache(ctypes.Structure):
@@ -52,6 +53,10 @@ def _load():
     lib.iq_strerror.argtypes = [ctypes.c_int]
     lib.iq_row_bytes.restype = ctypes.c_size_t
     lib.iq_row_bytes.argtypes = [_i32]
+    lib.iq_row_bytes_bits.restype = ctypes.c_size_t
+    lib.iq_row_bytes_bits.argtypes = [_i32, _i32]
+    lib.iq_lloyd_max_codebook.argtypes = [_i32, _i32, _i32, ctypes.POINTER(_IqCodebook)]
+    lib.iq_codebook_set_v.argtypes = [ctypes.POINTER(_IqCodebook), ctypes.POINTER(_IqCodebook)]
     lib.iq_rotation_floats.restype = ctypes.c_size_t
     lib.iq_rotation_floats.argtypes = [_i32, _i32]
     lib.iq_default_codebook.argtypes = [_i32, ctypes.POINTER(_IqCodebook)]
@@ -72,7 +77,7 @@ def _load():
                                         ctypes.POINTER(_IqCache), _i32, _vp, _vp, _vp, _vp, _i32, _vp, _vp]
     lib.iq_rotated_histogram.argtypes = [ctypes.POINTER(_IqShape), _vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, _vp,
                                          _i32, _vp, _i32, ctypes.c_float, _vp]
-    lib.iq_fit_codebook.argtypes = [_vp, _i32, ctypes.c_float, _i32, _i32, ctypes.POINTER(_IqCodebook)]
+    lib.iq_fit_codebook.argtypes = [_vp, _i32, ctypes.c_float, _i32, _i32, _i32, ctypes.POINTER(_IqCodebook)]
     lib.iq_suggest_splits.restype = _i32
     lib.iq_suggest_splits.argtypes = [ctypes.POINTER(_IqShape), _i32]
     lib.iq_wht_coordinates.argtypes = [ctypes.POINTER(_IqShape), _vp, _i64, _i64, _i64, _vp, _i32, _vp, _vp]
@@ -110,19 +115,60 @@ class Shape:
 
 @dataclass(frozen=True)
 class Codebook:
+    """2^b ascending levels and 2^b - 1 thresholds (b = 2, 3 or 4, read off the number of levels); v_levels / v_thresholds:
+    a codebook of their own for the V rows (None: the V rows use the same one)."""
     levels: tuple
     thresholds: tuple
+    v_levels: tuple = None
+    v_thresholds: tuple = None
+
+    @property
+    def bits(self) -> int:
+        return {4: 2, 8: 3, 16: 4}[len(self.levels)]
 
     def c(self) -> _IqCodebook:
         cb = self.__dict__.get("_c")
         if cb is None:
+            n = len(self.levels)
+            assert len(self.thresholds) == n - 1
             cb = _IqCodebook()
-            for i in range(8):
+            cb.bits = self.bits
+            for i in range(n):
                 cb.levels[i] = float(self.levels[i])
-            for i in range(7):
+            for i in range(n - 1):
                 cb.thresholds[i] = float(self.thresholds[i])
+            if self.v_levels is not None:
+                assert len(self.v_levels) == n and len(self.v_thresholds) == n - 1
+                cb.separate_v = 1
+                for i in range(n):
+                    cb.v_levels[i] = float(self.v_levels[i])
+                for i in range(n - 1):
+                    cb.v_thresholds[i] = float(self.v_thresholds[i])
             object.__setattr__(self, "_c", cb)
         return cb
+
+    def with_v(self, v_side: "Codebook") -> "Codebook":
+        """This codebook for the K rows, v_side's (K side) for the V rows."""
+        assert v_side.bits == self.bits
+        return Codebook(self.levels, self.thresholds, tuple(v_side.levels), tuple(v_side.thresholds))
+
+
+def _from_c(cb: _IqCodebook) -> Codebook:
+    n = 1 << cb.bits
+    if cb.separate_v:
+        return Codebook(tuple(cb.levels[:n]), tuple(cb.thresholds[:n - 1]), tuple(cb.v_levels[:n]), tuple(cb.v_thresholds[:n - 1]))
+    return Codebook(tuple(cb.levels[:n]), tuple(cb.thresholds[:n - 1]))
+
+
+def iq_codebook_set_v(codebook: Codebook, v_side: Codebook) -> Codebook:
+    """A two-sided codebook: `codebook` for the K rows, the K side of `v_side` for the V rows (through the C ABI)."""
+    a, b = _IqCodebook.from_buffer_copy(codebook.c()), v_side.c()
+    _check(_lib.iq_codebook_set_v(ctypes.byref(a), ctypes.byref(b)), "iq_codebook_set_v")
+    return _from_c(a)
+
+
+def iq_row_bytes_bits(head_dim: int, bits: int) -> int:
+    return int(_lib.iq_row_bytes_bits(head_dim, bits))
 
 
 @dataclass
@@ -173,8 +219,15 @@ def iq_strerror(code: int) -> str:
     return _lib.iq_strerror(int(code)).decode()
 
 
-def iq_row_bytes(head_dim: int) -> int:
-    return int(_lib.iq_row_bytes(head_dim))
+def iq_row_bytes(head_dim: int, bits: int = 3) -> int:
+    return int(_lib.iq_row_bytes_bits(head_dim, bits))
+
+
+def iq_lloyd_max_codebook(head_dim: int, bits: int, grid: str = "int8") -> Codebook:
+    """2^bits Lloyd-Max levels for the post-rotation marginal; grid "int8" (integer decode path) or "fp16"."""
+    cb = _IqCodebook()
+    _check(_lib.iq_lloyd_max_codebook(head_dim, bits, {"fp16": 0, "int8": 1}[grid], ctypes.byref(cb)), "iq_lloyd_max_codebook")
+    return _from_c(cb)
 
 
 def iq_rotation_floats(head_dim: int, n_kv_heads: int) -> int:
@@ -184,13 +237,13 @@ def iq_rotation_floats(head_dim: int, n_kv_heads: int) -> int:
 def iq_default_codebook(head_dim: int) -> Codebook:
     cb = _IqCodebook()
     _check(_lib.iq_default_codebook(head_dim, ctypes.byref(cb)), "iq_default_codebook")
-    return Codebook(tuple(cb.levels), tuple(cb.thresholds))
+    return _from_c(cb)
 
 
 def iq_int8_codebook(head_dim: int) -> Codebook:
     cb = _IqCodebook()
     _check(_lib.iq_int8_codebook(head_dim, ctypes.byref(cb)), "iq_int8_codebook")
-    return Codebook(tuple(cb.levels), tuple(cb.thresholds))
+    return _from_c(cb)
 
 
 def iq_make_rotation(head_dim: int, n_kv_heads: int, seed: int, quats_host, rot_dev: torch.Tensor, stream=None) -> None:
@@ -308,15 +361,15 @@ def iq_rotated_histogram(shape: Shape, rot_dev, x, n_rows_dev, hist_dev, rng_hal
                                      _stream(stream)), "iq_rotated_histogram")
 
 
-def iq_fit_codebook(hist_host, rng_half: float, symmetric: bool = True, grid: str = "int8") -> Codebook:
+def iq_fit_codebook(hist_host, rng_half: float, symmetric: bool = True, grid: str = "int8", bits: int = 3) -> Codebook:
     """Lloyd-Max codebook fitted to a histogram from iq_rotated_histogram (a contiguous int32/uint32 numpy array or CPU
     tensor). grid: "int8" (integer tensor-core decode path) or "fp16" (exact binary16 levels)."""
     h = hist_host.numpy() if isinstance(hist_host, torch.Tensor) else hist_host
     assert h.dtype.itemsize == 4 and h.dtype.kind in "iu" and h.flags["C_CONTIGUOUS"]
     cb = _IqCodebook()
-    _check(_lib.iq_fit_codebook(h.ctypes.data, h.size, float(rng_half), 1 if symmetric else 0, {"fp16": 0, "int8": 1}[grid],
+    _check(_lib.iq_fit_codebook(h.ctypes.data, h.size, float(rng_half), bits, 1 if symmetric else 0, {"fp16": 0, "int8": 1}[grid],
                                 ctypes.byref(cb)), "iq_fit_codebook")
-    return Codebook(tuple(cb.levels), tuple(cb.thresholds))
+    return _from_c(cb)
 
 
 def iq_suggest_splits(shape: Shape, max_seq_len: int) -> int:
@@ -352,7 +405,7 @@ def iq_selftest_bounded_wait(status, polls: int, stream=None) -> None:
 # ------------------------------------------------------------------ small conveniences (allocation only)
 def new_cache(shape: Shape, device="cuda", scales_dtype=torch.float32) -> Cache:
     """scales_dtype: torch.float32, or torch.float16 for binary16 scale arrays."""
-    P = iq_row_bytes(shape.head_dim)
+    P = iq_row_bytes(shape.head_dim, shape.bits)
     n = (shape.batch, shape.n_kv_heads, shape.t_cap)
     return Cache(torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=scales_dtype, device=device),
                  torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=scales_dtype, device=device))
@@ -364,7 +417,7 @@ def new_paged_cache(shape: Shape, num_pages: int, page_rows: int, block_table: t
     (int32 device tensor [batch][t_cap / page_rows]) that maps the sequences' rows onto it."""
     assert page_rows % 128 == 0 and shape.t_cap % page_rows == 0
     assert tuple(block_table.shape) == (shape.batch, shape.t_cap // page_rows)
-    P = iq_row_bytes(shape.head_dim)
+    P = iq_row_bytes(shape.head_dim, shape.bits)
     n = (num_pages, shape.n_kv_heads, page_rows)
     return Cache(torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=scales_dtype, device=device),
                  torch.zeros(n + (P,), dtype=torch.uint8, device=device), torch.zeros(n, dtype=scales_dtype, device=device),

@@ -8,9 +8,11 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libisoquant.so")
-SOURCES = ["iq_api.cu", "iq_quantize.cu", "iq_decode.cu", "iq_combine.cu", "iq_static.cu", "iq_reconstruct.cu"]
-HEADERS = ["iq_common.cuh", "iq_decode_common.cuh", "iq_quantize_common.cuh", "iq_kernels.h", os.path.join("..", "..", "include", "isoquant.h")]
-NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+SOURCES = ["iq_api.cu", "iq_quantize.cu", "iq_decode.cu", "iq_decode_b2.cu", "iq_decode_b3.cu", "iq_decode_b4.cu", "iq_combine.cu",
+           "iq_static.cu", "iq_reconstruct.cu"]
+HEADERS = ["iq_common.cuh", "iq_decode_common.cuh", "iq_decode_kernel.cuh", "iq_quantize_common.cuh", "iq_append_row.cuh", "iq_format.cuh",
+           "iq_kernels.h", os.path.join("..", "..", "include", "isoquant.h")]
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-t", "0",
               "-Xcompiler", "-fPIC", "-shared"]
 
 

@@ -14,7 +14,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 int check_shape(const iq_shape* s) {
   if (!s) return IQ_ERR_NULL;
   if (s->head_dim != 128 && s->head_dim != 256) return IQ_ERR_SHAPE;
-  if (s->bits != 3) return IQ_ERR_SHAPE;
+  if (s->bits < 2 || s->bits > 4) return IQ_ERR_SHAPE;
   if (s->batch < 0 || s->batch > 65535) return IQ_ERR_SHAPE;
   if (s->n_kv_heads <= 0 || s->n_q_heads <= 0 || s->n_q_heads % s->n_kv_heads != 0) return IQ_ERR_SHAPE;
   if (s->t_cap <= 0 || (s->t_cap & 127) != 0) return IQ_ERR_SHAPE;
@@ -25,34 +25,49 @@ int check_shape(const iq_shape* s) {
 
 bool fp16_exact(float x) { return std::isfinite(x) && __half2float(__float2half_rn(x)) == x; }
 
-int check_codebook(const iq_codebook* cb, bool need_fp16_levels) {
+// The two sides of a codebook: K rows, V rows (the same unless separate_v).
+const float* side_levels(const iq_codebook* cb, int v) { return (v && cb->separate_v) ? cb->v_levels : cb->levels; }
+const float* side_thresholds(const iq_codebook* cb, int v) { return (v && cb->separate_v) ? cb->v_thresholds : cb->thresholds; }
+
+int check_codebook(const iq_codebook* cb, int bits, bool need_fp16_levels) {
   if (!cb) return IQ_ERR_NULL;
-  for (int i = 0; i < 8; i++) {
-    if (!std::isfinite(cb->levels[i])) return IQ_ERR_CODEBOOK;
-    if (i && !(cb->levels[i] > cb->levels[i - 1])) return IQ_ERR_CODEBOOK;
-    if (need_fp16_levels && !fp16_exact(cb->levels[i])) return IQ_ERR_CODEBOOK;
-  }
-  for (int i = 0; i < 7; i++) {
-    if (!std::isfinite(cb->thresholds[i])) return IQ_ERR_CODEBOOK;
-    if (i && !(cb->thresholds[i] > cb->thresholds[i - 1])) return IQ_ERR_CODEBOOK;
+  if (cb->bits != bits || bits < 2 || bits > 4) return IQ_ERR_CODEBOOK;
+  const int n = 1 << bits;
+  for (int v = 0; v < (cb->separate_v ? 2 : 1); v++) {
+    const float* lv = side_levels(cb, v);
+    const float* th = side_thresholds(cb, v);
+    for (int i = 0; i < n; i++) {
+      if (!std::isfinite(lv[i])) return IQ_ERR_CODEBOOK;
+      if (i && !(lv[i] > lv[i - 1])) return IQ_ERR_CODEBOOK;
+      if (need_fp16_levels && !fp16_exact(lv[i])) return IQ_ERR_CODEBOOK;
+    }
+    for (int i = 0; i < n - 1; i++) {
+      if (!std::isfinite(th[i])) return IQ_ERR_CODEBOOK;
+      if (i && !(th[i] > th[i - 1])) return IQ_ERR_CODEBOOK;
+    }
   }
   return IQ_OK;
 }
 
 // Levels on an 8-bit grid: level_j = n_j * delta with integer |n_j| <= 127 and delta = max|level| / 127 (to fp32
-// rounding). Fills n[8] and delta.
-bool int8_grid(const iq_codebook* cb, int (&n)[8], float& delta) {
+// rounding). Fills n[] and delta for one side of the codebook.
+bool int8_grid_side(const float* lv, int n_levels, int (&n)[16], float& delta) {
   float mx = 0.f;
-  for (int i = 0; i < 8; i++) mx = std::fmax(mx, std::fabs(cb->levels[i]));
+  for (int i = 0; i < n_levels; i++) mx = std::fmax(mx, std::fabs(lv[i]));
   if (!(mx > 0.f)) return false;
   delta = mx / 127.0f;
-  for (int i = 0; i < 8; i++) {
-    const double r = (double)cb->levels[i] / (double)delta;
+  for (int i = 0; i < n_levels; i++) {
+    const double r = (double)lv[i] / (double)delta;
     const double ri = std::nearbyint(r);
     if (std::fabs(r - ri) > 1e-4 || std::fabs(ri) > 127.0) return false;
     n[i] = (int)ri;
   }
   return true;
+}
+// Both sides on 8-bit grids (each its own): the integer decode path.
+bool int8_grid(const iq_codebook* cb, int (&nk)[16], float& delta_k, int (&nv)[16], float& delta_v) {
+  const int n = 1 << cb->bits;
+  return int8_grid_side(side_levels(cb, 0), n, nk, delta_k) && int8_grid_side(side_levels(cb, 1), n, nv, delta_v);
 }
 
 int check_cache(const iq_cache* c, const iq_shape* shape) {
@@ -98,17 +113,17 @@ struct SphereMarginal {
   }
 };
 
-void lloyd_max_sphere(int d, double (&lv)[8]) {
+void lloyd_max_sphere(int d, int n, double (&lv)[16]) {
   SphereMarginal f{(double)d};
   const double lim = std::sqrt((double)d);
-  for (int i = 0; i < 8; i++) lv[i] = -2.1 + 0.6 * i;
-  for (int iter = 0; iter < 5000; iter++) {
-    double edge[9];
+  for (int i = 0; i < n; i++) lv[i] = -2.4 + 4.8 * (i + 0.5) / n;
+  for (int iter = 0; iter < 20000; iter++) {
+    double edge[17];
     edge[0] = -lim;
-    edge[8] = lim;
-    for (int i = 1; i < 8; i++) edge[i] = 0.5 * (lv[i - 1] + lv[i]);
+    edge[n] = lim;
+    for (int i = 1; i < n; i++) edge[i] = 0.5 * (lv[i - 1] + lv[i]);
     double delta = 0;
-    for (int i = 0; i < 8; i++) {
+    for (int i = 0; i < n; i++) {
       double mass, mom;
       f.cell(edge[i], edge[i + 1], mass, mom);
       const double c = mom / mass;
@@ -121,7 +136,7 @@ void lloyd_max_sphere(int d, double (&lv)[8]) {
 
 // Lloyd's iteration on a histogram with uniform bins on [-range, range), read as a piecewise-constant density: a bin
 // cut by a threshold contributes to both cells in proportion. mass0 / mom0: mass and first moment below bin edge i.
-void lloyd_max_histogram(const std::vector<double>& c, double range, bool symmetric, double (&lv)[8]) {
+void lloyd_max_histogram(const std::vector<double>& c, double range, bool symmetric, int n, double (&lv)[16]) {
   const int bins = (int)c.size();
   const double w = 2.0 * range / bins;
   std::vector<double> mass0(bins + 1, 0.0), mom0(bins + 1, 0.0);
@@ -139,34 +154,34 @@ void lloyd_max_histogram(const std::vector<double>& c, double range, bool symmet
     mom = mom0[i] + dens * 0.5 * (t * t - lo * lo);
   };
   const double total = mass0[bins];
-  {  // start: the quantiles (k + 1/2) / 8
+  {  // start: the quantiles (k + 1/2) / n
     int i = 0;
-    for (int k = 0; k < 8; k++) {
-      const double target = total * (k + 0.5) / 8.0;
+    for (int k = 0; k < n; k++) {
+      const double target = total * (k + 0.5) / n;
       while (i < bins - 1 && mass0[i + 1] < target) i++;
       const double frac = c[i] > 0.0 ? (target - mass0[i]) / c[i] : 0.5;
       lv[k] = (i + frac) * w - range;
     }
   }
-  for (int iter = 0; iter < 5000; iter++) {
-    double cut[9], m[9], f[9];
+  for (int iter = 0; iter < 20000; iter++) {
+    double cut[17], m[17], f[17];
     cut[0] = -range;
-    cut[8] = range;
-    for (int i = 1; i < 8; i++) cut[i] = 0.5 * (lv[i - 1] + lv[i]);
-    for (int i = 0; i < 9; i++) below(cut[i], m[i], f[i]);
-    double nl[8];
-    for (int i = 0; i < 8; i++) {
+    cut[n] = range;
+    for (int i = 1; i < n; i++) cut[i] = 0.5 * (lv[i - 1] + lv[i]);
+    for (int i = 0; i <= n; i++) below(cut[i], m[i], f[i]);
+    double nl[16];
+    for (int i = 0; i < n; i++) {
       const double mass = m[i + 1] - m[i];
       nl[i] = mass > 0.0 ? (f[i + 1] - f[i]) / mass : lv[i];
     }
     if (symmetric)
-      for (int i = 0; i < 4; i++) {
-        const double a = 0.5 * (nl[7 - i] - nl[i]);
-        nl[7 - i] = a;
+      for (int i = 0; i < n / 2; i++) {
+        const double a = 0.5 * (nl[n - 1 - i] - nl[i]);
+        nl[n - 1 - i] = a;
         nl[i] = -a;
       }
     double delta = 0.0;
-    for (int i = 0; i < 8; i++) {
+    for (int i = 0; i < n; i++) {
       delta = std::fmax(delta, std::fabs(nl[i] - lv[i]));
       lv[i] = nl[i];
     }
@@ -176,16 +191,19 @@ void lloyd_max_histogram(const std::vector<double>& c, double range, bool symmet
 
 // Levels (fp64, ascending) -> the codebook handed to the kernels: levels exactly representable in binary16 (grid = 0)
 // or on an 8-bit grid (grid = 1: level = n * delta, |n| <= 127, delta = max |level| / 127), thresholds = midpoints.
-void finish_codebook(const double (&lv)[8], int grid, iq_codebook* out) {
+void finish_codebook(const double (&lv)[16], int bits, int grid, iq_codebook* out) {
+  const int n = 1 << bits;
+  std::memset(out, 0, sizeof(*out));
+  out->bits = bits;
   if (grid == 1) {
     double amax = 0.0;
-    for (int i = 0; i < 8; i++) amax = std::fmax(amax, std::fabs(lv[i]));
+    for (int i = 0; i < n; i++) amax = std::fmax(amax, std::fabs(lv[i]));
     const float delta = (float)(amax / 127.0);
-    for (int i = 0; i < 8; i++) out->levels[i] = delta > 0.f ? (float)std::nearbyint(lv[i] / (double)delta) * delta : 0.f;
+    for (int i = 0; i < n; i++) out->levels[i] = delta > 0.f ? (float)std::nearbyint(lv[i] / (double)delta) * delta : 0.f;
   } else {
-    for (int i = 0; i < 8; i++) out->levels[i] = __half2float(__float2half_rn((float)lv[i]));
+    for (int i = 0; i < n; i++) out->levels[i] = __half2float(__float2half_rn((float)lv[i]));
   }
-  for (int i = 0; i < 7; i++) out->thresholds[i] = (float)(0.5 * ((double)out->levels[i] + (double)out->levels[i + 1]));
+  for (int i = 0; i < n - 1; i++) out->thresholds[i] = (float)(0.5 * ((double)out->levels[i] + (double)out->levels[i + 1]));
 }
 
 // ---- fitting the SO(4) blocks (host, fp64) ---------------------------------------------------------------------
@@ -241,7 +259,7 @@ double block_distortion(const float* z4, size_t stride, int n, const double (&M)
     for (int r = 0; r < 4; r++) {
       const double u = M[r][0] * z[0] + M[r][1] * z[1] + M[r][2] * z[2] + M[r][3] * z[3];
       int code = 0;
-      for (int j = 0; j < 7; j++) code += u > (double)cb.thresholds[j];
+      for (int j = 0; j < (1 << cb.bits) - 1; j++) code += u > (double)cb.thresholds[j];
       const double e = u - (double)cb.levels[code];
       total += e * e;
     }
@@ -292,53 +310,54 @@ const char* iq_strerror(int code) {
   switch (code) {
     case IQ_OK: return "ok";
     case IQ_ERR_NULL: return "a required pointer is NULL";
-    case IQ_ERR_SHAPE: return "unsupported shape (head_dim 128/256, bits 3, n_q_heads % n_kv_heads == 0, t_cap % 128 == 0, strides % 8 == 0)";
+    case IQ_ERR_SHAPE: return "unsupported shape (head_dim 128/256, bits 2/3/4, n_q_heads % n_kv_heads == 0, t_cap % 128 == 0, strides % 8 == 0)";
     case IQ_ERR_ALIGN: return "pointer or stride not 16-byte aligned";
-    case IQ_ERR_CODEBOOK: return "codebook not ascending, or (decode) its levels are neither on an 8-bit grid nor all exact binary16 values";
+    case IQ_ERR_CODEBOOK: return "codebook bits differ from the shape's, codebook not ascending, or (decode) its levels are neither on an 8-bit grid nor all exact binary16 values";
     case IQ_ERR_CUDA: return "CUDA runtime error at launch";
     case IQ_ERR_LIMIT: return "size exceeds the documented maximum of this entry point";
     default: return "unknown error code";
   }
 }
 
-size_t iq_row_bytes(int32_t head_dim) { return (head_dim == 128 || head_dim == 256) ? (size_t)(3 * head_dim / 8) : 0; }
+size_t iq_row_bytes_bits(int32_t head_dim, int32_t bits) {
+  return ((head_dim == 128 || head_dim == 256) && bits >= 2 && bits <= 4) ? (size_t)(bits * head_dim / 8) : 0;
+}
+size_t iq_row_bytes(int32_t head_dim) { return iq_row_bytes_bits(head_dim, 3); }
 
 size_t iq_rotation_floats(int32_t head_dim, int32_t n_kv_heads) {
   if ((head_dim != 128 && head_dim != 256) || n_kv_heads <= 0) return 0;
   return (size_t)n_kv_heads * (size_t)(head_dim / 4) * 8;
 }
 
-int iq_default_codebook(int32_t head_dim, iq_codebook* out_host) {
+int iq_lloyd_max_codebook(int32_t head_dim, int32_t bits, int32_t grid, iq_codebook* out_host) {
   if (!out_host) return IQ_ERR_NULL;
-  if (head_dim != 128 && head_dim != 256) return IQ_ERR_SHAPE;
-  double lv[8];
-  lloyd_max_sphere(head_dim, lv);
-  for (int i = 0; i < 4; i++) {  // enforce exact symmetry, then round to binary16
-    const double a = 0.5 * (lv[7 - i] - lv[i]);
-    const float r = __half2float(__float2half_rn((float)a));
-    out_host->levels[7 - i] = r;
+  if ((head_dim != 128 && head_dim != 256) || bits < 2 || bits > 4 || (grid != 0 && grid != 1)) return IQ_ERR_SHAPE;
+  const int n = 1 << bits;
+  double lv[16];
+  lloyd_max_sphere(head_dim, n, lv);
+  std::memset(out_host, 0, sizeof(*out_host));
+  out_host->bits = bits;
+  double a[8];
+  for (int i = 0; i < n / 2; i++) a[i] = 0.5 * (lv[n - 1 - i] - lv[i]);  // exact symmetry; a[0] is the largest magnitude
+  const float delta = (float)(a[0] / 127.0);
+  for (int i = 0; i < n / 2; i++) {  // rounded to binary16, or snapped to the 8-bit grid
+    const float r = grid ? (float)std::nearbyint(a[i] / (double)delta) * delta : __half2float(__float2half_rn((float)a[i]));
+    out_host->levels[n - 1 - i] = r;
     out_host->levels[i] = -r;
   }
-  for (int i = 0; i < 7; i++)
+  for (int i = 0; i < n - 1; i++)
     out_host->thresholds[i] = (float)(0.5 * ((double)out_host->levels[i] + (double)out_host->levels[i + 1]));
   return IQ_OK;
 }
+int iq_default_codebook(int32_t head_dim, iq_codebook* out_host) { return iq_lloyd_max_codebook(head_dim, 3, 0, out_host); }
+int iq_int8_codebook(int32_t head_dim, iq_codebook* out_host) { return iq_lloyd_max_codebook(head_dim, 3, 1, out_host); }
 
-int iq_int8_codebook(int32_t head_dim, iq_codebook* out_host) {
-  if (!out_host) return IQ_ERR_NULL;
-  if (head_dim != 128 && head_dim != 256) return IQ_ERR_SHAPE;
-  double lv[8];
-  lloyd_max_sphere(head_dim, lv);
-  double a[4];
-  for (int i = 0; i < 4; i++) a[i] = 0.5 * (lv[7 - i] - lv[i]);  // exact symmetry; a[0] is the largest magnitude
-  const float delta = (float)(a[0] / 127.0);
-  for (int i = 0; i < 4; i++) {
-    const float r = (float)std::nearbyint(a[i] / (double)delta) * delta;
-    out_host->levels[7 - i] = r;
-    out_host->levels[i] = -r;
-  }
-  for (int i = 0; i < 7; i++)
-    out_host->thresholds[i] = (float)(0.5 * ((double)out_host->levels[i] + (double)out_host->levels[i + 1]));
+int iq_codebook_set_v(iq_codebook* cb, const iq_codebook* v_side) {
+  if (!cb || !v_side) return IQ_ERR_NULL;
+  if (cb->bits != v_side->bits || cb->bits < 2 || cb->bits > 4) return IQ_ERR_CODEBOOK;
+  cb->separate_v = 1;
+  std::memcpy(cb->v_levels, v_side->levels, sizeof(cb->v_levels));
+  std::memcpy(cb->v_thresholds, v_side->thresholds, sizeof(cb->v_thresholds));
   return IQ_OK;
 }
 
@@ -368,7 +387,7 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
   int rc = check_shape(shape);
   if (rc) return rc;
   if (!rot_dev || !append_pos_dev) return IQ_ERR_NULL;
-  if ((rc = check_codebook(codebook, false))) return rc;
+  if ((rc = check_codebook(codebook, shape->bits, false))) return rc;
   if ((rc = check_cache(cache, shape))) return rc;
   if (n_new_max < 0) return IQ_ERR_SHAPE;
   if (n_new_max == 0 || shape->batch == 0) return IQ_OK;
@@ -387,7 +406,9 @@ int iq_quantize_append(const iq_shape* shape, const float* rot_dev, const iq_cod
   p.n_new = n_new_dev;
   p.n_new_max = n_new_max;
   p.rot = rot_dev;
-  std::memcpy(p.thresholds, codebook->thresholds, sizeof(p.thresholds));
+  p.bits = shape->bits;
+  std::memcpy(p.thresholds_k, side_thresholds(codebook, 0), sizeof(p.thresholds_k));
+  std::memcpy(p.thresholds_v, side_thresholds(codebook, 1), sizeof(p.thresholds_v));
   p.k_codes = cache->k_codes;
   p.k_scales = cache->k_scales;
   p.v_codes = cache->v_codes;
@@ -408,11 +429,11 @@ static int decode_params(const iq_shape* shape, const float* rot_dev, const iq_c
   int rc = check_shape(shape);
   if (rc) return rc;
   if (!rot_dev || !q || !seq_lens_dev || !part_acc || !part_ml) return IQ_ERR_NULL;
-  if ((rc = check_codebook(codebook, false))) return rc;
-  int n8[8];
-  float delta = 0.f;
-  const bool grid8 = int8_grid(codebook, n8, delta);  // integer tensor-core path; otherwise the levels must be exact fp16 values
-  if (!grid8 && (rc = check_codebook(codebook, true))) return rc;
+  if ((rc = check_codebook(codebook, shape->bits, false))) return rc;
+  int n8[16], n8v[16];
+  float delta = 0.f, delta_v = 0.f;
+  const bool grid8 = int8_grid(codebook, n8, delta, n8v, delta_v);  // integer tensor-core path; otherwise the levels must be exact fp16 values
+  if (!grid8 && (rc = check_codebook(codebook, shape->bits, true))) return rc;
   if ((rc = check_cache(cache, shape))) return rc;
   if (num_splits < 1 || num_splits > 65535) return IQ_ERR_SHAPE;
   {  // the kernel counts (sequence, KV head group, slot) units and 128-row blocks in 31 bits
@@ -442,23 +463,29 @@ static int decode_params(const iq_shape* shape, const float* rot_dev, const iq_c
   p.scale_f16 = cache->scales_fp16 ? 1 : 0;
   p.splits = num_splits;
   p.sm_scale = shape->sm_scale > 0.f ? shape->sm_scale : 1.0f / std::sqrt((float)shape->head_dim);
-  p.lut_lo[0] = p.lut_lo[1] = p.lut_hi[0] = p.lut_hi[1] = 0u;
-  for (int i = 0; i < 8; i++) {
-    const __half hv = __float2half_rn(codebook->levels[i]);
-    uint16_t bits;
-    std::memcpy(&bits, &hv, 2);
-    p.lut_lo[i >> 2] |= (uint32_t)(bits & 0xFFu) << (8 * (i & 3));
-    p.lut_hi[i >> 2] |= (uint32_t)(bits >> 8) << (8 * (i & 3));
+  p.bits = shape->bits;
+  const int n_levels = 1 << shape->bits;
+  for (int i = 0; i < 4; i++) p.lut_lo[i] = p.lut_hi[i] = p.lut_v_lo[i] = p.lut_v_hi[i] = p.lut8[i] = p.lut8_v[i] = 0u;
+  for (int v = 0; v < 2; v++) {
+    const float* lv = side_levels(codebook, v);
+    for (int i = 0; i < n_levels; i++) {
+      const __half hv = __float2half_rn(lv[i]);
+      uint16_t bits;
+      std::memcpy(&bits, &hv, 2);
+      (v ? p.lut_v_lo : p.lut_lo)[i >> 2] |= (uint32_t)(bits & 0xFFu) << (8 * (i & 3));
+      (v ? p.lut_v_hi : p.lut_hi)[i >> 2] |= (uint32_t)(bits >> 8) << (8 * (i & 3));
+      if (grid8) (v ? p.lut8_v : p.lut8)[i >> 2] |= (uint32_t)(uint8_t)(int8_t)(v ? n8v : n8)[i] << (8 * (i & 3));
+    }
   }
   p.use_i8 = grid8 ? 1 : 0;
   p.delta = delta;
-  p.lut8[0] = p.lut8[1] = 0u;
-  if (grid8)
-    for (int i = 0; i < 8; i++) p.lut8[i >> 2] |= (uint32_t)(uint8_t)(int8_t)n8[i] << (8 * (i & 3));
+  p.delta_v = delta_v;
   p.k_new = p.v_new = nullptr;
   p.new_acc = p.new_ml = nullptr;
-  std::memcpy(p.thresholds, codebook->thresholds, sizeof(p.thresholds));
-  std::memcpy(p.levels, codebook->levels, sizeof(p.levels));
+  std::memcpy(p.thresholds_k, side_thresholds(codebook, 0), sizeof(p.thresholds_k));
+  std::memcpy(p.thresholds_v, side_thresholds(codebook, 1), sizeof(p.thresholds_v));
+  std::memcpy(p.levels_k, side_levels(codebook, 0), sizeof(p.levels_k));
+  std::memcpy(p.levels_v, side_levels(codebook, 1), sizeof(p.levels_v));
   return IQ_OK;
 }
 
@@ -511,6 +538,7 @@ int iq_decode_step_fused(const iq_shape* shape, const float* rot_dev, const iq_c
   if (!aligned16(workspace_dev) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new)) return IQ_ERR_ALIGN;
   int rc = check_shape(shape);
   if (rc) return rc;
+  if (shape->bits != 3) return IQ_ERR_SHAPE;  // the append inside the decode launch is built for the 3-bit layout
   if (num_splits < 1 || num_splits > 65535) return IQ_ERR_SHAPE;
   const StepWorkspace w = step_workspace(shape, num_splits);
   uint8_t* ws = static_cast<uint8_t*>(workspace_dev);
@@ -587,7 +615,7 @@ int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_co
   if (rc) return rc;
   if (!rot_dev || !seq_lens_dev || !k_out || !v_out) return IQ_ERR_NULL;
   if (out_rows < 0) return IQ_ERR_SHAPE;
-  if ((rc = check_codebook(codebook, false))) return rc;
+  if ((rc = check_codebook(codebook, shape->bits, false))) return rc;
   if ((rc = check_cache(cache, shape))) return rc;
   if (!aligned16(k_out) || !aligned16(v_out) || !aligned16(rot_dev)) return IQ_ERR_ALIGN;
   if (stride_b < 0 || stride_t < 0 || stride_h < 0) return IQ_ERR_SHAPE;
@@ -612,7 +640,9 @@ int iq_reconstruct_rows(const iq_shape* shape, const float* rot_dev, const iq_co
   p.scale_f16 = cache->scales_fp16 ? 1 : 0;
   p.status = nullptr;
   p.out_rows = out_rows;
-  std::memcpy(p.levels, codebook->levels, sizeof(p.levels));
+  p.bits = shape->bits;
+  std::memcpy(p.levels_k, side_levels(codebook, 0), sizeof(p.levels_k));
+  std::memcpy(p.levels_v, side_levels(codebook, 1), sizeof(p.levels_v));
   const cudaError_t e = iq::launch_reconstruct_rows(p, shape->head_dim, shape->batch, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }
@@ -627,11 +657,11 @@ int iq_decode_step_host(const iq_shape* shape, const float* rot_dev, const iq_co
   if (!aligned16(inputs_dev)) return IQ_ERR_ALIGN;
   // everything the three calls below would refuse is refused here, before the copy and the append are enqueued
   if (!rot_dev || !append_pos_dev || !seq_lens_dev || !part_acc || !part_ml) return IQ_ERR_NULL;
-  if ((rc = check_codebook(codebook, false))) return rc;
+  if ((rc = check_codebook(codebook, shape->bits, false))) return rc;
   {
-    int n8[8];
-    float delta = 0.f;
-    if (!int8_grid(codebook, n8, delta) && (rc = check_codebook(codebook, true))) return rc;
+    int n8[16], n8v[16];
+    float delta = 0.f, delta_v = 0.f;
+    if (!int8_grid(codebook, n8, delta, n8v, delta_v) && (rc = check_codebook(codebook, shape->bits, true))) return rc;
   }
   if ((rc = check_cache(cache, shape))) return rc;
   if (num_splits < 1 || num_splits > 65535) return IQ_ERR_SHAPE;
@@ -684,19 +714,19 @@ int iq_rotated_histogram(const iq_shape* shape, const float* rot_dev, const void
   return e == cudaSuccess ? IQ_OK : IQ_ERR_CUDA;
 }
 
-int iq_fit_codebook(const uint32_t* hist_host, int32_t bins, float range, int32_t symmetric, int32_t grid,
+int iq_fit_codebook(const uint32_t* hist_host, int32_t bins, float range, int32_t bits, int32_t symmetric, int32_t grid,
                     iq_codebook* out_host) {
   if (!hist_host || !out_host) return IQ_ERR_NULL;
-  if (bins < 16 || bins > iq::HIST_MAX_BINS || !(range > 0.f) || (grid != 0 && grid != 1)) return IQ_ERR_SHAPE;
+  if (bins < 16 || bins > iq::HIST_MAX_BINS || !(range > 0.f) || (grid != 0 && grid != 1) || bits < 2 || bits > 4) return IQ_ERR_SHAPE;
   std::vector<double> c((size_t)bins);
   double total = 0.0;
   for (int i = 0; i < bins; i++) total += (double)hist_host[i];
   if (!(total > 0.0)) return IQ_ERR_SHAPE;
   for (int i = 0; i < bins; i++) c[i] = symmetric ? 0.5 * ((double)hist_host[i] + (double)hist_host[bins - 1 - i]) : (double)hist_host[i];
-  double lv[8];
-  lloyd_max_histogram(c, (double)range, symmetric != 0, lv);
-  finish_codebook(lv, grid, out_host);
-  for (int i = 0; i < 7; i++)
+  double lv[16];
+  lloyd_max_histogram(c, (double)range, symmetric != 0, 1 << bits, lv);
+  finish_codebook(lv, bits, grid, out_host);
+  for (int i = 0; i < (1 << bits) - 1; i++)
     if (!(out_host->levels[i] < out_host->levels[i + 1])) return IQ_ERR_CODEBOOK;  // too few distinct values in the data
   return IQ_OK;
 }
@@ -728,7 +758,7 @@ int iq_fit_rotation(const float* z_host, int32_t n_rows, int64_t row_stride, int
                     float* quats_host, double* distortion_host) {
   if (!z_host || !codebook || !quats_host) return IQ_ERR_NULL;
   if ((head_dim != 128 && head_dim != 256) || n_rows < 1 || row_stride < head_dim) return IQ_ERR_SHAPE;
-  const int rc = check_codebook(codebook, false);
+  const int rc = codebook ? check_codebook(codebook, codebook->bits, false) : IQ_ERR_NULL;  // (the K side of the codebook is fitted to)
   if (rc) return rc;
   double before = 0.0, after = 0.0;
   for (int b = 0; b < head_dim / 4; b++) {

@@ -1,24 +1,49 @@
 // One cache row appended by one warp (Algorithm 1 for a single row): shared by the few-rows append kernel and by the
 // one-launch decode step, whose auxiliary warp appends the step's new K and V rows itself.
 #pragma once
+#include "iq_format.cuh"
 #include "iq_quantize_common.cuh"
 
 namespace iq {
 
-template <int D>
+// code = #{ j : u > t_j } over NT ascending thresholds, and whether u is within `guard` of one of them.
+template <typename T, int NT>
+__device__ __forceinline__ int decide_code_n(T u, const float (&th)[NT], bool& near_boundary, T guard) {
+  if constexpr (NT == 7) {
+    return decide_code<T>(u, th, near_boundary, guard);
+  } else {
+    int code = 0;
+    T dmin = (T)1e30;
+#pragma unroll
+    for (int j = 0; j < NT; j++) {
+      code += u > (T)th[j];
+      dmin = fmin(dmin, fabs(u - (T)th[j]));
+    }
+    near_boundary = dmin <= guard;
+    return code;
+  }
+}
+
+template <int D, int BITS = 3>
 struct WarpRowQuantizer {
   static constexpr int E = D / 32;  // coordinates per lane
   static constexpr int NB = E / 4;  // SO(4) blocks per lane
+  static constexpr int NT = (1 << BITS) - 1;
   const float* qbase;
   float M[NB][4][4];
-  float th[7];
+  float th[NT];
 
   __device__ __forceinline__ void init(const float* rot_head, const float* thresholds, int lane) {
     qbase = rot_head + (size_t)lane * NB * 8;
 #pragma unroll
     for (int j = 0; j < NB; j++) so4_matrix<float>(qbase + 8 * j, M[j]);
 #pragma unroll
-    for (int i = 0; i < 7; i++) th[i] = thresholds[i];
+    for (int i = 0; i < NT; i++) th[i] = thresholds[i];
+  }
+
+  __device__ __forceinline__ void set_thresholds(const float* thresholds) {
+#pragma unroll
+    for (int i = 0; i < NT; i++) th[i] = thresholds[i];
   }
 
   // Algorithm 1, steps 1-3 for one row: returns the fp32 scale, fills code[E]. `src` points at this lane's E values.
@@ -52,7 +77,7 @@ struct WarpRowQuantizer {
 #pragma unroll
     for (int e = 0; e < E; e++) {
       bool nb;
-      code[e] = decide_code<float>(v[e] * inv_s, th, nb, GUARD_BAND);
+      code[e] = decide_code_n<float, NT>(v[e] * inv_s, th, nb, GUARD_BAND);
       any_near |= nb;
     }
     if (__any_sync(FULL, any_near)) {  // re-decide the row in fp64: the +-1 sums of fp16 values are exact there
@@ -70,7 +95,7 @@ struct WarpRowQuantizer {
 #pragma unroll
         for (int r = 0; r < 4; r++) {
           bool nb;
-          code[4 * j + r] = decide_code<double>(blk[r] * inv_sd, th, nb, 0.0);
+          code[4 * j + r] = decide_code_n<double, NT>(blk[r] * inv_sd, th, nb, 0.0);
         }
       }
       if (lane == 0 && status) atomicAdd(&status[1], 1u);
@@ -90,9 +115,26 @@ struct RowSink {
 };
 
 // K row `row` (index into the cache arrays): lane l holds the codes of coordinates l E .. l E + E - 1.
-template <int D>
+template <int D, int BITS = 3>
 __device__ __forceinline__ void warp_store_k_row(const RowSink& c, size_t row, const int (&code)[D / 32], float s, int lane) {
   constexpr int E = D / 32;
+  if constexpr (BITS != 3) {
+    // the lane's E coordinates lie in one word (8 or 16 entries per word): the lanes that share a word OR their parts
+    constexpr int EPW = BITS == 4 ? 8 : 16, LPW = EPW / E;
+    uint32_t w = 0u;
+#pragma unroll
+    for (int e = 0; e < E; e++) {
+      int word, sh;
+      packed_place<BITS>(lane * E + e, word, sh);
+      w |= (uint32_t)code[e] << sh;
+    }
+#pragma unroll
+    for (int o = 1; o < LPW; o <<= 1) w |= __shfl_xor_sync(FULL, w, o);
+    uint32_t* row_words = reinterpret_cast<uint32_t*>(c.k_codes + row * (size_t)(BITS * D / 8));
+    if (lane % LPW == 0) row_words[lane * E / EPW] = w;
+    if (lane == 0) store_scale(c.k_scales, row, s, c.scale_f16, c.status);
+    return;
+  }
   constexpr int LPU = 32 / E;  // lanes per 32-coordinate packing unit
   // packed row: a packing unit is 32 coordinates = LPU lanes = 3 words
   uint32_t w[3] = {0u, 0u, 0u};
@@ -124,10 +166,21 @@ __device__ __forceinline__ void warp_store_k_row(const RowSink& c, size_t row, c
 
 // V row t of its sequence (at `row` in the cache arrays) into the token-transposed records: row t is entry r = t % 32
 // of unit u = (t % 128) / 32 of block t / 128, for every coordinate; one read-modify-write per touched word.
-template <int D>
+template <int D, int BITS = 3>
 __device__ __forceinline__ void warp_store_v_row(const RowSink& c, size_t row, long long t, const int (&code)[D / 32], float s, int lane) {
   constexpr int E = D / 32;
   const size_t blk = row / 128;  // (a page holds whole 128-row blocks: row / 128 is the block's index in the V array)
+  if constexpr (BITS != 3) {
+    int word, sh;
+    packed_place<BITS>((int)(t % 128), word, sh);
+#pragma unroll
+    for (int e = 0; e < E; e++) {
+      uint32_t* dst = reinterpret_cast<uint32_t*>(c.v_codes + (blk * D + lane * E + e) * (size_t)(16 * BITS)) + word;
+      *dst = (*dst & ~(((1u << BITS) - 1u) << sh)) | ((uint32_t)code[e] << sh);
+    }
+    if (lane == 0) store_scale(c.v_scales, row, s, c.scale_f16, c.status);
+    return;
+  }
   const int u = (int)(t % 128) / 32, r = (int)(t % 32);
 #pragma unroll
   for (int e = 0; e < E; e++) {

@@ -118,6 +118,73 @@ __device__ __forceinline__ void dequant_unit8(uint32_t w0, uint32_t w1, uint32_t
     out[2 * k + 1] = prmt(l0, l1, shr_mul<16>(sel[k]));
   }
 }
+// ---- the same for every bit width: 32 consecutive entries of a packed run (BITS words at w) -> natural order.
+// b = 2: 16 entries per word, codes in the low (entries 0..7) and high (8..15) bit pair of the nibbles: one 4-byte table.
+// b = 4: 8 entries per word; a byte permute selects among 8 bytes, so the 16 levels are two tables of 8, looked up with
+// the low three bits of the code and chosen byte by byte with a mask made from its top bit.
+__device__ __forceinline__ uint32_t byte_select(uint32_t lo, uint32_t hi, uint32_t mask) { return (hi & mask) | (lo & ~mask); }
+
+template <int BITS>
+__device__ __forceinline__ void dequant32_i8(const uint32_t* w, const uint32_t (&t)[4], uint32_t* out) {
+  if constexpr (BITS == 3) {
+    dequant_unit8(w[0], w[1], w[2], t[0], t[1], out);
+  } else if constexpr (BITS == 2) {
+#pragma unroll
+    for (int j = 0; j < 2; j++) {
+      const uint32_t a = w[j] & 0x33333333u, b = shr_mul<2>(w[j]) & 0x33333333u;
+      out[4 * j] = prmt(t[0], t[0], a);
+      out[4 * j + 1] = prmt(t[0], t[0], shr_mul<16>(a));
+      out[4 * j + 2] = prmt(t[0], t[0], b);
+      out[4 * j + 3] = prmt(t[0], t[0], shr_mul<16>(b));
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      const uint32_t s7 = w[j] & 0x77777777u, s3 = shr_mul<3>(w[j]) & 0x11111111u;
+#pragma unroll
+      for (int hh = 0; hh < 2; hh++) {
+        const uint32_t x = hh ? shr_mul<16>(s7) : s7, mx = hh ? shr_mul<16>(s3) : s3;
+        out[2 * j + hh] = byte_select(prmt(t[0], t[1], x), prmt(t[2], t[3], x), prmt(0x0000FF00u, 0u, mx));
+      }
+    }
+  }
+}
+
+// fp16 levels: out[r] = (level[code 2r], level[code 2r+1]), 16 registers for the 32 entries.
+template <int BITS>
+__device__ __forceinline__ void dequant32_f16(const uint32_t* w, const uint32_t (&lo)[4], const uint32_t (&hi)[4], uint32_t (&out)[16]) {
+  if constexpr (BITS == 3) {
+    dequant_unit(w[0], w[1], w[2], lo[0], lo[1], hi[0], hi[1], out);
+  } else {
+    uint32_t sel[4], top[4];  // four selectors of 8 entries each (b = 4: and the top bits of their codes)
+    if constexpr (BITS == 2) {
+      sel[0] = w[0] & 0x33333333u; sel[1] = shr_mul<2>(w[0]) & 0x33333333u;
+      sel[2] = w[1] & 0x33333333u; sel[3] = shr_mul<2>(w[1]) & 0x33333333u;
+      top[0] = top[1] = top[2] = top[3] = 0u;
+    } else {
+#pragma unroll
+      for (int k = 0; k < 4; k++) { sel[k] = w[k] & 0x77777777u; top[k] = shr_mul<3>(w[k]) & 0x11111111u; }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; k++)
+#pragma unroll
+      for (int hh = 0; hh < 2; hh++) {
+        const uint32_t x = hh ? shr_mul<16>(sel[k]) : sel[k];
+        uint32_t l, h;
+        if constexpr (BITS == 2) {
+          l = prmt(lo[0], lo[0], x);
+          h = prmt(hi[0], hi[0], x);
+        } else {
+          const uint32_t m = prmt(0x0000FF00u, 0u, hh ? shr_mul<16>(top[k]) : top[k]);
+          l = byte_select(prmt(lo[0], lo[1], x), prmt(lo[2], lo[3], x), m);
+          h = byte_select(prmt(hi[0], hi[1], x), prmt(hi[2], hi[3], x), m);
+        }
+        out[4 * k + 2 * hh] = prmt(l, h, 0x5140u);
+        out[4 * k + 2 * hh + 1] = prmt(l, h, 0x7362u);
+      }
+  }
+}
+
 // int32 -> float for |x| < 2^22, on the integer and FMA pipes (the conversion instruction runs at a quarter of their rate).
 __device__ __forceinline__ float i2f_small(uint32_t x) { return __uint_as_float(x + 0x4B400000u) - 12582912.0f; }
 

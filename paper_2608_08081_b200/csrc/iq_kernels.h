@@ -26,7 +26,9 @@ struct QuantizeParams {
   const int32_t* n_new;
   int n_new_max;
   const float* rot;
-  float thresholds[7];
+  int bits;                 // 2, 3 or 4
+  float thresholds_k[15];   // the first 2^bits - 1 are read
+  float thresholds_v[15];
   uint8_t* k_codes;
   float* k_scales;
   uint8_t* v_codes;
@@ -85,10 +87,12 @@ struct DecodeParams {
   PageMap pm;
   int scale_f16;
   float sm_scale;
-  uint32_t lut_lo[2], lut_hi[2];  // low / high bytes of the 8 fp16 levels, 4 per register
-  // integer path (levels on an 8-bit grid): level_j = lut8 byte j (int8) * delta
-  uint32_t lut8[2];
-  float delta;
+  int bits;  // 2, 3 or 4
+  // fp16 path: low / high bytes of the fp16 levels of the K and V codebooks, 4 per register (2^bits / 4 registers used)
+  uint32_t lut_lo[4], lut_hi[4], lut_v_lo[4], lut_v_hi[4];
+  // integer path (levels on an 8-bit grid): level_j = lut8 byte j (int8) * delta, per side
+  uint32_t lut8[4], lut8_v[4];
+  float delta, delta_v;
   int use_i8;
   // Decode with append (k_new != nullptr; otherwise none of the following is read): the step's new K and V rows
   // [batch][n_kv_heads][head_dim] are quantised and appended at row seq_lens[b] by one warp per (sequence, KV head),
@@ -98,8 +102,8 @@ struct DecodeParams {
   const __half* v_new;
   float* new_acc;
   float* new_ml;
-  float thresholds[7];
-  float levels[8];
+  float thresholds_k[15], thresholds_v[15];
+  float levels_k[16], levels_v[16];
 };
 cudaError_t launch_decode_attention(const DecodeParams& p, int head_dim, cudaStream_t stream);
 int decode_ctas_per_sm(int head_dim);
@@ -143,7 +147,8 @@ struct ReconstructParams {
   PageMap pm;
   int scale_f16;
   uint32_t* status;
-  float levels[8];
+  int bits;
+  float levels_k[16], levels_v[16];
 };
 cudaError_t launch_reconstruct_rows(const ReconstructParams& p, int head_dim, int batch, cudaStream_t stream);
 

@@ -241,7 +241,7 @@ __global__ void __launch_bounds__(QA_WARPS * 32, 5) quantize_append_k_kernel(con
   const int pos0 = p.append_pos[b];
 
   RQ rq;
-  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane, m_s);
+  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds_k, lane, m_s);
   const int li = lane % LPR, sub = lane / LPR;  // lane within the row, row within the warp
   const __half* src_base = p.k_new + (size_t)b * p.stride_b + (size_t)h * p.stride_h + li * 16;
 
@@ -333,7 +333,7 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
   RQ::fill_matrices(p.rot + (size_t)h * (D / 4) * 8, m_s, tid, 128);
   __syncthreads();
   RQ rq;
-  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane, m_s);
+  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds_v, lane, m_s);
   const int li = lane % LPR, sub = lane / LPR;
   const __half* src_base = p.v_new + (size_t)b * p.stride_b + (size_t)h * p.stride_h + li * 16;
   const int n_rows = (int)(t_hi - t_lo);
@@ -435,27 +435,33 @@ __global__ void __launch_bounds__(128, 5) quantize_append_v_kernel(const __grid_
 // blocks), five shuffle stages of the butterfly -- a short instruction stream and no shared memory. The V row goes
 // straight into its transposed records with one read-modify-write per touched word.
 // ---------------------------------------------------------------------------------------------------------
-template <int D>
+template <int D, int BITS>
 __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_constant__ QuantizeParams p) {
   constexpr int E = D / 32;
   grid_dependency_wait();
   allow_dependent_launch();
   const int lane = threadIdx.x;
-  const bool is_v = blockIdx.x != 0;
+  const bool is_v = (blockIdx.x & 1) != 0;
+  const int chunk = blockIdx.x >> 1;  // the warp takes the rows that fall into one 128-row block of the cache
   const int h = blockIdx.y, b = blockIdx.z;
   int n_new = p.n_new ? p.n_new[b] : p.n_new_max;
   n_new = min(n_new, p.n_new_max);
   if (n_new <= 0) return;
   const long long pos0 = p.append_pos[b];
+  // rows i with floor((pos0 + i) / 128) == floor(pos0 / 128) + chunk (rows at negative positions: chunk 0, they are refused below)
+  const long long blk0 = pos0 >= 0 ? pos0 / 128 : 0;
+  const long long lo = max(0ll, (blk0 + chunk) * 128 - pos0), hi = min((long long)n_new, (blk0 + chunk + 1) * 128 - pos0);
+  const int i_lo = (int)((chunk == 0) ? 0 : lo), i_hi = (int)hi;
+  if (i_lo >= i_hi) return;
   const __half* src_base = (is_v ? p.v_new : p.k_new) + (size_t)b * p.stride_b + (size_t)h * p.stride_h + lane * E;
   __half2 raw[E / 2];  // the first row is requested before the rotation blocks are set up: two latencies in one
 #pragma unroll
-  for (int k = 0; k < E / 2; k++) raw[k] = reinterpret_cast<const __half2*>(src_base)[k];
-  WarpRowQuantizer<D> rq;
+  for (int k = 0; k < E / 2; k++) raw[k] = reinterpret_cast<const __half2*>(src_base + (size_t)i_lo * p.stride_t)[k];
+  WarpRowQuantizer<D, BITS> rq;
   const RowSink sink{p.k_codes, p.k_scales, p.v_codes, p.v_scales, p.status, p.scale_f16};
-  rq.init(p.rot + (size_t)h * (D / 4) * 8, p.thresholds, lane);
-  for (int i = 0; i < n_new; i++) {
-    if (i > 0) {
+  rq.init(p.rot + (size_t)h * (D / 4) * 8, is_v ? p.thresholds_v : p.thresholds_k, lane);
+  for (int i = i_lo; i < i_hi; i++) {
+    if (i > i_lo) {
 #pragma unroll
       for (int k = 0; k < E / 2; k++) raw[k] = reinterpret_cast<const __half2*>(src_base + (size_t)i * p.stride_t)[k];
     }
@@ -474,8 +480,8 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
     }
     int code[E];
     const float s = rq.run(raw, lane, code, p.status);
-    if (!is_v) warp_store_k_row<D>(sink, row, code, s, lane);
-    else warp_store_v_row<D>(sink, row, t, code, s, lane);
+    if (!is_v) warp_store_k_row<D, BITS>(sink, row, code, s, lane);
+    else warp_store_v_row<D, BITS>(sink, row, t, code, s, lane);
   }
 }
 
@@ -581,33 +587,40 @@ cudaError_t launch_wht_coordinates(const WhtParams& p, int head_dim, int batch, 
                          : launch_after_predecessor(wht_coordinates_kernel<256>, grid, dim3(QA_WARPS * 32), 0, stream, p);
 }
 
+template <int D, int BITS>
+static cudaError_t launch_few(const QuantizeParams& p, int batch, cudaStream_t stream) {
+  // x = 2 * chunk + (0: the K rows, 1: the V rows) of (sequence, KV head); a chunk is the part of the new rows inside
+  // one 128-row block of the cache (+1: the first row may sit in the middle of a block)
+  dim3 grid(2 * ((p.n_new_max + 127) / 128 + 1), p.n_kv_heads, batch);
+  return launch_after_predecessor(quantize_append_few_kernel<D, BITS>, grid, dim3(32), 0, stream, p);
+}
+
 cudaError_t launch_quantize_append(const QuantizeParams& p, int head_dim, int batch, cudaStream_t stream) {
   if (p.n_new_max <= 0 || batch <= 0) return cudaSuccess;
+  // 2 and 4 bits: one warp per row throughout (the row-tiled kernels below are written for the 3-bit layout)
+  if (p.bits == 2) return head_dim == 128 ? launch_few<128, 2>(p, batch, stream) : launch_few<256, 2>(p, batch, stream);
+  if (p.bits == 4) return head_dim == 128 ? launch_few<128, 4>(p, batch, stream) : launch_few<256, 4>(p, batch, stream);
   const int rows_per_cta = QA_WARPS * QA_ROWS_PER_WARP;
   dim3 kgrid((p.n_new_max + rows_per_cta - 1) / rows_per_cta, p.n_kv_heads, batch);
   dim3 vgrid((p.n_new_max + 127) / 128 + 1, p.n_kv_heads, batch);  // +1: the first row may sit in the middle of a block
-  if (p.n_new_max <= QA_FEW_ROWS) {
-    dim3 grid(2, p.n_kv_heads, batch);  // x = 0: the K rows, x = 1: the V rows of (sequence, KV head)
-    return head_dim == 128 ? launch_after_predecessor(quantize_append_few_kernel<128>, grid, dim3(32), 0, stream, p)
-                           : launch_after_predecessor(quantize_append_few_kernel<256>, grid, dim3(32), 0, stream, p);
-  }
+  if (p.n_new_max <= QA_FEW_ROWS) return head_dim == 128 ? launch_few<128, 3>(p, batch, stream) : launch_few<256, 3>(p, batch, stream);
   // (the V kernel may start under the K kernel: they write different arrays)
-  const float* t = p.thresholds;
-  const bool sym = t[3] == 0.f && t[0] == -t[6] && t[1] == -t[5] && t[2] == -t[4];  // two compares per coordinate instead of three
+  auto symmetric = [](const float* t) { return t[3] == 0.f && t[0] == -t[6] && t[1] == -t[5] && t[2] == -t[4]; };  // two compares per coordinate instead of three
+  const bool sym_k = symmetric(p.thresholds_k), sym_v = symmetric(p.thresholds_v);
   const dim3 kblock(QA_WARPS * 32), vblock(128);
   cudaError_t e;
   if (head_dim == 128)
-    e = sym ? launch_after_predecessor(quantize_append_k_kernel<128, true>, kgrid, kblock, 0, stream, p)
-            : launch_after_predecessor(quantize_append_k_kernel<128, false>, kgrid, kblock, 0, stream, p);
+    e = sym_k ? launch_after_predecessor(quantize_append_k_kernel<128, true>, kgrid, kblock, 0, stream, p)
+              : launch_after_predecessor(quantize_append_k_kernel<128, false>, kgrid, kblock, 0, stream, p);
   else
-    e = sym ? launch_after_predecessor(quantize_append_k_kernel<256, true>, kgrid, kblock, 0, stream, p)
-            : launch_after_predecessor(quantize_append_k_kernel<256, false>, kgrid, kblock, 0, stream, p);
+    e = sym_k ? launch_after_predecessor(quantize_append_k_kernel<256, true>, kgrid, kblock, 0, stream, p)
+              : launch_after_predecessor(quantize_append_k_kernel<256, false>, kgrid, kblock, 0, stream, p);
   if (e != cudaSuccess) return e;
   if (head_dim == 128)
-    return sym ? launch_after_predecessor(quantize_append_v_kernel<128, true>, vgrid, vblock, 0, stream, p)
-               : launch_after_predecessor(quantize_append_v_kernel<128, false>, vgrid, vblock, 0, stream, p);
-  return sym ? launch_after_predecessor(quantize_append_v_kernel<256, true>, vgrid, vblock, 0, stream, p)
-             : launch_after_predecessor(quantize_append_v_kernel<256, false>, vgrid, vblock, 0, stream, p);
+    return sym_v ? launch_after_predecessor(quantize_append_v_kernel<128, true>, vgrid, vblock, 0, stream, p)
+                 : launch_after_predecessor(quantize_append_v_kernel<128, false>, vgrid, vblock, 0, stream, p);
+  return sym_v ? launch_after_predecessor(quantize_append_v_kernel<256, true>, vgrid, vblock, 0, stream, p)
+               : launch_after_predecessor(quantize_append_v_kernel<256, false>, vgrid, vblock, 0, stream, p);
 }
 
 }  // namespace iq

@@ -3,6 +3,7 @@
 // tensors for a standard attention kernel. This is the execution model the fused decode path replaces; it exists so that
 // the two can be measured against each other on the same packed cache.
 #include "iq_common.cuh"
+#include "iq_format.cuh"
 #include "iq_kernels.h"
 
 namespace iq {
@@ -13,20 +14,12 @@ namespace iq {
 // across the row's lanes.
 constexpr int RC_WARPS = 8;
 
-// Code of entry e of a packing unit (three little-endian words): entries 0..23 sit in the low three bits of the
-// nibbles, entries 24..31 are spread over the top bits of the nibbles (bit k of the code in word k).
-__device__ __forceinline__ uint32_t unit_code(const uint32_t* w, int e) {
-  if (e < 24) return (w[e >> 3] >> (4 * (e & 7))) & 7u;
-  const int sh = 4 * (e - 24) + 3;
-  return ((w[0] >> sh) & 1u) | (((w[1] >> sh) & 1u) << 1) | (((w[2] >> sh) & 1u) << 2);
-}
-
-template <int D>
+template <int D, int BITS>
 __global__ void __launch_bounds__(RC_WARPS * 32) reconstruct_kernel(const ReconstructParams p) {
-  constexpr int ROWB = 3 * D / 8, LPR = D / 16, RPW = 32 / LPR, TB = 128;
+  constexpr int ROWB = BITS * D / 8, VREC = 16 * BITS, LPR = D / 16, RPW = 32 / LPR, TB = 128;
   __shared__ __align__(16) uint8_t k_s[TB * ROWB];
-  __shared__ __align__(16) uint8_t v_s[D * 48];
-  __shared__ float ks_s[TB], vs_s[TB], lv_s[8];
+  __shared__ __align__(16) uint8_t v_s[D * VREC];
+  __shared__ float ks_s[TB], vs_s[TB], lv_s[16], lvv_s[16];
 
   grid_dependency_wait();
   allow_dependent_launch();
@@ -38,16 +31,16 @@ __global__ void __launch_bounds__(RC_WARPS * 32) reconstruct_kernel(const Recons
   const int n = min(TB, len - r_begin);
   const size_t row0 = cache_row(p.pm, b, g, r_begin, p.status);  // the block's first row in the cache arrays
 
-  {  // stage the block: n packed K rows, the whole V record set of the block (128 * ROWB = D * 48 bytes), the scales
+  {  // stage the block: n packed K rows, the whole V record set of the block (128 * ROWB = D * 16 b bytes), the scales
     const uint4* ksrc = reinterpret_cast<const uint4*>(p.k_codes + row0 * ROWB);
     const uint4* vsrc = reinterpret_cast<const uint4*>(p.v_codes + row0 * ROWB);
     for (int i = tid; i < n * ROWB / 16; i += RC_WARPS * 32) reinterpret_cast<uint4*>(k_s)[i] = ksrc[i];
-    for (int i = tid; i < D * 48 / 16; i += RC_WARPS * 32) reinterpret_cast<uint4*>(v_s)[i] = vsrc[i];
+    for (int i = tid; i < D * VREC / 16; i += RC_WARPS * 32) reinterpret_cast<uint4*>(v_s)[i] = vsrc[i];
     if (tid < n) {
       ks_s[tid] = load_scale(p.k_scales, row0 + tid, p.scale_f16);
       vs_s[tid] = load_scale(p.v_scales, row0 + tid, p.scale_f16);
     }
-    if (tid < 8) lv_s[tid] = p.levels[tid];
+    if (tid < 16) { lv_s[tid] = p.levels_k[tid]; lvv_s[tid] = p.levels_v[tid]; }
   }
   const int li = lane % LPR, sub = lane / LPR;  // lane within the row, row within the warp
   float M[4][4][4];
@@ -92,7 +85,11 @@ __global__ void __launch_bounds__(RC_WARPS * 32) reconstruct_kernel(const Recons
     const int rr = active ? r : 0;
     const size_t out_off = (size_t)b * p.stride_b + (size_t)(r_begin + rr) * p.stride_t + (size_t)g * p.stride_h + (size_t)li * 16;
     float x[16];
-    {  // K row rr: this lane's half of packing unit li / 2
+    if constexpr (BITS != 3) {  // K row rr: the lane's 16 entries
+      const uint32_t* w = reinterpret_cast<const uint32_t*>(k_s + rr * ROWB);
+#pragma unroll
+      for (int e = 0; e < 16; e++) x[e] = lv_s[packed_code<BITS>(w, li * 16 + e)];
+    } else {  // K row rr: this lane's half of packing unit li / 2
       const uint32_t* w = reinterpret_cast<const uint32_t*>(k_s + rr * ROWB) + 3 * (li >> 1);
       const uint32_t w0 = w[0], w1 = w[1], w2 = w[2];
       uint32_t sa, sb;  // eight codes each, one per nibble
@@ -111,22 +108,27 @@ __global__ void __launch_bounds__(RC_WARPS * 32) reconstruct_kernel(const Recons
     }
     rotate_back_and_store(x, ks_s[rr], p.k_out + out_off, active);
     {  // V row rr: one record per coordinate, the row-in-block is the entry
-      const int u = rr >> 5, e_in = rr & 31;
 #pragma unroll
       for (int e = 0; e < 16; e++) {
-        const uint32_t* w = reinterpret_cast<const uint32_t*>(v_s + (size_t)(li * 16 + e) * 48) + 3 * u;
-        x[e] = lv_s[unit_code(w, e_in)];
+        const uint32_t* w = reinterpret_cast<const uint32_t*>(v_s + (size_t)(li * 16 + e) * VREC);
+        x[e] = lvv_s[packed_code<BITS>(w, rr)];
       }
     }
     rotate_back_and_store(x, vs_s[rr], p.v_out + out_off, active);
   }
 }
 
+template <int BITS>
+static cudaError_t launch_reconstruct_bits(const ReconstructParams& p, int head_dim, dim3 grid, cudaStream_t stream) {
+  if (head_dim == 128) return launch_after_predecessor(reconstruct_kernel<128, BITS>, grid, dim3(RC_WARPS * 32), 0, stream, p);
+  return launch_after_predecessor(reconstruct_kernel<256, BITS>, grid, dim3(RC_WARPS * 32), 0, stream, p);
+}
 cudaError_t launch_reconstruct_rows(const ReconstructParams& p, int head_dim, int batch, cudaStream_t stream) {
   if (batch <= 0 || p.t_cap <= 0 || p.out_rows <= 0) return cudaSuccess;
   dim3 grid((unsigned)((min(p.t_cap, p.out_rows) + 127) / 128), (unsigned)p.n_kv_heads, (unsigned)batch);
-  if (head_dim == 128) return launch_after_predecessor(reconstruct_kernel<128>, grid, dim3(RC_WARPS * 32), 0, stream, p);
-  return launch_after_predecessor(reconstruct_kernel<256>, grid, dim3(RC_WARPS * 32), 0, stream, p);
+  if (p.bits == 2) return launch_reconstruct_bits<2>(p, head_dim, grid, stream);
+  if (p.bits == 4) return launch_reconstruct_bits<4>(p, head_dim, grid, stream);
+  return launch_reconstruct_bits<3>(p, head_dim, grid, stream);
 }
 
 }  // namespace iq

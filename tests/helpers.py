@@ -126,11 +126,11 @@ ARGMAX_TIE_RTOL = 4e-6   # a different argmax row is a tie iff its fp64 score is
 ARGMAX_TIE_ATOL = 2e-6   # ... plus this: the kernel's scores are fp32 values of 21-bit (integer path) or 22-bit (fp16 path) queries
 
 
-def check_decode(w, lv, q_np, gpu_res, cache_np, lens, sm_scale=0.0, argmax_tol=None):
+def check_decode(w, lv, q_np, gpu_res, cache_np, lens, sm_scale=0.0, argmax_tol=None, levels_v=None):
     """Outputs within tolerance of the fp64 oracle run on the same packed cache; argmax identical, except that a row
     whose fp64 score ties with the maximum within the rounding of the kernel's fp32 scores is accepted (counted, and
     at most 2 % of the heads + 1)."""
-    ref = oracle.decode_attention(w.quats, lv, q_np, cache_np, lens, w.H_kv, sm_scale)
+    ref = oracle.decode_attention(w.quats, lv, q_np, cache_np, lens, w.H_kv, sm_scale, levels_v=levels_v)
     err = np.abs(gpu_res["out"] - ref["out"])
     bound = OUT_ATOL + OUT_RTOL * np.abs(ref["out"])
     assert np.all(err <= bound), f"max err {err.max():.3e} (worst excess {np.max(err - bound):.3e})"

@@ -23,7 +23,7 @@ def test_library_exports_every_declared_symbol(iq):
     lib = ctypes.CDLL(iq.lib_path())
     for n in sorted(names):
         assert hasattr(lib, n), f"{n} declared in isoquant.h but not exported"
-    assert iq.iq_version() == 200 and iq.iq_format_version() == 2
+    assert iq.iq_version() == 300 and iq.iq_format_version() == 3
     for n in sorted(names):
         assert hasattr(iq, n) or n in ("iq_shape", "iq_codebook", "iq_cache"), f"binding lacks {n}"
 
@@ -93,7 +93,8 @@ def test_argument_validation_happens_before_any_launch(iq, monkeypatch):
     def qa(shape, rot=A, cbk=cb, k=A, v=A, sb=1024 * 128, st=128, sh=128, pos=A, nn=None, n=1, c=cache):
         return lib.iq_quantize_append(ctypes.byref(shape), rot, ctypes.byref(cbk), k, v, sb, st, sh, pos, nn, n, ctypes.byref(c), None, None)
     assert qa(B._IqShape(1, 4, 1, 64, 1024, 3, 0.0)) == -2          # head_dim
-    assert qa(B._IqShape(1, 4, 1, 128, 1024, 4, 0.0)) == -2         # bits
+    assert qa(B._IqShape(1, 4, 1, 128, 1024, 5, 0.0)) == -2         # bits
+    assert qa(B._IqShape(1, 4, 1, 128, 1024, 4, 0.0)) == -4         # bits that the codebook is not for
     assert qa(B._IqShape(1, 5, 2, 128, 1024, 3, 0.0)) == -2         # n_q % n_kv
     assert qa(B._IqShape(1, 4, 1, 128, 1022, 3, 0.0)) == -2         # t_cap % 4
     assert qa(good, rot=None) == -1
