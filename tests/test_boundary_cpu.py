@@ -66,6 +66,29 @@ def test_codebook_fitted_to_a_histogram_matches_the_oracle(iq):
                 assert np.array_equal(np.array(cb8.levels)[::-1], -np.array(cb8.levels)) and cb8.thresholds[3] == 0.0
     with pytest.raises(iq.IQError):
         iq.iq_fit_codebook(np.zeros(bins, np.uint32), R)                 # no data
+    # 4 and 16 levels (Algorithm 1's b = 2 and 4)
+    for bits in (2, 4):
+        h = np.rint(hists["skewed"] * 1e8).astype(np.uint32)
+        for symmetric in (True, False):
+            lv, _, _ = lloyd_max.fit_histogram(h, R, n_levels=1 << bits, symmetric=symmetric)
+            cb16 = iq.iq_fit_codebook(h, R, symmetric=symmetric, grid="fp16", bits=bits)
+            assert cb16.bits == bits and len(cb16.levels) == 1 << bits
+            assert np.allclose(np.array(cb16.levels, np.float64), lv.astype(np.float16).astype(np.float64), rtol=0, atol=2e-3), (bits, symmetric)
+            cb8 = iq.iq_fit_codebook(h, R, symmetric=symmetric, grid="int8", bits=bits)
+            delta = np.max(np.abs(cb8.levels)) / 127.0
+            assert np.allclose(np.array(cb8.levels) / delta, np.rint(np.array(cb8.levels) / delta), atol=1e-4)
+            assert np.allclose(cb8.levels, lv, rtol=0, atol=0.6 * delta + 2e-3)
+    # the library's Lloyd-Max codebooks for the post-rotation marginal, every width and both grids
+    for d in (128, 256):
+        for bits in (2, 3, 4):
+            for kind, make in (("int8", lloyd_max.int8_codebook), ("fp16", lloyd_max.fp16_codebook)):
+                cb = iq.iq_lloyd_max_codebook(d, bits, kind)
+                lv, th = make(d, 1 << bits)
+                assert np.allclose(cb.levels, lv, rtol=0, atol=2e-3) and np.allclose(cb.thresholds, th, rtol=0, atol=2e-3), (d, bits, kind)
+    two = iq.iq_codebook_set_v(iq.iq_lloyd_max_codebook(128, 4, "int8"), iq.iq_lloyd_max_codebook(128, 4, "fp16"))
+    assert two.v_levels == iq.iq_lloyd_max_codebook(128, 4, "fp16").levels and two.levels == iq.iq_lloyd_max_codebook(128, 4, "int8").levels
+    with pytest.raises(iq.IQError):
+        iq.iq_codebook_set_v(iq.iq_lloyd_max_codebook(128, 4, "int8"), iq.iq_lloyd_max_codebook(128, 2, "int8"))
 
 
 class _P:
@@ -163,7 +186,7 @@ def test_rotation_fit_on_the_host_matches_the_oracle(iq, codebooks):
     must give, under the oracle's distortion, what the product reports, and no block may end above its start."""
     import oracle
     import workloads
-    from oracle import so4_fit
+    from oracle import lloyd_max, so4_fit
     d = 128
     lv, th = codebooks[d]
     cb = iq.Codebook(tuple(float(x) for x in lv), tuple(float(x) for x in th))
@@ -179,6 +202,12 @@ def test_rotation_fit_on_the_host_matches_the_oracle(iq, codebooks):
     assert abs(a_lib - a_ref) < 2e-3 * a_ref
     again = sum(so4_fit.block_distortion(z[:, 4 * b:4 * b + 4].astype(np.float64), oracle.so4_block(q_lib[b]), lv, th) for b in range(d // 4)) / d
     assert abs(again - a_lib) < 1e-5 * a_lib                                   # the pairs it returns are the rotation it found
+    for bits in (2, 4):                                                        # the same with 4 and 16 levels
+        lvb, thb = lloyd_max.int8_codebook(d, 1 << bits)
+        cbb = iq.Codebook(tuple(float(x) for x in lvb), tuple(float(x) for x in thb))
+        _, b_r, a_r = so4_fit.fit_rotation(z[:256].astype(np.float64), q0, lvb, thb)
+        _, b_l, a_l = iq.iq_fit_rotation(np.ascontiguousarray(z[:256]), d, cbb, q0)
+        assert abs(b_l - b_r) < 1e-12 * b_r and a_l <= b_l and abs(a_l - a_r) < 5e-3 * a_r, (bits, b_l, b_r, a_l, a_r)
     assert np.allclose(np.linalg.norm(q_lib.reshape(-1, 2, 4), axis=-1), 1.0, atol=1e-6)
     # argument checks, no CUDA involved
     import ctypes
