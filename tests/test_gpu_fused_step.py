@@ -111,3 +111,75 @@ def test_more_sequences_than_sms(iq, torch, codebooks):
     w = workloads.tiny(760, B, 4, 2, 128, 256, lens=lens)
     print(_step(iq, torch, codebooks, w, lens, 8, steps=2)[-1])
     print(_step(iq, torch, codebooks, w, lens, 3, steps=1)[-1])
+
+
+def test_paged_cache_and_binary16_scales(iq, torch, codebooks):
+    """The step's append inside the decode launch on a pool of scrambled pages with binary16 scale arrays: the new rows
+    land in the right pages (one of them on the first row of a fresh page), the output equals the oracle's with its
+    stored norms rounded the same way, and a page that is missing from the table costs the row, not another page."""
+    d, B, H_q, H_kv, T, page_rows = 128, 3, 8, 2, 768, 128
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    lens = np.array([700, 255, 0], np.int32)
+    w = workloads.tiny(770, B, H_q, H_kv, d, T, lens)
+    n_tab = T // page_rows
+    num_pages = B * n_tab + 2
+    table = np.random.default_rng(3).permutation(num_pages)[:B * n_tab].reshape(B, n_tab).astype(np.int32)
+    shape = iq.Shape(B, H_q, H_kv, d, T)
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(w.quats), rot)
+    cache = iq.new_paged_cache(shape, num_pages, page_rows, torch.from_numpy(table).cuda(), scales_dtype=torch.float16)
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(w.k).cuda(), torch.from_numpy(w.v).cuda(),
+                          torch.zeros(B, dtype=torch.int32, device="cuda"), torch.from_numpy(lens).cuda(), T, cache, status)
+    ref = oracle.new_cache(B, H_kv, d, T)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), lens, ref)
+    S = 8
+    ws = torch.empty(iq.iq_decode_step_workspace_bytes(shape, S), dtype=torch.uint8, device="cuda")
+    out = torch.empty((B, H_q, d), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, H_q), dtype=torch.float32, device="cuda")
+    am = torch.empty((B, H_q), dtype=torch.int32, device="cuda")
+    now = lens.copy()
+    q = torch.from_numpy(w.q).cuda()
+
+    def gathered():
+        def pool(a):
+            a = a.cpu().numpy()
+            return np.stack([np.concatenate([a[table[b, j]] for j in range(n_tab)], axis=1) for b in range(B)])
+        g = dict(k_codes=pool(cache.k_codes), v_codes=pool(cache.v_codes),
+                 k_scales=pool(cache.k_scales).astype(np.float32), v_scales=pool(cache.v_scales).astype(np.float32))
+        return g
+
+    for step in range(2):                                                # sequence 1: rows 255 and 256 (a fresh page)
+        kn = np.ascontiguousarray(np.stack([w.k[b, now[b]] for b in range(B)]))
+        vn = np.ascontiguousarray(np.stack([w.v[b, now[b]] for b in range(B)]))
+        iq.iq_decode_step_fused(shape, rot, cb, q, torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), cache,
+                                torch.from_numpy(now).cuda(), S, ws, out, lse, am, status)
+        torch.cuda.synchronize()
+        assert status.cpu().numpy()[0] == 0
+        oracle.quantize_append(w.quats, th, kn[:, None], vn[:, None], now.copy(), None, ref)
+        now = now + 1
+        ref16 = {k_: v_.copy() for k_, v_ in ref.items()}
+        oracle.round_scales_fp16(ref16)
+        g = gathered()
+        assert np.array_equal(g["k_codes"][0, :, :now[0]], ref16["k_codes"][0, :, :now[0]])
+        for b in range(B):
+            n = int(now[b])
+            assert np.array_equal(g["k_codes"][b, :, :n], ref16["k_codes"][b, :, :n])
+            assert np.mean(g["k_scales"][b, :, :n] != ref16["k_scales"][b, :, :n]) <= 2e-3 + 1.0 / max(n * H_kv, 1)
+        w2 = workloads.Workload("paged", B, H_q, H_kv, d, T, w.k, w.v, w.q, w.quats, now)
+        res = dict(out=out.cpu().numpy().astype(np.float64), lse=lse.cpu().numpy().astype(np.float64), argmax=am.cpu().numpy())
+        check_decode(w2, lv, w.q, res, g, now)
+    # a page missing from the table: the new row of that sequence is skipped and counted, every page stays as it was
+    bad = table.copy(); bad[1, int(now[1]) // page_rows] = -1
+    cache_bad = iq.Cache(cache.k_codes, cache.k_scales, cache.v_codes, cache.v_scales, torch.from_numpy(bad).cuda(), page_rows)
+    if True:
+        before = [t.clone() for t in (cache.k_codes, cache.v_codes)]
+        only1 = torch.tensor([-5, int(now[1]), -5], dtype=torch.int32, device="cuda")     # the other sequences: out of range, no row either
+        status.zero_()
+        kn = torch.from_numpy(np.ascontiguousarray(w.k[:, 0])).cuda()
+        iq.iq_decode_step_fused(shape, rot, cb, q, kn, kn, cache_bad, only1, S, ws, out, lse, am, status)
+        torch.cuda.synchronize()
+        st = status.cpu().numpy()
+        assert st[0] & 4 and st[0] & 1 and st[2] == 3 * 2 * H_kv
+        assert torch.equal(cache.k_codes, before[0]) and torch.equal(cache.v_codes, before[1])
