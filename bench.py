@@ -294,6 +294,39 @@ class StepRunner:
                 self._stamp(ev[1][1])   # fires when the decode kernel has completed
             iq.iq_combine_splits(self.gshape, st["rot"], S, ws.part_acc[g], ws.part_ml[g], None, (ws.out if out is None else out)[g], ws.lse[g], None)
 
+    def decode_alone(self, n: int = 20, replays: int = 7):
+        """The decode launch by itself: a CUDA graph of n decode launches (no append, no merge, no event nodes), replayed;
+        returns the median time per launch in ms, or None without a graph. Consecutive launches overlap their set-up with
+        the tail of the one before (programmatic dependent launch), as they do behind the append kernel in a step."""
+        iq, st, ws, S, torch = self.iq, self.st, self.ws, self.S, self.torch
+        i = self.W   # lengths of the first timed step
+
+        def launches():
+            for _ in range(n):
+                for j, g in enumerate(self.groups):
+                    iq.iq_decode_attention(self.gshape, st["rot"], st["cb"], self.q_all[i][g], self.gcache[j], self.lens_tab[i + 1][g], S,
+                                           ws.part_acc[g], ws.part_ml[g], None, ws.status)
+        try:
+            launches()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                launches()
+            graph.replay()
+            torch.cuda.synchronize()
+        except Exception:
+            return None
+        ts = []
+        for _ in range(replays):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            graph.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / (n * self.n_groups))
+        del graph
+        return float(np.median(ts))
+
     def one_step(self, i, ev=None):
         self.launches(i, self.q_all[i], self.k_all[i], self.v_all[i], None if ev is None else (i % self.n_groups, ev))
 
@@ -440,6 +473,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     # the timed region: the K steps R times, until it lasts args.min_region seconds (whatever --steps is)
     per_replay, dec_ms = r.timed_region(args.min_region, barrier=barrier)
     clocks = sampler.stop() if rank == 0 else None
+    alone_ms = r.decode_alone() if not args.no_graph else None
     assert int(ws.status[0].item()) == 0 and int(st["status"][0].item()) == 0, "device status flags set"
     R = len(per_replay)
     bytes_steps = r.bytes_of_steps()
@@ -532,7 +566,11 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                      "launch_ms_cv": round(float(np.std(dec_ms) / np.mean(dec_ms)), 4), "launches_timed": len(dec_ms),
                      "timing": ("CUDA event-record nodes beside every %d-th decode launch of the replayed graph: from the completion of the kernel before it to its own completion (sibling nodes: the kernels keep their direct dependencies)" % GRAPH_EVENT_STRIDE
                                 if r.graph is not None else "CUDA events on a side stream beside every decode launch: from the completion of the kernel before it to its own completion"),
-                     "algorithmic_bytes_per_launch": int(launch_bytes)},
+                     "algorithmic_bytes_per_launch": int(launch_bytes),
+                     "launch_alone": (None if not alone_ms else {
+                         "ms": round(alone_ms, 4), "gb_per_s": round(launch_bytes / (alone_ms * 1e-3) / 1e9, 1),
+                         "frac": round(launch_bytes / (alone_ms * 1e-3) / 1e9 / peak, 4),
+                         "what": "the same decode launch in a CUDA graph of 20 decode launches and nothing else (median of 7 replays, outside the timed region): what the event nodes and the neighbouring small kernels add to the bracketed figure above is the difference"})},
         "e2e": {"value": round(aggregate_gbs(e2e_bytes_pass * e2e_passes, e2e_ms, world), 1), "unit": "GB/s",
                 "h2d_bytes_per_step": int(B * (H_q + 2 * H_kv) * d * 2), "d2h_bytes_per_step": int(B * H_q * d * 2),
                 "ms_per_step": round(e2e_ms / max(n_e2e * e2e_passes, 1), 4), "steps": n_e2e * e2e_passes,
