@@ -266,6 +266,13 @@ class StepRunner:
         else:
             self.gcache = [iq.Cache(cache.k_codes[g], cache.k_scales[g], cache.v_codes[g], cache.v_scales[g]) for g in self.groups]
         self.n_groups = len(self.groups)
+        # Small launch groups take the one-call step whose decode launch also appends (iq_decode_step_fused: two launches);
+        # a group whose decode launch is bracketed by event records takes the three separate calls, so that the records
+        # can sit between them. For larger groups the one-call step enqueues the same three launches anyway.
+        gB = 1 if self.per_seq else B
+        self.one_call = BITS == 3 and gB * self.H_kv * (1 + self.H_q // self.H_kv) <= 180
+        self.step_ws = torch.empty(max(iq.iq_decode_step_workspace_bytes(self.gshape, self.S), 16), dtype=torch.uint8, device=device) if self.one_call else None
+        self.launch_count = 0   # kernels launched by launches() since the counter was last cleared
         self.graph, self.graph_evs, self.graph_error = None, None, None
         self.side = torch.cuda.Stream(device=device)   # carries the event records that bracket decode launches
 
@@ -286,6 +293,12 @@ class StepRunner:
         ev = (group, event pair) brackets that group's decode launch."""
         iq, st, ws, S, torch = self.iq, self.st, self.ws, self.S, self.torch
         for j, g in enumerate(self.groups):
+            if self.one_call and not (ev is not None and ev[0] == j):
+                iq.iq_decode_step_fused(self.gshape, st["rot"], st["cb"], q[g], k[g][:, 0], v[g][:, 0], self.gcache[j], self.lens_tab[i][g], S,
+                                        self.step_ws, (ws.out if out is None else out)[g], ws.lse[g], None, ws.status)
+                self.launch_count += 2
+                continue
+            self.launch_count += 3
             iq.iq_quantize_append(self.gshape, st["rot"], st["cb"], k[g], v[g], self.lens_tab[i][g], None, 1, self.gcache[j], st["status"])
             if ev is not None and ev[0] == j:
                 self._stamp(ev[1][0])   # fires when the append kernel has completed
@@ -346,11 +359,13 @@ class StepRunner:
             self.graph_evs = [(torch.cuda.Event(enable_timing=True, external=True), torch.cuda.Event(enable_timing=True, external=True))
                               for _ in range((K + GRAPH_EVENT_STRIDE - 1) // GRAPH_EVENT_STRIDE)]
             self.graph = torch.cuda.CUDAGraph()
+            self.launch_count = 0
             with torch.cuda.graph(self.graph):
                 self.side.wait_stream(torch.cuda.current_stream())     # the side stream joins the capture
                 for i in range(K):
                     self.one_step(W + i, self.graph_evs[i // GRAPH_EVENT_STRIDE] if i % GRAPH_EVENT_STRIDE == 0 else None)
                 torch.cuda.current_stream().wait_stream(self.side)     # and is joined back before the capture ends
+            self.graph_launches = self.launch_count                    # kernels in one replay
             self.graph.replay()                                        # untimed: first replay of a new graph
             torch.cuda.synchronize()
         except Exception as e:  # noqa: BLE001 -- reported in the JSON line; the host-launched loop is timed instead
@@ -469,7 +484,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
         for i in range(K):
             r.one_step(W + i, eager_evs[i])
 
+    r.launch_count = 0
     eager_ms, eager_dec_ms = r.timed_pass(eager_k_steps, eager_evs, barrier)
+    eager_launches = r.launch_count   # kernels of one pass of the K host-launched steps
     # the timed region: the K steps R times, until it lasts args.min_region seconds (whatever --steps is)
     per_replay, dec_ms = r.timed_region(args.min_region, barrier=barrier)
     clocks = sampler.stop() if rank == 0 else None
@@ -552,7 +569,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                    "t_cap": st["t_cap"], "lengths": "ctx" if r.per_seq else "ragged, floor(ctx*U[0.5,1.0])",
                    "launch_groups": n_groups, "ms_per_launch_group": round(ms_step / n_groups, 5), "cached_rows_per_kv_head": rows,
                    "num_splits": S, "bytes_per_row_per_kv_head": bytes_per_row(d), "l2": "inputs_larger_than_l2",
-                   "step": "quantize-append 1 row/seq + fused decode + combine", "codebook": CODEBOOK, "scales": "fp16" if SCALES_F16 else "fp32", "cache": (f"paged, {PAGE_ROWS} rows per page, scrambled" if PAGE_ROWS else "contiguous"), "parallelism": f"replicas x{world}",
+                   "step": ("one-call step (iq_decode_step_fused: the decode launch also appends the new rows, then the merge; two launches), every %d-th step's bracketed group by the three separate calls" % GRAPH_EVENT_STRIDE
+                            if r.one_call else "quantize-append 1 row/seq + fused decode + combine"), "codebook": CODEBOOK, "scales": "fp16" if SCALES_F16 else "fp32", "cache": (f"paged, {PAGE_ROWS} rows per page, scrambled" if PAGE_ROWS else "contiguous"), "parallelism": f"replicas x{world}",
                    "timed_region": ((f"{R} replays of a CUDA graph holding the K steps" if r.graph is not None else f"the K steps launched from the host, {R} times")
                                     + ", each replay between its own events and synchronizes; the replays' times are summed")},
         "decode_tokens_per_s": round(world * B / (ms_step * 1e-3), 1),
@@ -579,7 +597,9 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                           "ms_per_step": round(eager_ms / K, 4), "decode_launch_ms": round(sum(eager_dec_ms) / K, 4),
                           "note": "the same K steps launched call by call from the host (three binding calls per step), one pass"},
         "quantize_append": st["quantize_append"],
-        "gpu_launches": 3 * K * n_groups * R,   # per step and launch group: quantize_append_few_kernel, decode_kernel, combine_kernel
+        # counted as they are enqueued: per step and launch group quantize_append_few_kernel, decode_kernel, combine_kernel, or
+        # (one-call step of a small group) the decode kernel that also appends, and combine_kernel
+        "gpu_launches": (r.graph_launches if r.graph is not None else eager_launches) * R,
         "clocks": clocks,
     }
     if clocks and clocks.get("sm_mhz"):

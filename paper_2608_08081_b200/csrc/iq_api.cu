@@ -482,6 +482,8 @@ static int decode_params(const iq_shape* shape, const float* rot_dev, const iq_c
   p.delta_v = delta_v;
   p.k_new = p.v_new = nullptr;
   p.new_acc = p.new_ml = nullptr;
+  p.aux_ctas = 0;
+  p.len_bias = 0;
   std::memcpy(p.thresholds_k, side_thresholds(codebook, 0), sizeof(p.thresholds_k));
   std::memcpy(p.thresholds_v, side_thresholds(codebook, 1), sizeof(p.thresholds_v));
   std::memcpy(p.levels_k, side_levels(codebook, 0), sizeof(p.levels_k));
@@ -538,7 +540,6 @@ int iq_decode_step_fused(const iq_shape* shape, const float* rot_dev, const iq_c
   if (!aligned16(workspace_dev) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new)) return IQ_ERR_ALIGN;
   int rc = check_shape(shape);
   if (rc) return rc;
-  if (shape->bits != 3) return IQ_ERR_SHAPE;  // the append inside the decode launch is built for the 3-bit layout
   if (num_splits < 1 || num_splits > 65535) return IQ_ERR_SHAPE;
   const StepWorkspace w = step_workspace(shape, num_splits);
   uint8_t* ws = static_cast<uint8_t*>(workspace_dev);
@@ -549,12 +550,25 @@ int iq_decode_step_fused(const iq_shape* shape, const float* rot_dev, const iq_c
   rc = decode_params(shape, rot_dev, codebook, q, cache, seq_lens_dev, num_splits, part_acc, part_ml, part_argmax, status_dev, p);
   if (rc) return rc;
   if (shape->batch == 0) return IQ_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The append inside the decode launch pays while its tasks ((sequence, KV head) x (1 + heads per KV head), a warp
+  // each) fit the few SMs set aside for them in one round; beyond that the three launches are faster, and the same
+  // result is produced by them: append, decode over one more row per sequence, merge.
+  const long long tasks = (long long)shape->batch * shape->n_kv_heads * (1 + shape->n_q_heads / shape->n_kv_heads);
+  if (tasks > 180 || shape->bits != 3) {  // (the append inside the decode launch is built for the 3-bit layout)
+    const int64_t sh = shape->head_dim, sb = (int64_t)shape->n_kv_heads * sh;  // k_new, v_new: [B][1][H_kv][d]
+    rc = iq_quantize_append(shape, rot_dev, codebook, k_new, v_new, sb, sb, sh, seq_lens_dev, nullptr, 1, cache, status_dev, stream);
+    if (rc) return rc;
+    p.len_bias = 1;
+    if (iq::launch_decode_attention(p, shape->head_dim, st) != cudaSuccess) return IQ_ERR_CUDA;
+    return combine_with_new_row(shape, rot_dev, num_splits, 1, part_acc, part_ml, part_argmax, nullptr, nullptr, nullptr, nullptr, out,
+                                out_is_fp16, lse_out, argmax_out, stream);
+  }
   p.k_new = static_cast<const __half*>(k_new);
   p.v_new = static_cast<const __half*>(v_new);
   p.new_acc = reinterpret_cast<float*>(ws + w.new_acc);
   p.new_ml = reinterpret_cast<float*>(ws + w.new_ml);
-  const cudaError_t e = iq::launch_decode_attention(p, shape->head_dim, static_cast<cudaStream_t>(stream));
-  if (e != cudaSuccess) return IQ_ERR_CUDA;
+  if (iq::launch_decode_attention(p, shape->head_dim, st) != cudaSuccess) return IQ_ERR_CUDA;
   return combine_with_new_row(shape, rot_dev, num_splits, 1, part_acc, part_ml, part_argmax, nullptr, p.new_acc, p.new_ml, seq_lens_dev,
                               out, out_is_fp16, lse_out, argmax_out, stream);
 }

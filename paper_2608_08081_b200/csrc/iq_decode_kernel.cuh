@@ -150,7 +150,7 @@ template <int D>
 __device__ __forceinline__ void dec_draw(const DecodeParams& p, DecWalk& w, DecDrawn& d, int* next_s, int lane, int with_argmax) {
   constexpr int TB = DEC_BLOCK_TOKENS;
   const int S = p.splits, B = p.batch;
-  auto len_of = [&](int b) { return max(0, min(p.seq_lens[b], p.t_cap)); };
+  auto len_of = [&](int b) { return max(0, min(p.seq_lens[b] + p.len_bias, p.t_cap)); };
   auto warp_fill = [&](int b, int y, int slot) {
     const int kvh = y / p.head_groups, hg = y - kvh * p.head_groups;
     const int h0 = kvh * p.group + hg * DEC_HEADS, nh = min(DEC_HEADS, p.group - hg * DEC_HEADS);
@@ -276,85 +276,83 @@ static __device__ __noinline__ void dec_write_operand(uint8_t* dst, int hh, DecH
 }
 
 // Decode with append: the step's new K and V rows are quantised and appended (Algorithm 1) by the launch that attends
-// to them. CTA c takes (sequence, KV head) units c, c + grid, ...; one warp quantises the two rows, writes them to the
-// cache and writes the new row's own partial (m, l) = (z, 1), acc = v~ -- computed from the row's codes and stored
+// to them. The first aux_ctas CTAs of the grid do nothing else: their warps take the tasks of the (sequence, KV head)
+// units in turn; a unit's rows are quantised and written to the cache, and with them the new row's own partial (m, l) = (z, 1), acc = v~ -- computed from the row's codes and stored
 // scale, like a cached row's -- which the merge reads as one more slot. The blocks of the cache are read WITHOUT that
 // row (rows below seq_lens[b]), so nothing the other warps load depends on these writes.
 template <int D>
-static __device__ __noinline__ void dec_aux_work(const DecodeParams& p, int lane) {
+static __device__ __noinline__ void dec_aux_work(const DecodeParams& p, int lane, int first_task, int task_stride) {
   constexpr int E = D / 32;
-  const int n_units = p.batch * p.n_kv_heads;
-  for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+  // A (sequence, KV head) unit is 1 + group tasks, one warp each: task 0 quantises and stores the two rows and writes
+  // the value part of the partial; task 1 + j quantises the K row again (in registers) and writes head j's score.
+  const int per_unit = 1 + p.group;
+  const int n_tasks = p.batch * p.n_kv_heads * per_unit;
+  for (int t = first_task; t < n_tasks; t += task_stride) {
+    const int u = t / per_unit, part = t - u * per_unit;
     const int b = u / p.n_kv_heads, kvh = u - b * p.n_kv_heads;
     const int raw_len = p.seq_lens[b];
-    {
-      bool have_new = false;
-      size_t row = 0;
-      if (raw_len < 0 || raw_len >= p.t_cap) {
-        if (lane == 0 && p.status) {  // counted per (row, KV head, tensor)
-          atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
-          atomicAdd(&p.status[2], 2u);
-        }
-      } else if (!cache_row_for_write(p.pm, b, kvh, raw_len, p.status, row)) {  // no such page: skipped and counted
-        if (lane == 0 && p.status) atomicAdd(&p.status[2], 2u);
-      } else {
-        have_new = true;
+    bool have_new = false;
+    size_t row = 0;
+    if (raw_len < 0 || raw_len >= p.t_cap) {
+      if (part == 0 && lane == 0 && p.status) {  // counted per (row, KV head, tensor)
+        atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
+        atomicAdd(&p.status[2], 2u);
       }
-      if (have_new) {
-        const RowSink sink{const_cast<uint8_t*>(p.k_codes), const_cast<float*>(p.k_scales), const_cast<uint8_t*>(p.v_codes),
-                           const_cast<float*>(p.v_scales), p.status, p.scale_f16};
-        const size_t src = ((size_t)b * p.n_kv_heads + kvh) * D + lane * E;
-        __half2 raw_k[E / 2], raw_v[E / 2];
-#pragma unroll
-        for (int k = 0; k < E / 2; k++) {
-          raw_k[k] = reinterpret_cast<const __half2*>(p.k_new + src)[k];
-          raw_v[k] = reinterpret_cast<const __half2*>(p.v_new + src)[k];
-        }
-        WarpRowQuantizer<D> rq;
-        rq.init(p.rot + (size_t)kvh * (D / 4) * 8, p.thresholds_k, lane);
-        int code[E];
-        float lk[E], lv[E];
-        float sk = rq.run(raw_k, lane, code, p.status);
-        warp_store_k_row<D>(sink, row, code, sk, lane);
-#pragma unroll
-        for (int e = 0; e < E; e++) lk[e] = p.levels_k[code[e]];
-        rq.set_thresholds(p.thresholds_v);
-        float sv = rq.run(raw_v, lane, code, p.status);
-        warp_store_v_row<D>(sink, row, raw_len, code, sv, lane);
-#pragma unroll
-        for (int e = 0; e < E; e++) lv[e] = p.levels_v[code[e]];
-        if (p.scale_f16) {  // the scales as the cache holds them
-          sk = __half2float(__float2half_rn(fminf(sk, 65504.f)));
-          sv = __half2float(__float2half_rn(fminf(sv, 65504.f)));
-        }
-        const float vf = sv * rsqrtf((float)D);
-        for (int j = 0; j < p.group; j++) {  // z = sm_scale q~ . k~ of the new row, head by head; (m, l) = (z, 1), acc = v~
-          const size_t bh = (size_t)b * p.n_q_heads + kvh * p.group + j;
-          const DecHeadCoords<D> c = dec_rotate_head<D>(p.q + bh * D, p.rot + (size_t)kvh * (D / 4) * 8, lane);
-          float dot = 0.f;
-#pragma unroll
-          for (int e = 0; e < E; e++) dot = fmaf(c.v[e], lk[e], dot);
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(FULL, dot, o);
-          float4* a = reinterpret_cast<float4*>(p.new_acc + bh * D + lane * E);
-#pragma unroll
-          for (int e4 = 0; e4 < E / 4; e4++) a[e4] = make_float4(lv[4 * e4] * vf, lv[4 * e4 + 1] * vf, lv[4 * e4 + 2] * vf, lv[4 * e4 + 3] * vf);
-          if (lane == 0) {
-            p.new_ml[2 * bh] = dot * sk * p.sm_scale * rsqrtf((float)D);  // z = sm_scale q~ . (s level / sqrt d)
-            p.new_ml[2 * bh + 1] = 1.f;
-          }
-        }
-      } else if (lane < p.group) {
-        const size_t bh = (size_t)b * p.n_q_heads + kvh * p.group + lane;
-        p.new_ml[2 * bh] = -INFINITY;
-        p.new_ml[2 * bh + 1] = 0.f;
-      }
-      if (!have_new)
-        for (int j = 32 + lane; j < p.group; j += 32) {  // (more than 32 heads per KV head)
+    } else if (!cache_row_for_write(p.pm, b, kvh, raw_len, part == 0 ? p.status : nullptr, row)) {  // no such page: skipped and counted
+      if (part == 0 && lane == 0 && p.status) atomicAdd(&p.status[2], 2u);
+    } else {
+      have_new = true;
+    }
+    if (!have_new) {
+      if (part == 0)
+        for (int j = lane; j < p.group; j += 32) {
           const size_t bh = (size_t)b * p.n_q_heads + kvh * p.group + j;
           p.new_ml[2 * bh] = -INFINITY;
           p.new_ml[2 * bh + 1] = 0.f;
         }
+      continue;
+    }
+    const size_t src = ((size_t)b * p.n_kv_heads + kvh) * D + lane * E;
+    __half2 raw[E / 2];
+#pragma unroll
+    for (int k = 0; k < E / 2; k++) raw[k] = reinterpret_cast<const __half2*>(p.k_new + src)[k];
+    WarpRowQuantizer<D> rq;
+    rq.init(p.rot + (size_t)kvh * (D / 4) * 8, p.thresholds_k, lane);
+    int code[E];
+    if (part == 0) {
+      const RowSink sink{const_cast<uint8_t*>(p.k_codes), const_cast<float*>(p.k_scales), const_cast<uint8_t*>(p.v_codes),
+                         const_cast<float*>(p.v_scales), p.status, p.scale_f16};
+      const float sk = rq.run(raw, lane, code, p.status);
+      warp_store_k_row<D>(sink, row, code, sk, lane);
+#pragma unroll
+      for (int k = 0; k < E / 2; k++) raw[k] = reinterpret_cast<const __half2*>(p.v_new + src)[k];
+      rq.set_thresholds(p.thresholds_v);
+      float sv = rq.run(raw, lane, code, p.status);
+      warp_store_v_row<D>(sink, row, raw_len, code, sv, lane);
+      if (p.scale_f16) sv = __half2float(__float2half_rn(fminf(sv, 65504.f)));  // the scale as the cache holds it
+      const float vf = sv * rsqrtf((float)D);
+      float lv[E];
+#pragma unroll
+      for (int e = 0; e < E; e++) lv[e] = p.levels_v[code[e]] * vf;
+      for (int j = 0; j < p.group; j++) {  // acc = v~, the same for every head of the KV head
+        float4* a = reinterpret_cast<float4*>(p.new_acc + ((size_t)b * p.n_q_heads + kvh * p.group + j) * D + lane * E);
+#pragma unroll
+        for (int e4 = 0; e4 < E / 4; e4++) a[e4] = make_float4(lv[4 * e4], lv[4 * e4 + 1], lv[4 * e4 + 2], lv[4 * e4 + 3]);
+      }
+    } else {  // z = sm_scale q~ . k~ of the new row for one head; (m, l) = (z, 1)
+      const size_t bh = (size_t)b * p.n_q_heads + kvh * p.group + (part - 1);
+      float sk = rq.run(raw, lane, code, nullptr);
+      if (p.scale_f16) sk = __half2float(__float2half_rn(fminf(sk, 65504.f)));
+      const DecHeadCoords<D> c = dec_rotate_head<D>(p.q + bh * D, p.rot + (size_t)kvh * (D / 4) * 8, lane);
+      float dot = 0.f;
+#pragma unroll
+      for (int e = 0; e < E; e++) dot = fmaf(c.v[e], p.levels_k[code[e]], dot);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(FULL, dot, o);
+      if (lane == 0) {
+        p.new_ml[2 * bh] = dot * sk * p.sm_scale * rsqrtf((float)D);  // z = sm_scale q~ . (s level / sqrt d)
+        p.new_ml[2 * bh + 1] = 1.f;
+      }
     }
   }
 }
@@ -383,9 +381,17 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const bool control = warp >= NG * 4;
   const int grp = control ? warp - NG * 4 : warp >> 2;  // group of this warp
-  // decode with append: the last control warp first does the CTA's share of the appends; its group starts that much
-  // later, and the other groups draw the blocks meanwhile
-  const bool aux = APPEND && warp == NG * 5 - 1;
+  // Decode with append: the first aux_ctas CTAs append the new rows (every warp of them takes units) while the others
+  // work on the blocks; those see a grid of n_cta CTAs in which they are CTA number cta.
+  const int n_aux = APPEND ? p.aux_ctas : 0;
+  const int cta = (int)blockIdx.x - n_aux, n_cta = (int)gridDim.x - n_aux;
+  if constexpr (APPEND) {
+    if (cta < 0) {
+      grid_dependency_wait();
+      dec_aux_work<D>(p, lane, (int)blockIdx.x * (L::THREADS / 32) + warp, n_aux * (L::THREADS / 32));
+      return;
+    }
+  }
   const int gt = tid & (DEC_GROUP_THREADS - 1);         // compute thread within its group = TMEM lane
   const int bar_id = 1 + grp;                           // named barrier of the group's compute threads
 
@@ -420,7 +426,7 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
   const int B = p.batch;
   const int ips = p.n_kv_heads * p.head_groups;  // items per sequence
   const bool range_mode = S >= 2 * NG;
-  auto len_of = [&](int b) { return max(0, min(p.seq_lens[b], p.t_cap)); };
+  auto len_of = [&](int b) { return max(0, min(p.seq_lens[b] + p.len_bias, p.t_cap)); };
   auto nb_of = [&](int b) { return (len_of(b) + TB - 1) / TB; };
   auto item_heads = [&](int y, int& kvh, int& h0, int& nh) {
     kvh = y / p.head_groups;
@@ -479,10 +485,10 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
       n_cols = v;
       for (int i = 0; i < L::THREADS / 32; i++) nb_max = max(nb_max, scan_s[L::THREADS + i]);
     }
-    long long cper = (c_total + gridDim.x - 1) / gridDim.x;
+    long long cper = (c_total + n_cta - 1) / n_cta;
     cper = max(cper, (long long)((nb_max + W - 1) / (S / NG - 1) + 1));  // an item then spans at most S / NG ranges
     cper = max(cper, W + 1);                                              // and no range between two ranges of blocks is empty
-    const long long t_lo = (long long)blockIdx.x * cper;
+    const long long t_lo = (long long)cta * cper;
     if (t_lo >= c_total) no_work = true;
     if (tid == 0 && !no_work) {
       // the first block at or after cost position t: its sequence, item, block, and launch-wide block index
@@ -527,7 +533,7 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
       s0.item_g = before * ips + (long long)y * nb;
       s0.g0 = s0.item_g + blk;
       s0.count = (int)((b1 < B ? before1 * ips + (long long)y1 * nb1 + blk1 : before1 * ips) - s0.g0);
-      s0.piece = (int)((long long)blockIdx.x - (c_b + (long long)y * (nb + W) + W) / cper);  // CTAs since the one that holds the item's first block
+      s0.piece = (int)((long long)cta - (c_b + (long long)y * (nb + W) + W) / cper);  // CTAs since the one that holds the item's first block
       *start_s = s0;
       *next_s = 0;
       // the range's first segments: their query operands are prepared once for all groups
@@ -545,16 +551,10 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
     }
   } else {
     // unit mode: worker w = grp * grid + CTA takes units w, w + NG * grid, ...; a CTA none of whose groups has a unit leaves
-    if ((long long)blockIdx.x >= (long long)B * ips * S) no_work = true;
+    if ((long long)cta >= (long long)B * ips * S) no_work = true;
     if (tid == 0) *n_pre_s = 0;
   }
-  if (no_work) {  // a CTA without blocks still has its share of the appends
-    if (aux) {
-      grid_dependency_wait();
-      dec_aux_work<D>(p, lane);
-    }
-    return;
-  }
+  if (no_work) return;
 
   // ---------------------------------------------------------------- set-up: barriers, TMEM
   if (control && elect_one()) {  // every control warp initialises the barriers of its group
@@ -574,7 +574,7 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
   grid_dependency_wait();  // queries, cache rows and the partial buffers are not touched above this line
 
   // sequences without cached rows belong to no range and no unit: CTA c defines their partial slots for sequences c, c + grid, ...
-  for (int b = blockIdx.x; b < B; b += gridDim.x)
+  for (int b = cta; b < B; b += n_cta)
     if (len_of(b) == 0)
       for (int i = tid / DEC_HEADS; i < ips * S; i += L::THREADS / DEC_HEADS) fill_slot(b, i / S, i % S, tid % DEC_HEADS);
 
@@ -587,7 +587,6 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
   const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;                // this warp's 32 TMEM lanes
   bool failed = false;  // a bounded wait gave up; every later wait of this thread is skipped
 
-  if (aux) dec_aux_work<D>(p, lane);
   if (control) {
     // ================================================================ control warp of group grp: walks the work, fetches blocks, issues MMAs.
     // All 32 lanes run the loop and the waits (the walk is uniform over the warp); an elected lane issues.
@@ -614,8 +613,8 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
     if (range_mode) { wk.b = start_s->b; wk.y = start_s->y; wk.len = start_s->len; wk.nb = (wk.len + TB - 1) / TB; wk.piece = start_s->piece; wk.item_g = start_s->item_g; }
     else { wk.b = wk.y = wk.nb = wk.len = wk.piece = 0; wk.item_g = 0; }
     wk.n_units = B * ips * S;
-    wk.unit_step = NG * (int)gridDim.x;
-    wk.unit = min(wk.n_units, grp * (int)gridDim.x + (int)blockIdx.x);
+    wk.unit_step = NG * n_cta;
+    wk.unit = min(wk.n_units, grp * n_cta + cta);
     wk.ub = wk.uy = wk.uk = wk.ublk = wk.uhi = wk.unew = wk.ulen = 0;
     // The next block is drawn (shared counter; with a paged cache also its block-table entry, a load from global
     // memory) while the compute warps are busy with the softmax of the current one, and staged after the value MMAs.
@@ -1317,9 +1316,18 @@ static cudaError_t launch_one(const DecodeParams& p, cudaStream_t stream) {
   long long ctas = n_sm[dev];
   if (ctas > max_blocks) ctas = max_blocks;
   if (ctas < 1) ctas = 1;
-  if (APPEND) {  // the appends are spread over the CTAs whatever the number of blocks
-    const long long units = (long long)p.batch * p.n_kv_heads;
-    if (ctas < units) ctas = units < n_sm[dev] ? units : n_sm[dev];
+  if (APPEND) {
+    // A few CTAs of the grid only append: a warp takes ~5 us per task (a (sequence, KV head) unit is 1 + group tasks);
+    // enough CTAs for one round of tasks, never more than a sixteenth of the SMs.
+    const long long tasks = (long long)p.batch * p.n_kv_heads * (1 + p.group);
+    const int warps = L::THREADS / 32;
+    long long aux = (tasks + warps - 1) / warps;
+    if (aux > n_sm[dev] / 16) aux = n_sm[dev] / 16;
+    if (aux < 1) aux = 1;
+    if (ctas + aux > n_sm[dev] && ctas > 1) ctas = n_sm[dev] - aux;  // still one CTA per SM
+    DecodeParams q = p;
+    q.aux_ctas = (int)aux;
+    return launch_after_predecessor(kern, dim3((unsigned)(ctas + aux)), dim3(L::THREADS), L::SMEM_BYTES, stream, q);
   }
   return launch_after_predecessor(kern, dim3((unsigned)ctas), dim3(L::THREADS), L::SMEM_BYTES, stream, p);
 }

@@ -102,6 +102,8 @@ struct DecodeParams {
   const __half* v_new;
   float* new_acc;
   float* new_ml;
+  int aux_ctas;  // CTAs at the start of the grid that only append (set by the launcher)
+  int len_bias;  // added to every sequence length before it is clamped to [0, t_cap] (1: the lengths given are those before an append that has been enqueued)
   float thresholds_k[15], thresholds_v[15];
   float levels_k[16], levels_v[16];
 };

@@ -183,3 +183,42 @@ def test_paged_cache_and_binary16_scales(iq, torch, codebooks):
         st = status.cpu().numpy()
         assert st[0] & 4 and st[0] & 1 and st[2] == 3 * 2 * H_kv
         assert torch.equal(cache.k_codes, before[0]) and torch.equal(cache.v_codes, before[1])
+
+
+@pytest.mark.parametrize("bits", [2, 4])
+def test_other_bit_widths_take_the_three_launch_route(iq, torch, bits):
+    """The one-call step at 2 and 4 bits (the three launches behind the same contract) against the oracle."""
+    from oracle import lloyd_max
+    d, B, H_q, H_kv, T = 128, 2, 8, 2, 300
+    lv, th = lloyd_max.int8_codebook(d, 1 << bits)
+    cb = iq.Codebook(tuple(map(float, lv)), tuple(map(float, th)))
+    lens = np.array([259, 128], np.int32)
+    w = workloads.tiny(780 + bits, B, H_q, H_kv, d, T + 2, lens)
+    shape = iq.Shape(B, H_q, H_kv, d, w.t_cap, bits=bits)
+    rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+    iq.iq_make_rotation(d, H_kv, 0, np.ascontiguousarray(w.quats), rot)
+    cache = iq.new_cache(shape)
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(w.k).cuda(), torch.from_numpy(w.v).cuda(),
+                          torch.zeros(B, dtype=torch.int32, device="cuda"), torch.from_numpy(lens).cuda(), w.k.shape[1], cache, status)
+    ref = oracle.new_cache(B, H_kv, d, w.t_cap, bits)
+    oracle.quantize_append(w.quats, th, w.k, w.v, np.zeros(B, np.int32), lens, ref)
+    S = 8
+    ws = torch.empty(iq.iq_decode_step_workspace_bytes(shape, S), dtype=torch.uint8, device="cuda")
+    out = torch.empty((B, H_q, d), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, H_q), dtype=torch.float32, device="cuda")
+    am = torch.empty((B, H_q), dtype=torch.int32, device="cuda")
+    kn = np.ascontiguousarray(np.stack([w.k[b, lens[b]] for b in range(B)]))
+    vn = np.ascontiguousarray(np.stack([w.v[b, lens[b]] for b in range(B)]))
+    iq.iq_decode_step_fused(shape, rot, cb, torch.from_numpy(w.q).cuda(), torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), cache,
+                            torch.from_numpy(lens).cuda(), S, ws, out, lse, am, status)
+    torch.cuda.synchronize()
+    assert status.cpu().numpy()[0] == 0
+    oracle.quantize_append(w.quats, th, kn[:, None], vn[:, None], lens.copy(), None, ref)
+    now = lens + 1
+    g = cache_to_numpy(cache)
+    for b in range(B):
+        assert np.array_equal(g["k_codes"][b, :, :now[b]], ref["k_codes"][b, :, :now[b]])
+    w2 = workloads.Workload("bits", B, H_q, H_kv, d, w.t_cap, w.k, w.v, w.q, w.quats, now)
+    res = dict(out=out.cpu().numpy().astype(np.float64), lse=lse.cpu().numpy().astype(np.float64), argmax=am.cpu().numpy())
+    check_decode(w2, lv, w.q, res, g, now)
