@@ -704,6 +704,29 @@ def test_random_configurations(iq, torch, codebooks, case):
     S = int(g.choice([1, 2, 3, iq.iq_suggest_splits(shape, T)]))
     res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, now, S)
     check_decode(w2, lv, w.q, res, got, now)
+    # one more step through the one-call entry (the decode launch appends when the case is small, three launches otherwise)
+    kn = np.ascontiguousarray(np.stack([w.k[b, now[b]] for b in range(B)]))
+    vn = np.ascontiguousarray(np.stack([w.v[b, now[b]] for b in range(B)]))
+    ws = torch.empty(iq.iq_decode_step_workspace_bytes(shape, S), dtype=torch.uint8, device="cuda")
+    out = torch.empty((B, H_q, d), dtype=torch.float32, device="cuda")
+    lse = torch.empty((B, H_q), dtype=torch.float32, device="cuda")
+    am = torch.empty((B, H_q), dtype=torch.int32, device="cuda")
+    iq.iq_decode_step_fused(shape, rot, cb, torch.from_numpy(w.q).cuda(), torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), cache,
+                            torch.from_numpy(now).cuda(), S, ws, out, lse, am, status)
+    torch.cuda.synchronize()
+    assert status.cpu().numpy()[0] == 0
+    oracle.quantize_append(w.quats, th, kn[:, None], vn[:, None], now.copy(), None, ref)
+    if f16:
+        oracle.round_scales_fp16(ref)
+    now = now + 1
+    got = _gather_pages(cache, table, page_rows) if paged else cache_to_numpy(cache)
+    got["k_scales"] = got["k_scales"].astype(np.float32)
+    got["v_scales"] = got["v_scales"].astype(np.float32)
+    for b in range(B):
+        assert np.array_equal(got["k_codes"][b, :, :now[b]], ref["k_codes"][b, :, :now[b]])
+    w3 = workloads.Workload("rnd", B, H_q, H_kv, d, T, full_k, full_v, w.q, w.quats, now)
+    check_decode(w3, lv, w.q, dict(out=out.cpu().numpy().astype(np.float64), lse=lse.cpu().numpy().astype(np.float64), argmax=am.cpu().numpy()),
+                 got, now)
 
 
 def test_combine_splits_in_isolation(iq, torch, codebooks):
