@@ -6,21 +6,31 @@
 
 namespace iq {
 
-// code = #{ j : u > t_j } over NT ascending thresholds, and whether u is within `guard` of one of them.
+// code = #{ j : u > t_j } over NT = 3, 7 or 15 ascending thresholds, and whether u is within `guard` of one of them: a
+// binary search whose pivots are picked with selects (the thresholds stay in registers). The pivots visited include
+// both bounds of the final cell, so checking them covers every decision that could flip.
 template <typename T, int NT>
 __device__ __forceinline__ int decide_code_n(T u, const float (&th)[NT], bool& near_boundary, T guard) {
   if constexpr (NT == 7) {
     return decide_code<T>(u, th, near_boundary, guard);
+  } else if constexpr (NT == 3) {
+    const bool b1 = u > (T)th[1];
+    const T p0 = b1 ? (T)th[2] : (T)th[0];
+    const bool b0 = u > p0;
+    near_boundary = fmin(fabs(u - (T)th[1]), fabs(u - p0)) <= guard;
+    return (b1 ? 2 : 0) + (b0 ? 1 : 0);
   } else {
-    int code = 0;
-    T dmin = (T)1e30;
-#pragma unroll
-    for (int j = 0; j < NT; j++) {
-      code += u > (T)th[j];
-      dmin = fmin(dmin, fabs(u - (T)th[j]));
-    }
-    near_boundary = dmin <= guard;
-    return code;
+    static_assert(NT == 15, "2, 3 or 4 bits");
+    const bool b3 = u > (T)th[7];
+    const T p2 = b3 ? (T)th[11] : (T)th[3];
+    const bool b2 = u > p2;
+    const T p1 = b3 ? (b2 ? (T)th[13] : (T)th[9]) : (b2 ? (T)th[5] : (T)th[1]);
+    const bool b1 = u > p1;
+    const T p0 = b3 ? (b2 ? (b1 ? (T)th[14] : (T)th[12]) : (b1 ? (T)th[10] : (T)th[8]))
+                    : (b2 ? (b1 ? (T)th[6] : (T)th[4]) : (b1 ? (T)th[2] : (T)th[0]));
+    const bool b0 = u > p0;
+    near_boundary = fmin(fmin(fabs(u - (T)th[7]), fabs(u - p2)), fmin(fabs(u - p1), fabs(u - p0))) <= guard;
+    return (b3 ? 8 : 0) + (b2 ? 4 : 0) + (b1 ? 2 : 0) + (b0 ? 1 : 0);
   }
 }
 

@@ -460,29 +460,75 @@ __global__ void __launch_bounds__(32) quantize_append_few_kernel(const __grid_co
   WarpRowQuantizer<D, BITS> rq;
   const RowSink sink{p.k_codes, p.k_scales, p.v_codes, p.v_scales, p.status, p.scale_f16};
   rq.init(p.rot + (size_t)h * (D / 4) * 8, is_v ? p.thresholds_v : p.thresholds_k, lane);
-  for (int i = i_lo; i < i_hi; i++) {
-    if (i > i_lo) {
+  // 2 and 4 bits, V rows: the codes of consecutive rows that share a word of the records (8 or 16 rows) are collected in
+  // registers and the word is written once -- whole when every entry of it is new, merged with the old word otherwise --
+  // instead of one read-modify-write per row (this kernel is also the bulk path of those widths).
+  uint32_t pend[E];
+  uint32_t pend_mask = 0u;
+  int pend_word = -1;
+  size_t pend_blk = 0;
 #pragma unroll
-      for (int k = 0; k < E / 2; k++) raw[k] = reinterpret_cast<const __half2*>(src_base + (size_t)i * p.stride_t)[k];
+  for (int e = 0; e < E; e++) pend[e] = 0u;
+  auto flush_pending = [&]() {
+    if constexpr (BITS != 3) {
+      if (pend_word >= 0 && pend_mask != 0u) {
+#pragma unroll
+        for (int e = 0; e < E; e++) {
+          uint32_t* dst = reinterpret_cast<uint32_t*>(p.v_codes + (pend_blk * D + lane * E + e) * (size_t)(16 * BITS)) + pend_word;
+          *dst = (pend_mask == 0xFFFFFFFFu) ? pend[e] : ((*dst & ~pend_mask) | pend[e]);
+          pend[e] = 0u;
+        }
+      }
+      pend_mask = 0u;
+      pend_word = -1;
+    }
+  };
+  for (int i = i_lo; i < i_hi; i++) {
+    __half2 nxt[E / 2];  // the next row is requested before this one is worked on
+    if (i + 1 < i_hi) {
+#pragma unroll
+      for (int k = 0; k < E / 2; k++) nxt[k] = reinterpret_cast<const __half2*>(src_base + (size_t)(i + 1) * p.stride_t)[k];
     }
     const long long t = pos0 + i;
+    bool ok = true;
+    size_t row = 0;  // the row's place in the cache arrays
     if (t < 0 || t >= p.t_cap) {
       if (lane == 0 && p.status) {  // counted per (row, KV head, tensor), like the bulk kernels
         atomicOr(&p.status[0], IQ_STATUS_ROW_OUT_OF_RANGE);
         atomicAdd(&p.status[2], 1u);
       }
-      continue;
-    }
-    size_t row;  // the row's place in the cache arrays
-    if (!cache_row_for_write(p.pm, b, h, t, p.status, row)) {  // no such page: skipped and counted
+      ok = false;
+    } else if (!cache_row_for_write(p.pm, b, h, t, p.status, row)) {  // no such page: skipped and counted
       if (lane == 0 && p.status) atomicAdd(&p.status[2], 1u);
-      continue;
+      ok = false;
     }
-    int code[E];
-    const float s = rq.run(raw, lane, code, p.status);
-    if (!is_v) warp_store_k_row<D, BITS>(sink, row, code, s, lane);
-    else warp_store_v_row<D, BITS>(sink, row, t, code, s, lane);
+    if (ok) {
+      int code[E];
+      const float s = rq.run(raw, lane, code, p.status);
+      if (!is_v) {
+        warp_store_k_row<D, BITS>(sink, row, code, s, lane);
+      } else if constexpr (BITS == 3) {
+        warp_store_v_row<D, BITS>(sink, row, t, code, s, lane);
+      } else {
+        int word, sh;
+        packed_place<BITS>((int)(t % 128), word, sh);
+        if (word != pend_word || row / 128 != pend_blk) {
+          flush_pending();
+          pend_word = word;
+          pend_blk = row / 128;
+        }
+#pragma unroll
+        for (int e = 0; e < E; e++) pend[e] |= (uint32_t)code[e] << sh;
+        pend_mask |= ((1u << BITS) - 1u) << sh;
+        if (lane == 0) store_scale(p.v_scales, row, s, p.scale_f16, p.status);
+      }
+    }
+    if (i + 1 < i_hi) {
+#pragma unroll
+      for (int k = 0; k < E / 2; k++) raw[k] = nxt[k];
+    }
   }
+  flush_pending();
 }
 
 // ---------------------------------------------------------------------------------------------------------
