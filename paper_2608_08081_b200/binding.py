@@ -173,7 +173,7 @@ def iq_row_bytes_bits(head_dim: int, bits: int) -> int:
 
 @dataclass
 class Cache:
-    """Contiguous: k_codes uint8 [B][H_kv][t_cap][3d/8], k_scales fp32 [B][H_kv][t_cap] (V alike). Paged: the same
+    """Contiguous: k_codes uint8 [B][H_kv][t_cap][bits * d / 8], k_scales fp32 [B][H_kv][t_cap] (V alike). Paged: the same
     arrays with a pool of pages in place of the batch, [num_pages][H_kv][page_rows]..., and block_table int32
     [B][t_cap / page_rows] on the device."""
     k_codes: torch.Tensor
