@@ -26,7 +26,11 @@
 //   4. thread c dequantises coordinate c of the token-transposed V block (128 codes = one 48-byte row) into
 //      TMEM lane c; the control warp issues O[c][n] = sum_row A_V[c][row] * B_P[n][row].
 //   5. thread c folds O into its running accumulator for coordinate c.
-// Packed tiles arrive through a 1-D bulk-copy (TMA) pipeline; every mbarrier wait is bounded in time.
+// Packed tiles arrive through a 1-D bulk-copy (TMA) pipeline; every mbarrier wait is bounded (a poll count).
+//
+// Template parameters of the kernel: head_dim D; ARGMAX (exact slot maxima and their rows); I8 (levels on an 8-bit grid:
+// int8 operands, int32 accumulation; otherwise fp16 operands); APPEND (the launch also appends the step's new rows: a few
+// CTAs at the start of the grid do only that, see dec_aux_work); BITS (2, 3 or 4 bits per code: tile sizes and lookups).
 #pragma once
 #include <climits>
 
