@@ -459,6 +459,7 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
   long long g0 = 0;
   int count = 0;  // blocks of this CTA's range (read from shared memory after the set-up barrier)
   bool no_work = false;
+  int n_work = n_cta;  // CTAs of the grid that have blocks (they share the slots of the sequences without cached rows)
   if (range_mode) {
     constexpr long long W = DEC_SEG_COST;
     int* cnt_s = scan_s + L::THREADS + L::THREADS / 32;  // [THREADS] non-empty sequences per slice of the batch
@@ -494,6 +495,7 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
     cper = max(cper, W + 1);                                              // and no range between two ranges of blocks is empty
     const long long t_lo = (long long)cta * cper;
     if (t_lo >= c_total) no_work = true;
+    n_work = (int)min((long long)n_cta, (c_total + cper - 1) / cper);  // 0: no sequence has a cached row
     if (tid == 0 && !no_work) {
       // the first block at or after cost position t: its sequence, item, block, and launch-wide block index
       auto locate = [&](long long t, int& b, int& nb, int& y, int& blk, long long& before_nb, long long& c_b) {
@@ -556,9 +558,17 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
   } else {
     // unit mode: worker w = grp * grid + CTA takes units w, w + NG * grid, ...; a CTA none of whose groups has a unit leaves
     if ((long long)cta >= (long long)B * ips * S) no_work = true;
+    n_work = (int)min((long long)n_cta, (long long)B * ips * S);
     if (tid == 0) *n_pre_s = 0;
   }
-  if (no_work) return;
+  if (no_work) {
+    if (n_work == 0 && cta == 0) {  // not one cached row in the whole batch: this CTA marks every slot unused
+      grid_dependency_wait();
+      for (int b = 0; b < B; b++)
+        for (int i = tid / DEC_HEADS; i < ips * S; i += L::THREADS / DEC_HEADS) fill_slot(b, i / S, i % S, tid % DEC_HEADS);
+    }
+    return;
+  }
 
   // ---------------------------------------------------------------- set-up: barriers, TMEM
   if (control && elect_one()) {  // every control warp initialises the barriers of its group
@@ -577,8 +587,9 @@ __global__ void __launch_bounds__(DecLayout<D, BITS>::THREADS, 1) decode_kernel(
   }
   grid_dependency_wait();  // queries, cache rows and the partial buffers are not touched above this line
 
-  // sequences without cached rows belong to no range and no unit: CTA c defines their partial slots for sequences c, c + grid, ...
-  for (int b = cta; b < B; b += n_cta)
+  // sequences without cached rows belong to no range and no unit: the CTAs that have blocks define their partial slots, CTA c
+  // those of sequences c, c + n_work, ...
+  for (int b = cta; b < B; b += n_work)
     if (len_of(b) == 0)
       for (int i = tid / DEC_HEADS; i < ips * S; i += L::THREADS / DEC_HEADS) fill_slot(b, i / S, i % S, tid % DEC_HEADS);
 

@@ -986,3 +986,26 @@ def test_bench_line_keeps_its_contract():
     assert rf["bound"] == "hbm" and rf["unit"] == "GB/s" and abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-3 and rf["traffic"] > 0
     assert d["e2e"]["h2d_bytes_per_step"] > 0 and d["e2e"]["d2h_bytes_per_step"] > 0 and d["e2e"]["value"] > 0
     assert d["value"] > 0 and d["ms_per_step"] > 0
+
+
+@pytest.mark.parametrize("d", [128, 256])
+def test_empty_sequences_next_to_little_work(iq, torch, codebooks, d):
+    """Many sequences without cached rows and hardly any blocks: only a few CTAs have work, and they must still define every
+    partial slot of every empty sequence (the workspace is pre-filled with values a merge would take for live slots);
+    likewise a batch in which no sequence has a row."""
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    for lens in ([5] + [0] * 199, [0] * 150 + [130, 0, 0, 1], [0] * 64):
+        B = len(lens)
+        w = workloads.tiny(2300 + B, B, 4, 2, d, 256, lens=lens)
+        shape, rot, cache, status = gpu_quantize(iq, torch, w, cb, n_new=np.asarray(lens, np.int32))
+        g = cache_to_numpy(cache)
+        for S in (1, 3, 8, 24):
+            ws = iq.DecodeWorkspace(shape, S, want_argmax=True)
+            ws.part_acc.fill_(1.0); ws.part_ml.fill_(1.0); ws.part_argmax.fill_(7); ws.out.fill_(3.0); ws.lse.fill_(3.0)
+            iq.decode_step(shape, rot, cb, torch.from_numpy(w.q).cuda(), cache, torch.from_numpy(np.asarray(lens, np.int32)).cuda(), ws)
+            torch.cuda.synchronize()
+            res = dict(out=ws.out.cpu().numpy().astype(np.float64), lse=ws.lse.cpu().numpy().astype(np.float64), argmax=ws.argmax.cpu().numpy())
+            check_decode(w, lv, w.q, res, g, np.asarray(lens, np.int32))
+            empty = np.asarray(lens) == 0
+            assert np.all(res["argmax"][empty] == -1)
