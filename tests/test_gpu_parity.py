@@ -1009,3 +1009,10 @@ def test_empty_sequences_next_to_little_work(iq, torch, codebooks, d):
             check_decode(w, lv, w.q, res, g, np.asarray(lens, np.int32))
             empty = np.asarray(lens) == 0
             assert np.all(res["argmax"][empty] == -1)
+
+
+def test_very_many_slots(iq, torch, codebooks):
+    """Slot counts beyond what one pass of the wide merge covers (more than 32 slots per warp), and odd ones."""
+    lens = [700, 33, 0]
+    w = workloads.tiny(2400, 3, 8, 2, 128, 768, lens=lens)
+    print(_roundtrip(iq, torch, codebooks, w, [17, 33, 255, 257, 300, 1024], n_new=lens))
