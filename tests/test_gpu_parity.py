@@ -1016,3 +1016,36 @@ def test_very_many_slots(iq, torch, codebooks):
     lens = [700, 33, 0]
     w = workloads.tiny(2400, 3, 8, 2, 128, 768, lens=lens)
     print(_roundtrip(iq, torch, codebooks, w, [17, 33, 255, 257, 300, 1024], n_new=lens))
+
+
+@pytest.mark.parametrize("d", [128, 256])
+def test_softmax_scale_given_by_the_caller(iq, torch, codebooks, d):
+    """iq_shape.sm_scale > 0 replaces 1/sqrt(d) (Appendix A's scale) in the plain step and in the one-call step."""
+    lv, th = codebooks[d]
+    cb = codebook_for(iq, codebooks, d)
+    lens = np.array([300, 77], np.int32)
+    w = workloads.tiny(2500 + d, 2, 8, 2, d, 304, lens=lens)
+    for scale in (0.31, 0.02):
+        shape = iq.Shape(w.B, w.H_q, w.H_kv, d, w.t_cap, sm_scale=scale)
+        rot = torch.empty(iq.iq_rotation_floats(d, w.H_kv), dtype=torch.float32, device="cuda")
+        iq.iq_make_rotation(d, w.H_kv, 0, np.ascontiguousarray(w.quats), rot)
+        cache = iq.new_cache(shape)
+        status = torch.zeros(4, dtype=torch.int32, device="cuda")
+        iq.iq_quantize_append(shape, rot, cb, torch.from_numpy(w.k).cuda(), torch.from_numpy(w.v).cuda(),
+                              torch.zeros(w.B, dtype=torch.int32, device="cuda"), torch.from_numpy(lens).cuda(), w.k.shape[1], cache, status)
+        for S in (1, 8):
+            res = gpu_decode(iq, torch, shape, rot, cb, w.q, cache, lens, S)
+            check_decode(w, lv, w.q, res, cache_to_numpy(cache), lens, sm_scale=scale)
+        ws = torch.empty(iq.iq_decode_step_workspace_bytes(shape, 8), dtype=torch.uint8, device="cuda")
+        out = torch.empty((w.B, w.H_q, d), dtype=torch.float32, device="cuda")
+        lse = torch.empty((w.B, w.H_q), dtype=torch.float32, device="cuda")
+        am = torch.empty((w.B, w.H_q), dtype=torch.int32, device="cuda")
+        kn = np.ascontiguousarray(np.stack([w.k[b, lens[b]] for b in range(w.B)]))
+        vn = np.ascontiguousarray(np.stack([w.v[b, lens[b]] for b in range(w.B)]))
+        iq.iq_decode_step_fused(shape, rot, cb, torch.from_numpy(w.q).cuda(), torch.from_numpy(kn).cuda(), torch.from_numpy(vn).cuda(), cache,
+                                torch.from_numpy(lens).cuda(), 8, ws, out, lse, am, status)
+        torch.cuda.synchronize()
+        assert status.cpu().numpy()[0] == 0
+        w2 = workloads.Workload("scale", w.B, w.H_q, w.H_kv, d, w.t_cap, w.k, w.v, w.q, w.quats, lens + 1)
+        check_decode(w2, lv, w.q, dict(out=out.cpu().numpy().astype(np.float64), lse=lse.cpu().numpy().astype(np.float64), argmax=am.cpu().numpy()),
+                     cache_to_numpy(cache), lens + 1, sm_scale=scale)
