@@ -41,5 +41,6 @@ from .binding import (  # noqa: F401
     new_cache,
     new_paged_cache,
     DecodeWorkspace,
+    HostStepper,
     decode_step,
 )

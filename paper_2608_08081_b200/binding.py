@@ -351,6 +351,37 @@ def iq_decode_step_host(shape: Shape, rot_dev, codebook: Codebook, inputs_host, 
                                     _ptr(ws.status), _stream(stream)), "iq_decode_step_host")
 
 
+class HostStepper:
+    """iq_decode_step_host for a loop of steps with every argument marshalled once: the step's host inputs are rows of one
+    pinned tensor [n_steps][B * (H_q + 2 H_kv) * d], the lengths rows of one device table [n_steps + 1][B] (row i: before
+    step i), and a step only adds offsets to base pointers. Same call, same kernels; what it saves is the host's time
+    per step (tensor views, pointer queries, argument conversion), which sits inside an end-to-end step."""
+
+    def __init__(self, shape: Shape, rot_dev, codebook: Codebook, inputs_host_all, inputs_dev, lens_table_dev, cache: Cache,
+                 ws: "DecodeWorkspace", out_dev, out_host, stream=None):
+        n = shape.batch * (shape.n_q_heads + 2 * shape.n_kv_heads) * shape.head_dim
+        assert inputs_host_all.dtype == torch.float16 and inputs_host_all.dim() == 2 and inputs_host_all.shape[1] == n
+        assert inputs_host_all.is_contiguous() and inputs_dev.dtype == torch.float16 and inputs_dev.numel() == n
+        assert lens_table_dev.dtype == torch.int32 and lens_table_dev.is_contiguous() and lens_table_dev.shape[1] == shape.batch
+        assert out_dev.dtype == out_host.dtype
+        self._keep = (shape, codebook, cache, rot_dev, inputs_host_all, inputs_dev, lens_table_dev, ws, out_dev, out_host)
+        self._cs, self._cb, self._cc = shape.c(), codebook.c(), cache.c()
+        self._hin, self._hin_stride = inputs_host_all.data_ptr(), n * 2
+        self._lens, self._lens_stride = lens_table_dev.data_ptr(), shape.batch * 4
+        self.n_steps = min(inputs_host_all.shape[0], lens_table_dev.shape[0] - 1)
+        self._fixed = (ctypes.byref(self._cs), _ptr(rot_dev), ctypes.byref(self._cb))
+        self._tail = (ctypes.byref(self._cc), ws.num_splits, _ptr(ws.part_acc), _ptr(ws.part_ml), _ptr(out_dev), _ptr(out_host),
+                      1 if out_dev.dtype == torch.float16 else 0, _ptr(ws.status), _stream(stream))
+        self._din = _ptr(inputs_dev)
+
+    def step(self, i: int) -> None:
+        """Step i (blocking): inputs row i, lengths row i before and row i + 1 after the append."""
+        rc = _lib.iq_decode_step_host(*self._fixed, self._hin + i * self._hin_stride, self._din, self._lens + i * self._lens_stride,
+                                      self._lens + (i + 1) * self._lens_stride, *self._tail)
+        if rc != 0:
+            raise IQError(rc, "iq_decode_step_host")
+
+
 def iq_rotated_histogram(shape: Shape, rot_dev, x, n_rows_dev, hist_dev, rng_half: float, stream=None) -> None:
     """Adds the histogram of the rotated, normalised coordinates of the rows x (fp16 device tensor [B][T][H_kv][d]) to
     hist_dev (uint32/int32 device tensor [bins]); n_rows_dev: int32 [B] or None (all T rows)."""

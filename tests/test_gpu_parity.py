@@ -307,6 +307,29 @@ def test_decode_step_from_host_buffers(iq, torch, codebooks, out_dtype):
         assert np.all(np.abs(got - r["out"]) <= tol), float(np.max(np.abs(got - r["out"])))
     w2 = workloads.Workload("h", B, H_q, H_kv, d, t_cap, w.k, w.v, w.q, w.quats, rows.astype(np.int32))
     compare_caches(w2, th, cache_to_numpy(cache), ref, w2.seq_lens)
+    # two more steps through the stepper that marshals every argument once (rows of one pinned tensor, one length table)
+    more = 2
+    h_all = torch.empty((more, n_in), dtype=torch.float16).pin_memory()
+    tab = torch.from_numpy(np.stack([rows + j for j in range(more + 1)]).astype(np.int32)).cuda()
+    qs, kns, vns = [], [], []
+    for j in range(more):
+        kn = np.stack([w.k[b, min(rows[b] + j, w.k.shape[1] - 1)] for b in range(B)])[:, None]
+        vn = np.stack([w.v[b, min(rows[b] + j, w.k.shape[1] - 1)] for b in range(B)])[:, None]
+        qn = workloads.to_fp16(g.standard_normal((B, H_q, d)))
+        h_all[j].copy_(torch.from_numpy(np.concatenate([qn.reshape(-1), kn.reshape(-1), vn.reshape(-1)])))
+        qs.append(qn); kns.append(kn); vns.append(vn)
+    stepper = iq.HostStepper(shape, rot, cb, h_all, d_in, tab, cache, ws, out_dev, out_host)
+    assert stepper.n_steps == more
+    for j in range(more):
+        stepper.step(j)
+        got = out_host.numpy().astype(np.float64).copy()
+        oracle.quantize_append(w.quats, th, kns[j], vns[j], rows.astype(np.int32), None, ref)
+        rows += 1
+        r = oracle.decode_attention(w.quats, lv, qs[j], cache_to_numpy(cache), rows.astype(np.int32), H_kv)
+        tol = 2e-3 + 1e-3 * np.abs(r["out"]) + (2.0 ** -11 * np.abs(r["out"]) if out_dtype == "float16" else 0)
+        assert np.all(np.abs(got - r["out"]) <= tol), float(np.max(np.abs(got - r["out"])))
+    for b in range(B):
+        assert np.array_equal(cache_to_numpy(cache)["k_codes"][b, :, :rows[b]], ref["k_codes"][b, :, :rows[b]])
     assert status.cpu().numpy()[0] == 0 and ws.status.cpu().numpy()[0] == 0
 
 
