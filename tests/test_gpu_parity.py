@@ -1072,3 +1072,52 @@ def test_softmax_scale_given_by_the_caller(iq, torch, codebooks, d):
         w2 = workloads.Workload("scale", w.B, w.H_q, w.H_kv, d, w.t_cap, w.k, w.v, w.q, w.quats, lens + 1)
         check_decode(w2, lv, w.q, dict(out=out.cpu().numpy().astype(np.float64), lse=lse.cpu().numpy().astype(np.float64), argmax=am.cpu().numpy()),
                      cache_to_numpy(cache), lens + 1, sm_scale=scale)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_split_count_does_not_change_the_result(iq, torch, seed):
+    """A property that holds at any size: which slots cover which rows is the library's choice, so the merged result
+    of a launch must not depend on num_splits. Random caches (uniform codes, positive scales) with length mixes the
+    oracle would take minutes for -- thousands of short sequences, many empty ones, a few long ones -- are decoded with
+    one slot per head (one worker per item, no merge) and with balanced splits; outputs, lse and argmax must agree."""
+    g = np.random.default_rng(500 + seed)
+    for case in range(6):
+        d = int(g.choice([128, 256]))
+        H_kv = int(g.choice([1, 2, 4]))
+        G = int(g.choice([1, 4, 8, 12]))
+        H_q = H_kv * G
+        B, T = [(2, 20000), (500, 256), (60, 2048), (2500, 128), (12, 8192), (300, 640)][case]
+        lens = g.integers(0, T + 1, size=B).astype(np.int32)
+        lens[g.random(B) < g.choice([0.0, 0.3, 0.9])] = 0
+        lens[g.integers(0, B)] = T
+        t_cap = workloads.cap128(T)
+        shape = iq.Shape(B, H_q, H_kv, d, t_cap)
+        cb = iq.iq_int8_codebook(d) if (case + seed) % 2 == 0 else iq.iq_default_codebook(d)
+        rot = torch.empty(iq.iq_rotation_floats(d, H_kv), dtype=torch.float32, device="cuda")
+        iq.iq_make_rotation(d, H_kv, case, None, rot)
+        cache = iq.new_cache(shape)
+        gen = torch.Generator(device="cuda")
+        gen.manual_seed(1000 * seed + case)
+        cache.k_codes.copy_(torch.randint(0, 256, cache.k_codes.shape, dtype=torch.uint8, device="cuda", generator=gen))
+        cache.v_codes.copy_(torch.randint(0, 256, cache.v_codes.shape, dtype=torch.uint8, device="cuda", generator=gen))
+        cache.k_scales.copy_(torch.rand(cache.k_scales.shape, device="cuda", generator=gen) * 3 + 0.1)
+        cache.v_scales.copy_(torch.rand(cache.v_scales.shape, device="cuda", generator=gen) * 3 + 0.1)
+        q = torch.randn((B, H_q, d), device="cuda", generator=gen).half()
+        sl = torch.from_numpy(lens).cuda()
+        ref = None
+        for S in (1, 2, int(g.choice([8, 16, 24])), iq.iq_suggest_splits(shape, T), int(g.choice([9, 33, 100]))):
+            ws = iq.DecodeWorkspace(shape, S, want_argmax=True)
+            ws.part_ml.fill_(1.0); ws.part_acc.fill_(1.0); ws.part_argmax.fill_(5)   # what a merge would take for live slots
+            iq.decode_step(shape, rot, cb, q, cache, sl, ws)
+            torch.cuda.synchronize()
+            assert int(ws.status[0]) == 0
+            if ref is None:
+                ref = (ws.out.clone(), ws.lse.clone(), ws.argmax.clone())
+                continue
+            nz = sl > 0
+            assert float((ws.out - ref[0]).abs().max()) <= 2e-3, (case, S)
+            assert float((ws.lse[nz] - ref[1][nz]).abs().max()) <= 2e-3, (case, S)
+            assert int((ws.argmax != ref[2]).sum()) <= 0.02 * ref[2].numel() + 1, (case, S)
+            assert bool((ws.out[~nz] == 0).all()) and bool(torch.isneginf(ws.lse[~nz]).all()) and bool((ws.argmax[~nz] == -1).all())
+        del cache
+        torch.cuda.empty_cache()
