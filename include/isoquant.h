@@ -4,7 +4,8 @@
  * The library implements the data-parallel hot path of IsoQuant KV-cache compression:
  *
  *   quantize-append   Algorithm 1 of the paper: s = ||x||_2, x^ = x/s, x~ = R_SO4(H_d x^) (Eq. 2),
- *                     3-bit Lloyd-Max code per coordinate (Step 3), bit-pack (Step 4).
+ *                     b-bit Lloyd-Max code per coordinate (Step 3; b = 3 in the paper, 2 and 4 as well here),
+ *                     bit-pack (Step 4).
  *   fused decode      Appendix A: q~ = R q once, scores q~ . k~_j / sqrt(d_k) taken directly on the
  *                     packed codes, softmax, o~ = sum_j alpha_j v~_j accumulated directly on the packed
  *                     codes, o = R^T o~ once (Table 2, kernels A-D). FP16 K/V are never materialised.
